@@ -1,0 +1,475 @@
+"""Pins for the CPU oracle: every check compares ``oracle/`` with something that
+does not come from it -- dense brute force written here, closed forms, special
+cases that reduce to separately written textbook loops, invariants the paper
+proves.  A dropped term, a wrong sign or index, a missing conjugate or a
+transposed operand in the oracle fails at least one of them.
+"""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import bookkeeping, chunk_wy, recurrence
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ----------------------------------------------------------------------------
+# helpers written independently of oracle/ (dense matrices, no structure used)
+# ----------------------------------------------------------------------------
+def rand_inputs(seed, N, T, m, dv, alpha_lo=0.5, s0=True, unit_k=True):
+    rng = np.random.default_rng(seed)
+    q = rng.standard_normal((N, T, 2 * m))
+    k = rng.standard_normal((N, T, 2 * m))
+    if unit_k:
+        k /= np.linalg.norm(k, axis=-1, keepdims=True)
+    v = rng.standard_normal((N, T, dv))
+    alpha = rng.uniform(alpha_lo, 1.0, (N, T, m))
+    theta = rng.uniform(-np.pi, np.pi, (N, T, m))
+    beta = rng.uniform(0.0, 1.0, (N, T))
+    S0 = rng.standard_normal((N, 2 * m, dv)) if s0 else None
+    return q, k, v, alpha, theta, beta, S0
+
+
+def cplx(x):
+    return x[..., 0::2] + 1j * x[..., 1::2]
+
+
+def dense_A(kc, alpha, theta, beta):
+    """A_t = (I - beta k k^H) diag(alpha e^{i theta}) as a dense m x m matrix (Eq. AtBt)."""
+    m = kc.shape[0]
+    Lam = np.diag(alpha * np.exp(1j * theta))
+    return (np.eye(m) - beta * np.outer(kc, kc.conj())) @ Lam
+
+
+def dense_forward(q, k, v, alpha, theta, beta, S0):
+    """One sequence, dense matrices only.  Returns o [T,dv] complex, all states, all A_t."""
+    T = q.shape[0]
+    qc, kc = cplx(q), cplx(k)
+    S = np.zeros((kc.shape[1], v.shape[1]), complex) if S0 is None else S0[0::2] + 1j * S0[1::2]
+    o, states, As = [], [], []
+    for t in range(T):
+        A = dense_A(kc[t], alpha[t], theta[t], beta[t])
+        B = beta[t] * np.outer(kc[t], v[t])            # beta k v^* with v real
+        S = A @ S + B
+        o.append(S.conj().T @ qc[t])
+        states.append(S)
+        As.append(A)
+    return np.array(o), states, As
+
+
+def run_rec(q, k, v, alpha, theta, beta, S0):
+    return recurrence.sfda_recurrence(q, k, v, alpha, theta, beta, S0)
+
+
+# ----------------------------------------------------------------------------
+# P1: dense brute force (Theorem "Constructive left-to-right chunk-WY recursion")
+# ----------------------------------------------------------------------------
+@pytest.mark.parametrize("seed,m,dv,T", [(1, 3, 2, 12), (2, 8, 5, 32), (3, 1, 1, 7)])
+def test_both_oracles_match_dense_brute_force(seed, m, dv, T):
+    q, k, v, al, th, be, S0 = rand_inputs(seed, 2, T, m, dv)
+    o_re, o_im, ST = run_rec(q, k, v, al, th, be, S0)
+    for n in range(2):
+        o, states, _ = dense_forward(q[n], k[n], v[n], al[n], th[n], be[n], S0[n])
+        assert np.abs(o_re[n] - o.real).max() < 1e-12
+        assert np.abs(o_im[n] - o.imag).max() < 1e-12
+        assert np.abs(ST[n][0::2] - states[-1].real).max() < 1e-12
+        assert np.abs(ST[n][1::2] - states[-1].imag).max() < 1e-12
+        for C in (4, 5, T):
+            a, b, c = chunk_wy.forward_chunked(q[n], k[n], v[n], al[n], th[n], be[n], S0[n], C)
+            assert np.abs(a - o.real).max() < 1e-12
+            assert np.abs(b - o.imag).max() < 1e-12
+            assert np.abs(c[0::2] - states[-1].real).max() < 1e-12
+            assert np.abs(c[1::2] - states[-1].imag).max() < 1e-12
+
+
+@pytest.mark.parametrize("seed,m,C", [(4, 4, 9), (5, 8, 16), (6, 2, 6)])
+def test_prefix_products_equal_factor_form(seed, m, C):
+    """P_t = A_t ... A_1 = Gamma_t - Y_t M_t W_t^* for every t (Eq. constructive-invariant)."""
+    _, k, _, al, th, be, _ = rand_inputs(seed, 1, C, m, 1)
+    kc = cplx(k[0])
+    P = np.eye(m, dtype=complex)
+    worst = 0.0
+    for t, (G, Y, W, M) in enumerate(chunk_wy.chunk_factor_steps(kc, al[0], th[0], be[0])):
+        P = dense_A(kc[t], al[0, t], th[0, t], be[0, t]) @ P
+        F = np.diag(G) - Y @ M @ W.conj().T
+        worst = max(worst, np.abs(P - F).max())
+        assert Y.shape == (m, t + 1) and W.shape == (m, t + 1) and M.shape == (t + 1, t + 1)
+        assert np.allclose(np.triu(M, 1), 0) and np.allclose(np.diag(M), 1)
+    assert worst < 1e-13          # the paper prints 1.9e-15 for this identity (Table 8)
+
+
+def test_single_step_diag_plus_rank_one():
+    """A_t = Lambda_t - u_t w_t^*, u = beta k, w = Lambda^* k (Eq. single-step-wy)."""
+    _, k, _, al, th, be, _ = rand_inputs(7, 1, 1, 5, 1)
+    kc = cplx(k[0, 0])
+    lam = al[0, 0] * np.exp(1j * th[0, 0])
+    A = dense_A(kc, al[0, 0], th[0, 0], be[0, 0])
+    G, Y, W, M = chunk_wy.chunk_factors(kc[None], al[0], th[0], be[0])
+    assert np.allclose(Y[:, 0], be[0, 0] * kc)
+    assert np.allclose(W[:, 0], np.conj(lam) * kc)
+    assert np.allclose(A, np.diag(lam) - np.outer(Y[:, 0], W[:, 0].conj()))
+
+
+# ----------------------------------------------------------------------------
+# P2: theta = 0 reduces to KDA (Prop. "KDA is a special case")
+# ----------------------------------------------------------------------------
+def real_kda(q, k, v, alpha, beta, S0):
+    """Textbook real KDA of dimension m: S = (I - b k k^T) diag(a) S + b k v^T; o = S^T q."""
+    T, m = k.shape
+    S = S0.copy()
+    o = np.zeros((T, v.shape[1]))
+    for t in range(T):
+        S = alpha[t][:, None] * S
+        S = S - beta[t] * np.outer(k[t], k[t] @ S) + beta[t] * np.outer(k[t], v[t])
+        o[t] = S.T @ q[t]
+    return o, S
+
+
+def test_theta_zero_real_channels_is_real_kda():
+    N, T, m, dv = 2, 50, 6, 4
+    q, k, v, al, th, be, S0 = rand_inputs(11, N, T, m, dv)
+    th[:] = 0.0
+    q[..., 1::2] = 0.0
+    k[..., 1::2] = 0.0
+    S0[:, 1::2] = 0.0
+    o_re, o_im, ST = run_rec(q, k, v, al, th, be, S0)
+    for n in range(N):
+        o, S = real_kda(q[n][:, 0::2], k[n][:, 0::2], v[n], al[n], be[n], S0[n][0::2])
+        assert np.abs(o_re[n] - o).max() < 1e-13
+        assert np.abs(o_im[n]).max() == 0.0
+        assert np.abs(ST[n][0::2] - S).max() < 1e-13
+        assert np.abs(ST[n][1::2]).max() == 0.0
+        a, b, c = chunk_wy.forward_chunked(q[n], k[n], v[n], al[n], th[n], be[n], S0[n], 16)
+        assert np.abs(a - o).max() < 1e-12 and np.abs(b).max() < 1e-13
+        assert np.abs(c[0::2] - S).max() < 1e-12
+
+
+def test_theta_zero_general_is_complex_kda():
+    T, m, dv = 30, 5, 3
+    q, k, v, al, th, be, S0 = rand_inputs(12, 1, T, m, dv)
+    th[:] = 0.0
+    o_re, o_im, ST = run_rec(q, k, v, al, th, be, S0)
+    qc, kc = cplx(q[0]), cplx(k[0])
+    S = S0[0][0::2] + 1j * S0[0][1::2]
+    for t in range(T):
+        S = (np.eye(m) - be[0, t] * np.outer(kc[t], kc[t].conj())) @ np.diag(al[0, t]) @ S \
+            + be[0, t] * np.outer(kc[t], v[0, t])
+        o = S.conj().T @ qc[t]
+        assert np.abs(o_re[0, t] - o.real).max() < 1e-13
+        assert np.abs(o_im[0, t] - o.imag).max() < 1e-13
+
+
+# ----------------------------------------------------------------------------
+# P3/P4: beta = 0 gives pure diagonal phase-decay (Prop. "Interpolation ...")
+# ----------------------------------------------------------------------------
+def test_beta_zero_closed_form():
+    N, T, m, dv = 1, 64, 4, 3
+    q, k, v, al, th, be, S0 = rand_inputs(13, N, T, m, dv)
+    be[:] = 0.0
+    o_re, o_im, ST = run_rec(q, k, v, al, th, be, S0)
+    gam = np.cumprod(al[0] * np.exp(1j * th[0]), axis=0)        # global cumulative product
+    S0c = S0[0][0::2] + 1j * S0[0][1::2]
+    qc = cplx(q[0])
+    for t in range(T):
+        o = S0c.conj().T @ (np.conj(gam[t]) * qc[t])
+        assert np.abs(o_re[0, t] - o.real).max() < 1e-12
+        assert np.abs(o_im[0, t] - o.imag).max() < 1e-12
+    S_T = gam[-1][:, None] * S0c
+    assert np.abs(ST[0][0::2] - S_T.real).max() < 1e-12
+    assert np.abs(ST[0][1::2] - S_T.imag).max() < 1e-12
+    a, b, c = chunk_wy.forward_chunked(q[0], k[0], v[0], al[0], th[0], be[0], S0[0], 16)
+    assert np.abs(c[0::2] - S_T.real).max() < 1e-12 and np.abs(c[1::2] - S_T.imag).max() < 1e-12
+
+
+def test_unit_decay_no_write_preserves_row_norms():
+    """alpha = 1, beta = 0: |z_t| = |z_0| (Prop. "Bounded cyclic phase memory")."""
+    N, T, m, dv = 1, 4096, 3, 2
+    q, k, v, al, th, be, S0 = rand_inputs(14, N, T, m, dv)
+    al[:] = 1.0
+    be[:] = 0.0
+    _, _, ST = run_rec(q, k, v, al, th, be, S0)
+    n0 = np.hypot(S0[0][0::2], S0[0][1::2])
+    nT = np.hypot(ST[0][0::2], ST[0][1::2])
+    assert np.abs(nT - n0).max() < 1e-12          # the paper prints 3.0e-14 drift at T = 16384
+
+
+# ----------------------------------------------------------------------------
+# P5: quantised phases 2 pi a / p (Prop. "Bounded cyclic phase memory")
+# ----------------------------------------------------------------------------
+def test_constant_quantised_phase_returns_after_p_steps():
+    m, dv = 4, 2
+    p = np.array([2, 3, 5, 7])
+    a = np.array([1, 2, 3, 4])
+    lcm = 210
+    T = 2 * lcm
+    rng = np.random.default_rng(15)
+    q = rng.standard_normal((1, T, 2 * m))
+    k = rng.standard_normal((1, T, 2 * m))
+    v = rng.standard_normal((1, T, dv))
+    S0 = rng.standard_normal((1, 2 * m, dv))
+    al = np.ones((1, T, m))
+    th = np.broadcast_to(2 * np.pi * a / p, (1, T, m)).copy()
+    be = np.zeros((1, T))
+    for Tcut in (lcm, 2 * lcm):
+        _, _, ST = run_rec(q[:, :Tcut], k[:, :Tcut], v[:, :Tcut], al[:, :Tcut], th[:, :Tcut], be[:, :Tcut], S0)
+        assert np.abs(ST - S0).max() < 1e-11
+    # after p_j steps coordinate j alone is back
+    for j in range(m):
+        _, _, ST = run_rec(q[:, :p[j]], k[:, :p[j]], v[:, :p[j]], al[:, :p[j]], th[:, :p[j]], be[:, :p[j]], S0)
+        assert np.abs(ST[0, 2 * j:2 * j + 2] - S0[0, 2 * j:2 * j + 2]).max() < 1e-13
+
+
+def test_mod5_counter_fixture():
+    """z_t = exp(2 pi i (sum a_s mod 5) / 5) z_0: the symbols and residues of the
+    fixture were written by hand from the closed form of Prop. "Bounded cyclic
+    phase memory"; nothing in it comes from the oracle."""
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "mod5_counter.txt")) if l.strip() and l[0] != "#"]
+    a = np.array([int(r[0]) for r in rows])
+    resid = np.array([int(r[1]) for r in rows])
+    T = len(a)
+    q = np.zeros((1, T, 2))
+    q[..., 0] = 1.0                                   # q = 1 reads conj(z_t)
+    k = np.zeros((1, T, 2))
+    v = np.zeros((1, T, 1))
+    al = np.ones((1, T, 1))
+    th = (2 * np.pi * a / 5).reshape(1, T, 1)
+    be = np.zeros((1, T))
+    S0 = np.array([[[1.0], [0.0]]])                   # z_0 = 1
+    o_re, o_im, ST = run_rec(q, k, v, al, th, be, S0)
+    z = o_re[0, :, 0] - 1j * o_im[0, :, 0]            # o = conj(z) * 1
+    want = np.exp(2j * np.pi * resid / 5)
+    assert np.abs(z - want).max() < 1e-13
+    a2, b2, _ = chunk_wy.forward_chunked(q[0], k[0], v[0], al[0], th[0], be[0], S0[0], 4)
+    assert np.abs((a2[:, 0] - 1j * b2[:, 0]) - want).max() < 1e-13
+
+
+def test_random_quantised_phase_tracks_integer_sum():
+    T, m, dv = 500, 4, 1
+    p = np.array([2, 3, 5, 7])
+    rng = np.random.default_rng(16)
+    a = rng.integers(0, p, size=(T, m))
+    th = (2 * np.pi * a / p)[None]
+    q = rng.standard_normal((1, T, 2 * m))
+    k = rng.standard_normal((1, T, 2 * m))
+    v = rng.standard_normal((1, T, dv))
+    S0 = rng.standard_normal((1, 2 * m, dv))
+    _, _, ST = run_rec(q, k, v, np.ones((1, T, m)), th, np.zeros((1, T)), S0)
+    resid = a.sum(0) % p                               # exact integer bookkeeping
+    S0c = S0[0][0::2] + 1j * S0[0][1::2]
+    want = np.exp(2j * np.pi * resid / p)[:, None] * S0c
+    assert np.abs(ST[0][0::2] - want.real).max() < 1e-11      # paper: modular error 3.0e-12
+    assert np.abs(ST[0][1::2] - want.imag).max() < 1e-11
+
+
+# ----------------------------------------------------------------------------
+# P6: register write (Theorem on register memory): Lambda = I, beta = 1, k = e_i
+# ----------------------------------------------------------------------------
+def test_register_overwrite():
+    m, dv = 5, 3
+    rng = np.random.default_rng(17)
+    S0 = rng.standard_normal((1, 2 * m, dv))
+    i = 2
+    k = np.zeros((1, 1, 2 * m))
+    k[0, 0, 2 * i] = 1.0
+    a = rng.standard_normal((1, 1, dv))
+    q = rng.standard_normal((1, 1, 2 * m))
+    _, _, ST = run_rec(q, k, a, np.ones((1, 1, m)), np.zeros((1, 1, m)), np.ones((1, 1)), S0)
+    want = S0[0].copy()
+    want[2 * i] = a[0, 0]
+    want[2 * i + 1] = 0.0
+    assert np.abs(ST[0] - want).max() < 1e-15
+
+
+# ----------------------------------------------------------------------------
+# P7: chunk-size invariance and split-sequence continuation (Theorem "Chunk-bounded exactness")
+# ----------------------------------------------------------------------------
+def test_chunk_size_invariance_and_continuation():
+    N, T, m, dv = 1, 96, 6, 4
+    q, k, v, al, th, be, S0 = rand_inputs(18, N, T, m, dv)
+    ref = run_rec(q, k, v, al, th, be, S0)
+    for C in (16, 32, 64, 7):
+        got = chunk_wy.forward_chunked(q[0], k[0], v[0], al[0], th[0], be[0], S0[0], C)
+        for g, r in zip(got, ref):
+            assert np.abs(g - r[0]).max() < 1e-12
+    T1 = 37
+    o1 = run_rec(q[:, :T1], k[:, :T1], v[:, :T1], al[:, :T1], th[:, :T1], be[:, :T1], S0)
+    o2 = run_rec(q[:, T1:], k[:, T1:], v[:, T1:], al[:, T1:], th[:, T1:], be[:, T1:], o1[2])
+    assert np.abs(np.concatenate([o1[0], o2[0]], 1) - ref[0]).max() < 1e-13
+    assert np.abs(np.concatenate([o1[1], o2[1]], 1) - ref[1]).max() < 1e-13
+    assert np.abs(o2[2] - ref[2]).max() < 1e-13
+
+
+# ----------------------------------------------------------------------------
+# P8: affine transfer (Theorem "Exact affine chunk transfer")
+# ----------------------------------------------------------------------------
+def test_affine_transfer_against_dense_sum():
+    T, m, dv = 12, 5, 3
+    q, k, v, al, th, be, S0 = rand_inputs(19, 1, T, m, dv)
+    kc = cplx(k[0])
+    _, states, As = dense_forward(q[0], k[0], v[0], al[0], th[0], be[0], S0[0])
+    # B^chunk = sum_i A_{C:i+1} B_i with dense products
+    Bc = np.zeros((m, dv), complex)
+    for i in range(T):
+        P = np.eye(m, dtype=complex)
+        for s in range(i + 1, T):
+            P = As[s] @ P
+        Bc += P @ (be[0, i] * np.outer(kc[i], v[0, i]))
+    G, Y, W, M = chunk_wy.chunk_factors(kc, al[0], th[0], be[0])
+    S0c = S0[0][0::2] + 1j * S0[0][1::2]
+    S_out = G[:, None] * S0c - Y @ (M @ (W.conj().T @ S0c)) + Bc
+    assert np.abs(S_out - states[-1]).max() < 1e-13
+    # zero-state run of the C oracle gives the same write summary
+    _, _, ST0 = run_rec(q, k, v, al, th, be, None)
+    assert np.abs((ST0[0][0::2] + 1j * ST0[0][1::2]) - Bc).max() < 1e-13
+
+
+# ----------------------------------------------------------------------------
+# P9/P10: rank and stability (Cor. "SFDA admits exact constructive block-WY products",
+# Prop. "Basic numerical stability")
+# ----------------------------------------------------------------------------
+@pytest.mark.parametrize("m,C", [(8, 4), (8, 8), (6, 10)])
+def test_correction_rank(m, C):
+    _, k, _, al, th, be, _ = rand_inputs(20, 1, C, m, 1)
+    be = np.maximum(be, 0.2)
+    G, Y, W, M = chunk_wy.chunk_factors(cplx(k[0]), al[0], th[0], be[0])
+    corr = Y @ M @ W.conj().T
+    assert np.linalg.matrix_rank(corr, tol=1e-10) == min(C, m)
+
+
+def test_spectral_and_frobenius_bounds():
+    N, T, m, dv = 1, 200, 6, 4
+    q, k, v, al, th, be, S0 = rand_inputs(21, N, T, m, dv, alpha_lo=0.0)
+    kc = cplx(k[0])
+    worst = 0.0
+    for t in range(T):
+        worst = max(worst, np.linalg.norm(dense_A(kc[t], al[0, t], th[0, t], be[0, t]), 2))
+    assert worst <= 1.0 + 1e-12
+    bound = np.linalg.norm(S0[0]) + np.cumsum(be[0] * np.linalg.norm(k[0], axis=1) * np.linalg.norm(v[0], axis=1))
+    for Tcut in (1, 50, 200):
+        _, _, ST = run_rec(q[:, :Tcut], k[:, :Tcut], v[:, :Tcut], al[:, :Tcut], th[:, :Tcut], be[:, :Tcut], S0)
+        assert np.linalg.norm(ST[0]) <= bound[Tcut - 1] + 1e-9
+
+
+# ----------------------------------------------------------------------------
+# P11: block-WY closure (Theorem "Block-WY closure") on two exported chunk tuples
+# ----------------------------------------------------------------------------
+def test_closure_of_two_chunks():
+    m, C = 6, 5
+    _, k, _, al, th, be, _ = rand_inputs(22, 1, 2 * C, m, 1)
+    kc = cplx(k[0])
+    G1, Y1, W1, M1 = chunk_wy.chunk_factors(kc[:C], al[0, :C], th[0, :C], be[0, :C])
+    G2, Y2, W2, M2 = chunk_wy.chunk_factors(kc[C:], al[0, C:], th[0, C:], be[0, C:])
+    G21 = G2 * G1
+    Y21 = np.concatenate([G2[:, None] * Y1, Y2], 1)
+    W21 = np.concatenate([W1, np.conj(G1)[:, None] * W2], 1)
+    M21 = np.block([[M1, np.zeros((C, C))], [-M2 @ W2.conj().T @ Y1 @ M1, M2]])
+    P = np.eye(m, dtype=complex)
+    for t in range(2 * C):
+        P = dense_A(kc[t], al[0, t], th[0, t], be[0, t]) @ P
+    assert np.abs(np.diag(G21) - Y21 @ M21 @ W21.conj().T - P).max() < 1e-13
+    # and the 2C-token recursion yields exactly these composed factors
+    G, Y, W, M = chunk_wy.chunk_factors(kc, al[0], th[0], be[0])
+    assert np.abs(G - G21).max() < 1e-13 and np.abs(Y - Y21).max() < 1e-13
+    assert np.abs(W - W21).max() < 1e-13 and np.abs(M - M21).max() < 1e-12
+
+
+# ----------------------------------------------------------------------------
+# P12: realification (Prop. "Complex phases are real block rotations")
+# ----------------------------------------------------------------------------
+def test_real_block_formulation():
+    """Same map on R^{2m}: 2x2 blocks alpha R(theta); the complex rank-one k k^*
+    is the real rank-two projector k k^T + (Jk)(Jk)^T."""
+    T, m, dv = 25, 4, 3
+    q, k, v, al, th, be, S0 = rand_inputs(23, 1, T, m, dv)
+    o_re, o_im, ST = run_rec(q, k, v, al, th, be, S0)
+    S = S0[0].copy()
+    J = np.kron(np.eye(m), np.array([[0.0, -1.0], [1.0, 0.0]]))
+    for t in range(T):
+        Lam = np.zeros((2 * m, 2 * m))
+        for j in range(m):
+            c, s = np.cos(th[0, t, j]), np.sin(th[0, t, j])
+            Lam[2 * j:2 * j + 2, 2 * j:2 * j + 2] = al[0, t, j] * np.array([[c, -s], [s, c]])
+        kr = k[0, t]
+        Jk = J @ kr
+        E = np.eye(2 * m) - be[0, t] * (np.outer(kr, kr) + np.outer(Jk, Jk))
+        S = E @ Lam @ S + be[0, t] * np.outer(kr, v[0, t])
+        assert np.abs(o_re[0, t] - S.T @ q[0, t]).max() < 1e-12
+        assert np.abs(o_im[0, t] + S.T @ (J @ q[0, t])).max() < 1e-12
+    assert np.abs(ST[0] - S).max() < 1e-12
+
+
+# ----------------------------------------------------------------------------
+# closed forms the GPU kernels use, checked against the literal recursion
+# ----------------------------------------------------------------------------
+def test_closed_form_factors():
+    m, C = 7, 12
+    _, k, _, al, th, be, _ = rand_inputs(24, 1, C, m, 1)
+    kc = cplx(k[0])
+    G, Y, W, M = chunk_wy.chunk_factors(kc, al[0], th[0], be[0])
+    gam = np.cumprod(al[0] * np.exp(1j * th[0]), axis=0)           # gamma_t
+    assert np.abs(G - gam[-1]).max() < 1e-14
+    assert np.abs(W - (np.conj(gam) * kc).T).max() < 1e-14
+    assert np.abs(Y - ((gam[-1] / gam) * be[0][:, None] * kc).T).max() < 1e-13
+    Kt = np.zeros((C, C), complex)
+    for t in range(C):
+        for i in range(t):
+            Kt[t, i] = np.sum(np.conj(kc[t]) * (gam[t] / gam[i]) * kc[i])
+    N = Kt * be[0][None, :]
+    assert np.abs(M - np.linalg.inv(np.eye(C) + N)).max() < 1e-12
+
+
+# ----------------------------------------------------------------------------
+# integer bookkeeping
+# ----------------------------------------------------------------------------
+PI50 = "3.14159265358979323846264338327950288419716939937510"
+
+
+def test_phase_turns_match_exact_rational_rounding():
+    from decimal import Decimal, getcontext, ROUND_HALF_EVEN
+    getcontext().prec = 60
+    rng = np.random.default_rng(25)
+    th = np.concatenate([rng.uniform(-np.pi, np.pi, 2000), [0.0, np.pi, -np.pi, 1e-9, -1e-9, 100.0, -7.5]]).astype(np.float32)
+    got = bookkeeping.phase_to_turns(th)
+    scale = Decimal(2 ** 32) / (2 * Decimal(PI50))
+    exact_mismatch = 0
+    for x, g in zip(th, got):
+        e = int((Decimal(float(x)) * scale).to_integral_value(rounding=ROUND_HALF_EVEN)) % 2 ** 32
+        d = (int(g) - e) % 2 ** 32
+        assert d in (0, 1, 2 ** 32 - 1)        # double rounding may move a near-tie by one unit
+        exact_mismatch += d != 0
+    assert exact_mismatch <= 2
+    assert np.array_equal(bookkeeping.phase_to_turns(-th), (-got.astype(np.int64) & 0xFFFFFFFF).astype(np.uint32))
+
+
+def test_cumulative_turns_are_chunk_local_integer_sums():
+    rng = np.random.default_rng(26)
+    T, m, C = 50, 3, 16
+    th = rng.uniform(-np.pi, np.pi, (2, T, m)).astype(np.float32)
+    u = bookkeeping.phase_to_turns(th)
+    cum = bookkeeping.cumulative_phase_turns(th, C)
+    for n in range(2):
+        for j in range(m):
+            acc = 0
+            for t in range(T):
+                if t % C == 0:
+                    acc = 0
+                acc = (acc + int(u[n, t, j])) % 2 ** 32
+                assert int(cum[n, t, j]) == acc
+    # quantised phases: p steps of 2 pi / p come back to within p rounding units of zero
+    for p in (2, 3, 5, 7):
+        thp = np.full((1, p, 1), 2 * np.pi / p, np.float32)
+        last = int(bookkeeping.cumulative_phase_turns(thp, 64)[0, -1, 0])
+        dist = min(last, 2 ** 32 - last)
+        assert dist <= 2 ** 32 * 2.0 ** -24 * p      # float32 spacing of theta, p times
+    assert int(bookkeeping.cumulative_phase_turns(np.full((1, 2, 1), np.pi, np.float32), 64)[0, -1, 0]) \
+        == (2 * int(bookkeeping.phase_to_turns(np.float32(np.pi)))) % 2 ** 32
+
+
+def test_chunk_plan():
+    assert bookkeeping.chunk_plan(256, 16) == (16, 16)
+    assert bookkeeping.chunk_plan(257, 16) == (17, 1)
+    assert bookkeeping.chunk_plan(5, 64) == (1, 5)
+    assert bookkeeping.chunk_plan(131072, 64) == (2048, 64)
+    with pytest.raises(ValueError):
+        bookkeeping.chunk_plan(0, 16)
