@@ -1,0 +1,188 @@
+/*
+ * sfda.h -- C ABI of the B200 (sm_100a) Semidirect Fourier Delta Attention library.
+ *
+ * The library computes the chunkwise constructive chunk-WY forward, the per-chunk
+ * factor export and the one-token decode step of the tied SFDA recurrence
+ * (Section 3, Eq. "sfda"):
+ *
+ *     S_t = (I - beta_t k_t k_t^*) Lambda_t S_{t-1} + beta_t k_t v_t^*,
+ *     Lambda_t = diag(alpha_t * exp(i theta_t)),        o_t = S_t^* q_t.
+ *
+ * Storage conventions shared by every entry point
+ * -----------------------------------------------
+ *  - All tensors are dense, row-major, with the index order written beside them.
+ *  - The key space is R^{d_k} ~ C^m, m = d_k / 2: real channel 2j is the real part
+ *    and channel 2j+1 the imaginary part of complex coordinate j (the aligned 2x2
+ *    rotation-decay blocks of Prop. "Complex phases are real block rotations").
+ *    This holds for q, k and for the ROWS of a state S[d_k][d_v].
+ *  - v, o and the columns of S are plain real channels (v real, so v^* = v^T).
+ *  - alpha, theta are per complex coordinate ([..., m]); beta is one scalar per
+ *    token and head.  alpha in (0, 1], beta in [0, 1], |k| <= 1 are preconditions
+ *    of the method (Prop. "Basic numerical stability"); they are NOT checked, and
+ *    k is not normalised here.
+ *  - `dtype` selects the element type of q, k, v, o, o_im: SFDA_F32 (float) or
+ *    SFDA_BF16 (bfloat16).  alpha, theta, beta and every state are float.
+ *  - o = Re(S_t^* q_t);  o_im = Im(S_t^* q_t) is written when o_im is not NULL.
+ *
+ * Ownership and execution
+ * -----------------------
+ *  Unless an argument says "host", pointers are DEVICE pointers owned by the
+ *  caller; they must be 16-byte aligned.  The library allocates and frees nothing,
+ *  never synchronises, and enqueues all work on `stream` (a cudaStream_t passed as
+ *  void*; NULL is the default stream).  Results are ready when the stream reaches
+ *  the end of the enqueued work.
+ *
+ * Errors
+ * ------
+ *  Every int-returning function returns SFDA_OK (0) or a negative sfda_status.
+ *  Arguments are validated on the host before anything is launched; on an error
+ *  nothing has been enqueued.  No exceptions, no exit(), no output.
+ */
+#ifndef SFDA_H
+#define SFDA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define SFDA_API __attribute__((visibility("default")))
+#else
+#define SFDA_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SFDA_OK = 0,
+    SFDA_ERR_NULL = -1,        /* a required pointer is NULL                          */
+    SFDA_ERR_SHAPE = -2,       /* B, T, H < 1, odd d_k, non-positive chunk            */
+    SFDA_ERR_UNSUPPORTED = -3, /* d_k, d_v not in {64,128}; chunk not in {16,32,64};  */
+                               /* unknown dtype                                       */
+    SFDA_ERR_ALIGN = -4,       /* a pointer is not 16-byte aligned                    */
+    SFDA_ERR_WORKSPACE = -5,   /* workspace NULL or smaller than sfda_workspace_bytes */
+    SFDA_ERR_CUDA = -6,        /* the CUDA runtime reported an error at launch        */
+    SFDA_ERR_TIMEOUT = -7      /* a bounded device-side wait ran out                  */
+} sfda_status;
+
+typedef enum { SFDA_F32 = 0, SFDA_BF16 = 1 } sfda_dtype;
+
+/* Text for a status code (static storage, never NULL). Host only. */
+SFDA_API const char *sfda_status_string(int status);
+
+/*
+ * Chunk bookkeeping (host only, integer).  Chunks are [j*chunk, (j+1)*chunk); the
+ * factors restart at every chunk (Gamma_0 = I, Theorem "Constructive left-to-right
+ * chunk-WY recursion").  T need not be a multiple of chunk: the last chunk holds
+ * tail_len tokens and is completed with neutral tokens (alpha = 1, theta = 0,
+ * beta = 0, k = q = v = 0, for which A_t = I and B_t = 0 by Eq. "AtBt").
+ * Writes n_chunks = ceil(T / chunk) and tail_len in [1, chunk].
+ */
+SFDA_API int sfda_plan(int T, int chunk, int *n_chunks, int *tail_len);
+
+/*
+ * Bytes of device scratch sfda_forward needs for these sizes (0 when it needs
+ * none).  Returns 0 for invalid sizes as well; sfda_forward reports those.
+ */
+SFDA_API size_t sfda_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int dtype);
+
+/*
+ * Chunkwise forward: o_t for every token and the final state, by Algorithm 1
+ * ("Constructive SFDA-WY chunk summary"), Eq. "apply-transfer" and Theorem "Prefix
+ * outputs inside a chunk", scanning boundary states over the chunks of every
+ * (batch, head) pair (the "boundary-state scan").
+ *
+ *  q, k   [B][T][H][d_k]   dtype          v   [B][T][H][d_v]  dtype
+ *  alpha, theta [B][T][H][m] float        beta [B][T][H]      float
+ *  S0     [B][H][d_k][d_v] float, or NULL for a zero initial state
+ *  o      [B][T][H][d_v]   dtype          o_im same shape, or NULL
+ *  S_T    [B][H][d_k][d_v] float, or NULL; may alias S0
+ *  workspace: device scratch of at least sfda_workspace_bytes(...) bytes (may be
+ *             NULL when that is 0); contents are clobbered.
+ *
+ * Supported: d_k, d_v in {64, 128}; chunk in {16, 32, 64}.
+ * bf16 inputs with d_k = d_v = 128 and chunk = 64 take the tensor-core path
+ * (bf16 operands, fp32 accumulation and state); everything else runs in fp32 on
+ * the CUDA cores.  The tensor-core path forms 1/gamma_t inside a chunk and so
+ * additionally assumes prod_{t in chunk} alpha_{t,j} >= exp(-80) for every
+ * coordinate j; beyond that results lose accuracy but stay finite.
+ */
+SFDA_API int sfda_forward(const void *q, const void *k, const void *v,
+                 const float *alpha, const float *theta, const float *beta,
+                 const float *S0, void *o, void *o_im, float *S_T,
+                 int B, int T, int H, int d_k, int d_v, int chunk, int dtype,
+                 void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Same computation forced onto the fp32 CUDA-core path for any dtype (the
+ * reference path of this library; used to cross-check the tensor-core path).
+ * Needs no workspace.
+ */
+SFDA_API int sfda_forward_simt(const void *q, const void *k, const void *v,
+                      const float *alpha, const float *theta, const float *beta,
+                      const float *S0, void *o, void *o_im, float *S_T,
+                      int B, int T, int H, int d_k, int d_v, int chunk, int dtype,
+                      void *stream);
+
+/*
+ * Per-chunk factors of P = A_C ... A_1 = Gamma - Y M W^* in the convention of
+ * Theorem "Constructive left-to-right chunk-WY recursion" with u_t = beta_t k_t,
+ * r_t = Lambda_t^* k_t (Cor. "SFDA admits exact constructive block-WY products"):
+ *
+ *  Gamma [B][H][NC][m][2]       gamma_C = prod_t lambda_t          (Re, Im)
+ *  Y     [B][H][NC][m][C][2]    Y[:,t] = (gamma_C / gamma_t) beta_t k_t
+ *  M     [B][H][NC][C][C][2]    unit lower triangular
+ *  W     [B][H][NC][m][C][2]    W[:,t] = conj(gamma_t) k_t
+ *  phase_turns [B][T][H][m] uint32, or NULL: the chunk-local inclusive prefix sum,
+ *         modulo 2^32, of  rint((double)theta * 2^32 / (2 pi))  -- the integer
+ *         cumulative phase every kernel of this library derives gamma's angle from.
+ *
+ * NC = ceil(T / chunk), C = chunk.  Columns (and rows of M) of padded tail tokens
+ * are those of neutral tokens (zero columns in Y and W, identity rows in M).
+ * Any of Gamma, Y, M, W may be NULL to skip that output.  fp32 arithmetic.
+ */
+SFDA_API int sfda_chunk_factors(const void *k, const float *alpha, const float *theta, const float *beta,
+                       float *Gamma, float *Y, float *M, float *W, uint32_t *phase_turns,
+                       int B, int T, int H, int d_k, int chunk, int dtype, void *stream);
+
+/*
+ * One-token recurrent decode: one application of Eq. "sfda" followed by
+ * o = S^* q, for B*H independent states, updating S in place.
+ *
+ *  q, k [B][H][d_k] dtype     v [B][H][d_v] dtype
+ *  alpha, theta [B][H][m] float     beta [B][H] float
+ *  S [B][H][d_k][d_v] float, read and overwritten
+ *  o [B][H][d_v] dtype;  o_im same shape or NULL
+ */
+SFDA_API int sfda_step(const void *q, const void *k, const void *v,
+              const float *alpha, const float *theta, const float *beta,
+              float *S, void *o, void *o_im,
+              int B, int H, int d_k, int d_v, int dtype, void *stream);
+
+/*
+ * Host-buffer forward: the call a user with data in host memory makes.  Copies the
+ * inputs from HOST memory (pinned for asynchronous copies) into `arena`, runs
+ * sfda_forward there and copies o (and o_im, S_T when not NULL) back to HOST
+ * memory, all enqueued on `stream`.  Host pointers: q, k, v, alpha, theta, beta,
+ * S0, o, o_im, S_T.  Device pointer: arena, at least sfda_forward_host_arena_bytes
+ * bytes, 256-byte aligned, clobbered.  bytes_h2d / bytes_d2h (host, may be NULL)
+ * receive the bytes copied in each direction.
+ */
+SFDA_API size_t sfda_forward_host_arena_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int dtype,
+                                     int want_o_im, int have_S0, int want_S_T);
+SFDA_API int sfda_forward_host(const void *q, const void *k, const void *v,
+                      const float *alpha, const float *theta, const float *beta,
+                      const float *S0, void *o, void *o_im, float *S_T,
+                      int B, int T, int H, int d_k, int d_v, int chunk, int dtype,
+                      void *arena, size_t arena_bytes, void *stream,
+                      size_t *bytes_h2d, size_t *bytes_d2h);
+
+/* Number of kernels the last sfda_forward / sfda_step / sfda_chunk_factors call of
+ * this thread enqueued (host only; for launch accounting in benchmarks). */
+SFDA_API int sfda_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SFDA_H */

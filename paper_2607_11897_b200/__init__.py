@@ -1,0 +1,13 @@
+"""Python binding of the SFDA C-ABI library (``libsfda.so``, hand-written CUDA for sm_100a).
+
+Argument marshalling only: every step of the path runs in the library's kernels.
+PyTorch is used for device memory and streams.  There is no CPU or PyTorch
+fallback: a missing library raises.
+"""
+from .binding import (SFDA_BF16, SFDA_F32, SfdaError, last_launch_count, lib_path, load, sfda_chunk_factors,
+                      sfda_forward, sfda_forward_host, sfda_forward_host_arena_bytes, sfda_forward_simt, sfda_plan, sfda_status_string, sfda_step,
+                      sfda_workspace_bytes)
+
+__all__ = ["SFDA_BF16", "SFDA_F32", "SfdaError", "last_launch_count", "lib_path", "load", "sfda_chunk_factors",
+           "sfda_forward", "sfda_forward_host", "sfda_forward_host_arena_bytes", "sfda_forward_simt", "sfda_plan", "sfda_status_string", "sfda_step",
+           "sfda_workspace_bytes"]

@@ -1,0 +1,186 @@
+"""ctypes marshalling for ``include/sfda.h``.  Same names, same argument order."""
+import ctypes
+import os
+
+import torch
+
+SFDA_F32, SFDA_BF16 = 0, 1
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB = None
+
+_vp, _ci, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+
+
+class SfdaError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__("%s failed: %d (%s)" % (where, status, sfda_status_string(status)))
+
+
+def lib_path() -> str:
+    return os.path.join(_HERE, "libsfda.so")
+
+
+def load():
+    """Load ``libsfda.so``; raise if it has not been built (no fallback exists)."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = lib_path()
+    if not os.path.exists(path):
+        raise ImportError("%s is missing: run `python -m paper_2607_11897_b200.build` "
+                          "(or __graft_entry__.build()) first" % path)
+    lib = ctypes.CDLL(path)
+    lib.sfda_status_string.restype = ctypes.c_char_p
+    lib.sfda_status_string.argtypes = [_ci]
+    lib.sfda_plan.argtypes = [_ci, _ci, ctypes.POINTER(_ci), ctypes.POINTER(_ci)]
+    lib.sfda_workspace_bytes.restype = _sz
+    lib.sfda_workspace_bytes.argtypes = [_ci] * 7
+    lib.sfda_forward.argtypes = [_vp] * 10 + [_ci] * 7 + [_vp, _sz, _vp]
+    lib.sfda_forward_simt.argtypes = [_vp] * 10 + [_ci] * 7 + [_vp]
+    lib.sfda_chunk_factors.argtypes = [_vp] * 9 + [_ci] * 6 + [_vp]
+    lib.sfda_step.argtypes = [_vp] * 9 + [_ci] * 5 + [_vp]
+    lib.sfda_forward_host_arena_bytes.restype = _sz
+    lib.sfda_forward_host_arena_bytes.argtypes = [_ci] * 10
+    lib.sfda_forward_host.argtypes = [_vp] * 10 + [_ci] * 7 + [_vp, _sz, _vp, ctypes.POINTER(_sz),
+                                                          ctypes.POINTER(_sz)]
+    lib.sfda_last_launch_count.restype = _ci
+    _LIB = lib
+    return lib
+
+
+def sfda_status_string(status: int) -> str:
+    return load().sfda_status_string(int(status)).decode()
+
+
+def last_launch_count() -> int:
+    return int(load().sfda_last_launch_count())
+
+
+def sfda_plan(T: int, chunk: int):
+    n, tail = _ci(), _ci()
+    rc = load().sfda_plan(T, chunk, ctypes.byref(n), ctypes.byref(tail))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_plan")
+    return n.value, tail.value
+
+
+def sfda_workspace_bytes(B, T, H, d_k, d_v, chunk, dtype) -> int:
+    return int(load().sfda_workspace_bytes(B, T, H, d_k, d_v, chunk, dtype))
+
+
+def _ptr(t):
+    return None if t is None else _vp(t.data_ptr())
+
+
+def _dtype_code(t):
+    if t.dtype == torch.float32:
+        return SFDA_F32
+    if t.dtype == torch.bfloat16:
+        return SFDA_BF16
+    raise TypeError("q, k, v must be float32 or bfloat16")
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return _vp(s.cuda_stream)
+
+
+def _check(t, name, dtype=None, device="cuda"):
+    if t is None:
+        return
+    if not t.is_contiguous():
+        raise ValueError(name + " must be contiguous")
+    if t.device.type != device:
+        raise ValueError("%s must live on %s" % (name, device))
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError("%s must be %s" % (name, dtype))
+
+
+def _forward_common(fn_name, q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chunk, workspace, stream):
+    lib = load()
+    B, T, H, d_k = q.shape
+    d_v = v.shape[-1]
+    dt = _dtype_code(q)
+    for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o"), (o_im, "o_im")):
+        _check(t, n, q.dtype)
+    for t, n in ((alpha, "alpha"), (theta, "theta"), (beta, "beta"), (S0, "S0"), (S_T, "S_T")):
+        _check(t, n, torch.float32)
+    if fn_name == "sfda_forward":
+        ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+        rc = lib.sfda_forward(_ptr(q), _ptr(k), _ptr(v), _ptr(alpha), _ptr(theta), _ptr(beta), _ptr(S0), _ptr(o),
+                              _ptr(o_im), _ptr(S_T), B, T, H, d_k, d_v, chunk, dt, _ptr(workspace), ws_bytes,
+                              _stream(stream))
+    else:
+        rc = lib.sfda_forward_simt(_ptr(q), _ptr(k), _ptr(v), _ptr(alpha), _ptr(theta), _ptr(beta), _ptr(S0),
+                                   _ptr(o), _ptr(o_im), _ptr(S_T), B, T, H, d_k, d_v, chunk, dt, _stream(stream))
+    if rc != 0:
+        raise SfdaError(rc, fn_name)
+
+
+def sfda_forward(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chunk, workspace=None, stream=None):
+    """``sfda_forward`` of ``include/sfda.h``; tensors are CUDA tensors the caller allocated."""
+    _forward_common("sfda_forward", q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chunk, workspace, stream)
+
+
+def sfda_forward_simt(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chunk, stream=None):
+    """``sfda_forward_simt`` of ``include/sfda.h`` (fp32 CUDA-core path for any dtype)."""
+    _forward_common("sfda_forward_simt", q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chunk, None, stream)
+
+
+def sfda_chunk_factors(k, alpha, theta, beta, Gamma, Y, M, W, phase_turns, chunk, stream=None):
+    """``sfda_chunk_factors`` of ``include/sfda.h``; any output may be None."""
+    B, T, H, d_k = k.shape
+    _check(k, "k")
+    for t, n in ((alpha, "alpha"), (theta, "theta"), (beta, "beta"), (Gamma, "Gamma"), (Y, "Y"), (M, "M"),
+                 (W, "W")):
+        _check(t, n, torch.float32)
+    _check(phase_turns, "phase_turns", torch.int32)
+    rc = load().sfda_chunk_factors(_ptr(k), _ptr(alpha), _ptr(theta), _ptr(beta), _ptr(Gamma), _ptr(Y), _ptr(M),
+                                   _ptr(W), _ptr(phase_turns), B, T, H, d_k, chunk, _dtype_code(k),
+                                   _stream(stream))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_chunk_factors")
+
+
+def sfda_step(q, k, v, alpha, theta, beta, S, o, o_im, stream=None):
+    """``sfda_step`` of ``include/sfda.h``; S is updated in place."""
+    B, H, d_k = q.shape
+    d_v = v.shape[-1]
+    for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o"), (o_im, "o_im")):
+        _check(t, n, q.dtype)
+    for t, n in ((alpha, "alpha"), (theta, "theta"), (beta, "beta"), (S, "S")):
+        _check(t, n, torch.float32)
+    rc = load().sfda_step(_ptr(q), _ptr(k), _ptr(v), _ptr(alpha), _ptr(theta), _ptr(beta), _ptr(S), _ptr(o),
+                          _ptr(o_im), B, H, d_k, d_v, _dtype_code(q), _stream(stream))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_step")
+
+
+def sfda_forward_host(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chunk, arena, stream=None):
+    """``sfda_forward_host``: q..S_T are HOST tensors (pinned), arena a CUDA byte tensor.
+
+    Returns (bytes_h2d, bytes_d2h) the call copied.
+    """
+    lib = load()
+    B, T, H, d_k = q.shape
+    d_v = v.shape[-1]
+    dt = _dtype_code(q)
+    for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o"), (o_im, "o_im")):
+        _check(t, n, q.dtype, "cpu")
+    for t, n in ((alpha, "alpha"), (theta, "theta"), (beta, "beta"), (S0, "S0"), (S_T, "S_T")):
+        _check(t, n, torch.float32, "cpu")
+    _check(arena, "arena")
+    h2d, d2h = _sz(), _sz()
+    rc = lib.sfda_forward_host(_ptr(q), _ptr(k), _ptr(v), _ptr(alpha), _ptr(theta), _ptr(beta), _ptr(S0), _ptr(o),
+                               _ptr(o_im), _ptr(S_T), B, T, H, d_k, d_v, chunk, dt, _ptr(arena),
+                               arena.numel() * arena.element_size(), _stream(stream), ctypes.byref(h2d),
+                               ctypes.byref(d2h))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_forward_host")
+    return h2d.value, d2h.value
+
+
+def sfda_forward_host_arena_bytes(B, T, H, d_k, d_v, chunk, dtype, want_o_im, have_S0, want_S_T) -> int:
+    return int(load().sfda_forward_host_arena_bytes(B, T, H, d_k, d_v, chunk, dtype, int(want_o_im), int(have_S0),
+                                                    int(want_S_T)))

@@ -1,0 +1,238 @@
+// C ABI of the library: argument validation on the host, dispatch to the kernels.
+#include "../../include/sfda.h"
+
+#include "sfda_internal.h"
+
+namespace {
+
+thread_local int g_last_launches = 0;
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_dims(int d_k, int d_v, int chunk, int dtype)
+{
+    if (d_k < 2 || (d_k & 1) || d_v < 1 || chunk < 1) return SFDA_ERR_SHAPE;
+    if (d_k != 64 && d_k != 128) return SFDA_ERR_UNSUPPORTED;
+    if (d_v != 64 && d_v != 128) return SFDA_ERR_UNSUPPORTED;
+    if (chunk != 16 && chunk != 32 && chunk != 64) return SFDA_ERR_UNSUPPORTED;
+    if (dtype != SFDA_F32 && dtype != SFDA_BF16) return SFDA_ERR_UNSUPPORTED;
+    return SFDA_OK;
+}
+
+size_t elem_bytes(int dtype) { return dtype == SFDA_BF16 ? 2 : 4; }
+
+int validate_forward(const void *q, const void *k, const void *v, const float *alpha, const float *theta,
+                     const float *beta, const float *S0, void *o, void *o_im, float *S_T, int B, int T, int H,
+                     int d_k, int d_v, int chunk, int dtype)
+{
+    if (!q || !k || !v || !alpha || !theta || !beta || !o) return SFDA_ERR_NULL;
+    if (B < 1 || T < 1 || H < 1) return SFDA_ERR_SHAPE;
+    const int rc = check_dims(d_k, d_v, chunk, dtype);
+    if (rc != SFDA_OK) return rc;
+    const void *ptrs[] = {q, k, v, alpha, theta, beta, S0, o, o_im, S_T};
+    for (const void *p : ptrs)
+        if (p && !aligned16(p)) return SFDA_ERR_ALIGN;
+    return SFDA_OK;
+}
+
+sfda::ForwardArgs pack(const void *q, const void *k, const void *v, const float *alpha, const float *theta,
+                       const float *beta, const float *S0, void *o, void *o_im, float *S_T, int B, int T, int H,
+                       int d_k, int d_v, int chunk, int dtype)
+{
+    sfda::ForwardArgs a;
+    a.q = q; a.k = k; a.v = v; a.alpha = alpha; a.theta = theta; a.beta = beta; a.S0 = S0;
+    a.o = o; a.o_im = o_im; a.S_T = S_T;
+    a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.chunk = chunk; a.dtype = dtype;
+    return a;
+}
+
+size_t round256(size_t x) { return (x + 255u) & ~(size_t)255u; }
+
+}  // namespace
+
+extern "C" {
+
+const char *sfda_status_string(int status)
+{
+    switch (status) {
+        case SFDA_OK: return "ok";
+        case SFDA_ERR_NULL: return "a required pointer is NULL";
+        case SFDA_ERR_SHAPE: return "invalid shape (B, T, H >= 1; d_k even; chunk >= 1)";
+        case SFDA_ERR_UNSUPPORTED: return "unsupported d_k / d_v / chunk / dtype";
+        case SFDA_ERR_ALIGN: return "a pointer is not 16-byte aligned";
+        case SFDA_ERR_WORKSPACE: return "workspace missing or too small";
+        case SFDA_ERR_CUDA: return "CUDA runtime error at launch";
+        case SFDA_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        default: return "unknown status";
+    }
+}
+
+int sfda_plan(int T, int chunk, int *n_chunks, int *tail_len)
+{
+    if (!n_chunks || !tail_len) return SFDA_ERR_NULL;
+    if (T < 1 || chunk < 1) return SFDA_ERR_SHAPE;
+    const int nc = (T + chunk - 1) / chunk;
+    *n_chunks = nc;
+    *tail_len = T - (nc - 1) * chunk;
+    return SFDA_OK;
+}
+
+size_t sfda_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int dtype)
+{
+    (void)B; (void)T; (void)H; (void)d_k; (void)d_v; (void)chunk; (void)dtype;
+    return 0;
+}
+
+int sfda_forward_simt(const void *q, const void *k, const void *v, const float *alpha, const float *theta,
+                      const float *beta, const float *S0, void *o, void *o_im, float *S_T, int B, int T, int H,
+                      int d_k, int d_v, int chunk, int dtype, void *stream)
+{
+    g_last_launches = 0;
+    const int rc = validate_forward(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
+    if (rc != SFDA_OK) return rc;
+    const sfda::ForwardArgs a = pack(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
+    return sfda::launch_forward_simt(a, static_cast<cudaStream_t>(stream), &g_last_launches) == cudaSuccess
+               ? SFDA_OK
+               : SFDA_ERR_CUDA;
+}
+
+int sfda_forward(const void *q, const void *k, const void *v, const float *alpha, const float *theta,
+                 const float *beta, const float *S0, void *o, void *o_im, float *S_T, int B, int T, int H, int d_k,
+                 int d_v, int chunk, int dtype, void *workspace, size_t workspace_bytes, void *stream)
+{
+    g_last_launches = 0;
+    const int rc = validate_forward(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
+    if (rc != SFDA_OK) return rc;
+    const size_t need = sfda_workspace_bytes(B, T, H, d_k, d_v, chunk, dtype);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return SFDA_ERR_WORKSPACE;
+    if (workspace && !aligned16(workspace)) return SFDA_ERR_ALIGN;
+    const sfda::ForwardArgs a = pack(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
+    return sfda::launch_forward_simt(a, static_cast<cudaStream_t>(stream), &g_last_launches) == cudaSuccess
+               ? SFDA_OK
+               : SFDA_ERR_CUDA;
+}
+
+int sfda_chunk_factors(const void *k, const float *alpha, const float *theta, const float *beta, float *Gamma,
+                       float *Y, float *M, float *W, uint32_t *phase_turns, int B, int T, int H, int d_k, int chunk,
+                       int dtype, void *stream)
+{
+    g_last_launches = 0;
+    if (!k || !alpha || !theta || !beta) return SFDA_ERR_NULL;
+    if (B < 1 || T < 1 || H < 1) return SFDA_ERR_SHAPE;
+    const int rc = check_dims(d_k, 64, chunk, dtype);
+    if (rc != SFDA_OK) return rc;
+    const void *ptrs[] = {k, alpha, theta, beta, Gamma, Y, M, W, phase_turns};
+    for (const void *p : ptrs)
+        if (p && !aligned16(p)) return SFDA_ERR_ALIGN;
+    sfda::FactorArgs a;
+    a.k = k; a.alpha = alpha; a.theta = theta; a.beta = beta;
+    a.Gamma = Gamma; a.Y = Y; a.M = M; a.W = W; a.phase_turns = phase_turns;
+    a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.chunk = chunk; a.dtype = dtype;
+    return sfda::launch_chunk_factors(a, static_cast<cudaStream_t>(stream), &g_last_launches) == cudaSuccess
+               ? SFDA_OK
+               : SFDA_ERR_CUDA;
+}
+
+int sfda_step(const void *q, const void *k, const void *v, const float *alpha, const float *theta,
+              const float *beta, float *S, void *o, void *o_im, int B, int H, int d_k, int d_v, int dtype,
+              void *stream)
+{
+    g_last_launches = 0;
+    if (!q || !k || !v || !alpha || !theta || !beta || !S || !o) return SFDA_ERR_NULL;
+    if (B < 1 || H < 1) return SFDA_ERR_SHAPE;
+    const int rc = check_dims(d_k, d_v, 64, dtype);
+    if (rc != SFDA_OK) return rc;
+    const void *ptrs[] = {q, k, v, alpha, theta, beta, S, o, o_im};
+    for (const void *p : ptrs)
+        if (p && !aligned16(p)) return SFDA_ERR_ALIGN;
+    sfda::StepArgs a;
+    a.q = q; a.k = k; a.v = v; a.alpha = alpha; a.theta = theta; a.beta = beta;
+    a.S = S; a.o = o; a.o_im = o_im;
+    a.B = B; a.H = H; a.d_k = d_k; a.d_v = d_v; a.dtype = dtype;
+    return sfda::launch_step(a, static_cast<cudaStream_t>(stream), &g_last_launches) == cudaSuccess ? SFDA_OK
+                                                                                                    : SFDA_ERR_CUDA;
+}
+
+size_t sfda_forward_host_arena_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int dtype, int want_o_im,
+                                     int have_S0, int want_S_T)
+{
+    if (B < 1 || T < 1 || H < 1 || check_dims(d_k, d_v, chunk, dtype) != SFDA_OK) return 0;
+    const size_t n = (size_t)B * T * H, eb = elem_bytes(dtype), m = d_k / 2;
+    size_t total = 0;
+    total += 2 * round256(n * d_k * eb);                      // q, k
+    total += round256(n * d_v * eb);                          // v
+    total += 2 * round256(n * m * 4) + round256(n * 4);       // alpha, theta, beta
+    total += (want_o_im ? 2 : 1) * round256(n * d_v * eb);    // o, o_im
+    if (have_S0 || want_S_T) total += round256((size_t)B * H * d_k * d_v * 4);
+    total += round256(sfda_workspace_bytes(B, T, H, d_k, d_v, chunk, dtype));
+    return total;
+}
+
+int sfda_forward_host(const void *q, const void *k, const void *v, const float *alpha, const float *theta,
+                      const float *beta, const float *S0, void *o, void *o_im, float *S_T, int B, int T, int H,
+                      int d_k, int d_v, int chunk, int dtype, void *arena, size_t arena_bytes, void *stream,
+                      size_t *bytes_h2d, size_t *bytes_d2h)
+{
+    g_last_launches = 0;
+    if (!q || !k || !v || !alpha || !theta || !beta || !o) return SFDA_ERR_NULL;
+    if (B < 1 || T < 1 || H < 1) return SFDA_ERR_SHAPE;
+    const int rc = check_dims(d_k, d_v, chunk, dtype);
+    if (rc != SFDA_OK) return rc;
+    const size_t need = sfda_forward_host_arena_bytes(B, T, H, d_k, d_v, chunk, dtype, o_im != nullptr,
+                                                      S0 != nullptr, S_T != nullptr);
+    if (!arena || arena_bytes < need) return SFDA_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(arena) & 255u) return SFDA_ERR_ALIGN;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t n = (size_t)B * T * H, eb = elem_bytes(dtype), m = d_k / 2;
+    char *cur = static_cast<char *>(arena);
+    auto take = [&](size_t bytes) { char *p = cur; cur += round256(bytes); return p; };
+    size_t h2d = 0, d2h = 0;
+    bool ok = true;
+    auto up = [&](const void *src, size_t bytes) {
+        char *dst = take(bytes);
+        ok = ok && cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+        h2d += bytes;
+        return dst;
+    };
+    void *dq = up(q, n * d_k * eb);
+    void *dk = up(k, n * d_k * eb);
+    void *dv = up(v, n * d_v * eb);
+    float *da = reinterpret_cast<float *>(up(alpha, n * m * 4));
+    float *dt = reinterpret_cast<float *>(up(theta, n * m * 4));
+    float *db = reinterpret_cast<float *>(up(beta, n * 4));
+    void *dout = take(n * d_v * eb);
+    void *dout_im = o_im ? take(n * d_v * eb) : nullptr;
+    float *dS = nullptr;
+    const size_t state_bytes = (size_t)B * H * d_k * d_v * 4;
+    if (S0 || S_T) dS = reinterpret_cast<float *>(take(state_bytes));
+    if (S0) {
+        ok = ok && cudaMemcpyAsync(dS, S0, state_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+        h2d += state_bytes;
+    }
+    const size_t ws_bytes = sfda_workspace_bytes(B, T, H, d_k, d_v, chunk, dtype);
+    void *ws = ws_bytes ? take(ws_bytes) : nullptr;
+    if (!ok) return SFDA_ERR_CUDA;
+
+    const int frc = sfda_forward(dq, dk, dv, da, dt, db, S0 ? dS : nullptr, dout, dout_im, S_T ? dS : nullptr, B, T,
+                                 H, d_k, d_v, chunk, dtype, ws, ws_bytes, stream);
+    if (frc != SFDA_OK) return frc;
+
+    ok = ok && cudaMemcpyAsync(o, dout, n * d_v * eb, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    d2h += n * d_v * eb;
+    if (o_im) {
+        ok = ok && cudaMemcpyAsync(o_im, dout_im, n * d_v * eb, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+        d2h += n * d_v * eb;
+    }
+    if (S_T) {
+        ok = ok && cudaMemcpyAsync(S_T, dS, state_bytes, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+        d2h += state_bytes;
+    }
+    if (bytes_h2d) *bytes_h2d = h2d;
+    if (bytes_d2h) *bytes_d2h = d2h;
+    return ok ? SFDA_OK : SFDA_ERR_CUDA;
+}
+
+int sfda_last_launch_count(void) { return g_last_launches; }
+
+}  // extern "C"

@@ -1,0 +1,465 @@
+// fp32 CUDA-core chunk-WY forward and per-chunk factor export.
+//
+// What is computed per chunk (C tokens, one (batch, head) pair, gamma_t = prod_{s<=t} lambda_s inside
+// the chunk, written gamma_t = a_t e^{i phi_t}):
+//
+//   k'_t = e^{-i phi_t} k_t,  q'_t = e^{-i phi_t} q_t            (rotated keys / queries)
+//   Kt[t][i] = k_t^* diag(gamma_t/gamma_i) k_i = sum_j conj(k'_tj) k'_ij a_tj/a_ij      (i < t)
+//   Aq[t][i] = q_t^* diag(gamma_t/gamma_i) k_i = sum_j conj(q'_tj) k'_ij a_tj/a_ij      (i <= t)
+//   R = V - W^* S_0,  W_t = conj(gamma_t) k_t                      (W of Theorem "Constructive ... recursion")
+//   (I + D_beta Kt) E = D_beta R                                   (the unit lower triangular WY system;
+//        rows e_t^T = beta_t (v_t^T - k_t^* Lambda_t S_{t-1}); this is M of Eq. "constructive-M" applied)
+//   o_t^* = (conj(gamma_t) q_t)^* S_0 + sum_{i<=t} Aq[t][i] e_i^T   (Theorem "Prefix outputs inside a chunk")
+//   S_C = Gamma_C S_0 + sum_t (gamma_C/gamma_t) k_t e_t^T          (Eq. "apply-transfer" with B = Y M V)
+//
+// Only ratios a_t/a_i <= 1 are ever formed, so any alpha in [0, 1] is safe here.
+#include "sfda_common.cuh"
+#include "sfda_internal.h"
+
+namespace sfda {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kSlice = 32;  // value columns per CTA of the forward kernel
+
+// Index of the pair (t, i), i <= t, in row-major order of the lower triangle.
+__device__ __forceinline__ void tri_decode(int p, int *t, int *i)
+{
+    int r = (int)((sqrtf(8.f * (float)p + 1.f) - 1.f) * 0.5f);
+    while ((r + 1) * (r + 2) / 2 <= p) ++r;
+    while (r * (r + 1) / 2 > p) --r;
+    *t = r;
+    *i = p - r * (r + 1) / 2;
+}
+
+template <int DK, int C>
+struct ChunkSmem {
+    static constexpr int M = DK / 2;
+    static constexpr int KS = DK + 2;  // row stride of kp / qp (floats): spreads rows over banks
+    static constexpr int LS = M + 1;   // row stride of lg
+    static constexpr int GS = C + 1;   // row stride of the Gram matrices
+    float *kp, *qp, *lg, *gcr, *gci, *lgC, *beta;
+    __device__ explicit ChunkSmem(float *base)
+    {
+        kp = base;
+        qp = kp + C * KS;
+        lg = qp + C * KS;
+        gcr = lg + C * LS;
+        gci = gcr + M;
+        lgC = gci + M;
+        beta = lgC + M;
+    }
+    static constexpr int floats = 2 * C * KS + C * LS + 3 * M + C;
+};
+
+// Loads one chunk of k (and q when given), alpha, theta, beta; leaves in shared memory the rotated
+// keys / queries, the cumulative log-decay lg[t][j] = sum_{s<=t} log alpha_sj, the closing phase
+// e^{i phi_C} and lg_C.  Tokens past `len` are neutral (alpha = 1, theta = 0, beta = 0, k = q = 0).
+// When turns_out is not NULL the chunk-local cumulative phase turns of real tokens are written there.
+template <int DK, int C, typename T>
+__device__ void load_and_rotate(const ChunkSmem<DK, C> &sm, const T *__restrict__ k, const T *__restrict__ q,
+                                const float *__restrict__ alpha, const float *__restrict__ theta,
+                                const float *__restrict__ beta, uint32_t *__restrict__ turns_out, int b,
+                                int h, int T_, int H, int t0, int len)
+{
+    constexpr int M = DK / 2;
+    using S = ChunkSmem<DK, C>;
+    const int tid = threadIdx.x;
+    for (int idx = tid; idx < C * DK; idx += kThreads) {
+        const int t = idx / DK, x = idx % DK;
+        float kv = 0.f, qv = 0.f;
+        if (t < len) {
+            const size_t g = (((size_t)b * T_ + t0 + t) * H + h) * DK + x;
+            kv = ld_val(k, g);
+            if (q) qv = ld_val(q, g);
+        }
+        sm.kp[t * S::KS + x] = kv;
+        sm.qp[t * S::KS + x] = qv;
+    }
+    if (tid < C) sm.beta[tid] = tid < len ? beta[((size_t)b * T_ + t0 + tid) * H + h] : 0.f;
+    __syncthreads();
+    if (tid < M) {
+        const int j = tid;
+        float acc = 0.f, cs = 1.f, sn = 0.f;
+        uint32_t turns = 0u;
+#pragma unroll 4
+        for (int t = 0; t < C; ++t) {
+            if (t < len) {
+                const size_t g = (((size_t)b * T_ + t0 + t) * H + h) * M + j;
+                acc += log_decay(alpha[g]);
+                turns += phase_to_turns(theta[g]);
+                if (turns_out) turns_out[g] = turns;
+            }
+            sm.lg[t * S::LS + j] = acc;
+            turns_to_cos_sin(turns, &cs, &sn);
+            const float kr = sm.kp[t * S::KS + 2 * j], ki = sm.kp[t * S::KS + 2 * j + 1];
+            sm.kp[t * S::KS + 2 * j] = kr * cs + ki * sn;      // e^{-i phi} (kr + i ki)
+            sm.kp[t * S::KS + 2 * j + 1] = ki * cs - kr * sn;
+            const float qr = sm.qp[t * S::KS + 2 * j], qi = sm.qp[t * S::KS + 2 * j + 1];
+            sm.qp[t * S::KS + 2 * j] = qr * cs + qi * sn;
+            sm.qp[t * S::KS + 2 * j + 1] = qi * cs - qr * sn;
+        }
+        sm.gcr[j] = cs;
+        sm.gci[j] = sn;
+        sm.lgC[j] = acc;
+    }
+    __syncthreads();
+}
+
+// ------------------------------------------------------------------------------------------------
+// forward
+// ------------------------------------------------------------------------------------------------
+template <int DK, int C>
+constexpr int forward_smem_floats()
+{
+    return ChunkSmem<DK, C>::floats + 2 * (DK / 2) * kSlice  // state (re, im)
+           + 4 * C * (C + 1)                                  // Kt, Aq (re, im)
+           + 2 * C * kSlice;                                  // E (re, im)
+}
+
+template <int DK, int C, typename T>
+__global__ void __launch_bounds__(kThreads)
+sfda_forward_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v,
+                         const float *__restrict__ alpha, const float *__restrict__ theta,
+                         const float *__restrict__ beta, const float *__restrict__ S0, T *__restrict__ o,
+                         T *__restrict__ o_im, float *__restrict__ S_T, int T_, int H, int dv)
+{
+    constexpr int M = DK / 2;
+    using SM = ChunkSmem<DK, C>;
+    extern __shared__ __align__(16) float smem[];
+    const SM sm(smem);
+    float *Sre = smem + SM::floats;
+    float *Sim = Sre + M * kSlice;
+    float *Ktr = Sim + M * kSlice;
+    float *Kti = Ktr + C * SM::GS;
+    float *Aqr = Kti + C * SM::GS;
+    float *Aqi = Aqr + C * SM::GS;
+    float *Er = Aqi + C * SM::GS;
+    float *Ei = Er + C * kSlice;
+
+    const int tid = threadIdx.x, lane = tid % 32, wid = tid / 32;
+    const int nsl = dv / kSlice;
+    const int slice = blockIdx.x % nsl;
+    const int bh = blockIdx.x / nsl;
+    const int h = bh % H, b = bh / H;
+    const int c0 = slice * kSlice;
+
+    for (int idx = tid; idx < M * kSlice; idx += kThreads) {
+        const int j = idx / kSlice, c = idx % kSlice;
+        Sre[idx] = S0 ? S0[((size_t)bh * DK + 2 * j) * dv + c0 + c] : 0.f;
+        Sim[idx] = S0 ? S0[((size_t)bh * DK + 2 * j + 1) * dv + c0 + c] : 0.f;
+    }
+
+    const int n_chunks = (T_ + C - 1) / C;
+    for (int ci = 0; ci < n_chunks; ++ci) {
+        const int t0 = ci * C;
+        const int len = min(C, T_ - t0);
+        __syncthreads();
+        load_and_rotate<DK, C, T>(sm, k, q, alpha, theta, beta, nullptr, b, h, T_, H, t0, len);
+
+        // Gram blocks Kt (i < t) and Aq (i <= t).
+        for (int p = tid; p < C * (C + 1) / 2; p += kThreads) {
+            int t, i;
+            tri_decode(p, &t, &i);
+            float kr_ = 0.f, ki_ = 0.f, ar_ = 0.f, ai_ = 0.f;
+            const float *kt = sm.kp + t * SM::KS, *ki = sm.kp + i * SM::KS, *qt = sm.qp + t * SM::KS;
+            const float *lt = sm.lg + t * SM::LS, *li = sm.lg + i * SM::LS;
+            for (int j = 0; j < M; ++j) {
+                const float w = expf(lt[j] - li[j]);
+                const float br = w * ki[2 * j], bi = w * ki[2 * j + 1];
+                const float xr = kt[2 * j], xi = kt[2 * j + 1];
+                kr_ += xr * br + xi * bi;   // conj(x) * b
+                ki_ += xr * bi - xi * br;
+                const float yr = qt[2 * j], yi = qt[2 * j + 1];
+                ar_ += yr * br + yi * bi;
+                ai_ += yr * bi - yi * br;
+            }
+            Ktr[t * SM::GS + i] = kr_;
+            Kti[t * SM::GS + i] = ki_;
+            Aqr[t * SM::GS + i] = ar_;
+            Aqi[t * SM::GS + i] = ai_;
+        }
+
+        // R = V - W^* S_0 (kept in E).
+        for (int t = wid; t < C; t += kThreads / 32) {
+            float rr = 0.f, ri = 0.f;
+            if (t < len) rr = ld_val(v, (((size_t)b * T_ + t0 + t) * H + h) * dv + c0 + lane);
+            const float *kt = sm.kp + t * SM::KS, *lt = sm.lg + t * SM::LS;
+            for (int j = 0; j < M; ++j) {
+                const float w = expf(lt[j]);
+                const float wr = w * kt[2 * j], wi = w * kt[2 * j + 1];
+                const float sr = Sre[j * kSlice + lane], si = Sim[j * kSlice + lane];
+                rr -= wr * sr + wi * si;   // conj(w) * s
+                ri -= wr * si - wi * sr;
+            }
+            Er[t * kSlice + lane] = rr;
+            Ei[t * kSlice + lane] = ri;
+        }
+        __syncthreads();
+
+        // Forward substitution of (I + D_beta Kt) E = D_beta R.  A warp owns four columns; the sum
+        // over earlier tokens is split over eight lanes and folded with shuffles.
+        {
+            const int cc = 4 * wid + lane / 8, part = lane % 8;
+            for (int t = 0; t < C; ++t) {
+                float sr = 0.f, si = 0.f;
+                for (int i = part; i < t; i += 8) {
+                    const float xr = Ktr[t * SM::GS + i], xi = Kti[t * SM::GS + i];
+                    const float er = Er[i * kSlice + cc], ei = Ei[i * kSlice + cc];
+                    sr += xr * er - xi * ei;
+                    si += xr * ei + xi * er;
+                }
+#pragma unroll
+                for (int off = 1; off < 8; off <<= 1) {
+                    sr += __shfl_xor_sync(0xffffffffu, sr, off);
+                    si += __shfl_xor_sync(0xffffffffu, si, off);
+                }
+                const float bt = sm.beta[t];
+                const float er = bt * (Er[t * kSlice + cc] - sr);
+                const float ei = bt * (Ei[t * kSlice + cc] - si);
+                __syncwarp();
+                if (part == 0) {
+                    Er[t * kSlice + cc] = er;
+                    Ei[t * kSlice + cc] = ei;
+                }
+                __syncwarp();
+            }
+        }
+        __syncthreads();
+
+        // Outputs: o_t^* = (conj(gamma_t) q_t)^* S_0 + sum_{i<=t} Aq[t][i] e_i^T ; o = conj of that row.
+        for (int t = wid; t < len; t += kThreads / 32) {
+            float rr = 0.f, ri = 0.f;
+            const float *qt = sm.qp + t * SM::KS, *lt = sm.lg + t * SM::LS;
+            for (int j = 0; j < M; ++j) {
+                const float w = expf(lt[j]);
+                const float wr = w * qt[2 * j], wi = w * qt[2 * j + 1];
+                const float sr = Sre[j * kSlice + lane], si = Sim[j * kSlice + lane];
+                rr += wr * sr + wi * si;
+                ri += wr * si - wi * sr;
+            }
+            for (int i = 0; i <= t; ++i) {
+                const float xr = Aqr[t * SM::GS + i], xi = Aqi[t * SM::GS + i];
+                const float er = Er[i * kSlice + lane], ei = Ei[i * kSlice + lane];
+                rr += xr * er - xi * ei;
+                ri += xr * ei + xi * er;
+            }
+            const size_t g = (((size_t)b * T_ + t0 + t) * H + h) * dv + c0 + lane;
+            st_val(o, g, rr);
+            if (o_im) st_val(o_im, g, -ri);
+        }
+        __syncthreads();
+
+        // S_C = Gamma_C S_0 + sum_t (gamma_C / gamma_t) k_t e_t^T.
+        for (int j = wid; j < M; j += kThreads / 32) {
+            const float aC = expf(sm.lgC[j]);
+            float nr = aC * Sre[j * kSlice + lane], ni = aC * Sim[j * kSlice + lane];
+            for (int t = 0; t < C; ++t) {
+                const float w = expf(sm.lgC[j] - sm.lg[t * SM::LS + j]);
+                const float yr = w * sm.kp[t * SM::KS + 2 * j], yi = w * sm.kp[t * SM::KS + 2 * j + 1];
+                const float er = Er[t * kSlice + lane], ei = Ei[t * kSlice + lane];
+                nr += yr * er - yi * ei;
+                ni += yr * ei + yi * er;
+            }
+            const float gr = sm.gcr[j], gi = sm.gci[j];   // e^{i phi_C}
+            Sre[j * kSlice + lane] = gr * nr - gi * ni;
+            Sim[j * kSlice + lane] = gr * ni + gi * nr;
+        }
+    }
+    __syncthreads();
+    if (S_T) {
+        for (int idx = tid; idx < M * kSlice; idx += kThreads) {
+            const int j = idx / kSlice, c = idx % kSlice;
+            S_T[((size_t)bh * DK + 2 * j) * dv + c0 + c] = Sre[idx];
+            S_T[((size_t)bh * DK + 2 * j + 1) * dv + c0 + c] = Sim[idx];
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// factor export
+// ------------------------------------------------------------------------------------------------
+template <int DK, int C>
+constexpr int factor_smem_floats()
+{
+    return ChunkSmem<DK, C>::floats + 4 * C * (C + 1);  // N (re, im), X = (I + N)^{-1} (re, im)
+}
+
+template <int DK, int C, typename T>
+__global__ void __launch_bounds__(kThreads)
+sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alpha,
+                          const float *__restrict__ theta, const float *__restrict__ beta,
+                          float *__restrict__ Gamma, float *__restrict__ Y, float *__restrict__ Mo,
+                          float *__restrict__ W, uint32_t *__restrict__ turns_out, int T_, int H, int NC)
+{
+    constexpr int M = DK / 2;
+    using SM = ChunkSmem<DK, C>;
+    extern __shared__ __align__(16) float smem[];
+    const SM sm(smem);
+    float *Nr = smem + SM::floats;
+    float *Ni = Nr + C * SM::GS;
+    float *Xr = Ni + C * SM::GS;
+    float *Xi = Xr + C * SM::GS;
+
+    const int tid = threadIdx.x;
+    const int ci = blockIdx.x % NC;
+    const int bh = blockIdx.x / NC;
+    const int h = bh % H, b = bh / H;
+    const int t0 = ci * C;
+    const int len = min(C, T_ - t0);
+    const size_t chunk_id = (size_t)bh * NC + ci;
+
+    load_and_rotate<DK, C, T>(sm, k, static_cast<const T *>(nullptr), alpha, theta, beta, turns_out, b, h, T_,
+                              H, t0, len);
+
+    // N[t][i] = beta_i * k_t^* diag(gamma_t / gamma_i) k_i, i < t  (the block-inverse of Eq. "constructive-M").
+    for (int p = tid; p < C * (C + 1) / 2; p += kThreads) {
+        int t, i;
+        tri_decode(p, &t, &i);
+        float ar = 0.f, ai = 0.f;
+        if (i < t) {
+            const float *kt = sm.kp + t * SM::KS, *ki = sm.kp + i * SM::KS;
+            const float *lt = sm.lg + t * SM::LS, *li = sm.lg + i * SM::LS;
+            for (int j = 0; j < M; ++j) {
+                const float w = expf(lt[j] - li[j]);
+                const float br = w * ki[2 * j], bi = w * ki[2 * j + 1];
+                ar += kt[2 * j] * br + kt[2 * j + 1] * bi;
+                ai += kt[2 * j] * bi - kt[2 * j + 1] * br;
+            }
+            ar *= sm.beta[i];
+            ai *= sm.beta[i];
+        }
+        Nr[t * SM::GS + i] = ar;
+        Ni[t * SM::GS + i] = ai;
+    }
+    __syncthreads();
+
+    // M = (I + N)^{-1}: thread c solves column c by forward substitution (it only reads its own column).
+    if (tid < C) {
+        const int c = tid;
+        for (int t = 0; t < C; ++t) {
+            float xr = t == c ? 1.f : 0.f, xi = 0.f;
+            if (t > c) {
+                for (int i = c; i < t; ++i) {
+                    const float nr = Nr[t * SM::GS + i], ni = Ni[t * SM::GS + i];
+                    const float yr = Xr[i * SM::GS + c], yi = Xi[i * SM::GS + c];
+                    xr -= nr * yr - ni * yi;
+                    xi -= nr * yi + ni * yr;
+                }
+            }
+            Xr[t * SM::GS + c] = xr;
+            Xi[t * SM::GS + c] = xi;
+        }
+    }
+    __syncthreads();
+
+    if (Gamma) {
+        for (int j = tid; j < M; j += kThreads) {
+            const float a = expf(sm.lgC[j]);
+            Gamma[(chunk_id * M + j) * 2] = a * sm.gcr[j];
+            Gamma[(chunk_id * M + j) * 2 + 1] = a * sm.gci[j];
+        }
+    }
+    for (int idx = tid; idx < M * C; idx += kThreads) {
+        const int j = idx / C, t = idx % C;
+        const float kr = sm.kp[t * SM::KS + 2 * j], ki = sm.kp[t * SM::KS + 2 * j + 1];
+        if (W) {   // W[:,t] = conj(gamma_t) k_t = a_t k'_t
+            const float a = expf(sm.lg[t * SM::LS + j]);
+            reinterpret_cast<float2 *>(W)[(chunk_id * M + j) * C + t] = make_float2(a * kr, a * ki);
+        }
+        if (Y) {   // Y[:,t] = (gamma_C / gamma_t) beta_t k_t = (a_C / a_t) e^{i phi_C} beta_t k'_t
+            const float w = sm.beta[t] * expf(sm.lgC[j] - sm.lg[t * SM::LS + j]);
+            const float gr = sm.gcr[j], gi = sm.gci[j];
+            reinterpret_cast<float2 *>(Y)[(chunk_id * M + j) * C + t] =
+                make_float2(w * (gr * kr - gi * ki), w * (gr * ki + gi * kr));
+        }
+    }
+    if (Mo) {
+        for (int idx = tid; idx < C * C; idx += kThreads) {
+            const int t = idx / C, i = idx % C;
+            reinterpret_cast<float2 *>(Mo)[chunk_id * C * C + idx] =
+                i <= t ? make_float2(Xr[t * SM::GS + i], Xi[t * SM::GS + i]) : make_float2(0.f, 0.f);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// launchers
+// ------------------------------------------------------------------------------------------------
+template <int DK, int C, typename T>
+cudaError_t launch_fwd(const ForwardArgs &a, cudaStream_t stream)
+{
+    constexpr size_t smem = sizeof(float) * forward_smem_floats<DK, C>();
+    auto kern = sfda_forward_simt_kernel<DK, C, T>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const unsigned grid = (unsigned)a.B * a.H * (a.d_v / kSlice);
+    kern<<<grid, kThreads, smem, stream>>>(static_cast<const T *>(a.q), static_cast<const T *>(a.k),
+                                           static_cast<const T *>(a.v), a.alpha, a.theta, a.beta, a.S0,
+                                           static_cast<T *>(a.o), static_cast<T *>(a.o_im), a.S_T, a.T, a.H,
+                                           a.d_v);
+    return cudaGetLastError();
+}
+
+template <int DK, int C, typename T>
+cudaError_t launch_fac(const FactorArgs &a, cudaStream_t stream)
+{
+    constexpr size_t smem = sizeof(float) * factor_smem_floats<DK, C>();
+    auto kern = sfda_chunk_factors_kernel<DK, C, T>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const int NC = (a.T + C - 1) / C;
+    const unsigned grid = (unsigned)a.B * a.H * NC;
+    kern<<<grid, kThreads, smem, stream>>>(static_cast<const T *>(a.k), a.alpha, a.theta, a.beta, a.Gamma, a.Y,
+                                           a.M, a.W, a.phase_turns, a.T, a.H, NC);
+    return cudaGetLastError();
+}
+
+template <typename Args, typename T, typename F64_16, typename F64_32, typename F64_64, typename F128_16,
+          typename F128_32, typename F128_64>
+cudaError_t by_shape(const Args &a, F64_16 f1, F64_32 f2, F64_64 f3, F128_16 f4, F128_32 f5, F128_64 f6)
+{
+    if (a.d_k == 64 && a.chunk == 16) return f1();
+    if (a.d_k == 64 && a.chunk == 32) return f2();
+    if (a.d_k == 64 && a.chunk == 64) return f3();
+    if (a.d_k == 128 && a.chunk == 16) return f4();
+    if (a.d_k == 128 && a.chunk == 32) return f5();
+    if (a.d_k == 128 && a.chunk == 64) return f6();
+    return cudaErrorInvalidValue;
+}
+
+template <typename T>
+cudaError_t dispatch_fwd(const ForwardArgs &a, cudaStream_t s)
+{
+    return by_shape<ForwardArgs, T>(
+        a, [&] { return launch_fwd<64, 16, T>(a, s); }, [&] { return launch_fwd<64, 32, T>(a, s); },
+        [&] { return launch_fwd<64, 64, T>(a, s); }, [&] { return launch_fwd<128, 16, T>(a, s); },
+        [&] { return launch_fwd<128, 32, T>(a, s); }, [&] { return launch_fwd<128, 64, T>(a, s); });
+}
+
+template <typename T>
+cudaError_t dispatch_fac(const FactorArgs &a, cudaStream_t s)
+{
+    return by_shape<FactorArgs, T>(
+        a, [&] { return launch_fac<64, 16, T>(a, s); }, [&] { return launch_fac<64, 32, T>(a, s); },
+        [&] { return launch_fac<64, 64, T>(a, s); }, [&] { return launch_fac<128, 16, T>(a, s); },
+        [&] { return launch_fac<128, 32, T>(a, s); }, [&] { return launch_fac<128, 64, T>(a, s); });
+}
+
+}  // namespace
+
+cudaError_t launch_forward_simt(const ForwardArgs &a, cudaStream_t stream, int *launches)
+{
+    const cudaError_t e = a.dtype == 1 ? dispatch_fwd<__nv_bfloat16>(a, stream) : dispatch_fwd<float>(a, stream);
+    if (e == cudaSuccess && launches) ++*launches;
+    return e;
+}
+
+cudaError_t launch_chunk_factors(const FactorArgs &a, cudaStream_t stream, int *launches)
+{
+    const cudaError_t e = a.dtype == 1 ? dispatch_fac<__nv_bfloat16>(a, stream) : dispatch_fac<float>(a, stream);
+    if (e == cudaSuccess && launches) ++*launches;
+    return e;
+}
+
+}  // namespace sfda

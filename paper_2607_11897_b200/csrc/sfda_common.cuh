@@ -1,0 +1,38 @@
+// Shared device helpers of the SFDA kernels (sm_100a).  Nothing here is used by,
+// or shared with, the CPU oracle.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace sfda {
+
+// ---- element IO in the caller's dtype --------------------------------------------------------
+__device__ __forceinline__ float ld_val(const float *p, size_t i) { return p[i]; }
+__device__ __forceinline__ float ld_val(const __nv_bfloat16 *p, size_t i) { return __bfloat162float(p[i]); }
+__device__ __forceinline__ void st_val(float *p, size_t i, float x) { p[i] = x; }
+__device__ __forceinline__ void st_val(__nv_bfloat16 *p, size_t i, float x) { p[i] = __float2bfloat16_rn(x); }
+
+// ---- integer cumulative phase ------------------------------------------------------------------
+// A phase is carried as an unsigned 32-bit count of 2*pi/2^32 turns so that the chunk-local prefix
+// product Gamma_t = Lambda_t Gamma_{t-1} (Eq. "constructive-Gamma") has, for its unit-modulus part,
+// one right answer whatever order a scan adds it in.  theta -> rint((double)theta * 2^32/(2 pi)).
+__device__ __forceinline__ uint32_t phase_to_turns(float theta)
+{
+    const double turns_per_radian = 0x1.45f306dc9c883p+29;  // 2^32 / (2 pi), nearest double
+    const long long r = __double2ll_rn(__dmul_rn((double)theta, turns_per_radian));
+    return (uint32_t)(unsigned long long)r;
+}
+
+// cos / sin of a phase given in turns (signed view keeps the float argument in [-1, 1)).
+__device__ __forceinline__ void turns_to_cos_sin(uint32_t turns, float *c, float *s)
+{
+    const float x = (float)(int32_t)turns * 0x1p-31f;  // phase / pi
+    sincospif(x, s, c);
+}
+
+// log of a decay factor, floored so that sums of 64 of them stay finite and differences of two
+// such sums never give inf - inf (alpha = 0 is admissible in the recurrence).
+__device__ __forceinline__ float log_decay(float alpha) { return fmaxf(logf(alpha), -1.0e4f); }
+
+}  // namespace sfda

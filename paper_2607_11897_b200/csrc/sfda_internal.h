@@ -1,0 +1,38 @@
+// Host-side launcher prototypes shared by the translation units of the library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace sfda {
+
+struct ForwardArgs {
+    const void *q, *k, *v;
+    const float *alpha, *theta, *beta, *S0;
+    void *o, *o_im;
+    float *S_T;
+    int B, T, H, d_k, d_v, chunk, dtype;
+};
+
+struct FactorArgs {
+    const void *k;
+    const float *alpha, *theta, *beta;
+    float *Gamma, *Y, *M, *W;
+    uint32_t *phase_turns;
+    int B, T, H, d_k, chunk, dtype;
+};
+
+struct StepArgs {
+    const void *q, *k, *v;
+    const float *alpha, *theta, *beta;
+    float *S;
+    void *o, *o_im;
+    int B, H, d_k, d_v, dtype;
+};
+
+// Each returns a cudaError_t from configuring / launching; *launches is incremented per kernel.
+cudaError_t launch_forward_simt(const ForwardArgs &a, cudaStream_t stream, int *launches);
+cudaError_t launch_chunk_factors(const FactorArgs &a, cudaStream_t stream, int *launches);
+cudaError_t launch_step(const StepArgs &a, cudaStream_t stream, int *launches);
+
+}  // namespace sfda

@@ -1,0 +1,341 @@
+"""GPU parity: every entry point of the C-ABI library against the CPU oracle,
+element by element, on the same seeded inputs.
+
+Error measure (the paper defines none): err = max|x - y| / max|y| per output
+tensor, with y the oracle.  Bars: 1e-4 for fp32 inputs, 2e-2 for bf16 inputs with
+fp32 accumulation; integer bookkeeping (chunk plan, cumulative phase turns) must be
+bit-exact.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2607_11897_b200 as sfda
+import workloads
+from oracle import bookkeeping, chunk_wy, recurrence
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-4, "bf16": 2e-2}
+DEV = "cuda:0"
+
+
+def rel_err(got, want):
+    got = np.asarray(got, dtype=np.float64)
+    want = np.asarray(want, dtype=np.float64)
+    assert np.isfinite(got).all(), "non-finite GPU output"
+    return float(np.abs(got - want).max() / max(np.abs(want).max(), 1e-30))
+
+
+def to_dev(x, cfg, key):
+    t = torch.from_numpy(np.ascontiguousarray(x)).to(DEV)
+    if key in ("q", "k", "v") and cfg.dtype == "bf16":
+        t = t.to(torch.bfloat16)          # exact: the values already lie on the bf16 grid
+    return t
+
+
+def run_forward(cfg, inp, want_im=True, simt=False, want_state=True):
+    d = {k: (None if v is None else to_dev(v, cfg, k)) for k, v in inp.items()}
+    B, T, H = d["q"].shape[:3]
+    o = torch.empty(B, T, H, cfg.d_v, device=DEV, dtype=d["q"].dtype)
+    o_im = torch.empty_like(o) if want_im else None
+    S_T = torch.empty(B, H, cfg.d_k, cfg.d_v, device=DEV, dtype=torch.float32) if want_state else None
+    ws_bytes = sfda.sfda_workspace_bytes(B, T, H, cfg.d_k, cfg.d_v, cfg.chunk, 1 if cfg.dtype == "bf16" else 0)
+    ws = torch.empty(max(ws_bytes, 16), device=DEV, dtype=torch.uint8)
+    if simt:
+        sfda.sfda_forward_simt(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im, S_T,
+                               cfg.chunk)
+    else:
+        sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im, S_T,
+                          cfg.chunk, ws)
+    torch.cuda.synchronize()
+    assert sfda.last_launch_count() >= 1
+    return (o.float().cpu().numpy(), None if o_im is None else o_im.float().cpu().numpy(),
+            None if S_T is None else S_T.cpu().numpy())
+
+
+def oracle_pairs(inp, pairs):
+    s = workloads.sequences(inp, pairs)
+    return recurrence.sfda_recurrence(s["q"], s["k"], s["v"], s["alpha"], s["theta"], s["beta"], s["S0"])
+
+
+def check_forward(cfg, inp, pairs, tol, **kw):
+    o, o_im, S_T = run_forward(cfg, inp, **kw)
+    w_re, w_im, w_S = oracle_pairs(inp, pairs)
+    g_re = np.stack([o[b, :, h] for b, h in pairs])
+    errs = {"o_re": rel_err(g_re, w_re)}
+    if o_im is not None:
+        errs["o_im"] = rel_err(np.stack([o_im[b, :, h] for b, h in pairs]), w_im)
+    if S_T is not None:
+        errs["S_T"] = rel_err(np.stack([S_T[b, h] for b, h in pairs]), w_S)
+    for name, e in errs.items():
+        assert e <= tol, "%s: %s rel err %.3e > %.1e (%s)" % (cfg.name, name, e, tol, errs)
+    return errs
+
+
+def all_pairs(cfg):
+    return [(b, h) for b in range(cfg.B) for h in range(cfg.H)]
+
+
+# ------------------------------------------------------------------------------------------------
+# forward
+# ------------------------------------------------------------------------------------------------
+def test_forward_cfg0_tiny_fp32():
+    cfg = workloads.CONFIGS[0]
+    inp = workloads.forward_inputs(cfg)
+    check_forward(cfg, inp, all_pairs(cfg), TOL["f32"])
+
+
+@pytest.mark.parametrize("d_k,d_v,chunk,T", [(64, 64, 16, 100), (64, 128, 32, 77), (128, 64, 64, 130),
+                                             (128, 128, 64, 200), (128, 128, 32, 64), (128, 128, 16, 33),
+                                             (64, 64, 64, 1), (128, 128, 64, 5)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_forward_simt_shapes_ragged_tail_and_state(d_k, d_v, chunk, T, dtype):
+    cfg = workloads.CONFIGS[0].scaled(name="t", B=2, T=T, H=3, d_k=d_k, d_v=d_v, chunk=chunk, dtype=dtype,
+                                      s0_std=0.5, seed=100 + d_k + d_v + chunk + T)
+    inp = workloads.forward_inputs(cfg)
+    # the fp32 path with bf16 storage only rounds the stored outputs: 2^-9 relative
+    check_forward(cfg, inp, all_pairs(cfg), 1e-4 if dtype == "f32" else 5e-3, simt=True)
+
+
+@pytest.mark.parametrize("alpha,beta", [("u(0.3,1)", "u(0,1)"), ("u(0.0,1)", "u(0,1)"),
+                                        ("u(0.9,1)", "bernoulli(0.05)"), ("u(1.0,1.0)", "u(0,1)")])
+def test_forward_simt_decay_and_write_edges(alpha, beta):
+    cfg = workloads.CONFIGS[0].scaled(name="edge", B=1, T=192, H=2, d_k=128, d_v=64, chunk=64, alpha=alpha,
+                                      beta=beta, s0_std=1.0, seed=7)
+    inp = workloads.forward_inputs(cfg)
+    if alpha == "u(0.0,1)":
+        inp["alpha"][:, ::17, :, ::5] = 0.0            # exact zeros are admissible (alpha in [0, 1])
+    check_forward(cfg, inp, all_pairs(cfg), 1e-4, simt=True)
+
+
+def test_forward_beta_all_zero_and_all_one():
+    for val in (0.0, 1.0):
+        cfg = workloads.CONFIGS[0].scaled(name="b", B=1, T=96, H=2, chunk=32, s0_std=1.0, seed=9)
+        inp = workloads.forward_inputs(cfg)
+        inp["beta"][:] = val
+        check_forward(cfg, inp, all_pairs(cfg), 1e-4, simt=True)
+
+
+def test_forward_outputs_optional():
+    cfg = workloads.CONFIGS[0].scaled(name="opt", T=64, seed=3)
+    inp = workloads.forward_inputs(cfg)
+    check_forward(cfg, inp, all_pairs(cfg), 1e-4, want_im=False, want_state=False)
+
+
+def test_forward_split_sequence_continues_from_state():
+    """forward(T1) then forward(T2, S0 = S_T1) equals forward(T1 + T2) (Theorem "Chunk-bounded exactness")."""
+    cfg = workloads.CONFIGS[0].scaled(name="split", T=160, seed=4)
+    inp = workloads.forward_inputs(cfg)
+    o, o_im, S_T = run_forward(cfg, inp)
+    T1 = 64
+    first = {k: (None if v is None else v[:, :T1]) for k, v in inp.items()}
+    o1, _, S1 = run_forward(cfg, first)
+    second = {k: (None if v is None else v[:, T1:]) for k, v in inp.items()}
+    second["S0"] = S1
+    o2, _, S2 = run_forward(cfg, second)
+    assert rel_err(np.concatenate([o1, o2], 1), o) < 1e-5
+    assert rel_err(S2, S_T) < 1e-5
+
+
+@pytest.mark.parametrize("idx", [1, 2])
+def test_forward_full_size_bf16_configs_sampled(idx):
+    """Configurations 1 and 2 at full size, in the launch configuration bench.py times;
+    the oracle recomputes a sample of (batch, head) sequences end to end."""
+    cfg = workloads.CONFIGS[idx]
+    inp = workloads.forward_inputs(cfg)
+    pairs = [(0, 0), (cfg.B - 1, cfg.H - 1), (cfg.B // 2, 5), (1, cfg.H // 2)]
+    check_forward(cfg, inp, pairs, TOL["bf16"])
+
+
+def test_forward_long_context_stability():
+    """Configuration 3 (T = 131072): parity on sampled heads, finite outputs, the Frobenius
+    bound of Prop. "Basic numerical stability", bit-exact cumulative phase turns."""
+    cfg = workloads.CONFIGS[3]
+    inp = workloads.forward_inputs(cfg)
+    pairs = [(0, 0), (0, 9)]
+    o, o_im, S_T = run_forward(cfg, inp)
+    assert np.isfinite(o).all() and np.isfinite(o_im).all() and np.isfinite(S_T).all()
+    w_re, w_im, w_S = oracle_pairs(inp, pairs)
+    assert rel_err(np.stack([o[b, :, h] for b, h in pairs]), w_re) <= TOL["bf16"]
+    assert rel_err(np.stack([o_im[b, :, h] for b, h in pairs]), w_im) <= TOL["bf16"]
+    assert rel_err(np.stack([S_T[b, h] for b, h in pairs]), w_S) <= TOL["bf16"]
+    # ||S_T||_F <= ||S_0||_F + sum beta |k| |v|
+    for h in range(cfg.H):
+        bound = np.sum(inp["beta"][0, :, h].astype(np.float64)
+                       * np.linalg.norm(inp["k"][0, :, h].astype(np.float64), axis=-1)
+                       * np.linalg.norm(inp["v"][0, :, h].astype(np.float64), axis=-1))
+        assert np.linalg.norm(S_T[0, h].astype(np.float64)) <= bound * (1 + 1e-2) + 1e-6
+    k = to_dev(inp["k"], cfg, "k")
+    turns = torch.empty(cfg.B, cfg.T, cfg.H, cfg.m, device=DEV, dtype=torch.int32)
+    sfda.sfda_chunk_factors(k, to_dev(inp["alpha"], cfg, "alpha"), to_dev(inp["theta"], cfg, "theta"),
+                            to_dev(inp["beta"], cfg, "beta"), None, None, None, None, turns, cfg.chunk)
+    torch.cuda.synchronize()
+    got = turns.cpu().numpy().view(np.uint32)
+    want = np.moveaxis(bookkeeping.cumulative_phase_turns(np.moveaxis(inp["theta"], 1, 2), cfg.chunk), 2, 1)
+    assert np.array_equal(got, want)
+
+
+# ------------------------------------------------------------------------------------------------
+# factor export
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("d_k,chunk,T,dtype", [(64, 16, 50, "f32"), (128, 64, 150, "f32"), (128, 32, 64, "bf16"),
+                                               (64, 64, 64, "f32")])
+def test_chunk_factors_match_constructive_recursion(d_k, chunk, T, dtype):
+    cfg = workloads.CONFIGS[0].scaled(name="fac", B=2, T=T, H=2, d_k=d_k, chunk=chunk, dtype=dtype, seed=5 + T)
+    inp = workloads.forward_inputs(cfg)
+    B, H, m, C = cfg.B, cfg.H, cfg.m, chunk
+    NC, tail = sfda.sfda_plan(T, chunk)
+    assert (NC, tail) == bookkeeping.chunk_plan(T, chunk)
+    G = torch.full((B, H, NC, m, 2), float("nan"), device=DEV)
+    Y = torch.full((B, H, NC, m, C, 2), float("nan"), device=DEV)
+    M = torch.full((B, H, NC, C, C, 2), float("nan"), device=DEV)
+    W = torch.full((B, H, NC, m, C, 2), float("nan"), device=DEV)
+    turns = torch.zeros(B, T, H, m, device=DEV, dtype=torch.int32)
+    sfda.sfda_chunk_factors(to_dev(inp["k"], cfg, "k"), to_dev(inp["alpha"], cfg, "alpha"),
+                            to_dev(inp["theta"], cfg, "theta"), to_dev(inp["beta"], cfg, "beta"), G, Y, M, W, turns,
+                            chunk)
+    torch.cuda.synchronize()
+    cx = lambda t: t.cpu().numpy().astype(np.float64)[..., 0] + 1j * t.cpu().numpy().astype(np.float64)[..., 1]
+    G, Y, M, W = cx(G), cx(Y), cx(M), cx(W)
+    got_turns = turns.cpu().numpy().view(np.uint32)
+    want_turns = np.moveaxis(bookkeeping.cumulative_phase_turns(np.moveaxis(inp["theta"], 1, 2), chunk), 2, 1)
+    assert np.array_equal(got_turns, want_turns)
+    worst = 0.0
+    for b in range(B):
+        for h in range(H):
+            kc = chunk_wy.pair(inp["k"][b, :, h])
+            for c in range(NC):
+                sl = slice(c * C, min((c + 1) * C, T))
+                L = sl.stop - sl.start
+                g, y, w, mm = chunk_wy.chunk_factors(kc[sl], inp["alpha"][b, sl, h].astype(np.float64),
+                                                     inp["theta"][b, sl, h].astype(np.float64),
+                                                     inp["beta"][b, sl, h].astype(np.float64))
+                worst = max(worst, rel_err(G[b, h, c].view(np.float64), g.view(np.float64)),
+                            rel_err(Y[b, h, c][:, :L].copy().view(np.float64), y.copy().view(np.float64)),
+                            rel_err(W[b, h, c][:, :L].copy().view(np.float64), w.copy().view(np.float64)),
+                            rel_err(M[b, h, c][:L, :L].copy().view(np.float64), mm.copy().view(np.float64)))
+                # padded tail tokens are neutral: zero columns, identity rows
+                assert np.all(Y[b, h, c][:, L:] == 0) and np.all(W[b, h, c][:, L:] == 0)
+                assert np.array_equal(M[b, h, c][L:, :], np.eye(C)[L:, :])
+                # the product the factors stand for, P = Gamma - Y M W^*, against the oracle's
+                P_gpu = np.diag(G[b, h, c]) - Y[b, h, c] @ M[b, h, c] @ W[b, h, c].conj().T
+                P_ref = np.diag(g) - y @ mm @ w.conj().T
+                assert np.abs(P_gpu - P_ref).max() < 2e-5
+    assert worst < 1e-4, worst
+
+
+# ------------------------------------------------------------------------------------------------
+# decode
+# ------------------------------------------------------------------------------------------------
+def run_decode(cfg, steps, pairs):
+    """Run `steps` decode steps on the GPU; keep inputs and outputs of the sampled (b, h) pairs only."""
+    from concurrent.futures import ThreadPoolExecutor
+    S0 = workloads.decode_initial_state(cfg)
+    S = torch.from_numpy(S0).to(DEV)
+    dt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    o = torch.empty(cfg.B, cfg.H, cfg.d_v, device=DEV, dtype=dt)
+    o_im = torch.empty_like(o)
+    bi = torch.tensor([p[0] for p in pairs], device=DEV)
+    hi = torch.tensor([p[1] for p in pairs], device=DEV)
+    out = torch.empty(steps, len(pairs), cfg.d_v, device=DEV)
+    out_im = torch.empty_like(out)
+    keys = ("q", "k", "v", "alpha", "theta", "beta")
+    sampled = {k: [] for k in keys}
+    window = 32
+    with ThreadPoolExecutor(max_workers=8) as pool:
+        for s0 in range(0, steps, window):
+            batch = list(pool.map(lambda s: workloads.decode_step_inputs(cfg, s), range(s0, min(s0 + window, steps))))
+            for i, x in enumerate(batch):
+                for k in keys:
+                    sampled[k].append(np.stack([x[k][b, h] for b, h in pairs]))
+                d = {k: to_dev(v, cfg, k) for k, v in x.items()}
+                sfda.sfda_step(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], S, o, o_im)
+                out[s0 + i] = o[bi, hi].float()
+                out_im[s0 + i] = o_im[bi, hi].float()
+    torch.cuda.synchronize()
+    seqs = {k: np.stack(v, axis=1).astype(np.float64) for k, v in sampled.items()}     # [N, steps, ...]
+    S0s = np.stack([S0[b, h] for b, h in pairs]).astype(np.float64)
+    S_end = np.stack([S[b, h].cpu().numpy() for b, h in pairs])
+    return seqs, S0s, out.cpu().numpy().transpose(1, 0, 2), out_im.cpu().numpy().transpose(1, 0, 2), S_end
+
+
+def check_decode(cfg, pairs, tol_o, tol_S):
+    seqs, S0s, o, o_im, S_end = run_decode(cfg, cfg.steps, pairs)
+    w_re, w_im, w_S = recurrence.sfda_recurrence(seqs["q"], seqs["k"], seqs["v"], seqs["alpha"], seqs["theta"],
+                                                 seqs["beta"], S0s)
+    assert rel_err(o, w_re) <= tol_o
+    assert rel_err(o_im, w_im) <= tol_o
+    assert rel_err(S_end, w_S) <= tol_S
+
+
+@pytest.mark.parametrize("d_k,d_v,dtype", [(64, 64, "f32"), (64, 128, "f32"), (128, 64, "bf16"), (128, 128, "f32"),
+                                           (128, 128, "bf16")])
+def test_step_small(d_k, d_v, dtype):
+    cfg = workloads.CONFIGS[4].scaled(name="dec", B=3, H=2, d_k=d_k, d_v=d_v, dtype=dtype, s0_std=0.5, steps=40)
+    # fp32 arithmetic; bf16 storage only rounds o
+    check_decode(cfg, all_pairs(cfg), 1e-4 if dtype == "f32" else 5e-3, 1e-4)
+
+
+def test_step_full_size_decode_config():
+    """Configuration 4: B = 256 sequences, H = 32, 1024 consecutive steps; the oracle follows a
+    sample of (batch, head) states through all steps."""
+    cfg = workloads.CONFIGS[4]
+    check_decode(cfg, [(0, 0), (255, 31), (100, 7), (31, 16)], TOL["bf16"], 1e-4)
+
+
+def test_iterated_step_equals_forward():
+    """Decode step by step == chunked forward on the same tokens."""
+    cfg = workloads.CONFIGS[0].scaled(name="it", B=2, T=48, H=2, d_k=128, d_v=128, chunk=16, s0_std=0.3, seed=12)
+    inp = workloads.forward_inputs(cfg)
+    o_f, o_im_f, S_f = run_forward(cfg, inp)
+    S = torch.from_numpy(inp["S0"]).to(DEV)
+    o = torch.empty(cfg.B, cfg.H, cfg.d_v, device=DEV)
+    o_im = torch.empty_like(o)
+    for t in range(cfg.T):
+        d = {k: to_dev(np.ascontiguousarray(inp[k][:, t]), cfg, k) for k in ("q", "k", "v", "alpha", "theta", "beta")}
+        sfda.sfda_step(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], S, o, o_im)
+        assert rel_err(o.cpu().numpy(), o_f[:, t]) < 1e-4
+        assert rel_err(o_im.cpu().numpy(), o_im_f[:, t]) < 1e-4
+    assert rel_err(S.cpu().numpy(), S_f) < 1e-4
+
+
+# ------------------------------------------------------------------------------------------------
+# host-buffer entry point and argument errors
+# ------------------------------------------------------------------------------------------------
+def test_forward_host_matches_device_call():
+    cfg = workloads.CONFIGS[1].scaled(name="host", B=2, T=256, H=2, s0_std=0.1)
+    inp = workloads.forward_inputs(cfg)
+    o_d, o_im_d, S_d = run_forward(cfg, inp)
+    h = {}
+    for key, val in inp.items():
+        t = torch.from_numpy(np.ascontiguousarray(val))
+        if key in ("q", "k", "v"):
+            t = t.to(torch.bfloat16)
+        h[key] = t.pin_memory()
+    o = torch.empty(cfg.B, cfg.T, cfg.H, cfg.d_v, dtype=torch.bfloat16).pin_memory()
+    o_im = torch.empty_like(o).pin_memory()
+    S_T = torch.empty(cfg.B, cfg.H, cfg.d_k, cfg.d_v).pin_memory()
+    n = sfda.sfda_forward_host_arena_bytes(cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk, 1, True, True, True)
+    arena = torch.empty(n, dtype=torch.uint8, device=DEV)
+    h2d, d2h = sfda.sfda_forward_host(h["q"], h["k"], h["v"], h["alpha"], h["theta"], h["beta"], h["S0"], o, o_im,
+                                      S_T, cfg.chunk, arena)
+    torch.cuda.synchronize()
+    assert h2d == sum(h[k].numel() * h[k].element_size() for k in h)
+    assert d2h == 2 * o.numel() * 2 + S_T.numel() * 4
+    assert np.array_equal(o.float().numpy(), o_d) and np.array_equal(o_im.float().numpy(), o_im_d)
+    assert np.array_equal(S_T.numpy(), S_d)
+
+
+def test_argument_errors_launch_nothing():
+    cfg = workloads.CONFIGS[0]
+    inp = workloads.forward_inputs(cfg)
+    d = {k: (None if v is None else to_dev(v, cfg, k)) for k, v in inp.items()}
+    o = torch.empty(1, cfg.T, cfg.H, cfg.d_v, device=DEV)
+    with pytest.raises(sfda.SfdaError) as e:
+        sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], None, o, None, None, 48)
+    assert e.value.status == -3
+    with pytest.raises(sfda.SfdaError) as e:
+        sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], None, o[..., 1:].reshape(-1)[1:33],
+                          None, None, 16)
+    assert e.value.status == -4
