@@ -1,0 +1,322 @@
+#!/usr/bin/env python
+"""Benchmark of the SFDA chunk-WY forward on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+One "step" is one pass of the whole hot path (sfda_forward: cumulative phase-decay,
+operand construction, Gram blocks, the WY triangular system, state-dependent
+contractions, outputs, boundary-state scan) over one batch of synthetic input of the
+headline configuration (B=8, T=8192, H=32, d_k=d_v=128, chunk=64, bf16 q/k/v, fp32
+alpha/theta/beta/state, S0 ~ N(0, 0.02), o = Re + Im).  Prints ONE JSON line.
+
+With N > 1 (launched by torch.distributed.run) every rank runs the same per-GPU
+workload on its own batch (the path shards over (batch, head) with no collective):
+weak scaling, value = all ranks' tokens / max-over-ranks time.
+
+`--impl reference` times the CPU oracle (the deliberately plain per-token recurrence)
+on a bounded sample of the same workload.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import workloads  # noqa: E402
+
+METRIC = "SFDA chunk-WY forward tokens/sec at B=8,T=8192,H=32,d=128"
+UNIT = "tokens/s"
+HEADLINE = 2
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def algorithmic_bytes(cfg, want_im=True):
+    """Compulsory HBM traffic of one forward: q, k, v, alpha, theta, beta read once, o (and o_im)
+    written once, S0 read and S_T written once per (batch, head)."""
+    eb = 2 if cfg.dtype == "bf16" else 4
+    per_token_head = 2 * cfg.d_k * eb + cfg.d_v * eb + 2 * cfg.m * 4 + 4 + (2 if want_im else 1) * cfg.d_v * eb
+    return cfg.B * cfg.T * cfg.H * per_token_head + cfg.B * cfg.H * 2 * cfg.d_k * cfg.d_v * 4
+
+
+def algorithmic_flops(cfg, want_im=True):
+    """F_chunk = 4 d_k C^2 + 12 C d_k d_v + 8 C^2 d_v real flops per chunk for Re + Im outputs
+    (complex MAC = 8 flops, triangular products at their triangular size)."""
+    C = cfg.chunk
+    f = 4 * cfg.d_k * C * C + 12 * C * cfg.d_k * cfg.d_v + 8 * C * C * cfg.d_v
+    if not want_im:
+        f -= 2 * C * cfg.d_k * cfg.d_v + 2 * C * C * cfg.d_v
+    return cfg.B * cfg.H * (-(-cfg.T // C)) * f
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self._stop = threading.Event()
+        self._thread = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5)
+                if out.returncode == 0 and out.stdout.strip():
+                    self.rows.append([c.strip() for c in out.stdout.strip().splitlines()[0].split(",")])
+            except Exception:
+                pass
+            self._stop.wait(0.05)
+
+    def __enter__(self):
+        self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        self._thread.join(timeout=10)
+
+    def summary(self):
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                smax.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, val in zip(names, r[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def cpu_oracle_throughput(cfg, n_pairs, T):
+    """Time the oracle, as it stands, on n_pairs (batch, head) sequences of T tokens of the workload."""
+    from oracle import recurrence
+    sub = cfg.scaled(T=T)
+    per_b = max(1, min(cfg.H, n_pairs))
+    pairs = [(i // per_b, i % per_b) for i in range(n_pairs)]
+    inp = workloads.forward_inputs(sub, batch=sorted({b for b, _ in pairs}))
+    s = workloads.sequences(inp, pairs)
+    recurrence.sfda_recurrence(s["q"][:, :64], s["k"][:, :64], s["v"][:, :64], s["alpha"][:, :64],
+                               s["theta"][:, :64], s["beta"][:, :64], s["S0"])       # load + warm the library
+    t0 = time.perf_counter()
+    recurrence.sfda_recurrence(s["q"], s["k"], s["v"], s["alpha"], s["theta"], s["beta"], s["S0"])
+    dt = time.perf_counter() - t0
+    tokens = n_pairs * T / cfg.H          # a token carries all H heads
+    return tokens / dt, dt, recurrence.num_threads()
+
+
+def run_reference(args, rank):
+    """--impl reference: the CPU oracle on a bounded sample; rank 0 only."""
+    if rank != 0:
+        return
+    cfg = workloads.CONFIGS[HEADLINE]
+    cores = len(os.sched_getaffinity(0))
+    n_pairs, T = max(8, 2 * cores), 2048
+    vals, times = [], []
+    for i in range(args.warmup + args.steps):
+        v, dt, threads = cpu_oracle_throughput(cfg, n_pairs, T)
+        if i >= args.warmup:
+            vals.append(v)
+            times.append(dt)
+    value = float(statistics.median(vals))
+    sample = "%d (batch, head) sequences x first %d tokens of the headline workload per step" % (n_pairs, T)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * float(statistics.median(times)),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "T": cfg.T, "H": cfg.H, "d_k": cfg.d_k, "d_v": cfg.d_v,
+                   "chunk": cfg.chunk, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--re-only", action="store_true", help="write o = Re only (default: Re and Im)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else max(args.warmup, 0)
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_2607_11897_b200 as sfda
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    sfda.load()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg = workloads.CONFIGS[HEADLINE]
+    want_im = not args.re_only
+    # every rank draws its own batch: batch elements rank*B .. rank*B + B - 1 of the same recipe
+    inp = workloads.forward_inputs(cfg, batch=range(rank * cfg.B, (rank + 1) * cfg.B))
+    host = {}
+    for key, val in inp.items():
+        t = torch.from_numpy(np.ascontiguousarray(val))
+        if key in ("q", "k", "v"):
+            t = t.to(torch.bfloat16)
+        host[key] = t.pin_memory()
+    d = {k: v.to(dev, non_blocking=True) for k, v in host.items()}
+    o = torch.empty(cfg.B, cfg.T, cfg.H, cfg.d_v, device=dev, dtype=torch.bfloat16)
+    o_im = torch.empty_like(o) if want_im else None
+    S_T = torch.empty(cfg.B, cfg.H, cfg.d_k, cfg.d_v, device=dev)
+    ws = torch.empty(max(sfda.sfda_workspace_bytes(cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk, 1), 256),
+                     dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im, S_T,
+                          cfg.chunk, ws, stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    launches_per_step = sfda.last_launch_count()
+    barrier()
+    events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        start.record(stream)
+        for e0, e1 in events:
+            e0.record(stream)
+            step()
+            e1.record(stream)
+        stop.record(stream)
+        barrier()
+    total_ms = start.elapsed_time(stop)
+    kernel_ms = [e0.elapsed_time(e1) for e0, e1 in events]      # one forward = one launch of the chunk kernel
+    t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    tokens_per_step = world * cfg.B * cfg.T
+    value = tokens_per_step / (ms_per_step * 1e-3)
+
+    # end to end through the host-buffer entry point: H2D of the inputs and D2H of the results inside the timing
+    e2e = None
+    if args.e2e_steps > 0:
+        oh = torch.empty(cfg.B, cfg.T, cfg.H, cfg.d_v, dtype=torch.bfloat16).pin_memory()
+        oh_im = torch.empty_like(oh).pin_memory() if want_im else None
+        Sh = torch.empty(cfg.B, cfg.H, cfg.d_k, cfg.d_v).pin_memory()
+        n = sfda.sfda_forward_host_arena_bytes(cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk, 1, want_im, True, True)
+        arena = torch.empty(n, dtype=torch.uint8, device=dev)
+        h2d = d2h = 0
+        for i in range(1 + args.e2e_steps):
+            if i == 1:
+                barrier()
+                t0 = time.perf_counter()
+            h2d, d2h = sfda.sfda_forward_host(host["q"], host["k"], host["v"], host["alpha"], host["theta"],
+                                              host["beta"], host["S0"], oh, oh_im, Sh, cfg.chunk, arena, stream)
+            stream.synchronize()
+        barrier()
+        e2e_s = (time.perf_counter() - t0) / args.e2e_steps
+        t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e = {"value": tokens_per_step / float(t.item()), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": int(d2h), "ms_per_step": 1e3 * float(t.item())}
+        del arena
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    abytes = algorithmic_bytes(cfg, want_im)
+    aflops = algorithmic_flops(cfg, want_im)
+    k_ms = float(statistics.mean(kernel_ms))
+    achieved_gbs = abytes / (k_ms * 1e-3) / 1e9
+    achieved_tf = aflops / (k_ms * 1e-3) / 1e12
+    hbm_time = abytes / (peaks["hbm_gbs"] * 1e9)
+    tensor_time = aflops / (peaks["bf16_tflops"] * 1e12)
+    roofline = {
+        "bound": "hbm", "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+        "frac": achieved_gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": "of " + peaks["source"],
+        "kernel": "sfda_forward chunk kernel (1 launch per step)", "kernel_ms": k_ms,
+        "algorithmic_bytes": abytes, "algorithmic_flops": aflops, "achieved_tflops": achieved_tf,
+        "tensor_frac": achieved_tf / peaks["bf16_tflops"],
+        "roofline_ms": 1e3 * max(hbm_time, tensor_time),
+    }
+    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(traffic_path):
+        with open(traffic_path) as f:
+            roofline["traffic"] = json.load(f).get("sfda_forward_headline_bytes_per_launch")
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        cores = len(os.sched_getaffinity(0))
+        n_pairs, T = max(8, 4 * cores), cfg.T
+        v, dt, threads = cpu_oracle_throughput(cfg, n_pairs, T)
+        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": dt,
+               "sample": "%d of the %d (batch, head) sequences, all %d tokens" % (n_pairs, cfg.B * cfg.H, T)}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "T": cfg.T, "H": cfg.H, "d_k": cfg.d_k, "d_v": cfg.d_v,
+                   "chunk": cfg.chunk, "outputs": "Re+Im" if want_im else "Re", "state": "fp32", "S0": "N(0,0.02)",
+                   "parallelism": "dp%d over (batch, head), no collective" % world,
+                   "l2": "inputs+outputs %.2f GB per step, far larger than the 126 MB L2; no flush" % (abytes / 1e9)},
+        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
+        "gpu_launches": launches_per_step * args.steps, "clocks": clocks.summary(),
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

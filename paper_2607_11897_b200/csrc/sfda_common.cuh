@@ -31,8 +31,9 @@ __device__ __forceinline__ void turns_to_cos_sin(uint32_t turns, float *c, float
     sincospif(x, s, c);
 }
 
-// log of a decay factor, floored so that sums of 64 of them stay finite and differences of two
-// such sums never give inf - inf (alpha = 0 is admissible in the recurrence).
-__device__ __forceinline__ float log_decay(float alpha) { return fmaxf(logf(alpha), -1.0e4f); }
+// log of a decay factor, floored at -30: alpha below e^-30 (alpha = 0 is admissible in the
+// recurrence) then acts as e^-30 ~ 9e-14, far below fp32 resolution of anything it multiplies, while
+// cumulative sums over a chunk stay small enough that differences of two of them keep fp32 precision.
+__device__ __forceinline__ float log_decay(float alpha) { return fmaxf(logf(alpha), -30.0f); }
 
 }  // namespace sfda
