@@ -83,7 +83,7 @@ SFDA_API int sfda_plan(int T, int chunk, int *n_chunks, int *tail_len);
 
 /*
  * Bytes of device scratch sfda_forward needs for these sizes (0 when it needs
- * none).  Returns 0 for invalid sizes as well; sfda_forward reports those.
+ * none; 256 for the tensor-core path, which keeps a status word there).  Returns 0 for invalid sizes as well; sfda_forward reports those.
  */
 SFDA_API size_t sfda_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int dtype);
 
@@ -113,6 +113,16 @@ SFDA_API int sfda_forward(const void *q, const void *k, const void *v,
                  const float *S0, void *o, void *o_im, float *S_T,
                  int B, int T, int H, int d_k, int d_v, int chunk, int dtype,
                  void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * After work enqueued by sfda_forward with a non-empty workspace: waits for `stream`
+ * and reads the status word the tensor-core kernel keeps at the start of the
+ * workspace.  Returns SFDA_OK, or SFDA_ERR_TIMEOUT when a bounded device-side wait
+ * (on a TMA copy or a tensor-core commit) ran out, in which case the kernel returned
+ * early and o, o_im, S_T of that call are invalid; *detail (host, may be NULL) gets
+ * the raw word.  Synchronises the stream.  Host only.
+ */
+SFDA_API int sfda_workspace_status(const void *workspace, void *stream, uint32_t *detail);
 
 /*
  * Same computation forced onto the fp32 CUDA-core path for any dtype (the

@@ -45,6 +45,7 @@ def load():
     lib.sfda_forward_host.argtypes = [_vp] * 10 + [_ci] * 7 + [_vp, _sz, _vp, ctypes.POINTER(_sz),
                                                           ctypes.POINTER(_sz)]
     lib.sfda_last_launch_count.restype = _ci
+    lib.sfda_workspace_status.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_uint32)]
     _LIB = lib
     return lib
 
@@ -121,6 +122,15 @@ def _forward_common(fn_name, q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chun
 def sfda_forward(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chunk, workspace=None, stream=None):
     """``sfda_forward`` of ``include/sfda.h``; tensors are CUDA tensors the caller allocated."""
     _forward_common("sfda_forward", q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chunk, workspace, stream)
+
+
+def sfda_workspace_status(workspace, stream=None) -> int:
+    """``sfda_workspace_status``: 0, or raises SfdaError(-7) when a device-side wait ran out."""
+    word = ctypes.c_uint32()
+    rc = load().sfda_workspace_status(_ptr(workspace), _stream(stream), ctypes.byref(word))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_workspace_status")
+    return int(word.value)
 
 
 def sfda_forward_simt(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chunk, stream=None):

@@ -79,8 +79,10 @@ int sfda_plan(int T, int chunk, int *n_chunks, int *tail_len)
 
 size_t sfda_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int dtype)
 {
-    (void)B; (void)T; (void)H; (void)d_k; (void)d_v; (void)chunk; (void)dtype;
-    return 0;
+    if (B < 1 || T < 1 || H < 1 || check_dims(d_k, d_v, chunk, dtype) != SFDA_OK) return 0;
+    sfda::ForwardArgs a{};
+    a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.chunk = chunk; a.dtype = dtype;
+    return sfda::forward_tc_supported(a) ? 256 : 0;   // the tensor-core path keeps a status word there
 }
 
 int sfda_forward_simt(const void *q, const void *k, const void *v, const float *alpha, const float *theta,
@@ -107,9 +109,24 @@ int sfda_forward(const void *q, const void *k, const void *v, const float *alpha
     if (need > 0 && (!workspace || workspace_bytes < need)) return SFDA_ERR_WORKSPACE;
     if (workspace && !aligned16(workspace)) return SFDA_ERR_ALIGN;
     const sfda::ForwardArgs a = pack(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
-    return sfda::launch_forward_simt(a, static_cast<cudaStream_t>(stream), &g_last_launches) == cudaSuccess
-               ? SFDA_OK
-               : SFDA_ERR_CUDA;
+    const cudaError_t e =
+        sfda::forward_tc_supported(a)
+            ? sfda::launch_forward_tc(a, static_cast<uint32_t *>(workspace), static_cast<cudaStream_t>(stream),
+                                      &g_last_launches)
+            : sfda::launch_forward_simt(a, static_cast<cudaStream_t>(stream), &g_last_launches);
+    return e == cudaSuccess ? SFDA_OK : SFDA_ERR_CUDA;
+}
+
+int sfda_workspace_status(const void *workspace, void *stream, uint32_t *detail)
+{
+    if (!workspace) return SFDA_ERR_NULL;
+    uint32_t word = 0;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess)
+        return SFDA_ERR_CUDA;
+    if (detail) *detail = word;
+    return word == 0 ? SFDA_OK : SFDA_ERR_TIMEOUT;
 }
 
 int sfda_chunk_factors(const void *k, const float *alpha, const float *theta, const float *beta, float *Gamma,

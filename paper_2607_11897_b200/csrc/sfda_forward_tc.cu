@@ -1,0 +1,750 @@
+// Tensor-core chunk-WY forward for sm_100a: bf16 q/k/v, d_k = d_v = 128, chunk C = 64.
+//
+// One CTA walks the chunks of one (batch, head) pair.  The fp32 state lives in tensor memory for the
+// whole sequence, transposed: TMEM lane c = value channel, column = key channel in de-interleaved order
+// [Re j = 0..63 | Im j = 0..63].  Every dense contraction is a tcgen05.mma (kind::f16, bf16 operands,
+// fp32 accumulators in TMEM); the state-dependent ones take their A operand (bf16 copies of S, R, E) from
+// TMEM and their B operand from 128-byte-swizzled K-major shared-memory tiles that the CUDA cores build.
+//
+// With gamma_t = a_t e^{i phi_t} the chunk-local cumulative phase-decay (Eq. "constructive-Gamma"),
+// k'_t = e^{-i phi_t} k_t, q'_t = e^{-i phi_t} q_t:
+//
+//   W_t   = a_t k'_t                (= conj(gamma_t) k_t, Eq. "constructive-W")
+//   Kc_t  = k'_t / a_t              (= k_t / gamma_t)
+//   Qt_t  = a_t q'_t                (= conj(gamma_t) q_t)
+//   Y'_t  = (a_C / a_t) k'_t        (= e^{-i phi_C} (gamma_C / gamma_t) k_t, cf. Eq. "constructive-Y")
+//   Kt[t][i] = W_t^* Kc_i (i < t),  Aq[t][i] = Qt_t^* Kc_i (i <= t)          -- Gram blocks
+//   M_beta = (I + D_beta Kt)^{-1} D_beta                                     -- unit-lower WY system
+//   R = V - W^* S_0,  E = M_beta R                                           -- Eq. "apply-transfer"
+//   rho_t = Qt_t^* S_0 + sum_{i<=t} Aq[t][i] e_i^T,  o_t = conj(rho_t)       -- Thm "Prefix outputs"
+//   S_C = e^{i phi_C} (a_C S_0 + sum_t Y'_t e_t^T)                           -- boundary-state scan
+//
+// Complex products are real block products over the de-interleaved halves; where a minus sign is needed
+// the instruction descriptor's negate-B bit supplies it, so no operand is stored twice.
+#include <cuda.h>
+
+#include "sfda_common.cuh"
+#include "sfda_internal.h"
+
+namespace sfda {
+namespace {
+
+constexpr int C = 64;         // chunk
+constexpr int DK = 128, DV = 128, M = 64;
+constexpr int kThreads = 256;
+
+// ---- shared memory map (bytes from a 1024-aligned base) -------------------------------------------
+constexpr int kTile = 8192;                      // 64 rows x 128 B, K-major, 128B swizzle
+constexpr int OFF_WQ_RE = 0;                     // 128 rows: W (0..63) then Qt (64..127), Re halves
+constexpr int OFF_WQ_IM = OFF_WQ_RE + 2 * kTile;
+constexpr int OFF_KC_RE = OFF_WQ_IM + 2 * kTile;
+constexpr int OFF_KC_IM = OFF_KC_RE + kTile;
+constexpr int OFF_YT_RE = OFF_KC_IM + kTile;     // Y'^T [j][t]
+constexpr int OFF_YT_IM = OFF_YT_RE + kTile;
+constexpr int OFF_MB_RE = OFF_YT_IM + kTile;     // M_beta [t][i]
+constexpr int OFF_MB_IM = OFF_MB_RE + kTile;
+constexpr int OFF_AQ_RE = OFF_MB_IM + kTile;     // Aq [t][i], upper triangle zero
+constexpr int OFF_AQ_IM = OFF_AQ_RE + kTile;
+constexpr int OFF_V = OFF_AQ_IM + kTile;         // v staging [t][128] bf16 (TMA, no swizzle)
+constexpr int OFF_Q = OFF_V + 16384;             // q staging [t][128] bf16
+constexpr int OFF_K = OFF_Q + 16384;             // k staging
+constexpr int OFF_ALPHA = OFF_K + 16384;         // alpha staging [t][64] fp32
+constexpr int OFF_THETA = OFF_ALPHA + 16384;     // theta staging
+constexpr int OFF_SOLVE = OFF_Q;                 // L, X (fp32 complex 64x64) alias the staging buffers
+constexpr int OFF_MISC = OFF_THETA + 16384;
+constexpr int kSmemBytes = OFF_MISC + 16384 + 1024;   // + slack for the 1024-byte alignment
+
+struct Misc {
+    float part_lg[4][M];
+    uint32_t part_turns[4][M];
+    float aC[M];
+    float closing_cos[2][M], closing_sin[2][M];
+    float beta[C];
+    float Tr[4][16][16], Ti[4][16][16];
+    unsigned long long bar_mma, bar_in, bar_v;
+    uint32_t tmem_base;
+};
+static_assert(sizeof(Misc) <= 16384, "misc area too small");
+
+// ---- tensor memory map (columns) -------------------------------------------------------------------
+constexpr uint32_t TM_S32 = 0;     // state fp32: [Re j | Im j]
+constexpr uint32_t TM_S16 = 128;   // bf16 copy of the chunk-start state (A operand), 64 packed columns
+constexpr uint32_t TM_X16 = 192;   // bf16 R, then E (A operand)
+constexpr uint32_t TM_ACC = 256;   // [D1/E re | rho re | D1/E im | rho im], 64 columns each; Gram uses 0..127
+
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+// ---- small PTX wrappers ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(unsigned long long *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Bounded wait: returns false when the phase did not complete within the spin limit.
+__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, uint32_t parity)
+{
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+            : "=r"(ok)
+            : "r"(smem_u32(bar)), "r"(parity)
+            : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, unsigned long long *bar, int c0, int c1,
+                                            int c2, int c3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2),
+        "r"(c3)
+        : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// K-major, 128-byte-swizzled operand tile: 8-row atoms of 1024 B (stride-dimension offset 1024).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// kind::f16 instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, M = 128.
+__device__ __forceinline__ constexpr uint32_t idesc(int N, int neg_b)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)neg_b << 14) | ((uint32_t)(N >> 3) << 17) |
+           ((uint32_t)(128 >> 4) << 24);
+}
+__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t id, uint32_t acc)
+{
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+                 ::"r"(d), "l"(a), "l"(b), "r"(id), "r"(acc)
+                 : "memory");
+}
+__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t id, uint32_t acc)
+{
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
+                 ::"r"(d), "r"(a), "l"(b), "r"(id), "r"(acc)
+                 : "memory");
+}
+__device__ __forceinline__ void mma_commit(unsigned long long *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+// K = 64 (one swizzle span) product: four K = 16 instructions. A from shared memory / from TMEM.
+__device__ __forceinline__ void mma_k64_ss(uint32_t d, uint32_t a_saddr, uint32_t b_saddr, uint32_t id, bool acc)
+{
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks)
+        mma_ss(d, smem_desc(a_saddr + 32 * ks), smem_desc(b_saddr + 32 * ks), id, (acc || ks > 0) ? 1u : 0u);
+}
+__device__ __forceinline__ void mma_k64_ts(uint32_t d, uint32_t a_tmem, uint32_t b_saddr, uint32_t id, bool acc)
+{
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks) mma_ts(d, a_tmem + 8 * ks, smem_desc(b_saddr + 32 * ks), id, (acc || ks > 0) ? 1u : 0u);
+}
+
+#define SFDA_R32(r, o) \
+    "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), "=r"(r[o + 6]), \
+    "=r"(r[o + 7]), "=r"(r[o + 8]), "=r"(r[o + 9]), "=r"(r[o + 10]), "=r"(r[o + 11]), "=r"(r[o + 12]),               \
+    "=r"(r[o + 13]), "=r"(r[o + 14]), "=r"(r[o + 15])
+#define SFDA_W32(r, o) \
+    "r"(r[o + 0]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]), "r"(r[o + 6]), \
+    "r"(r[o + 7]), "r"(r[o + 8]), "r"(r[o + 9]), "r"(r[o + 10]), "r"(r[o + 11]), "r"(r[o + 12]), "r"(r[o + 13]), \
+    "r"(r[o + 14]), "r"(r[o + 15])
+
+// 16 consecutive 32-bit columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t *r)
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : SFDA_R32(r, 0)
+                 : "r"(addr));
+}
+__device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t *r)
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+                 ::"r"(addr), SFDA_W32(r, 0)
+                 : "memory");
+}
+template <int N>
+__device__ __forceinline__ void tmem_ld(uint32_t addr, uint32_t *r)
+{
+#pragma unroll
+    for (int i = 0; i < N; i += 16) tmem_ld16(addr + i, r + i);
+}
+template <int N>
+__device__ __forceinline__ void tmem_st(uint32_t addr, const uint32_t *r)
+{
+#pragma unroll
+    for (int i = 0; i < N; i += 16) tmem_st16(addr + i, r + i);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) |
+           ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
+}
+// Byte offset of element (row r, k-element e < 64) in a K-major 128B-swizzled tile.
+__device__ __forceinline__ int sw_off(int r, int e)
+{
+    return (r >> 3) * 1024 + (r & 7) * 128 + ((((e >> 3) ^ r) & 7) << 4) + ((e & 7) << 1);
+}
+// fp32 64x64 scratch matrices of the triangular solve, XOR-swizzled so that one column read by 32 rows
+// and one row read by 32 columns are both conflict-free.
+__device__ __forceinline__ int lx(int r, int k) { return r * 64 + (k ^ (r & 31)); }
+
+struct Params {
+    const float *beta, *S0;
+    __nv_bfloat16 *o, *o_im;
+    float *S_T;
+    uint32_t *status;
+    int T, H;
+};
+
+// ---- the kernel -------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads, 1)
+sfda_forward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                       const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_alpha,
+                       const __grid_constant__ CUtensorMap tm_theta, const Params p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    Misc &mi = *reinterpret_cast<Misc *>(smem + OFF_MISC);
+    float *Lr = reinterpret_cast<float *>(smem + OFF_SOLVE);
+    float *Li = Lr + 4096, *Xr = Li + 4096, *Xi = Xr + 4096;
+    const uint32_t sbase = smem_u32(smem);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int quad = warp & 3, half = warp >> 2;
+    const int bh = blockIdx.x, h = bh % p.H, b = bh / p.H;
+    const int n_chunks = (p.T + C - 1) / C;
+
+    if (tid == 0) {
+        mbar_init(&mi.bar_mma, 1);
+        mbar_init(&mi.bar_in, 1);
+        mbar_init(&mi.bar_v, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&mi.tmem_base)));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = mi.tmem_base;
+    const uint32_t tlane = tmem + ((uint32_t)(quad * 32) << 16);   // this warp's lane quadrant
+
+    if (tid == 0) {
+        mbar_expect_tx(&mi.bar_in, 4 * 16384);
+        tma_load_4d(smem + OFF_Q, &tm_q, &mi.bar_in, 0, h, 0, b);
+        tma_load_4d(smem + OFF_K, &tm_k, &mi.bar_in, 0, h, 0, b);
+        tma_load_4d(smem + OFF_ALPHA, &tm_alpha, &mi.bar_in, 0, h, 0, b);
+        tma_load_4d(smem + OFF_THETA, &tm_theta, &mi.bar_in, 0, h, 0, b);
+        mbar_expect_tx(&mi.bar_v, 16384);
+        tma_load_4d(smem + OFF_V, &tm_v, &mi.bar_v, 0, h, 0, b);
+    }
+
+    uint32_t ph_mma = 0, ph_in = 0, ph_v = 0;
+    bool in_flight_in = true, in_flight_v = true;
+    int failed = 0;
+
+    for (int ci = 0; ci < n_chunks; ++ci) {
+        const int t0 = ci * C;
+        const int len = min(C, p.T - t0);
+        const int cur = ci & 1;
+
+        // ================= prep: cumulative phase-decay and the operand tiles =======================
+        failed = __syncthreads_or(mbar_wait(&mi.bar_in, ph_in) ? 0 : 1);
+        ph_in ^= 1;
+        in_flight_in = false;
+        if (failed) break;
+        {
+            const int j = tid & 63, tq = tid >> 6;
+            const float *s_alpha = reinterpret_cast<const float *>(smem + OFF_ALPHA);
+            const float *s_theta = reinterpret_cast<const float *>(smem + OFF_THETA);
+            float lg[16];
+            uint32_t tu[16];
+            float acc = 0.f;
+            uint32_t tacc = 0u;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int t = tq * 16 + i;
+                if (t < len) {
+                    acc += fmaxf(__log2f(s_alpha[t * M + j]), -43.28f);   // floor e^-30, as in log_decay
+                    tacc += phase_to_turns(s_theta[t * M + j]);
+                }
+                lg[i] = acc;
+                tu[i] = tacc;
+            }
+            mi.part_lg[tq][j] = acc;
+            mi.part_turns[tq][j] = tacc;
+            if (tid < C) mi.beta[tid] = tid < len ? p.beta[((size_t)b * p.T + t0 + tid) * p.H + h] : 0.f;
+            __syncthreads();
+            float base = 0.f, total = 0.f;
+            uint32_t tbase = 0u, ttotal = 0u;
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                const float pl = mi.part_lg[g][j];
+                const uint32_t pt = mi.part_turns[g][j];
+                if (g < tq) { base += pl; tbase += pt; }
+                total += pl;
+                ttotal += pt;
+            }
+            if (tq == 0) {
+                mi.aC[j] = exp2f(total);
+                float cs, sn;
+                const float ang = (float)(int32_t)ttotal * 0x1.921fb6p-30f;   // turns * 2 pi / 2^32
+                __sincosf(ang, &sn, &cs);
+                mi.closing_cos[cur][j] = cs;
+                mi.closing_sin[cur][j] = sn;
+            }
+            const uint32_t *s_q = reinterpret_cast<const uint32_t *>(smem + OFF_Q);
+            const uint32_t *s_k = reinterpret_cast<const uint32_t *>(smem + OFF_K);
+            uint32_t ytr[8], yti[8];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int t = tq * 16 + i;
+                const float l2 = base + lg[i];
+                const float a = exp2f(l2);
+                const float ainv = exp2f(fminf(-l2, 115.4f));                 // 1/a_t, capped at e^80
+                const float ay = exp2f(total - l2);                           // a_C / a_t <= 1
+                float cs, sn;
+                __sincosf((float)(int32_t)(tbase + tu[i]) * 0x1.921fb6p-30f, &sn, &cs);
+                const uint32_t kw = s_k[t * 64 + j], qw = s_q[t * 64 + j];
+                const float kr = __uint_as_float(kw << 16), ki = __uint_as_float(kw & 0xffff0000u);
+                const float qr = __uint_as_float(qw << 16), qi = __uint_as_float(qw & 0xffff0000u);
+                const float kpr = kr * cs + ki * sn, kpi = ki * cs - kr * sn;   // e^{-i phi} k
+                const float qpr = qr * cs + qi * sn, qpi = qi * cs - qr * sn;
+                const int o1 = sw_off(t, j);
+                *reinterpret_cast<__nv_bfloat16 *>(smem + OFF_WQ_RE + o1) = __float2bfloat16_rn(a * kpr);
+                *reinterpret_cast<__nv_bfloat16 *>(smem + OFF_WQ_IM + o1) = __float2bfloat16_rn(a * kpi);
+                *reinterpret_cast<__nv_bfloat16 *>(smem + OFF_WQ_RE + kTile + o1) = __float2bfloat16_rn(a * qpr);
+                *reinterpret_cast<__nv_bfloat16 *>(smem + OFF_WQ_IM + kTile + o1) = __float2bfloat16_rn(a * qpi);
+                *reinterpret_cast<__nv_bfloat16 *>(smem + OFF_KC_RE + o1) = __float2bfloat16_rn(ainv * kpr);
+                *reinterpret_cast<__nv_bfloat16 *>(smem + OFF_KC_IM + o1) = __float2bfloat16_rn(ainv * kpi);
+                const float yr = ay * kpr, yi = ay * kpi;
+                if (i & 1) {
+                    ytr[i >> 1] |= (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(yr)) << 16;
+                    yti[i >> 1] |= (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(yi)) << 16;
+                } else {
+                    ytr[i >> 1] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(yr));
+                    yti[i >> 1] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(yi));
+                }
+            }
+            // Y'^T row j, tokens 16 tq .. 16 tq + 15: two 16-byte chunks per half.
+#pragma unroll
+            for (int cidx = 0; cidx < 2; ++cidx) {
+                const int off = sw_off(j, tq * 16 + cidx * 8);
+                *reinterpret_cast<uint4 *>(smem + OFF_YT_RE + off) =
+                    make_uint4(ytr[4 * cidx], ytr[4 * cidx + 1], ytr[4 * cidx + 2], ytr[4 * cidx + 3]);
+                *reinterpret_cast<uint4 *>(smem + OFF_YT_IM + off) =
+                    make_uint4(yti[4 * cidx], yti[4 * cidx + 1], yti[4 * cidx + 2], yti[4 * cidx + 3]);
+            }
+        }
+        fence_async_smem();
+        tc_fence_before();
+        __syncthreads();
+
+        // ================= Gram blocks Kt (rows 0..63) and Aq (rows 64..127) ==========================
+        if (tid == 0) {
+            tc_fence_after();
+            const uint32_t d_re = tmem + TM_ACC, d_im = tmem + TM_ACC + 64;
+            mma_k64_ss(d_re, sbase + OFF_WQ_RE, sbase + OFF_KC_RE, idesc(64, 0), false);
+            mma_k64_ss(d_re, sbase + OFF_WQ_IM, sbase + OFF_KC_IM, idesc(64, 0), true);
+            mma_k64_ss(d_im, sbase + OFF_WQ_RE, sbase + OFF_KC_IM, idesc(64, 0), false);
+            mma_k64_ss(d_im, sbase + OFF_WQ_IM, sbase + OFF_KC_RE, idesc(64, 1), true);
+            mma_commit(&mi.bar_mma);
+        }
+        failed = __syncthreads_or(mbar_wait(&mi.bar_mma, ph_mma) ? 0 : 1);
+        ph_mma ^= 1;
+        if (failed) break;
+        tc_fence_after();
+        {
+            uint32_t r[64];
+            tmem_ld<64>(tlane + TM_ACC + 64 * half, r);
+            tc_wait_ld();
+            const int row = quad * 32 + lane;
+            if (row < 64) {                       // L = D_beta Kt, strictly lower
+                const int t = row;
+                const float bt = mi.beta[t];
+                float *dst = half ? Li : Lr;
+#pragma unroll
+                for (int i = 0; i < 64; ++i) dst[lx(t, i)] = i < t ? bt * __uint_as_float(r[i]) : 0.f;
+            } else {                              // Aq, lower incl. diagonal, as a bf16 operand tile
+                const int t = row - 64;
+                uint8_t *tile = smem + (half ? OFF_AQ_IM : OFF_AQ_RE);
+#pragma unroll
+                for (int c8 = 0; c8 < 8; ++c8) {
+                    uint32_t w[4];
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) {
+                        const int i0 = c8 * 8 + 2 * x;
+                        w[x] = pack_bf16(i0 <= t ? __uint_as_float(r[i0]) : 0.f,
+                                         i0 + 1 <= t ? __uint_as_float(r[i0 + 1]) : 0.f);
+                    }
+                    *reinterpret_cast<uint4 *>(tile + sw_off(t, c8 * 8)) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+            }
+        }
+        tc_fence_before();
+        __syncthreads();
+
+        // ================= X = (I + L)^{-1} in fp32 by 16x16 blocks; M_beta = X D_beta ================
+        if (tid < 64) {
+            const int blk = tid >> 4, c = tid & 15, o = 16 * blk;
+            float xr[16], xi[16];
+#pragma unroll
+            for (int r = 0; r < 16; ++r) {
+                float ar = r == c ? 1.f : 0.f, ai = 0.f;
+#pragma unroll
+                for (int i = 0; i < 15; ++i) {
+                    if (i < r && i >= c) {
+                        const float lr_ = Lr[lx(o + r, o + i)], li_ = Li[lx(o + r, o + i)];
+                        ar -= lr_ * xr[i] - li_ * xi[i];
+                        ai -= lr_ * xi[i] + li_ * xr[i];
+                    }
+                }
+                xr[r] = r >= c ? ar : 0.f;
+                xi[r] = r >= c ? ai : 0.f;
+                Xr[lx(o + r, o + c)] = xr[r];
+                Xi[lx(o + r, o + c)] = xi[r];
+            }
+        }
+        __syncthreads();
+        {
+            const int r = tid >> 4, c = tid & 15;
+            for (int d = 1; d < 4; ++d) {
+                for (int rb = d; rb < 4; ++rb) {      // T_rb = sum_kb L[rb][kb] X[kb][cb]
+                    const int cb = rb - d;
+                    float ar = 0.f, ai = 0.f;
+                    for (int kb = cb; kb < rb; ++kb) {
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) {
+                            const float lr_ = Lr[lx(16 * rb + r, 16 * kb + k)], li_ = Li[lx(16 * rb + r, 16 * kb + k)];
+                            const float vr = Xr[lx(16 * kb + k, 16 * cb + c)], vi = Xi[lx(16 * kb + k, 16 * cb + c)];
+                            ar += lr_ * vr - li_ * vi;
+                            ai += lr_ * vi + li_ * vr;
+                        }
+                    }
+                    mi.Tr[rb][r][c] = ar;
+                    mi.Ti[rb][r][c] = ai;
+                }
+                __syncthreads();
+                for (int rb = d; rb < 4; ++rb) {      // X[rb][cb] = -X[rb][rb] T_rb
+                    const int cb = rb - d;
+                    float ar = 0.f, ai = 0.f;
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) {
+                        const float vr = Xr[lx(16 * rb + r, 16 * rb + k)], vi = Xi[lx(16 * rb + r, 16 * rb + k)];
+                        const float tr = mi.Tr[rb][k][c], ti = mi.Ti[rb][k][c];
+                        ar -= vr * tr - vi * ti;
+                        ai -= vr * ti + vi * tr;
+                    }
+                    Xr[lx(16 * rb + r, 16 * cb + c)] = ar;
+                    Xi[lx(16 * rb + r, 16 * cb + c)] = ai;
+                }
+                __syncthreads();
+            }
+        }
+        {
+            const int t = tid >> 2, part = tid & 3;     // row t, columns 16 part .. 16 part + 15
+#pragma unroll
+            for (int cidx = 0; cidx < 2; ++cidx) {
+                uint32_t wr[4], wi[4];
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {
+                    const int i0 = part * 16 + cidx * 8 + 2 * x;
+                    const float b0 = mi.beta[i0], b1 = mi.beta[i0 + 1];
+                    const bool in0 = i0 <= t, in1 = i0 + 1 <= t;
+                    wr[x] = pack_bf16(in0 ? Xr[lx(t, i0)] * b0 : 0.f, in1 ? Xr[lx(t, i0 + 1)] * b1 : 0.f);
+                    wi[x] = pack_bf16(in0 ? Xi[lx(t, i0)] * b0 : 0.f, in1 ? Xi[lx(t, i0 + 1)] * b1 : 0.f);
+                }
+                const int off = sw_off(t, part * 16 + cidx * 8);
+                *reinterpret_cast<uint4 *>(smem + OFF_MB_RE + off) = make_uint4(wr[0], wr[1], wr[2], wr[3]);
+                *reinterpret_cast<uint4 *>(smem + OFF_MB_IM + off) = make_uint4(wi[0], wi[1], wi[2], wi[3]);
+            }
+        }
+
+        // ================= state pass: S16 <- bf16(S_start), S32 <- a_C * S_start ======================
+        {
+            const int c = quad * 32 + lane;        // value channel = TMEM lane
+            const int j0 = half * 32;              // this warp's complex rows
+            uint32_t sre[32], sim[32];
+            if (ci == 0) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int j = j0 + i;
+                    sre[i] = p.S0 ? __float_as_uint(p.S0[((size_t)bh * DK + 2 * j) * DV + c]) : 0u;
+                    sim[i] = p.S0 ? __float_as_uint(p.S0[((size_t)bh * DK + 2 * j + 1) * DV + c]) : 0u;
+                }
+            } else {
+                tmem_ld<32>(tlane + TM_S32 + j0, sre);
+                tmem_ld<32>(tlane + TM_S32 + 64 + j0, sim);
+                tc_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {     // closing phase of the previous chunk
+                    const float cs = mi.closing_cos[cur ^ 1][j0 + i], sn = mi.closing_sin[cur ^ 1][j0 + i];
+                    const float xr = __uint_as_float(sre[i]), xi = __uint_as_float(sim[i]);
+                    sre[i] = __float_as_uint(cs * xr - sn * xi);
+                    sim[i] = __float_as_uint(cs * xi + sn * xr);
+                }
+            }
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(__uint_as_float(sre[2 * i]), __uint_as_float(sre[2 * i + 1]));
+            tmem_st<16>(tlane + TM_S16 + j0 / 2, pk);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(__uint_as_float(sim[2 * i]), __uint_as_float(sim[2 * i + 1]));
+            tmem_st<16>(tlane + TM_S16 + 32 + j0 / 2, pk);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float a = mi.aC[j0 + i];
+                sre[i] = __float_as_uint(a * __uint_as_float(sre[i]));
+                sim[i] = __float_as_uint(a * __uint_as_float(sim[i]));
+            }
+            tmem_st<32>(tlane + TM_S32 + j0, sre);
+            tmem_st<32>(tlane + TM_S32 + 64 + j0, sim);
+            tc_wait_st();
+        }
+        fence_async_smem();
+        tc_fence_before();
+        __syncthreads();
+
+        // ================= D1 = W^* S_0 and rho_1 = Qt^* S_0 (N = 128: W rows then Qt rows) ==========
+        if (tid == 0) {
+            tc_fence_after();
+            if (ci + 1 < n_chunks) {               // staging (aliased by the solve scratch) is free again
+                mbar_expect_tx(&mi.bar_in, 4 * 16384);
+                tma_load_4d(smem + OFF_Q, &tm_q, &mi.bar_in, 0, h, t0 + C, b);
+                tma_load_4d(smem + OFF_K, &tm_k, &mi.bar_in, 0, h, t0 + C, b);
+                tma_load_4d(smem + OFF_ALPHA, &tm_alpha, &mi.bar_in, 0, h, t0 + C, b);
+                tma_load_4d(smem + OFF_THETA, &tm_theta, &mi.bar_in, 0, h, t0 + C, b);
+            }
+            const uint32_t d_re = tmem + TM_ACC, d_im = tmem + TM_ACC + 128;
+            const uint32_t s_re = tmem + TM_S16, s_im = tmem + TM_S16 + 32;
+            mma_k64_ts(d_re, s_re, sbase + OFF_WQ_RE, idesc(128, 0), false);
+            mma_k64_ts(d_re, s_im, sbase + OFF_WQ_IM, idesc(128, 0), true);
+            mma_k64_ts(d_im, s_im, sbase + OFF_WQ_RE, idesc(128, 0), false);
+            mma_k64_ts(d_im, s_re, sbase + OFF_WQ_IM, idesc(128, 1), true);
+            mma_commit(&mi.bar_mma);
+        }
+        in_flight_in = ci + 1 < n_chunks;
+        {
+            const int ok_mma = mbar_wait(&mi.bar_mma, ph_mma) ? 1 : 0;
+            const int ok_v = mbar_wait(&mi.bar_v, ph_v) ? 1 : 0;
+            failed = __syncthreads_or((ok_mma & ok_v) ? 0 : 1);
+        }
+        ph_mma ^= 1;
+        ph_v ^= 1;
+        in_flight_v = false;
+        if (failed) break;
+        tc_fence_after();
+
+        // ================= R = V - D1 -> bf16 A operand ================================================
+        {
+            const int c = quad * 32 + lane;
+            uint32_t r[64], pk[32];
+            tmem_ld<64>(tlane + TM_ACC + 128 * half, r);
+            tc_wait_ld();
+            if (half == 0) {
+                const __nv_bfloat16 *sv = reinterpret_cast<const __nv_bfloat16 *>(smem + OFF_V);
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    pk[i] = pack_bf16(__bfloat162float(sv[(2 * i) * DV + c]) - __uint_as_float(r[2 * i]),
+                                      __bfloat162float(sv[(2 * i + 1) * DV + c]) - __uint_as_float(r[2 * i + 1]));
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) pk[i] = pack_bf16(-__uint_as_float(r[2 * i]), -__uint_as_float(r[2 * i + 1]));
+            }
+            tmem_st<32>(tlane + TM_X16 + 32 * half, pk);
+            tc_wait_st();
+        }
+        tc_fence_before();
+        __syncthreads();
+
+        // ================= E = M_beta R ================================================================
+        if (tid == 0) {
+            tc_fence_after();
+            if (ci + 1 < n_chunks) {
+                mbar_expect_tx(&mi.bar_v, 16384);
+                tma_load_4d(smem + OFF_V, &tm_v, &mi.bar_v, 0, h, t0 + C, b);
+            }
+            const uint32_t e_re = tmem + TM_ACC, e_im = tmem + TM_ACC + 128;
+            const uint32_t r_re = tmem + TM_X16, r_im = tmem + TM_X16 + 32;
+            mma_k64_ts(e_re, r_re, sbase + OFF_MB_RE, idesc(64, 0), false);
+            mma_k64_ts(e_re, r_im, sbase + OFF_MB_IM, idesc(64, 1), true);
+            mma_k64_ts(e_im, r_im, sbase + OFF_MB_RE, idesc(64, 0), false);
+            mma_k64_ts(e_im, r_re, sbase + OFF_MB_IM, idesc(64, 0), true);
+            mma_commit(&mi.bar_mma);
+        }
+        in_flight_v = ci + 1 < n_chunks;
+        failed = __syncthreads_or(mbar_wait(&mi.bar_mma, ph_mma) ? 0 : 1);
+        ph_mma ^= 1;
+        if (failed) break;
+        tc_fence_after();
+        {
+            uint32_t r[64], pk[32];
+            tmem_ld<64>(tlane + TM_ACC + 128 * half, r);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) pk[i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+            tmem_st<32>(tlane + TM_X16 + 32 * half, pk);
+            tc_wait_st();
+        }
+        tc_fence_before();
+        __syncthreads();
+
+        // ================= S += E^T Y'  and  rho += Aq E ================================================
+        if (tid == 0) {
+            tc_fence_after();
+            const uint32_t e_re = tmem + TM_X16, e_im = tmem + TM_X16 + 32;
+            const uint32_t s_re = tmem + TM_S32, s_im = tmem + TM_S32 + 64;
+            mma_k64_ts(s_re, e_re, sbase + OFF_YT_RE, idesc(64, 0), true);
+            mma_k64_ts(s_re, e_im, sbase + OFF_YT_IM, idesc(64, 1), true);
+            mma_k64_ts(s_im, e_re, sbase + OFF_YT_IM, idesc(64, 0), true);
+            mma_k64_ts(s_im, e_im, sbase + OFF_YT_RE, idesc(64, 0), true);
+            const uint32_t o_re = tmem + TM_ACC + 64, o_imc = tmem + TM_ACC + 192;
+            mma_k64_ts(o_re, e_re, sbase + OFF_AQ_RE, idesc(64, 0), true);
+            mma_k64_ts(o_re, e_im, sbase + OFF_AQ_IM, idesc(64, 1), true);
+            mma_k64_ts(o_imc, e_im, sbase + OFF_AQ_RE, idesc(64, 0), true);
+            mma_k64_ts(o_imc, e_re, sbase + OFF_AQ_IM, idesc(64, 0), true);
+            mma_commit(&mi.bar_mma);
+        }
+        failed = __syncthreads_or(mbar_wait(&mi.bar_mma, ph_mma) ? 0 : 1);
+        ph_mma ^= 1;
+        if (failed) break;
+        tc_fence_after();
+
+        // ================= outputs: o = Re rho, o_im = -Im rho ==========================================
+        {
+            const int c = quad * 32 + lane;
+            __nv_bfloat16 *dst = half ? p.o_im : p.o;
+            if (dst) {
+                uint32_t r[64];
+                tmem_ld<64>(tlane + TM_ACC + 64 + 128 * half, r);
+                tc_wait_ld();
+                const float sgn = half ? -1.f : 1.f;
+#pragma unroll
+                for (int t = 0; t < 64; ++t)
+                    if (t < len)
+                        dst[(((size_t)b * p.T + t0 + t) * p.H + h) * DV + c] = __float2bfloat16_rn(sgn * __uint_as_float(r[t]));
+            }
+        }
+        tc_fence_before();
+        __syncthreads();
+    }
+
+    if (failed) {
+        if (tid == 0) atomicExch(p.status, 1u);
+        // let copies that are still in flight land before the shared memory goes away
+        if (in_flight_in) mbar_wait(&mi.bar_in, ph_in);
+        if (in_flight_v) mbar_wait(&mi.bar_v, ph_v);
+    } else if (p.S_T) {
+        // final state: closing phase of the last chunk, back to paired rows
+        tc_fence_after();
+        const int c = quad * 32 + lane, j0 = half * 32, last = (n_chunks - 1) & 1;
+        uint32_t sre[32], sim[32];
+        tmem_ld<32>(tlane + TM_S32 + j0, sre);
+        tmem_ld<32>(tlane + TM_S32 + 64 + j0, sim);
+        tc_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const int j = j0 + i;
+            const float cs = mi.closing_cos[last][j], sn = mi.closing_sin[last][j];
+            const float xr = __uint_as_float(sre[i]), xi = __uint_as_float(sim[i]);
+            p.S_T[((size_t)bh * DK + 2 * j) * DV + c] = cs * xr - sn * xi;
+            p.S_T[((size_t)bh * DK + 2 * j + 1) * DV + c] = cs * xi + sn * xr;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem));
+}
+
+// ---- host side --------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = [] {
+        void *f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            f = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(f);
+    }();
+    return fn;
+}
+
+// [B][T][H][inner] tensor, box = 64 tokens of one head.
+bool make_map(CUtensorMap *map, const void *base, CUtensorMapDataType dt, int elem_bytes, int inner, int B, int T, int H)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[4] = {(cuuint64_t)inner, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {(cuuint64_t)inner * elem_bytes, (cuuint64_t)H * inner * elem_bytes,
+                                   (cuuint64_t)T * H * inner * elem_bytes};
+    const cuuint32_t box[4] = {(cuuint32_t)inner, 1, (cuuint32_t)C, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, dt, 4, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool forward_tc_supported(const ForwardArgs &a)
+{
+    return a.dtype == 1 && a.d_k == DK && a.d_v == DV && a.chunk == C;
+}
+
+cudaError_t launch_forward_tc(const ForwardArgs &a, uint32_t *status, cudaStream_t stream, int *launches)
+{
+    CUtensorMap tq, tk, tv, ta, tt;
+    if (!make_map(&tq, a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, DK, a.B, a.T, a.H) ||
+        !make_map(&tk, a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, DK, a.B, a.T, a.H) ||
+        !make_map(&tv, a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, DV, a.B, a.T, a.H) ||
+        !make_map(&ta, a.alpha, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, M, a.B, a.T, a.H) ||
+        !make_map(&tt, a.theta, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, M, a.B, a.T, a.H))
+        return cudaErrorInvalidValue;
+    cudaError_t e = cudaFuncSetAttribute(sfda_forward_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(status, 0, sizeof(uint32_t), stream);
+    if (e != cudaSuccess) return e;
+    Params p;
+    p.beta = a.beta;
+    p.S0 = a.S0;
+    p.o = static_cast<__nv_bfloat16 *>(a.o);
+    p.o_im = static_cast<__nv_bfloat16 *>(a.o_im);
+    p.S_T = a.S_T;
+    p.status = status;
+    p.T = a.T;
+    p.H = a.H;
+    sfda_forward_tc_kernel<<<(unsigned)(a.B * a.H), kThreads, kSmemBytes, stream>>>(tq, tk, tv, ta, tt, p);
+    e = cudaGetLastError();
+    if (e == cudaSuccess && launches) ++*launches;
+    return e;
+}
+
+}  // namespace sfda

@@ -50,6 +50,8 @@ def run_forward(cfg, inp, want_im=True, simt=False, want_state=True):
                           cfg.chunk, ws)
     torch.cuda.synchronize()
     assert sfda.last_launch_count() >= 1
+    if ws_bytes and not simt:
+        assert sfda.sfda_workspace_status(ws) == 0
     return (o.float().cpu().numpy(), None if o_im is None else o_im.float().cpu().numpy(),
             None if S_T is None else S_T.cpu().numpy())
 
@@ -136,6 +138,28 @@ def test_forward_split_sequence_continues_from_state():
     o2, _, S2 = run_forward(cfg, second)
     assert rel_err(np.concatenate([o1, o2], 1), o) < 1e-5
     assert rel_err(S2, S_T) < 1e-5
+
+
+@pytest.mark.parametrize("T,H,s0,alpha", [(64, 1, 0.0, "sigmoid(n(3,1))"), (256, 2, 0.02, "sigmoid(n(3,1))"),
+                                         (200, 3, 0.5, "sigmoid(n(3,1))"), (1, 2, 1.0, "sigmoid(n(3,1))"),
+                                         (130, 2, 1.0, "u(0.5,1)"), (192, 2, 0.3, "u(1.0,1.0)"),
+                                         (192, 2, 0.3, "u(0.3,1)")])
+def test_forward_tensor_core_path(T, H, s0, alpha):
+    """bf16, d_k = d_v = 128, chunk = 64: the tcgen05 path, several chunks, ragged tails, nonzero S0."""
+    cfg = workloads.CONFIGS[1].scaled(name="tc", B=2, T=T, H=H, s0_std=s0, alpha=alpha, seed=40 + T)
+    assert sfda.sfda_workspace_bytes(cfg.B, T, H, 128, 128, 64, 1) > 0          # takes the tensor-core path
+    inp = workloads.forward_inputs(cfg)
+    errs = check_forward(cfg, inp, all_pairs(cfg), TOL["bf16"])
+    print(errs)
+
+
+def test_forward_tensor_core_matches_cuda_core_path():
+    cfg = workloads.CONFIGS[1].scaled(name="tc2", B=1, T=512, H=4, s0_std=0.1, seed=77)
+    inp = workloads.forward_inputs(cfg)
+    a = run_forward(cfg, inp)
+    b = run_forward(cfg, inp, simt=True)
+    for x, y in zip(a, b):
+        assert rel_err(x, y) < TOL["bf16"]
 
 
 @pytest.mark.parametrize("idx", [1, 2])
