@@ -50,21 +50,24 @@ constexpr int OFF_Q = OFF_V + 16384;             // q staging [t][128] bf16
 constexpr int OFF_K = OFF_Q + 16384;             // k staging
 constexpr int OFF_ALPHA = OFF_K + 16384;         // alpha staging [t][64] fp32
 constexpr int OFF_THETA = OFF_ALPHA + 16384;     // theta staging
-constexpr int OFF_SOLVE = OFF_Q;                 // L, X (fp32 complex 64x64) alias the staging buffers
-constexpr int OFF_MISC = OFF_THETA + 16384;
-constexpr int kSmemBytes = OFF_MISC + 16384 + 1024;   // + slack for the 1024-byte alignment
+constexpr int OFF_SOLVE = OFF_Q;                 // L, X (fp32 complex 64 x 64, row stride 68) alias the staging
+constexpr int LS = 68;                           // row stride (floats) of L and X: conflict-free A fragments
+constexpr int TS = 40;                           // row stride of the T scratch: conflict-free B fragments
+constexpr int OFF_MISC = OFF_SOLVE + 4 * 64 * LS * 4;
+constexpr int kSmemBytes = OFF_MISC + 20480 + 1024;   // + slack for the 1024-byte alignment
+static_assert(OFF_MISC >= OFF_THETA + 16384, "solve scratch must cover the staging buffers it aliases");
 
 struct Misc {
-    float part_lg[4][M];
-    uint32_t part_turns[4][M];
+    float part_lg[8][M];
+    uint32_t part_turns[8][M];
     float aC[M];
     float closing_cos[2][M], closing_sin[2][M];
     float beta[C];
-    float Tr[4][16][16], Ti[4][16][16];
+    float Tr[32 * TS], Ti[32 * TS];
     unsigned long long bar_mma, bar_in, bar_v;
     uint32_t tmem_base;
 };
-static_assert(sizeof(Misc) <= 16384, "misc area too small");
+static_assert(sizeof(Misc) <= 20480, "misc area too small");
 
 // ---- tensor memory map (columns) -------------------------------------------------------------------
 constexpr uint32_t TM_S32 = 0;     // state fp32: [Re j | Im j]
@@ -108,6 +111,16 @@ __device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, u
         "r"(c3)
         : "memory");
 }
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap *map, const void *src, int c0, int c1, int c2, int c3)
+{
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(
+                     reinterpret_cast<uint64_t>(map)),
+                 "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -206,11 +219,86 @@ __device__ __forceinline__ int sw_off(int r, int e)
 {
     return (r >> 3) * 1024 + (r & 7) * 128 + ((((e >> 3) ^ r) & 7) << 4) + ((e & 7) << 1);
 }
-// fp32 64x64 scratch matrices of the triangular solve, XOR-swizzled so that one column read by 32 rows
-// and one row read by 32 columns are both conflict-free.
-__device__ __forceinline__ int lx(int r, int k) { return r * 64 + (k ^ (r & 31)); }
+// ---- warp-level tf32 MMA used by the triangular solve ------------------------------------------------
+__device__ __forceinline__ uint32_t to_tf32(float x)
+{
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2])
+{
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+// (cr + i ci) += A[a_row0 .. +15][a_col0 + 8 s ..] * B[b_row0 + 8 s ..][b_col0 .. +7] over k-steps s in [s0, s1),
+// complex fp32 matrices in shared memory (row strides a_ld, b_ld); one 16 x 8 output tile per warp.
+__device__ __forceinline__ void cmma_16x8(float (&cr)[4], float (&ci)[4], const float *Ar, const float *Ai, int a_ld,
+                                          int a_row0, int a_col0, const float *Br, const float *Bi, int b_ld,
+                                          int b_row0, int b_col0, int s0, int s1, int lane)
+{
+    const int g = lane >> 2, tg = lane & 3;
+    for (int s = s0; s < s1; ++s) {
+        const int ao = (a_row0 + g) * a_ld + a_col0 + 8 * s + tg;
+        uint32_t ar[4], ai[4], nai[4], br[2], bi[2];
+        ar[0] = to_tf32(Ar[ao]);
+        ar[1] = to_tf32(Ar[ao + 8 * a_ld]);
+        ar[2] = to_tf32(Ar[ao + 4]);
+        ar[3] = to_tf32(Ar[ao + 8 * a_ld + 4]);
+        ai[0] = to_tf32(Ai[ao]);
+        ai[1] = to_tf32(Ai[ao + 8 * a_ld]);
+        ai[2] = to_tf32(Ai[ao + 4]);
+        ai[3] = to_tf32(Ai[ao + 8 * a_ld + 4]);
+#pragma unroll
+        for (int x = 0; x < 4; ++x) nai[x] = ai[x] ^ 0x80000000u;
+        const int bo = (b_row0 + 8 * s + tg) * b_ld + b_col0 + g;
+        br[0] = to_tf32(Br[bo]);
+        br[1] = to_tf32(Br[bo + 4 * b_ld]);
+        bi[0] = to_tf32(Bi[bo]);
+        bi[1] = to_tf32(Bi[bo + 4 * b_ld]);
+        mma_tf32(cr, ar, br);
+        mma_tf32(cr, nai, bi);
+        mma_tf32(ci, ar, bi);
+        mma_tf32(ci, ai, br);
+    }
+}
+// Store a 16 x 8 accumulator tile (times `scale`) at rows row0.., columns col0.. of a complex fp32 matrix.
+__device__ __forceinline__ void store_tile(const float (&cr)[4], const float (&ci)[4], float scale, float *Dr, float *Di,
+                                           int ld, int row0, int col0, int lane)
+{
+    const int g = lane >> 2, tg = lane & 3;
+    const int o = (row0 + g) * ld + col0 + 2 * tg;
+    Dr[o] = scale * cr[0];
+    Dr[o + 1] = scale * cr[1];
+    Dr[o + 8 * ld] = scale * cr[2];
+    Dr[o + 8 * ld + 1] = scale * cr[3];
+    Di[o] = scale * ci[0];
+    Di[o + 1] = scale * ci[1];
+    Di[o + 8 * ld] = scale * ci[2];
+    Di[o + 8 * ld + 1] = scale * ci[3];
+}
+
+// Optional per-phase cycle counters (development builds only, -DSFDA_TC_TIMING).
+#ifdef SFDA_TC_TIMING
+#define SFDA_MARK(i)                                                          \
+    do {                                                                      \
+        if (tid == 0 && bh == 0 && p.timing) {                                \
+            const long long now_ = clock64();                                 \
+            p.timing[i] += now_ - mark_;                                      \
+            mark_ = now_;                                                     \
+        }                                                                     \
+    } while (0)
+#else
+#define SFDA_MARK(i) \
+    do {             \
+    } while (0)
+#endif
 
 struct Params {
+#ifdef SFDA_TC_TIMING
+    long long *timing;
+#endif
     const float *beta, *S0;
     __nv_bfloat16 *o, *o_im;
     float *S_T;
@@ -222,13 +310,14 @@ struct Params {
 __global__ void __launch_bounds__(kThreads, 1)
 sfda_forward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_alpha,
-                       const __grid_constant__ CUtensorMap tm_theta, const Params p)
+                       const __grid_constant__ CUtensorMap tm_theta, const __grid_constant__ CUtensorMap tm_o,
+                       const __grid_constant__ CUtensorMap tm_oim, const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     Misc &mi = *reinterpret_cast<Misc *>(smem + OFF_MISC);
     float *Lr = reinterpret_cast<float *>(smem + OFF_SOLVE);
-    float *Li = Lr + 4096, *Xr = Li + 4096, *Xi = Xr + 4096;
+    float *Li = Lr + 64 * LS, *Xr = Li + 64 * LS, *Xi = Xr + 64 * LS;
     const uint32_t sbase = smem_u32(smem);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -262,6 +351,9 @@ sfda_forward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         tma_load_4d(smem + OFF_V, &tm_v, &mi.bar_v, 0, h, 0, b);
     }
 
+#ifdef SFDA_TC_TIMING
+    long long mark_ = clock64();
+#endif
     uint32_t ph_mma = 0, ph_in = 0, ph_v = 0;
     bool in_flight_in = true, in_flight_v = true;
     int failed = 0;
@@ -272,97 +364,119 @@ sfda_forward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const int cur = ci & 1;
 
         // ================= prep: cumulative phase-decay and the operand tiles =======================
+        if (tid == 0) tma_store_wait_read();   // the previous chunk's output store still reads the WQ tiles
         failed = __syncthreads_or(mbar_wait(&mi.bar_in, ph_in) ? 0 : 1);
         ph_in ^= 1;
         in_flight_in = false;
         if (failed) break;
+        SFDA_MARK(0);
         {
-            const int j = tid & 63, tq = tid >> 6;
-            const float *s_alpha = reinterpret_cast<const float *>(smem + OFF_ALPHA);
-            const float *s_theta = reinterpret_cast<const float *>(smem + OFF_THETA);
-            float lg[16];
-            uint32_t tu[16];
-            float acc = 0.f;
-            uint32_t tacc = 0u;
+            // thread = (channel pair jp: channels 2jp, 2jp+1 ; token octet tq = warp)
+            const int jp = tid & 31, tq = tid >> 5;
+            const float2 *s_alpha = reinterpret_cast<const float2 *>(smem + OFF_ALPHA);
+            const float2 *s_theta = reinterpret_cast<const float2 *>(smem + OFF_THETA);
+            float lg0[8], lg1[8];
+            uint32_t tu0[8], tu1[8];
+            float acc0 = 0.f, acc1 = 0.f;
+            uint32_t tacc0 = 0u, tacc1 = 0u;
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int t = tq * 16 + i;
+            for (int i = 0; i < 8; ++i) {
+                const int t = tq * 8 + i;
                 if (t < len) {
-                    acc += fmaxf(__log2f(s_alpha[t * M + j]), -43.28f);   // floor e^-30, as in log_decay
-                    tacc += phase_to_turns(s_theta[t * M + j]);
+                    const float2 al = s_alpha[t * 32 + jp], th = s_theta[t * 32 + jp];
+                    acc0 += fmaxf(__log2f(al.x), -43.28f);   // floor e^-30, as in log_decay
+                    acc1 += fmaxf(__log2f(al.y), -43.28f);
+                    tacc0 += phase_to_turns(th.x);
+                    tacc1 += phase_to_turns(th.y);
                 }
-                lg[i] = acc;
-                tu[i] = tacc;
+                lg0[i] = acc0; lg1[i] = acc1;
+                tu0[i] = tacc0; tu1[i] = tacc1;
             }
-            mi.part_lg[tq][j] = acc;
-            mi.part_turns[tq][j] = tacc;
+            mi.part_lg[tq][2 * jp] = acc0;
+            mi.part_lg[tq][2 * jp + 1] = acc1;
+            mi.part_turns[tq][2 * jp] = tacc0;
+            mi.part_turns[tq][2 * jp + 1] = tacc1;
             if (tid < C) mi.beta[tid] = tid < len ? p.beta[((size_t)b * p.T + t0 + tid) * p.H + h] : 0.f;
             __syncthreads();
-            float base = 0.f, total = 0.f;
-            uint32_t tbase = 0u, ttotal = 0u;
+            float base0 = 0.f, base1 = 0.f, tot0 = 0.f, tot1 = 0.f;
+            uint32_t tb0 = 0u, tb1 = 0u, tt0 = 0u, tt1 = 0u;
 #pragma unroll
-            for (int g = 0; g < 4; ++g) {
-                const float pl = mi.part_lg[g][j];
-                const uint32_t pt = mi.part_turns[g][j];
-                if (g < tq) { base += pl; tbase += pt; }
-                total += pl;
-                ttotal += pt;
+            for (int g = 0; g < 8; ++g) {
+                const float2 pl = *reinterpret_cast<const float2 *>(&mi.part_lg[g][2 * jp]);
+                const uint2 pt = *reinterpret_cast<const uint2 *>(&mi.part_turns[g][2 * jp]);
+                if (g < tq) { base0 += pl.x; base1 += pl.y; tb0 += pt.x; tb1 += pt.y; }
+                tot0 += pl.x; tot1 += pl.y; tt0 += pt.x; tt1 += pt.y;
             }
             if (tq == 0) {
-                mi.aC[j] = exp2f(total);
                 float cs, sn;
-                const float ang = (float)(int32_t)ttotal * 0x1.921fb6p-30f;   // turns * 2 pi / 2^32
-                __sincosf(ang, &sn, &cs);
-                mi.closing_cos[cur][j] = cs;
-                mi.closing_sin[cur][j] = sn;
+                mi.aC[2 * jp] = exp2f(tot0);
+                mi.aC[2 * jp + 1] = exp2f(tot1);
+                __sincosf((float)(int32_t)tt0 * 0x1.921fb6p-30f, &sn, &cs);   // turns * 2 pi / 2^32
+                mi.closing_cos[cur][2 * jp] = cs;
+                mi.closing_sin[cur][2 * jp] = sn;
+                __sincosf((float)(int32_t)tt1 * 0x1.921fb6p-30f, &sn, &cs);
+                mi.closing_cos[cur][2 * jp + 1] = cs;
+                mi.closing_sin[cur][2 * jp + 1] = sn;
             }
-            const uint32_t *s_q = reinterpret_cast<const uint32_t *>(smem + OFF_Q);
-            const uint32_t *s_k = reinterpret_cast<const uint32_t *>(smem + OFF_K);
-            uint32_t ytr[8], yti[8];
+            const uint2 *s_q = reinterpret_cast<const uint2 *>(smem + OFF_Q);
+            const uint2 *s_k = reinterpret_cast<const uint2 *>(smem + OFF_K);
+            uint32_t y0r[4], y0i[4], y1r[4], y1i[4];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int t = tq * 16 + i;
-                const float l2 = base + lg[i];
-                const float a = exp2f(l2);
-                const float ainv = exp2f(fminf(-l2, 115.4f));                 // 1/a_t, capped at e^80
-                const float ay = exp2f(total - l2);                           // a_C / a_t <= 1
-                float cs, sn;
-                __sincosf((float)(int32_t)(tbase + tu[i]) * 0x1.921fb6p-30f, &sn, &cs);
-                const uint32_t kw = s_k[t * 64 + j], qw = s_q[t * 64 + j];
-                const float kr = __uint_as_float(kw << 16), ki = __uint_as_float(kw & 0xffff0000u);
-                const float qr = __uint_as_float(qw << 16), qi = __uint_as_float(qw & 0xffff0000u);
-                const float kpr = kr * cs + ki * sn, kpi = ki * cs - kr * sn;   // e^{-i phi} k
-                const float qpr = qr * cs + qi * sn, qpi = qi * cs - qr * sn;
-                const int o1 = sw_off(t, j);
-                *reinterpret_cast<__nv_bfloat16 *>(smem + OFF_WQ_RE + o1) = __float2bfloat16_rn(a * kpr);
-                *reinterpret_cast<__nv_bfloat16 *>(smem + OFF_WQ_IM + o1) = __float2bfloat16_rn(a * kpi);
-                *reinterpret_cast<__nv_bfloat16 *>(smem + OFF_WQ_RE + kTile + o1) = __float2bfloat16_rn(a * qpr);
-                *reinterpret_cast<__nv_bfloat16 *>(smem + OFF_WQ_IM + kTile + o1) = __float2bfloat16_rn(a * qpi);
-                *reinterpret_cast<__nv_bfloat16 *>(smem + OFF_KC_RE + o1) = __float2bfloat16_rn(ainv * kpr);
-                *reinterpret_cast<__nv_bfloat16 *>(smem + OFF_KC_IM + o1) = __float2bfloat16_rn(ainv * kpi);
-                const float yr = ay * kpr, yi = ay * kpi;
+            for (int i = 0; i < 8; ++i) {
+                const int t = tq * 8 + i;
+                const uint2 kw = s_k[t * 32 + jp], qw = s_q[t * 32 + jp];
+                float wr[2], wi[2], cr_[2], ci_[2], qr_[2], qi_[2], yr[2], yi[2];
+#pragma unroll
+                for (int x = 0; x < 2; ++x) {
+                    const float l2 = x ? base1 + lg1[i] : base0 + lg0[i];
+                    const float tot = x ? tot1 : tot0;
+                    const uint32_t tu = x ? tb1 + tu1[i] : tb0 + tu0[i];
+                    const uint32_t kx = x ? kw.y : kw.x, qx = x ? qw.y : qw.x;
+                    const float a = exp2f(l2);
+                    const float ainv = exp2f(fminf(-l2, 115.4f));                 // 1/a_t, capped at e^80
+                    const float ay = exp2f(tot - l2);                             // a_C / a_t <= 1
+                    float cs, sn;
+                    __sincosf((float)(int32_t)tu * 0x1.921fb6p-30f, &sn, &cs);
+                    const float kr = __uint_as_float(kx << 16), ki = __uint_as_float(kx & 0xffff0000u);
+                    const float qr = __uint_as_float(qx << 16), qi = __uint_as_float(qx & 0xffff0000u);
+                    const float kpr = kr * cs + ki * sn, kpi = ki * cs - kr * sn;   // e^{-i phi} k
+                    const float qpr = qr * cs + qi * sn, qpi = qi * cs - qr * sn;
+                    wr[x] = a * kpr; wi[x] = a * kpi;
+                    qr_[x] = a * qpr; qi_[x] = a * qpi;
+                    cr_[x] = ainv * kpr; ci_[x] = ainv * kpi;
+                    yr[x] = ay * kpr; yi[x] = ay * kpi;
+                }
+                const int o1 = sw_off(t, 2 * jp);
+                *reinterpret_cast<uint32_t *>(smem + OFF_WQ_RE + o1) = pack_bf16(wr[0], wr[1]);
+                *reinterpret_cast<uint32_t *>(smem + OFF_WQ_IM + o1) = pack_bf16(wi[0], wi[1]);
+                *reinterpret_cast<uint32_t *>(smem + OFF_WQ_RE + kTile + o1) = pack_bf16(qr_[0], qr_[1]);
+                *reinterpret_cast<uint32_t *>(smem + OFF_WQ_IM + kTile + o1) = pack_bf16(qi_[0], qi_[1]);
+                *reinterpret_cast<uint32_t *>(smem + OFF_KC_RE + o1) = pack_bf16(cr_[0], cr_[1]);
+                *reinterpret_cast<uint32_t *>(smem + OFF_KC_IM + o1) = pack_bf16(ci_[0], ci_[1]);
+                const uint32_t h0r = __bfloat16_as_ushort(__float2bfloat16_rn(yr[0]));
+                const uint32_t h0i = __bfloat16_as_ushort(__float2bfloat16_rn(yi[0]));
+                const uint32_t h1r = __bfloat16_as_ushort(__float2bfloat16_rn(yr[1]));
+                const uint32_t h1i = __bfloat16_as_ushort(__float2bfloat16_rn(yi[1]));
                 if (i & 1) {
-                    ytr[i >> 1] |= (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(yr)) << 16;
-                    yti[i >> 1] |= (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(yi)) << 16;
+                    y0r[i >> 1] |= h0r << 16; y0i[i >> 1] |= h0i << 16;
+                    y1r[i >> 1] |= h1r << 16; y1i[i >> 1] |= h1i << 16;
                 } else {
-                    ytr[i >> 1] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(yr));
-                    yti[i >> 1] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(yi));
+                    y0r[i >> 1] = h0r; y0i[i >> 1] = h0i;
+                    y1r[i >> 1] = h1r; y1i[i >> 1] = h1i;
                 }
             }
-            // Y'^T row j, tokens 16 tq .. 16 tq + 15: two 16-byte chunks per half.
-#pragma unroll
-            for (int cidx = 0; cidx < 2; ++cidx) {
-                const int off = sw_off(j, tq * 16 + cidx * 8);
-                *reinterpret_cast<uint4 *>(smem + OFF_YT_RE + off) =
-                    make_uint4(ytr[4 * cidx], ytr[4 * cidx + 1], ytr[4 * cidx + 2], ytr[4 * cidx + 3]);
-                *reinterpret_cast<uint4 *>(smem + OFF_YT_IM + off) =
-                    make_uint4(yti[4 * cidx], yti[4 * cidx + 1], yti[4 * cidx + 2], yti[4 * cidx + 3]);
-            }
+            // Y'^T rows 2jp and 2jp+1, tokens 8 tq .. 8 tq + 7: one 16-byte chunk per row and half.
+            const int oa = sw_off(2 * jp, tq * 8), ob = sw_off(2 * jp + 1, tq * 8);
+            *reinterpret_cast<uint4 *>(smem + OFF_YT_RE + oa) = make_uint4(y0r[0], y0r[1], y0r[2], y0r[3]);
+            *reinterpret_cast<uint4 *>(smem + OFF_YT_IM + oa) = make_uint4(y0i[0], y0i[1], y0i[2], y0i[3]);
+            *reinterpret_cast<uint4 *>(smem + OFF_YT_RE + ob) = make_uint4(y1r[0], y1r[1], y1r[2], y1r[3]);
+            *reinterpret_cast<uint4 *>(smem + OFF_YT_IM + ob) = make_uint4(y1i[0], y1i[1], y1i[2], y1i[3]);
         }
         fence_async_smem();
         tc_fence_before();
         __syncthreads();
 
+        SFDA_MARK(1);
         // ================= Gram blocks Kt (rows 0..63) and Aq (rows 64..127) ==========================
         if (tid == 0) {
             tc_fence_after();
@@ -377,6 +491,7 @@ sfda_forward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         ph_mma ^= 1;
         if (failed) break;
         tc_fence_after();
+        SFDA_MARK(2);
         {
             uint32_t r[64];
             tmem_ld<64>(tlane + TM_ACC + 64 * half, r);
@@ -385,9 +500,13 @@ sfda_forward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             if (row < 64) {                       // L = D_beta Kt, strictly lower
                 const int t = row;
                 const float bt = mi.beta[t];
-                float *dst = half ? Li : Lr;
+                float4 *dst = reinterpret_cast<float4 *>((half ? Li : Lr) + t * LS);
 #pragma unroll
-                for (int i = 0; i < 64; ++i) dst[lx(t, i)] = i < t ? bt * __uint_as_float(r[i]) : 0.f;
+                for (int i = 0; i < 64; i += 4)
+                    dst[i >> 2] = make_float4(i < t ? bt * __uint_as_float(r[i]) : 0.f,
+                                              i + 1 < t ? bt * __uint_as_float(r[i + 1]) : 0.f,
+                                              i + 2 < t ? bt * __uint_as_float(r[i + 2]) : 0.f,
+                                              i + 3 < t ? bt * __uint_as_float(r[i + 3]) : 0.f);
             } else {                              // Aq, lower incl. diagonal, as a bf16 operand tile
                 const int t = row - 64;
                 uint8_t *tile = smem + (half ? OFF_AQ_IM : OFF_AQ_RE);
@@ -407,63 +526,59 @@ sfda_forward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         tc_fence_before();
         __syncthreads();
 
-        // ================= X = (I + L)^{-1} in fp32 by 16x16 blocks; M_beta = X D_beta ================
-        if (tid < 64) {
-            const int blk = tid >> 4, c = tid & 15, o = 16 * blk;
+        SFDA_MARK(3);
+        // ================= X = (I + L)^{-1}: 16x16 diagonal blocks by substitution, merges on mma.sync ===
+        if (warp < 4 && lane < 16) {                  // warp b inverts diagonal block b, lane = column
+            const int o = 16 * warp, c = lane;
             float xr[16], xi[16];
 #pragma unroll
             for (int r = 0; r < 16; ++r) {
                 float ar = r == c ? 1.f : 0.f, ai = 0.f;
 #pragma unroll
                 for (int i = 0; i < 15; ++i) {
-                    if (i < r && i >= c) {
-                        const float lr_ = Lr[lx(o + r, o + i)], li_ = Li[lx(o + r, o + i)];
-                        ar -= lr_ * xr[i] - li_ * xi[i];
-                        ai -= lr_ * xi[i] + li_ * xr[i];
+                    if (i < r) {
+                        const float lr_ = Lr[(o + r) * LS + o + i], li_ = Li[(o + r) * LS + o + i];
+                        const float vr = i >= c ? xr[i] : 0.f, vi = i >= c ? xi[i] : 0.f;
+                        ar -= lr_ * vr - li_ * vi;
+                        ai -= lr_ * vi + li_ * vr;
                     }
                 }
                 xr[r] = r >= c ? ar : 0.f;
                 xi[r] = r >= c ? ai : 0.f;
-                Xr[lx(o + r, o + c)] = xr[r];
-                Xi[lx(o + r, o + c)] = xi[r];
+                Xr[(o + r) * LS + o + c] = xr[r];
+                Xi[(o + r) * LS + o + c] = xi[r];
             }
         }
         __syncthreads();
-        {
-            const int r = tid >> 4, c = tid & 15;
-            for (int d = 1; d < 4; ++d) {
-                for (int rb = d; rb < 4; ++rb) {      // T_rb = sum_kb L[rb][kb] X[kb][cb]
-                    const int cb = rb - d;
-                    float ar = 0.f, ai = 0.f;
-                    for (int kb = cb; kb < rb; ++kb) {
+        if (warp < 2) {                               // level 1: X[b1][b0] = -X[b1][b1] (L[b1][b0] X[b0][b0])
+            const int r0 = 32 * warp + 16, c0 = 32 * warp;
+            float *tr = mi.Tr + 16 * warp * TS, *ti = mi.Ti + 16 * warp * TS;
 #pragma unroll
-                        for (int k = 0; k < 16; ++k) {
-                            const float lr_ = Lr[lx(16 * rb + r, 16 * kb + k)], li_ = Li[lx(16 * rb + r, 16 * kb + k)];
-                            const float vr = Xr[lx(16 * kb + k, 16 * cb + c)], vi = Xi[lx(16 * kb + k, 16 * cb + c)];
-                            ar += lr_ * vr - li_ * vi;
-                            ai += lr_ * vi + li_ * vr;
-                        }
-                    }
-                    mi.Tr[rb][r][c] = ar;
-                    mi.Ti[rb][r][c] = ai;
-                }
-                __syncthreads();
-                for (int rb = d; rb < 4; ++rb) {      // X[rb][cb] = -X[rb][rb] T_rb
-                    const int cb = rb - d;
-                    float ar = 0.f, ai = 0.f;
+            for (int nt = 0; nt < 2; ++nt) {
+                float cr[4] = {0.f, 0.f, 0.f, 0.f}, ci[4] = {0.f, 0.f, 0.f, 0.f};
+                cmma_16x8(cr, ci, Lr, Li, LS, r0, c0, Xr, Xi, LS, c0, c0 + 8 * nt, nt, 2, lane);
+                store_tile(cr, ci, 1.f, tr, ti, TS, 0, 8 * nt, lane);
+            }
+            __syncwarp();
 #pragma unroll
-                    for (int k = 0; k < 16; ++k) {
-                        const float vr = Xr[lx(16 * rb + r, 16 * rb + k)], vi = Xi[lx(16 * rb + r, 16 * rb + k)];
-                        const float tr = mi.Tr[rb][k][c], ti = mi.Ti[rb][k][c];
-                        ar -= vr * tr - vi * ti;
-                        ai -= vr * ti + vi * tr;
-                    }
-                    Xr[lx(16 * rb + r, 16 * cb + c)] = ar;
-                    Xi[lx(16 * rb + r, 16 * cb + c)] = ai;
-                }
-                __syncthreads();
+            for (int nt = 0; nt < 2; ++nt) {
+                float cr[4] = {0.f, 0.f, 0.f, 0.f}, ci[4] = {0.f, 0.f, 0.f, 0.f};
+                cmma_16x8(cr, ci, Xr, Xi, LS, r0, r0, tr, ti, TS, 0, 8 * nt, 0, 2, lane);
+                store_tile(cr, ci, -1.f, Xr, Xi, LS, r0, c0 + 8 * nt, lane);
             }
         }
+        __syncthreads();
+        {                                             // level 2: X[BL] = -X[BR] (L[BL] X[TL]); one tile per warp
+            const int mt = warp >> 2, nt = warp & 3;
+            float cr[4] = {0.f, 0.f, 0.f, 0.f}, ci[4] = {0.f, 0.f, 0.f, 0.f};
+            cmma_16x8(cr, ci, Lr, Li, LS, 32 + 16 * mt, 0, Xr, Xi, LS, 0, 8 * nt, nt, 4, lane);
+            store_tile(cr, ci, 1.f, mi.Tr, mi.Ti, TS, 16 * mt, 8 * nt, lane);
+            __syncthreads();
+            float dr[4] = {0.f, 0.f, 0.f, 0.f}, di[4] = {0.f, 0.f, 0.f, 0.f};
+            cmma_16x8(dr, di, Xr, Xi, LS, 32 + 16 * mt, 32, mi.Tr, mi.Ti, TS, 0, 8 * nt, 0, 2 * mt + 2, lane);
+            store_tile(dr, di, -1.f, Xr, Xi, LS, 32 + 16 * mt, 8 * nt, lane);
+        }
+        __syncthreads();
         {
             const int t = tid >> 2, part = tid & 3;     // row t, columns 16 part .. 16 part + 15
 #pragma unroll
@@ -474,8 +589,8 @@ sfda_forward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     const int i0 = part * 16 + cidx * 8 + 2 * x;
                     const float b0 = mi.beta[i0], b1 = mi.beta[i0 + 1];
                     const bool in0 = i0 <= t, in1 = i0 + 1 <= t;
-                    wr[x] = pack_bf16(in0 ? Xr[lx(t, i0)] * b0 : 0.f, in1 ? Xr[lx(t, i0 + 1)] * b1 : 0.f);
-                    wi[x] = pack_bf16(in0 ? Xi[lx(t, i0)] * b0 : 0.f, in1 ? Xi[lx(t, i0 + 1)] * b1 : 0.f);
+                    wr[x] = pack_bf16(in0 ? Xr[t * LS + i0] * b0 : 0.f, in1 ? Xr[t * LS + i0 + 1] * b1 : 0.f);
+                    wi[x] = pack_bf16(in0 ? Xi[t * LS + i0] * b0 : 0.f, in1 ? Xi[t * LS + i0 + 1] * b1 : 0.f);
                 }
                 const int off = sw_off(t, part * 16 + cidx * 8);
                 *reinterpret_cast<uint4 *>(smem + OFF_MB_RE + off) = make_uint4(wr[0], wr[1], wr[2], wr[3]);
@@ -483,6 +598,7 @@ sfda_forward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             }
         }
 
+        SFDA_MARK(4);
         // ================= state pass: S16 <- bf16(S_start), S32 <- a_C * S_start ======================
         {
             const int c = quad * 32 + lane;        // value channel = TMEM lane
@@ -528,6 +644,7 @@ sfda_forward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         tc_fence_before();
         __syncthreads();
 
+        SFDA_MARK(5);
         // ================= D1 = W^* S_0 and rho_1 = Qt^* S_0 (N = 128: W rows then Qt rows) ==========
         if (tid == 0) {
             tc_fence_after();
@@ -558,6 +675,7 @@ sfda_forward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         if (failed) break;
         tc_fence_after();
 
+        SFDA_MARK(6);
         // ================= R = V - D1 -> bf16 A operand ================================================
         {
             const int c = quad * 32 + lane;
@@ -580,6 +698,7 @@ sfda_forward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         tc_fence_before();
         __syncthreads();
 
+        SFDA_MARK(7);
         // ================= E = M_beta R ================================================================
         if (tid == 0) {
             tc_fence_after();
@@ -612,6 +731,7 @@ sfda_forward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         tc_fence_before();
         __syncthreads();
 
+        SFDA_MARK(8);
         // ================= S += E^T Y'  and  rho += Aq E ================================================
         if (tid == 0) {
             tc_fence_after();
@@ -633,23 +753,30 @@ sfda_forward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         if (failed) break;
         tc_fence_after();
 
-        // ================= outputs: o = Re rho, o_im = -Im rho ==========================================
+        SFDA_MARK(9);
+        // ================= outputs: o = Re rho, o_im = -Im rho, staged in the (now dead) WQ tiles =======
         {
             const int c = quad * 32 + lane;
-            __nv_bfloat16 *dst = half ? p.o_im : p.o;
-            if (dst) {
+            const bool want = half ? p.o_im != nullptr : true;
+            if (want) {
                 uint32_t r[64];
                 tmem_ld<64>(tlane + TM_ACC + 64 + 128 * half, r);
                 tc_wait_ld();
+                __nv_bfloat16 *stage = reinterpret_cast<__nv_bfloat16 *>(smem + (half ? OFF_WQ_IM : OFF_WQ_RE));
                 const float sgn = half ? -1.f : 1.f;
 #pragma unroll
-                for (int t = 0; t < 64; ++t)
-                    if (t < len)
-                        dst[(((size_t)b * p.T + t0 + t) * p.H + h) * DV + c] = __float2bfloat16_rn(sgn * __uint_as_float(r[t]));
+                for (int t = 0; t < 64; ++t) stage[t * DV + c] = __float2bfloat16_rn(sgn * __uint_as_float(r[t]));
             }
         }
+        fence_async_smem();
         tc_fence_before();
         __syncthreads();
+        if (tid == 0) {
+            tma_store_4d(&tm_o, smem + OFF_WQ_RE, 0, h, t0, b);
+            if (p.o_im) tma_store_4d(&tm_oim, smem + OFF_WQ_IM, 0, h, t0, b);
+            tma_store_commit();
+        }
+        SFDA_MARK(10);
     }
 
     if (failed) {
@@ -674,12 +801,17 @@ sfda_forward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             p.S_T[((size_t)bh * DK + 2 * j + 1) * DV + c] = cs * xi + sn * xr;
         }
     }
+    if (tid == 0) tma_store_wait_all();
     tc_fence_before();
     __syncthreads();
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem));
 }
 
 // ---- host side --------------------------------------------------------------------------------------
+#ifdef SFDA_TC_TIMING
+long long *g_timing = nullptr;
+#endif
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -721,18 +853,23 @@ bool forward_tc_supported(const ForwardArgs &a)
 
 cudaError_t launch_forward_tc(const ForwardArgs &a, uint32_t *status, cudaStream_t stream, int *launches)
 {
-    CUtensorMap tq, tk, tv, ta, tt;
+    CUtensorMap tq, tk, tv, ta, tt, to, toi;
     if (!make_map(&tq, a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, DK, a.B, a.T, a.H) ||
         !make_map(&tk, a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, DK, a.B, a.T, a.H) ||
         !make_map(&tv, a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, DV, a.B, a.T, a.H) ||
         !make_map(&ta, a.alpha, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, M, a.B, a.T, a.H) ||
-        !make_map(&tt, a.theta, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, M, a.B, a.T, a.H))
+        !make_map(&tt, a.theta, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, M, a.B, a.T, a.H) ||
+        !make_map(&to, a.o, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, DV, a.B, a.T, a.H) ||
+        !make_map(&toi, a.o_im ? a.o_im : a.o, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, DV, a.B, a.T, a.H))
         return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(sfda_forward_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     e = cudaMemsetAsync(status, 0, sizeof(uint32_t), stream);
     if (e != cudaSuccess) return e;
     Params p;
+#ifdef SFDA_TC_TIMING
+    p.timing = g_timing;
+#endif
     p.beta = a.beta;
     p.S0 = a.S0;
     p.o = static_cast<__nv_bfloat16 *>(a.o);
@@ -741,7 +878,7 @@ cudaError_t launch_forward_tc(const ForwardArgs &a, uint32_t *status, cudaStream
     p.status = status;
     p.T = a.T;
     p.H = a.H;
-    sfda_forward_tc_kernel<<<(unsigned)(a.B * a.H), kThreads, kSmemBytes, stream>>>(tq, tk, tv, ta, tt, p);
+    sfda_forward_tc_kernel<<<(unsigned)(a.B * a.H), kThreads, kSmemBytes, stream>>>(tq, tk, tv, ta, tt, to, toi, p);
     e = cudaGetLastError();
     if (e == cudaSuccess && launches) ++*launches;
     return e;
