@@ -111,7 +111,7 @@ int sfda_forward(const void *q, const void *k, const void *v, const float *alpha
     const sfda::ForwardArgs a = pack(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
     const cudaError_t e =
         sfda::forward_tc_supported(a)
-            ? sfda::launch_forward_tc(a, static_cast<uint32_t *>(workspace), static_cast<cudaStream_t>(stream),
+            ? sfda::launch_forward_ws(a, static_cast<uint32_t *>(workspace), static_cast<cudaStream_t>(stream),
                                       &g_last_launches)
             : sfda::launch_forward_simt(a, static_cast<cudaStream_t>(stream), &g_last_launches);
     return e == cudaSuccess ? SFDA_OK : SFDA_ERR_CUDA;

@@ -25,9 +25,12 @@
 
 #include "sfda_common.cuh"
 #include "sfda_internal.h"
+#include "sfda_tc_ptx.cuh"
 
 namespace sfda {
 namespace {
+
+using namespace tc;
 
 constexpr int C = 64;         // chunk
 constexpr int DK = 128, DV = 128, M = 64;
@@ -74,210 +77,6 @@ constexpr uint32_t TM_S32 = 0;     // state fp32: [Re j | Im j]
 constexpr uint32_t TM_S16 = 128;   // bf16 copy of the chunk-start state (A operand), 64 packed columns
 constexpr uint32_t TM_X16 = 192;   // bf16 R, then E (A operand)
 constexpr uint32_t TM_ACC = 256;   // [D1/E re | rho re | D1/E im | rho im], 64 columns each; Gram uses 0..127
-
-constexpr uint32_t kSpinLimit = 1u << 22;
-
-// ---- small PTX wrappers ---------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(unsigned long long *bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-// Bounded wait: returns false when the phase did not complete within the spin limit.
-__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, uint32_t parity)
-{
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
-        uint32_t ok;
-        asm volatile(
-            "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
-            : "=r"(ok)
-            : "r"(smem_u32(bar)), "r"(parity)
-            : "memory");
-        if (ok) return true;
-    }
-    return false;
-}
-__device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, unsigned long long *bar, int c0, int c1,
-                                            int c2, int c3)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2),
-        "r"(c3)
-        : "memory");
-}
-__device__ __forceinline__ void tma_store_4d(const CUtensorMap *map, const void *src, int c0, int c1, int c2, int c3)
-{
-    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(
-                     reinterpret_cast<uint64_t>(map)),
-                 "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-                 : "memory");
-}
-__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-// K-major, 128-byte-swizzled operand tile: 8-row atoms of 1024 B (stride-dimension offset 1024).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)1 << 16;
-    d |= (uint64_t)(1024 >> 4) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
-// kind::f16 instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, M = 128.
-__device__ __forceinline__ constexpr uint32_t idesc(int N, int neg_b)
-{
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)neg_b << 14) | ((uint32_t)(N >> 3) << 17) |
-           ((uint32_t)(128 >> 4) << 24);
-}
-__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t id, uint32_t acc)
-{
-    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
-                 ::"r"(d), "l"(a), "l"(b), "r"(id), "r"(acc)
-                 : "memory");
-}
-__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t id, uint32_t acc)
-{
-    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
-                 ::"r"(d), "r"(a), "l"(b), "r"(id), "r"(acc)
-                 : "memory");
-}
-__device__ __forceinline__ void mma_commit(unsigned long long *bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-                 : "memory");
-}
-// K = 64 (one swizzle span) product: four K = 16 instructions. A from shared memory / from TMEM.
-__device__ __forceinline__ void mma_k64_ss(uint32_t d, uint32_t a_saddr, uint32_t b_saddr, uint32_t id, bool acc)
-{
-#pragma unroll
-    for (int ks = 0; ks < 4; ++ks)
-        mma_ss(d, smem_desc(a_saddr + 32 * ks), smem_desc(b_saddr + 32 * ks), id, (acc || ks > 0) ? 1u : 0u);
-}
-__device__ __forceinline__ void mma_k64_ts(uint32_t d, uint32_t a_tmem, uint32_t b_saddr, uint32_t id, bool acc)
-{
-#pragma unroll
-    for (int ks = 0; ks < 4; ++ks) mma_ts(d, a_tmem + 8 * ks, smem_desc(b_saddr + 32 * ks), id, (acc || ks > 0) ? 1u : 0u);
-}
-
-#define SFDA_R32(r, o) \
-    "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), "=r"(r[o + 6]), \
-    "=r"(r[o + 7]), "=r"(r[o + 8]), "=r"(r[o + 9]), "=r"(r[o + 10]), "=r"(r[o + 11]), "=r"(r[o + 12]),               \
-    "=r"(r[o + 13]), "=r"(r[o + 14]), "=r"(r[o + 15])
-#define SFDA_W32(r, o) \
-    "r"(r[o + 0]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]), "r"(r[o + 6]), \
-    "r"(r[o + 7]), "r"(r[o + 8]), "r"(r[o + 9]), "r"(r[o + 10]), "r"(r[o + 11]), "r"(r[o + 12]), "r"(r[o + 13]), \
-    "r"(r[o + 14]), "r"(r[o + 15])
-
-// 16 consecutive 32-bit columns of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t *r)
-{
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-                 : SFDA_R32(r, 0)
-                 : "r"(addr));
-}
-__device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t *r)
-{
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
-                 ::"r"(addr), SFDA_W32(r, 0)
-                 : "memory");
-}
-template <int N>
-__device__ __forceinline__ void tmem_ld(uint32_t addr, uint32_t *r)
-{
-#pragma unroll
-    for (int i = 0; i < N; i += 16) tmem_ld16(addr + i, r + i);
-}
-template <int N>
-__device__ __forceinline__ void tmem_st(uint32_t addr, const uint32_t *r)
-{
-#pragma unroll
-    for (int i = 0; i < N; i += 16) tmem_st16(addr + i, r + i);
-}
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
-{
-    return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) |
-           ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
-}
-// Byte offset of element (row r, k-element e < 64) in a K-major 128B-swizzled tile.
-__device__ __forceinline__ int sw_off(int r, int e)
-{
-    return (r >> 3) * 1024 + (r & 7) * 128 + ((((e >> 3) ^ r) & 7) << 4) + ((e & 7) << 1);
-}
-// ---- warp-level tf32 MMA used by the triangular solve ------------------------------------------------
-__device__ __forceinline__ uint32_t to_tf32(float x)
-{
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return r;
-}
-__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2])
-{
-    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
-}
-// (cr + i ci) += A[a_row0 .. +15][a_col0 + 8 s ..] * B[b_row0 + 8 s ..][b_col0 .. +7] over k-steps s in [s0, s1),
-// complex fp32 matrices in shared memory (row strides a_ld, b_ld); one 16 x 8 output tile per warp.
-__device__ __forceinline__ void cmma_16x8(float (&cr)[4], float (&ci)[4], const float *Ar, const float *Ai, int a_ld,
-                                          int a_row0, int a_col0, const float *Br, const float *Bi, int b_ld,
-                                          int b_row0, int b_col0, int s0, int s1, int lane)
-{
-    const int g = lane >> 2, tg = lane & 3;
-    for (int s = s0; s < s1; ++s) {
-        const int ao = (a_row0 + g) * a_ld + a_col0 + 8 * s + tg;
-        uint32_t ar[4], ai[4], nai[4], br[2], bi[2];
-        ar[0] = to_tf32(Ar[ao]);
-        ar[1] = to_tf32(Ar[ao + 8 * a_ld]);
-        ar[2] = to_tf32(Ar[ao + 4]);
-        ar[3] = to_tf32(Ar[ao + 8 * a_ld + 4]);
-        ai[0] = to_tf32(Ai[ao]);
-        ai[1] = to_tf32(Ai[ao + 8 * a_ld]);
-        ai[2] = to_tf32(Ai[ao + 4]);
-        ai[3] = to_tf32(Ai[ao + 8 * a_ld + 4]);
-#pragma unroll
-        for (int x = 0; x < 4; ++x) nai[x] = ai[x] ^ 0x80000000u;
-        const int bo = (b_row0 + 8 * s + tg) * b_ld + b_col0 + g;
-        br[0] = to_tf32(Br[bo]);
-        br[1] = to_tf32(Br[bo + 4 * b_ld]);
-        bi[0] = to_tf32(Bi[bo]);
-        bi[1] = to_tf32(Bi[bo + 4 * b_ld]);
-        mma_tf32(cr, ar, br);
-        mma_tf32(cr, nai, bi);
-        mma_tf32(ci, ar, bi);
-        mma_tf32(ci, ai, br);
-    }
-}
-// Store a 16 x 8 accumulator tile (times `scale`) at rows row0.., columns col0.. of a complex fp32 matrix.
-__device__ __forceinline__ void store_tile(const float (&cr)[4], const float (&ci)[4], float scale, float *Dr, float *Di,
-                                           int ld, int row0, int col0, int lane)
-{
-    const int g = lane >> 2, tg = lane & 3;
-    const int o = (row0 + g) * ld + col0 + 2 * tg;
-    Dr[o] = scale * cr[0];
-    Dr[o + 1] = scale * cr[1];
-    Dr[o + 8 * ld] = scale * cr[2];
-    Dr[o + 8 * ld + 1] = scale * cr[3];
-    Di[o] = scale * ci[0];
-    Di[o + 1] = scale * ci[1];
-    Di[o + 8 * ld] = scale * ci[2];
-    Di[o + 8 * ld + 1] = scale * ci[3];
-}
 
 // Optional per-phase cycle counters (development builds only, -DSFDA_TC_TIMING).
 #ifdef SFDA_TC_TIMING

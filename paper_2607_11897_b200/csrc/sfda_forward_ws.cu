@@ -1,0 +1,842 @@
+// Warp-specialised tensor-core chunk-WY forward for sm_100a: bf16 q/k/v, d_k = d_v = 128, chunk C = 64.
+//
+// One CTA (17 warps) walks the chunks of one (batch, head) pair; four roles run concurrently on
+// different chunks and hand tiles to one another through mbarriers:
+//
+//   PREP  (4 warps)  chunk j+1..j+2: cumulative phase-decay gamma_t = a_t e^{i phi_t} (Eq. "constructive-Gamma";
+//                    log2-sum and integer-turn prefix scans), rotated/decayed operand tiles in shared memory.
+//   SOLVE (4 warps)  chunk j+1: drains the Gram blocks from tensor memory, inverts the unit-lower WY system
+//                    (Eq. "constructive-M": M = (I + L)^{-1}) by 16x16 blocks, writes M_beta and Aq tiles.
+//   CHAIN (8 warps)  chunk j: the state-dependent conversions between the tcgen05 products
+//                    (state pass, R = V - W^* S_0, E, outputs); they own the TMEM <-> register traffic.
+//   CTRL  (1 warp)   one thread issues every tcgen05.mma / commit and the TMA copies.
+//
+// Algebra (k'_t = e^{-i phi_t} k_t, q'_t = e^{-i phi_t} q_t, all tiles bf16, de-interleaved [Re | Im]):
+//   W_t = a_t k'_t (= conj(gamma_t) k_t, Eq. "constructive-W"),  Qt_t = a_t q'_t,  Kc_t = k'_t / a_t
+//   Kt[t][i] = W_t^* Kc_i (i < t),  Aq[t][i] = Qt_t^* Kc_i (i <= t)
+//   M_beta = (I + D_beta Kt)^{-1} D_beta,  R = V - W^* S_0,  E = M_beta R            (Eq. "apply-transfer")
+//   rho_t = Qt_t^* S_0 + sum_{i<=t} Aq[t][i] e_i^T,  o_t = conj(rho_t)               (Thm "Prefix outputs")
+//   S_C = e^{i phi_C} a_C (S_0 + sum_t Kc_t e_t^T)                                    (boundary-state scan)
+// The fp32 state lives in tensor memory, transposed (lane = value channel, column = key channel
+// [Re j | Im j]); the update accumulates onto the unscaled S_0 and the factor e^{i phi_C} a_C is applied by
+// the next chunk's state pass, so no operand depends on the chunk's total decay.
+#include <cuda.h>
+
+#include "sfda_common.cuh"
+#include "sfda_internal.h"
+#include "sfda_tc_ptx.cuh"
+
+namespace sfda {
+namespace {
+
+using namespace tc;
+
+constexpr int C = 64, DK = 128, DV = 128, M = 64;
+constexpr int kChainWarps = 8, kSolveWarps = 4, kPrepWarps = 4;
+constexpr int kCtrlWarps = 4;   // a full warpgroup, so that it can hand its registers to the others; one thread works
+constexpr int kThreads = 32 * (kChainWarps + kSolveWarps + kPrepWarps + kCtrlWarps);   // 640
+// The CTA is launched with 96 registers per thread (640 * 96 = 61440); the roles then rebalance that pool:
+// 8 * 96 + 4 * 96 + 4 * 128 + 4 * 64 = 1920 warp rows = 61440 registers.
+constexpr int kRegsChain = 96, kRegsSolve = 96, kRegsPrep = 128, kRegsCtrl = 64;
+constexpr int kChainThreads = 32 * kChainWarps, kSolveThreads = 32 * kSolveWarps, kPrepThreads = 32 * kPrepWarps;
+
+// ---- shared memory map (bytes from a 1024-aligned base) -------------------------------------------------
+constexpr int kTile = 8192;                       // 64 rows x 128 B, K-major, 128B swizzle
+constexpr int OFF_WQ = 0;                         // [2 slots][re | im][128 rows: W then Qt]      64 KB
+constexpr int OFF_KC = OFF_WQ + 2 * 4 * kTile;    // Kc [i][j], re | im (Gram B operand)          16 KB
+constexpr int OFF_KT = OFF_KC + 2 * kTile;        // [2 slots] Kc^T [j][t], re | im (update B)    32 KB
+constexpr int OFF_MB = OFF_KT + 2 * 2 * kTile;    // M_beta [t][i], re | im                       16 KB
+constexpr int OFF_AQ = OFF_MB + 2 * kTile;        // [2 slots] Aq [t][i], re | im                 32 KB
+constexpr int OFF_V = OFF_AQ + 2 * 2 * kTile;     // v staging [t][128] bf16 (TMA)                16 KB
+constexpr int LS = 68;                            // row stride (floats) of the solve scratch
+constexpr int OFF_LX = OFF_V + 16384;             // L -> X in place, fp32 [64][LS], re | im      34 KB
+constexpr int OFF_MISC = OFF_LX + 2 * 64 * LS * 4;
+constexpr int kSmemBytes = OFF_MISC + 7168 + 1024;
+
+enum Bar {
+    B_PREP_FULL0, B_PREP_FULL1, B_KT_FULL0, B_KT_FULL1, B_WQ_FREE0, B_WQ_FREE1, B_KC_FREE, B_STORE_DONE0,
+    B_STORE_DONE1, B_GRAM_FULL, B_GRAM_DRAINED, B_MB_FULL, B_AQ_FULL0, B_AQ_FULL1, B_D1_DONE, B_E_DONE, B_UPD_DONE,
+    B_S16_READY, B_R16_READY, B_E16_READY, B_O_STAGED, B_V_FULL, B_SYNC_PREP, B_SYNC_SOLVE, kNumBars
+};
+
+struct Misc {
+    float part_lg[4][M];
+    uint32_t part_turns[4][M];
+    float aC[4][M], closing_cos[4][M], closing_sin[4][M];   // ring of four chunks
+    float beta[4][C];
+    unsigned long long bars[kNumBars];
+    uint32_t tmem_base;
+    volatile int abort;
+};
+static_assert(sizeof(Misc) <= 7168, "misc area too small");
+static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA exceeded");
+
+// ---- tensor memory map (columns) ----------------------------------------------------------------------
+constexpr uint32_t TM_S32 = 0;      // state fp32 [Re j | Im j]
+constexpr uint32_t TM_X16 = 128;    // bf16 A operand: S_0, then R, then E (64 packed columns)
+constexpr uint32_t TM_GRAM = 192;   // Gram half (Re, then Im): lanes 0..63 Kt rows, 64..127 Aq rows
+constexpr uint32_t TM_ACC = 256;    // [D1/E re | rho re | D1/E im | rho im], 64 columns each
+
+struct Params {
+    const __nv_bfloat16 *q, *k;
+    const float *alpha, *theta, *beta, *S0;
+    float *S_T;
+    uint32_t *status;
+    int T, H, has_o_im;
+};
+
+__device__ __forceinline__ void mbar_arrive(unsigned long long *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+template <int N>
+__device__ __forceinline__ void regs_inc()
+{
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void regs_dec()
+{
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+
+__device__ __forceinline__ unsigned long long now_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // no wait of this kernel may last longer than 2 s
+
+// Non-blocking test of completion number k (0-based) of a barrier.
+__device__ __forceinline__ bool test_k(Misc &mi, int bar, int k)
+{
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+                 : "=r"(ok)
+                 : "r"(smem_u32(&mi.bars[bar])), "r"((uint32_t)k & 1u)
+                 : "memory");
+    return ok != 0;
+}
+// Wait for completion number k; gives up after kWaitLimitNs or when another role has raised the abort flag.
+// Returns false in that case, after raising the flag itself.
+__device__ __forceinline__ bool wait_k(Misc &mi, int bar, int k)
+{
+    if (test_k(mi, bar, k)) return true;
+    const unsigned long long t0 = now_ns();
+    for (uint32_t it = 0;; ++it) {
+        if (test_k(mi, bar, k)) return true;
+        if ((it & 255u) == 255u) {
+            if (mi.abort) return false;
+            if (now_ns() - t0 > kWaitLimitNs) break;
+        }
+    }
+    mi.abort = 1;
+    return false;
+}
+// Barrier among the threads of one role, with the same bounded wait as everything else (a plain bar.sync
+// could wait forever for a thread that has given up).  `n` counts the calls of the role.
+__device__ __forceinline__ bool group_sync(Misc &mi, int bar, int &n)
+{
+    mbar_arrive(&mi.bars[bar]);
+    return wait_k(mi, bar, n++);
+}
+
+// ---- CTRL: one thread issues all tensor-core and TMA work ------------------------------------------------
+__device__ __forceinline__ void run_ctrl(uint8_t *smem, Misc &mi, uint32_t tmem, const CUtensorMap *tm_v, const CUtensorMap *tm_o,
+                         const CUtensorMap *tm_oim, const Params &p, int b, int h, int n_chunks)
+{
+    const uint32_t sbase = smem_u32(smem);
+    auto wq = [&](int s, int im) { return sbase + OFF_WQ + (s * 2 + im) * 2 * kTile; };   // 128-row tile
+    auto kc = [&](int im) { return sbase + OFF_KC + im * kTile; };
+    auto kt = [&](int s, int im) { return sbase + OFF_KT + (s * 2 + im) * kTile; };
+    auto mb = [&](int im) { return sbase + OFF_MB + im * kTile; };
+    auto aq = [&](int s, int im) { return sbase + OFF_AQ + (s * 2 + im) * kTile; };
+    unsigned long long *bars = mi.bars;
+
+    auto gram_half = [&](int j, int im) {   // Kt/Aq half into TM_GRAM: rows = [W; Qt] of slot j&1, columns = tokens i
+        const int s = j & 1;
+        const uint32_t d = tmem + TM_GRAM;
+        if (!im) {
+            mma_k64_ss(d, wq(s, 0), kc(0), idesc(64, 0), false);
+            mma_k64_ss(d, wq(s, 1), kc(1), idesc(64, 0), true);
+        } else {
+            mma_k64_ss(d, wq(s, 0), kc(1), idesc(64, 0), false);
+            mma_k64_ss(d, wq(s, 1), kc(0), idesc(64, 1), true);
+        }
+        mma_commit(&bars[B_GRAM_FULL]);
+    };
+
+    mbar_expect_tx(&bars[B_V_FULL], 16384);
+    tma_load_4d(smem + OFF_V, tm_v, &bars[B_V_FULL], 0, h, 0, b);
+
+    // The Gram products run ahead of the chain: chunk g, half gh is issued as soon as its operands are ready and
+    // the Gram columns have been drained; the chain's own waits keep trying in the meantime.
+    int g = 0, gh = 0;
+    auto pump_gram = [&]() {
+        if (g >= n_chunks) return;
+        if (gh == 0) {
+            if (!test_k(mi, g & 1 ? B_PREP_FULL1 : B_PREP_FULL0, g >> 1)) return;
+            if (g > 0 && !test_k(mi, B_GRAM_DRAINED, 2 * g - 1)) return;
+            tc_fence_after();
+            gram_half(g, 0);
+            gh = 1;
+        } else {
+            if (!test_k(mi, B_GRAM_DRAINED, 2 * g)) return;
+            tc_fence_after();
+            gram_half(g, 1);
+            mma_commit(&bars[B_KC_FREE]);
+            gh = 0;
+            ++g;
+        }
+    };
+    auto wait_pump = [&](int bar, int k) {
+        if (test_k(mi, bar, k)) return true;
+        const unsigned long long t0 = now_ns();
+        for (uint32_t it = 0;; ++it) {
+            if (test_k(mi, bar, k)) return true;
+            pump_gram();
+            if ((it & 255u) == 255u) {
+                if (mi.abort) return false;
+                if (now_ns() - t0 > kWaitLimitNs) break;
+            }
+        }
+        mi.abort = 1;
+        return false;
+    };
+
+    const uint32_t x_re = tmem + TM_X16, x_im = tmem + TM_X16 + 32;
+    for (int j = 0; j < n_chunks; ++j) {
+        const int s = j & 1, u = j >> 1;
+        // D1 = W^* S_0
+        if (!wait_pump(B_S16_READY, j)) return;
+        if (!wait_pump(s ? B_PREP_FULL1 : B_PREP_FULL0, u)) return;
+        tc_fence_after();
+        {
+            const uint32_t d_re = tmem + TM_ACC, d_im = tmem + TM_ACC + 128;
+            mma_k64_ts(d_re, x_re, wq(s, 0), idesc(64, 0), false);
+            mma_k64_ts(d_re, x_im, wq(s, 1), idesc(64, 0), true);
+            mma_k64_ts(d_im, x_im, wq(s, 0), idesc(64, 0), false);
+            mma_k64_ts(d_im, x_re, wq(s, 1), idesc(64, 1), true);
+            mma_commit(&bars[B_D1_DONE]);
+        }
+        // outputs of the previous chunk are staged: store them; rho is free again
+        if (j > 0) {
+            if (!wait_pump(B_O_STAGED, j - 1)) return;
+            tc_fence_after();
+            const int sp = (j - 1) & 1;
+            tma_store_4d(tm_o, smem + OFF_KT + sp * 2 * kTile, 0, h, (j - 1) * C, b);
+            if (p.has_o_im) tma_store_4d(tm_oim, smem + OFF_AQ + sp * 2 * kTile, 0, h, (j - 1) * C, b);
+            tma_store_commit();
+        }
+        // rho_1 = Qt^* S_0
+        {
+            const uint32_t o_re = tmem + TM_ACC + 64, o_im = tmem + TM_ACC + 192;
+            mma_k64_ts(o_re, x_re, wq(s, 0) + kTile, idesc(64, 0), false);
+            mma_k64_ts(o_re, x_im, wq(s, 1) + kTile, idesc(64, 0), true);
+            mma_k64_ts(o_im, x_im, wq(s, 0) + kTile, idesc(64, 0), false);
+            mma_k64_ts(o_im, x_re, wq(s, 1) + kTile, idesc(64, 1), true);
+            mma_commit(&bars[s ? B_WQ_FREE1 : B_WQ_FREE0]);
+        }
+        pump_gram();
+        if (j > 0) {   // the store of chunk j-1 has read its staging tiles (Kt / Aq of slot (j-1)&1)
+            tma_store_wait_read();
+            mbar_arrive(&bars[(j - 1) & 1 ? B_STORE_DONE1 : B_STORE_DONE0]);
+        }
+        // E = M_beta R
+        if (!wait_pump(B_R16_READY, j)) return;
+        if (!wait_pump(B_MB_FULL, j)) return;
+        tc_fence_after();
+        {
+            const uint32_t e_re = tmem + TM_ACC, e_im = tmem + TM_ACC + 128;
+            mma_k64_ts(e_re, x_re, mb(0), idesc(64, 0), false);
+            mma_k64_ts(e_re, x_im, mb(1), idesc(64, 1), true);
+            mma_k64_ts(e_im, x_im, mb(0), idesc(64, 0), false);
+            mma_k64_ts(e_im, x_re, mb(1), idesc(64, 0), true);
+            mma_commit(&bars[B_E_DONE]);
+        }
+        if (j + 1 < n_chunks) {   // v of chunk j has been consumed
+            mbar_expect_tx(&bars[B_V_FULL], 16384);
+            tma_load_4d(smem + OFF_V, tm_v, &bars[B_V_FULL], 0, h, (j + 1) * C, b);
+        }
+        pump_gram();
+        // S += E^T Kc ,  rho += Aq E
+        if (!wait_pump(B_E16_READY, j)) return;
+        if (!wait_pump(s ? B_KT_FULL1 : B_KT_FULL0, u)) return;
+        if (!wait_pump(s ? B_AQ_FULL1 : B_AQ_FULL0, u)) return;
+        tc_fence_after();
+        {
+            const uint32_t s_re = tmem + TM_S32, s_im = tmem + TM_S32 + 64;
+            mma_k64_ts(s_re, x_re, kt(s, 0), idesc(64, 0), true);
+            mma_k64_ts(s_re, x_im, kt(s, 1), idesc(64, 1), true);
+            mma_k64_ts(s_im, x_re, kt(s, 1), idesc(64, 0), true);
+            mma_k64_ts(s_im, x_im, kt(s, 0), idesc(64, 0), true);
+            const uint32_t o_re = tmem + TM_ACC + 64, o_im = tmem + TM_ACC + 192;
+            mma_k64_ts(o_re, x_re, aq(s, 0), idesc(64, 0), true);
+            mma_k64_ts(o_re, x_im, aq(s, 1), idesc(64, 1), true);
+            mma_k64_ts(o_im, x_im, aq(s, 0), idesc(64, 0), true);
+            mma_k64_ts(o_im, x_re, aq(s, 1), idesc(64, 0), true);
+            mma_commit(&bars[B_UPD_DONE]);
+        }
+        pump_gram();
+    }
+    if (!wait_pump(B_O_STAGED, n_chunks - 1)) return;
+    {
+        const int sp = (n_chunks - 1) & 1;
+        tma_store_4d(tm_o, smem + OFF_KT + sp * 2 * kTile, 0, h, (n_chunks - 1) * C, b);
+        if (p.has_o_im) tma_store_4d(tm_oim, smem + OFF_AQ + sp * 2 * kTile, 0, h, (n_chunks - 1) * C, b);
+        tma_store_commit();
+    }
+    tma_store_wait_all();
+}
+
+// ---- PREP ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, const Params &p, int b, int h, int n_chunks, int pt)
+{
+    const int jp = pt & 31, tq = pt >> 5;   // channel pair (channels 2jp, 2jp+1), token quarter (16 tokens)
+    int nsync = 0;
+    for (int j = 0; j < n_chunks; ++j) {
+        const int s = j & 1, ring = j & 3;
+        const int t0 = j * C, len = min(C, p.T - t0);
+        const size_t row0 = ((size_t)b * p.T + t0) * p.H + h;   // token t of this head: row0 + t * H
+
+        // pass 1: prefix sums of log2 alpha and of the integer phase over this thread's 16 tokens
+        float lg0[16], lg1[16];
+        uint32_t tu0[16], tu1[16];
+        {
+            float2 al[16], th[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int t = tq * 16 + i;
+                if (t < len) {
+                    al[i] = __ldg(reinterpret_cast<const float2 *>(p.alpha + (row0 + (size_t)t * p.H) * M) + jp);
+                    th[i] = __ldg(reinterpret_cast<const float2 *>(p.theta + (row0 + (size_t)t * p.H) * M) + jp);
+                } else {
+                    al[i] = make_float2(1.f, 1.f);
+                    th[i] = make_float2(0.f, 0.f);
+                }
+            }
+            float a0 = 0.f, a1 = 0.f;
+            uint32_t u0 = 0u, u1 = 0u;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                a0 += fmaxf(__log2f(al[i].x), -43.28f);   // floor e^-30, as in log_decay
+                a1 += fmaxf(__log2f(al[i].y), -43.28f);
+                u0 += phase_to_turns(th[i].x);
+                u1 += phase_to_turns(th[i].y);
+                lg0[i] = a0; lg1[i] = a1; tu0[i] = u0; tu1[i] = u1;
+            }
+            mi.part_lg[tq][2 * jp] = a0;
+            mi.part_lg[tq][2 * jp + 1] = a1;
+            mi.part_turns[tq][2 * jp] = u0;
+            mi.part_turns[tq][2 * jp + 1] = u1;
+        }
+        if (!group_sync(mi, B_SYNC_PREP, nsync)) return;
+        float base0 = 0.f, base1 = 0.f, tot0 = 0.f, tot1 = 0.f;
+        uint32_t tb0 = 0u, tb1 = 0u, tt0 = 0u, tt1 = 0u;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const float2 pl = *reinterpret_cast<const float2 *>(&mi.part_lg[g][2 * jp]);
+            const uint2 pu = *reinterpret_cast<const uint2 *>(&mi.part_turns[g][2 * jp]);
+            if (g < tq) { base0 += pl.x; base1 += pl.y; tb0 += pu.x; tb1 += pu.y; }
+            tot0 += pl.x; tot1 += pl.y; tt0 += pu.x; tt1 += pu.y;
+        }
+        if (!group_sync(mi, B_SYNC_PREP, nsync)) return;   // partials may be overwritten from here on
+        if (tq == 0) {                    // chunk totals: a_C and the closing phase e^{i phi_C}
+            float cs, sn;
+            mi.aC[ring][2 * jp] = exp2f(tot0);
+            mi.aC[ring][2 * jp + 1] = exp2f(tot1);
+            __sincosf((float)(int32_t)tt0 * 0x1.921fb6p-30f, &sn, &cs);   // turns * 2 pi / 2^32
+            mi.closing_cos[ring][2 * jp] = cs;
+            mi.closing_sin[ring][2 * jp] = sn;
+            __sincosf((float)(int32_t)tt1 * 0x1.921fb6p-30f, &sn, &cs);
+            mi.closing_cos[ring][2 * jp + 1] = cs;
+            mi.closing_sin[ring][2 * jp + 1] = sn;
+        }
+        if (pt < C) mi.beta[ring][pt] = pt < len ? __ldg(p.beta + row0 + (size_t)pt * p.H) : 0.f;
+
+        // the W/Qt tiles of this slot and the Kc tile must have been consumed
+        if (j >= 2 && !wait_k(mi, s ? B_WQ_FREE1 : B_WQ_FREE0, (j >> 1) - 1)) return;
+        if (j >= 1 && !wait_k(mi, B_KC_FREE, j - 1)) return;
+
+        // pass 2a: rotated / decayed operands
+        uint8_t *wq_re = smem + OFF_WQ + (s * 2) * 2 * kTile, *wq_im = wq_re + 2 * kTile;
+        uint8_t *kc_re = smem + OFF_KC, *kc_im = kc_re + kTile;
+        uint32_t k0r[8], k0i[8], k1r[8], k1i[8];   // Kc^T rows 2jp and 2jp+1, 16 tokens, packed bf16 pairs
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int t = tq * 16 + i;
+            uint2 kw = make_uint2(0u, 0u), qw = make_uint2(0u, 0u);
+            if (t < len) {
+                kw = __ldg(reinterpret_cast<const uint2 *>(p.k + (row0 + (size_t)t * p.H) * DK) + jp);
+                qw = __ldg(reinterpret_cast<const uint2 *>(p.q + (row0 + (size_t)t * p.H) * DK) + jp);
+            }
+            float wr[2], wi[2], cr_[2], ci_[2], qr_[2], qi_[2];
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+                const float l2 = x ? base1 + lg1[i] : base0 + lg0[i];
+                const uint32_t tu = x ? tb1 + tu1[i] : tb0 + tu0[i];
+                const uint32_t kx = x ? kw.y : kw.x, qx = x ? qw.y : qw.x;
+                const float a = exp2f(l2);
+                const float ainv = exp2f(fminf(-l2, 115.4f));                 // 1/a_t, capped at e^80
+                float cs, sn;
+                __sincosf((float)(int32_t)tu * 0x1.921fb6p-30f, &sn, &cs);
+                const float kr = __uint_as_float(kx << 16), ki = __uint_as_float(kx & 0xffff0000u);
+                const float qr = __uint_as_float(qx << 16), qi = __uint_as_float(qx & 0xffff0000u);
+                const float kpr = kr * cs + ki * sn, kpi = ki * cs - kr * sn;   // e^{-i phi} k
+                const float qpr = qr * cs + qi * sn, qpi = qi * cs - qr * sn;
+                wr[x] = a * kpr; wi[x] = a * kpi;
+                qr_[x] = a * qpr; qi_[x] = a * qpi;
+                cr_[x] = ainv * kpr; ci_[x] = ainv * kpi;
+            }
+            const int o1 = sw_off(t, 2 * jp);
+            *reinterpret_cast<uint32_t *>(wq_re + o1) = pack_bf16(wr[0], wr[1]);
+            *reinterpret_cast<uint32_t *>(wq_im + o1) = pack_bf16(wi[0], wi[1]);
+            *reinterpret_cast<uint32_t *>(wq_re + kTile + o1) = pack_bf16(qr_[0], qr_[1]);
+            *reinterpret_cast<uint32_t *>(wq_im + kTile + o1) = pack_bf16(qi_[0], qi_[1]);
+            *reinterpret_cast<uint32_t *>(kc_re + o1) = pack_bf16(cr_[0], cr_[1]);
+            *reinterpret_cast<uint32_t *>(kc_im + o1) = pack_bf16(ci_[0], ci_[1]);
+            const uint32_t h0r = __bfloat16_as_ushort(__float2bfloat16_rn(cr_[0]));
+            const uint32_t h0i = __bfloat16_as_ushort(__float2bfloat16_rn(ci_[0]));
+            const uint32_t h1r = __bfloat16_as_ushort(__float2bfloat16_rn(cr_[1]));
+            const uint32_t h1i = __bfloat16_as_ushort(__float2bfloat16_rn(ci_[1]));
+            if (i & 1) {
+                k0r[i >> 1] |= h0r << 16; k0i[i >> 1] |= h0i << 16;
+                k1r[i >> 1] |= h1r << 16; k1i[i >> 1] |= h1i << 16;
+            } else {
+                k0r[i >> 1] = h0r; k0i[i >> 1] = h0i;
+                k1r[i >> 1] = h1r; k1i[i >> 1] = h1i;
+            }
+        }
+        fence_async_smem();
+        mbar_arrive(&mi.bars[s ? B_PREP_FULL1 : B_PREP_FULL0]);
+
+        // pass 2b: Kc^T once the slot's previous occupant (update operand, then output staging) is done with
+        if (j >= 2 && !wait_k(mi, s ? B_STORE_DONE1 : B_STORE_DONE0, (j >> 1) - 1)) return;
+        uint8_t *kt_re = smem + OFF_KT + (s * 2) * kTile, *kt_im = kt_re + kTile;
+#pragma unroll
+        for (int cidx = 0; cidx < 2; ++cidx) {
+            const int oa = sw_off(2 * jp, tq * 16 + cidx * 8), ob = sw_off(2 * jp + 1, tq * 16 + cidx * 8);
+            *reinterpret_cast<uint4 *>(kt_re + oa) = make_uint4(k0r[4 * cidx], k0r[4 * cidx + 1], k0r[4 * cidx + 2], k0r[4 * cidx + 3]);
+            *reinterpret_cast<uint4 *>(kt_im + oa) = make_uint4(k0i[4 * cidx], k0i[4 * cidx + 1], k0i[4 * cidx + 2], k0i[4 * cidx + 3]);
+            *reinterpret_cast<uint4 *>(kt_re + ob) = make_uint4(k1r[4 * cidx], k1r[4 * cidx + 1], k1r[4 * cidx + 2], k1r[4 * cidx + 3]);
+            *reinterpret_cast<uint4 *>(kt_im + ob) = make_uint4(k1i[4 * cidx], k1i[4 * cidx + 1], k1i[4 * cidx + 2], k1i[4 * cidx + 3]);
+        }
+        fence_async_smem();
+        mbar_arrive(&mi.bars[s ? B_KT_FULL1 : B_KT_FULL0]);
+    }
+}
+
+// ---- SOLVE --------------------------------------------------------------------------------------------
+__device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem, int n_chunks, int st)
+{
+    const int lane = st & 31, w = st >> 5;    // w = TMEM lane quadrant of this warp
+    float *Lr = reinterpret_cast<float *>(smem + OFF_LX), *Li = Lr + 64 * LS;
+    const uint32_t tlane = tmem + ((uint32_t)(w * 32) << 16);
+    const int row = w * 32 + lane;            // Gram row held by this thread: < 64 -> Kt row, else Aq row
+    int nsync = 0;
+    for (int j = 0; j < n_chunks; ++j) {
+        const int s = j & 1, ring = j & 3;
+        // The Aq tile of this slot also staged the outputs of chunk j-2: its rows are written straight from the
+        // drain, so the warps that hold them wait for that store first.
+        if (row >= 64 && j >= 2 && !wait_k(mi, s ? B_STORE_DONE1 : B_STORE_DONE0, (j >> 1) - 1)) return;
+        // ---- drain the two Gram halves
+#pragma unroll
+        for (int im = 0; im < 2; ++im) {
+            if (!wait_k(mi, B_GRAM_FULL, 2 * j + im)) return;
+            tc_fence_after();
+#pragma unroll
+            for (int hc = 0; hc < 2; ++hc) {      // 32 columns at a time keeps the register footprint down
+                uint32_t r[32];
+                tmem_ld<32>(tlane + TM_GRAM + 32 * hc, r);
+                tc_wait_ld();
+                if (hc == 1) {
+                    tc_fence_before();
+                    mbar_arrive(&mi.bars[B_GRAM_DRAINED]);
+                }
+                if (row < 64) {                   // L = D_beta Kt, strictly lower
+                    const int t = row;
+                    const float bt = mi.beta[ring][t];
+                    float4 *dst = reinterpret_cast<float4 *>((im ? Li : Lr) + t * LS + 32 * hc);
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) {
+                        const int ii = 32 * hc + i;
+                        dst[i >> 2] = make_float4(ii < t ? bt * __uint_as_float(r[i]) : 0.f,
+                                                  ii + 1 < t ? bt * __uint_as_float(r[i + 1]) : 0.f,
+                                                  ii + 2 < t ? bt * __uint_as_float(r[i + 2]) : 0.f,
+                                                  ii + 3 < t ? bt * __uint_as_float(r[i + 3]) : 0.f);
+                    }
+                } else {                          // Aq, lower incl. diagonal, as a bf16 operand tile
+                    const int t = row - 64;
+                    uint8_t *tile = smem + OFF_AQ + (s * 2 + im) * kTile;
+#pragma unroll
+                    for (int c8 = 0; c8 < 4; ++c8) {
+                        uint32_t wv[4];
+#pragma unroll
+                        for (int x = 0; x < 4; ++x) {
+                            const int ii = 32 * hc + 8 * c8 + 2 * x;
+                            wv[x] = pack_bf16(ii <= t ? __uint_as_float(r[8 * c8 + 2 * x]) : 0.f,
+                                              ii + 1 <= t ? __uint_as_float(r[8 * c8 + 2 * x + 1]) : 0.f);
+                        }
+                        *reinterpret_cast<uint4 *>(tile + sw_off(t, 32 * hc + 8 * c8)) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+                    }
+                }
+            }
+        }
+        fence_async_smem();
+        mbar_arrive(&mi.bars[s ? B_AQ_FULL1 : B_AQ_FULL0]);
+        if (!group_sync(mi, B_SYNC_SOLVE, nsync)) return;
+
+        // ---- X = (I + L)^{-1} in place: diagonal 16x16 blocks by substitution, merges on mma.sync
+        if (lane < 16) {                      // warp w inverts diagonal block w, lane = column
+            const int o = 16 * w, c = lane;
+            float xr[16], xi[16];
+#pragma unroll
+            for (int r = 0; r < 16; ++r) {
+                float ar = r == c ? 1.f : 0.f, ai = 0.f;
+#pragma unroll
+                for (int i = 0; i < 15; ++i) {
+                    if (i < r) {
+                        const float lr_ = Lr[(o + r) * LS + o + i], li_ = Li[(o + r) * LS + o + i];
+                        const float vr = i >= c ? xr[i] : 0.f, vi = i >= c ? xi[i] : 0.f;
+                        ar -= lr_ * vr - li_ * vi;
+                        ai -= lr_ * vi + li_ * vr;
+                    }
+                }
+                xr[r] = r >= c ? ar : 0.f;
+                xi[r] = r >= c ? ai : 0.f;
+            }
+            __syncwarp(0x0000ffffu);          // every lane has read its L rows before the block is overwritten
+#pragma unroll
+            for (int r = 0; r < 16; ++r) {
+                Lr[(o + r) * LS + o + c] = xr[r];
+                Li[(o + r) * LS + o + c] = xi[r];
+            }
+        }
+        if (!group_sync(mi, B_SYNC_SOLVE, nsync)) return;
+        {   // level 1: X[b1][b0] = -X[b1][b1] (L[b1][b0] X[b0][b0]); T in the unused block above the diagonal
+            const int pr = w >> 1, nt = w & 1;
+            const int r0 = 32 * pr + 16, c0 = 32 * pr;
+            float cr[4] = {0.f, 0.f, 0.f, 0.f}, ci[4] = {0.f, 0.f, 0.f, 0.f};
+            cmma_16x8(cr, ci, Lr, Li, LS, r0, c0, Lr, Li, LS, c0, c0 + 8 * nt, nt, 2, lane);
+            store_tile(cr, ci, 1.f, Lr, Li, LS, c0, r0 + 8 * nt, lane);          // T at block (b0, b1)
+            if (!group_sync(mi, B_SYNC_SOLVE, nsync)) return;
+            float dr[4] = {0.f, 0.f, 0.f, 0.f}, di[4] = {0.f, 0.f, 0.f, 0.f};
+            cmma_16x8(dr, di, Lr, Li, LS, r0, r0, Lr, Li, LS, c0, r0 + 8 * nt, 0, 2, lane);
+            if (!group_sync(mi, B_SYNC_SOLVE, nsync)) return;                                     // L[b1][b0] fully read
+            store_tile(dr, di, -1.f, Lr, Li, LS, r0, c0 + 8 * nt, lane);
+        }
+        if (!group_sync(mi, B_SYNC_SOLVE, nsync)) return;
+        {   // level 2: X[BL] = -X[BR] (L[BL] X[TL]); T in the top-right quadrant; warp w owns column tile w
+            const int nt = w;
+            float c0r[4] = {0.f, 0.f, 0.f, 0.f}, c0i[4] = {0.f, 0.f, 0.f, 0.f};
+            float c1r[4] = {0.f, 0.f, 0.f, 0.f}, c1i[4] = {0.f, 0.f, 0.f, 0.f};
+            cmma_16x8(c0r, c0i, Lr, Li, LS, 32, 0, Lr, Li, LS, 0, 8 * nt, nt, 4, lane);
+            cmma_16x8(c1r, c1i, Lr, Li, LS, 48, 0, Lr, Li, LS, 0, 8 * nt, nt, 4, lane);
+            store_tile(c0r, c0i, 1.f, Lr, Li, LS, 0, 32 + 8 * nt, lane);
+            store_tile(c1r, c1i, 1.f, Lr, Li, LS, 16, 32 + 8 * nt, lane);
+            if (!group_sync(mi, B_SYNC_SOLVE, nsync)) return;
+            float d0r[4] = {0.f, 0.f, 0.f, 0.f}, d0i[4] = {0.f, 0.f, 0.f, 0.f};
+            float d1r[4] = {0.f, 0.f, 0.f, 0.f}, d1i[4] = {0.f, 0.f, 0.f, 0.f};
+            cmma_16x8(d0r, d0i, Lr, Li, LS, 32, 32, Lr, Li, LS, 0, 32 + 8 * nt, 0, 2, lane);
+            cmma_16x8(d1r, d1i, Lr, Li, LS, 48, 32, Lr, Li, LS, 0, 32 + 8 * nt, 0, 4, lane);
+            if (!group_sync(mi, B_SYNC_SOLVE, nsync)) return;                                     // L[BL] fully read
+            store_tile(d0r, d0i, -1.f, Lr, Li, LS, 32, 8 * nt, lane);
+            store_tile(d1r, d1i, -1.f, Lr, Li, LS, 48, 8 * nt, lane);
+        }
+        if (!group_sync(mi, B_SYNC_SOLVE, nsync)) return;
+
+        // ---- M_beta = X D_beta as a bf16 operand tile, once E of the previous chunk has read the old one
+        if (j >= 1 && !wait_k(mi, B_E_DONE, j - 1)) return;
+        {
+            const int t = st >> 1, part = st & 1;   // row t, columns 32 part .. 32 part + 31
+#pragma unroll
+            for (int cidx = 0; cidx < 4; ++cidx) {
+                uint32_t wr[4], wi[4];
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {
+                    const int i0 = part * 32 + cidx * 8 + 2 * x;
+                    const float b0 = mi.beta[ring][i0], b1 = mi.beta[ring][i0 + 1];
+                    const bool in0 = i0 <= t, in1 = i0 + 1 <= t;
+                    wr[x] = pack_bf16(in0 ? Lr[t * LS + i0] * b0 : 0.f, in1 ? Lr[t * LS + i0 + 1] * b1 : 0.f);
+                    wi[x] = pack_bf16(in0 ? Li[t * LS + i0] * b0 : 0.f, in1 ? Li[t * LS + i0 + 1] * b1 : 0.f);
+                }
+                const int off = sw_off(t, part * 32 + cidx * 8);
+                *reinterpret_cast<uint4 *>(smem + OFF_MB + off) = make_uint4(wr[0], wr[1], wr[2], wr[3]);
+                *reinterpret_cast<uint4 *>(smem + OFF_MB + kTile + off) = make_uint4(wi[0], wi[1], wi[2], wi[3]);
+            }
+        }
+        fence_async_smem();
+        mbar_arrive(&mi.bars[B_MB_FULL]);
+        if (!group_sync(mi, B_SYNC_SOLVE, nsync)) return;      // the scratch may be overwritten by the next chunk's drain
+
+    }
+}
+
+// ---- CHAIN --------------------------------------------------------------------------------------------
+__device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int bh, int n_chunks, int ct)
+{
+    const int lane = ct & 31, warp = ct >> 5;
+    const int quad = warp & 3, half = warp >> 2;
+    const int c = quad * 32 + lane;            // value channel = TMEM lane
+    const int j0 = half * 32;                  // this warp's complex rows in the state pass
+    const uint32_t tlane = tmem + ((uint32_t)(quad * 32) << 16);
+
+    auto drain_outputs = [&](int jd) {         // rho of chunk jd -> bf16 staging tiles [t][128]
+        const bool want = half ? p.has_o_im != 0 : true;
+        if (want) {
+            __nv_bfloat16 *stage = reinterpret_cast<__nv_bfloat16 *>(
+                smem + (half ? OFF_AQ : OFF_KT) + (jd & 1) * 2 * kTile);
+            const float sgn = half ? -1.f : 1.f;   // o = conj(rho)
+#pragma unroll
+            for (int hc = 0; hc < 2; ++hc) {
+                uint32_t r[32];
+                tmem_ld<32>(tlane + TM_ACC + 64 + 128 * half + 32 * hc, r);
+                tc_wait_ld();
+#pragma unroll
+                for (int t = 0; t < 32; ++t)
+                    stage[(32 * hc + t) * DV + c] = __float2bfloat16_rn(sgn * __uint_as_float(r[t]));
+            }
+        }
+        fence_async_smem();
+        tc_fence_before();
+        mbar_arrive(&mi.bars[B_O_STAGED]);
+    };
+    // One 16-row piece of the state pass: rows j0 + 16 pc .. + 15 (Re and Im), scaled/rotated by (cs, sn).
+    auto state_piece = [&](int pc, int ring, bool first) {
+        uint32_t sre[16], sim[16], pk[8];
+        const int jb = j0 + 16 * pc;
+        if (first) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int jj = jb + i;
+                sre[i] = p.S0 ? __float_as_uint(p.S0[((size_t)bh * DK + 2 * jj) * DV + c]) : 0u;
+                sim[i] = p.S0 ? __float_as_uint(p.S0[((size_t)bh * DK + 2 * jj + 1) * DV + c]) : 0u;
+            }
+        } else {
+            tmem_ld<16>(tlane + TM_S32 + jb, sre);
+            tmem_ld<16>(tlane + TM_S32 + 64 + jb, sim);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float a = mi.aC[ring][jb + i];
+                const float cs = a * mi.closing_cos[ring][jb + i], sn = a * mi.closing_sin[ring][jb + i];
+                const float xr = __uint_as_float(sre[i]), xi = __uint_as_float(sim[i]);
+                sre[i] = __float_as_uint(cs * xr - sn * xi);
+                sim[i] = __float_as_uint(cs * xi + sn * xr);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) pk[i] = pack_bf16(__uint_as_float(sre[2 * i]), __uint_as_float(sre[2 * i + 1]));
+        tmem_st8(tlane + TM_X16 + jb / 2, pk);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) pk[i] = pack_bf16(__uint_as_float(sim[2 * i]), __uint_as_float(sim[2 * i + 1]));
+        tmem_st8(tlane + TM_X16 + 32 + jb / 2, pk);
+        tmem_st<16>(tlane + TM_S32 + jb, sre);
+        tmem_st<16>(tlane + TM_S32 + 64 + jb, sim);
+    };
+    // bf16 A operand from 64 fp32 accumulator columns of this warp's half; `sub_v`: R = V - D1 (Re half only).
+    auto convert_acc = [&](bool sub_v, bool negate, int gate_bar, int gate_k) -> bool {
+        uint32_t pk[32];
+#pragma unroll
+        for (int hc = 0; hc < 2; ++hc) {
+            uint32_t r[32];
+            tmem_ld<32>(tlane + TM_ACC + 128 * half + 32 * hc, r);
+            tc_wait_ld();
+            if (sub_v) {
+                const __nv_bfloat16 *sv = reinterpret_cast<const __nv_bfloat16 *>(smem + OFF_V);
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    pk[16 * hc + i] = pack_bf16(__bfloat162float(sv[(32 * hc + 2 * i) * DV + c]) - __uint_as_float(r[2 * i]),
+                                                __bfloat162float(sv[(32 * hc + 2 * i + 1) * DV + c]) - __uint_as_float(r[2 * i + 1]));
+            } else {
+                const float sgn = negate ? -1.f : 1.f;
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    pk[16 * hc + i] = pack_bf16(sgn * __uint_as_float(r[2 * i]), sgn * __uint_as_float(r[2 * i + 1]));
+            }
+        }
+        if (gate_bar >= 0 && !wait_k(mi, gate_bar, gate_k)) return false;
+        tmem_st<32>(tlane + TM_X16 + 32 * half, pk);
+        tc_wait_st();
+        return true;
+    };
+
+    for (int j = 0; j < n_chunks; ++j) {
+        const int s = j & 1;
+        // ---- state pass: S_0 of this chunk = e^{i phi_C} a_C (accumulated state of the previous chunk)
+        if (j > 0) {
+            if (!wait_k(mi, B_UPD_DONE, j - 1)) return;
+            tc_fence_after();
+        }
+        state_piece(0, (j - 1) & 3, j == 0);
+        state_piece(1, (j - 1) & 3, j == 0);
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(&mi.bars[B_S16_READY]);
+
+        // ---- outputs of the previous chunk, while D1 runs
+        if (j > 0) drain_outputs(j - 1);
+
+        // ---- R = V - D1 -> bf16 A operand (rho_1 still reads S_0 from the same columns: gate on its commit)
+        if (!wait_k(mi, B_D1_DONE, j)) return;
+        if (!wait_k(mi, B_V_FULL, j)) return;
+        tc_fence_after();
+        if (!convert_acc(half == 0, half == 1, s ? B_WQ_FREE1 : B_WQ_FREE0, j >> 1)) return;
+        tc_fence_before();
+        mbar_arrive(&mi.bars[B_R16_READY]);
+
+        // ---- E -> bf16 A operand
+        if (!wait_k(mi, B_E_DONE, j)) return;
+        tc_fence_after();
+        if (!convert_acc(false, false, -1, 0)) return;
+        tc_fence_before();
+        mbar_arrive(&mi.bars[B_E16_READY]);
+    }
+
+    // ---- last chunk: outputs and the final state
+    if (!wait_k(mi, B_UPD_DONE, n_chunks - 1)) return;
+    tc_fence_after();
+    drain_outputs(n_chunks - 1);
+    if (p.S_T) {
+        const int ring = (n_chunks - 1) & 3;
+#pragma unroll
+        for (int pc = 0; pc < 2; ++pc) {
+            uint32_t sre[16], sim[16];
+            const int jb = j0 + 16 * pc;
+            tmem_ld<16>(tlane + TM_S32 + jb, sre);
+            tmem_ld<16>(tlane + TM_S32 + 64 + jb, sim);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int jj = jb + i;
+                const float a = mi.aC[ring][jj];
+                const float cs = a * mi.closing_cos[ring][jj], sn = a * mi.closing_sin[ring][jj];
+                const float xr = __uint_as_float(sre[i]), xi = __uint_as_float(sim[i]);
+                p.S_T[((size_t)bh * DK + 2 * jj) * DV + c] = cs * xr - sn * xi;
+                p.S_T[((size_t)bh * DK + 2 * jj + 1) * DV + c] = cs * xi + sn * xr;
+            }
+        }
+    }
+}
+
+// ---- the kernel ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads, 1)
+sfda_forward_ws_kernel(const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                       const __grid_constant__ CUtensorMap tm_oim, const Params p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    Misc &mi = *reinterpret_cast<Misc *>(smem + OFF_MISC);
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int bh = blockIdx.x, h = bh % p.H, b = bh / p.H;
+    const int n_chunks = (p.T + C - 1) / C;
+
+    if (tid == 0) {
+        auto init = [&](int bar, uint32_t count) { mbar_init(&mi.bars[bar], count); };
+        init(B_PREP_FULL0, kPrepThreads); init(B_PREP_FULL1, kPrepThreads);
+        init(B_KT_FULL0, kPrepThreads); init(B_KT_FULL1, kPrepThreads);
+        init(B_WQ_FREE0, 1); init(B_WQ_FREE1, 1); init(B_KC_FREE, 1);
+        init(B_STORE_DONE0, 1); init(B_STORE_DONE1, 1);
+        init(B_GRAM_FULL, 1); init(B_GRAM_DRAINED, kSolveThreads);
+        init(B_MB_FULL, kSolveThreads); init(B_AQ_FULL0, kSolveThreads); init(B_AQ_FULL1, kSolveThreads);
+        init(B_D1_DONE, 1); init(B_E_DONE, 1); init(B_UPD_DONE, 1);
+        init(B_S16_READY, kChainThreads); init(B_R16_READY, kChainThreads); init(B_E16_READY, kChainThreads);
+        init(B_O_STAGED, kChainThreads); init(B_V_FULL, 1);
+        init(B_SYNC_PREP, kPrepThreads); init(B_SYNC_SOLVE, kSolveThreads);
+        mi.abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&mi.tmem_base)));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = mi.tmem_base;
+
+    if (warp < kChainWarps) {
+        run_chain(smem, mi, tmem, p, bh, n_chunks, tid);
+    } else if (warp < kChainWarps + kSolveWarps) {
+        run_solve(smem, mi, tmem, n_chunks, tid - kChainThreads);
+    } else if (warp < kChainWarps + kSolveWarps + kPrepWarps) {
+        regs_inc<kRegsPrep>();
+        run_prep(smem, mi, p, b, h, n_chunks, tid - kChainThreads - kSolveThreads);
+    } else {
+        regs_dec<kRegsCtrl>();
+        if (tid == kChainThreads + kSolveThreads + kPrepThreads)
+            run_ctrl(smem, mi, tmem, &tm_v, &tm_o, &tm_oim, p, b, h, n_chunks);
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0 && mi.abort) atomicExch(p.status, 1u);
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem));
+}
+
+// ---- host side ----------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = [] {
+        void *f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            f = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(f);
+    }();
+    return fn;
+}
+
+// [B][T][H][128] bf16 tensor, box = 64 tokens of one head.
+bool make_map(CUtensorMap *map, const void *base, int B, int T, int H)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[4] = {(cuuint64_t)DV, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {(cuuint64_t)DV * 2, (cuuint64_t)H * DV * 2, (cuuint64_t)T * H * DV * 2};
+    const cuuint32_t box[4] = {(cuuint32_t)DV, 1, (cuuint32_t)C, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+cudaError_t launch_forward_ws(const ForwardArgs &a, uint32_t *status, cudaStream_t stream, int *launches)
+{
+    CUtensorMap tv, to, toi;
+    if (!make_map(&tv, a.v, a.B, a.T, a.H) || !make_map(&to, a.o, a.B, a.T, a.H) ||
+        !make_map(&toi, a.o_im ? a.o_im : a.o, a.B, a.T, a.H))
+        return cudaErrorInvalidValue;
+    cudaError_t e = cudaFuncSetAttribute(sfda_forward_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(status, 0, sizeof(uint32_t), stream);
+    if (e != cudaSuccess) return e;
+    Params p;
+    p.q = static_cast<const __nv_bfloat16 *>(a.q);
+    p.k = static_cast<const __nv_bfloat16 *>(a.k);
+    p.alpha = a.alpha;
+    p.theta = a.theta;
+    p.beta = a.beta;
+    p.S0 = a.S0;
+    p.S_T = a.S_T;
+    p.status = status;
+    p.T = a.T;
+    p.H = a.H;
+    p.has_o_im = a.o_im != nullptr;
+    sfda_forward_ws_kernel<<<(unsigned)(a.B * a.H), kThreads, kSmemBytes, stream>>>(tv, to, toi, p);
+    e = cudaGetLastError();
+    if (e == cudaSuccess && launches) ++*launches;
+    return e;
+}
+
+}  // namespace sfda
