@@ -20,8 +20,13 @@ __device__ __forceinline__ void st_val(__nv_bfloat16 *p, size_t i, float x) { p[
 __device__ __forceinline__ uint32_t phase_to_turns(float theta)
 {
     const double turns_per_radian = 0x1.45f306dc9c883p+29;  // 2^32 / (2 pi), nearest double
-    const long long r = __double2ll_rn(__dmul_rn((double)theta, turns_per_radian));
-    return (uint32_t)(unsigned long long)r;
+    const double d = __dmul_rn((double)theta, turns_per_radian);
+    if (fabsf(theta) < 1.0e6f) {
+        // |d| < 2^51: adding 1.5 * 2^52 rounds d to an integer (to nearest, ties to even) and leaves that
+        // integer, modulo 2^32, in the low word of the sum -- the same value as the conversion below.
+        return (uint32_t)__double2loint(__dadd_rn(d, 6755399441055744.0));
+    }
+    return (uint32_t)(unsigned long long)__double2ll_rn(d);
 }
 
 // cos / sin of a phase given in turns (signed view keeps the float argument in [-1, 1)).

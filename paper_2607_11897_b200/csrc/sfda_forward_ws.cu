@@ -1,15 +1,15 @@
 // Warp-specialised tensor-core chunk-WY forward for sm_100a: bf16 q/k/v, d_k = d_v = 128, chunk C = 64.
 //
-// One CTA (17 warps) walks the chunks of one (batch, head) pair; four roles run concurrently on
-// different chunks and hand tiles to one another through mbarriers:
+// One CTA walks the chunks of one (batch, head) pair; four roles run concurrently on different chunks
+// and hand tiles to one another through mbarriers:
 //
-//   PREP  (4 warps)  chunk j+1..j+2: cumulative phase-decay gamma_t = a_t e^{i phi_t} (Eq. "constructive-Gamma";
+//   PREP  (4 warps)  chunk j+1: cumulative phase-decay gamma_t = a_t e^{i phi_t} (Eq. "constructive-Gamma";
 //                    log2-sum and integer-turn prefix scans), rotated/decayed operand tiles in shared memory.
 //   SOLVE (4 warps)  chunk j+1: drains the Gram blocks from tensor memory, inverts the unit-lower WY system
 //                    (Eq. "constructive-M": M = (I + L)^{-1}) by 16x16 blocks, writes M_beta and Aq tiles.
 //   CHAIN (8 warps)  chunk j: the state-dependent conversions between the tcgen05 products
 //                    (state pass, R = V - W^* S_0, E, outputs); they own the TMEM <-> register traffic.
-//   CTRL  (1 warp)   one thread issues every tcgen05.mma / commit and the TMA copies.
+//   CTRL  (1 thread) issues every tcgen05.mma / commit and the TMA copies.
 //
 // Algebra (k'_t = e^{-i phi_t} k_t, q'_t = e^{-i phi_t} q_t, all tiles bf16, de-interleaved [Re | Im]):
 //   W_t = a_t k'_t (= conj(gamma_t) k_t, Eq. "constructive-W"),  Qt_t = a_t q'_t,  Kc_t = k'_t / a_t
@@ -32,44 +32,53 @@ namespace {
 using namespace tc;
 
 constexpr int C = 64, DK = 128, DV = 128, M = 64;
-constexpr int kChainWarps = 8, kSolveWarps = 4, kPrepWarps = 4;
+constexpr int kChainWarps = 8, kSolveWarps = 4, kPrepWarps = 8;
 constexpr int kCtrlWarps = 4;   // a full warpgroup, so that it can hand its registers to the others; one thread works
-constexpr int kThreads = 32 * (kChainWarps + kSolveWarps + kPrepWarps + kCtrlWarps);   // 640
-// The CTA is launched with 96 registers per thread (640 * 96 = 61440); the roles then rebalance that pool:
-// 8 * 96 + 4 * 96 + 4 * 128 + 4 * 64 = 1920 warp rows = 61440 registers.
-constexpr int kRegsChain = 96, kRegsSolve = 96, kRegsPrep = 128, kRegsCtrl = 64;
+constexpr int kThreads = 32 * (kChainWarps + kSolveWarps + kPrepWarps + kCtrlWarps);   // 768
 constexpr int kChainThreads = 32 * kChainWarps, kSolveThreads = 32 * kSolveWarps, kPrepThreads = 32 * kPrepWarps;
+// The CTA is launched with 80 registers per thread (768 * 80 = 61440); the working roles take what CTRL gives up:
+// (8 + 4 + 8) * 88 + 4 * 40 = 1920 warp rows = 61440 registers.
+constexpr int kRegsWork = 88, kRegsCtrl = 40;
 
 // ---- shared memory map (bytes from a 1024-aligned base) -------------------------------------------------
-constexpr int kTile = 8192;                       // 64 rows x 128 B, K-major, 128B swizzle
-constexpr int OFF_WQ = 0;                         // [2 slots][re | im][128 rows: W then Qt]      64 KB
-constexpr int OFF_KC = OFF_WQ + 2 * 4 * kTile;    // Kc [i][j], re | im (Gram B operand)          16 KB
-constexpr int OFF_KT = OFF_KC + 2 * kTile;        // [2 slots] Kc^T [j][t], re | im (update B)    32 KB
-constexpr int OFF_MB = OFF_KT + 2 * 2 * kTile;    // M_beta [t][i], re | im                       16 KB
-constexpr int OFF_AQ = OFF_MB + 2 * kTile;        // [2 slots] Aq [t][i], re | im                 32 KB
-constexpr int OFF_V = OFF_AQ + 2 * 2 * kTile;     // v staging [t][128] bf16 (TMA)                16 KB
+constexpr int kTile = 8192;                       // 64 rows x 128 B, 128B swizzle
+constexpr int OFF_WQ = 0;                         // [2 slots][re | im][128 rows: W then Qt], K-major     64 KB
+constexpr int OFF_KC = OFF_WQ + 2 * 4 * kTile;    // [2 slots] Kc [t][j], re | im: K-major B of the Gram, 32 KB
+                                                  //           MN-major B of the state update
+constexpr int OFF_MB = OFF_KC + 2 * 2 * kTile;    // M_beta [t][i], re | im                                16 KB
+constexpr int OFF_AQ = OFF_MB + 2 * kTile;        // [2 slots] Aq [t][i], re | im; also stages o_im        32 KB
+constexpr int OFF_V = OFF_AQ + 2 * 2 * kTile;     // v staging [t][128] bf16 (TMA load)                    16 KB
+constexpr int OFF_OST = OFF_V + 16384;            // o staging [t][128] bf16 (TMA store)                   16 KB
 constexpr int LS = 68;                            // row stride (floats) of the solve scratch
-constexpr int OFF_LX = OFF_V + 16384;             // L -> X in place, fp32 [64][LS], re | im      34 KB
+constexpr int OFF_LX = OFF_OST + 16384;           // L -> X in place, fp32 [64][LS], re | im               34 KB
 constexpr int OFF_MISC = OFF_LX + 2 * 64 * LS * 4;
-constexpr int kSmemBytes = OFF_MISC + 7168 + 1024;
+constexpr int kMiscBytes = 9216;
+constexpr int kSmemBytes = OFF_MISC + kMiscBytes + 1024;   // + slack for the 1024-byte alignment
+static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA exceeded");
 
 enum Bar {
-    B_PREP_FULL0, B_PREP_FULL1, B_KT_FULL0, B_KT_FULL1, B_WQ_FREE0, B_WQ_FREE1, B_KC_FREE, B_STORE_DONE0,
-    B_STORE_DONE1, B_GRAM_FULL, B_GRAM_DRAINED, B_MB_FULL, B_AQ_FULL0, B_AQ_FULL1, B_D1_DONE, B_E_DONE, B_UPD_DONE,
-    B_S16_READY, B_R16_READY, B_E16_READY, B_O_STAGED, B_V_FULL, B_SYNC_PREP, B_SYNC_SOLVE, kNumBars
+    B_PREP_FULL0, B_PREP_FULL1,     // PREP -> CTRL: W/Qt/Kc tiles of the slot are written
+    B_WQ_FREE0, B_WQ_FREE1,         // commit: rho_1 (last reader of the slot's W/Qt tiles) has run
+    B_KC_FREE0, B_KC_FREE1,         // commit: the state update (last reader of the slot's Kc tile) has run
+    B_STORE_DONE0, B_STORE_DONE1,   // CTRL: the output store of a chunk of this parity has read its staging
+    B_GRAM_FULL, B_GRAM_DRAINED,    // commit / SOLVE: one Gram half is in tensor memory / has been read out
+    B_MB_FULL, B_AQ_FULL0, B_AQ_FULL1,
+    B_D1_DONE, B_E_DONE, B_UPD_DONE,
+    B_S16_READY, B_R16_READY, B_E16_READY, B_O_STAGED,
+    B_V_FULL,
+    kNumBars
 };
 
 struct Misc {
-    float part_lg[4][M];
-    uint32_t part_turns[4][M];
-    float aC[4][M], closing_cos[4][M], closing_sin[4][M];   // ring of four chunks
+    float part_lg[8][M];
+    uint32_t part_turns[8][M];
+    float close_re[4][M], close_im[4][M];   // a_C e^{i phi_C} of a ring of four chunks
     float beta[4][C];
     unsigned long long bars[kNumBars];
     uint32_t tmem_base;
     volatile int abort;
 };
-static_assert(sizeof(Misc) <= 7168, "misc area too small");
-static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA exceeded");
+static_assert(sizeof(Misc) <= kMiscBytes, "misc area too small");
 
 // ---- tensor memory map (columns) ----------------------------------------------------------------------
 constexpr uint32_t TM_S32 = 0;      // state fp32 [Re j | Im j]
@@ -77,7 +86,27 @@ constexpr uint32_t TM_X16 = 128;    // bf16 A operand: S_0, then R, then E (64 p
 constexpr uint32_t TM_GRAM = 192;   // Gram half (Re, then Im): lanes 0..63 Kt rows, 64..127 Aq rows
 constexpr uint32_t TM_ACC = 256;    // [D1/E re | rho re | D1/E im | rho im], 64 columns each
 
+// Optional per-role cycle accounting of CTA 0 (development builds only, -DSFDA_WS_TIMING): each role's first
+// thread adds the cycles since its previous mark to slot i.
+#ifdef SFDA_WS_TIMING
+#define SFDA_TDECL(cond) long long tmark_ = clock64(); const bool ton_ = blockIdx.x == 0 && timing != nullptr && (cond)
+#define SFDA_T(i)                                   \
+    do {                                            \
+        if (ton_) {                                 \
+            const long long now_ = clock64();       \
+            timing[i] += now_ - tmark_;             \
+            tmark_ = now_;                          \
+        }                                           \
+    } while (0)
+#else
+#define SFDA_TDECL(cond)
+#define SFDA_T(i) \
+    do {          \
+    } while (0)
+#endif
+
 struct Params {
+    long long *timing;
     const __nv_bfloat16 *q, *k;
     const float *alpha, *theta, *beta, *S0;
     float *S_T;
@@ -89,7 +118,6 @@ __device__ __forceinline__ void mbar_arrive(unsigned long long *bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-
 template <int N>
 __device__ __forceinline__ void regs_inc()
 {
@@ -99,6 +127,21 @@ template <int N>
 __device__ __forceinline__ void regs_dec()
 {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+// Barrier among the threads of one role (hardware barrier `id`); returns the OR of `flag` over the role.
+__device__ __forceinline__ bool role_sync_or(int id, int nthreads, bool flag)
+{
+    uint32_t out;
+    asm volatile(
+        "{\n.reg .pred p, q;\nsetp.ne.b32 q, %3, 0;\nbarrier.cta.red.or.pred p, %1, %2, q;\nselp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(out)
+        : "r"(id), "r"(nthreads), "r"((uint32_t)flag)
+        : "memory");
+    return out != 0;
+}
+__device__ __forceinline__ void role_sync(int id, int nthreads)
+{
+    asm volatile("barrier.cta.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
 __device__ __forceinline__ unsigned long long now_ns()
@@ -120,50 +163,69 @@ __device__ __forceinline__ bool test_k(Misc &mi, int bar, int k)
     return ok != 0;
 }
 // Wait for completion number k; gives up after kWaitLimitNs or when another role has raised the abort flag.
-// Returns false in that case, after raising the flag itself.
+// Returns false in that case, after raising the flag itself.  try_wait parks the thread in hardware for up to
+// the hinted time, so waiting warps do not compete with working ones for issue slots.
 __device__ __forceinline__ bool wait_k(Misc &mi, int bar, int k)
 {
-    if (test_k(mi, bar, k)) return true;
-    const unsigned long long t0 = now_ns();
+    const uint32_t addr = smem_u32(&mi.bars[bar]), parity = (uint32_t)k & 1u;
+    unsigned long long t0 = 0;
     for (uint32_t it = 0;; ++it) {
-        if (test_k(mi, bar, k)) return true;
-        if ((it & 255u) == 255u) {
-            if (mi.abort) return false;
-            if (now_ns() - t0 > kWaitLimitNs) break;
-        }
+        uint32_t ok;
+        asm volatile(
+            "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}\n"
+            : "=r"(ok)
+            : "r"(addr), "r"(parity), "r"(20000u)
+            : "memory");
+        if (ok) return true;
+        if (mi.abort) return false;
+        const unsigned long long t = now_ns();
+        if (it == 0) t0 = t;
+        else if (t - t0 > kWaitLimitNs) break;
     }
     mi.abort = 1;
     return false;
 }
-// Barrier among the threads of one role, with the same bounded wait as everything else (a plain bar.sync
-// could wait forever for a thread that has given up).  `n` counts the calls of the role.
-__device__ __forceinline__ bool group_sync(Misc &mi, int bar, int &n)
-{
-    mbar_arrive(&mi.bars[bar]);
-    return wait_k(mi, bar, n++);
-}
 
 // ---- CTRL: one thread issues all tensor-core and TMA work ------------------------------------------------
-__device__ __forceinline__ void run_ctrl(uint8_t *smem, Misc &mi, uint32_t tmem, const CUtensorMap *tm_v, const CUtensorMap *tm_o,
-                         const CUtensorMap *tm_oim, const Params &p, int b, int h, int n_chunks)
+// Four K = 16 instructions over one 64-element swizzle span.  `b_step` is the descriptor advance per K = 16:
+// 2 (32 bytes) for a K-major operand, 128 (2048 bytes = 16 rows) for an MN-major one.
+__device__ __forceinline__ void mma4_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t id, uint32_t acc, uint32_t b_step = 2)
 {
-    const uint32_t sbase = smem_u32(smem);
-    auto wq = [&](int s, int im) { return sbase + OFF_WQ + (s * 2 + im) * 2 * kTile; };   // 128-row tile
-    auto kc = [&](int im) { return sbase + OFF_KC + im * kTile; };
-    auto kt = [&](int s, int im) { return sbase + OFF_KT + (s * 2 + im) * kTile; };
-    auto mb = [&](int im) { return sbase + OFF_MB + im * kTile; };
-    auto aq = [&](int s, int im) { return sbase + OFF_AQ + (s * 2 + im) * kTile; };
-    unsigned long long *bars = mi.bars;
+    mma_ts(d, a, b, id, acc);
+    mma_ts(d, a + 8, b + b_step, id, 1u);
+    mma_ts(d, a + 16, b + 2 * b_step, id, 1u);
+    mma_ts(d, a + 24, b + 3 * b_step, id, 1u);
+}
+__device__ __forceinline__ void mma4_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t id, uint32_t acc)
+{
+    mma_ss(d, a, b, id, acc);
+    mma_ss(d, a + 2, b + 2, id, 1u);
+    mma_ss(d, a + 4, b + 4, id, 1u);
+    mma_ss(d, a + 6, b + 6, id, 1u);
+}
 
-    auto gram_half = [&](int j, int im) {   // Kt/Aq half into TM_GRAM: rows = [W; Qt] of slot j&1, columns = tokens i
+__device__ __forceinline__ void run_ctrl(uint8_t *smem, Misc &mi, uint32_t tmem, const CUtensorMap *tm_v,
+                                         const CUtensorMap *tm_o, const CUtensorMap *tm_oim, const Params &p, int b,
+                                         int h, int n_chunks)
+{
+    long long *timing = p.timing;
+    const uint64_t dbase = smem_desc(smem_u32(smem));                     // descriptor of byte offset 0
+    auto desc = [&](int off) { return dbase + (uint64_t)(off >> 4); };    // offsets are multiples of 16
+    unsigned long long *bars = mi.bars;
+    constexpr uint32_t I64 = idesc(64, 0), I64N = idesc(64, 1);           // N = 64, B K-major (negated)
+    constexpr uint32_t I64M = idesc(64, 0) | (1u << 16), I64MN = idesc(64, 1) | (1u << 16);   // B MN-major
+
+    auto gram_half = [&](int j, int im) {   // Kt/Aq half: rows = [W; Qt], columns = tokens i
         const int s = j & 1;
+        const uint64_t w_re = desc(OFF_WQ + s * 4 * kTile), w_im = w_re + (2 * kTile >> 4);
+        const uint64_t k_re = desc(OFF_KC + s * 2 * kTile), k_im = k_re + (kTile >> 4);
         const uint32_t d = tmem + TM_GRAM;
         if (!im) {
-            mma_k64_ss(d, wq(s, 0), kc(0), idesc(64, 0), false);
-            mma_k64_ss(d, wq(s, 1), kc(1), idesc(64, 0), true);
+            mma4_ss(d, w_re, k_re, I64, 0u);
+            mma4_ss(d, w_im, k_im, I64, 1u);
         } else {
-            mma_k64_ss(d, wq(s, 0), kc(1), idesc(64, 0), false);
-            mma_k64_ss(d, wq(s, 1), kc(0), idesc(64, 1), true);
+            mma4_ss(d, w_re, k_im, I64, 0u);
+            mma4_ss(d, w_im, k_re, I64N, 1u);
         }
         mma_commit(&bars[B_GRAM_FULL]);
     };
@@ -186,7 +248,6 @@ __device__ __forceinline__ void run_ctrl(uint8_t *smem, Misc &mi, uint32_t tmem,
             if (!test_k(mi, B_GRAM_DRAINED, 2 * g)) return;
             tc_fence_after();
             gram_half(g, 1);
-            mma_commit(&bars[B_KC_FREE]);
             gh = 0;
             ++g;
         }
@@ -207,120 +268,141 @@ __device__ __forceinline__ void run_ctrl(uint8_t *smem, Misc &mi, uint32_t tmem,
     };
 
     const uint32_t x_re = tmem + TM_X16, x_im = tmem + TM_X16 + 32;
+    const uint32_t acc_re = tmem + TM_ACC, rho_re = tmem + TM_ACC + 64, acc_im = tmem + TM_ACC + 128,
+                   rho_im = tmem + TM_ACC + 192;
+    SFDA_TDECL(true);
     for (int j = 0; j < n_chunks; ++j) {
         const int s = j & 1, u = j >> 1;
+        const uint64_t w_re = desc(OFF_WQ + s * 4 * kTile), w_im = w_re + (2 * kTile >> 4);
+        const uint64_t q_re = w_re + (kTile >> 4), q_im = w_im + (kTile >> 4);
+        const uint64_t k_re = desc(OFF_KC + s * 2 * kTile), k_im = k_re + (kTile >> 4);
+        const uint64_t a_re = desc(OFF_AQ + s * 2 * kTile), a_im = a_re + (kTile >> 4);
+        const uint64_t m_re = desc(OFF_MB), m_im = m_re + (kTile >> 4);
         // D1 = W^* S_0
         if (!wait_pump(B_S16_READY, j)) return;
         if (!wait_pump(s ? B_PREP_FULL1 : B_PREP_FULL0, u)) return;
         tc_fence_after();
-        {
-            const uint32_t d_re = tmem + TM_ACC, d_im = tmem + TM_ACC + 128;
-            mma_k64_ts(d_re, x_re, wq(s, 0), idesc(64, 0), false);
-            mma_k64_ts(d_re, x_im, wq(s, 1), idesc(64, 0), true);
-            mma_k64_ts(d_im, x_im, wq(s, 0), idesc(64, 0), false);
-            mma_k64_ts(d_im, x_re, wq(s, 1), idesc(64, 1), true);
-            mma_commit(&bars[B_D1_DONE]);
-        }
+        SFDA_T(0);
+        mma4_ts(acc_re, x_re, w_re, I64, 0u);
+        mma4_ts(acc_re, x_im, w_im, I64, 1u);
+        mma4_ts(acc_im, x_im, w_re, I64, 0u);
+        mma4_ts(acc_im, x_re, w_im, I64N, 1u);
+        mma_commit(&bars[B_D1_DONE]);
+        SFDA_T(1);
         // outputs of the previous chunk are staged: store them; rho is free again
         if (j > 0) {
             if (!wait_pump(B_O_STAGED, j - 1)) return;
             tc_fence_after();
-            const int sp = (j - 1) & 1;
-            tma_store_4d(tm_o, smem + OFF_KT + sp * 2 * kTile, 0, h, (j - 1) * C, b);
-            if (p.has_o_im) tma_store_4d(tm_oim, smem + OFF_AQ + sp * 2 * kTile, 0, h, (j - 1) * C, b);
+            SFDA_T(2);
+            tma_store_4d(tm_o, smem + OFF_OST, 0, h, (j - 1) * C, b);
+            if (p.has_o_im) tma_store_4d(tm_oim, smem + OFF_AQ + ((j - 1) & 1) * 2 * kTile, 0, h, (j - 1) * C, b);
             tma_store_commit();
         }
         // rho_1 = Qt^* S_0
-        {
-            const uint32_t o_re = tmem + TM_ACC + 64, o_im = tmem + TM_ACC + 192;
-            mma_k64_ts(o_re, x_re, wq(s, 0) + kTile, idesc(64, 0), false);
-            mma_k64_ts(o_re, x_im, wq(s, 1) + kTile, idesc(64, 0), true);
-            mma_k64_ts(o_im, x_im, wq(s, 0) + kTile, idesc(64, 0), false);
-            mma_k64_ts(o_im, x_re, wq(s, 1) + kTile, idesc(64, 1), true);
-            mma_commit(&bars[s ? B_WQ_FREE1 : B_WQ_FREE0]);
-        }
+        mma4_ts(rho_re, x_re, q_re, I64, 0u);
+        mma4_ts(rho_re, x_im, q_im, I64, 1u);
+        mma4_ts(rho_im, x_im, q_re, I64, 0u);
+        mma4_ts(rho_im, x_re, q_im, I64N, 1u);
+        mma_commit(&bars[s ? B_WQ_FREE1 : B_WQ_FREE0]);
         pump_gram();
-        if (j > 0) {   // the store of chunk j-1 has read its staging tiles (Kt / Aq of slot (j-1)&1)
+        if (j > 0) {   // by now the store of chunk j-1 has read its staging tiles
             tma_store_wait_read();
             mbar_arrive(&bars[(j - 1) & 1 ? B_STORE_DONE1 : B_STORE_DONE0]);
         }
+        SFDA_T(3);
         // E = M_beta R
         if (!wait_pump(B_R16_READY, j)) return;
+        SFDA_T(4);
         if (!wait_pump(B_MB_FULL, j)) return;
         tc_fence_after();
-        {
-            const uint32_t e_re = tmem + TM_ACC, e_im = tmem + TM_ACC + 128;
-            mma_k64_ts(e_re, x_re, mb(0), idesc(64, 0), false);
-            mma_k64_ts(e_re, x_im, mb(1), idesc(64, 1), true);
-            mma_k64_ts(e_im, x_im, mb(0), idesc(64, 0), false);
-            mma_k64_ts(e_im, x_re, mb(1), idesc(64, 0), true);
-            mma_commit(&bars[B_E_DONE]);
-        }
+        SFDA_T(5);
+        mma4_ts(acc_re, x_re, m_re, I64, 0u);
+        mma4_ts(acc_re, x_im, m_im, I64N, 1u);
+        mma4_ts(acc_im, x_im, m_re, I64, 0u);
+        mma4_ts(acc_im, x_re, m_im, I64, 1u);
+        mma_commit(&bars[B_E_DONE]);
         if (j + 1 < n_chunks) {   // v of chunk j has been consumed
             mbar_expect_tx(&bars[B_V_FULL], 16384);
             tma_load_4d(smem + OFF_V, tm_v, &bars[B_V_FULL], 0, h, (j + 1) * C, b);
         }
         pump_gram();
-        // S += E^T Kc ,  rho += Aq E
+        SFDA_T(6);
+        // S += E^T Kc (Kc as MN-major B: rows = tokens) ,  rho += Aq E
         if (!wait_pump(B_E16_READY, j)) return;
-        if (!wait_pump(s ? B_KT_FULL1 : B_KT_FULL0, u)) return;
+        SFDA_T(7);
         if (!wait_pump(s ? B_AQ_FULL1 : B_AQ_FULL0, u)) return;
         tc_fence_after();
-        {
-            const uint32_t s_re = tmem + TM_S32, s_im = tmem + TM_S32 + 64;
-            mma_k64_ts(s_re, x_re, kt(s, 0), idesc(64, 0), true);
-            mma_k64_ts(s_re, x_im, kt(s, 1), idesc(64, 1), true);
-            mma_k64_ts(s_im, x_re, kt(s, 1), idesc(64, 0), true);
-            mma_k64_ts(s_im, x_im, kt(s, 0), idesc(64, 0), true);
-            const uint32_t o_re = tmem + TM_ACC + 64, o_im = tmem + TM_ACC + 192;
-            mma_k64_ts(o_re, x_re, aq(s, 0), idesc(64, 0), true);
-            mma_k64_ts(o_re, x_im, aq(s, 1), idesc(64, 1), true);
-            mma_k64_ts(o_im, x_im, aq(s, 0), idesc(64, 0), true);
-            mma_k64_ts(o_im, x_re, aq(s, 1), idesc(64, 0), true);
-            mma_commit(&bars[B_UPD_DONE]);
-        }
+        SFDA_T(8);
+        mma4_ts(tmem + TM_S32, x_re, k_re, I64M, 1u, 128);
+        mma4_ts(tmem + TM_S32, x_im, k_im, I64MN, 1u, 128);
+        mma4_ts(tmem + TM_S32 + 64, x_re, k_im, I64M, 1u, 128);
+        mma4_ts(tmem + TM_S32 + 64, x_im, k_re, I64M, 1u, 128);
+        mma_commit(&bars[s ? B_KC_FREE1 : B_KC_FREE0]);
+        mma4_ts(rho_re, x_re, a_re, I64, 1u);
+        mma4_ts(rho_re, x_im, a_im, I64N, 1u);
+        mma4_ts(rho_im, x_im, a_re, I64, 1u);
+        mma4_ts(rho_im, x_re, a_im, I64, 1u);
+        mma_commit(&bars[B_UPD_DONE]);
         pump_gram();
+        SFDA_T(9);
     }
     if (!wait_pump(B_O_STAGED, n_chunks - 1)) return;
-    {
-        const int sp = (n_chunks - 1) & 1;
-        tma_store_4d(tm_o, smem + OFF_KT + sp * 2 * kTile, 0, h, (n_chunks - 1) * C, b);
-        if (p.has_o_im) tma_store_4d(tm_oim, smem + OFF_AQ + sp * 2 * kTile, 0, h, (n_chunks - 1) * C, b);
-        tma_store_commit();
-    }
+    tma_store_4d(tm_o, smem + OFF_OST, 0, h, (n_chunks - 1) * C, b);
+    if (p.has_o_im) tma_store_4d(tm_oim, smem + OFF_AQ + ((n_chunks - 1) & 1) * 2 * kTile, 0, h, (n_chunks - 1) * C, b);
+    tma_store_commit();
     tma_store_wait_all();
 }
 
 // ---- PREP ---------------------------------------------------------------------------------------------
+// e^{-i phi} from the integer phase: the top 23 bits of the turn count make a float in [1, 2); centred to
+// [-0.5, 0.5) turns it is well inside the accurate range of the fast sine / cosine.
+__device__ __forceinline__ void turns_sincos(uint32_t turns, float *sn, float *cs)
+{
+    float f = __uint_as_float(0x3f800000u | (turns >> 9)) - 1.0f;
+    f -= f >= 0.5f ? 1.0f : 0.0f;
+    __sincosf(f * 6.283185307f, sn, cs);
+}
+
 __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, const Params &p, int b, int h, int n_chunks, int pt)
 {
-    const int jp = pt & 31, tq = pt >> 5;   // channel pair (channels 2jp, 2jp+1), token quarter (16 tokens)
-    int nsync = 0;
+    long long *timing = p.timing;
+    const int jp = pt & 31, tq = pt >> 5;   // channel pair (channels 2jp, 2jp+1), token octet (8 tokens)
+    bool dead = false;
+    SFDA_TDECL(pt == 0);
     for (int j = 0; j < n_chunks; ++j) {
+        if (role_sync_or(2, kPrepThreads, dead || mi.abort)) break;
         const int s = j & 1, ring = j & 3;
         const int t0 = j * C, len = min(C, p.T - t0);
         const size_t row0 = ((size_t)b * p.T + t0) * p.H + h;   // token t of this head: row0 + t * H
+        const int nt = min(8, max(0, len - tq * 8));             // real tokens in this thread's octet
 
-        // pass 1: prefix sums of log2 alpha and of the integer phase over this thread's 16 tokens
-        float lg0[16], lg1[16];
-        uint32_t tu0[16], tu1[16];
-        {
-            float2 al[16], th[16];
+        // all loads of this thread for the chunk, issued together
+        float2 al[8], th[8];
+        uint2 kw[8], qw[8];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int t = tq * 16 + i;
-                if (t < len) {
-                    al[i] = __ldg(reinterpret_cast<const float2 *>(p.alpha + (row0 + (size_t)t * p.H) * M) + jp);
-                    th[i] = __ldg(reinterpret_cast<const float2 *>(p.theta + (row0 + (size_t)t * p.H) * M) + jp);
-                } else {
-                    al[i] = make_float2(1.f, 1.f);
-                    th[i] = make_float2(0.f, 0.f);
-                }
+        for (int i = 0; i < 8; ++i) {
+            const size_t row = row0 + (size_t)(tq * 8 + i) * p.H;
+            al[i] = make_float2(1.f, 1.f);
+            th[i] = make_float2(0.f, 0.f);
+            kw[i] = make_uint2(0u, 0u);
+            qw[i] = make_uint2(0u, 0u);
+            if (i < nt) {
+                al[i] = __ldg(reinterpret_cast<const float2 *>(p.alpha + row * M) + jp);
+                th[i] = __ldg(reinterpret_cast<const float2 *>(p.theta + row * M) + jp);
+                kw[i] = __ldg(reinterpret_cast<const uint2 *>(p.k + row * DK) + jp);
+                qw[i] = __ldg(reinterpret_cast<const uint2 *>(p.q + row * DK) + jp);
             }
+        }
+        if (pt < C) mi.beta[ring][pt] = pt < len ? __ldg(p.beta + row0 + (size_t)pt * p.H) : 0.f;
+
+        // pass 1: prefix sums of log2 alpha and of the integer phase over this thread's 8 tokens
+        float lg0[8], lg1[8];
+        uint32_t tu0[8], tu1[8];
+        {
             float a0 = 0.f, a1 = 0.f;
             uint32_t u0 = 0u, u1 = 0u;
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
+            for (int i = 0; i < 8; ++i) {
                 a0 += fmaxf(__log2f(al[i].x), -43.28f);   // floor e^-30, as in log_decay
                 a1 += fmaxf(__log2f(al[i].y), -43.28f);
                 u0 += phase_to_turns(th[i].x);
@@ -332,56 +414,52 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, const Params &
             mi.part_turns[tq][2 * jp] = u0;
             mi.part_turns[tq][2 * jp + 1] = u1;
         }
-        if (!group_sync(mi, B_SYNC_PREP, nsync)) return;
+        SFDA_T(30);
+        role_sync(2, kPrepThreads);
         float base0 = 0.f, base1 = 0.f, tot0 = 0.f, tot1 = 0.f;
         uint32_t tb0 = 0u, tb1 = 0u, tt0 = 0u, tt1 = 0u;
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            const float2 pl = *reinterpret_cast<const float2 *>(&mi.part_lg[g][2 * jp]);
-            const uint2 pu = *reinterpret_cast<const uint2 *>(&mi.part_turns[g][2 * jp]);
-            if (g < tq) { base0 += pl.x; base1 += pl.y; tb0 += pu.x; tb1 += pu.y; }
+        for (int gq = 0; gq < 8; ++gq) {
+            const float2 pl = *reinterpret_cast<const float2 *>(&mi.part_lg[gq][2 * jp]);
+            const uint2 pu = *reinterpret_cast<const uint2 *>(&mi.part_turns[gq][2 * jp]);
+            if (gq < tq) { base0 += pl.x; base1 += pl.y; tb0 += pu.x; tb1 += pu.y; }
             tot0 += pl.x; tot1 += pl.y; tt0 += pu.x; tt1 += pu.y;
         }
-        if (!group_sync(mi, B_SYNC_PREP, nsync)) return;   // partials may be overwritten from here on
-        if (tq == 0) {                    // chunk totals: a_C and the closing phase e^{i phi_C}
+        if (tq == 0) {                    // chunk totals: a_C e^{i phi_C}, applied by the next state pass
             float cs, sn;
-            mi.aC[ring][2 * jp] = exp2f(tot0);
-            mi.aC[ring][2 * jp + 1] = exp2f(tot1);
-            __sincosf((float)(int32_t)tt0 * 0x1.921fb6p-30f, &sn, &cs);   // turns * 2 pi / 2^32
-            mi.closing_cos[ring][2 * jp] = cs;
-            mi.closing_sin[ring][2 * jp] = sn;
-            __sincosf((float)(int32_t)tt1 * 0x1.921fb6p-30f, &sn, &cs);
-            mi.closing_cos[ring][2 * jp + 1] = cs;
-            mi.closing_sin[ring][2 * jp + 1] = sn;
+            const float a0 = exp2f(tot0), a1 = exp2f(tot1);
+            turns_sincos(tt0, &sn, &cs);
+            mi.close_re[ring][2 * jp] = a0 * cs;
+            mi.close_im[ring][2 * jp] = a0 * sn;
+            turns_sincos(tt1, &sn, &cs);
+            mi.close_re[ring][2 * jp + 1] = a1 * cs;
+            mi.close_im[ring][2 * jp + 1] = a1 * sn;
         }
-        if (pt < C) mi.beta[ring][pt] = pt < len ? __ldg(p.beta + row0 + (size_t)pt * p.H) : 0.f;
+        SFDA_T(31);
 
-        // the W/Qt tiles of this slot and the Kc tile must have been consumed
-        if (j >= 2 && !wait_k(mi, s ? B_WQ_FREE1 : B_WQ_FREE0, (j >> 1) - 1)) return;
-        if (j >= 1 && !wait_k(mi, B_KC_FREE, j - 1)) return;
+        // the slot's tiles must have been consumed: W/Qt by rho_1 of chunk j-2, Kc by its state update
+        if (j >= 2) {
+            if (!dead && !wait_k(mi, s ? B_WQ_FREE1 : B_WQ_FREE0, (j >> 1) - 1)) dead = true;
+            if (!dead && !wait_k(mi, s ? B_KC_FREE1 : B_KC_FREE0, (j >> 1) - 1)) dead = true;
+        }
+        SFDA_T(32);
 
-        // pass 2a: rotated / decayed operands
-        uint8_t *wq_re = smem + OFF_WQ + (s * 2) * 2 * kTile, *wq_im = wq_re + 2 * kTile;
-        uint8_t *kc_re = smem + OFF_KC, *kc_im = kc_re + kTile;
-        uint32_t k0r[8], k0i[8], k1r[8], k1i[8];   // Kc^T rows 2jp and 2jp+1, 16 tokens, packed bf16 pairs
+        // pass 2: rotated / decayed operands
+        uint8_t *wq_re = smem + OFF_WQ + s * 4 * kTile, *wq_im = wq_re + 2 * kTile;
+        uint8_t *kc_re = smem + OFF_KC + s * 2 * kTile, *kc_im = kc_re + kTile;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const int t = tq * 16 + i;
-            uint2 kw = make_uint2(0u, 0u), qw = make_uint2(0u, 0u);
-            if (t < len) {
-                kw = __ldg(reinterpret_cast<const uint2 *>(p.k + (row0 + (size_t)t * p.H) * DK) + jp);
-                qw = __ldg(reinterpret_cast<const uint2 *>(p.q + (row0 + (size_t)t * p.H) * DK) + jp);
-            }
+        for (int i = 0; i < 8; ++i) {
+            const int t = tq * 8 + i;
             float wr[2], wi[2], cr_[2], ci_[2], qr_[2], qi_[2];
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
                 const float l2 = x ? base1 + lg1[i] : base0 + lg0[i];
                 const uint32_t tu = x ? tb1 + tu1[i] : tb0 + tu0[i];
-                const uint32_t kx = x ? kw.y : kw.x, qx = x ? qw.y : qw.x;
+                const uint32_t kx = x ? kw[i].y : kw[i].x, qx = x ? qw[i].y : qw[i].x;
                 const float a = exp2f(l2);
                 const float ainv = exp2f(fminf(-l2, 115.4f));                 // 1/a_t, capped at e^80
                 float cs, sn;
-                __sincosf((float)(int32_t)tu * 0x1.921fb6p-30f, &sn, &cs);
+                turns_sincos(tu, &sn, &cs);
                 const float kr = __uint_as_float(kx << 16), ki = __uint_as_float(kx & 0xffff0000u);
                 const float qr = __uint_as_float(qx << 16), qi = __uint_as_float(qx & 0xffff0000u);
                 const float kpr = kr * cs + ki * sn, kpi = ki * cs - kr * sn;   // e^{-i phi} k
@@ -397,55 +475,36 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, const Params &
             *reinterpret_cast<uint32_t *>(wq_im + kTile + o1) = pack_bf16(qi_[0], qi_[1]);
             *reinterpret_cast<uint32_t *>(kc_re + o1) = pack_bf16(cr_[0], cr_[1]);
             *reinterpret_cast<uint32_t *>(kc_im + o1) = pack_bf16(ci_[0], ci_[1]);
-            const uint32_t h0r = __bfloat16_as_ushort(__float2bfloat16_rn(cr_[0]));
-            const uint32_t h0i = __bfloat16_as_ushort(__float2bfloat16_rn(ci_[0]));
-            const uint32_t h1r = __bfloat16_as_ushort(__float2bfloat16_rn(cr_[1]));
-            const uint32_t h1i = __bfloat16_as_ushort(__float2bfloat16_rn(ci_[1]));
-            if (i & 1) {
-                k0r[i >> 1] |= h0r << 16; k0i[i >> 1] |= h0i << 16;
-                k1r[i >> 1] |= h1r << 16; k1i[i >> 1] |= h1i << 16;
-            } else {
-                k0r[i >> 1] = h0r; k0i[i >> 1] = h0i;
-                k1r[i >> 1] = h1r; k1i[i >> 1] = h1i;
-            }
         }
         fence_async_smem();
         mbar_arrive(&mi.bars[s ? B_PREP_FULL1 : B_PREP_FULL0]);
-
-        // pass 2b: Kc^T once the slot's previous occupant (update operand, then output staging) is done with
-        if (j >= 2 && !wait_k(mi, s ? B_STORE_DONE1 : B_STORE_DONE0, (j >> 1) - 1)) return;
-        uint8_t *kt_re = smem + OFF_KT + (s * 2) * kTile, *kt_im = kt_re + kTile;
-#pragma unroll
-        for (int cidx = 0; cidx < 2; ++cidx) {
-            const int oa = sw_off(2 * jp, tq * 16 + cidx * 8), ob = sw_off(2 * jp + 1, tq * 16 + cidx * 8);
-            *reinterpret_cast<uint4 *>(kt_re + oa) = make_uint4(k0r[4 * cidx], k0r[4 * cidx + 1], k0r[4 * cidx + 2], k0r[4 * cidx + 3]);
-            *reinterpret_cast<uint4 *>(kt_im + oa) = make_uint4(k0i[4 * cidx], k0i[4 * cidx + 1], k0i[4 * cidx + 2], k0i[4 * cidx + 3]);
-            *reinterpret_cast<uint4 *>(kt_re + ob) = make_uint4(k1r[4 * cidx], k1r[4 * cidx + 1], k1r[4 * cidx + 2], k1r[4 * cidx + 3]);
-            *reinterpret_cast<uint4 *>(kt_im + ob) = make_uint4(k1i[4 * cidx], k1i[4 * cidx + 1], k1i[4 * cidx + 2], k1i[4 * cidx + 3]);
-        }
-        fence_async_smem();
-        mbar_arrive(&mi.bars[s ? B_KT_FULL1 : B_KT_FULL0]);
+        SFDA_T(33);
     }
 }
 
 // ---- SOLVE --------------------------------------------------------------------------------------------
-__device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem, int n_chunks, int st)
+__device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int n_chunks, int st)
 {
+    long long *timing = p.timing;
     const int lane = st & 31, w = st >> 5;    // w = TMEM lane quadrant of this warp
     float *Lr = reinterpret_cast<float *>(smem + OFF_LX), *Li = Lr + 64 * LS;
     const uint32_t tlane = tmem + ((uint32_t)(w * 32) << 16);
     const int row = w * 32 + lane;            // Gram row held by this thread: < 64 -> Kt row, else Aq row
-    int nsync = 0;
+    bool dead = false;
+    SFDA_TDECL(st == 0);
     for (int j = 0; j < n_chunks; ++j) {
+        if (role_sync_or(1, kSolveThreads, dead || mi.abort)) break;   // also: scratch of the last chunk is free
         const int s = j & 1, ring = j & 3;
-        // The Aq tile of this slot also staged the outputs of chunk j-2: its rows are written straight from the
-        // drain, so the warps that hold them wait for that store first.
-        if (row >= 64 && j >= 2 && !wait_k(mi, s ? B_STORE_DONE1 : B_STORE_DONE0, (j >> 1) - 1)) return;
+        // The Aq tile of this slot also staged o_im of chunk j-2: its rows are written straight from the drain,
+        // so the warps that hold them wait for that store first.
+        if (row >= 64 && j >= 2 && !dead && !wait_k(mi, s ? B_STORE_DONE1 : B_STORE_DONE0, (j >> 1) - 1)) dead = true;
         // ---- drain the two Gram halves
 #pragma unroll
         for (int im = 0; im < 2; ++im) {
-            if (!wait_k(mi, B_GRAM_FULL, 2 * j + im)) return;
+            SFDA_T(20 + 2 * im);
+            if (!dead && !wait_k(mi, B_GRAM_FULL, 2 * j + im)) dead = true;
             tc_fence_after();
+            SFDA_T(21 + 2 * im);
 #pragma unroll
             for (int hc = 0; hc < 2; ++hc) {      // 32 columns at a time keeps the register footprint down
                 uint32_t r[32];
@@ -486,48 +545,51 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
         }
         fence_async_smem();
         mbar_arrive(&mi.bars[s ? B_AQ_FULL1 : B_AQ_FULL0]);
-        if (!group_sync(mi, B_SYNC_SOLVE, nsync)) return;
+        role_sync(1, kSolveThreads);
+        SFDA_T(24);
 
-        // ---- X = (I + L)^{-1} in place: diagonal 16x16 blocks by substitution, merges on mma.sync
-        if (lane < 16) {                      // warp w inverts diagonal block w, lane = column
+        // ---- X = (I + L)^{-1} in place.  Diagonal 16x16 blocks: warp w, lane = column c solves (I + L) x = e_c
+        // right-looking (after x_i is final, every later row is updated at once: independent operations).
+        if (lane < 16) {
             const int o = 16 * w, c = lane;
             float xr[16], xi[16];
 #pragma unroll
             for (int r = 0; r < 16; ++r) {
-                float ar = r == c ? 1.f : 0.f, ai = 0.f;
-#pragma unroll
-                for (int i = 0; i < 15; ++i) {
-                    if (i < r) {
-                        const float lr_ = Lr[(o + r) * LS + o + i], li_ = Li[(o + r) * LS + o + i];
-                        const float vr = i >= c ? xr[i] : 0.f, vi = i >= c ? xi[i] : 0.f;
-                        ar -= lr_ * vr - li_ * vi;
-                        ai -= lr_ * vi + li_ * vr;
-                    }
-                }
-                xr[r] = r >= c ? ar : 0.f;
-                xi[r] = r >= c ? ai : 0.f;
+                xr[r] = r == c ? 1.f : 0.f;
+                xi[r] = 0.f;
             }
-            __syncwarp(0x0000ffffu);          // every lane has read its L rows before the block is overwritten
+#pragma unroll
+            for (int i = 0; i < 15; ++i) {
+                const float vr = xr[i], vi = xi[i];      // zero above the diagonal (i < c)
+#pragma unroll
+                for (int r = i + 1; r < 16; ++r) {
+                    const float lr_ = Lr[(o + r) * LS + o + i], li_ = Li[(o + r) * LS + o + i];
+                    xr[r] -= lr_ * vr - li_ * vi;
+                    xi[r] -= lr_ * vi + li_ * vr;
+                }
+            }
+            __syncwarp(0x0000ffffu);          // every lane has read its L block before it is overwritten
 #pragma unroll
             for (int r = 0; r < 16; ++r) {
                 Lr[(o + r) * LS + o + c] = xr[r];
                 Li[(o + r) * LS + o + c] = xi[r];
             }
         }
-        if (!group_sync(mi, B_SYNC_SOLVE, nsync)) return;
+        role_sync(1, kSolveThreads);
+        SFDA_T(25);
         {   // level 1: X[b1][b0] = -X[b1][b1] (L[b1][b0] X[b0][b0]); T in the unused block above the diagonal
             const int pr = w >> 1, nt = w & 1;
             const int r0 = 32 * pr + 16, c0 = 32 * pr;
             float cr[4] = {0.f, 0.f, 0.f, 0.f}, ci[4] = {0.f, 0.f, 0.f, 0.f};
             cmma_16x8(cr, ci, Lr, Li, LS, r0, c0, Lr, Li, LS, c0, c0 + 8 * nt, nt, 2, lane);
             store_tile(cr, ci, 1.f, Lr, Li, LS, c0, r0 + 8 * nt, lane);          // T at block (b0, b1)
-            if (!group_sync(mi, B_SYNC_SOLVE, nsync)) return;
+            role_sync(1, kSolveThreads);
             float dr[4] = {0.f, 0.f, 0.f, 0.f}, di[4] = {0.f, 0.f, 0.f, 0.f};
             cmma_16x8(dr, di, Lr, Li, LS, r0, r0, Lr, Li, LS, c0, r0 + 8 * nt, 0, 2, lane);
-            if (!group_sync(mi, B_SYNC_SOLVE, nsync)) return;                                     // L[b1][b0] fully read
             store_tile(dr, di, -1.f, Lr, Li, LS, r0, c0 + 8 * nt, lane);
         }
-        if (!group_sync(mi, B_SYNC_SOLVE, nsync)) return;
+        role_sync(1, kSolveThreads);
+        SFDA_T(26);
         {   // level 2: X[BL] = -X[BR] (L[BL] X[TL]); T in the top-right quadrant; warp w owns column tile w
             const int nt = w;
             float c0r[4] = {0.f, 0.f, 0.f, 0.f}, c0i[4] = {0.f, 0.f, 0.f, 0.f};
@@ -536,19 +598,20 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
             cmma_16x8(c1r, c1i, Lr, Li, LS, 48, 0, Lr, Li, LS, 0, 8 * nt, nt, 4, lane);
             store_tile(c0r, c0i, 1.f, Lr, Li, LS, 0, 32 + 8 * nt, lane);
             store_tile(c1r, c1i, 1.f, Lr, Li, LS, 16, 32 + 8 * nt, lane);
-            if (!group_sync(mi, B_SYNC_SOLVE, nsync)) return;
+            role_sync(1, kSolveThreads);
             float d0r[4] = {0.f, 0.f, 0.f, 0.f}, d0i[4] = {0.f, 0.f, 0.f, 0.f};
             float d1r[4] = {0.f, 0.f, 0.f, 0.f}, d1i[4] = {0.f, 0.f, 0.f, 0.f};
             cmma_16x8(d0r, d0i, Lr, Li, LS, 32, 32, Lr, Li, LS, 0, 32 + 8 * nt, 0, 2, lane);
             cmma_16x8(d1r, d1i, Lr, Li, LS, 48, 32, Lr, Li, LS, 0, 32 + 8 * nt, 0, 4, lane);
-            if (!group_sync(mi, B_SYNC_SOLVE, nsync)) return;                                     // L[BL] fully read
             store_tile(d0r, d0i, -1.f, Lr, Li, LS, 32, 8 * nt, lane);
             store_tile(d1r, d1i, -1.f, Lr, Li, LS, 48, 8 * nt, lane);
         }
-        if (!group_sync(mi, B_SYNC_SOLVE, nsync)) return;
+        role_sync(1, kSolveThreads);
+        SFDA_T(27);
 
         // ---- M_beta = X D_beta as a bf16 operand tile, once E of the previous chunk has read the old one
-        if (j >= 1 && !wait_k(mi, B_E_DONE, j - 1)) return;
+        if (j >= 1 && !dead && !wait_k(mi, B_E_DONE, j - 1)) dead = true;
+        SFDA_T(28);
         {
             const int t = st >> 1, part = st & 1;   // row t, columns 32 part .. 32 part + 31
 #pragma unroll
@@ -569,25 +632,28 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
         }
         fence_async_smem();
         mbar_arrive(&mi.bars[B_MB_FULL]);
-        if (!group_sync(mi, B_SYNC_SOLVE, nsync)) return;      // the scratch may be overwritten by the next chunk's drain
-
+        SFDA_T(29);
     }
 }
 
 // ---- CHAIN --------------------------------------------------------------------------------------------
-__device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int bh, int n_chunks, int ct)
+__device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int bh, int n_chunks,
+                                          int ct)
 {
+    long long *timing = p.timing;
     const int lane = ct & 31, warp = ct >> 5;
     const int quad = warp & 3, half = warp >> 2;
     const int c = quad * 32 + lane;            // value channel = TMEM lane
     const int j0 = half * 32;                  // this warp's complex rows in the state pass
     const uint32_t tlane = tmem + ((uint32_t)(quad * 32) << 16);
 
-    auto drain_outputs = [&](int jd) {         // rho of chunk jd -> bf16 staging tiles [t][128]
+    auto drain_outputs = [&](int jd) -> bool {   // rho of chunk jd -> bf16 staging tiles [t][128]
         const bool want = half ? p.has_o_im != 0 : true;
+        // the Re staging tile is shared by all chunks: the store of chunk jd-1 must have read it
+        if (jd >= 1 && !wait_k(mi, (jd - 1) & 1 ? B_STORE_DONE1 : B_STORE_DONE0, (jd - 1) >> 1)) return false;
         if (want) {
-            __nv_bfloat16 *stage = reinterpret_cast<__nv_bfloat16 *>(
-                smem + (half ? OFF_AQ : OFF_KT) + (jd & 1) * 2 * kTile);
+            __nv_bfloat16 *stage =
+                reinterpret_cast<__nv_bfloat16 *>(smem + (half ? OFF_AQ + (jd & 1) * 2 * kTile : OFF_OST));
             const float sgn = half ? -1.f : 1.f;   // o = conj(rho)
 #pragma unroll
             for (int hc = 0; hc < 2; ++hc) {
@@ -602,8 +668,9 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
         fence_async_smem();
         tc_fence_before();
         mbar_arrive(&mi.bars[B_O_STAGED]);
+        return true;
     };
-    // One 16-row piece of the state pass: rows j0 + 16 pc .. + 15 (Re and Im), scaled/rotated by (cs, sn).
+    // One 16-row piece of the state pass: rows j0 + 16 pc .. + 15 (Re and Im).
     auto state_piece = [&](int pc, int ring, bool first) {
         uint32_t sre[16], sim[16], pk[8];
         const int jb = j0 + 16 * pc;
@@ -620,8 +687,7 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
             tc_wait_ld();
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
-                const float a = mi.aC[ring][jb + i];
-                const float cs = a * mi.closing_cos[ring][jb + i], sn = a * mi.closing_sin[ring][jb + i];
+                const float cs = mi.close_re[ring][jb + i], sn = mi.close_im[ring][jb + i];
                 const float xr = __uint_as_float(sre[i]), xi = __uint_as_float(sim[i]);
                 sre[i] = __float_as_uint(cs * xr - sn * xi);
                 sim[i] = __float_as_uint(cs * xi + sn * xr);
@@ -663,6 +729,7 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
         return true;
     };
 
+    SFDA_TDECL(ct == 0);
     for (int j = 0; j < n_chunks; ++j) {
         const int s = j & 1;
         // ---- state pass: S_0 of this chunk = e^{i phi_C} a_C (accumulated state of the previous chunk)
@@ -670,35 +737,42 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
             if (!wait_k(mi, B_UPD_DONE, j - 1)) return;
             tc_fence_after();
         }
+        SFDA_T(10);
         state_piece(0, (j - 1) & 3, j == 0);
         state_piece(1, (j - 1) & 3, j == 0);
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(&mi.bars[B_S16_READY]);
+        SFDA_T(11);
 
         // ---- outputs of the previous chunk, while D1 runs
-        if (j > 0) drain_outputs(j - 1);
+        if (j > 0 && !drain_outputs(j - 1)) return;
+        SFDA_T(12);
 
         // ---- R = V - D1 -> bf16 A operand (rho_1 still reads S_0 from the same columns: gate on its commit)
         if (!wait_k(mi, B_D1_DONE, j)) return;
         if (!wait_k(mi, B_V_FULL, j)) return;
         tc_fence_after();
+        SFDA_T(13);
         if (!convert_acc(half == 0, half == 1, s ? B_WQ_FREE1 : B_WQ_FREE0, j >> 1)) return;
         tc_fence_before();
         mbar_arrive(&mi.bars[B_R16_READY]);
+        SFDA_T(14);
 
         // ---- E -> bf16 A operand
         if (!wait_k(mi, B_E_DONE, j)) return;
         tc_fence_after();
+        SFDA_T(15);
         if (!convert_acc(false, false, -1, 0)) return;
         tc_fence_before();
         mbar_arrive(&mi.bars[B_E16_READY]);
+        SFDA_T(16);
     }
 
     // ---- last chunk: outputs and the final state
     if (!wait_k(mi, B_UPD_DONE, n_chunks - 1)) return;
     tc_fence_after();
-    drain_outputs(n_chunks - 1);
+    if (!drain_outputs(n_chunks - 1)) return;
     if (p.S_T) {
         const int ring = (n_chunks - 1) & 3;
 #pragma unroll
@@ -711,8 +785,7 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
                 const int jj = jb + i;
-                const float a = mi.aC[ring][jj];
-                const float cs = a * mi.closing_cos[ring][jj], sn = a * mi.closing_sin[ring][jj];
+                const float cs = mi.close_re[ring][jj], sn = mi.close_im[ring][jj];
                 const float xr = __uint_as_float(sre[i]), xi = __uint_as_float(sim[i]);
                 p.S_T[((size_t)bh * DK + 2 * jj) * DV + c] = cs * xr - sn * xi;
                 p.S_T[((size_t)bh * DK + 2 * jj + 1) * DV + c] = cs * xi + sn * xr;
@@ -737,15 +810,13 @@ sfda_forward_ws_kernel(const __grid_constant__ CUtensorMap tm_v, const __grid_co
     if (tid == 0) {
         auto init = [&](int bar, uint32_t count) { mbar_init(&mi.bars[bar], count); };
         init(B_PREP_FULL0, kPrepThreads); init(B_PREP_FULL1, kPrepThreads);
-        init(B_KT_FULL0, kPrepThreads); init(B_KT_FULL1, kPrepThreads);
-        init(B_WQ_FREE0, 1); init(B_WQ_FREE1, 1); init(B_KC_FREE, 1);
+        init(B_WQ_FREE0, 1); init(B_WQ_FREE1, 1); init(B_KC_FREE0, 1); init(B_KC_FREE1, 1);
         init(B_STORE_DONE0, 1); init(B_STORE_DONE1, 1);
         init(B_GRAM_FULL, 1); init(B_GRAM_DRAINED, kSolveThreads);
         init(B_MB_FULL, kSolveThreads); init(B_AQ_FULL0, kSolveThreads); init(B_AQ_FULL1, kSolveThreads);
         init(B_D1_DONE, 1); init(B_E_DONE, 1); init(B_UPD_DONE, 1);
         init(B_S16_READY, kChainThreads); init(B_R16_READY, kChainThreads); init(B_E16_READY, kChainThreads);
         init(B_O_STAGED, kChainThreads); init(B_V_FULL, 1);
-        init(B_SYNC_PREP, kPrepThreads); init(B_SYNC_SOLVE, kSolveThreads);
         mi.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -759,11 +830,13 @@ sfda_forward_ws_kernel(const __grid_constant__ CUtensorMap tm_v, const __grid_co
     const uint32_t tmem = mi.tmem_base;
 
     if (warp < kChainWarps) {
+        regs_inc<kRegsWork>();
         run_chain(smem, mi, tmem, p, bh, n_chunks, tid);
     } else if (warp < kChainWarps + kSolveWarps) {
-        run_solve(smem, mi, tmem, n_chunks, tid - kChainThreads);
+        regs_inc<kRegsWork>();
+        run_solve(smem, mi, tmem, p, n_chunks, tid - kChainThreads);
     } else if (warp < kChainWarps + kSolveWarps + kPrepWarps) {
-        regs_inc<kRegsPrep>();
+        regs_inc<kRegsWork>();
         run_prep(smem, mi, p, b, h, n_chunks, tid - kChainThreads - kSolveThreads);
     } else {
         regs_dec<kRegsCtrl>();
@@ -778,6 +851,8 @@ sfda_forward_ws_kernel(const __grid_constant__ CUtensorMap tm_v, const __grid_co
 }
 
 // ---- host side ----------------------------------------------------------------------------------------
+long long *g_ws_timing = nullptr;   // set by development probes built with -DSFDA_WS_TIMING
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -822,6 +897,7 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, uint32_t *status, cudaStream
     e = cudaMemsetAsync(status, 0, sizeof(uint32_t), stream);
     if (e != cudaSuccess) return e;
     Params p;
+    p.timing = g_ws_timing;
     p.q = static_cast<const __nv_bfloat16 *>(a.q);
     p.k = static_cast<const __nv_bfloat16 *>(a.k);
     p.alpha = a.alpha;

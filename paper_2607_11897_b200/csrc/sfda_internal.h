@@ -37,6 +37,7 @@ cudaError_t launch_forward_simt(const ForwardArgs &a, cudaStream_t stream, int *
 bool forward_tc_supported(const ForwardArgs &a);
 cudaError_t launch_forward_tc(const ForwardArgs &a, uint32_t *status, cudaStream_t stream, int *launches);
 // Warp-specialised, chunk-pipelined version of the same path (the one sfda_forward uses).
+bool forward_ws_supported(const ForwardArgs &a);
 cudaError_t launch_forward_ws(const ForwardArgs &a, uint32_t *status, cudaStream_t stream, int *launches);
 cudaError_t launch_chunk_factors(const FactorArgs &a, cudaStream_t stream, int *launches);
 cudaError_t launch_step(const StepArgs &a, cudaStream_t stream, int *launches);
