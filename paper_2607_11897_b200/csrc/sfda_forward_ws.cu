@@ -187,170 +187,169 @@ __device__ __forceinline__ bool wait_k(Misc &mi, int bar, int k)
 }
 
 // ---- CTRL: one thread issues all tensor-core and TMA work ------------------------------------------------
-// Four K = 16 instructions over one 64-element swizzle span.  `b_step` is the descriptor advance per K = 16:
-// 2 (32 bytes) for a K-major operand, 128 (2048 bytes = 16 rows) for an MN-major one.
-__device__ __forceinline__ void mma4_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t id, uint32_t acc, uint32_t b_step = 2)
+// Four K = 16 instructions over one 64-element swizzle span; `b` is the low half of the operand's descriptor,
+// `hi` the (common) high half.  `b_step` is the descriptor advance per K = 16: 2 (32 bytes) for a K-major
+// operand, 128 (2048 bytes = 16 rows) for an MN-major one.
+__device__ __forceinline__ void mma4_ts(uint32_t d, uint32_t a, uint32_t b, uint32_t hi, uint32_t id, uint32_t acc,
+                                        uint32_t b_step = 2)
 {
-    mma_ts(d, a, b, id, acc);
-    mma_ts(d, a + 8, b + b_step, id, 1u);
-    mma_ts(d, a + 16, b + 2 * b_step, id, 1u);
-    mma_ts(d, a + 24, b + 3 * b_step, id, 1u);
+    mma_ts2(d, a, b, hi, id, acc);
+    mma_ts2(d, a + 8, b + b_step, hi, id, 1u);
+    mma_ts2(d, a + 16, b + 2 * b_step, hi, id, 1u);
+    mma_ts2(d, a + 24, b + 3 * b_step, hi, id, 1u);
 }
-__device__ __forceinline__ void mma4_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t id, uint32_t acc)
+__device__ __forceinline__ void mma4_ss(uint32_t d, uint32_t a, uint32_t b, uint32_t hi, uint32_t id, uint32_t acc)
 {
-    mma_ss(d, a, b, id, acc);
-    mma_ss(d, a + 2, b + 2, id, 1u);
-    mma_ss(d, a + 4, b + 4, id, 1u);
-    mma_ss(d, a + 6, b + 6, id, 1u);
+    mma_ss2(d, a, hi, b, hi, id, acc);
+    mma_ss2(d, a + 2, hi, b + 2, hi, id, 1u);
+    mma_ss2(d, a + 4, hi, b + 4, hi, id, 1u);
+    mma_ss2(d, a + 6, hi, b + 6, hi, id, 1u);
 }
 
-__device__ __forceinline__ void run_ctrl(uint8_t *smem, Misc &mi, uint32_t tmem, const CUtensorMap *tm_v,
+// The issuing work is split over three threads (one per warp, so they sit on different schedulers):
+//   role 0  the products on the state's dependency chain: D1, E, the state update
+//   role 1  the output products rho_1 and rho += Aq E, and the output stores
+//   role 2  the Gram products (they run ahead of the chain) and the v loads
+__device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint32_t tmem, const CUtensorMap *tm_v,
                                          const CUtensorMap *tm_o, const CUtensorMap *tm_oim, const Params &p, int b,
                                          int h, int n_chunks)
 {
     long long *timing = p.timing;
     const uint64_t dbase = smem_desc(smem_u32(smem));                     // descriptor of byte offset 0
-    auto desc = [&](int off) { return dbase + (uint64_t)(off >> 4); };    // offsets are multiples of 16
+    const uint32_t dlo = (uint32_t)dbase, dhi = (uint32_t)(dbase >> 32);
+    auto desc = [&](int off) { return dlo + (uint32_t)(off >> 4); };      // low half; offsets are multiples of 16
     unsigned long long *bars = mi.bars;
     constexpr uint32_t I64 = idesc(64, 0), I64N = idesc(64, 1);           // N = 64, B K-major (negated)
+    constexpr uint32_t I128 = idesc(128, 0), I128N = idesc(128, 1);       // N = 128
     constexpr uint32_t I64M = idesc(64, 0) | (1u << 16), I64MN = idesc(64, 1) | (1u << 16);   // B MN-major
-
-    auto gram_half = [&](int j, int im) {   // Kt/Aq half: rows = [W; Qt], columns = tokens i
-        const int s = j & 1;
-        const uint64_t w_re = desc(OFF_WQ + s * 4 * kTile), w_im = w_re + (2 * kTile >> 4);
-        const uint64_t k_re = desc(OFF_KC + s * 2 * kTile), k_im = k_re + (kTile >> 4);
-        const uint32_t d = tmem + TM_GRAM;
-        if (!im) {
-            mma4_ss(d, w_re, k_re, I64, 0u);
-            mma4_ss(d, w_im, k_im, I64, 1u);
-        } else {
-            mma4_ss(d, w_re, k_im, I64, 0u);
-            mma4_ss(d, w_im, k_re, I64N, 1u);
-        }
-        mma_commit(&bars[B_GRAM_FULL]);
-    };
-
-    mbar_expect_tx(&bars[B_V_FULL], 16384);
-    tma_load_4d(smem + OFF_V, tm_v, &bars[B_V_FULL], 0, h, 0, b);
-
-    // The Gram products run ahead of the chain: chunk g, half gh is issued as soon as its operands are ready and
-    // the Gram columns have been drained; the chain's own waits keep trying in the meantime.
-    int g = 0, gh = 0;
-    auto pump_gram = [&]() {
-        if (g >= n_chunks) return;
-        if (gh == 0) {
-            if (!test_k(mi, g & 1 ? B_PREP_FULL1 : B_PREP_FULL0, g >> 1)) return;
-            if (g > 0 && !test_k(mi, B_GRAM_DRAINED, 2 * g - 1)) return;
-            tc_fence_after();
-            gram_half(g, 0);
-            gh = 1;
-        } else {
-            if (!test_k(mi, B_GRAM_DRAINED, 2 * g)) return;
-            tc_fence_after();
-            gram_half(g, 1);
-            gh = 0;
-            ++g;
-        }
-    };
-    auto wait_pump = [&](int bar, int k) {
-        if (test_k(mi, bar, k)) return true;
-        const unsigned long long t0 = now_ns();
-        for (uint32_t it = 0;; ++it) {
-            if (test_k(mi, bar, k)) return true;
-            pump_gram();
-            if ((it & 255u) == 255u) {
-                if (mi.abort) return false;
-                if (now_ns() - t0 > kWaitLimitNs) break;
-            }
-        }
-        mi.abort = 1;
-        return false;
-    };
-
     const uint32_t x_re = tmem + TM_X16, x_im = tmem + TM_X16 + 32;
     const uint32_t acc_re = tmem + TM_ACC, rho_re = tmem + TM_ACC + 64, acc_im = tmem + TM_ACC + 128,
                    rho_im = tmem + TM_ACC + 192;
-    SFDA_TDECL(true);
-    for (int j = 0; j < n_chunks; ++j) {
-        const int s = j & 1, u = j >> 1;
-        const uint64_t w_re = desc(OFF_WQ + s * 4 * kTile), w_im = w_re + (2 * kTile >> 4);
-        const uint64_t q_re = w_re + (kTile >> 4), q_im = w_im + (kTile >> 4);
-        const uint64_t k_re = desc(OFF_KC + s * 2 * kTile), k_im = k_re + (kTile >> 4);
-        const uint64_t a_re = desc(OFF_AQ + s * 2 * kTile), a_im = a_re + (kTile >> 4);
-        const uint64_t m_re = desc(OFF_MB), m_im = m_re + (kTile >> 4);
-        // D1 = W^* S_0
-        if (!wait_pump(B_S16_READY, j)) return;
-        if (!wait_pump(s ? B_PREP_FULL1 : B_PREP_FULL0, u)) return;
-        tc_fence_after();
-        SFDA_T(0);
-        mma4_ts(acc_re, x_re, w_re, I64, 0u);
-        mma4_ts(acc_re, x_im, w_im, I64, 1u);
-        mma4_ts(acc_im, x_im, w_re, I64, 0u);
-        mma4_ts(acc_im, x_re, w_im, I64N, 1u);
-        mma_commit(&bars[B_D1_DONE]);
-        SFDA_T(1);
-        // outputs of the previous chunk are staged: store them; rho is free again
-        if (j > 0) {
-            if (!wait_pump(B_O_STAGED, j - 1)) return;
+
+    if (role == 0) {
+        SFDA_TDECL(true);
+        for (int j = 0; j < n_chunks; ++j) {
+            const int s = j & 1, u = j >> 1;
+            const uint32_t w_re = desc(OFF_WQ + s * 4 * kTile), w_im = w_re + (2 * kTile >> 4);
+            const uint32_t k_re = desc(OFF_KC + s * 2 * kTile), k_im = k_re + (kTile >> 4);
+            const uint32_t m_re = desc(OFF_MB), m_im = m_re + (kTile >> 4);
+            // [D1 | rho_1] = [W ; Qt]^* S_0 : N = 128 over the slot's 128-row tiles; rho of the previous chunk
+            // must have been read out
+            if (!wait_k(mi, B_S16_READY, j)) return;
+            if (!wait_k(mi, s ? B_PREP_FULL1 : B_PREP_FULL0, u)) return;
+            if (j > 0 && !wait_k(mi, B_O_STAGED, j - 1)) return;
             tc_fence_after();
+            SFDA_T(0);
+            mma4_ts(acc_re, x_re, w_re, dhi, I128, 0u);
+            mma4_ts(acc_re, x_im, w_im, dhi, I128, 1u);
+            mma4_ts(acc_im, x_im, w_re, dhi, I128, 0u);
+            mma4_ts(acc_im, x_re, w_im, dhi, I128N, 1u);
+            mma_commit(&bars[B_D1_DONE]);
+            mma_commit(&bars[s ? B_WQ_FREE1 : B_WQ_FREE0]);
+            SFDA_T(1);
+            // E = M_beta R
+            if (!wait_k(mi, B_R16_READY, j)) return;
             SFDA_T(2);
-            tma_store_4d(tm_o, smem + OFF_OST, 0, h, (j - 1) * C, b);
-            if (p.has_o_im) tma_store_4d(tm_oim, smem + OFF_AQ + ((j - 1) & 1) * 2 * kTile, 0, h, (j - 1) * C, b);
-            tma_store_commit();
+            if (!wait_k(mi, B_MB_FULL, j)) return;
+            tc_fence_after();
+            SFDA_T(3);
+            mma4_ts(acc_re, x_re, m_re, dhi, I64, 0u);
+            mma4_ts(acc_re, x_im, m_im, dhi, I64N, 1u);
+            mma4_ts(acc_im, x_im, m_re, dhi, I64, 0u);
+            mma4_ts(acc_im, x_re, m_im, dhi, I64, 1u);
+            mma_commit(&bars[B_E_DONE]);
+            SFDA_T(4);
+            // S += E^T Kc (Kc as MN-major B: rows = tokens)
+            if (!wait_k(mi, B_E16_READY, j)) return;
+            tc_fence_after();
+            SFDA_T(5);
+            mma4_ts(tmem + TM_S32, x_re, k_re, dhi, I64M, 1u, 128);
+            mma4_ts(tmem + TM_S32, x_im, k_im, dhi, I64MN, 1u, 128);
+            mma4_ts(tmem + TM_S32 + 64, x_re, k_im, dhi, I64M, 1u, 128);
+            mma4_ts(tmem + TM_S32 + 64, x_im, k_re, dhi, I64M, 1u, 128);
+            mma_commit(&bars[s ? B_KC_FREE1 : B_KC_FREE0]);
+            mma_commit(&bars[B_UPD_DONE]);
+            SFDA_T(6);
         }
-        // rho_1 = Qt^* S_0
-        mma4_ts(rho_re, x_re, q_re, I64, 0u);
-        mma4_ts(rho_re, x_im, q_im, I64, 1u);
-        mma4_ts(rho_im, x_im, q_re, I64, 0u);
-        mma4_ts(rho_im, x_re, q_im, I64N, 1u);
-        mma_commit(&bars[s ? B_WQ_FREE1 : B_WQ_FREE0]);
-        pump_gram();
-        if (j > 0) {   // by now the store of chunk j-1 has read its staging tiles
-            tma_store_wait_read();
-            mbar_arrive(&bars[(j - 1) & 1 ? B_STORE_DONE1 : B_STORE_DONE0]);
+    } else if (role == 1) {
+        for (int j = 0; j < n_chunks; ++j) {
+            const int s = j & 1, u = j >> 1;
+            const uint32_t a_re = desc(OFF_AQ + s * 2 * kTile), a_im = a_re + (kTile >> 4);
+            // outputs of the previous chunk are staged: store them
+            if (j > 0) {
+                if (!wait_k(mi, B_O_STAGED, j - 1)) return;
+                tma_store_4d(tm_o, smem + OFF_OST, 0, h, (j - 1) * C, b);
+                if (p.has_o_im) tma_store_4d(tm_oim, smem + OFF_AQ + ((j - 1) & 1) * 2 * kTile, 0, h, (j - 1) * C, b);
+                tma_store_commit();
+                tma_store_wait_read();
+                mbar_arrive(&bars[(j - 1) & 1 ? B_STORE_DONE1 : B_STORE_DONE0]);
+            }
+            // rho += Aq E
+            if (!wait_k(mi, B_E16_READY, j)) return;
+            if (!wait_k(mi, s ? B_AQ_FULL1 : B_AQ_FULL0, u)) return;
+            tc_fence_after();
+            mma4_ts(rho_re, x_re, a_re, dhi, I64, 1u);
+            mma4_ts(rho_re, x_im, a_im, dhi, I64N, 1u);
+            mma4_ts(rho_im, x_im, a_re, dhi, I64, 1u);
+            mma4_ts(rho_im, x_re, a_im, dhi, I64, 1u);
+            mma_commit(&bars[B_UPD_DONE]);
         }
-        SFDA_T(3);
-        // E = M_beta R
-        if (!wait_pump(B_R16_READY, j)) return;
-        SFDA_T(4);
-        if (!wait_pump(B_MB_FULL, j)) return;
-        tc_fence_after();
-        SFDA_T(5);
-        mma4_ts(acc_re, x_re, m_re, I64, 0u);
-        mma4_ts(acc_re, x_im, m_im, I64N, 1u);
-        mma4_ts(acc_im, x_im, m_re, I64, 0u);
-        mma4_ts(acc_im, x_re, m_im, I64, 1u);
-        mma_commit(&bars[B_E_DONE]);
-        if (j + 1 < n_chunks) {   // v of chunk j has been consumed
-            mbar_expect_tx(&bars[B_V_FULL], 16384);
-            tma_load_4d(smem + OFF_V, tm_v, &bars[B_V_FULL], 0, h, (j + 1) * C, b);
+        if (!wait_k(mi, B_O_STAGED, n_chunks - 1)) return;
+        tma_store_4d(tm_o, smem + OFF_OST, 0, h, (n_chunks - 1) * C, b);
+        if (p.has_o_im)
+            tma_store_4d(tm_oim, smem + OFF_AQ + ((n_chunks - 1) & 1) * 2 * kTile, 0, h, (n_chunks - 1) * C, b);
+        tma_store_commit();
+        tma_store_wait_all();
+    } else {
+        // Gram chunk g, half gh, as soon as its operands are written and the Gram columns have been drained;
+        // v of chunk jv as soon as v of chunk jv-1 has been consumed (R of that chunk is built).
+        mbar_expect_tx(&bars[B_V_FULL], 16384);
+        tma_load_4d(smem + OFF_V, tm_v, &bars[B_V_FULL], 0, h, 0, b);
+        int g = 0, gh = 0, jv = 1;
+        const unsigned long long t0 = now_ns();
+        for (uint32_t it = 0; g < n_chunks || jv < n_chunks; ++it) {
+            bool progress = false;
+            if (g < n_chunks) {
+                const bool ready = gh == 0 ? test_k(mi, g & 1 ? B_PREP_FULL1 : B_PREP_FULL0, g >> 1) &&
+                                                 (g == 0 || test_k(mi, B_GRAM_DRAINED, 2 * g - 1))
+                                           : test_k(mi, B_GRAM_DRAINED, 2 * g);
+                if (ready) {
+                    const int s = g & 1;
+                    const uint32_t w_re = desc(OFF_WQ + s * 4 * kTile), w_im = w_re + (2 * kTile >> 4);
+                    const uint32_t k_re = desc(OFF_KC + s * 2 * kTile), k_im = k_re + (kTile >> 4);
+                    const uint32_t d = tmem + TM_GRAM;
+                    tc_fence_after();
+                    if (gh == 0) {       // rows = [W; Qt], columns = tokens i
+                        mma4_ss(d, w_re, k_re, dhi, I64, 0u);
+                        mma4_ss(d, w_im, k_im, dhi, I64, 1u);
+                    } else {
+                        mma4_ss(d, w_re, k_im, dhi, I64, 0u);
+                        mma4_ss(d, w_im, k_re, dhi, I64N, 1u);
+                    }
+                    mma_commit(&bars[B_GRAM_FULL]);
+                    g += gh;
+                    gh ^= 1;
+                    progress = true;
+                }
+            }
+            if (jv < n_chunks && test_k(mi, B_R16_READY, jv - 1)) {
+                mbar_expect_tx(&bars[B_V_FULL], 16384);
+                tma_load_4d(smem + OFF_V, tm_v, &bars[B_V_FULL], 0, h, jv * C, b);
+                ++jv;
+                progress = true;
+            }
+            if (!progress) {
+                __nanosleep(64);
+                if ((it & 63u) == 63u) {
+                    if (mi.abort) return;
+                    if (now_ns() - t0 > 2 * kWaitLimitNs + 1000000ull * (unsigned long long)n_chunks) {
+                        mi.abort = 1;
+                        return;
+                    }
+                }
+            }
         }
-        pump_gram();
-        SFDA_T(6);
-        // S += E^T Kc (Kc as MN-major B: rows = tokens) ,  rho += Aq E
-        if (!wait_pump(B_E16_READY, j)) return;
-        SFDA_T(7);
-        if (!wait_pump(s ? B_AQ_FULL1 : B_AQ_FULL0, u)) return;
-        tc_fence_after();
-        SFDA_T(8);
-        mma4_ts(tmem + TM_S32, x_re, k_re, I64M, 1u, 128);
-        mma4_ts(tmem + TM_S32, x_im, k_im, I64MN, 1u, 128);
-        mma4_ts(tmem + TM_S32 + 64, x_re, k_im, I64M, 1u, 128);
-        mma4_ts(tmem + TM_S32 + 64, x_im, k_re, I64M, 1u, 128);
-        mma_commit(&bars[s ? B_KC_FREE1 : B_KC_FREE0]);
-        mma4_ts(rho_re, x_re, a_re, I64, 1u);
-        mma4_ts(rho_re, x_im, a_im, I64N, 1u);
-        mma4_ts(rho_im, x_im, a_re, I64, 1u);
-        mma4_ts(rho_im, x_re, a_im, I64, 1u);
-        mma_commit(&bars[B_UPD_DONE]);
-        pump_gram();
-        SFDA_T(9);
     }
-    if (!wait_pump(B_O_STAGED, n_chunks - 1)) return;
-    tma_store_4d(tm_o, smem + OFF_OST, 0, h, (n_chunks - 1) * C, b);
-    if (p.has_o_im) tma_store_4d(tm_oim, smem + OFF_AQ + ((n_chunks - 1) & 1) * 2 * kTile, 0, h, (n_chunks - 1) * C, b);
-    tma_store_commit();
-    tma_store_wait_all();
 }
 
 // ---- PREP ---------------------------------------------------------------------------------------------
@@ -363,14 +362,47 @@ __device__ __forceinline__ void turns_sincos(uint32_t turns, float *sn, float *c
     __sincosf(f * 6.283185307f, sn, cs);
 }
 
-__device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, const Params &p, int b, int h, int n_chunks, int pt)
+__device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int b, int h, int n_chunks,
+                                         int pt)
 {
     long long *timing = p.timing;
     const int jp = pt & 31, tq = pt >> 5;   // channel pair (channels 2jp, 2jp+1), token octet (8 tokens)
     bool dead = false;
+    // this role also reads the finished outputs out of tensor memory (its warps cover the four lane quadrants
+    // twice: the first four take rho's real part, the others the imaginary part)
+    const int lane = pt & 31, quad = (pt >> 5) & 3, half = pt >> 7;
+    const int c = quad * 32 + lane;
+    const uint32_t tlane = tmem + ((uint32_t)(quad * 32) << 16);
+    auto drain_outputs = [&](int jd) {           // rho of chunk jd -> bf16 staging tiles [t][128]
+        if (!dead && !wait_k(mi, B_UPD_DONE, jd)) dead = true;
+        // the Re staging tile is shared by all chunks: the store of chunk jd-1 must have read it
+        if (jd >= 1 && !dead && !wait_k(mi, (jd - 1) & 1 ? B_STORE_DONE1 : B_STORE_DONE0, (jd - 1) >> 1)) dead = true;
+        tc_fence_after();
+        if (half == 0 || p.has_o_im) {
+            __nv_bfloat16 *stage =
+                reinterpret_cast<__nv_bfloat16 *>(smem + (half ? OFF_AQ + (jd & 1) * 2 * kTile : OFF_OST));
+            const float sgn = half ? -1.f : 1.f;   // o = conj(rho)
+#pragma unroll
+            for (int hc = 0; hc < 2; ++hc) {
+                uint32_t r[32];
+                tmem_ld<32>(tlane + TM_ACC + 64 + 128 * half + 32 * hc, r);
+                tc_wait_ld();
+#pragma unroll
+                for (int t = 0; t < 32; ++t)
+                    stage[(32 * hc + t) * DV + c] = __float2bfloat16_rn(sgn * __uint_as_float(r[t]));
+            }
+        }
+        fence_async_smem();
+        tc_fence_before();
+        mbar_arrive(&mi.bars[B_O_STAGED]);
+    };
     SFDA_TDECL(pt == 0);
-    for (int j = 0; j < n_chunks; ++j) {
+    for (int j = 0; j < n_chunks + 2; ++j) {
         if (role_sync_or(2, kPrepThreads, dead || mi.abort)) break;
+        if (j >= n_chunks) {                     // only the outputs of the last two chunks are left
+            if (j >= 2) drain_outputs(j - 2);
+            continue;
+        }
         const int s = j & 1, ring = j & 3;
         const int t0 = j * C, len = min(C, p.T - t0);
         const size_t row0 = ((size_t)b * p.T + t0) * p.H + h;   // token t of this head: row0 + t * H
@@ -443,6 +475,10 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, const Params &
             if (!dead && !wait_k(mi, s ? B_KC_FREE1 : B_KC_FREE0, (j >> 1) - 1)) dead = true;
         }
         SFDA_T(32);
+        // the state update of chunk j-2 has just finished (it freed Kc above): read out that chunk's outputs,
+        // so that rho is free when the next chunk's first product is issued
+        if (j >= 2) drain_outputs(j - 2);
+        SFDA_T(34);
 
         // pass 2: rotated / decayed operands
         uint8_t *wq_re = smem + OFF_WQ + s * 4 * kTile, *wq_im = wq_re + 2 * kTile;
@@ -548,31 +584,56 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
         role_sync(1, kSolveThreads);
         SFDA_T(24);
 
-        // ---- X = (I + L)^{-1} in place.  Diagonal 16x16 blocks: warp w, lane = column c solves (I + L) x = e_c
-        // right-looking (after x_i is final, every later row is updated at once: independent operations).
-        if (lane < 16) {
-            const int o = 16 * w, c = lane;
-            float xr[16], xi[16];
+        // ---- X = (I + L)^{-1} in place.  Diagonal 8x8 blocks: lane = column c of block blk solves
+        // (I + L) x = e_c right-looking (after x_i is final every later row is updated at once).
+        if (w < 2) {
+            const int o = 8 * (4 * w + (lane >> 3)), c = lane & 7;
+            float xr[8], xi[8];
 #pragma unroll
-            for (int r = 0; r < 16; ++r) {
+            for (int r = 0; r < 8; ++r) {
                 xr[r] = r == c ? 1.f : 0.f;
                 xi[r] = 0.f;
             }
 #pragma unroll
-            for (int i = 0; i < 15; ++i) {
+            for (int i = 0; i < 7; ++i) {
                 const float vr = xr[i], vi = xi[i];      // zero above the diagonal (i < c)
 #pragma unroll
-                for (int r = i + 1; r < 16; ++r) {
+                for (int r = i + 1; r < 8; ++r) {
                     const float lr_ = Lr[(o + r) * LS + o + i], li_ = Li[(o + r) * LS + o + i];
                     xr[r] -= lr_ * vr - li_ * vi;
                     xi[r] -= lr_ * vi + li_ * vr;
                 }
             }
-            __syncwarp(0x0000ffffu);          // every lane has read its L block before it is overwritten
+            __syncwarp();                     // every lane has read its L block before it is overwritten
 #pragma unroll
-            for (int r = 0; r < 16; ++r) {
+            for (int r = 0; r < 8; ++r) {
                 Lr[(o + r) * LS + o + c] = xr[r];
                 Li[(o + r) * LS + o + c] = xi[r];
+            }
+        }
+        role_sync(1, kSolveThreads);
+        {   // level 0: 8 -> 16.  Warp w merges 16-block w: X21 = -X22 (L21 X11).  The m16 tile is placed on the
+            // whole 16-row block, so its lower eight rows (fragment elements 2, 3) are the rows that matter.
+            const int o = 16 * w;
+            float cr[4] = {0.f, 0.f, 0.f, 0.f}, ci[4] = {0.f, 0.f, 0.f, 0.f};
+            cmma_16x8(cr, ci, Lr, Li, LS, o, o, Lr, Li, LS, o, o, 0, 1, lane);           // rows 8..15: L21 X11
+            {   // T into the unused 8x8 block above the diagonal: rows o..o+7, columns o+8..o+15
+                const int g = lane >> 2, tg = lane & 3, at = (o + g) * LS + o + 8 + 2 * tg;
+                Lr[at] = cr[2]; Lr[at + 1] = cr[3];
+                Li[at] = ci[2]; Li[at + 1] = ci[3];
+            }
+            __syncwarp();
+            float dr[4] = {0.f, 0.f, 0.f, 0.f}, di[4] = {0.f, 0.f, 0.f, 0.f};
+            cmma_16x8(dr, di, Lr, Li, LS, o, o + 8, Lr, Li, LS, o, o + 8, 0, 1, lane);   // rows 8..15: X22 T
+            {
+                const int g = lane >> 2, tg = lane & 3, at = (o + 8 + g) * LS + o + 2 * tg;
+                Lr[at] = -dr[2]; Lr[at + 1] = -dr[3];
+                Li[at] = -di[2]; Li[at + 1] = -di[3];
+                // the block above the diagonal held T; later levels read the whole 16x16 diagonal block
+                const int zt = (o + g) * LS + o + 8 + 2 * tg;
+                __syncwarp();
+                Lr[zt] = 0.f; Lr[zt + 1] = 0.f;
+                Li[zt] = 0.f; Li[zt + 1] = 0.f;
             }
         }
         role_sync(1, kSolveThreads);
@@ -647,29 +708,6 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
     const int j0 = half * 32;                  // this warp's complex rows in the state pass
     const uint32_t tlane = tmem + ((uint32_t)(quad * 32) << 16);
 
-    auto drain_outputs = [&](int jd) -> bool {   // rho of chunk jd -> bf16 staging tiles [t][128]
-        const bool want = half ? p.has_o_im != 0 : true;
-        // the Re staging tile is shared by all chunks: the store of chunk jd-1 must have read it
-        if (jd >= 1 && !wait_k(mi, (jd - 1) & 1 ? B_STORE_DONE1 : B_STORE_DONE0, (jd - 1) >> 1)) return false;
-        if (want) {
-            __nv_bfloat16 *stage =
-                reinterpret_cast<__nv_bfloat16 *>(smem + (half ? OFF_AQ + (jd & 1) * 2 * kTile : OFF_OST));
-            const float sgn = half ? -1.f : 1.f;   // o = conj(rho)
-#pragma unroll
-            for (int hc = 0; hc < 2; ++hc) {
-                uint32_t r[32];
-                tmem_ld<32>(tlane + TM_ACC + 64 + 128 * half + 32 * hc, r);
-                tc_wait_ld();
-#pragma unroll
-                for (int t = 0; t < 32; ++t)
-                    stage[(32 * hc + t) * DV + c] = __float2bfloat16_rn(sgn * __uint_as_float(r[t]));
-            }
-        }
-        fence_async_smem();
-        tc_fence_before();
-        mbar_arrive(&mi.bars[B_O_STAGED]);
-        return true;
-    };
     // One 16-row piece of the state pass: rows j0 + 16 pc .. + 15 (Re and Im).
     auto state_piece = [&](int pc, int ring, bool first) {
         uint32_t sre[16], sim[16], pk[8];
@@ -731,7 +769,6 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
 
     SFDA_TDECL(ct == 0);
     for (int j = 0; j < n_chunks; ++j) {
-        const int s = j & 1;
         // ---- state pass: S_0 of this chunk = e^{i phi_C} a_C (accumulated state of the previous chunk)
         if (j > 0) {
             if (!wait_k(mi, B_UPD_DONE, j - 1)) return;
@@ -745,16 +782,12 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
         mbar_arrive(&mi.bars[B_S16_READY]);
         SFDA_T(11);
 
-        // ---- outputs of the previous chunk, while D1 runs
-        if (j > 0 && !drain_outputs(j - 1)) return;
-        SFDA_T(12);
-
-        // ---- R = V - D1 -> bf16 A operand (rho_1 still reads S_0 from the same columns: gate on its commit)
+        // ---- R = V - D1 -> bf16 A operand (D1 and rho_1, which read S_0 from the same columns, are both done)
         if (!wait_k(mi, B_D1_DONE, j)) return;
         if (!wait_k(mi, B_V_FULL, j)) return;
         tc_fence_after();
         SFDA_T(13);
-        if (!convert_acc(half == 0, half == 1, s ? B_WQ_FREE1 : B_WQ_FREE0, j >> 1)) return;
+        if (!convert_acc(half == 0, half == 1, -1, 0)) return;
         tc_fence_before();
         mbar_arrive(&mi.bars[B_R16_READY]);
         SFDA_T(14);
@@ -772,7 +805,6 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
     // ---- last chunk: outputs and the final state
     if (!wait_k(mi, B_UPD_DONE, n_chunks - 1)) return;
     tc_fence_after();
-    if (!drain_outputs(n_chunks - 1)) return;
     if (p.S_T) {
         const int ring = (n_chunks - 1) & 3;
 #pragma unroll
@@ -814,9 +846,9 @@ sfda_forward_ws_kernel(const __grid_constant__ CUtensorMap tm_v, const __grid_co
         init(B_STORE_DONE0, 1); init(B_STORE_DONE1, 1);
         init(B_GRAM_FULL, 1); init(B_GRAM_DRAINED, kSolveThreads);
         init(B_MB_FULL, kSolveThreads); init(B_AQ_FULL0, kSolveThreads); init(B_AQ_FULL1, kSolveThreads);
-        init(B_D1_DONE, 1); init(B_E_DONE, 1); init(B_UPD_DONE, 1);
+        init(B_D1_DONE, 1); init(B_E_DONE, 1); init(B_UPD_DONE, 2);   // state update and rho += Aq E
         init(B_S16_READY, kChainThreads); init(B_R16_READY, kChainThreads); init(B_E16_READY, kChainThreads);
-        init(B_O_STAGED, kChainThreads); init(B_V_FULL, 1);
+        init(B_O_STAGED, kPrepThreads); init(B_V_FULL, 1);
         mi.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -837,11 +869,11 @@ sfda_forward_ws_kernel(const __grid_constant__ CUtensorMap tm_v, const __grid_co
         run_solve(smem, mi, tmem, p, n_chunks, tid - kChainThreads);
     } else if (warp < kChainWarps + kSolveWarps + kPrepWarps) {
         regs_inc<kRegsWork>();
-        run_prep(smem, mi, p, b, h, n_chunks, tid - kChainThreads - kSolveThreads);
+        run_prep(smem, mi, tmem, p, b, h, n_chunks, tid - kChainThreads - kSolveThreads);
     } else {
         regs_dec<kRegsCtrl>();
-        if (tid == kChainThreads + kSolveThreads + kPrepThreads)
-            run_ctrl(smem, mi, tmem, &tm_v, &tm_o, &tm_oim, p, b, h, n_chunks);
+        const int cw = warp - (kChainWarps + kSolveWarps + kPrepWarps);
+        if ((tid & 31) == 0 && cw < 3) run_ctrl(cw, smem, mi, tmem, &tm_v, &tm_o, &tm_oim, p, b, h, n_chunks);
     }
 
     tc_fence_before();

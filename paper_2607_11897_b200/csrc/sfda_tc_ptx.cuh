@@ -90,6 +90,25 @@ __device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t b, uint3
                  ::"r"(d), "r"(a), "l"(b), "r"(id), "r"(acc)
                  : "memory");
 }
+// Same with the shared-memory descriptor given as its two 32-bit halves: advancing along K only changes the
+// low half, so the issuing thread spends one 32-bit add per instruction.
+__device__ __forceinline__ void mma_ts2(uint32_t d, uint32_t a, uint32_t b_lo, uint32_t b_hi, uint32_t id, uint32_t acc)
+{
+    asm volatile(
+        "{\n.reg .pred p;\n.reg .b64 db;\nmov.b64 db, {%2, %3};\nsetp.ne.b32 p, %5, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n}\n" ::"r"(d),
+        "r"(a), "r"(b_lo), "r"(b_hi), "r"(id), "r"(acc)
+        : "memory");
+}
+__device__ __forceinline__ void mma_ss2(uint32_t d, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi, uint32_t id,
+                                        uint32_t acc)
+{
+    asm volatile(
+        "{\n.reg .pred p;\n.reg .b64 da, db;\nmov.b64 da, {%1, %2};\nmov.b64 db, {%3, %4};\nsetp.ne.b32 p, %6, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n}\n" ::"r"(d),
+        "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(id), "r"(acc)
+        : "memory");
+}
 __device__ __forceinline__ void mma_commit(unsigned long long *bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
@@ -160,12 +179,9 @@ __device__ __forceinline__ int sw_off(int r, int e)
     return (r >> 3) * 1024 + (r & 7) * 128 + ((((e >> 3) ^ r) & 7) << 4) + ((e & 7) << 1);
 }
 // ---- warp-level tf32 MMA used by the triangular solve ------------------------------------------------
-__device__ __forceinline__ uint32_t to_tf32(float x)
-{
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return r;
-}
+// fp32 bits used directly as a tf32 operand: the tensor core ignores the low 13 mantissa bits (truncation,
+// relative error below 2^-10), and no conversion instruction is spent.
+__device__ __forceinline__ uint32_t to_tf32(float x) { return __float_as_uint(x); }
 __device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2])
 {
     asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
