@@ -167,6 +167,10 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--re-only", action="store_true", help="write o = Re only (default: Re and Im)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="profiling only: run the headline shapes with this batch size instead of 8 "
+                         "(the JSON line then names the reduced workload and is not a benchmark value)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else max(args.warmup, 0)
 
@@ -182,6 +186,7 @@ def main():
     import torch.distributed as dist
 
     import paper_2607_11897_b200 as sfda
+    from paper_2607_11897_b200 import dp
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
@@ -192,9 +197,11 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     cfg = workloads.CONFIGS[HEADLINE]
+    if args.batch > 0:
+        cfg = cfg.scaled(name="%s_batch%d_profiling_only" % (cfg.name, args.batch), B=args.batch)
     want_im = not args.re_only
     # every rank draws its own batch: batch elements rank*B .. rank*B + B - 1 of the same recipe
-    inp = workloads.forward_inputs(cfg, batch=range(rank * cfg.B, (rank + 1) * cfg.B))
+    inp = workloads.forward_inputs(cfg, batch=dp.rank_batch_range(cfg.B, rank))
     host = {}
     for key, val in inp.items():
         t = torch.from_numpy(np.ascontiguousarray(val))
@@ -235,13 +242,11 @@ def main():
         barrier()
     total_ms = start.elapsed_time(stop)
     kernel_ms = [e0.elapsed_time(e1) for e0, e1 in events]      # one forward = one launch of the chunk kernel
-    t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
+    total_ms = dp.max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / args.steps
     tokens_per_step = world * cfg.B * cfg.T
-    value = tokens_per_step / (ms_per_step * 1e-3)
+    value = dp.whole_job_throughput(cfg.B * cfg.T, world, ms_per_step * 1e-3)
+    assert sfda.sfda_workspace_status(ws, stream) == 0      # no bounded device-side wait ran out
 
     # end to end through the host-buffer entry point: H2D of the inputs and D2H of the results inside the timing
     e2e = None
@@ -260,13 +265,46 @@ def main():
                                               host["beta"], host["S0"], oh, oh_im, Sh, cfg.chunk, arena, stream)
             stream.synchronize()
         barrier()
-        e2e_s = (time.perf_counter() - t0) / args.e2e_steps
-        t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e = {"value": tokens_per_step / float(t.item()), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
-               "d2h_bytes_per_step": int(d2h), "ms_per_step": 1e3 * float(t.item())}
+        e2e_s = dp.max_over_ranks((time.perf_counter() - t0) / args.e2e_steps, dev)
+        e2e = {"value": tokens_per_step / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": int(d2h), "ms_per_step": 1e3 * e2e_s}
         del arena
+
+    # one-token decode (sfda_step) on the decode configuration: HBM-bound, reported beside the headline
+    decode = None
+    if rank == 0 and not args.no_decode:
+        del d, o, o_im
+        torch.cuda.empty_cache()
+        dcfg = workloads.CONFIGS[4]
+        S = torch.from_numpy(workloads.decode_initial_state(dcfg)).to(dev)
+        ring = []
+        for st in range(8):                                  # eight distinct steps of inputs, cycled
+            x = workloads.decode_step_inputs(dcfg, st)
+            ring.append({k: (torch.from_numpy(v).to(dev).to(torch.bfloat16) if k in ("q", "k", "v")
+                             else torch.from_numpy(v).to(dev)) for k, v in x.items()})
+        od = torch.empty(dcfg.B, dcfg.H, dcfg.d_v, device=dev, dtype=torch.bfloat16)
+        od_im = torch.empty_like(od)
+
+        def dstep(i):
+            x = ring[i % len(ring)]
+            sfda.sfda_step(x["q"], x["k"], x["v"], x["alpha"], x["theta"], x["beta"], S, od, od_im, stream)
+
+        for i in range(8):
+            dstep(i)
+        nd = 200
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        d0.record(stream)
+        for i in range(nd):
+            dstep(i)
+        d1.record(stream)
+        torch.cuda.synchronize()
+        step_ms = d0.elapsed_time(d1) / nd
+        dbytes = dcfg.B * dcfg.H * (2 * dcfg.d_k * dcfg.d_v * 4 + 2 * dcfg.d_k * 2 + dcfg.d_v * 2 + 2 * dcfg.m * 4 + 4
+                                     + 2 * dcfg.d_v * 2)
+        decode = {"workload": dcfg.name, "ms_per_step": step_ms, "tokens_per_s": dcfg.B / (step_ms * 1e-3),
+                  "algorithmic_bytes_per_step": dbytes, "achieved_gbs": dbytes / (step_ms * 1e-3) / 1e9,
+                  "state_bytes": int(S.numel() * 4), "note": "state (537 MB) far larger than L2"}
 
     if rank != 0:
         if world > 1:
@@ -289,11 +327,15 @@ def main():
         "tensor_frac": achieved_tf / peaks["bf16_tflops"],
         "roofline_ms": 1e3 * max(hbm_time, tensor_time),
     }
-    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(traffic_path):
-        with open(traffic_path) as f:
-            roofline["traffic"] = json.load(f).get("sfda_forward_headline_bytes_per_launch")
+    if args.batch == 0:
+        # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this kernel at B = 4 (1.870 GB,
+        # profiles/sfda_forward_ws_kernel_batch4_ncu_full.md), scaled by the units processed (traffic grows with B)
+        roofline["traffic"] = 1.870e9 * cfg.B / 4
+        roofline["traffic_source"] = "ncu capture at B=4 scaled to B=%d; Re+Im outputs" % cfg.B
 
+    if decode is not None:
+        decode["frac"] = decode["achieved_gbs"] / peaks["hbm_gbs"]
+        decode["peak_source"] = "of " + peaks["source"]
     cpu = None
     if not args.no_cpu_baseline:
         cores = len(os.sched_getaffinity(0))
@@ -310,7 +352,7 @@ def main():
                    "chunk": cfg.chunk, "outputs": "Re+Im" if want_im else "Re", "state": "fp32", "S0": "N(0,0.02)",
                    "parallelism": "dp%d over (batch, head), no collective" % world,
                    "l2": "inputs+outputs %.2f GB per step, far larger than the 126 MB L2; no flush" % (abytes / 1e9)},
-        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
+        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "decode": decode,
         "gpu_launches": launches_per_step * args.steps, "clocks": clocks.summary(),
     }
     print(json.dumps(line), flush=True)

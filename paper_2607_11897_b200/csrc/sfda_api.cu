@@ -82,7 +82,7 @@ size_t sfda_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, in
     if (B < 1 || T < 1 || H < 1 || check_dims(d_k, d_v, chunk, dtype) != SFDA_OK) return 0;
     sfda::ForwardArgs a{};
     a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.chunk = chunk; a.dtype = dtype;
-    return sfda::forward_tc_supported(a) ? 256 : 0;   // the tensor-core path keeps a status word there
+    return sfda::forward_ws_supported(a) ? 256 : 0;   // the tensor-core path keeps a status word there
 }
 
 int sfda_forward_simt(const void *q, const void *k, const void *v, const float *alpha, const float *theta,
@@ -110,7 +110,7 @@ int sfda_forward(const void *q, const void *k, const void *v, const float *alpha
     if (workspace && !aligned16(workspace)) return SFDA_ERR_ALIGN;
     const sfda::ForwardArgs a = pack(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
     const cudaError_t e =
-        sfda::forward_tc_supported(a)
+        sfda::forward_ws_supported(a)
             ? sfda::launch_forward_ws(a, static_cast<uint32_t *>(workspace), static_cast<cudaStream_t>(stream),
                                       &g_last_launches)
             : sfda::launch_forward_simt(a, static_cast<cudaStream_t>(stream), &g_last_launches);

@@ -3,7 +3,7 @@
 // One CTA walks the chunks of one (batch, head) pair; four roles run concurrently on different chunks
 // and hand tiles to one another through mbarriers:
 //
-//   PREP  (4 warps)  chunk j+1: cumulative phase-decay gamma_t = a_t e^{i phi_t} (Eq. "constructive-Gamma";
+//   PREP  (8 warps)  chunk j+1: cumulative phase-decay gamma_t = a_t e^{i phi_t} (Eq. "constructive-Gamma";
 //                    log2-sum and integer-turn prefix scans), rotated/decayed operand tiles in shared memory.
 //   SOLVE (4 warps)  chunk j+1: drains the Gram blocks from tensor memory, inverts the unit-lower WY system
 //                    (Eq. "constructive-M": M = (I + L)^{-1}) by 16x16 blocks, writes M_beta and Aq tiles.
@@ -917,6 +917,8 @@ bool make_map(CUtensorMap *map, const void *base, int B, int T, int H)
 }
 
 }  // namespace
+
+bool forward_ws_supported(const ForwardArgs &a) { return a.dtype == 1 && a.d_k == DK && a.d_v == DV && a.chunk == C; }
 
 cudaError_t launch_forward_ws(const ForwardArgs &a, uint32_t *status, cudaStream_t stream, int *launches)
 {

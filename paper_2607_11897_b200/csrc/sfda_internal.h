@@ -32,11 +32,9 @@ struct StepArgs {
 
 // Each returns a cudaError_t from configuring / launching; *launches is incremented per kernel.
 cudaError_t launch_forward_simt(const ForwardArgs &a, cudaStream_t stream, int *launches);
-// Tensor-core path (bf16, d_k = d_v = 128, chunk = 64).  `status` is one device word the kernel sets
-// when a bounded wait runs out; it is cleared on the stream before the launch.
-bool forward_tc_supported(const ForwardArgs &a);
-cudaError_t launch_forward_tc(const ForwardArgs &a, uint32_t *status, cudaStream_t stream, int *launches);
-// Warp-specialised, chunk-pipelined version of the same path (the one sfda_forward uses).
+// Tensor-core path (bf16, d_k = d_v = 128, chunk = 64): warp-specialised, chunk-pipelined tcgen05 kernel.
+// `status` is one device word the kernel sets when a bounded wait runs out; it is cleared on the stream
+// before the launch.
 bool forward_ws_supported(const ForwardArgs &a);
 cudaError_t launch_forward_ws(const ForwardArgs &a, uint32_t *status, cudaStream_t stream, int *launches);
 cudaError_t launch_chunk_factors(const FactorArgs &a, cudaStream_t stream, int *launches);

@@ -1,0 +1,156 @@
+"""Host-side checks that need no GPU: the C-ABI library loads and exports what the header declares,
+its integer bookkeeping and argument validation behave as documented, the input generators are
+deterministic, and the multi-process sharding covers every (batch, head) pair exactly once."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2607_11897_b200 as sfda
+import workloads
+from oracle import bookkeeping
+from paper_2607_11897_b200 import build as cuda_build
+from paper_2607_11897_b200 import dp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    cuda_build.build()
+    return sfda.load()
+
+
+def test_library_exports_every_declared_symbol(lib):
+    header = open(os.path.join(ROOT, "include", "sfda.h")).read()
+    names = re.findall(r"SFDA_API\s+[\w\s\*]+?\b(sfda_\w+)\s*\(", header)
+    assert len(names) >= 10 and len(set(names)) == len(names)
+    for name in names:
+        assert hasattr(lib, name), "libsfda.so does not export %s" % name
+
+
+def test_plan_matches_integer_bookkeeping(lib):
+    for T in (1, 5, 63, 64, 65, 256, 257, 8192, 131072):
+        for chunk in (16, 32, 64):
+            assert sfda.sfda_plan(T, chunk) == bookkeeping.chunk_plan(T, chunk)
+    with pytest.raises(sfda.SfdaError) as e:
+        sfda.sfda_plan(0, 64)
+    assert e.value.status == -2
+
+
+def test_status_strings(lib):
+    seen = {sfda.sfda_status_string(c) for c in range(0, -8, -1)}
+    assert len(seen) == 8 and "ok" in seen
+    assert sfda.sfda_status_string(-99) == "unknown status"
+
+
+def test_workspace_bytes(lib):
+    assert sfda.sfda_workspace_bytes(8, 8192, 32, 128, 128, 64, sfda.SFDA_BF16) == 256
+    assert sfda.sfda_workspace_bytes(1, 256, 2, 64, 64, 16, sfda.SFDA_F32) == 0
+    assert sfda.sfda_workspace_bytes(1, 256, 2, 128, 128, 64, sfda.SFDA_F32) == 0
+    assert sfda.sfda_workspace_bytes(0, 256, 2, 128, 128, 64, sfda.SFDA_BF16) == 0
+
+
+def test_argument_validation_happens_before_any_launch(lib):
+    """Every error below is found on the host; nothing touches a device (there is none here)."""
+    vp, ci = ctypes.c_void_p, ctypes.c_int
+    ok = vp(0x1000)                      # never dereferenced: validation fails first
+    fwd = lambda ptrs, dims: lib.sfda_forward(*ptrs, *[ci(d) for d in dims], vp(0x2000), ctypes.c_size_t(256), None)
+    base = [ok] * 6 + [None, ok, None, None]
+    dims = [1, 64, 1, 128, 128, 64, 1]
+    assert fwd([None] + base[1:], dims) == -1
+    assert fwd(base, [0] + dims[1:]) == -2
+    assert fwd(base, dims[:3] + [127] + dims[4:]) == -2          # odd d_k
+    assert fwd(base, dims[:3] + [96] + dims[4:]) == -3
+    assert fwd(base, dims[:5] + [48, 1]) == -3
+    assert fwd(base, dims[:6] + [7]) == -3
+    assert fwd([vp(0x1004)] + base[1:], dims) == -4
+    assert lib.sfda_forward(*base, *[ci(d) for d in dims], None, ctypes.c_size_t(0), None) == -5
+    step = lambda ptrs, d: lib.sfda_step(*ptrs, *[ci(x) for x in d], None)
+    sbase = [ok] * 8 + [None]
+    assert step([None] + sbase[1:], [1, 1, 128, 128, 1]) == -1
+    assert step(sbase, [1, 0, 128, 128, 1]) == -2
+    assert step(sbase, [1, 1, 128, 32, 1]) == -3
+    fac = lambda ptrs, d: lib.sfda_chunk_factors(*ptrs, *[ci(x) for x in d], None)
+    fbase = [ok] * 4 + [None] * 5
+    assert fac([None] + fbase[1:], [1, 64, 1, 128, 64, 0]) == -1
+    assert fac(fbase, [1, 64, 1, 128, 24, 0]) == -3
+    n = lib.sfda_forward_host_arena_bytes(1, 64, 1, 128, 128, 64, 1, 1, 1, 1)
+    assert n >= 64 * (3 * 256 + 2 * 256 + 4 + 2 * 256) + 65536
+    assert lib.sfda_forward_host_arena_bytes(1, 64, 1, 100, 128, 64, 1, 1, 1, 1) == 0
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    from paper_2607_11897_b200 import binding
+    monkeypatch.setattr(binding, "_LIB", None)
+    monkeypatch.setattr(binding, "lib_path", lambda: "/nonexistent/libsfda.so")
+    with pytest.raises(ImportError):
+        binding.load()
+
+
+def test_generators_are_deterministic_and_on_the_storage_grid():
+    cfg = workloads.CONFIGS[1].scaled(B=2, T=64, H=2, s0_std=0.02)
+    a, b = workloads.forward_inputs(cfg), workloads.forward_inputs(cfg)
+    for key in a:
+        assert np.array_equal(a[key], b[key])
+    one = workloads.forward_inputs(cfg, batch=[1])
+    assert np.array_equal(one["q"][0], a["q"][1])                    # per-batch-element streams
+    for key in ("q", "k", "v"):
+        assert np.array_equal(workloads.bf16_round(a[key]), a[key])  # exactly representable in bf16
+    assert np.abs(np.linalg.norm(a["k"].astype(np.float64), axis=-1) - 1).max() < 4e-3
+    assert ((a["alpha"] > 0) & (a["alpha"] < 1)).all() and ((a["beta"] > 0) & (a["beta"] < 1)).all()
+    # bf16 rounding: ties to even
+    x = np.array([1.0 + 2 ** -8, 1.0 + 3 * 2 ** -8, 1.0 + 2 ** -9], np.float32)
+    assert np.array_equal(workloads.bf16_round(x), np.array([1.0, 1.0 + 2 ** -6, 1.0], np.float32))
+    c3 = workloads.CONFIGS[3].scaled(T=256, H=4)
+    z = workloads.forward_batch_element(c3, 0)
+    p = workloads.moduli(c3)
+    j = np.rint(np.mod(z["theta"].astype(np.float64), 2 * np.pi) * p / (2 * np.pi))
+    assert np.abs(np.mod(z["theta"].astype(np.float64), 2 * np.pi) - 2 * np.pi * j / p).max() < 1e-6
+    assert set(np.unique(z["beta"])) <= {0.0, 1.0}
+
+
+def _dp_worker(rank, world, port, out_dir):
+    import torch
+    import torch.distributed as dist
+    from oracle import recurrence
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    cfg = workloads.CONFIGS[0].scaled(B=3, T=32, H=2, s0_std=0.1)
+    mine = list(dp.split_batch(cfg.B, world, rank))
+    inp = workloads.forward_inputs(cfg, batch=mine)
+    pairs = [(i, h) for i in range(len(mine)) for h in range(cfg.H)]
+    s = workloads.sequences(inp, pairs)
+    o_re, _, _ = recurrence.sfda_recurrence(s["q"], s["k"], s["v"], s["alpha"], s["theta"], s["beta"], s["S0"])
+    np.save(os.path.join(out_dir, "o_%d.npy" % rank), o_re)
+    np.save(os.path.join(out_dir, "b_%d.npy" % rank), np.array(mine))
+    slowest = dp.max_over_ranks(1.0 + rank)            # rank r pretends to need 1 + r seconds
+    assert slowest == float(world)
+    assert dp.whole_job_throughput(10, world, slowest) == 10 * world / world
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_process_sharding_needs_no_collective(tmp_path):
+    import socket
+    import torch.multiprocessing as mp
+    from oracle import recurrence
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    world = 2
+    mp.spawn(_dp_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    cfg = workloads.CONFIGS[0].scaled(B=3, T=32, H=2, s0_std=0.1)
+    owned = np.concatenate([np.load(tmp_path / ("b_%d.npy" % r)) for r in range(world)])
+    assert sorted(owned.tolist()) == list(range(cfg.B))           # every batch element exactly once
+    inp = workloads.forward_inputs(cfg)
+    pairs = [(b, h) for b in range(cfg.B) for h in range(cfg.H)]
+    s = workloads.sequences(inp, pairs)
+    want, _, _ = recurrence.sfda_recurrence(s["q"], s["k"], s["v"], s["alpha"], s["theta"], s["beta"], s["S0"])
+    got = np.concatenate([np.load(tmp_path / ("o_%d.npy" % r)) for r in range(world)])
+    assert np.array_equal(got, want)                              # shards simply concatenate
+    assert list(dp.rank_batch_range(8, 3)) == list(range(24, 32))
+    assert [len(dp.split_batch(7, 3, r)) for r in range(3)] == [3, 2, 2]
