@@ -4,12 +4,14 @@
 // and hand tiles to one another through mbarriers:
 //
 //   PREP  (8 warps)  chunk j+1: cumulative phase-decay gamma_t = a_t e^{i phi_t} (Eq. "constructive-Gamma";
-//                    log2-sum and integer-turn prefix scans), rotated/decayed operand tiles in shared memory.
+//                    log2-sum and integer-turn prefix scans), rotated/decayed operand tiles in shared memory;
+//                    it also reads the finished outputs of chunk j-1 out of tensor memory for the TMA store.
 //   SOLVE (4 warps)  chunk j+1: drains the Gram blocks from tensor memory, inverts the unit-lower WY system
-//                    (Eq. "constructive-M": M = (I + L)^{-1}) by 16x16 blocks, writes M_beta and Aq tiles.
+//                    (Eq. "constructive-M": M = (I + L)^{-1}) by 8x8 blocks and tensor-core merges, writes the
+//                    M_beta and Aq tiles.
 //   CHAIN (8 warps)  chunk j: the state-dependent conversions between the tcgen05 products
-//                    (state pass, R = V - W^* S_0, E, outputs); they own the TMEM <-> register traffic.
-//   CTRL  (1 thread) issues every tcgen05.mma / commit and the TMA copies.
+//                    (state pass, R = V - W^* S_0, E); they own the TMEM <-> register traffic of the chain.
+//   CTRL  (3 threads) issue every tcgen05.mma / commit and the TMA copies.
 //
 // Algebra (k'_t = e^{-i phi_t} k_t, q'_t = e^{-i phi_t} q_t, all tiles bf16, de-interleaved [Re | Im]):
 //   W_t = a_t k'_t (= conj(gamma_t) k_t, Eq. "constructive-W"),  Qt_t = a_t q'_t,  Kc_t = k'_t / a_t
