@@ -125,6 +125,38 @@ SFDA_API int sfda_forward(const void *q, const void *k, const void *v,
 SFDA_API int sfda_workspace_status(const void *workspace, void *stream, uint32_t *detail);
 
 /*
+ * sfda_forward for callers that cannot hand the library any scratch memory.  (The paper has no counterpart
+ * to this entry point; it exists for deployment reasons only.)
+ *
+ * Who needs it: programs that give all device memory to their own pool at start-up and must not call the
+ * CUDA allocator afterwards -- inference servers with a fixed memory plan, plug-ins running inside another
+ * application's memory budget, real-time loops that cannot afford the device-wide synchronisation an
+ * allocation or a free may cause.  Such a caller can still pass its inputs and outputs (it owns those), but it
+ * has nowhere to take the workspace of sfda_forward from.  Here the workspace is a block of
+ * SFDA_STATIC_SCRATCH_BYTES bytes that is part of the library image itself: every GPU that loads the library
+ * holds that block until the process exits.  This call allocates and frees nothing, directly or through any
+ * library.
+ *
+ * Same arguments, layouts and results as sfda_forward, without workspace.  Restrictions:
+ *  - only the shapes of the tensor-core path (bf16, d_k = d_v = 128, chunk = 64; others need no workspace with
+ *    sfda_forward in the first place) -> SFDA_ERR_UNSUPPORTED otherwise;
+ *  - sizes whose scratch need (sfda_workspace_bytes) exceeds SFDA_STATIC_SCRATCH_BYTES -> SFDA_ERR_WORKSPACE;
+ *  - the first call on each device looks up the block's device address (with that device current); make that
+ *    first call before any stream capture begins;
+ *  - all calls on a device share the one block, which still holds what the previous call left there: this
+ *    call clears the status word on `stream` before the kernel, and two calls whose work overlaps on the GPU
+ *    (different streams) race on it.  Calls on one stream are safe.
+ * sfda_noalloc_status is the counterpart of sfda_workspace_status for that block (synchronises `stream`).
+ */
+#define SFDA_STATIC_SCRATCH_BYTES 256
+SFDA_API int sfda_forward_noalloc(const void *q, const void *k, const void *v,
+                                  const float *alpha, const float *theta, const float *beta,
+                                  const float *S0, void *o, void *o_im, float *S_T,
+                                  int B, int T, int H, int d_k, int d_v, int chunk, int dtype,
+                                  void *stream);
+SFDA_API int sfda_noalloc_status(void *stream, uint32_t *detail);
+
+/*
  * Same computation forced onto the fp32 CUDA-core path for any dtype (the
  * reference path of this library; used to cross-check the tensor-core path).
  * Needs no workspace.

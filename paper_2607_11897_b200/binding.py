@@ -45,6 +45,8 @@ def load():
     lib.sfda_forward_host.argtypes = [_vp] * 10 + [_ci] * 7 + [_vp, _sz, _vp, ctypes.POINTER(_sz),
                                                           ctypes.POINTER(_sz)]
     lib.sfda_last_launch_count.restype = _ci
+    lib.sfda_forward_noalloc.argtypes = [_vp] * 10 + [_ci] * 7 + [_vp]
+    lib.sfda_noalloc_status.argtypes = [_vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.sfda_workspace_status.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_uint32)]
     _LIB = lib
     return lib
@@ -107,7 +109,10 @@ def _forward_common(fn_name, q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chun
         _check(t, n, q.dtype)
     for t, n in ((alpha, "alpha"), (theta, "theta"), (beta, "beta"), (S0, "S0"), (S_T, "S_T")):
         _check(t, n, torch.float32)
-    if fn_name == "sfda_forward":
+    if fn_name == "sfda_forward_noalloc":
+        rc = lib.sfda_forward_noalloc(_ptr(q), _ptr(k), _ptr(v), _ptr(alpha), _ptr(theta), _ptr(beta), _ptr(S0),
+                                      _ptr(o), _ptr(o_im), _ptr(S_T), B, T, H, d_k, d_v, chunk, dt, _stream(stream))
+    elif fn_name == "sfda_forward":
         ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
         rc = lib.sfda_forward(_ptr(q), _ptr(k), _ptr(v), _ptr(alpha), _ptr(theta), _ptr(beta), _ptr(S0), _ptr(o),
                               _ptr(o_im), _ptr(S_T), B, T, H, d_k, d_v, chunk, dt, _ptr(workspace), ws_bytes,
@@ -130,6 +135,22 @@ def sfda_workspace_status(workspace, stream=None) -> int:
     rc = load().sfda_workspace_status(_ptr(workspace), _stream(stream), ctypes.byref(word))
     if rc != 0:
         raise SfdaError(rc, "sfda_workspace_status")
+    return int(word.value)
+
+
+def sfda_forward_noalloc(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chunk, stream=None):
+    """``sfda_forward_noalloc`` of ``include/sfda.h``: the forward on the library's own static scratch block,
+    for callers that may not allocate device memory.  Same tensors as ``sfda_forward``, no workspace."""
+    _forward_common("sfda_forward_noalloc", q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chunk, None, stream)
+
+
+def sfda_noalloc_status(stream=None) -> int:
+    """``sfda_noalloc_status``: 0, or raises SfdaError(-7) when a device-side wait of the last
+    ``sfda_forward_noalloc`` call ran out.  Synchronises the stream."""
+    word = ctypes.c_uint32()
+    rc = load().sfda_noalloc_status(_stream(stream), ctypes.byref(word))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_noalloc_status")
     return int(word.value)
 
 

@@ -117,6 +117,29 @@ int sfda_forward(const void *q, const void *k, const void *v, const float *alpha
     return e == cudaSuccess ? SFDA_OK : SFDA_ERR_CUDA;
 }
 
+int sfda_forward_noalloc(const void *q, const void *k, const void *v, const float *alpha, const float *theta,
+                         const float *beta, const float *S0, void *o, void *o_im, float *S_T, int B, int T, int H,
+                         int d_k, int d_v, int chunk, int dtype, void *stream)
+{
+    g_last_launches = 0;
+    const int rc = validate_forward(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
+    if (rc != SFDA_OK) return rc;
+    const sfda::ForwardArgs a = pack(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
+    if (!sfda::forward_ws_supported(a)) return SFDA_ERR_UNSUPPORTED;     // only the kernel that uses scratch
+    if (sfda_workspace_bytes(B, T, H, d_k, d_v, chunk, dtype) > SFDA_STATIC_SCRATCH_BYTES) return SFDA_ERR_WORKSPACE;
+    return sfda::launch_forward_ws_static(a, static_cast<cudaStream_t>(stream), &g_last_launches) == cudaSuccess
+               ? SFDA_OK
+               : SFDA_ERR_CUDA;
+}
+
+int sfda_noalloc_status(void *stream, uint32_t *detail)
+{
+    uint32_t word = 0;
+    if (sfda::read_static_status(static_cast<cudaStream_t>(stream), &word) != cudaSuccess) return SFDA_ERR_CUDA;
+    if (detail) *detail = word;
+    return word == 0 ? SFDA_OK : SFDA_ERR_TIMEOUT;
+}
+
 int sfda_workspace_status(const void *workspace, void *stream, uint32_t *detail)
 {
     if (!workspace) return SFDA_ERR_NULL;

@@ -24,6 +24,8 @@
 // the next chunk's state pass, so no operand depends on the chunk's total decay.
 #include <cuda.h>
 
+#include <mutex>
+
 #include "sfda_common.cuh"
 #include "sfda_internal.h"
 #include "sfda_tc_ptx.cuh"
@@ -919,6 +921,56 @@ bool make_map(CUtensorMap *map, const void *base, int B, int T, int H)
 }
 
 }  // namespace
+
+// ---- scratch that nobody allocates -------------------------------------------------------------------
+// The tensor-core kernel keeps its status word in caller-provided scratch.  For callers that cannot provide
+// any, the same kernel can run on this statically allocated block instead: it is part of the library image,
+// so every GPU that loads the library holds these bytes until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void *g_static_ptr[kMaxDevices] = {};   // device address of g_static_scratch, per device ordinal
+
+// In host code `g_static_scratch` is only a handle, not a device address; the address has to be asked for,
+// once per device, with that device current.
+cudaError_t static_scratch_address(void **out)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void *ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        g_static_ptr[dev] = ptr;
+    }
+    *out = g_static_ptr[dev];
+    return cudaSuccess;
+}
+}  // namespace
+
+cudaError_t launch_forward_ws_static(const ForwardArgs &a, cudaStream_t stream, int *launches)
+{
+    void *scratch = nullptr;
+    const cudaError_t e = static_scratch_address(&scratch);
+    if (e != cudaSuccess) return e;
+    // the block keeps whatever the last call left in it; the launcher clears the status word on the stream
+    return launch_forward_ws(a, static_cast<uint32_t *>(scratch), stream, launches);
+}
+
+cudaError_t read_static_status(cudaStream_t stream, uint32_t *word)
+{
+    void *scratch = nullptr;
+    cudaError_t e = static_scratch_address(&scratch);
+    if (e != cudaSuccess) return e;
+    e = cudaMemcpyAsync(word, scratch, sizeof(uint32_t), cudaMemcpyDeviceToHost, stream);
+    if (e != cudaSuccess) return e;
+    return cudaStreamSynchronize(stream);
+}
 
 bool forward_ws_supported(const ForwardArgs &a) { return a.dtype == 1 && a.d_k == DK && a.d_v == DV && a.chunk == C; }
 

@@ -37,6 +37,11 @@ cudaError_t launch_forward_simt(const ForwardArgs &a, cudaStream_t stream, int *
 // before the launch.
 bool forward_ws_supported(const ForwardArgs &a);
 cudaError_t launch_forward_ws(const ForwardArgs &a, uint32_t *status, cudaStream_t stream, int *launches);
+// The same kernel on the library's own statically allocated scratch block (kStaticScratchBytes), and a read of
+// the status word kept there (synchronises the stream).  Neither allocates.
+constexpr size_t kStaticScratchBytes = 256;
+cudaError_t launch_forward_ws_static(const ForwardArgs &a, cudaStream_t stream, int *launches);
+cudaError_t read_static_status(cudaStream_t stream, uint32_t *word);
 cudaError_t launch_chunk_factors(const FactorArgs &a, cudaStream_t stream, int *launches);
 cudaError_t launch_step(const StepArgs &a, cudaStream_t stream, int *launches);
 
