@@ -356,6 +356,31 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
     }
 }
 
+__device__ __forceinline__ void prefetch_l2(const void *ptr)
+{
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+}
+// ---- input prefetch ------------------------------------------------------------------------------------
+// PREP reads q, k, alpha, theta straight from global memory (no shared memory is left to stage them).  So that
+// those loads find their lines in L2 instead of stalling on HBM in a burst, one otherwise idle warp touches the
+// rows of a chunk two chunks before PREP gets there: 64 tokens x 4 arrays x 256 bytes = 512 lines per chunk.
+__device__ __forceinline__ void run_prefetch(Misc &mi, const Params &p, int b, int h, int n_chunks, int lane)
+{
+    for (int j = 0; j < n_chunks; ++j) {
+        if (j >= 2 && !wait_k(mi, (j - 2) & 1 ? B_PREP_FULL1 : B_PREP_FULL0, (j - 2) >> 1)) return;
+        const int t0 = j * C, len = min(C, p.T - t0);
+        const size_t row0 = ((size_t)b * p.T + t0) * p.H + h;
+        for (int idx = lane; idx < 2 * len; idx += 32) {
+            const size_t row = row0 + (size_t)(idx >> 1) * p.H;
+            const size_t off = (size_t)(idx & 1) * 128;
+            prefetch_l2(reinterpret_cast<const char *>(p.alpha + row * M) + off);
+            prefetch_l2(reinterpret_cast<const char *>(p.theta + row * M) + off);
+            prefetch_l2(reinterpret_cast<const char *>(p.k + row * DK) + off);
+            prefetch_l2(reinterpret_cast<const char *>(p.q + row * DK) + off);
+        }
+    }
+}
+
 // ---- PREP ---------------------------------------------------------------------------------------------
 // e^{-i phi} from the integer phase: the top 23 bits of the turn count make a float in [1, 2); centred to
 // [-0.5, 0.5) turns it is well inside the accurate range of the fast sine / cosine.
@@ -411,6 +436,7 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
         const int t0 = j * C, len = min(C, p.T - t0);
         const size_t row0 = ((size_t)b * p.T + t0) * p.H + h;   // token t of this head: row0 + t * H
         const int nt = min(8, max(0, len - tq * 8));             // real tokens in this thread's octet
+        SFDA_T(35);
 
         // all loads of this thread for the chunk, issued together
         float2 al[8], th[8];
@@ -429,18 +455,20 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
                 qw[i] = __ldg(reinterpret_cast<const uint2 *>(p.q + row * DK) + jp);
             }
         }
+        SFDA_T(36);
         if (pt < C) mi.beta[ring][pt] = pt < len ? __ldg(p.beta + row0 + (size_t)pt * p.H) : 0.f;
-
-        // pass 1: prefix sums of log2 alpha and of the integer phase over this thread's 8 tokens
+        SFDA_T(37);
+        // pass 1: prefix products of alpha (a_t: fp32 products of at most 64 factors, relative error far below
+        // bf16's) and prefix sums of the integer phase over this thread's 8 tokens
         float lg0[8], lg1[8];
         uint32_t tu0[8], tu1[8];
         {
-            float a0 = 0.f, a1 = 0.f;
+            float a0 = 1.f, a1 = 1.f;
             uint32_t u0 = 0u, u1 = 0u;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                a0 += fmaxf(__log2f(al[i].x), -43.28f);   // floor e^-30, as in log_decay
-                a1 += fmaxf(__log2f(al[i].y), -43.28f);
+                a0 *= fmaxf(al[i].x, 9.0e-14f);           // floor e^-30, as in log_decay
+                a1 *= fmaxf(al[i].y, 9.0e-14f);
                 u0 += phase_to_turns(th[i].x);
                 u1 += phase_to_turns(th[i].y);
                 lg0[i] = a0; lg1[i] = a1; tu0[i] = u0; tu1[i] = u1;
@@ -452,18 +480,18 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
         }
         SFDA_T(30);
         role_sync(2, kPrepThreads);
-        float base0 = 0.f, base1 = 0.f, tot0 = 0.f, tot1 = 0.f;
+        float base0 = 1.f, base1 = 1.f, tot0 = 1.f, tot1 = 1.f;
         uint32_t tb0 = 0u, tb1 = 0u, tt0 = 0u, tt1 = 0u;
 #pragma unroll
         for (int gq = 0; gq < 8; ++gq) {
             const float2 pl = *reinterpret_cast<const float2 *>(&mi.part_lg[gq][2 * jp]);
             const uint2 pu = *reinterpret_cast<const uint2 *>(&mi.part_turns[gq][2 * jp]);
-            if (gq < tq) { base0 += pl.x; base1 += pl.y; tb0 += pu.x; tb1 += pu.y; }
-            tot0 += pl.x; tot1 += pl.y; tt0 += pu.x; tt1 += pu.y;
+            if (gq < tq) { base0 *= pl.x; base1 *= pl.y; tb0 += pu.x; tb1 += pu.y; }
+            tot0 *= pl.x; tot1 *= pl.y; tt0 += pu.x; tt1 += pu.y;
         }
         if (tq == 0) {                    // chunk totals: a_C e^{i phi_C}, applied by the next state pass
             float cs, sn;
-            const float a0 = exp2f(tot0), a1 = exp2f(tot1);
+            const float a0 = tot0, a1 = tot1;
             turns_sincos(tt0, &sn, &cs);
             mi.close_re[ring][2 * jp] = a0 * cs;
             mi.close_im[ring][2 * jp] = a0 * sn;
@@ -493,11 +521,10 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
             float wr[2], wi[2], cr_[2], ci_[2], qr_[2], qi_[2];
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
-                const float l2 = x ? base1 + lg1[i] : base0 + lg0[i];
+                const float a = x ? base1 * lg1[i] : base0 * lg0[i];           // a_t
                 const uint32_t tu = x ? tb1 + tu1[i] : tb0 + tu0[i];
                 const uint32_t kx = x ? kw[i].y : kw[i].x, qx = x ? qw[i].y : qw[i].x;
-                const float a = exp2f(l2);
-                const float ainv = exp2f(fminf(-l2, 115.4f));                 // 1/a_t, capped at e^80
+                const float ainv = fminf(__fdividef(1.0f, a), 5.5e34f);              // 1/a_t, capped at e^80
                 float cs, sn;
                 turns_sincos(tu, &sn, &cs);
                 const float kr = __uint_as_float(kx << 16), ki = __uint_as_float(kx & 0xffff0000u);
@@ -559,13 +586,11 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
                     const float bt = mi.beta[ring][t];
                     float4 *dst = reinterpret_cast<float4 *>((im ? Li : Lr) + t * LS + 32 * hc);
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        const int ii = 32 * hc + i;
-                        dst[i >> 2] = make_float4(ii < t ? bt * __uint_as_float(r[i]) : 0.f,
-                                                  ii + 1 < t ? bt * __uint_as_float(r[i + 1]) : 0.f,
-                                                  ii + 2 < t ? bt * __uint_as_float(r[i + 2]) : 0.f,
-                                                  ii + 3 < t ? bt * __uint_as_float(r[i + 3]) : 0.f);
-                    }
+                    // no mask: the substitution reads only entries below the diagonal of an 8x8 block and then
+                    // overwrites the whole block; the merges read whole blocks strictly below the diagonal
+                    for (int i = 0; i < 32; i += 4)
+                        dst[i >> 2] = make_float4(bt * __uint_as_float(r[i]), bt * __uint_as_float(r[i + 1]),
+                                                  bt * __uint_as_float(r[i + 2]), bt * __uint_as_float(r[i + 3]));
                 } else {                          // Aq, lower incl. diagonal, as a bf16 operand tile
                     const int t = row - 64;
                     uint8_t *tile = smem + OFF_AQ + (s * 2 + im) * kTile;
@@ -877,7 +902,10 @@ sfda_forward_ws_kernel(const __grid_constant__ CUtensorMap tm_v, const __grid_co
     } else {
         regs_dec<kRegsCtrl>();
         const int cw = warp - (kChainWarps + kSolveWarps + kPrepWarps);
-        if ((tid & 31) == 0 && cw < 3) run_ctrl(cw, smem, mi, tmem, &tm_v, &tm_o, &tm_oim, p, b, h, n_chunks);
+        if (cw == 3)
+            run_prefetch(mi, p, b, h, n_chunks, tid & 31);
+        else if ((tid & 31) == 0)
+            run_ctrl(cw, smem, mi, tmem, &tm_v, &tm_o, &tm_oim, p, b, h, n_chunks);
     }
 
     tc_fence_before();
