@@ -122,6 +122,13 @@ __device__ __forceinline__ void mbar_arrive(unsigned long long *bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// One arrival per warp: the warp's lanes order their writes among themselves with __syncwarp, then one lane
+// arrives (a barrier counted in warps completes after a handful of shared-memory atomics instead of hundreds).
+__device__ __forceinline__ void warp_arrive(unsigned long long *bar)
+{
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
+}
 template <int N>
 __device__ __forceinline__ void regs_inc()
 {
@@ -423,7 +430,7 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
         }
         fence_async_smem();
         tc_fence_before();
-        mbar_arrive(&mi.bars[B_O_STAGED]);
+        warp_arrive(&mi.bars[B_O_STAGED]);
     };
     SFDA_TDECL(pt == 0);
     for (int j = 0; j < n_chunks + 2; ++j) {
@@ -544,7 +551,7 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
             *reinterpret_cast<uint32_t *>(kc_im + o1) = pack_bf16(ci_[0], ci_[1]);
         }
         fence_async_smem();
-        mbar_arrive(&mi.bars[s ? B_PREP_FULL1 : B_PREP_FULL0]);
+        warp_arrive(&mi.bars[s ? B_PREP_FULL1 : B_PREP_FULL0]);
         SFDA_T(33);
     }
 }
@@ -579,7 +586,7 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
                 tc_wait_ld();
                 if (hc == 1) {
                     tc_fence_before();
-                    mbar_arrive(&mi.bars[B_GRAM_DRAINED]);
+                    warp_arrive(&mi.bars[B_GRAM_DRAINED]);
                 }
                 if (row < 64) {                   // L = D_beta Kt, strictly lower
                     const int t = row;
@@ -609,7 +616,7 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
             }
         }
         fence_async_smem();
-        mbar_arrive(&mi.bars[s ? B_AQ_FULL1 : B_AQ_FULL0]);
+        warp_arrive(&mi.bars[s ? B_AQ_FULL1 : B_AQ_FULL0]);
         role_sync(1, kSolveThreads);
         SFDA_T(24);
 
@@ -721,12 +728,18 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
             }
         }
         fence_async_smem();
-        mbar_arrive(&mi.bars[B_MB_FULL]);
+        warp_arrive(&mi.bars[B_MB_FULL]);
         SFDA_T(29);
     }
 }
 
 // ---- CHAIN --------------------------------------------------------------------------------------------
+// wait_k with a warp-uniform outcome, so that a warp leaves (or stays) as a whole
+__device__ __forceinline__ bool wait_k_warp(Misc &mi, int bar, int k)
+{
+    return __all_sync(0xffffffffu, wait_k(mi, bar, k) ? 1 : 0) != 0;
+}
+
 __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int bh, int n_chunks,
                                           int ct)
 {
@@ -790,7 +803,7 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
                     pk[16 * hc + i] = pack_bf16(sgn * __uint_as_float(r[2 * i]), sgn * __uint_as_float(r[2 * i + 1]));
             }
         }
-        if (gate_bar >= 0 && !wait_k(mi, gate_bar, gate_k)) return false;
+        if (gate_bar >= 0 && !wait_k_warp(mi, gate_bar, gate_k)) return false;
         tmem_st<32>(tlane + TM_X16 + 32 * half, pk);
         tc_wait_st();
         return true;
@@ -800,7 +813,7 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
     for (int j = 0; j < n_chunks; ++j) {
         // ---- state pass: S_0 of this chunk = e^{i phi_C} a_C (accumulated state of the previous chunk)
         if (j > 0) {
-            if (!wait_k(mi, B_UPD_DONE, j - 1)) return;
+            if (!wait_k_warp(mi, B_UPD_DONE, j - 1)) return;
             tc_fence_after();
         }
         SFDA_T(10);
@@ -808,31 +821,31 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
         state_piece(1, (j - 1) & 3, j == 0);
         tc_wait_st();
         tc_fence_before();
-        mbar_arrive(&mi.bars[B_S16_READY]);
+        warp_arrive(&mi.bars[B_S16_READY]);
         SFDA_T(11);
 
         // ---- R = V - D1 -> bf16 A operand (D1 and rho_1, which read S_0 from the same columns, are both done)
-        if (!wait_k(mi, B_D1_DONE, j)) return;
-        if (!wait_k(mi, B_V_FULL, j)) return;
+        if (!wait_k_warp(mi, B_D1_DONE, j)) return;
+        if (!wait_k_warp(mi, B_V_FULL, j)) return;
         tc_fence_after();
         SFDA_T(13);
         if (!convert_acc(half == 0, half == 1, -1, 0)) return;
         tc_fence_before();
-        mbar_arrive(&mi.bars[B_R16_READY]);
+        warp_arrive(&mi.bars[B_R16_READY]);
         SFDA_T(14);
 
         // ---- E -> bf16 A operand
-        if (!wait_k(mi, B_E_DONE, j)) return;
+        if (!wait_k_warp(mi, B_E_DONE, j)) return;
         tc_fence_after();
         SFDA_T(15);
         if (!convert_acc(false, false, -1, 0)) return;
         tc_fence_before();
-        mbar_arrive(&mi.bars[B_E16_READY]);
+        warp_arrive(&mi.bars[B_E16_READY]);
         SFDA_T(16);
     }
 
     // ---- last chunk: outputs and the final state
-    if (!wait_k(mi, B_UPD_DONE, n_chunks - 1)) return;
+    if (!wait_k_warp(mi, B_UPD_DONE, n_chunks - 1)) return;
     tc_fence_after();
     if (p.S_T) {
         const int ring = (n_chunks - 1) & 3;
@@ -870,14 +883,14 @@ sfda_forward_ws_kernel(const __grid_constant__ CUtensorMap tm_v, const __grid_co
 
     if (tid == 0) {
         auto init = [&](int bar, uint32_t count) { mbar_init(&mi.bars[bar], count); };
-        init(B_PREP_FULL0, kPrepThreads); init(B_PREP_FULL1, kPrepThreads);
+        init(B_PREP_FULL0, kPrepWarps); init(B_PREP_FULL1, kPrepWarps);
         init(B_WQ_FREE0, 1); init(B_WQ_FREE1, 1); init(B_KC_FREE0, 1); init(B_KC_FREE1, 1);
         init(B_STORE_DONE0, 1); init(B_STORE_DONE1, 1);
-        init(B_GRAM_FULL, 1); init(B_GRAM_DRAINED, kSolveThreads);
-        init(B_MB_FULL, kSolveThreads); init(B_AQ_FULL0, kSolveThreads); init(B_AQ_FULL1, kSolveThreads);
+        init(B_GRAM_FULL, 1); init(B_GRAM_DRAINED, kSolveWarps);
+        init(B_MB_FULL, kSolveWarps); init(B_AQ_FULL0, kSolveWarps); init(B_AQ_FULL1, kSolveWarps);
         init(B_D1_DONE, 1); init(B_E_DONE, 1); init(B_UPD_DONE, 2);   // state update and rho += Aq E
-        init(B_S16_READY, kChainThreads); init(B_R16_READY, kChainThreads); init(B_E16_READY, kChainThreads);
-        init(B_O_STAGED, kPrepThreads); init(B_V_FULL, 1);
+        init(B_S16_READY, kChainWarps); init(B_R16_READY, kChainWarps); init(B_E16_READY, kChainWarps);
+        init(B_O_STAGED, kPrepWarps); init(B_V_FULL, 1);
         mi.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
