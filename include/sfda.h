@@ -82,8 +82,11 @@ SFDA_API const char *sfda_status_string(int status);
 SFDA_API int sfda_plan(int T, int chunk, int *n_chunks, int *tail_len);
 
 /*
- * Bytes of device scratch sfda_forward needs for these sizes (0 when it needs
- * none; 256 for the tensor-core path, which keeps a status word there).  Returns 0 for invalid sizes as well; sfda_forward reports those.
+ * Bytes of device scratch sfda_forward should be given for these sizes (0 when it
+ * needs none).  The tensor-core path keeps a 256-byte status block there and, when it
+ * gets the full size (256 + 4*B*H rounded up to 256 + B*H*d_k*d_v*4 bytes), also the
+ * boundary states of the time slices it may cut long sequences into to keep every SM
+ * busy; with at least 256 bytes it still runs, one (batch, head) pair per CTA at a time.  Returns 0 for invalid sizes as well; sfda_forward reports those.
  */
 SFDA_API size_t sfda_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int dtype);
 
@@ -98,8 +101,9 @@ SFDA_API size_t sfda_workspace_bytes(int B, int T, int H, int d_k, int d_v, int 
  *  S0     [B][H][d_k][d_v] float, or NULL for a zero initial state
  *  o      [B][T][H][d_v]   dtype          o_im same shape, or NULL
  *  S_T    [B][H][d_k][d_v] float, or NULL; may alias S0
- *  workspace: device scratch of at least sfda_workspace_bytes(...) bytes (may be
- *             NULL when that is 0); contents are clobbered.
+ *  workspace: device scratch, sfda_workspace_bytes(...) bytes for full speed (may be
+ *             NULL when that is 0; the tensor-core path needs at least 256 bytes);
+ *             contents are clobbered.
  *
  * Supported: d_k, d_v in {64, 128}; chunk in {16, 32, 64}.
  * bf16 inputs with d_k = d_v = 128 and chunk = 64 take the tensor-core path
@@ -140,7 +144,9 @@ SFDA_API int sfda_workspace_status(const void *workspace, void *stream, uint32_t
  * Same arguments, layouts and results as sfda_forward, without workspace.  Restrictions:
  *  - only the shapes of the tensor-core path (bf16, d_k = d_v = 128, chunk = 64; others need no workspace with
  *    sfda_forward in the first place) -> SFDA_ERR_UNSUPPORTED otherwise;
- *  - sizes whose scratch need (sfda_workspace_bytes) exceeds SFDA_STATIC_SCRATCH_BYTES -> SFDA_ERR_WORKSPACE;
+ *  - it runs on the kernel's minimum scratch (the status block), so without the time slicing sfda_forward does
+ *    with a full workspace; a kernel whose minimum exceeded SFDA_STATIC_SCRATCH_BYTES would be refused with
+ *    SFDA_ERR_WORKSPACE;
  *  - the first call on each device looks up the block's device address (with that device current); make that
  *    first call before any stream capture begins;
  *  - all calls on a device share the one block, which still holds what the previous call left there: this

@@ -82,7 +82,8 @@ size_t sfda_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, in
     if (B < 1 || T < 1 || H < 1 || check_dims(d_k, d_v, chunk, dtype) != SFDA_OK) return 0;
     sfda::ForwardArgs a{};
     a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.chunk = chunk; a.dtype = dtype;
-    return sfda::forward_ws_supported(a) ? 256 : 0;   // the tensor-core path keeps a status word there
+    // the tensor-core path keeps a status word there, and the boundary states of its time slices
+    return sfda::forward_ws_supported(a) ? sfda::forward_ws_scratch_bytes(B, H) : 0;
 }
 
 int sfda_forward_simt(const void *q, const void *k, const void *v, const float *alpha, const float *theta,
@@ -105,13 +106,14 @@ int sfda_forward(const void *q, const void *k, const void *v, const float *alpha
     g_last_launches = 0;
     const int rc = validate_forward(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
     if (rc != SFDA_OK) return rc;
-    const size_t need = sfda_workspace_bytes(B, T, H, d_k, d_v, chunk, dtype);
+    const sfda::ForwardArgs a = pack(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
+    // the tensor-core path runs with as little as its status block; the full size enables time slicing
+    const size_t need = sfda::forward_ws_supported(a) ? sfda::kWsMinScratchBytes : 0;
     if (need > 0 && (!workspace || workspace_bytes < need)) return SFDA_ERR_WORKSPACE;
     if (workspace && !aligned16(workspace)) return SFDA_ERR_ALIGN;
-    const sfda::ForwardArgs a = pack(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
     const cudaError_t e =
         sfda::forward_ws_supported(a)
-            ? sfda::launch_forward_ws(a, static_cast<uint32_t *>(workspace), static_cast<cudaStream_t>(stream),
+            ? sfda::launch_forward_ws(a, workspace, workspace_bytes, static_cast<cudaStream_t>(stream),
                                       &g_last_launches)
             : sfda::launch_forward_simt(a, static_cast<cudaStream_t>(stream), &g_last_launches);
     return e == cudaSuccess ? SFDA_OK : SFDA_ERR_CUDA;
@@ -126,7 +128,7 @@ int sfda_forward_noalloc(const void *q, const void *k, const void *v, const floa
     if (rc != SFDA_OK) return rc;
     const sfda::ForwardArgs a = pack(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
     if (!sfda::forward_ws_supported(a)) return SFDA_ERR_UNSUPPORTED;     // only the kernel that uses scratch
-    if (sfda_workspace_bytes(B, T, H, d_k, d_v, chunk, dtype) > SFDA_STATIC_SCRATCH_BYTES) return SFDA_ERR_WORKSPACE;
+    if (sfda::kWsMinScratchBytes > SFDA_STATIC_SCRATCH_BYTES) return SFDA_ERR_WORKSPACE;
     return sfda::launch_forward_ws_static(a, static_cast<cudaStream_t>(stream), &g_last_launches) == cudaSuccess
                ? SFDA_OK
                : SFDA_ERR_CUDA;

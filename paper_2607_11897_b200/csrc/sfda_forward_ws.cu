@@ -115,8 +115,68 @@ struct Params {
     const float *alpha, *theta, *beta, *S0;
     float *S_T;
     uint32_t *status;
+    uint32_t *flags;     // [B*H] progress counters of the time slices (only used when Q > 1)
+    float *handoff;      // [B*H][d_k][d_v] boundary states between time slices (only used when Q > 1)
     int T, H, has_o_im;
+    int BH, U, Q, n_units;   // sequences, chunks per work unit, time slices per sequence, Q * BH
 };
+
+// Work units.  A sequence is cut into Q time slices of U chunks; unit u = slice * BH + sequence.  CTA c works
+// through units c, c + gridDim, ... as ONE stream of chunks, so its pipeline never drains between units; only
+// the state pass notices a unit boundary (it writes the finished state out and takes the next one in).  A slice
+// q > 0 starts from the boundary state slice q - 1 left in `handoff`; its CTA waits for that (bounded).  Units
+// are handed out in increasing order and every CTA is resident, so the unit a CTA waits for is always already
+// running or done.
+struct ChunkInfo {
+    int b, h, bh, jg, q;   // sequence, chunk index inside the sequence, time slice
+    bool first, last;      // first / last chunk of its unit
+};
+// Walks the stream chunk by chunk; the divisions happen once per unit, not once per chunk.
+struct ChunkCursor {
+    ChunkInfo ci;
+    int jl, u;
+    __device__ __forceinline__ void set_unit(const Params &p)
+    {
+        ci.q = u / p.BH;
+        ci.bh = u - ci.q * p.BH;
+        ci.b = ci.bh / p.H;
+        ci.h = ci.bh - ci.b * p.H;
+    }
+    __device__ __forceinline__ void refresh(const Params &p)
+    {
+        ci.jg = ci.q * p.U + jl;
+        ci.first = jl == 0;
+        ci.last = jl == p.U - 1;
+    }
+    __device__ __forceinline__ explicit ChunkCursor(const Params &p) : jl(0), u((int)blockIdx.x)
+    {
+        set_unit(p);
+        refresh(p);
+    }
+    __device__ __forceinline__ void next(const Params &p)
+    {
+        if (++jl == p.U) {
+            jl = 0;
+            u += (int)gridDim.x;
+            set_unit(p);
+        }
+        refresh(p);
+    }
+};
+__device__ __forceinline__ ChunkInfo chunk_info(const Params &p, int jj)
+{
+    const int ul = jj / p.U, jl = jj - ul * p.U;
+    const int u = (int)blockIdx.x + ul * (int)gridDim.x;
+    ChunkInfo ci;
+    ci.q = u / p.BH;
+    ci.bh = u - ci.q * p.BH;
+    ci.b = ci.bh / p.H;
+    ci.h = ci.bh - ci.b * p.H;
+    ci.jg = ci.q * p.U + jl;
+    ci.first = jl == 0;
+    ci.last = jl == p.U - 1;
+    return ci;
+}
 
 __device__ __forceinline__ void mbar_arrive(unsigned long long *bar)
 {
@@ -155,13 +215,17 @@ __device__ __forceinline__ void role_sync(int id, int nthreads)
     asm volatile("barrier.cta.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
+// Waits are bounded in ticks of the SM's own clock counter, which is cheap to read.
+__device__ __forceinline__ unsigned long long now_ticks() { return (unsigned long long)clock64(); }
+constexpr unsigned long long kWaitLimitTicks = 4000000000ull;   // about 2 s at the maximum SM clock
+#ifdef SFDA_WS_TIMING
 __device__ __forceinline__ unsigned long long now_ns()
 {
     unsigned long long t;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // no wait of this kernel may last longer than 2 s
+#endif
 
 // Non-blocking test of completion number k (0-based) of a barrier.
 __device__ __forceinline__ bool test_k(Misc &mi, int bar, int k)
@@ -173,7 +237,7 @@ __device__ __forceinline__ bool test_k(Misc &mi, int bar, int k)
                  : "memory");
     return ok != 0;
 }
-// Wait for completion number k; gives up after kWaitLimitNs or when another role has raised the abort flag.
+// Wait for completion number k; gives up after kWaitLimitTicks or when another role has raised the abort flag.
 // Returns false in that case, after raising the flag itself.  try_wait parks the thread in hardware for up to
 // the hinted time, so waiting warps do not compete with working ones for issue slots.
 __device__ __forceinline__ bool wait_k(Misc &mi, int bar, int k)
@@ -189,9 +253,9 @@ __device__ __forceinline__ bool wait_k(Misc &mi, int bar, int k)
             : "memory");
         if (ok) return true;
         if (mi.abort) return false;
-        const unsigned long long t = now_ns();
+        const unsigned long long t = now_ticks();
         if (it == 0) t0 = t;
-        else if (t - t0 > kWaitLimitNs) break;
+        else if (t - t0 > kWaitLimitTicks) break;
     }
     mi.abort = 1;
     return false;
@@ -222,8 +286,8 @@ __device__ __forceinline__ void mma4_ss(uint32_t d, uint32_t a, uint32_t b, uint
 //   role 1  the output products rho_1 and rho += Aq E, and the output stores
 //   role 2  the Gram products (they run ahead of the chain) and the v loads
 __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint32_t tmem, const CUtensorMap *tm_v,
-                                         const CUtensorMap *tm_o, const CUtensorMap *tm_oim, const Params &p, int b,
-                                         int h, int n_chunks)
+                                         const CUtensorMap *tm_o, const CUtensorMap *tm_oim, const Params &p,
+                                         int n_chunks)
 {
     long long *timing = p.timing;
     const uint64_t dbase = smem_desc(smem_u32(smem));                     // descriptor of byte offset 0
@@ -283,14 +347,18 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
             SFDA_T(6);
         }
     } else if (role == 1) {
+        ChunkCursor prev(p);             // chunk j - 1 inside the loop
         for (int j = 0; j < n_chunks; ++j) {
             const int s = j & 1, u = j >> 1;
             const uint32_t a_re = desc(OFF_AQ + s * 2 * kTile), a_im = a_re + (kTile >> 4);
             // outputs of the previous chunk are staged: store them
             if (j > 0) {
                 if (!wait_k(mi, B_O_STAGED, j - 1)) return;
-                tma_store_4d(tm_o, smem + OFF_OST, 0, h, (j - 1) * C, b);
-                if (p.has_o_im) tma_store_4d(tm_oim, smem + OFF_AQ + ((j - 1) & 1) * 2 * kTile, 0, h, (j - 1) * C, b);
+                const ChunkInfo pc = prev.ci;
+                prev.next(p);
+                tma_store_4d(tm_o, smem + OFF_OST, 0, pc.h, pc.jg * C, pc.b);
+                if (p.has_o_im)
+                    tma_store_4d(tm_oim, smem + OFF_AQ + ((j - 1) & 1) * 2 * kTile, 0, pc.h, pc.jg * C, pc.b);
                 tma_store_commit();
                 tma_store_wait_read();
                 mbar_arrive(&bars[(j - 1) & 1 ? B_STORE_DONE1 : B_STORE_DONE0]);
@@ -306,18 +374,20 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
             mma_commit(&bars[B_UPD_DONE]);
         }
         if (!wait_k(mi, B_O_STAGED, n_chunks - 1)) return;
-        tma_store_4d(tm_o, smem + OFF_OST, 0, h, (n_chunks - 1) * C, b);
+        const ChunkInfo pc = prev.ci;
+        tma_store_4d(tm_o, smem + OFF_OST, 0, pc.h, pc.jg * C, pc.b);
         if (p.has_o_im)
-            tma_store_4d(tm_oim, smem + OFF_AQ + ((n_chunks - 1) & 1) * 2 * kTile, 0, h, (n_chunks - 1) * C, b);
+            tma_store_4d(tm_oim, smem + OFF_AQ + ((n_chunks - 1) & 1) * 2 * kTile, 0, pc.h, pc.jg * C, pc.b);
         tma_store_commit();
         tma_store_wait_all();
     } else {
         // Gram chunk g, half gh, as soon as its operands are written and the Gram columns have been drained;
         // v of chunk jv as soon as v of chunk jv-1 has been consumed (R of that chunk is built).
+        ChunkCursor vcur(p);             // chunk jv - 1 below, advanced before each further load
         mbar_expect_tx(&bars[B_V_FULL], 16384);
-        tma_load_4d(smem + OFF_V, tm_v, &bars[B_V_FULL], 0, h, 0, b);
+        tma_load_4d(smem + OFF_V, tm_v, &bars[B_V_FULL], 0, vcur.ci.h, vcur.ci.jg * C, vcur.ci.b);
         int g = 0, gh = 0, jv = 1;
-        const unsigned long long t0 = now_ns();
+        const unsigned long long t0 = now_ticks();
         for (uint32_t it = 0; g < n_chunks || jv < n_chunks; ++it) {
             bool progress = false;
             if (g < n_chunks) {
@@ -344,8 +414,10 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
                 }
             }
             if (jv < n_chunks && test_k(mi, B_R16_READY, jv - 1)) {
+                vcur.next(p);
+                const ChunkInfo cv = vcur.ci;
                 mbar_expect_tx(&bars[B_V_FULL], 16384);
-                tma_load_4d(smem + OFF_V, tm_v, &bars[B_V_FULL], 0, h, jv * C, b);
+                tma_load_4d(smem + OFF_V, tm_v, &bars[B_V_FULL], 0, cv.h, cv.jg * C, cv.b);
                 ++jv;
                 progress = true;
             }
@@ -353,7 +425,7 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
                 __nanosleep(64);
                 if ((it & 63u) == 63u) {
                     if (mi.abort) return;
-                    if (now_ns() - t0 > 2 * kWaitLimitNs + 1000000ull * (unsigned long long)n_chunks) {
+                    if (now_ticks() - t0 > 2 * kWaitLimitTicks + 2000000ull * (unsigned long long)n_chunks) {
                         mi.abort = 1;
                         return;
                     }
@@ -371,12 +443,14 @@ __device__ __forceinline__ void prefetch_l2(const void *ptr)
 // PREP reads q, k, alpha, theta straight from global memory (no shared memory is left to stage them).  So that
 // those loads find their lines in L2 instead of stalling on HBM in a burst, one otherwise idle warp touches the
 // rows of a chunk two chunks before PREP gets there: 64 tokens x 4 arrays x 256 bytes = 512 lines per chunk.
-__device__ __forceinline__ void run_prefetch(Misc &mi, const Params &p, int b, int h, int n_chunks, int lane)
+__device__ __forceinline__ void run_prefetch(Misc &mi, const Params &p, int n_chunks, int lane)
 {
-    for (int j = 0; j < n_chunks; ++j) {
+    ChunkCursor cur(p);
+    for (int j = 0; j < n_chunks; ++j, cur.next(p)) {
         if (j >= 2 && !wait_k(mi, (j - 2) & 1 ? B_PREP_FULL1 : B_PREP_FULL0, (j - 2) >> 1)) return;
-        const int t0 = j * C, len = min(C, p.T - t0);
-        const size_t row0 = ((size_t)b * p.T + t0) * p.H + h;
+        const ChunkInfo ci = cur.ci;
+        const int t0 = ci.jg * C, len = min(C, p.T - t0);
+        const size_t row0 = ((size_t)ci.b * p.T + t0) * p.H + ci.h;
         for (int idx = lane; idx < 2 * len; idx += 32) {
             const size_t row = row0 + (size_t)(idx >> 1) * p.H;
             const size_t off = (size_t)(idx & 1) * 128;
@@ -398,8 +472,7 @@ __device__ __forceinline__ void turns_sincos(uint32_t turns, float *sn, float *c
     __sincosf(f * 6.283185307f, sn, cs);
 }
 
-__device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int b, int h, int n_chunks,
-                                         int pt)
+__device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int n_chunks, int pt)
 {
     long long *timing = p.timing;
     const int jp = pt & 31, tq = pt >> 5;   // channel pair (channels 2jp, 2jp+1), token octet (8 tokens)
@@ -418,7 +491,7 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
             __nv_bfloat16 *stage =
                 reinterpret_cast<__nv_bfloat16 *>(smem + (half ? OFF_AQ + (jd & 1) * 2 * kTile : OFF_OST));
             const float sgn = half ? -1.f : 1.f;   // o = conj(rho)
-#pragma unroll
+#pragma unroll 1
             for (int hc = 0; hc < 2; ++hc) {
                 uint32_t r[32];
                 tmem_ld<32>(tlane + TM_ACC + 64 + 128 * half + 32 * hc, r);
@@ -433,91 +506,95 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
         warp_arrive(&mi.bars[B_O_STAGED]);
     };
     SFDA_TDECL(pt == 0);
+    ChunkCursor cur(p);
     for (int j = 0; j < n_chunks + 2; ++j) {
         if (role_sync_or(2, kPrepThreads, dead || mi.abort)) break;
-        if (j >= n_chunks) {                     // only the outputs of the last two chunks are left
-            if (j >= 2) drain_outputs(j - 2);
-            continue;
-        }
+        const bool live = j < n_chunks;          // after the last chunk only the outputs of two chunks are left
         const int s = j & 1, ring = j & 3;
-        const int t0 = j * C, len = min(C, p.T - t0);
-        const size_t row0 = ((size_t)b * p.T + t0) * p.H + h;   // token t of this head: row0 + t * H
-        const int nt = min(8, max(0, len - tq * 8));             // real tokens in this thread's octet
-        SFDA_T(35);
-
-        // all loads of this thread for the chunk, issued together
         float2 al[8], th[8];
         uint2 kw[8], qw[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const size_t row = row0 + (size_t)(tq * 8 + i) * p.H;
-            al[i] = make_float2(1.f, 1.f);
-            th[i] = make_float2(0.f, 0.f);
-            kw[i] = make_uint2(0u, 0u);
-            qw[i] = make_uint2(0u, 0u);
-            if (i < nt) {
-                al[i] = __ldg(reinterpret_cast<const float2 *>(p.alpha + row * M) + jp);
-                th[i] = __ldg(reinterpret_cast<const float2 *>(p.theta + row * M) + jp);
-                kw[i] = __ldg(reinterpret_cast<const uint2 *>(p.k + row * DK) + jp);
-                qw[i] = __ldg(reinterpret_cast<const uint2 *>(p.q + row * DK) + jp);
-            }
-        }
-        SFDA_T(36);
-        if (pt < C) mi.beta[ring][pt] = pt < len ? __ldg(p.beta + row0 + (size_t)pt * p.H) : 0.f;
-        SFDA_T(37);
-        // pass 1: prefix products of alpha (a_t: fp32 products of at most 64 factors, relative error far below
-        // bf16's) and prefix sums of the integer phase over this thread's 8 tokens
         float lg0[8], lg1[8];
         uint32_t tu0[8], tu1[8];
-        {
-            float a0 = 1.f, a1 = 1.f;
-            uint32_t u0 = 0u, u1 = 0u;
+        float base0 = 1.f, base1 = 1.f;
+        uint32_t tb0 = 0u, tb1 = 0u;
+        if (live) {
+            const ChunkInfo ci = cur.ci;
+            cur.next(p);
+            const int t0 = ci.jg * C, len = min(C, p.T - t0);
+            const size_t row0 = ((size_t)ci.b * p.T + t0) * p.H + ci.h;   // token t of this head: row0 + t * H
+            const int nt = min(8, max(0, len - tq * 8));             // real tokens in this thread's octet
+            SFDA_T(35);
+
+            // all loads of this thread for the chunk, issued together
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                a0 *= fmaxf(al[i].x, 9.0e-14f);           // floor e^-30, as in log_decay
-                a1 *= fmaxf(al[i].y, 9.0e-14f);
-                u0 += phase_to_turns(th[i].x);
-                u1 += phase_to_turns(th[i].y);
-                lg0[i] = a0; lg1[i] = a1; tu0[i] = u0; tu1[i] = u1;
+                const size_t row = row0 + (size_t)(tq * 8 + i) * p.H;
+                al[i] = make_float2(1.f, 1.f);
+                th[i] = make_float2(0.f, 0.f);
+                kw[i] = make_uint2(0u, 0u);
+                qw[i] = make_uint2(0u, 0u);
+                if (i < nt) {
+                    al[i] = __ldg(reinterpret_cast<const float2 *>(p.alpha + row * M) + jp);
+                    th[i] = __ldg(reinterpret_cast<const float2 *>(p.theta + row * M) + jp);
+                    kw[i] = __ldg(reinterpret_cast<const uint2 *>(p.k + row * DK) + jp);
+                    qw[i] = __ldg(reinterpret_cast<const uint2 *>(p.q + row * DK) + jp);
+                }
             }
-            mi.part_lg[tq][2 * jp] = a0;
-            mi.part_lg[tq][2 * jp + 1] = a1;
-            mi.part_turns[tq][2 * jp] = u0;
-            mi.part_turns[tq][2 * jp + 1] = u1;
-        }
-        SFDA_T(30);
-        role_sync(2, kPrepThreads);
-        float base0 = 1.f, base1 = 1.f, tot0 = 1.f, tot1 = 1.f;
-        uint32_t tb0 = 0u, tb1 = 0u, tt0 = 0u, tt1 = 0u;
+            SFDA_T(36);
+            if (pt < C) mi.beta[ring][pt] = pt < len ? __ldg(p.beta + row0 + (size_t)pt * p.H) : 0.f;
+            SFDA_T(37);
+            // pass 1: prefix products of alpha (a_t: fp32 products of at most 64 factors, relative error far
+            // below bf16's) and prefix sums of the integer phase over this thread's 8 tokens
+            {
+                float a0 = 1.f, a1 = 1.f;
+                uint32_t u0 = 0u, u1 = 0u;
 #pragma unroll
-        for (int gq = 0; gq < 8; ++gq) {
-            const float2 pl = *reinterpret_cast<const float2 *>(&mi.part_lg[gq][2 * jp]);
-            const uint2 pu = *reinterpret_cast<const uint2 *>(&mi.part_turns[gq][2 * jp]);
-            if (gq < tq) { base0 *= pl.x; base1 *= pl.y; tb0 += pu.x; tb1 += pu.y; }
-            tot0 *= pl.x; tot1 *= pl.y; tt0 += pu.x; tt1 += pu.y;
-        }
-        if (tq == 0) {                    // chunk totals: a_C e^{i phi_C}, applied by the next state pass
-            float cs, sn;
-            const float a0 = tot0, a1 = tot1;
-            turns_sincos(tt0, &sn, &cs);
-            mi.close_re[ring][2 * jp] = a0 * cs;
-            mi.close_im[ring][2 * jp] = a0 * sn;
-            turns_sincos(tt1, &sn, &cs);
-            mi.close_re[ring][2 * jp + 1] = a1 * cs;
-            mi.close_im[ring][2 * jp + 1] = a1 * sn;
-        }
-        SFDA_T(31);
+                for (int i = 0; i < 8; ++i) {
+                    a0 *= fmaxf(al[i].x, 9.0e-14f);           // floor e^-30, as in log_decay
+                    a1 *= fmaxf(al[i].y, 9.0e-14f);
+                    u0 += phase_to_turns(th[i].x);
+                    u1 += phase_to_turns(th[i].y);
+                    lg0[i] = a0; lg1[i] = a1; tu0[i] = u0; tu1[i] = u1;
+                }
+                mi.part_lg[tq][2 * jp] = a0;
+                mi.part_lg[tq][2 * jp + 1] = a1;
+                mi.part_turns[tq][2 * jp] = u0;
+                mi.part_turns[tq][2 * jp + 1] = u1;
+            }
+            SFDA_T(30);
+            role_sync(2, kPrepThreads);
+            float tot0 = 1.f, tot1 = 1.f;
+            uint32_t tt0 = 0u, tt1 = 0u;
+#pragma unroll
+            for (int gq = 0; gq < 8; ++gq) {
+                const float2 pl = *reinterpret_cast<const float2 *>(&mi.part_lg[gq][2 * jp]);
+                const uint2 pu = *reinterpret_cast<const uint2 *>(&mi.part_turns[gq][2 * jp]);
+                if (gq < tq) { base0 *= pl.x; base1 *= pl.y; tb0 += pu.x; tb1 += pu.y; }
+                tot0 *= pl.x; tot1 *= pl.y; tt0 += pu.x; tt1 += pu.y;
+            }
+            if (tq == 0) {                    // chunk totals: a_C e^{i phi_C}, applied by the next state pass
+                float cs, sn;
+                turns_sincos(tt0, &sn, &cs);
+                mi.close_re[ring][2 * jp] = tot0 * cs;
+                mi.close_im[ring][2 * jp] = tot0 * sn;
+                turns_sincos(tt1, &sn, &cs);
+                mi.close_re[ring][2 * jp + 1] = tot1 * cs;
+                mi.close_im[ring][2 * jp + 1] = tot1 * sn;
+            }
+            SFDA_T(31);
 
-        // the slot's tiles must have been consumed: W/Qt by rho_1 of chunk j-2, Kc by its state update
-        if (j >= 2) {
-            if (!dead && !wait_k(mi, s ? B_WQ_FREE1 : B_WQ_FREE0, (j >> 1) - 1)) dead = true;
-            if (!dead && !wait_k(mi, s ? B_KC_FREE1 : B_KC_FREE0, (j >> 1) - 1)) dead = true;
+            // the slot's tiles must have been consumed: W/Qt by rho_1 of chunk j-2, Kc by its state update
+            if (j >= 2) {
+                if (!dead && !wait_k(mi, s ? B_WQ_FREE1 : B_WQ_FREE0, (j >> 1) - 1)) dead = true;
+                if (!dead && !wait_k(mi, s ? B_KC_FREE1 : B_KC_FREE0, (j >> 1) - 1)) dead = true;
+            }
+            SFDA_T(32);
         }
-        SFDA_T(32);
         // the state update of chunk j-2 has just finished (it freed Kc above): read out that chunk's outputs,
         // so that rho is free when the next chunk's first product is issued
         if (j >= 2) drain_outputs(j - 2);
         SFDA_T(34);
+        if (!live) continue;
 
         // pass 2: rotated / decayed operands
         uint8_t *wq_re = smem + OFF_WQ + s * 4 * kTile, *wq_im = wq_re + 2 * kTile;
@@ -573,13 +650,13 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
         // so the warps that hold them wait for that store first.
         if (row >= 64 && j >= 2 && !dead && !wait_k(mi, s ? B_STORE_DONE1 : B_STORE_DONE0, (j >> 1) - 1)) dead = true;
         // ---- drain the two Gram halves
-#pragma unroll
+#pragma unroll 1
         for (int im = 0; im < 2; ++im) {
             SFDA_T(20 + 2 * im);
             if (!dead && !wait_k(mi, B_GRAM_FULL, 2 * j + im)) dead = true;
             tc_fence_after();
             SFDA_T(21 + 2 * im);
-#pragma unroll
+#pragma unroll 1
             for (int hc = 0; hc < 2; ++hc) {      // 32 columns at a time keeps the register footprint down
                 uint32_t r[32];
                 tmem_ld<32>(tlane + TM_GRAM + 32 * hc, r);
@@ -740,8 +817,7 @@ __device__ __forceinline__ bool wait_k_warp(Misc &mi, int bar, int k)
     return __all_sync(0xffffffffu, wait_k(mi, bar, k) ? 1 : 0) != 0;
 }
 
-__device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int bh, int n_chunks,
-                                          int ct)
+__device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int n_chunks, int ct)
 {
     long long *timing = p.timing;
     const int lane = ct & 31, warp = ct >> 5;
@@ -750,16 +826,18 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
     const int j0 = half * 32;                  // this warp's complex rows in the state pass
     const uint32_t tlane = tmem + ((uint32_t)(quad * 32) << 16);
 
-    // One 16-row piece of the state pass: rows j0 + 16 pc .. + 15 (Re and Im).
-    auto state_piece = [&](int pc, int ring, bool first) {
+    // One 16-row piece of the state pass: rows j0 + 16 pc .. + 15 (Re and Im).  Inside a unit the chunk-start
+    // state is the accumulated state of the previous chunk times a_C e^{i phi_C}; at the first chunk of a unit it
+    // comes from global memory (`src`, NULL = zero state).
+    auto state_piece = [&](int pc, int ring, bool first, const float *src) {
         uint32_t sre[16], sim[16], pk[8];
         const int jb = j0 + 16 * pc;
         if (first) {
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
                 const int jj = jb + i;
-                sre[i] = p.S0 ? __float_as_uint(p.S0[((size_t)bh * DK + 2 * jj) * DV + c]) : 0u;
-                sim[i] = p.S0 ? __float_as_uint(p.S0[((size_t)bh * DK + 2 * jj + 1) * DV + c]) : 0u;
+                sre[i] = src ? __float_as_uint(__ldcg(src + (size_t)(2 * jj) * DV + c)) : 0u;
+                sim[i] = src ? __float_as_uint(__ldcg(src + (size_t)(2 * jj + 1) * DV + c)) : 0u;
             }
         } else {
             tmem_ld<16>(tlane + TM_S32 + jb, sre);
@@ -782,34 +860,85 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
         tmem_st<16>(tlane + TM_S32 + jb, sre);
         tmem_st<16>(tlane + TM_S32 + 64 + jb, sim);
     };
-    // bf16 A operand from 64 fp32 accumulator columns of this warp's half; `sub_v`: R = V - D1 (Re half only).
-    auto convert_acc = [&](bool sub_v, bool negate, int gate_bar, int gate_k) -> bool {
-        uint32_t pk[32];
+    // The unit that ended with stream chunk `jl` is finished: its final state e^{i phi_C} a_C S goes to S_T (last
+    // time slice) or to the hand-off buffer, where the CTA that runs the next slice is told about it.
+    auto write_out_state = [&](int jl, const ChunkInfo &pi) {
+        const int ring = jl & 3;
+        float *dst = pi.q == p.Q - 1 ? p.S_T : p.handoff;
+        if (dst) {
+            dst += (size_t)pi.bh * DK * DV;
 #pragma unroll
-        for (int hc = 0; hc < 2; ++hc) {
-            uint32_t r[32];
-            tmem_ld<32>(tlane + TM_ACC + 128 * half + 32 * hc, r);
-            tc_wait_ld();
-            if (sub_v) {
-                const __nv_bfloat16 *sv = reinterpret_cast<const __nv_bfloat16 *>(smem + OFF_V);
+            for (int pc = 0; pc < 2; ++pc) {
+                uint32_t sre[16], sim[16];
+                const int jb = j0 + 16 * pc;
+                tmem_ld<16>(tlane + TM_S32 + jb, sre);
+                tmem_ld<16>(tlane + TM_S32 + 64 + jb, sim);
+                tc_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    pk[16 * hc + i] = pack_bf16(__bfloat162float(sv[(32 * hc + 2 * i) * DV + c]) - __uint_as_float(r[2 * i]),
-                                                __bfloat162float(sv[(32 * hc + 2 * i + 1) * DV + c]) - __uint_as_float(r[2 * i + 1]));
-            } else {
-                const float sgn = negate ? -1.f : 1.f;
-#pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    pk[16 * hc + i] = pack_bf16(sgn * __uint_as_float(r[2 * i]), sgn * __uint_as_float(r[2 * i + 1]));
+                for (int i = 0; i < 16; ++i) {
+                    const int jj = jb + i;
+                    const float cs = mi.close_re[ring][jj], sn = mi.close_im[ring][jj];
+                    const float xr = __uint_as_float(sre[i]), xi = __uint_as_float(sim[i]);
+                    __stcg(dst + (size_t)(2 * jj) * DV + c, cs * xr - sn * xi);
+                    __stcg(dst + (size_t)(2 * jj + 1) * DV + c, cs * xi + sn * xr);
+                }
             }
         }
-        if (gate_bar >= 0 && !wait_k_warp(mi, gate_bar, gate_k)) return false;
-        tmem_st<32>(tlane + TM_X16 + 32 * half, pk);
+        if (pi.q < p.Q - 1) {              // one count per warp: slice q + 1 may start once all eight have arrived
+            __threadfence();
+            __syncwarp();
+            if (lane == 0) atomicAdd(p.flags + pi.bh, 1u);
+        }
+    };
+    // Wait until the boundary state of this sequence's previous time slice has been written (eight warp counts
+    // per slice).  Bounded like every other wait; warp-uniform result.
+    auto wait_handoff = [&](const ChunkInfo &ci) -> bool {
+        int ok = 1;
+        if (lane == 0) {
+            const uint32_t want = 8u * (uint32_t)ci.q;
+            const unsigned long long t0 = now_ticks();
+            ok = 0;
+            for (uint32_t it = 0;; ++it) {
+                uint32_t seen;
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(p.flags + ci.bh) : "memory");
+                if (seen >= want) { ok = 1; break; }
+                __nanosleep(200);
+                if ((it & 63u) == 63u && (mi.abort || now_ticks() - t0 > kWaitLimitTicks)) break;
+            }
+            if (!ok) mi.abort = 1;
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        __threadfence();
+        return ok != 0;
+    };
+    // bf16 A operand from 64 fp32 accumulator columns of this warp's half, 32 columns at a time.
+    // mode 1: R = V - D1 (Re half); mode 2: negated (Im half of R = -D1); mode 0: as is (E).
+    auto convert_acc = [&](int mode) {
+#pragma unroll 1
+        for (int hc = 0; hc < 2; ++hc) {
+            uint32_t r[32], pk[16];
+            tmem_ld<32>(tlane + TM_ACC + 128 * half + 32 * hc, r);
+            tc_wait_ld();
+            if (mode == 1) {
+                const __nv_bfloat16 *sv = reinterpret_cast<const __nv_bfloat16 *>(smem + OFF_V) + (32 * hc) * DV + c;
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    pk[i] = pack_bf16(__bfloat162float(sv[(2 * i) * DV]) - __uint_as_float(r[2 * i]),
+                                      __bfloat162float(sv[(2 * i + 1) * DV]) - __uint_as_float(r[2 * i + 1]));
+            } else {
+                const float sgn = mode == 2 ? -1.f : 1.f;
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    pk[i] = pack_bf16(sgn * __uint_as_float(r[2 * i]), sgn * __uint_as_float(r[2 * i + 1]));
+            }
+            tmem_st<16>(tlane + TM_X16 + 32 * half + 16 * hc, pk);
+        }
         tc_wait_st();
-        return true;
     };
 
     SFDA_TDECL(ct == 0);
+    ChunkCursor cur(p);
+    ChunkInfo prev_ci = cur.ci;
     for (int j = 0; j < n_chunks; ++j) {
         // ---- state pass: S_0 of this chunk = e^{i phi_C} a_C (accumulated state of the previous chunk)
         if (j > 0) {
@@ -817,55 +946,52 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
             tc_fence_after();
         }
         SFDA_T(10);
-        state_piece(0, (j - 1) & 3, j == 0);
-        state_piece(1, (j - 1) & 3, j == 0);
+        const ChunkInfo ci = cur.ci;
+        const float *src = nullptr;
+        if (ci.first) {
+            if (j > 0) write_out_state(j - 1, prev_ci);
+#ifdef SFDA_WS_TIMING
+            if (j > 0 && ct == 0 && p.timing) p.timing[512 + blockIdx.x] = (long long)now_ns();
+#endif
+            if (ci.q == 0) {
+                src = p.S0 ? p.S0 + (size_t)ci.bh * DK * DV : nullptr;
+            } else {
+                if (!wait_handoff(ci)) return;
+                src = p.handoff + (size_t)ci.bh * DK * DV;
+            }
+        }
+#pragma unroll 1
+        for (int pc = 0; pc < 2; ++pc) state_piece(pc, (j - 1) & 3, ci.first, src);
+        prev_ci = ci;
+        cur.next(p);
         tc_wait_st();
         tc_fence_before();
         warp_arrive(&mi.bars[B_S16_READY]);
         SFDA_T(11);
 
-        // ---- R = V - D1 -> bf16 A operand (D1 and rho_1, which read S_0 from the same columns, are both done)
-        if (!wait_k_warp(mi, B_D1_DONE, j)) return;
-        if (!wait_k_warp(mi, B_V_FULL, j)) return;
-        tc_fence_after();
-        SFDA_T(13);
-        if (!convert_acc(half == 0, half == 1, -1, 0)) return;
-        tc_fence_before();
-        warp_arrive(&mi.bars[B_R16_READY]);
-        SFDA_T(14);
-
-        // ---- E -> bf16 A operand
-        if (!wait_k_warp(mi, B_E_DONE, j)) return;
-        tc_fence_after();
-        SFDA_T(15);
-        if (!convert_acc(false, false, -1, 0)) return;
-        tc_fence_before();
-        warp_arrive(&mi.bars[B_E16_READY]);
-        SFDA_T(16);
-    }
-
-    // ---- last chunk: outputs and the final state
-    if (!wait_k_warp(mi, B_UPD_DONE, n_chunks - 1)) return;
-    tc_fence_after();
-    if (p.S_T) {
-        const int ring = (n_chunks - 1) & 3;
-#pragma unroll
-        for (int pc = 0; pc < 2; ++pc) {
-            uint32_t sre[16], sim[16];
-            const int jb = j0 + 16 * pc;
-            tmem_ld<16>(tlane + TM_S32 + jb, sre);
-            tmem_ld<16>(tlane + TM_S32 + 64 + jb, sim);
-            tc_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int jj = jb + i;
-                const float cs = mi.close_re[ring][jj], sn = mi.close_im[ring][jj];
-                const float xr = __uint_as_float(sre[i]), xi = __uint_as_float(sim[i]);
-                p.S_T[((size_t)bh * DK + 2 * jj) * DV + c] = cs * xr - sn * xi;
-                p.S_T[((size_t)bh * DK + 2 * jj + 1) * DV + c] = cs * xi + sn * xr;
+        // ---- R = V - D1, then E, -> bf16 A operand (D1 and rho_1, which read S_0 from the same columns, are both
+        // done when D1 is)
+#pragma unroll 1
+        for (int ph = 0; ph < 2; ++ph) {
+            if (ph == 0) {
+                if (!wait_k_warp(mi, B_D1_DONE, j)) return;
+                if (!wait_k_warp(mi, B_V_FULL, j)) return;
+            } else {
+                if (!wait_k_warp(mi, B_E_DONE, j)) return;
             }
+            tc_fence_after();
+            SFDA_T(13 + 2 * ph);
+            convert_acc(ph == 0 ? 1 + half : 0);
+            tc_fence_before();
+            warp_arrive(&mi.bars[ph == 0 ? B_R16_READY : B_E16_READY]);
+            SFDA_T(14 + 2 * ph);
         }
     }
+
+    // ---- the last unit's final state
+    if (!wait_k_warp(mi, B_UPD_DONE, n_chunks - 1)) return;
+    tc_fence_after();
+    write_out_state(n_chunks - 1, prev_ci);
 }
 
 // ---- the kernel ---------------------------------------------------------------------------------------
@@ -878,9 +1004,12 @@ sfda_forward_ws_kernel(const __grid_constant__ CUtensorMap tm_v, const __grid_co
     Misc &mi = *reinterpret_cast<Misc *>(smem + OFF_MISC);
 
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int bh = blockIdx.x, h = bh % p.H, b = bh / p.H;
-    const int n_chunks = (p.T + C - 1) / C;
+    // this CTA's stream: units blockIdx, blockIdx + gridDim, ... of U chunks each
+    const int n_chunks = ((p.n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * p.U;
 
+#ifdef SFDA_WS_TIMING
+    if (tid == 0 && p.timing) { p.timing[64 + 2 * blockIdx.x] = (long long)now_ns(); if (blockIdx.x == 0) p.timing[400] = clock64(); unsigned sm; asm volatile("mov.u32 %0, %smid;" : "=r"(sm)); p.timing[700 + blockIdx.x] = sm; }
+#endif
     if (tid == 0) {
         auto init = [&](int bar, uint32_t count) { mbar_init(&mi.bars[bar], count); };
         init(B_PREP_FULL0, kPrepWarps); init(B_PREP_FULL1, kPrepWarps);
@@ -905,30 +1034,37 @@ sfda_forward_ws_kernel(const __grid_constant__ CUtensorMap tm_v, const __grid_co
 
     if (warp < kChainWarps) {
         regs_inc<kRegsWork>();
-        run_chain(smem, mi, tmem, p, bh, n_chunks, tid);
+        run_chain(smem, mi, tmem, p, n_chunks, tid);
     } else if (warp < kChainWarps + kSolveWarps) {
         regs_inc<kRegsWork>();
         run_solve(smem, mi, tmem, p, n_chunks, tid - kChainThreads);
     } else if (warp < kChainWarps + kSolveWarps + kPrepWarps) {
         regs_inc<kRegsWork>();
-        run_prep(smem, mi, tmem, p, b, h, n_chunks, tid - kChainThreads - kSolveThreads);
+        run_prep(smem, mi, tmem, p, n_chunks, tid - kChainThreads - kSolveThreads);
     } else {
         regs_dec<kRegsCtrl>();
         const int cw = warp - (kChainWarps + kSolveWarps + kPrepWarps);
         if (cw == 3)
-            run_prefetch(mi, p, b, h, n_chunks, tid & 31);
+            run_prefetch(mi, p, n_chunks, tid & 31);
         else if ((tid & 31) == 0)
-            run_ctrl(cw, smem, mi, tmem, &tm_v, &tm_o, &tm_oim, p, b, h, n_chunks);
+            run_ctrl(cw, smem, mi, tmem, &tm_v, &tm_o, &tm_oim, p, n_chunks);
     }
 
     tc_fence_before();
     __syncthreads();
+#ifdef SFDA_WS_TIMING
+    if (tid == 0 && p.timing) { p.timing[64 + 2 * blockIdx.x + 1] = (long long)now_ns(); if (blockIdx.x == 0) p.timing[401] = clock64(); }
+#endif
     if (tid == 0 && mi.abort) atomicExch(p.status, 1u);
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem));
 }
 
 // ---- host side ----------------------------------------------------------------------------------------
 long long *g_ws_timing = nullptr;   // set by development probes built with -DSFDA_WS_TIMING
+int g_ws_last_slices = 0;           // time slices chosen by the last launch (read by development probes)
+#ifdef SFDA_WS_TIMING
+int g_ws_grid_cap = 0, g_ws_force_q = 0;   // development probes only
+#endif
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -1000,7 +1136,7 @@ cudaError_t launch_forward_ws_static(const ForwardArgs &a, cudaStream_t stream, 
     const cudaError_t e = static_scratch_address(&scratch);
     if (e != cudaSuccess) return e;
     // the block keeps whatever the last call left in it; the launcher clears the status word on the stream
-    return launch_forward_ws(a, static_cast<uint32_t *>(scratch), stream, launches);
+    return launch_forward_ws(a, scratch, kStaticScratchBytes, stream, launches);
 }
 
 cudaError_t read_static_status(cudaStream_t stream, uint32_t *word)
@@ -1015,7 +1151,15 @@ cudaError_t read_static_status(cudaStream_t stream, uint32_t *word)
 
 bool forward_ws_supported(const ForwardArgs &a) { return a.dtype == 1 && a.d_k == DK && a.d_v == DV && a.chunk == C; }
 
-cudaError_t launch_forward_ws(const ForwardArgs &a, uint32_t *status, cudaStream_t stream, int *launches)
+// Scratch layout: [0, 256) status word; then, when the block is large enough for time slicing,
+// [256, 256 + round256(4 BH)) slice counters and BH boundary states of d_k x d_v floats.
+size_t forward_ws_scratch_bytes(int B, int H)
+{
+    const size_t bh = (size_t)B * H;
+    return kWsMinScratchBytes + ((bh * 4 + 255) & ~(size_t)255) + bh * DK * DV * 4;
+}
+
+cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratch_bytes, cudaStream_t stream, int *launches)
 {
     CUtensorMap tv, to, toi;
     if (!make_map(&tv, a.v, a.B, a.T, a.H) || !make_map(&to, a.o, a.B, a.T, a.H) ||
@@ -1023,7 +1167,32 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, uint32_t *status, cudaStream
         return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(sfda_forward_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    e = cudaMemsetAsync(status, 0, sizeof(uint32_t), stream);
+    int dev = 0, n_sm = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+
+    // Time slices per sequence: one CTA per SM works through ceil(units / SMs) units of NC / Q chunks.  More
+    // slices even out the last round, but every unit boundary costs about two chunk periods (the state goes
+    // through global memory and the next slice waits for it), so slicing is chosen only when it removes at least
+    // 15 % of the rounds' chunk count (for instance a few more sequences than SMs, or few very long sequences).
+    const int BH = a.B * a.H, NC = (a.T + C - 1) / C;
+    int Q = 1;
+    if (scratch_bytes >= forward_ws_scratch_bytes(a.B, a.H)) {
+        double best = 0.0;
+        for (int q = 1; q <= 8; q *= 2) {
+            if (NC % q != 0 || NC / q < 4) break;
+            const long units = (long)BH * q;
+            const double cost = (double)((units + n_sm - 1) / n_sm) * (NC / q + 2.0);
+            if (q == 1) best = cost;
+            else if (cost < 0.85 * best) { best = cost / 0.85; Q = q; }
+        }
+    }
+#ifdef SFDA_WS_TIMING
+    if (g_ws_force_q) Q = g_ws_force_q;
+    if (g_ws_grid_cap && g_ws_grid_cap < n_sm) n_sm = g_ws_grid_cap;
+#endif
+    const size_t header = kWsMinScratchBytes + (Q > 1 ? (((size_t)BH * 4 + 255) & ~(size_t)255) : 0);
+    e = cudaMemsetAsync(scratch, 0, header, stream);
     if (e != cudaSuccess) return e;
     Params p;
     p.timing = g_ws_timing;
@@ -1034,11 +1203,19 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, uint32_t *status, cudaStream
     p.beta = a.beta;
     p.S0 = a.S0;
     p.S_T = a.S_T;
-    p.status = status;
+    p.status = static_cast<uint32_t *>(scratch);
+    p.flags = reinterpret_cast<uint32_t *>(static_cast<char *>(scratch) + kWsMinScratchBytes);
+    p.handoff = reinterpret_cast<float *>(static_cast<char *>(scratch) + header);
     p.T = a.T;
     p.H = a.H;
     p.has_o_im = a.o_im != nullptr;
-    sfda_forward_ws_kernel<<<(unsigned)(a.B * a.H), kThreads, kSmemBytes, stream>>>(tv, to, toi, p);
+    p.BH = BH;
+    p.Q = Q;
+    p.U = NC / Q;
+    p.n_units = BH * Q;
+    g_ws_last_slices = Q;
+    const unsigned grid = (unsigned)(p.n_units < n_sm ? p.n_units : n_sm);
+    sfda_forward_ws_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tv, to, toi, p);
     e = cudaGetLastError();
     if (e == cudaSuccess && launches) ++*launches;
     return e;

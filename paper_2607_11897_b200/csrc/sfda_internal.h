@@ -36,7 +36,12 @@ cudaError_t launch_forward_simt(const ForwardArgs &a, cudaStream_t stream, int *
 // `status` is one device word the kernel sets when a bounded wait runs out; it is cleared on the stream
 // before the launch.
 bool forward_ws_supported(const ForwardArgs &a);
-cudaError_t launch_forward_ws(const ForwardArgs &a, uint32_t *status, cudaStream_t stream, int *launches);
+// `scratch` starts with that word (kWsMinScratchBytes suffice); with forward_ws_scratch_bytes(B, H) bytes the
+// launcher may also cut every sequence into time slices that hand their boundary state over through the scratch.
+constexpr size_t kWsMinScratchBytes = 256;
+size_t forward_ws_scratch_bytes(int B, int H);
+cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratch_bytes, cudaStream_t stream,
+                              int *launches);
 // The same kernel on the library's own statically allocated scratch block (kStaticScratchBytes), and a read of
 // the status word kept there (synchronises the stream).  Neither allocates.
 constexpr size_t kStaticScratchBytes = 256;

@@ -195,6 +195,7 @@ __device__ __forceinline__ void cmma_16x8(float (&cr)[4], float (&ci)[4], const 
                                           int b_row0, int b_col0, int s0, int s1, int lane)
 {
     const int g = lane >> 2, tg = lane & 3;
+#pragma unroll 1
     for (int s = s0; s < s1; ++s) {
         const int ao = (a_row0 + g) * a_ld + a_col0 + 8 * s + tg;
         uint32_t ar[4], ai[4], nai[4], br[2], bi[2];

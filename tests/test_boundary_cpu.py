@@ -47,7 +47,8 @@ def test_status_strings(lib):
 
 
 def test_workspace_bytes(lib):
-    assert sfda.sfda_workspace_bytes(8, 8192, 32, 128, 128, 64, sfda.SFDA_BF16) == 256
+    # status block + one counter per (batch, head) + one boundary state per (batch, head) for the time slices
+    assert sfda.sfda_workspace_bytes(8, 8192, 32, 128, 128, 64, sfda.SFDA_BF16) == 256 + 1024 + 256 * 128 * 128 * 4
     assert sfda.sfda_workspace_bytes(1, 256, 2, 64, 64, 16, sfda.SFDA_F32) == 0
     assert sfda.sfda_workspace_bytes(1, 256, 2, 128, 128, 64, sfda.SFDA_F32) == 0
     assert sfda.sfda_workspace_bytes(0, 256, 2, 128, 128, 64, sfda.SFDA_BF16) == 0

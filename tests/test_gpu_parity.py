@@ -153,6 +153,26 @@ def test_forward_tensor_core_path(T, H, s0, alpha):
     print(errs)
 
 
+def test_forward_tensor_core_time_slices():
+    """More sequences than SMs: the launcher cuts every sequence into time slices that hand their boundary
+    state over through the workspace; with only the status block as workspace it does not.  Same results."""
+    cfg = workloads.CONFIGS[1].scaled(name="slices", B=5, T=512, H=40, s0_std=0.05, seed=91)
+    inp = workloads.forward_inputs(cfg)
+    pairs = [(0, 0), (4, 39), (2, 17), (3, 5), (1, 30), (4, 0)]
+    check_forward(cfg, inp, pairs, TOL["bf16"])
+    d = {k: (None if v is None else to_dev(v, cfg, k)) for k, v in inp.items()}
+    outs = []
+    for nbytes in (sfda.sfda_workspace_bytes(cfg.B, cfg.T, cfg.H, 128, 128, 64, 1), 256):
+        o = torch.empty(cfg.B, cfg.T, cfg.H, cfg.d_v, device=DEV, dtype=torch.bfloat16)
+        o_im, S_T = torch.empty_like(o), torch.empty(cfg.B, cfg.H, 128, 128, device=DEV)
+        ws = torch.empty(nbytes, device=DEV, dtype=torch.uint8)
+        sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im, S_T, 64, ws)
+        assert sfda.sfda_workspace_status(ws) == 0
+        outs.append((o.float().cpu().numpy(), o_im.float().cpu().numpy(), S_T.cpu().numpy()))
+    for x, y in zip(*outs):
+        assert np.array_equal(x, y)          # slicing only moves the fp32 state through memory: bit-identical
+
+
 def test_forward_tensor_core_matches_cuda_core_path():
     cfg = workloads.CONFIGS[1].scaled(name="tc2", B=1, T=512, H=4, s0_std=0.1, seed=77)
     inp = workloads.forward_inputs(cfg)
