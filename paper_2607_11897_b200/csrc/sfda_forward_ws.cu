@@ -237,14 +237,15 @@ __device__ __forceinline__ bool test_k(Misc &mi, int bar, int k)
                  : "memory");
     return ok != 0;
 }
-// Wait for completion number k; gives up after kWaitLimitTicks or when another role has raised the abort flag.
-// Returns false in that case, after raising the flag itself.  try_wait parks the thread in hardware for up to
-// the hinted time, so waiting warps do not compete with working ones for issue slots.
+// Wait for completion number k of a barrier; gives up after about a second (2^31 ticks of the SM clock) and
+// raises the abort flag.  try_wait parks the thread in hardware for up to the hinted time, so waiting warps do
+// not compete with working ones for issue slots.  Kept to a handful of instructions: it is inlined at every
+// wait, and the kernel's per-chunk code has to stay inside the SM's instruction cache.
 __device__ __forceinline__ bool wait_k(Misc &mi, int bar, int k)
 {
     const uint32_t addr = smem_u32(&mi.bars[bar]), parity = (uint32_t)k & 1u;
-    unsigned long long t0 = 0;
-    for (uint32_t it = 0;; ++it) {
+    const uint32_t t0 = (uint32_t)clock();
+    do {
         uint32_t ok;
         asm volatile(
             "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}\n"
@@ -252,38 +253,71 @@ __device__ __forceinline__ bool wait_k(Misc &mi, int bar, int k)
             : "r"(addr), "r"(parity), "r"(20000u)
             : "memory");
         if (ok) return true;
-        if (mi.abort) return false;
-        const unsigned long long t = now_ticks();
-        if (it == 0) t0 = t;
-        else if (t - t0 > kWaitLimitTicks) break;
-    }
+    } while ((uint32_t)clock() - t0 < 0x80000000u);
     mi.abort = 1;
     return false;
 }
 
-// ---- CTRL: one thread issues all tensor-core and TMA work ------------------------------------------------
-// Four K = 16 instructions over one 64-element swizzle span; `b` is the low half of the operand's descriptor,
-// `hi` the (common) high half.  `b_step` is the descriptor advance per K = 16: 2 (32 bytes) for a K-major
-// operand, 128 (2048 bytes = 16 rows) for an MN-major one.
-__device__ __forceinline__ void mma4_ts(uint32_t d, uint32_t a, uint32_t b, uint32_t hi, uint32_t id, uint32_t acc,
-                                        uint32_t b_step = 2)
+// ---- CTRL: three warps issue all tensor-core and TMA work ------------------------------------------------
+// A CTRL warp runs its loop with all 32 lanes converged and elects one lane only around the instructions that
+// a single thread must issue.  (Issued from inside a one-thread branch, every tensor-core instruction costs some
+// thirty instructions that move its operands into uniform registers; from converged code it costs about five.)
+__device__ __forceinline__ bool elect_one()
 {
-    mma_ts2(d, a, b, hi, id, acc);
-    mma_ts2(d, a + 8, b + b_step, hi, id, 1u);
-    mma_ts2(d, a + 16, b + 2 * b_step, hi, id, 1u);
-    mma_ts2(d, a + 24, b + 3 * b_step, hi, id, 1u);
+    uint32_t pred;
+    asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\nselp.u32 %0, 1, 0, p;\n}\n" : "=r"(pred));
+    return pred != 0;
 }
-__device__ __forceinline__ void mma4_ss(uint32_t d, uint32_t a, uint32_t b, uint32_t hi, uint32_t id, uint32_t acc)
+// wait_k with a warp-uniform outcome, so that a warp leaves (or stays) as a whole
+__device__ __forceinline__ bool wait_k_warp(Misc &mi, int bar, int k)
 {
-    mma_ss2(d, a, hi, b, hi, id, acc);
-    mma_ss2(d, a + 2, hi, b + 2, hi, id, 1u);
-    mma_ss2(d, a + 4, hi, b + 4, hi, id, 1u);
-    mma_ss2(d, a + 6, hi, b + 6, hi, id, 1u);
+    return __all_sync(0xffffffffu, wait_k(mi, bar, k) ? 1 : 0) != 0;
+}
+__device__ __forceinline__ bool test_k_warp(Misc &mi, int bar, int k)
+{
+    return __all_sync(0xffffffffu, test_k(mi, bar, k) ? 1 : 0) != 0;
 }
 
-// The issuing work is split over three threads (one per warp, so they sit on different schedulers):
-//   role 0  the products on the state's dependency chain: D1, E, the state update
-//   role 1  the output products rho_1 and rho += Aq E, and the output stores
+// One complex product as four real ones (g = 0..3), each of four K = 16 instructions:
+//   Re += x_re b_re,  Re -+= x_im b_im,  Im += x_im b_re,  Im +-= x_re b_im
+// A (x) is the bf16 operand in tensor memory (or, for the Gram, tiles in shared memory); `a_im`, `b_im`, `d_im`
+// are the imaginary parts' addresses; `neg_g` is the g whose product is subtracted; `fresh`:
+// the accumulators start from zero.  `b_step`: descriptor advance of B per K = 16 (2 for a K-major tile,
+// 128 for an MN-major one).  The state update uses the same products with conj(E)-side roles swapped, which
+// `swap` selects: Re += x_re b_re, Re -= x_im b_im, Im += x_re b_im, Im += x_im b_re.
+template <bool kTmemA>
+__device__ __forceinline__ void issue_complex(uint32_t d_re, uint32_t d_im, uint32_t a_re, uint32_t a_im,
+                                              uint32_t b_re, uint32_t b_im, uint32_t dhi, uint32_t id, int neg_g,
+                                              bool fresh, bool swap, uint32_t b_step)
+{
+#pragma unroll 1
+    for (int g = 0; g < 4; ++g) {
+        const bool odd = g & 1, mid = g == 1 || g == 2;
+        const uint32_t d = g < 2 ? d_re : d_im;
+        const uint32_t a = (swap ? odd : mid) ? a_im : a_re;
+        const uint32_t b = (swap ? mid : odd) ? b_im : b_re;
+        const uint32_t idg = id | (g == neg_g ? 1u << 14 : 0u);
+        const uint32_t acc0 = (!fresh || odd) ? 1u : 0u;
+        if (elect_one()) {
+            if (kTmemA) {
+                mma_ts2(d, a, b, dhi, idg, acc0);
+                mma_ts2(d, a + 8, b + b_step, dhi, idg, 1u);
+                mma_ts2(d, a + 16, b + 2 * b_step, dhi, idg, 1u);
+                mma_ts2(d, a + 24, b + 3 * b_step, dhi, idg, 1u);
+            } else {
+                mma_ss2(d, a, dhi, b, dhi, idg, acc0);
+                mma_ss2(d, a + 2, dhi, b + 2, dhi, idg, 1u);
+                mma_ss2(d, a + 4, dhi, b + 4, dhi, idg, 1u);
+                mma_ss2(d, a + 6, dhi, b + 6, dhi, idg, 1u);
+            }
+        }
+        __syncwarp();
+    }
+}
+
+// The issuing work is split over three warps (they sit on different schedulers):
+//   role 0  the products on the state's dependency chain: D1 (with rho_1), E, the state update
+//   role 1  the output product rho += Aq E and the output stores
 //   role 2  the Gram products (they run ahead of the chain) and the v loads
 __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint32_t tmem, const CUtensorMap *tm_v,
                                          const CUtensorMap *tm_o, const CUtensorMap *tm_oim, const Params &p,
@@ -292,143 +326,139 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
     long long *timing = p.timing;
     const uint64_t dbase = smem_desc(smem_u32(smem));                     // descriptor of byte offset 0
     const uint32_t dlo = (uint32_t)dbase, dhi = (uint32_t)(dbase >> 32);
-    auto desc = [&](int off) { return dlo + (uint32_t)(off >> 4); };      // low half; offsets are multiples of 16
     unsigned long long *bars = mi.bars;
-    constexpr uint32_t I64 = idesc(64, 0), I64N = idesc(64, 1);           // N = 64, B K-major (negated)
-    constexpr uint32_t I128 = idesc(128, 0), I128N = idesc(128, 1);       // N = 128
-    constexpr uint32_t I64M = idesc(64, 0) | (1u << 16), I64MN = idesc(64, 1) | (1u << 16);   // B MN-major
-    const uint32_t x_re = tmem + TM_X16, x_im = tmem + TM_X16 + 32;
-    const uint32_t acc_re = tmem + TM_ACC, rho_re = tmem + TM_ACC + 64, acc_im = tmem + TM_ACC + 128,
-                   rho_im = tmem + TM_ACC + 192;
+    constexpr uint32_t I64 = idesc(64, 0), I128 = idesc(128, 0), I64M = idesc(64, 0) | (1u << 16);   // M: B MN-major
+    constexpr uint32_t kIm = kTile >> 4;                                  // re -> im tile, in descriptor units
+    const uint32_t x_re = tmem + TM_X16, acc = tmem + TM_ACC;
+    const uint32_t m_re = dlo + (OFF_MB >> 4);
 
     if (role == 0) {
-        SFDA_TDECL(true);
+        SFDA_TDECL((threadIdx.x & 31) == 0);
+#pragma unroll 1
         for (int j = 0; j < n_chunks; ++j) {
             const int s = j & 1, u = j >> 1;
-            const uint32_t w_re = desc(OFF_WQ + s * 4 * kTile), w_im = w_re + (2 * kTile >> 4);
-            const uint32_t k_re = desc(OFF_KC + s * 2 * kTile), k_im = k_re + (kTile >> 4);
-            const uint32_t m_re = desc(OFF_MB), m_im = m_re + (kTile >> 4);
-            // [D1 | rho_1] = [W ; Qt]^* S_0 : N = 128 over the slot's 128-row tiles; rho of the previous chunk
-            // must have been read out
-            if (!wait_k(mi, B_S16_READY, j)) return;
-            if (!wait_k(mi, s ? B_PREP_FULL1 : B_PREP_FULL0, u)) return;
-            if (j > 0 && !wait_k(mi, B_O_STAGED, j - 1)) return;
+            const uint32_t w_re = dlo + ((OFF_WQ + s * 4 * kTile) >> 4), k_re = dlo + ((OFF_KC + s * 2 * kTile) >> 4);
+            // [D1 | rho_1] = [W ; Qt]^* S_0: N = 128 over the slot's 128-row tiles; rho of the previous chunk must
+            // have been read out
+            if (!wait_k_warp(mi, B_S16_READY, j)) return;
+            if (!wait_k_warp(mi, B_PREP_FULL0 + s, u)) return;
+            if (j > 0 && !wait_k_warp(mi, B_O_STAGED, j - 1)) return;
             tc_fence_after();
             SFDA_T(0);
-            mma4_ts(acc_re, x_re, w_re, dhi, I128, 0u);
-            mma4_ts(acc_re, x_im, w_im, dhi, I128, 1u);
-            mma4_ts(acc_im, x_im, w_re, dhi, I128, 0u);
-            mma4_ts(acc_im, x_re, w_im, dhi, I128N, 1u);
-            mma_commit(&bars[B_D1_DONE]);
-            mma_commit(&bars[s ? B_WQ_FREE1 : B_WQ_FREE0]);
+            issue_complex<true>(acc, acc + 128, x_re, x_re + 32, w_re, w_re + 2 * kIm, dhi, I128, 3, true, false, 2);
+            if (elect_one()) {
+                mma_commit(&bars[B_D1_DONE]);
+                mma_commit(&bars[B_WQ_FREE0 + s]);
+            }
             SFDA_T(1);
             // E = M_beta R
-            if (!wait_k(mi, B_R16_READY, j)) return;
+            if (!wait_k_warp(mi, B_R16_READY, j)) return;
             SFDA_T(2);
-            if (!wait_k(mi, B_MB_FULL, j)) return;
+            if (!wait_k_warp(mi, B_MB_FULL, j)) return;
             tc_fence_after();
             SFDA_T(3);
-            mma4_ts(acc_re, x_re, m_re, dhi, I64, 0u);
-            mma4_ts(acc_re, x_im, m_im, dhi, I64N, 1u);
-            mma4_ts(acc_im, x_im, m_re, dhi, I64, 0u);
-            mma4_ts(acc_im, x_re, m_im, dhi, I64, 1u);
-            mma_commit(&bars[B_E_DONE]);
+            issue_complex<true>(acc, acc + 128, x_re, x_re + 32, m_re, m_re + kIm, dhi, I64, 1, true, false, 2);
+            if (elect_one()) mma_commit(&bars[B_E_DONE]);
             SFDA_T(4);
             // S += E^T Kc (Kc as MN-major B: rows = tokens)
-            if (!wait_k(mi, B_E16_READY, j)) return;
+            if (!wait_k_warp(mi, B_E16_READY, j)) return;
             tc_fence_after();
             SFDA_T(5);
-            mma4_ts(tmem + TM_S32, x_re, k_re, dhi, I64M, 1u, 128);
-            mma4_ts(tmem + TM_S32, x_im, k_im, dhi, I64MN, 1u, 128);
-            mma4_ts(tmem + TM_S32 + 64, x_re, k_im, dhi, I64M, 1u, 128);
-            mma4_ts(tmem + TM_S32 + 64, x_im, k_re, dhi, I64M, 1u, 128);
-            mma_commit(&bars[s ? B_KC_FREE1 : B_KC_FREE0]);
-            mma_commit(&bars[B_UPD_DONE]);
+            issue_complex<true>(tmem + TM_S32, tmem + TM_S32 + 64, x_re, x_re + 32, k_re, k_re + kIm, dhi, I64M, 1, false, true, 128);
+            if (elect_one()) {
+                mma_commit(&bars[B_KC_FREE0 + s]);
+                mma_commit(&bars[B_UPD_DONE]);
+            }
             SFDA_T(6);
         }
     } else if (role == 1) {
-        ChunkCursor prev(p);             // chunk j - 1 inside the loop
-        for (int j = 0; j < n_chunks; ++j) {
-            const int s = j & 1, u = j >> 1;
-            const uint32_t a_re = desc(OFF_AQ + s * 2 * kTile), a_im = a_re + (kTile >> 4);
-            // outputs of the previous chunk are staged: store them
+        ChunkCursor prev(p);             // the chunk whose outputs are stored next
+        // iteration j: store the outputs of chunk j - 1 (once staged), then issue rho += Aq E of chunk j
+#pragma unroll 1
+        for (int j = 0; j <= n_chunks; ++j) {
             if (j > 0) {
-                if (!wait_k(mi, B_O_STAGED, j - 1)) return;
+                if (!wait_k_warp(mi, B_O_STAGED, j - 1)) return;
                 const ChunkInfo pc = prev.ci;
                 prev.next(p);
-                tma_store_4d(tm_o, smem + OFF_OST, 0, pc.h, pc.jg * C, pc.b);
-                if (p.has_o_im)
-                    tma_store_4d(tm_oim, smem + OFF_AQ + ((j - 1) & 1) * 2 * kTile, 0, pc.h, pc.jg * C, pc.b);
-                tma_store_commit();
-                tma_store_wait_read();
-                mbar_arrive(&bars[(j - 1) & 1 ? B_STORE_DONE1 : B_STORE_DONE0]);
+                if (elect_one()) {
+                    tma_store_4d(tm_o, smem + OFF_OST, 0, pc.h, pc.jg * C, pc.b);
+                    if (p.has_o_im)
+                        tma_store_4d(tm_oim, smem + OFF_AQ + ((j - 1) & 1) * 2 * kTile, 0, pc.h, pc.jg * C, pc.b);
+                    tma_store_commit();
+                    if (j < n_chunks) {
+                        tma_store_wait_read();
+                        mbar_arrive(&bars[B_STORE_DONE0 + ((j - 1) & 1)]);
+                    } else {
+                        tma_store_wait_all();
+                    }
+                }
+                __syncwarp();
+                if (j == n_chunks) break;
             }
-            // rho += Aq E
-            if (!wait_k(mi, B_E16_READY, j)) return;
-            if (!wait_k(mi, s ? B_AQ_FULL1 : B_AQ_FULL0, u)) return;
+            if (!wait_k_warp(mi, B_E16_READY, j)) return;
+            if (!wait_k_warp(mi, B_AQ_FULL0 + (j & 1), j >> 1)) return;
             tc_fence_after();
-            mma4_ts(rho_re, x_re, a_re, dhi, I64, 1u);
-            mma4_ts(rho_re, x_im, a_im, dhi, I64N, 1u);
-            mma4_ts(rho_im, x_im, a_re, dhi, I64, 1u);
-            mma4_ts(rho_im, x_re, a_im, dhi, I64, 1u);
-            mma_commit(&bars[B_UPD_DONE]);
+            const uint32_t a_re = dlo + ((OFF_AQ + (j & 1) * 2 * kTile) >> 4);
+            issue_complex<true>(acc + 64, acc + 192, x_re, x_re + 32, a_re, a_re + kIm, dhi, I64, 1, false, false, 2);
+            if (elect_one()) mma_commit(&bars[B_UPD_DONE]);
         }
-        if (!wait_k(mi, B_O_STAGED, n_chunks - 1)) return;
-        const ChunkInfo pc = prev.ci;
-        tma_store_4d(tm_o, smem + OFF_OST, 0, pc.h, pc.jg * C, pc.b);
-        if (p.has_o_im)
-            tma_store_4d(tm_oim, smem + OFF_AQ + ((n_chunks - 1) & 1) * 2 * kTile, 0, pc.h, pc.jg * C, pc.b);
-        tma_store_commit();
-        tma_store_wait_all();
     } else {
         // Gram chunk g, half gh, as soon as its operands are written and the Gram columns have been drained;
         // v of chunk jv as soon as v of chunk jv-1 has been consumed (R of that chunk is built).
-        ChunkCursor vcur(p);             // chunk jv - 1 below, advanced before each further load
-        mbar_expect_tx(&bars[B_V_FULL], 16384);
-        tma_load_4d(smem + OFF_V, tm_v, &bars[B_V_FULL], 0, vcur.ci.h, vcur.ci.jg * C, vcur.ci.b);
-        int g = 0, gh = 0, jv = 1;
-        const unsigned long long t0 = now_ticks();
-        for (uint32_t it = 0; g < n_chunks || jv < n_chunks; ++it) {
+        ChunkCursor vcur(p);
+        int g = 0, gh = 0, jv = 0;
+        uint32_t t0 = (uint32_t)clock();
+#pragma unroll 1
+        while (g < n_chunks || jv < n_chunks) {
             bool progress = false;
             if (g < n_chunks) {
-                const bool ready = gh == 0 ? test_k(mi, g & 1 ? B_PREP_FULL1 : B_PREP_FULL0, g >> 1) &&
-                                                 (g == 0 || test_k(mi, B_GRAM_DRAINED, 2 * g - 1))
-                                           : test_k(mi, B_GRAM_DRAINED, 2 * g);
+                const bool ready = gh == 0 ? test_k_warp(mi, B_PREP_FULL0 + (g & 1), g >> 1) &&
+                                                 (g == 0 || test_k_warp(mi, B_GRAM_DRAINED, 2 * g - 1))
+                                           : test_k_warp(mi, B_GRAM_DRAINED, 2 * g);
                 if (ready) {
                     const int s = g & 1;
-                    const uint32_t w_re = desc(OFF_WQ + s * 4 * kTile), w_im = w_re + (2 * kTile >> 4);
-                    const uint32_t k_re = desc(OFF_KC + s * 2 * kTile), k_im = k_re + (kTile >> 4);
-                    const uint32_t d = tmem + TM_GRAM;
+                    const uint32_t w_re = dlo + ((OFF_WQ + s * 4 * kTile) >> 4), k_re = dlo + ((OFF_KC + s * 2 * kTile) >> 4);
+                    const uint32_t k_b = gh ? k_re + kIm : k_re;
                     tc_fence_after();
-                    if (gh == 0) {       // rows = [W; Qt], columns = tokens i
-                        mma4_ss(d, w_re, k_re, dhi, I64, 0u);
-                        mma4_ss(d, w_im, k_im, dhi, I64, 1u);
-                    } else {
-                        mma4_ss(d, w_re, k_im, dhi, I64, 0u);
-                        mma4_ss(d, w_im, k_re, dhi, I64N, 1u);
+                    // rows = [W ; Qt], columns = tokens i.  Re: W_re Kc_re + W_im Kc_im; Im: W_re Kc_im - W_im Kc_re
+                    if (elect_one()) {
+                        const uint32_t d = tmem + TM_GRAM, w_a = w_re, w_im = w_re + 2 * kIm;
+                        const uint32_t k2 = gh ? k_re : k_re + kIm;      // partner of the second product
+                        const uint32_t id2 = gh ? I64 | (1u << 14) : I64;
+                        mma_ss2(d, w_a, dhi, k_b, dhi, I64, 0u);
+                        mma_ss2(d, w_a + 2, dhi, k_b + 2, dhi, I64, 1u);
+                        mma_ss2(d, w_a + 4, dhi, k_b + 4, dhi, I64, 1u);
+                        mma_ss2(d, w_a + 6, dhi, k_b + 6, dhi, I64, 1u);
+                        mma_ss2(d, w_im, dhi, k2, dhi, id2, 1u);
+                        mma_ss2(d, w_im + 2, dhi, k2 + 2, dhi, id2, 1u);
+                        mma_ss2(d, w_im + 4, dhi, k2 + 4, dhi, id2, 1u);
+                        mma_ss2(d, w_im + 6, dhi, k2 + 6, dhi, id2, 1u);
+                        mma_commit(&bars[B_GRAM_FULL]);
                     }
-                    mma_commit(&bars[B_GRAM_FULL]);
+                    __syncwarp();
                     g += gh;
                     gh ^= 1;
                     progress = true;
                 }
             }
-            if (jv < n_chunks && test_k(mi, B_R16_READY, jv - 1)) {
-                vcur.next(p);
+            if (jv < n_chunks && (jv == 0 || test_k_warp(mi, B_R16_READY, jv - 1))) {
                 const ChunkInfo cv = vcur.ci;
-                mbar_expect_tx(&bars[B_V_FULL], 16384);
-                tma_load_4d(smem + OFF_V, tm_v, &bars[B_V_FULL], 0, cv.h, cv.jg * C, cv.b);
+                vcur.next(p);
+                if (elect_one()) {
+                    mbar_expect_tx(&bars[B_V_FULL], 16384);
+                    tma_load_4d(smem + OFF_V, tm_v, &bars[B_V_FULL], 0, cv.h, cv.jg * C, cv.b);
+                }
+                __syncwarp();
                 ++jv;
                 progress = true;
             }
-            if (!progress) {
+            if (progress) {
+                t0 = (uint32_t)clock();
+            } else {
                 __nanosleep(64);
-                if ((it & 63u) == 63u) {
-                    if (mi.abort) return;
-                    if (now_ticks() - t0 > 2 * kWaitLimitTicks + 2000000ull * (unsigned long long)n_chunks) {
-                        mi.abort = 1;
-                        return;
-                    }
+                if (mi.abort || (uint32_t)clock() - t0 > 0x80000000u) {      // a second without progress
+                    mi.abort = 1;
+                    return;
                 }
             }
         }
@@ -811,12 +841,6 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
 }
 
 // ---- CHAIN --------------------------------------------------------------------------------------------
-// wait_k with a warp-uniform outcome, so that a warp leaves (or stays) as a whole
-__device__ __forceinline__ bool wait_k_warp(Misc &mi, int bar, int k)
-{
-    return __all_sync(0xffffffffu, wait_k(mi, bar, k) ? 1 : 0) != 0;
-}
-
 __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int n_chunks, int ct)
 {
     long long *timing = p.timing;
@@ -1046,7 +1070,7 @@ sfda_forward_ws_kernel(const __grid_constant__ CUtensorMap tm_v, const __grid_co
         const int cw = warp - (kChainWarps + kSolveWarps + kPrepWarps);
         if (cw == 3)
             run_prefetch(mi, p, n_chunks, tid & 31);
-        else if ((tid & 31) == 0)
+        else
             run_ctrl(cw, smem, mi, tmem, &tm_v, &tm_o, &tm_oim, p, n_chunks);
     }
 
@@ -1172,9 +1196,9 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
     if ((e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
 
     // Time slices per sequence: one CTA per SM works through ceil(units / SMs) units of NC / Q chunks.  More
-    // slices even out the last round, but every unit boundary costs about two chunk periods (the state goes
-    // through global memory and the next slice waits for it), so slicing is chosen only when it removes at least
-    // 15 % of the rounds' chunk count (for instance a few more sequences than SMs, or few very long sequences).
+    // slices even out the last round (256 sequences on 148 SMs: two rounds of 128 chunks, or seven rounds of
+    // 32); every unit boundary costs about one chunk period (the state goes through global memory and the next
+    // slice waits for it).  The smallest Q within 3 % of the cheapest is taken.
     const int BH = a.B * a.H, NC = (a.T + C - 1) / C;
     int Q = 1;
     if (scratch_bytes >= forward_ws_scratch_bytes(a.B, a.H)) {
@@ -1182,9 +1206,8 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
         for (int q = 1; q <= 8; q *= 2) {
             if (NC % q != 0 || NC / q < 4) break;
             const long units = (long)BH * q;
-            const double cost = (double)((units + n_sm - 1) / n_sm) * (NC / q + 2.0);
-            if (q == 1) best = cost;
-            else if (cost < 0.85 * best) { best = cost / 0.85; Q = q; }
+            const double cost = (double)((units + n_sm - 1) / n_sm) * (NC / q + 1.0);
+            if (q == 1 || cost < 0.97 * best) { best = cost; Q = q; }
         }
     }
 #ifdef SFDA_WS_TIMING
