@@ -21,12 +21,14 @@ __device__ __forceinline__ uint32_t phase_to_turns(float theta)
 {
     const double turns_per_radian = 0x1.45f306dc9c883p+29;  // 2^32 / (2 pi), nearest double
     const double d = __dmul_rn((double)theta, turns_per_radian);
-    if (fabsf(theta) < 1.0e6f) {
-        // |d| < 2^51: adding 1.5 * 2^52 rounds d to an integer (to nearest, ties to even) and leaves that
-        // integer, modulo 2^32, in the low word of the sum -- the same value as the conversion below.
-        return (uint32_t)__double2loint(__dadd_rn(d, 6755399441055744.0));
-    }
-    return (uint32_t)(unsigned long long)__double2ll_rn(d);
+    // |theta| < 1e6 gives |d| < 2^51: adding 1.5 * 2^52 rounds d to an integer (to nearest, ties to even) and
+    // leaves that integer, modulo 2^32, in the low word of the sum.  Larger angles take the (slow) conversion
+    // instruction instead, under a predicate rather than a branch so that the common case stays straight-line.
+    uint32_t u = (uint32_t)__double2loint(__dadd_rn(d, 6755399441055744.0));
+    asm("{\n.reg .pred p;\n.reg .s64 t;\nsetp.ge.f32 p, %2, 0f49742400;\n@p cvt.rni.s64.f64 t, %1;\n@p cvt.u32.u64 %0, t;\n}\n"
+        : "+r"(u)
+        : "d"(d), "f"(fabsf(theta)));
+    return u;
 }
 
 // cos / sin of a phase given in turns (signed view keeps the float argument in [-1, 1)).

@@ -43,6 +43,8 @@ constexpr int kChainThreads = 32 * kChainWarps, kSolveThreads = 32 * kSolveWarps
 // The CTA is launched with 80 registers per thread (768 * 80 = 61440); the working roles take what CTRL gives up:
 // (8 + 4 + 8) * 88 + 4 * 40 = 1920 warp rows = 61440 registers.
 constexpr int kRegsWork = 88, kRegsCtrl = 40;
+constexpr int kTB = 2;
+            // tokens per trip of PREP's operand loop
 
 // ---- shared memory map (bytes from a 1024-aligned base) -------------------------------------------------
 constexpr int kTile = 8192;                       // 64 rows x 128 B, 128B swizzle
@@ -515,20 +517,19 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
     auto drain_outputs = [&](int jd) {           // rho of chunk jd -> bf16 staging tiles [t][128]
         if (!dead && !wait_k(mi, B_UPD_DONE, jd)) dead = true;
         // the Re staging tile is shared by all chunks: the store of chunk jd-1 must have read it
-        if (jd >= 1 && !dead && !wait_k(mi, (jd - 1) & 1 ? B_STORE_DONE1 : B_STORE_DONE0, (jd - 1) >> 1)) dead = true;
+        if (jd >= 1 && !dead && !wait_k(mi, B_STORE_DONE0 + ((jd - 1) & 1), (jd - 1) >> 1)) dead = true;
         tc_fence_after();
         if (half == 0 || p.has_o_im) {
             __nv_bfloat16 *stage =
-                reinterpret_cast<__nv_bfloat16 *>(smem + (half ? OFF_AQ + (jd & 1) * 2 * kTile : OFF_OST));
+                reinterpret_cast<__nv_bfloat16 *>(smem + (half ? OFF_AQ + (jd & 1) * 2 * kTile : OFF_OST)) + c;
             const float sgn = half ? -1.f : 1.f;   // o = conj(rho)
 #pragma unroll 1
-            for (int hc = 0; hc < 2; ++hc) {
-                uint32_t r[32];
-                tmem_ld<32>(tlane + TM_ACC + 64 + 128 * half + 32 * hc, r);
+            for (int pc = 0; pc < 4; ++pc) {
+                uint32_t r[16];
+                tmem_ld<16>(tlane + TM_ACC + 64 + 128 * half + 16 * pc, r);
                 tc_wait_ld();
 #pragma unroll
-                for (int t = 0; t < 32; ++t)
-                    stage[(32 * hc + t) * DV + c] = __float2bfloat16_rn(sgn * __uint_as_float(r[t]));
+                for (int t = 0; t < 16; ++t) stage[(16 * pc + t) * DV] = __float2bfloat16_rn(sgn * __uint_as_float(r[t]));
             }
         }
         fence_async_smem();
@@ -537,44 +538,52 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
     };
     SFDA_TDECL(pt == 0);
     ChunkCursor cur(p);
+#pragma unroll 1
     for (int j = 0; j < n_chunks + 2; ++j) {
         if (role_sync_or(2, kPrepThreads, dead || mi.abort)) break;
         const bool live = j < n_chunks;          // after the last chunk only the outputs of two chunks are left
         const int s = j & 1, ring = j & 3;
-        float2 al[8], th[8];
-        uint2 kw[8], qw[8];
-        float lg0[8], lg1[8];
-        uint32_t tu0[8], tu1[8];
         float base0 = 1.f, base1 = 1.f;
         uint32_t tb0 = 0u, tb1 = 0u;
+        size_t off = 0, step = 0;                // byte offset of this thread's first token in q/k/alpha/theta
+        int nt = 0;                              // real tokens in this thread's octet
+        struct Tok { uint2 al, th, k, q; } tk[kTB];   // alpha and theta as raw bits
+        auto load_token = [&](Tok &t, int i) {   // inputs of token i of the octet; neutral beyond the sequence
+            t.al = make_uint2(0x3f800000u, 0x3f800000u); t.th = make_uint2(0u, 0u);
+            t.k = make_uint2(0u, 0u); t.q = make_uint2(0u, 0u);
+            const size_t o = off + (size_t)i * step;
+            const bool on = i < nt;
+            ldg64_if(t.al.x, t.al.y, reinterpret_cast<const char *>(p.alpha) + o, on);
+            ldg64_if(t.th.x, t.th.y, reinterpret_cast<const char *>(p.theta) + o, on);
+            ldg64_if(t.k.x, t.k.y, reinterpret_cast<const char *>(p.k) + o, on);
+            ldg64_if(t.q.x, t.q.y, reinterpret_cast<const char *>(p.q) + o, on);
+        };
         if (live) {
             const ChunkInfo ci = cur.ci;
             cur.next(p);
             const int t0 = ci.jg * C, len = min(C, p.T - t0);
             const size_t row0 = ((size_t)ci.b * p.T + t0) * p.H + ci.h;   // token t of this head: row0 + t * H
-            const int nt = min(8, max(0, len - tq * 8));             // real tokens in this thread's octet
+            nt = min(8, max(0, len - tq * 8));
+            // all four arrays have 256 bytes per (token, head): the same byte offset serves them all
+            step = (size_t)p.H * 256;
+            off = (row0 + (size_t)(tq * 8) * p.H) * 256 + 8 * jp;
             SFDA_T(35);
 
-            // all loads of this thread for the chunk, issued together
+            // pass 1: this thread's product of alpha (fp32 products of at most 64 factors: relative error far
+            // below bf16's) and sum of the integer phase over its 8 tokens
+            float2 al[8], th[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                const size_t row = row0 + (size_t)(tq * 8 + i) * p.H;
                 al[i] = make_float2(1.f, 1.f);
                 th[i] = make_float2(0.f, 0.f);
-                kw[i] = make_uint2(0u, 0u);
-                qw[i] = make_uint2(0u, 0u);
                 if (i < nt) {
-                    al[i] = __ldg(reinterpret_cast<const float2 *>(p.alpha + row * M) + jp);
-                    th[i] = __ldg(reinterpret_cast<const float2 *>(p.theta + row * M) + jp);
-                    kw[i] = __ldg(reinterpret_cast<const uint2 *>(p.k + row * DK) + jp);
-                    qw[i] = __ldg(reinterpret_cast<const uint2 *>(p.q + row * DK) + jp);
+                    al[i] = __ldg(reinterpret_cast<const float2 *>(reinterpret_cast<const char *>(p.alpha) + off + i * step));
+                    th[i] = __ldg(reinterpret_cast<const float2 *>(reinterpret_cast<const char *>(p.theta) + off + i * step));
                 }
             }
             SFDA_T(36);
             if (pt < C) mi.beta[ring][pt] = pt < len ? __ldg(p.beta + row0 + (size_t)pt * p.H) : 0.f;
             SFDA_T(37);
-            // pass 1: prefix products of alpha (a_t: fp32 products of at most 64 factors, relative error far
-            // below bf16's) and prefix sums of the integer phase over this thread's 8 tokens
             {
                 float a0 = 1.f, a1 = 1.f;
                 uint32_t u0 = 0u, u1 = 0u;
@@ -584,39 +593,39 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
                     a1 *= fmaxf(al[i].y, 9.0e-14f);
                     u0 += phase_to_turns(th[i].x);
                     u1 += phase_to_turns(th[i].y);
-                    lg0[i] = a0; lg1[i] = a1; tu0[i] = u0; tu1[i] = u1;
                 }
-                mi.part_lg[tq][2 * jp] = a0;
-                mi.part_lg[tq][2 * jp + 1] = a1;
-                mi.part_turns[tq][2 * jp] = u0;
-                mi.part_turns[tq][2 * jp + 1] = u1;
+                *reinterpret_cast<float2 *>(&mi.part_lg[tq][2 * jp]) = make_float2(a0, a1);
+                *reinterpret_cast<uint2 *>(&mi.part_turns[tq][2 * jp]) = make_uint2(u0, u1);
             }
             SFDA_T(30);
-            role_sync(2, kPrepThreads);
-            float tot0 = 1.f, tot1 = 1.f;
-            uint32_t tt0 = 0u, tt1 = 0u;
 #pragma unroll
-            for (int gq = 0; gq < 8; ++gq) {
+            for (int ii = 0; ii < kTB; ++ii) load_token(tk[ii], ii);
+            role_sync(2, kPrepThreads);
+            // octet tq starts from the product of the octets before it; octet 0 instead multiplies all eight:
+            // the chunk totals a_C e^{i phi_C}, applied by the next state pass
+            const int n_before = tq == 0 ? 8 : tq;
+#pragma unroll 1
+            for (int gq = 0; gq < n_before; ++gq) {
                 const float2 pl = *reinterpret_cast<const float2 *>(&mi.part_lg[gq][2 * jp]);
                 const uint2 pu = *reinterpret_cast<const uint2 *>(&mi.part_turns[gq][2 * jp]);
-                if (gq < tq) { base0 *= pl.x; base1 *= pl.y; tb0 += pu.x; tb1 += pu.y; }
-                tot0 *= pl.x; tot1 *= pl.y; tt0 += pu.x; tt1 += pu.y;
+                base0 *= pl.x; base1 *= pl.y; tb0 += pu.x; tb1 += pu.y;
             }
-            if (tq == 0) {                    // chunk totals: a_C e^{i phi_C}, applied by the next state pass
+            if (tq == 0) {
                 float cs, sn;
-                turns_sincos(tt0, &sn, &cs);
-                mi.close_re[ring][2 * jp] = tot0 * cs;
-                mi.close_im[ring][2 * jp] = tot0 * sn;
-                turns_sincos(tt1, &sn, &cs);
-                mi.close_re[ring][2 * jp + 1] = tot1 * cs;
-                mi.close_im[ring][2 * jp + 1] = tot1 * sn;
+                turns_sincos(tb0, &sn, &cs);
+                mi.close_re[ring][2 * jp] = base0 * cs;
+                mi.close_im[ring][2 * jp] = base0 * sn;
+                turns_sincos(tb1, &sn, &cs);
+                mi.close_re[ring][2 * jp + 1] = base1 * cs;
+                mi.close_im[ring][2 * jp + 1] = base1 * sn;
+                base0 = 1.f; base1 = 1.f; tb0 = 0u; tb1 = 0u;
             }
             SFDA_T(31);
 
             // the slot's tiles must have been consumed: W/Qt by rho_1 of chunk j-2, Kc by its state update
             if (j >= 2) {
-                if (!dead && !wait_k(mi, s ? B_WQ_FREE1 : B_WQ_FREE0, (j >> 1) - 1)) dead = true;
-                if (!dead && !wait_k(mi, s ? B_KC_FREE1 : B_KC_FREE0, (j >> 1) - 1)) dead = true;
+                if (!dead && !wait_k(mi, B_WQ_FREE0 + s, (j >> 1) - 1)) dead = true;
+                if (!dead && !wait_k(mi, B_KC_FREE0 + s, (j >> 1) - 1)) dead = true;
             }
             SFDA_T(32);
         }
@@ -626,39 +635,49 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
         SFDA_T(34);
         if (!live) continue;
 
-        // pass 2: rotated / decayed operands
-        uint8_t *wq_re = smem + OFF_WQ + s * 4 * kTile, *wq_im = wq_re + 2 * kTile;
-        uint8_t *kc_re = smem + OFF_KC + s * 2 * kTile, *kc_im = kc_re + kTile;
+        // pass 2: rotated / decayed operands.  A rolled loop over groups of kTB tokens keeps the code small; each
+        // token's inputs (from L1 / L2: pass 1 or the prefetch warp brought them in) are fetched into the
+        // registers of the token kTB places before it as soon as that one has been worked on.
+        const uint32_t wq_re = smem_u32(smem) + OFF_WQ + s * 4 * kTile + tq * 1024 + (jp & 3) * 4;   // + row, swizzle
+        const uint32_t kc_re = smem_u32(smem) + OFF_KC + s * 2 * kTile + tq * 1024 + (jp & 3) * 4;
+#pragma unroll 1
+        for (int h = 0; h < 8 / kTB; ++h) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int t = tq * 8 + i;
-            float wr[2], wi[2], cr_[2], ci_[2], qr_[2], qi_[2];
+            for (int ii = 0; ii < kTB; ++ii) {
+                const int i = h * kTB + ii;
+                base0 *= fmaxf(__uint_as_float(tk[ii].al.x), 9.0e-14f);                  // a_t, phase of token t
+                base1 *= fmaxf(__uint_as_float(tk[ii].al.y), 9.0e-14f);
+                tb0 += phase_to_turns(__uint_as_float(tk[ii].th.x));
+                tb1 += phase_to_turns(__uint_as_float(tk[ii].th.y));
+                float wr[2], wi[2], cr_[2], ci_[2], qr_[2], qi_[2];
 #pragma unroll
-            for (int x = 0; x < 2; ++x) {
-                const float a = x ? base1 * lg1[i] : base0 * lg0[i];           // a_t
-                const uint32_t tu = x ? tb1 + tu1[i] : tb0 + tu0[i];
-                const uint32_t kx = x ? kw[i].y : kw[i].x, qx = x ? qw[i].y : qw[i].x;
-                const float ainv = fminf(__fdividef(1.0f, a), 5.5e34f);              // 1/a_t, capped at e^80
-                float cs, sn;
-                turns_sincos(tu, &sn, &cs);
-                const float kr = __uint_as_float(kx << 16), ki = __uint_as_float(kx & 0xffff0000u);
-                const float qr = __uint_as_float(qx << 16), qi = __uint_as_float(qx & 0xffff0000u);
-                const float kpr = kr * cs + ki * sn, kpi = ki * cs - kr * sn;   // e^{-i phi} k
-                const float qpr = qr * cs + qi * sn, qpi = qi * cs - qr * sn;
-                wr[x] = a * kpr; wi[x] = a * kpi;
-                qr_[x] = a * qpr; qi_[x] = a * qpi;
-                cr_[x] = ainv * kpr; ci_[x] = ainv * kpi;
+                for (int x = 0; x < 2; ++x) {
+                    const float a = x ? base1 : base0;
+                    const uint32_t tu = x ? tb1 : tb0;
+                    const uint32_t kx = x ? tk[ii].k.y : tk[ii].k.x, qx = x ? tk[ii].q.y : tk[ii].q.x;
+                    const float ainv = fminf(__fdividef(1.0f, a), 5.5e34f);              // 1/a_t, capped at e^80
+                    float cs, sn;
+                    turns_sincos(tu, &sn, &cs);
+                    const float kr = __uint_as_float(kx << 16), ki = __uint_as_float(kx & 0xffff0000u);
+                    const float qr = __uint_as_float(qx << 16), qi = __uint_as_float(qx & 0xffff0000u);
+                    const float kpr = kr * cs + ki * sn, kpi = ki * cs - kr * sn;   // e^{-i phi} k
+                    const float qpr = qr * cs + qi * sn, qpi = qi * cs - qr * sn;
+                    wr[x] = a * kpr; wi[x] = a * kpi;
+                    qr_[x] = a * qpr; qi_[x] = a * qpi;
+                    cr_[x] = ainv * kpr; ci_[x] = ainv * kpi;
+                }
+                load_token(tk[ii], i + kTB);
+                const int o1 = i * 128 + ((((jp >> 2) ^ i) & 7) << 4);      // row i of the octet's 8-row swizzle atom
+                sts32(wq_re + o1, pack_bf16(wr[0], wr[1]));
+                sts32(wq_re + 2 * kTile + o1, pack_bf16(wi[0], wi[1]));
+                sts32(wq_re + kTile + o1, pack_bf16(qr_[0], qr_[1]));
+                sts32(wq_re + 3 * kTile + o1, pack_bf16(qi_[0], qi_[1]));
+                sts32(kc_re + o1, pack_bf16(cr_[0], cr_[1]));
+                sts32(kc_re + kTile + o1, pack_bf16(ci_[0], ci_[1]));
             }
-            const int o1 = sw_off(t, 2 * jp);
-            *reinterpret_cast<uint32_t *>(wq_re + o1) = pack_bf16(wr[0], wr[1]);
-            *reinterpret_cast<uint32_t *>(wq_im + o1) = pack_bf16(wi[0], wi[1]);
-            *reinterpret_cast<uint32_t *>(wq_re + kTile + o1) = pack_bf16(qr_[0], qr_[1]);
-            *reinterpret_cast<uint32_t *>(wq_im + kTile + o1) = pack_bf16(qi_[0], qi_[1]);
-            *reinterpret_cast<uint32_t *>(kc_re + o1) = pack_bf16(cr_[0], cr_[1]);
-            *reinterpret_cast<uint32_t *>(kc_im + o1) = pack_bf16(ci_[0], ci_[1]);
         }
         fence_async_smem();
-        warp_arrive(&mi.bars[s ? B_PREP_FULL1 : B_PREP_FULL0]);
+        warp_arrive(&mi.bars[B_PREP_FULL0 + s]);
         SFDA_T(33);
     }
 }

@@ -168,10 +168,33 @@ __device__ __forceinline__ void tmem_st(uint32_t addr, const uint32_t *r)
     for (int i = 0; i < N; i += 16) tmem_st16(addr + i, r + i);
 }
 
+// Two floats -> packed bf16x2 (low half = lo), one conversion instruction.
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
-    return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) |
-           ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+// Shared-memory stores / loads by 32-bit shared address (no 64-bit generic address arithmetic).
+__device__ __forceinline__ void sts32(uint32_t saddr, uint32_t v)
+{
+    asm volatile("st.shared.b32 [%0], %1;" ::"r"(saddr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void sts16(uint32_t saddr, uint16_t v)
+{
+    asm volatile("st.shared.b16 [%0], %1;" ::"r"(saddr), "h"(v) : "memory");
+}
+__device__ __forceinline__ void sts128(uint32_t saddr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+// Global loads through the read-only path that only happen when `on` is set (the destination keeps its value
+// otherwise): no branch, so neighbouring work can be scheduled across them.
+__device__ __forceinline__ void ldg64_if(uint32_t &x, uint32_t &y, const void *ptr, bool on)
+{
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %3, 0;\n@p ld.global.nc.v2.b32 {%0, %1}, [%2];\n}\n"
+                 : "+r"(x), "+r"(y)
+                 : "l"(ptr), "r"((uint32_t)on));
 }
 // Byte offset of element (row r, k-element e < 64) in a K-major 128B-swizzled tile.
 __device__ __forceinline__ int sw_off(int r, int e)
