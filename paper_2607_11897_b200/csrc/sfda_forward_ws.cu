@@ -78,7 +78,7 @@ enum Bar {
 struct Misc {
     float part_lg[8][M];
     uint32_t part_turns[8][M];
-    float close_re[4][M], close_im[4][M];   // a_C e^{i phi_C} of a ring of four chunks
+    float2 close[4][M];                     // a_C e^{i phi_C} of a ring of four chunks
     float beta[4][C];
     unsigned long long bars[kNumBars];
     uint32_t tmem_base;
@@ -582,7 +582,9 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
                 }
             }
             SFDA_T(36);
-            if (pt < C) mi.beta[ring][pt] = pt < len ? __ldg(p.beta + row0 + (size_t)pt * p.H) : 0.f;
+            // beta of token pt: fetched now, written after the pass below so that its latency is covered
+            float beta_t = 0.f;
+            if (pt < len) beta_t = __ldg(p.beta + row0 + (size_t)pt * p.H);
             SFDA_T(37);
             {
                 float a0 = 1.f, a1 = 1.f;
@@ -597,6 +599,7 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
                 *reinterpret_cast<float2 *>(&mi.part_lg[tq][2 * jp]) = make_float2(a0, a1);
                 *reinterpret_cast<uint2 *>(&mi.part_turns[tq][2 * jp]) = make_uint2(u0, u1);
             }
+            if (pt < C) mi.beta[ring][pt] = beta_t;
             SFDA_T(30);
 #pragma unroll
             for (int ii = 0; ii < kTB; ++ii) load_token(tk[ii], ii);
@@ -613,11 +616,9 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
             if (tq == 0) {
                 float cs, sn;
                 turns_sincos(tb0, &sn, &cs);
-                mi.close_re[ring][2 * jp] = base0 * cs;
-                mi.close_im[ring][2 * jp] = base0 * sn;
+                mi.close[ring][2 * jp] = make_float2(base0 * cs, base0 * sn);
                 turns_sincos(tb1, &sn, &cs);
-                mi.close_re[ring][2 * jp + 1] = base1 * cs;
-                mi.close_im[ring][2 * jp + 1] = base1 * sn;
+                mi.close[ring][2 * jp + 1] = make_float2(base1 * cs, base1 * sn);
                 base0 = 1.f; base1 = 1.f; tb0 = 0u; tb1 = 0u;
             }
             SFDA_T(31);
@@ -868,121 +869,13 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
     const int c = quad * 32 + lane;            // value channel = TMEM lane
     const int j0 = half * 32;                  // this warp's complex rows in the state pass
     const uint32_t tlane = tmem + ((uint32_t)(quad * 32) << 16);
-
-    // One 16-row piece of the state pass: rows j0 + 16 pc .. + 15 (Re and Im).  Inside a unit the chunk-start
-    // state is the accumulated state of the previous chunk times a_C e^{i phi_C}; at the first chunk of a unit it
-    // comes from global memory (`src`, NULL = zero state).
-    auto state_piece = [&](int pc, int ring, bool first, const float *src) {
-        uint32_t sre[16], sim[16], pk[8];
-        const int jb = j0 + 16 * pc;
-        if (first) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int jj = jb + i;
-                sre[i] = src ? __float_as_uint(__ldcg(src + (size_t)(2 * jj) * DV + c)) : 0u;
-                sim[i] = src ? __float_as_uint(__ldcg(src + (size_t)(2 * jj + 1) * DV + c)) : 0u;
-            }
-        } else {
-            tmem_ld<16>(tlane + TM_S32 + jb, sre);
-            tmem_ld<16>(tlane + TM_S32 + 64 + jb, sim);
-            tc_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const float cs = mi.close_re[ring][jb + i], sn = mi.close_im[ring][jb + i];
-                const float xr = __uint_as_float(sre[i]), xi = __uint_as_float(sim[i]);
-                sre[i] = __float_as_uint(cs * xr - sn * xi);
-                sim[i] = __float_as_uint(cs * xi + sn * xr);
-            }
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) pk[i] = pack_bf16(__uint_as_float(sre[2 * i]), __uint_as_float(sre[2 * i + 1]));
-        tmem_st8(tlane + TM_X16 + jb / 2, pk);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) pk[i] = pack_bf16(__uint_as_float(sim[2 * i]), __uint_as_float(sim[2 * i + 1]));
-        tmem_st8(tlane + TM_X16 + 32 + jb / 2, pk);
-        tmem_st<16>(tlane + TM_S32 + jb, sre);
-        tmem_st<16>(tlane + TM_S32 + 64 + jb, sim);
-    };
-    // The unit that ended with stream chunk `jl` is finished: its final state e^{i phi_C} a_C S goes to S_T (last
-    // time slice) or to the hand-off buffer, where the CTA that runs the next slice is told about it.
-    auto write_out_state = [&](int jl, const ChunkInfo &pi) {
-        const int ring = jl & 3;
-        float *dst = pi.q == p.Q - 1 ? p.S_T : p.handoff;
-        if (dst) {
-            dst += (size_t)pi.bh * DK * DV;
-#pragma unroll
-            for (int pc = 0; pc < 2; ++pc) {
-                uint32_t sre[16], sim[16];
-                const int jb = j0 + 16 * pc;
-                tmem_ld<16>(tlane + TM_S32 + jb, sre);
-                tmem_ld<16>(tlane + TM_S32 + 64 + jb, sim);
-                tc_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const int jj = jb + i;
-                    const float cs = mi.close_re[ring][jj], sn = mi.close_im[ring][jj];
-                    const float xr = __uint_as_float(sre[i]), xi = __uint_as_float(sim[i]);
-                    __stcg(dst + (size_t)(2 * jj) * DV + c, cs * xr - sn * xi);
-                    __stcg(dst + (size_t)(2 * jj + 1) * DV + c, cs * xi + sn * xr);
-                }
-            }
-        }
-        if (pi.q < p.Q - 1) {              // one count per warp: slice q + 1 may start once all eight have arrived
-            __threadfence();
-            __syncwarp();
-            if (lane == 0) atomicAdd(p.flags + pi.bh, 1u);
-        }
-    };
-    // Wait until the boundary state of this sequence's previous time slice has been written (eight warp counts
-    // per slice).  Bounded like every other wait; warp-uniform result.
-    auto wait_handoff = [&](const ChunkInfo &ci) -> bool {
-        int ok = 1;
-        if (lane == 0) {
-            const uint32_t want = 8u * (uint32_t)ci.q;
-            const unsigned long long t0 = now_ticks();
-            ok = 0;
-            for (uint32_t it = 0;; ++it) {
-                uint32_t seen;
-                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(p.flags + ci.bh) : "memory");
-                if (seen >= want) { ok = 1; break; }
-                __nanosleep(200);
-                if ((it & 63u) == 63u && (mi.abort || now_ticks() - t0 > kWaitLimitTicks)) break;
-            }
-            if (!ok) mi.abort = 1;
-        }
-        ok = __shfl_sync(0xffffffffu, ok, 0);
-        __threadfence();
-        return ok != 0;
-    };
-    // bf16 A operand from 64 fp32 accumulator columns of this warp's half, 32 columns at a time.
-    // mode 1: R = V - D1 (Re half); mode 2: negated (Im half of R = -D1); mode 0: as is (E).
-    auto convert_acc = [&](int mode) {
-#pragma unroll 1
-        for (int hc = 0; hc < 2; ++hc) {
-            uint32_t r[32], pk[16];
-            tmem_ld<32>(tlane + TM_ACC + 128 * half + 32 * hc, r);
-            tc_wait_ld();
-            if (mode == 1) {
-                const __nv_bfloat16 *sv = reinterpret_cast<const __nv_bfloat16 *>(smem + OFF_V) + (32 * hc) * DV + c;
-#pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    pk[i] = pack_bf16(__bfloat162float(sv[(2 * i) * DV]) - __uint_as_float(r[2 * i]),
-                                      __bfloat162float(sv[(2 * i + 1) * DV]) - __uint_as_float(r[2 * i + 1]));
-            } else {
-                const float sgn = mode == 2 ? -1.f : 1.f;
-#pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    pk[i] = pack_bf16(sgn * __uint_as_float(r[2 * i]), sgn * __uint_as_float(r[2 * i + 1]));
-            }
-            tmem_st<16>(tlane + TM_X16 + 32 * half + 16 * hc, pk);
-        }
-        tc_wait_st();
-    };
+    const uint32_t sv = smem_u32(smem) + OFF_V + 2 * c;   // v[t][c], rows of 256 bytes
 
     SFDA_TDECL(ct == 0);
     ChunkCursor cur(p);
     ChunkInfo prev_ci = cur.ci;
-    for (int j = 0; j < n_chunks; ++j) {
+#pragma unroll 1
+    for (int j = 0; j <= n_chunks; ++j) {
         // ---- state pass: S_0 of this chunk = e^{i phi_C} a_C (accumulated state of the previous chunk)
         if (j > 0) {
             if (!wait_k_warp(mi, B_UPD_DONE, j - 1)) return;
@@ -990,21 +883,97 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
         }
         SFDA_T(10);
         const ChunkInfo ci = cur.ci;
+        const bool fin = j == n_chunks;
+        const float2 *close = mi.close[(j - 1) & 3];
         const float *src = nullptr;
-        if (ci.first) {
-            if (j > 0) write_out_state(j - 1, prev_ci);
+        if (fin || ci.first) {
+            // A unit ends (chunk j - 1 was its last): its final state e^{i phi_C} a_C S goes to S_T (last time
+            // slice) or to the hand-off buffer, where the CTA that runs the next slice is told about it.
+            if (j > 0) {
+                float *dst = prev_ci.q == p.Q - 1 ? p.S_T : p.handoff;
+                if (dst) {
+                    dst += (size_t)prev_ci.bh * DK * DV + c;
+#pragma unroll 1
+                    for (int pc = 0; pc < 4; ++pc) {
+                        uint32_t sre[8], sim[8];
+                        const int jb = j0 + 8 * pc;
+                        tmem_ld8(tlane + TM_S32 + jb, sre);
+                        tmem_ld8(tlane + TM_S32 + 64 + jb, sim);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const float2 cl = close[jb + i];
+                            const float xr = __uint_as_float(sre[i]), xi = __uint_as_float(sim[i]);
+                            __stcg(dst + (size_t)(2 * (jb + i)) * DV, cl.x * xr - cl.y * xi);
+                            __stcg(dst + (size_t)(2 * (jb + i) + 1) * DV, cl.x * xi + cl.y * xr);
+                        }
+                    }
+                }
+                if (prev_ci.q < p.Q - 1) {     // one count per warp: slice q + 1 may start once all eight have arrived
+                    __threadfence();
+                    __syncwarp();
+                    if (lane == 0) atomicAdd(p.flags + prev_ci.bh, 1u);
+                }
 #ifdef SFDA_WS_TIMING
-            if (j > 0 && ct == 0 && p.timing) p.timing[512 + blockIdx.x] = (long long)now_ns();
+                if (ct == 0 && p.timing) p.timing[512 + blockIdx.x] = (long long)now_ns();
 #endif
+            }
+            if (fin) break;
             if (ci.q == 0) {
-                src = p.S0 ? p.S0 + (size_t)ci.bh * DK * DV : nullptr;
+                src = p.S0 ? p.S0 + (size_t)ci.bh * DK * DV + c : nullptr;
             } else {
-                if (!wait_handoff(ci)) return;
-                src = p.handoff + (size_t)ci.bh * DK * DV;
+                // the boundary state of this sequence's previous time slice must have been written (eight warp
+                // counts per slice); bounded like every other wait, warp-uniform result
+                int ok = 1;
+                if (lane == 0) {
+                    const uint32_t want = 8u * (uint32_t)ci.q, t0 = (uint32_t)clock();
+                    uint32_t seen;
+                    do {
+                        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(p.flags + ci.bh) : "memory");
+                        if (seen >= want) break;
+                        __nanosleep(200);
+                    } while (!mi.abort && (uint32_t)clock() - t0 < 0x80000000u);
+                    ok = seen >= want;
+                    if (!ok) mi.abort = 1;
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                __threadfence();
+                if (!ok) return;
+                src = p.handoff + (size_t)ci.bh * DK * DV + c;
             }
         }
+        // 16 complex rows at a time: fp32 state (decayed and rotated in place) and its bf16 copy, the A operand
 #pragma unroll 1
-        for (int pc = 0; pc < 2; ++pc) state_piece(pc, (j - 1) & 3, ci.first, src);
+        for (int pc = 0; pc < 2; ++pc) {
+            uint32_t sre[16], sim[16], pk[8];
+            const int jb = j0 + 16 * pc;
+            if (ci.first) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    sre[i] = src ? __float_as_uint(__ldcg(src + (size_t)(2 * (jb + i)) * DV)) : 0u;
+                    sim[i] = src ? __float_as_uint(__ldcg(src + (size_t)(2 * (jb + i) + 1) * DV)) : 0u;
+                }
+            } else {
+                tmem_ld<16>(tlane + TM_S32 + jb, sre);
+                tmem_ld<16>(tlane + TM_S32 + 64 + jb, sim);
+                tc_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float2 cl = close[jb + i];
+                    const float xr = __uint_as_float(sre[i]), xi = __uint_as_float(sim[i]);
+                    sre[i] = __float_as_uint(cl.x * xr - cl.y * xi);
+                    sim[i] = __float_as_uint(cl.x * xi + cl.y * xr);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pk[i] = pack_bf16(__uint_as_float(sre[2 * i]), __uint_as_float(sre[2 * i + 1]));
+            tmem_st8(tlane + TM_X16 + jb / 2, pk);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pk[i] = pack_bf16(__uint_as_float(sim[2 * i]), __uint_as_float(sim[2 * i + 1]));
+            tmem_st8(tlane + TM_X16 + 32 + jb / 2, pk);
+            tmem_st<16>(tlane + TM_S32 + jb, sre);
+            tmem_st<16>(tlane + TM_S32 + 64 + jb, sim);
+        }
         prev_ci = ci;
         cur.next(p);
         tc_wait_st();
@@ -1012,8 +981,9 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
         warp_arrive(&mi.bars[B_S16_READY]);
         SFDA_T(11);
 
-        // ---- R = V - D1, then E, -> bf16 A operand (D1 and rho_1, which read S_0 from the same columns, are both
-        // done when D1 is)
+        // ---- R = V - D1 (ph 0), then E (ph 1), -> bf16 A operand: 64 fp32 accumulator columns of this warp's half
+        // (Re for the first four warps, Im for the others), 16 at a time.  D1 and rho_1, which read S_0 from the
+        // same columns, are both done when D1 is.
 #pragma unroll 1
         for (int ph = 0; ph < 2; ++ph) {
             if (ph == 0) {
@@ -1024,17 +994,30 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
             }
             tc_fence_after();
             SFDA_T(13 + 2 * ph);
-            convert_acc(ph == 0 ? 1 + half : 0);
+            const bool sub_v = ph == 0 && half == 0;            // R_re = V - D1_re
+            const float sgn = ph == 0 ? -1.f : 1.f;             // R_im = -D1_im
+#pragma unroll 1
+            for (int pc = 0; pc < 4; ++pc) {
+                uint32_t r[16], pk[8];
+                tmem_ld<16>(tlane + TM_ACC + 128 * half + 16 * pc, r);
+                tc_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    float v0 = 0.f, v1 = 0.f;
+                    if (sub_v) {
+                        v0 = __uint_as_float((uint32_t)lds16(sv + (16 * pc + 2 * i) * 2 * DV) << 16);
+                        v1 = __uint_as_float((uint32_t)lds16(sv + (16 * pc + 2 * i + 1) * 2 * DV) << 16);
+                    }
+                    pk[i] = pack_bf16(fmaf(sgn, __uint_as_float(r[2 * i]), v0), fmaf(sgn, __uint_as_float(r[2 * i + 1]), v1));
+                }
+                tmem_st8(tlane + TM_X16 + 32 * half + 8 * pc, pk);
+            }
+            tc_wait_st();
             tc_fence_before();
             warp_arrive(&mi.bars[ph == 0 ? B_R16_READY : B_E16_READY]);
             SFDA_T(14 + 2 * ph);
         }
     }
-
-    // ---- the last unit's final state
-    if (!wait_k_warp(mi, B_UPD_DONE, n_chunks - 1)) return;
-    tc_fence_after();
-    write_out_state(n_chunks - 1, prev_ci);
 }
 
 // ---- the kernel ---------------------------------------------------------------------------------------
