@@ -684,22 +684,87 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
 }
 
 // ---- SOLVE --------------------------------------------------------------------------------------------
+// NRT stacked 16 x 8 tiles of a complex product A B, operands in the solve scratch (fp32, row stride LS, Re at
+// shared address `lx`, Im 64 rows further): tile rt covers rows a_row0 + 16 rt .. + 15 of A and k-steps
+// s0 <= s < s1[rt] (8 columns of A / rows of B per step; s1[0] <= s1[1]).  B's 8 columns start at b_col0.  Each
+// tile keeps four independent accumulators (Re: ar br and -ai bi; Im: ar bi and ai br), summed at the end, so
+// that consecutive tensor-core instructions do not wait for one another.
+template <int NRT>
+__device__ __forceinline__ void cmma_tiles(float (&cr)[NRT][4], float (&ci)[NRT][4], uint32_t lx, int a_row0, int a_col0,
+                                           int b_row0, int b_col0, int s0, int s1a, int s1b, int lane)
+{
+    constexpr uint32_t kIm = 64 * LS * 4;
+    const int g = lane >> 2, tg = lane & 3, m = lane >> 3, r = lane & 7;
+    float acc[NRT][4][4];
+#pragma unroll
+    for (int rt = 0; rt < NRT; ++rt)
+#pragma unroll
+        for (int x = 0; x < 4; ++x)
+#pragma unroll
+            for (int y = 0; y < 4; ++y) acc[rt][x][y] = 0.f;
+    // lane's row address for the A blocks: block m = (rows 0-7 | 8-15) x (k 0-3 | 4-7)
+    uint32_t a_addr = lx + (uint32_t)(((a_row0 + r + 8 * (m & 1)) * LS + a_col0 + 8 * s0 + 4 * (m >> 1)) * 4);
+    uint32_t b_addr = lx + (uint32_t)(((b_row0 + 8 * s0 + tg) * LS + b_col0 + g) * 4);
+#pragma unroll 2
+    for (int s = s0; s < s1b; ++s, a_addr += 32, b_addr += 8 * LS * 4) {
+        uint32_t br[2], bi[2], nbi[2];
+        br[0] = lds32(b_addr);
+        br[1] = lds32(b_addr + 4 * LS * 4);
+        bi[0] = lds32(b_addr + kIm);
+        bi[1] = lds32(b_addr + kIm + 4 * LS * 4);
+        nbi[0] = bi[0] ^ 0x80000000u;
+        nbi[1] = bi[1] ^ 0x80000000u;
+#pragma unroll
+        for (int rt = 0; rt < NRT; ++rt) {
+            if (NRT == 2 && rt == 0 && s >= s1a) continue;
+            uint32_t ar[4], ai[4];
+            ldmatrix_x4(ar, a_addr + rt * 16 * LS * 4);
+            ldmatrix_x4(ai, a_addr + rt * 16 * LS * 4 + kIm);
+            mma_tf32(acc[rt][0], ar, br);
+            mma_tf32(acc[rt][1], ai, nbi);
+            mma_tf32(acc[rt][2], ar, bi);
+            mma_tf32(acc[rt][3], ai, br);
+        }
+    }
+#pragma unroll
+    for (int rt = 0; rt < NRT; ++rt)
+#pragma unroll
+        for (int y = 0; y < 4; ++y) {
+            cr[rt][y] = acc[rt][0][y] + acc[rt][1][y];
+            ci[rt][y] = acc[rt][2][y] + acc[rt][3][y];
+        }
+}
+// Store a 16 x 8 accumulator tile (times `scale`) at rows row0.., columns col0.. of the scratch.
+__device__ __forceinline__ void store_tile_s(const float (&cr)[4], const float (&ci)[4], float scale, uint32_t lx, int row0,
+                                             int col0, int lane)
+{
+    constexpr uint32_t kIm = 64 * LS * 4;
+    const int g = lane >> 2, tg = lane & 3;
+    const uint32_t o = lx + (uint32_t)(((row0 + g) * LS + col0 + 2 * tg) * 4);
+    sts64(o, __float_as_uint(scale * cr[0]), __float_as_uint(scale * cr[1]));
+    sts64(o + 8 * LS * 4, __float_as_uint(scale * cr[2]), __float_as_uint(scale * cr[3]));
+    sts64(o + kIm, __float_as_uint(scale * ci[0]), __float_as_uint(scale * ci[1]));
+    sts64(o + kIm + 8 * LS * 4, __float_as_uint(scale * ci[2]), __float_as_uint(scale * ci[3]));
+}
+
 __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int n_chunks, int st)
 {
     long long *timing = p.timing;
     const int lane = st & 31, w = st >> 5;    // w = TMEM lane quadrant of this warp
-    float *Lr = reinterpret_cast<float *>(smem + OFF_LX), *Li = Lr + 64 * LS;
+    constexpr uint32_t kIm = 64 * LS * 4;     // Re -> Im in the scratch
+    const uint32_t sbase = smem_u32(smem), lx = sbase + OFF_LX;
     const uint32_t tlane = tmem + ((uint32_t)(w * 32) << 16);
     const int row = w * 32 + lane;            // Gram row held by this thread: < 64 -> Kt row, else Aq row
     bool dead = false;
     SFDA_TDECL(st == 0);
+#pragma unroll 1
     for (int j = 0; j < n_chunks; ++j) {
         if (role_sync_or(1, kSolveThreads, dead || mi.abort)) break;   // also: scratch of the last chunk is free
         const int s = j & 1, ring = j & 3;
         // The Aq tile of this slot also staged o_im of chunk j-2: its rows are written straight from the drain,
         // so the warps that hold them wait for that store first.
-        if (row >= 64 && j >= 2 && !dead && !wait_k(mi, s ? B_STORE_DONE1 : B_STORE_DONE0, (j >> 1) - 1)) dead = true;
-        // ---- drain the two Gram halves
+        if (row >= 64 && j >= 2 && !dead && !wait_k(mi, B_STORE_DONE0 + s, (j >> 1) - 1)) dead = true;
+        // ---- drain the two Gram halves (Re, then Im), 32 columns at a time
 #pragma unroll 1
         for (int im = 0; im < 2; ++im) {
             SFDA_T(20 + 2 * im);
@@ -707,7 +772,7 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
             tc_fence_after();
             SFDA_T(21 + 2 * im);
 #pragma unroll 1
-            for (int hc = 0; hc < 2; ++hc) {      // 32 columns at a time keeps the register footprint down
+            for (int hc = 0; hc < 2; ++hc) {
                 uint32_t r[32];
                 tmem_ld<32>(tlane + TM_GRAM + 32 * hc, r);
                 tc_wait_ld();
@@ -716,18 +781,19 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
                     warp_arrive(&mi.bars[B_GRAM_DRAINED]);
                 }
                 if (row < 64) {                   // L = D_beta Kt, strictly lower
-                    const int t = row;
-                    const float bt = mi.beta[ring][t];
-                    float4 *dst = reinterpret_cast<float4 *>((im ? Li : Lr) + t * LS + 32 * hc);
-#pragma unroll
+                    const float bt = mi.beta[ring][row];
+                    const uint32_t dst = lx + im * kIm + (uint32_t)((row * LS + 32 * hc) * 4);
                     // no mask: the substitution reads only entries below the diagonal of an 8x8 block and then
                     // overwrites the whole block; the merges read whole blocks strictly below the diagonal
+#pragma unroll
                     for (int i = 0; i < 32; i += 4)
-                        dst[i >> 2] = make_float4(bt * __uint_as_float(r[i]), bt * __uint_as_float(r[i + 1]),
-                                                  bt * __uint_as_float(r[i + 2]), bt * __uint_as_float(r[i + 3]));
+                        sts128(dst + 4 * i, __float_as_uint(bt * __uint_as_float(r[i])),
+                               __float_as_uint(bt * __uint_as_float(r[i + 1])),
+                               __float_as_uint(bt * __uint_as_float(r[i + 2])),
+                               __float_as_uint(bt * __uint_as_float(r[i + 3])));
                 } else {                          // Aq, lower incl. diagonal, as a bf16 operand tile
                     const int t = row - 64;
-                    uint8_t *tile = smem + OFF_AQ + (s * 2 + im) * kTile;
+                    const uint32_t tile = sbase + OFF_AQ + (s * 2 + im) * kTile;
 #pragma unroll
                     for (int c8 = 0; c8 < 4; ++c8) {
                         uint32_t wv[4];
@@ -737,13 +803,13 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
                             wv[x] = pack_bf16(ii <= t ? __uint_as_float(r[8 * c8 + 2 * x]) : 0.f,
                                               ii + 1 <= t ? __uint_as_float(r[8 * c8 + 2 * x + 1]) : 0.f);
                         }
-                        *reinterpret_cast<uint4 *>(tile + sw_off(t, 32 * hc + 8 * c8)) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+                        sts128(tile + sw_off(t, 32 * hc + 8 * c8), wv[0], wv[1], wv[2], wv[3]);
                     }
                 }
             }
         }
         fence_async_smem();
-        warp_arrive(&mi.bars[s ? B_AQ_FULL1 : B_AQ_FULL0]);
+        warp_arrive(&mi.bars[B_AQ_FULL0 + s]);
         role_sync(1, kSolveThreads);
         SFDA_T(24);
 
@@ -751,6 +817,7 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
         // (I + L) x = e_c right-looking (after x_i is final every later row is updated at once).
         if (w < 2) {
             const int o = 8 * (4 * w + (lane >> 3)), c = lane & 7;
+            const uint32_t blk = lx + (uint32_t)((o * LS + o) * 4);
             float xr[8], xi[8];
 #pragma unroll
             for (int r = 0; r < 8; ++r) {
@@ -762,7 +829,8 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
                 const float vr = xr[i], vi = xi[i];      // zero above the diagonal (i < c)
 #pragma unroll
                 for (int r = i + 1; r < 8; ++r) {
-                    const float lr_ = Lr[(o + r) * LS + o + i], li_ = Li[(o + r) * LS + o + i];
+                    const float lr_ = __uint_as_float(lds32(blk + (r * LS + i) * 4));
+                    const float li_ = __uint_as_float(lds32(blk + kIm + (r * LS + i) * 4));
                     xr[r] -= lr_ * vr - li_ * vi;
                     xi[r] -= lr_ * vi + li_ * vr;
                 }
@@ -770,65 +838,56 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
             __syncwarp();                     // every lane has read its L block before it is overwritten
 #pragma unroll
             for (int r = 0; r < 8; ++r) {
-                Lr[(o + r) * LS + o + c] = xr[r];
-                Li[(o + r) * LS + o + c] = xi[r];
+                sts32(blk + (r * LS + c) * 4, __float_as_uint(xr[r]));
+                sts32(blk + kIm + (r * LS + c) * 4, __float_as_uint(xi[r]));
             }
         }
         role_sync(1, kSolveThreads);
-        {   // level 0: 8 -> 16.  Warp w merges 16-block w: X21 = -X22 (L21 X11).  The m16 tile is placed on the
-            // whole 16-row block, so its lower eight rows (fragment elements 2, 3) are the rows that matter.
+        // ---- three merge levels: X[lower-left] = -X[lower-right] (L[lower-left] X[upper-left]); the intermediate
+        // product T is parked in the (unused) block above the diagonal
+        {   // level 0: 8 -> 16.  Warp w merges 16-block w.  The m16 tile is placed on the whole 16-row block, so
+            // its lower eight rows (fragment elements 2, 3) are the rows that matter.
             const int o = 16 * w;
-            float cr[4] = {0.f, 0.f, 0.f, 0.f}, ci[4] = {0.f, 0.f, 0.f, 0.f};
-            cmma_16x8(cr, ci, Lr, Li, LS, o, o, Lr, Li, LS, o, o, 0, 1, lane);           // rows 8..15: L21 X11
-            {   // T into the unused 8x8 block above the diagonal: rows o..o+7, columns o+8..o+15
-                const int g = lane >> 2, tg = lane & 3, at = (o + g) * LS + o + 8 + 2 * tg;
-                Lr[at] = cr[2]; Lr[at + 1] = cr[3];
-                Li[at] = ci[2]; Li[at + 1] = ci[3];
-            }
+            const int g = lane >> 2, tg = lane & 3;
+            float cr[1][4], ci[1][4];
+            cmma_tiles<1>(cr, ci, lx, o, o, o, o, 0, 1, 1, lane);               // rows 8..15: L21 X11
+            const uint32_t tpos = lx + (uint32_t)(((o + g) * LS + o + 8 + 2 * tg) * 4);   // rows o.., columns o+8..
+            sts64(tpos, __float_as_uint(cr[0][2]), __float_as_uint(cr[0][3]));
+            sts64(tpos + kIm, __float_as_uint(ci[0][2]), __float_as_uint(ci[0][3]));
             __syncwarp();
-            float dr[4] = {0.f, 0.f, 0.f, 0.f}, di[4] = {0.f, 0.f, 0.f, 0.f};
-            cmma_16x8(dr, di, Lr, Li, LS, o, o + 8, Lr, Li, LS, o, o + 8, 0, 1, lane);   // rows 8..15: X22 T
-            {
-                const int g = lane >> 2, tg = lane & 3, at = (o + 8 + g) * LS + o + 2 * tg;
-                Lr[at] = -dr[2]; Lr[at + 1] = -dr[3];
-                Li[at] = -di[2]; Li[at + 1] = -di[3];
-                // the block above the diagonal held T; later levels read the whole 16x16 diagonal block
-                const int zt = (o + g) * LS + o + 8 + 2 * tg;
-                __syncwarp();
-                Lr[zt] = 0.f; Lr[zt + 1] = 0.f;
-                Li[zt] = 0.f; Li[zt + 1] = 0.f;
-            }
+            cmma_tiles<1>(cr, ci, lx, o, o + 8, o, o + 8, 0, 1, 1, lane);       // rows 8..15: X22 T
+            const uint32_t xpos = lx + (uint32_t)(((o + 8 + g) * LS + o + 2 * tg) * 4);
+            sts64(xpos, __float_as_uint(-cr[0][2]), __float_as_uint(-cr[0][3]));
+            sts64(xpos + kIm, __float_as_uint(-ci[0][2]), __float_as_uint(-ci[0][3]));
+            // the block above the diagonal held T; later levels read the whole 16x16 diagonal block
+            __syncwarp();
+            sts64(tpos, 0u, 0u);
+            sts64(tpos + kIm, 0u, 0u);
         }
         role_sync(1, kSolveThreads);
         SFDA_T(25);
-        {   // level 1: X[b1][b0] = -X[b1][b1] (L[b1][b0] X[b0][b0]); T in the unused block above the diagonal
+        {   // level 1: 16 -> 32.  Warp pair pr merges 32-block pr; warp's column tile nt of the 16 columns
             const int pr = w >> 1, nt = w & 1;
             const int r0 = 32 * pr + 16, c0 = 32 * pr;
-            float cr[4] = {0.f, 0.f, 0.f, 0.f}, ci[4] = {0.f, 0.f, 0.f, 0.f};
-            cmma_16x8(cr, ci, Lr, Li, LS, r0, c0, Lr, Li, LS, c0, c0 + 8 * nt, nt, 2, lane);
-            store_tile(cr, ci, 1.f, Lr, Li, LS, c0, r0 + 8 * nt, lane);          // T at block (b0, b1)
+            float cr[1][4], ci[1][4];
+            cmma_tiles<1>(cr, ci, lx, r0, c0, c0, c0 + 8 * nt, nt, 2, 2, lane);
+            store_tile_s(cr[0], ci[0], 1.f, lx, c0, r0 + 8 * nt, lane);          // T at block (b0, b1)
             role_sync(1, kSolveThreads);
-            float dr[4] = {0.f, 0.f, 0.f, 0.f}, di[4] = {0.f, 0.f, 0.f, 0.f};
-            cmma_16x8(dr, di, Lr, Li, LS, r0, r0, Lr, Li, LS, c0, r0 + 8 * nt, 0, 2, lane);
-            store_tile(dr, di, -1.f, Lr, Li, LS, r0, c0 + 8 * nt, lane);
+            cmma_tiles<1>(cr, ci, lx, r0, r0, c0, r0 + 8 * nt, 0, 2, 2, lane);
+            store_tile_s(cr[0], ci[0], -1.f, lx, r0, c0 + 8 * nt, lane);
         }
         role_sync(1, kSolveThreads);
         SFDA_T(26);
-        {   // level 2: X[BL] = -X[BR] (L[BL] X[TL]); T in the top-right quadrant; warp w owns column tile w
+        {   // level 2: 32 -> 64.  T in the top-right quadrant; warp w owns column tile w of the 32 columns
             const int nt = w;
-            float c0r[4] = {0.f, 0.f, 0.f, 0.f}, c0i[4] = {0.f, 0.f, 0.f, 0.f};
-            float c1r[4] = {0.f, 0.f, 0.f, 0.f}, c1i[4] = {0.f, 0.f, 0.f, 0.f};
-            cmma_16x8(c0r, c0i, Lr, Li, LS, 32, 0, Lr, Li, LS, 0, 8 * nt, nt, 4, lane);
-            cmma_16x8(c1r, c1i, Lr, Li, LS, 48, 0, Lr, Li, LS, 0, 8 * nt, nt, 4, lane);
-            store_tile(c0r, c0i, 1.f, Lr, Li, LS, 0, 32 + 8 * nt, lane);
-            store_tile(c1r, c1i, 1.f, Lr, Li, LS, 16, 32 + 8 * nt, lane);
+            float cr[2][4], ci[2][4];
+            cmma_tiles<2>(cr, ci, lx, 32, 0, 0, 8 * nt, nt, 4, 4, lane);
+            store_tile_s(cr[0], ci[0], 1.f, lx, 0, 32 + 8 * nt, lane);
+            store_tile_s(cr[1], ci[1], 1.f, lx, 16, 32 + 8 * nt, lane);
             role_sync(1, kSolveThreads);
-            float d0r[4] = {0.f, 0.f, 0.f, 0.f}, d0i[4] = {0.f, 0.f, 0.f, 0.f};
-            float d1r[4] = {0.f, 0.f, 0.f, 0.f}, d1i[4] = {0.f, 0.f, 0.f, 0.f};
-            cmma_16x8(d0r, d0i, Lr, Li, LS, 32, 32, Lr, Li, LS, 0, 32 + 8 * nt, 0, 2, lane);
-            cmma_16x8(d1r, d1i, Lr, Li, LS, 48, 32, Lr, Li, LS, 0, 32 + 8 * nt, 0, 4, lane);
-            store_tile(d0r, d0i, -1.f, Lr, Li, LS, 32, 8 * nt, lane);
-            store_tile(d1r, d1i, -1.f, Lr, Li, LS, 48, 8 * nt, lane);
+            cmma_tiles<2>(cr, ci, lx, 32, 32, 0, 32 + 8 * nt, 0, 2, 4, lane);    // X22 lower triangular
+            store_tile_s(cr[0], ci[0], -1.f, lx, 32, 8 * nt, lane);
+            store_tile_s(cr[1], ci[1], -1.f, lx, 48, 8 * nt, lane);
         }
         role_sync(1, kSolveThreads);
         SFDA_T(27);
@@ -838,20 +897,27 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
         SFDA_T(28);
         {
             const int t = st >> 1, part = st & 1;   // row t, columns 32 part .. 32 part + 31
-#pragma unroll
+            const uint32_t src = lx + (uint32_t)((t * LS + 32 * part) * 4);
+            const uint32_t bsrc = smem_u32(&mi.beta[ring][32 * part]);
+#pragma unroll 1
             for (int cidx = 0; cidx < 4; ++cidx) {
                 uint32_t wr[4], wi[4];
 #pragma unroll
-                for (int x = 0; x < 4; ++x) {
-                    const int i0 = part * 32 + cidx * 8 + 2 * x;
-                    const float b0 = mi.beta[ring][i0], b1 = mi.beta[ring][i0 + 1];
-                    const bool in0 = i0 <= t, in1 = i0 + 1 <= t;
-                    wr[x] = pack_bf16(in0 ? Lr[t * LS + i0] * b0 : 0.f, in1 ? Lr[t * LS + i0 + 1] * b1 : 0.f);
-                    wi[x] = pack_bf16(in0 ? Li[t * LS + i0] * b0 : 0.f, in1 ? Li[t * LS + i0 + 1] * b1 : 0.f);
+                for (int hx = 0; hx < 2; ++hx) {
+                    const uint4 b4 = lds128(bsrc + (8 * cidx + 4 * hx) * 4);
+                    const uint4 r4 = lds128(src + (8 * cidx + 4 * hx) * 4);
+                    const uint4 i4 = lds128(src + kIm + (8 * cidx + 4 * hx) * 4);
+                    const int i0 = 32 * part + 8 * cidx + 4 * hx;
+                    const float m0 = i0 <= t ? __uint_as_float(b4.x) : 0.f, m1 = i0 + 1 <= t ? __uint_as_float(b4.y) : 0.f;
+                    const float m2 = i0 + 2 <= t ? __uint_as_float(b4.z) : 0.f, m3 = i0 + 3 <= t ? __uint_as_float(b4.w) : 0.f;
+                    wr[2 * hx] = pack_bf16(__uint_as_float(r4.x) * m0, __uint_as_float(r4.y) * m1);
+                    wr[2 * hx + 1] = pack_bf16(__uint_as_float(r4.z) * m2, __uint_as_float(r4.w) * m3);
+                    wi[2 * hx] = pack_bf16(__uint_as_float(i4.x) * m0, __uint_as_float(i4.y) * m1);
+                    wi[2 * hx + 1] = pack_bf16(__uint_as_float(i4.z) * m2, __uint_as_float(i4.w) * m3);
                 }
-                const int off = sw_off(t, part * 32 + cidx * 8);
-                *reinterpret_cast<uint4 *>(smem + OFF_MB + off) = make_uint4(wr[0], wr[1], wr[2], wr[3]);
-                *reinterpret_cast<uint4 *>(smem + OFF_MB + kTile + off) = make_uint4(wi[0], wi[1], wi[2], wi[3]);
+                const uint32_t off = sbase + OFF_MB + sw_off(t, 32 * part + 8 * cidx);
+                sts128(off, wr[0], wr[1], wr[2], wr[3]);
+                sts128(off + kTile, wi[0], wi[1], wi[2], wi[3]);
             }
         }
         fence_async_smem();

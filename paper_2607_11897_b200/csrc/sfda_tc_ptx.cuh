@@ -200,6 +200,31 @@ __device__ __forceinline__ void sts128(uint32_t saddr, uint32_t a, uint32_t b, u
 {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
+__device__ __forceinline__ void sts64(uint32_t saddr, uint32_t a, uint32_t b)
+{
+    asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(saddr), "r"(a), "r"(b) : "memory");
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t saddr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(saddr));
+    return v;
+}
+__device__ __forceinline__ uint4 lds128(uint32_t saddr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr));
+    return v;
+}
+// Four 8 x 8 matrices of 16-bit elements = four 8-row x 4-column blocks of 32-bit elements: lane l supplies the
+// 16-byte row address of row l % 8 of block l / 8; thread T receives element (T / 4, T % 4) of every block, which
+// is the A-fragment layout of the m16n8k8 tf32 MMA when the blocks are (rows 0-7 | rows 8-15) x (k 0-3 | k 4-7).
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t saddr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(saddr));
+}
 // Global loads through the read-only path that only happen when `on` is set (the destination keeps its value
 // otherwise): no branch, so neighbouring work can be scheduled across them.
 __device__ __forceinline__ void ldg64_if(uint32_t &x, uint32_t &y, const void *ptr, bool on)
