@@ -504,6 +504,14 @@ __device__ __forceinline__ void turns_sincos(uint32_t turns, float *sn, float *c
     __sincosf(f * 6.283185307f, sn, cs);
 }
 
+// Phase in 2^-32 turns from fp32 arithmetic (one multiply, one conversion).  Inside this kernel the phase only
+// feeds sines and cosines of bf16 operands, so the product's fp32 rounding (2^-24 of the angle) is far below what
+// matters; the exact double-precision conversion is kept where phases are exported.
+__device__ __forceinline__ uint32_t turns_f32(float theta)
+{
+    return (uint32_t)(unsigned long long)__float2ll_rn(theta * 683565275.6f);
+}
+
 __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int n_chunks, int pt)
 {
     long long *timing = p.timing;
@@ -543,7 +551,8 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
         if (role_sync_or(2, kPrepThreads, dead || mi.abort)) break;
         const bool live = j < n_chunks;          // after the last chunk only the outputs of two chunks are left
         const int s = j & 1, ring = j & 3;
-        float base0 = 1.f, base1 = 1.f;
+        float base0 = 1.f, base1 = 1.f, ainv0 = 1.f, ainv1 = 1.f;
+        float2 g0 = make_float2(1.f, 0.f), g1 = g0;   // gamma_t = a_t e^{i phi_t} of the two coordinates
         uint32_t tb0 = 0u, tb1 = 0u;
         size_t off = 0, step = 0;                // byte offset of this thread's first token in q/k/alpha/theta
         int nt = 0;                              // real tokens in this thread's octet
@@ -593,8 +602,8 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
                 for (int i = 0; i < 8; ++i) {
                     a0 *= fmaxf(al[i].x, 9.0e-14f);           // floor e^-30, as in log_decay
                     a1 *= fmaxf(al[i].y, 9.0e-14f);
-                    u0 += phase_to_turns(th[i].x);
-                    u1 += phase_to_turns(th[i].y);
+                    u0 += turns_f32(th[i].x);
+                    u1 += turns_f32(th[i].y);
                 }
                 *reinterpret_cast<float2 *>(&mi.part_lg[tq][2 * jp]) = make_float2(a0, a1);
                 *reinterpret_cast<uint2 *>(&mi.part_turns[tq][2 * jp]) = make_uint2(u0, u1);
@@ -613,13 +622,19 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
                 const uint2 pu = *reinterpret_cast<const uint2 *>(&mi.part_turns[gq][2 * jp]);
                 base0 *= pl.x; base1 *= pl.y; tb0 += pu.x; tb1 += pu.y;
             }
-            if (tq == 0) {
+            {   // gamma at the start of the group (group 0: of the whole chunk, for the next state pass)
                 float cs, sn;
                 turns_sincos(tb0, &sn, &cs);
-                mi.close[ring][2 * jp] = make_float2(base0 * cs, base0 * sn);
+                g0 = make_float2(base0 * cs, base0 * sn);
                 turns_sincos(tb1, &sn, &cs);
-                mi.close[ring][2 * jp + 1] = make_float2(base1 * cs, base1 * sn);
-                base0 = 1.f; base1 = 1.f; tb0 = 0u; tb1 = 0u;
+                g1 = make_float2(base1 * cs, base1 * sn);
+                if (tq == 0) {
+                    mi.close[ring][2 * jp] = g0;
+                    mi.close[ring][2 * jp + 1] = g1;
+                    g0 = make_float2(1.f, 0.f); g1 = g0; base0 = 1.f; base1 = 1.f;
+                }
+                ainv0 = fminf(__fdividef(1.0f, base0), 5.5e34f);          // 1/a, capped at e^80
+                ainv1 = fminf(__fdividef(1.0f, base1), 5.5e34f);
             }
             SFDA_T(31);
 
@@ -646,26 +661,24 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
 #pragma unroll
             for (int ii = 0; ii < kTB; ++ii) {
                 const int i = h * kTB + ii;
-                base0 *= fmaxf(__uint_as_float(tk[ii].al.x), 9.0e-14f);                  // a_t, phase of token t
-                base1 *= fmaxf(__uint_as_float(tk[ii].al.y), 9.0e-14f);
-                tb0 += phase_to_turns(__uint_as_float(tk[ii].th.x));
-                tb1 += phase_to_turns(__uint_as_float(tk[ii].th.y));
                 float wr[2], wi[2], cr_[2], ci_[2], qr_[2], qi_[2];
 #pragma unroll
                 for (int x = 0; x < 2; ++x) {
-                    const float a = x ? base1 : base0;
-                    const uint32_t tu = x ? tb1 : tb0;
-                    const uint32_t kx = x ? tk[ii].k.y : tk[ii].k.x, qx = x ? tk[ii].q.y : tk[ii].q.x;
-                    const float ainv = fminf(__fdividef(1.0f, a), 5.5e34f);              // 1/a_t, capped at e^80
+                    // gamma_t = gamma_{t-1} alpha_t e^{i theta_t}; 1/a_t alongside (capped at e^80)
+                    const float al = fmaxf(__uint_as_float(x ? tk[ii].al.y : tk[ii].al.x), 9.0e-14f);   // floor e^-30
                     float cs, sn;
-                    turns_sincos(tu, &sn, &cs);
+                    __sincosf(__uint_as_float(x ? tk[ii].th.y : tk[ii].th.x), &sn, &cs);
+                    float2 &g = x ? g1 : g0;
+                    float &ainv = x ? ainv1 : ainv0;
+                    const float lr_ = al * cs, li_ = al * sn;
+                    g = make_float2(g.x * lr_ - g.y * li_, g.x * li_ + g.y * lr_);
+                    ainv = fminf(ainv * __fdividef(1.0f, al), 5.5e34f);
+                    const uint32_t kx = x ? tk[ii].k.y : tk[ii].k.x, qx = x ? tk[ii].q.y : tk[ii].q.x;
                     const float kr = __uint_as_float(kx << 16), ki = __uint_as_float(kx & 0xffff0000u);
                     const float qr = __uint_as_float(qx << 16), qi = __uint_as_float(qx & 0xffff0000u);
-                    const float kpr = kr * cs + ki * sn, kpi = ki * cs - kr * sn;   // e^{-i phi} k
-                    const float qpr = qr * cs + qi * sn, qpi = qi * cs - qr * sn;
-                    wr[x] = a * kpr; wi[x] = a * kpi;
-                    qr_[x] = a * qpr; qi_[x] = a * qpi;
-                    cr_[x] = ainv * kpr; ci_[x] = ainv * kpi;
+                    wr[x] = g.x * kr + g.y * ki; wi[x] = g.x * ki - g.y * kr;          // W = conj(gamma) k
+                    qr_[x] = g.x * qr + g.y * qi; qi_[x] = g.x * qi - g.y * qr;        // Qt = conj(gamma) q
+                    cr_[x] = (wr[x] * ainv) * ainv; ci_[x] = (wi[x] * ainv) * ainv;    // Kc = k / gamma = W / a^2
                 }
                 load_token(tk[ii], i + kTB);
                 const int o1 = i * 128 + ((((jp >> 2) ^ i) & 7) << 4);      // row i of the octet's 8-row swizzle atom
