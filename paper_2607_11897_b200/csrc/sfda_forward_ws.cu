@@ -58,7 +58,7 @@ constexpr int OFF_OST = OFF_V + 16384;            // o staging [t][128] bf16 (TM
 constexpr int LS = 68;                            // row stride (floats) of the solve scratch
 constexpr int OFF_LX = OFF_OST + 16384;           // L -> X in place, fp32 [64][LS], re | im               34 KB
 constexpr int OFF_MISC = OFF_LX + 2 * 64 * LS * 4;
-constexpr int kMiscBytes = 9216;
+constexpr int kMiscBytes = 13312;
 constexpr int kSmemBytes = OFF_MISC + kMiscBytes + 1024;   // + slack for the 1024-byte alignment
 static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA exceeded");
 
@@ -76,8 +76,8 @@ enum Bar {
 };
 
 struct Misc {
-    float part_lg[8][M];
-    uint32_t part_turns[8][M];
+    float part_lg[2][8][M];                 // per-group partial products / phase sums, two chunks deep
+    uint32_t part_turns[2][8][M];
     float2 close[4][M];                     // a_C e^{i phi_C} of a ring of four chunks
     float beta[4][C];
     unsigned long long bars[kNumBars];
@@ -121,6 +121,7 @@ struct Params {
     float *handoff;      // [B*H][d_k][d_v] boundary states between time slices (only used when Q > 1)
     int T, H, has_o_im;
     int BH, U, Q, n_units;   // sequences, chunks per work unit, time slices per sequence, Q * BH
+    uint32_t magic_BH, magic_H;   // floor(2^32 / d) + 1 (0 for d = 1): quotients by multiplication
 };
 
 // Work units.  A sequence is cut into Q time slices of U chunks; unit u = slice * BH + sequence.  CTA c works
@@ -137,11 +138,13 @@ struct ChunkInfo {
 struct ChunkCursor {
     ChunkInfo ci;
     int jl, u;
+    // n / d for n * d < 2^32 from the precomputed floor(2^32 / d) + 1 (d = 1 is flagged by 0)
+    static __device__ __forceinline__ int quot(int n, uint32_t magic) { return magic ? (int)__umulhi((uint32_t)n, magic) : n; }
     __device__ __forceinline__ void set_unit(const Params &p)
     {
-        ci.q = u / p.BH;
+        ci.q = quot(u, p.magic_BH);
         ci.bh = u - ci.q * p.BH;
-        ci.b = ci.bh / p.H;
+        ci.b = quot(ci.bh, p.magic_H);
         ci.h = ci.bh - ci.b * p.H;
     }
     __device__ __forceinline__ void refresh(const Params &p)
@@ -165,20 +168,6 @@ struct ChunkCursor {
         refresh(p);
     }
 };
-__device__ __forceinline__ ChunkInfo chunk_info(const Params &p, int jj)
-{
-    const int ul = jj / p.U, jl = jj - ul * p.U;
-    const int u = (int)blockIdx.x + ul * (int)gridDim.x;
-    ChunkInfo ci;
-    ci.q = u / p.BH;
-    ci.bh = u - ci.q * p.BH;
-    ci.b = ci.bh / p.H;
-    ci.h = ci.bh - ci.b * p.H;
-    ci.jg = ci.q * p.U + jl;
-    ci.first = jl == 0;
-    ci.last = jl == p.U - 1;
-    return ci;
-}
 
 __device__ __forceinline__ void mbar_arrive(unsigned long long *bar)
 {
@@ -287,34 +276,24 @@ __device__ __forceinline__ bool test_k_warp(Misc &mi, int bar, int k)
 // the accumulators start from zero.  `b_step`: descriptor advance of B per K = 16 (2 for a K-major tile,
 // 128 for an MN-major one).  The state update uses the same products with conj(E)-side roles swapped, which
 // `swap` selects: Re += x_re b_re, Re -= x_im b_im, Im += x_re b_im, Im += x_im b_re.
-template <bool kTmemA>
-__device__ __forceinline__ void issue_complex(uint32_t d_re, uint32_t d_im, uint32_t a_re, uint32_t a_im,
-                                              uint32_t b_re, uint32_t b_im, uint32_t dhi, uint32_t id, int neg_g,
-                                              bool fresh, bool swap, uint32_t b_step)
+template <int kNegG, bool kFresh, bool kSwap, uint32_t kBStep>
+__device__ __forceinline__ void issue_complex(uint32_t d_re, uint32_t d_im, uint32_t a_re, uint32_t a_im, uint32_t b_re,
+                                              uint32_t b_im, uint32_t dhi, uint32_t id)
 {
-#pragma unroll 1
-    for (int g = 0; g < 4; ++g) {
-        const bool odd = g & 1, mid = g == 1 || g == 2;
-        const uint32_t d = g < 2 ? d_re : d_im;
-        const uint32_t a = (swap ? odd : mid) ? a_im : a_re;
-        const uint32_t b = (swap ? mid : odd) ? b_im : b_re;
-        const uint32_t idg = id | (g == neg_g ? 1u << 14 : 0u);
-        const uint32_t acc0 = (!fresh || odd) ? 1u : 0u;
-        if (elect_one()) {
-            if (kTmemA) {
-                mma_ts2(d, a, b, dhi, idg, acc0);
-                mma_ts2(d, a + 8, b + b_step, dhi, idg, 1u);
-                mma_ts2(d, a + 16, b + 2 * b_step, dhi, idg, 1u);
-                mma_ts2(d, a + 24, b + 3 * b_step, dhi, idg, 1u);
-            } else {
-                mma_ss2(d, a, dhi, b, dhi, idg, acc0);
-                mma_ss2(d, a + 2, dhi, b + 2, dhi, idg, 1u);
-                mma_ss2(d, a + 4, dhi, b + 4, dhi, idg, 1u);
-                mma_ss2(d, a + 6, dhi, b + 6, dhi, idg, 1u);
-            }
+    if (elect_one()) {
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const bool odd = g & 1, mid = g == 1 || g == 2;
+            const uint32_t d = g < 2 ? d_re : d_im;
+            const uint32_t a = (kSwap ? odd : mid) ? a_im : a_re;
+            const uint32_t b = (kSwap ? mid : odd) ? b_im : b_re;
+            const uint32_t idg = id | (g == kNegG ? 1u << 14 : 0u);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+                mma_ts2(d, a + 8 * ks, b + kBStep * ks, dhi, idg, (!kFresh || odd || ks > 0) ? 1u : 0u);
         }
-        __syncwarp();
     }
+    __syncwarp();
 }
 
 // The issuing work is split over three warps (they sit on different schedulers):
@@ -347,7 +326,7 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
             if (j > 0 && !wait_k_warp(mi, B_O_STAGED, j - 1)) return;
             tc_fence_after();
             SFDA_T(0);
-            issue_complex<true>(acc, acc + 128, x_re, x_re + 32, w_re, w_re + 2 * kIm, dhi, I128, 3, true, false, 2);
+            issue_complex<3, true, false, 2>(acc, acc + 128, x_re, x_re + 32, w_re, w_re + 2 * kIm, dhi, I128);
             if (elect_one()) {
                 mma_commit(&bars[B_D1_DONE]);
                 mma_commit(&bars[B_WQ_FREE0 + s]);
@@ -359,14 +338,14 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
             if (!wait_k_warp(mi, B_MB_FULL, j)) return;
             tc_fence_after();
             SFDA_T(3);
-            issue_complex<true>(acc, acc + 128, x_re, x_re + 32, m_re, m_re + kIm, dhi, I64, 1, true, false, 2);
+            issue_complex<1, true, false, 2>(acc, acc + 128, x_re, x_re + 32, m_re, m_re + kIm, dhi, I64);
             if (elect_one()) mma_commit(&bars[B_E_DONE]);
             SFDA_T(4);
             // S += E^T Kc (Kc as MN-major B: rows = tokens)
             if (!wait_k_warp(mi, B_E16_READY, j)) return;
             tc_fence_after();
             SFDA_T(5);
-            issue_complex<true>(tmem + TM_S32, tmem + TM_S32 + 64, x_re, x_re + 32, k_re, k_re + kIm, dhi, I64M, 1, false, true, 128);
+            issue_complex<1, false, true, 128>(tmem + TM_S32, tmem + TM_S32 + 64, x_re, x_re + 32, k_re, k_re + kIm, dhi, I64M);
             if (elect_one()) {
                 mma_commit(&bars[B_KC_FREE0 + s]);
                 mma_commit(&bars[B_UPD_DONE]);
@@ -401,7 +380,7 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
             if (!wait_k_warp(mi, B_AQ_FULL0 + (j & 1), j >> 1)) return;
             tc_fence_after();
             const uint32_t a_re = dlo + ((OFF_AQ + (j & 1) * 2 * kTile) >> 4);
-            issue_complex<true>(acc + 64, acc + 192, x_re, x_re + 32, a_re, a_re + kIm, dhi, I64, 1, false, false, 2);
+            issue_complex<1, false, false, 2>(acc + 64, acc + 192, x_re, x_re + 32, a_re, a_re + kIm, dhi, I64);
             if (elect_one()) mma_commit(&bars[B_UPD_DONE]);
         }
     } else {
@@ -548,7 +527,6 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
     ChunkCursor cur(p);
 #pragma unroll 1
     for (int j = 0; j < n_chunks + 2; ++j) {
-        if (role_sync_or(2, kPrepThreads, dead || mi.abort)) break;
         const bool live = j < n_chunks;          // after the last chunk only the outputs of two chunks are left
         const int s = j & 1, ring = j & 3;
         float base0 = 1.f, base1 = 1.f, ainv0 = 1.f, ainv1 = 1.f;
@@ -605,21 +583,23 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
                     u0 += turns_f32(th[i].x);
                     u1 += turns_f32(th[i].y);
                 }
-                *reinterpret_cast<float2 *>(&mi.part_lg[tq][2 * jp]) = make_float2(a0, a1);
-                *reinterpret_cast<uint2 *>(&mi.part_turns[tq][2 * jp]) = make_uint2(u0, u1);
+                *reinterpret_cast<float2 *>(&mi.part_lg[s][tq][2 * jp]) = make_float2(a0, a1);
+                *reinterpret_cast<uint2 *>(&mi.part_turns[s][tq][2 * jp]) = make_uint2(u0, u1);
             }
             if (pt < C) mi.beta[ring][pt] = beta_t;
             SFDA_T(30);
 #pragma unroll
             for (int ii = 0; ii < kTB; ++ii) load_token(tk[ii], ii);
-            role_sync(2, kPrepThreads);
+            // The only barrier of the role.  The partial sums are kept two chunks deep: a warp that runs ahead
+            // writes the other copy, and cannot come back to this one before everybody has passed the next barrier.
+            if (role_sync_or(2, kPrepThreads, dead || mi.abort)) break;
             // octet tq starts from the product of the octets before it; octet 0 instead multiplies all eight:
             // the chunk totals a_C e^{i phi_C}, applied by the next state pass
             const int n_before = tq == 0 ? 8 : tq;
 #pragma unroll 1
             for (int gq = 0; gq < n_before; ++gq) {
-                const float2 pl = *reinterpret_cast<const float2 *>(&mi.part_lg[gq][2 * jp]);
-                const uint2 pu = *reinterpret_cast<const uint2 *>(&mi.part_turns[gq][2 * jp]);
+                const float2 pl = *reinterpret_cast<const float2 *>(&mi.part_lg[s][gq][2 * jp]);
+                const uint2 pu = *reinterpret_cast<const uint2 *>(&mi.part_turns[s][gq][2 * jp]);
                 base0 *= pl.x; base1 *= pl.y; tb0 += pu.x; tb1 += pu.y;
             }
             {   // gamma at the start of the group (group 0: of the whole chunk, for the next state pass)
@@ -1254,7 +1234,11 @@ cudaError_t read_static_status(cudaStream_t stream, uint32_t *word)
     return cudaStreamSynchronize(stream);
 }
 
-bool forward_ws_supported(const ForwardArgs &a) { return a.dtype == 1 && a.d_k == DK && a.d_v == DV && a.chunk == C; }
+// (B * H is bounded so that the unit cursor's quotients by multiplication stay exact.)
+bool forward_ws_supported(const ForwardArgs &a)
+{
+    return a.dtype == 1 && a.d_k == DK && a.d_v == DV && a.chunk == C && (long long)a.B * a.H <= 16384;
+}
 
 // Scratch layout: [0, 256) status word; then, when the block is large enough for time slicing,
 // [256, 256 + round256(4 BH)) slice counters and BH boundary states of d_k x d_v floats.
@@ -1317,6 +1301,8 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
     p.Q = Q;
     p.U = NC / Q;
     p.n_units = BH * Q;
+    p.magic_BH = BH > 1 ? (uint32_t)(0x100000000ull / (unsigned)BH) + 1u : 0u;
+    p.magic_H = a.H > 1 ? (uint32_t)(0x100000000ull / (unsigned)a.H) + 1u : 0u;
     g_ws_last_slices = Q;
     const unsigned grid = (unsigned)(p.n_units < n_sm ? p.n_units : n_sm);
     sfda_forward_ws_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tv, to, toi, p);
