@@ -240,6 +240,13 @@ def main():
             e1.record(stream)
         stop.record(stream)
         barrier()
+        # The timed region lasts tens of milliseconds, too short for nvidia-smi to see: the same launches go on,
+        # untimed, under the sampler until it has had about a second of this load.
+        t_load = time.perf_counter()
+        while time.perf_counter() - t_load < 1.0:
+            for _ in range(20):
+                step()
+            torch.cuda.synchronize()
     total_ms = start.elapsed_time(stop)
     kernel_ms = [e0.elapsed_time(e1) for e0, e1 in events]      # one forward = one launch of the chunk kernel
     total_ms = dp.max_over_ranks(total_ms, dev)

@@ -509,14 +509,19 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
         if (half == 0 || p.has_o_im) {
             __nv_bfloat16 *stage =
                 reinterpret_cast<__nv_bfloat16 *>(smem + (half ? OFF_AQ + (jd & 1) * 2 * kTile : OFF_OST)) + c;
-            const float sgn = half ? -1.f : 1.f;   // o = conj(rho)
+            const uint32_t flip = half ? 0x80008000u : 0u;   // o = conj(rho)
+            const uint32_t st = smem_u32(stage);
 #pragma unroll 1
-            for (int pc = 0; pc < 4; ++pc) {
-                uint32_t r[16];
-                tmem_ld<16>(tlane + TM_ACC + 64 + 128 * half + 16 * pc, r);
+            for (int pc = 0; pc < 2; ++pc) {
+                uint32_t r[32];
+                tmem_ld<32>(tlane + TM_ACC + 64 + 128 * half + 32 * pc, r);
                 tc_wait_ld();
 #pragma unroll
-                for (int t = 0; t < 16; ++t) stage[(16 * pc + t) * DV] = __float2bfloat16_rn(sgn * __uint_as_float(r[t]));
+                for (int t = 0; t < 32; t += 2) {
+                    const uint32_t pk = pack_bf16(__uint_as_float(r[t]), __uint_as_float(r[t + 1])) ^ flip;
+                    sts16(st + (32 * pc + t) * 2 * DV, (uint16_t)pk);
+                    sts16(st + (32 * pc + t + 1) * 2 * DV, (uint16_t)(pk >> 16));
+                }
             }
         }
         fence_async_smem();
@@ -534,10 +539,12 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
         uint32_t tb0 = 0u, tb1 = 0u;
         size_t off = 0, step = 0;                // byte offset of this thread's first token in q/k/alpha/theta
         int nt = 0;                              // real tokens in this thread's octet
-        struct Tok { uint2 al, th, k, q; } tk[kTB];   // alpha and theta as raw bits
-        auto load_token = [&](Tok &t, int i) {   // inputs of token i of the octet; neutral beyond the sequence
-            t.al = make_uint2(0x3f800000u, 0x3f800000u); t.th = make_uint2(0u, 0u);
-            t.k = make_uint2(0u, 0u); t.q = make_uint2(0u, 0u);
+        // Inputs of token i of the octet, alpha and theta as raw bits.  Beyond the end of the sequence nothing is
+        // loaded and the registers keep what they held (neutral values at first, then an earlier token's): such
+        // tokens have beta = 0 and stored-nowhere outputs, so any finite operand rows do for them; the chunk's
+        // closing factor comes from pass 1, which does count them as neutral.
+        struct Tok { uint2 al, th, k, q; } tk[kTB];
+        auto load_token = [&](Tok &t, int i) {
             const size_t o = off + (size_t)i * step;
             const bool on = i < nt;
             ldg64_if(t.al.x, t.al.y, reinterpret_cast<const char *>(p.alpha) + o, on);
@@ -545,6 +552,11 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
             ldg64_if(t.k.x, t.k.y, reinterpret_cast<const char *>(p.k) + o, on);
             ldg64_if(t.q.x, t.q.y, reinterpret_cast<const char *>(p.q) + o, on);
         };
+#pragma unroll
+        for (int ii = 0; ii < kTB; ++ii) {
+            tk[ii].al = make_uint2(0x3f800000u, 0x3f800000u); tk[ii].th = make_uint2(0u, 0u);
+            tk[ii].k = make_uint2(0u, 0u); tk[ii].q = make_uint2(0u, 0u);
+        }
         if (live) {
             const ChunkInfo ci = cur.ci;
             cur.next(p);
