@@ -69,7 +69,7 @@ enum Bar {
     B_STORE_DONE0, B_STORE_DONE1,   // CTRL: the output store of a chunk of this parity has read its staging
     B_GRAM_FULL, B_GRAM_DRAINED,    // commit / SOLVE: one Gram half is in tensor memory / has been read out
     B_MB_FULL, B_AQ_FULL0, B_AQ_FULL1,
-    B_D1_DONE, B_E_DONE, B_UPD_DONE,
+    B_D1_DONE, B_O1_DONE, B_E_DONE, B_UPD_DONE,
     B_S16_READY, B_R16_READY, B_E16_READY, B_O_STAGED,
     B_V_FULL,
     kNumBars
@@ -319,16 +319,19 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
         for (int j = 0; j < n_chunks; ++j) {
             const int s = j & 1, u = j >> 1;
             const uint32_t w_re = dlo + ((OFF_WQ + s * 4 * kTile) >> 4), k_re = dlo + ((OFF_KC + s * 2 * kTile) >> 4);
-            // [D1 | rho_1] = [W ; Qt]^* S_0: N = 128 over the slot's 128-row tiles; rho of the previous chunk must
-            // have been read out
+            // D1 = W^* S_0 as soon as S_0 is there; rho_1 = Qt^* S_0 (the Qt rows follow the W rows in the slot's
+            // tiles) once rho of the previous chunk has been read out.  Both read S_0 from the operand columns.
             if (!wait_k_warp(mi, B_S16_READY, j)) return;
             if (!wait_k_warp(mi, B_PREP_FULL0 + s, u)) return;
-            if (j > 0 && !wait_k_warp(mi, B_O_STAGED, j - 1)) return;
             tc_fence_after();
             SFDA_T(0);
-            issue_complex<3, true, false, 2>(acc, acc + 128, x_re, x_re + 32, w_re, w_re + 2 * kIm, dhi, I128);
+            issue_complex<3, true, false, 2>(acc, acc + 128, x_re, x_re + 32, w_re, w_re + 2 * kIm, dhi, I64);
+            if (elect_one()) mma_commit(&bars[B_D1_DONE]);
+            if (j > 0 && !wait_k_warp(mi, B_O_STAGED, j - 1)) return;
+            tc_fence_after();
+            issue_complex<3, true, false, 2>(acc + 64, acc + 192, x_re, x_re + 32, w_re + kIm, w_re + 3 * kIm, dhi, I64);
             if (elect_one()) {
-                mma_commit(&bars[B_D1_DONE]);
+                mma_commit(&bars[B_O1_DONE]);
                 mma_commit(&bars[B_WQ_FREE0 + s]);
             }
             SFDA_T(1);
@@ -1081,6 +1084,8 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
                     }
                     pk[i] = pack_bf16(fmaf(sgn, __uint_as_float(r[2 * i]), v0), fmaf(sgn, __uint_as_float(r[2 * i + 1]), v1));
                 }
+                // R replaces S_0 in the operand columns: rho_1, the last reader of S_0, must be done
+                if (ph == 0 && pc == 0 && !wait_k_warp(mi, B_O1_DONE, j)) return;
                 tmem_st8(tlane + TM_X16 + 32 * half + 8 * pc, pk);
             }
             tc_wait_st();
@@ -1114,7 +1119,7 @@ sfda_forward_ws_kernel(const __grid_constant__ CUtensorMap tm_v, const __grid_co
         init(B_STORE_DONE0, 1); init(B_STORE_DONE1, 1);
         init(B_GRAM_FULL, 1); init(B_GRAM_DRAINED, kSolveWarps);
         init(B_MB_FULL, kSolveWarps); init(B_AQ_FULL0, kSolveWarps); init(B_AQ_FULL1, kSolveWarps);
-        init(B_D1_DONE, 1); init(B_E_DONE, 1); init(B_UPD_DONE, 2);   // state update and rho += Aq E
+        init(B_D1_DONE, 1); init(B_O1_DONE, 1); init(B_E_DONE, 1); init(B_UPD_DONE, 2);   // state update and rho += Aq E
         init(B_S16_READY, kChainWarps); init(B_R16_READY, kChainWarps); init(B_E16_READY, kChainWarps);
         init(B_O_STAGED, kPrepWarps); init(B_V_FULL, 1);
         mi.abort = 0;
