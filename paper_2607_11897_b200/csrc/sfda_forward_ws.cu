@@ -387,45 +387,15 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
             if (elect_one()) mma_commit(&bars[B_UPD_DONE]);
         }
     } else {
-        // Gram chunk g, half gh, as soon as its operands are written and the Gram columns have been drained;
-        // v of chunk jv as soon as v of chunk jv-1 has been consumed (R of that chunk is built).
+        // Per chunk g, in the order in which the events normally happen: v of chunk g once v of chunk g-1 has been
+        // consumed (R of that chunk is built); then the two Gram halves of chunk g, each once its operands are
+        // written and the Gram columns have been read out.  Blocking waits: a polling loop here would take issue
+        // slots from the warps that do the work.
         ChunkCursor vcur(p);
-        int g = 0, gh = 0, jv = 0;
-        uint32_t t0 = (uint32_t)clock();
 #pragma unroll 1
-        while (g < n_chunks || jv < n_chunks) {
-            bool progress = false;
-            if (g < n_chunks) {
-                const bool ready = gh == 0 ? test_k_warp(mi, B_PREP_FULL0 + (g & 1), g >> 1) &&
-                                                 (g == 0 || test_k_warp(mi, B_GRAM_DRAINED, 2 * g - 1))
-                                           : test_k_warp(mi, B_GRAM_DRAINED, 2 * g);
-                if (ready) {
-                    const int s = g & 1;
-                    const uint32_t w_re = dlo + ((OFF_WQ + s * 4 * kTile) >> 4), k_re = dlo + ((OFF_KC + s * 2 * kTile) >> 4);
-                    const uint32_t k_b = gh ? k_re + kIm : k_re;
-                    tc_fence_after();
-                    // rows = [W ; Qt], columns = tokens i.  Re: W_re Kc_re + W_im Kc_im; Im: W_re Kc_im - W_im Kc_re
-                    if (elect_one()) {
-                        const uint32_t d = tmem + TM_GRAM, w_a = w_re, w_im = w_re + 2 * kIm;
-                        const uint32_t k2 = gh ? k_re : k_re + kIm;      // partner of the second product
-                        const uint32_t id2 = gh ? I64 | (1u << 14) : I64;
-                        mma_ss2(d, w_a, dhi, k_b, dhi, I64, 0u);
-                        mma_ss2(d, w_a + 2, dhi, k_b + 2, dhi, I64, 1u);
-                        mma_ss2(d, w_a + 4, dhi, k_b + 4, dhi, I64, 1u);
-                        mma_ss2(d, w_a + 6, dhi, k_b + 6, dhi, I64, 1u);
-                        mma_ss2(d, w_im, dhi, k2, dhi, id2, 1u);
-                        mma_ss2(d, w_im + 2, dhi, k2 + 2, dhi, id2, 1u);
-                        mma_ss2(d, w_im + 4, dhi, k2 + 4, dhi, id2, 1u);
-                        mma_ss2(d, w_im + 6, dhi, k2 + 6, dhi, id2, 1u);
-                        mma_commit(&bars[B_GRAM_FULL]);
-                    }
-                    __syncwarp();
-                    g += gh;
-                    gh ^= 1;
-                    progress = true;
-                }
-            }
-            if (jv < n_chunks && (jv == 0 || test_k_warp(mi, B_R16_READY, jv - 1))) {
+        for (int g = 0; g < n_chunks; ++g) {
+            if (g > 0 && !wait_k_warp(mi, B_R16_READY, g - 1)) return;
+            {
                 const ChunkInfo cv = vcur.ci;
                 vcur.next(p);
                 if (elect_one()) {
@@ -433,17 +403,26 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
                     tma_load_4d(smem + OFF_V, tm_v, &bars[B_V_FULL], 0, cv.h, cv.jg * C, cv.b);
                 }
                 __syncwarp();
-                ++jv;
-                progress = true;
             }
-            if (progress) {
-                t0 = (uint32_t)clock();
-            } else {
-                __nanosleep(64);
-                if (mi.abort || (uint32_t)clock() - t0 > 0x80000000u) {      // a second without progress
-                    mi.abort = 1;
-                    return;
+            const int s = g & 1;
+            const uint32_t w_re = dlo + ((OFF_WQ + s * 4 * kTile) >> 4), k_re = dlo + ((OFF_KC + s * 2 * kTile) >> 4);
+            if (!wait_k_warp(mi, B_PREP_FULL0 + s, g >> 1)) return;
+#pragma unroll 1
+            for (int gh = 0; gh < 2; ++gh) {
+                if (2 * g + gh > 0 && !wait_k_warp(mi, B_GRAM_DRAINED, 2 * g + gh - 1)) return;
+                tc_fence_after();
+                // rows = [W ; Qt], columns = tokens i.  Re: W_re Kc_re + W_im Kc_im; Im: W_re Kc_im - W_im Kc_re
+                if (elect_one()) {
+                    const uint32_t d = tmem + TM_GRAM, w_im = w_re + 2 * kIm;
+                    const uint32_t k1 = gh ? k_re + kIm : k_re, k2 = gh ? k_re : k_re + kIm;
+                    const uint32_t id2 = gh ? I64 | (1u << 14) : I64;
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) mma_ss2(d, w_re + 2 * ks, dhi, k1 + 2 * ks, dhi, I64, ks ? 1u : 0u);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) mma_ss2(d, w_im + 2 * ks, dhi, k2 + 2 * ks, dhi, id2, 1u);
+                    mma_commit(&bars[B_GRAM_FULL]);
                 }
+                __syncwarp();
             }
         }
     }
