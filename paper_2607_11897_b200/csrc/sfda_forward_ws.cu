@@ -124,6 +124,12 @@ struct Params {
     uint32_t magic_BH, magic_H;   // floor(2^32 / d) + 1 (0 for d = 1): quotients by multiplication
 };
 
+// Tensor maps of the arrays the copy engine touches: [B][T][H][128] bf16 (v, o, o_im, q, k) or [B][T][H][64] fp32
+// (alpha, theta), box = 64 tokens of one head.
+struct Maps {
+    CUtensorMap v, o, oim, q, k, al, th;
+};
+
 // Work units.  A sequence is cut into Q time slices of U chunks; unit u = slice * BH + sequence.  CTA c works
 // through units c, c + gridDim, ... as ONE stream of chunks, so its pipeline never drains between units; only
 // the state pass notices a unit boundary (it writes the finished state out and takes the next one in).  A slice
@@ -428,30 +434,31 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
     }
 }
 
-__device__ __forceinline__ void prefetch_l2(const void *ptr)
-{
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
-}
 // ---- input prefetch ------------------------------------------------------------------------------------
 // PREP reads q, k, alpha, theta straight from global memory (no shared memory is left to stage them).  So that
-// those loads find their lines in L2 instead of stalling on HBM in a burst, one otherwise idle warp touches the
-// rows of a chunk two chunks before PREP gets there: 64 tokens x 4 arrays x 256 bytes = 512 lines per chunk.
-__device__ __forceinline__ void run_prefetch(Misc &mi, const Params &p, int n_chunks, int lane)
+// those loads find their lines in L2 instead of stalling on HBM, the copy engine is asked to bring the four tiles
+// of a chunk into L2 two chunks before PREP gets there: four instructions per chunk.
+__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap *map, int c0, int c1, int c2, int c3)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(
+                     reinterpret_cast<uint64_t>(map)),
+                 "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+}
+__device__ __forceinline__ void run_prefetch(Misc &mi, const Params &p, const Maps &maps, int n_chunks)
 {
     ChunkCursor cur(p);
+#pragma unroll 1
     for (int j = 0; j < n_chunks; ++j, cur.next(p)) {
-        if (j >= 2 && !wait_k(mi, (j - 2) & 1 ? B_PREP_FULL1 : B_PREP_FULL0, (j - 2) >> 1)) return;
+        if (j >= 2 && !wait_k_warp(mi, B_PREP_FULL0 + (j & 1), (j - 2) >> 1)) return;
         const ChunkInfo ci = cur.ci;
-        const int t0 = ci.jg * C, len = min(C, p.T - t0);
-        const size_t row0 = ((size_t)ci.b * p.T + t0) * p.H + ci.h;
-        for (int idx = lane; idx < 2 * len; idx += 32) {
-            const size_t row = row0 + (size_t)(idx >> 1) * p.H;
-            const size_t off = (size_t)(idx & 1) * 128;
-            prefetch_l2(reinterpret_cast<const char *>(p.alpha + row * M) + off);
-            prefetch_l2(reinterpret_cast<const char *>(p.theta + row * M) + off);
-            prefetch_l2(reinterpret_cast<const char *>(p.k + row * DK) + off);
-            prefetch_l2(reinterpret_cast<const char *>(p.q + row * DK) + off);
+        if (elect_one()) {
+            tma_prefetch_4d(&maps.al, 0, ci.h, ci.jg * C, ci.b);
+            tma_prefetch_4d(&maps.th, 0, ci.h, ci.jg * C, ci.b);
+            tma_prefetch_4d(&maps.k, 0, ci.h, ci.jg * C, ci.b);
+            tma_prefetch_4d(&maps.q, 0, ci.h, ci.jg * C, ci.b);
         }
+        __syncwarp();
     }
 }
 
@@ -1077,8 +1084,7 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
 
 // ---- the kernel ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads, 1)
-sfda_forward_ws_kernel(const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
-                       const __grid_constant__ CUtensorMap tm_oim, const Params p)
+sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -1126,9 +1132,9 @@ sfda_forward_ws_kernel(const __grid_constant__ CUtensorMap tm_v, const __grid_co
         regs_dec<kRegsCtrl>();
         const int cw = warp - (kChainWarps + kSolveWarps + kPrepWarps);
         if (cw == 3)
-            run_prefetch(mi, p, n_chunks, tid & 31);
+            run_prefetch(mi, p, maps, n_chunks);
         else
-            run_ctrl(cw, smem, mi, tmem, &tm_v, &tm_o, &tm_oim, p, n_chunks);
+            run_ctrl(cw, smem, mi, tmem, &maps.v, &maps.o, &maps.oim, p, n_chunks);
     }
 
     tc_fence_before();
@@ -1164,18 +1170,19 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
-// [B][T][H][128] bf16 tensor, box = 64 tokens of one head.
-bool make_map(CUtensorMap *map, const void *base, int B, int T, int H)
+// [B][T][H][inner] tensor of bf16 (inner = 128) or fp32 (inner = 64), box = 64 tokens of one head.
+bool make_map(CUtensorMap *map, const void *base, int B, int T, int H, bool f32 = false)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    const cuuint64_t dims[4] = {(cuuint64_t)DV, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)B};
-    const cuuint64_t strides[3] = {(cuuint64_t)DV * 2, (cuuint64_t)H * DV * 2, (cuuint64_t)T * H * DV * 2};
-    const cuuint32_t box[4] = {(cuuint32_t)DV, 1, (cuuint32_t)C, 1};
+    const cuuint64_t inner = f32 ? M : DV, row = 256;      // elements, bytes per (token, head)
+    const cuuint64_t dims[4] = {inner, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {row, (cuuint64_t)H * row, (cuuint64_t)T * H * row};
+    const cuuint32_t box[4] = {(cuuint32_t)inner, 1, (cuuint32_t)C, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base),
+              dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace
@@ -1246,9 +1253,11 @@ size_t forward_ws_scratch_bytes(int B, int H)
 
 cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratch_bytes, cudaStream_t stream, int *launches)
 {
-    CUtensorMap tv, to, toi;
-    if (!make_map(&tv, a.v, a.B, a.T, a.H) || !make_map(&to, a.o, a.B, a.T, a.H) ||
-        !make_map(&toi, a.o_im ? a.o_im : a.o, a.B, a.T, a.H))
+    Maps maps;
+    if (!make_map(&maps.v, a.v, a.B, a.T, a.H) || !make_map(&maps.o, a.o, a.B, a.T, a.H) ||
+        !make_map(&maps.oim, a.o_im ? a.o_im : a.o, a.B, a.T, a.H) || !make_map(&maps.q, a.q, a.B, a.T, a.H) ||
+        !make_map(&maps.k, a.k, a.B, a.T, a.H) || !make_map(&maps.al, a.alpha, a.B, a.T, a.H, true) ||
+        !make_map(&maps.th, a.theta, a.B, a.T, a.H, true))
         return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(sfda_forward_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
@@ -1301,7 +1310,7 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
     p.magic_H = a.H > 1 ? (uint32_t)(0x100000000ull / (unsigned)a.H) + 1u : 0u;
     g_ws_last_slices = Q;
     const unsigned grid = (unsigned)(p.n_units < n_sm ? p.n_units : n_sm);
-    sfda_forward_ws_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tv, to, toi, p);
+    sfda_forward_ws_kernel<<<grid, kThreads, kSmemBytes, stream>>>(maps, p);
     e = cudaGetLastError();
     if (e == cudaSuccess && launches) ++*launches;
     return e;
