@@ -168,6 +168,9 @@ def main():
     ap.add_argument("--re-only", action="store_true", help="write o = Re only (default: Re and Im)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--clock-load-s", type=float, default=1.0,
+                    help="seconds of untimed continuation of the same launches under the clock sampler (0: none, "
+                         "for profiler runs)")
     ap.add_argument("--batch", type=int, default=0,
                     help="profiling only: run the headline shapes with this batch size instead of 8 "
                          "(the JSON line then names the reduced workload and is not a benchmark value)")
@@ -243,7 +246,7 @@ def main():
         # The timed region lasts tens of milliseconds, too short for nvidia-smi to see: the same launches go on,
         # untimed, under the sampler until it has had about a second of this load.
         t_load = time.perf_counter()
-        while time.perf_counter() - t_load < 1.0:
+        while time.perf_counter() - t_load < args.clock_load_s:
             for _ in range(20):
                 step()
             torch.cuda.synchronize()
@@ -335,9 +338,9 @@ def main():
         "roofline_ms": 1e3 * max(hbm_time, tensor_time),
     }
     if args.batch == 0:
-        # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this kernel at B = 4 (1.870 GB,
+        # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this kernel at B = 4 (1.951 GB,
         # profiles/sfda_forward_ws_kernel_batch4_ncu_full.md), scaled by the units processed (traffic grows with B)
-        roofline["traffic"] = 1.870e9 * cfg.B / 4
+        roofline["traffic"] = 1.951e9 * cfg.B / 4
         roofline["traffic_source"] = "ncu capture at B=4 scaled to B=%d; Re+Im outputs" % cfg.B
 
     if decode is not None:
