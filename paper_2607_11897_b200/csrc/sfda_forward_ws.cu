@@ -565,15 +565,13 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
 
             // pass 1: this thread's product of alpha (fp32 products of at most 64 factors: relative error far
             // below bf16's) and sum of the integer phase over its 8 tokens
-            float2 al[8], th[8];
+            uint2 al[8], th[8];                  // raw bits; neutral (alpha = 1, theta = 0) beyond the sequence
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                al[i] = make_float2(1.f, 1.f);
-                th[i] = make_float2(0.f, 0.f);
-                if (i < nt) {
-                    al[i] = __ldg(reinterpret_cast<const float2 *>(reinterpret_cast<const char *>(p.alpha) + off + i * step));
-                    th[i] = __ldg(reinterpret_cast<const float2 *>(reinterpret_cast<const char *>(p.theta) + off + i * step));
-                }
+                al[i] = make_uint2(0x3f800000u, 0x3f800000u);
+                th[i] = make_uint2(0u, 0u);
+                ldg64_if(al[i].x, al[i].y, reinterpret_cast<const char *>(p.alpha) + off + i * step, i < nt);
+                ldg64_if(th[i].x, th[i].y, reinterpret_cast<const char *>(p.theta) + off + i * step, i < nt);
             }
             SFDA_T(36);
             // beta of token pt: fetched now, written after the pass below so that its latency is covered
@@ -585,10 +583,10 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
                 uint32_t u0 = 0u, u1 = 0u;
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                    a0 *= fmaxf(al[i].x, 9.0e-14f);           // floor e^-30, as in log_decay
-                    a1 *= fmaxf(al[i].y, 9.0e-14f);
-                    u0 += turns_f32(th[i].x);
-                    u1 += turns_f32(th[i].y);
+                    a0 *= fmaxf(__uint_as_float(al[i].x), 9.0e-14f);           // floor e^-30, as in log_decay
+                    a1 *= fmaxf(__uint_as_float(al[i].y), 9.0e-14f);
+                    u0 += turns_f32(__uint_as_float(th[i].x));
+                    u1 += turns_f32(__uint_as_float(th[i].y));
                 }
                 *reinterpret_cast<float2 *>(&mi.part_lg[s][tq][2 * jp]) = make_float2(a0, a1);
                 *reinterpret_cast<uint2 *>(&mi.part_turns[s][tq][2 * jp]) = make_uint2(u0, u1);

@@ -229,7 +229,7 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t saddr)
 // otherwise): no branch, so neighbouring work can be scheduled across them.
 __device__ __forceinline__ void ldg64_if(uint32_t &x, uint32_t &y, const void *ptr, bool on)
 {
-    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %3, 0;\n@p ld.global.nc.v2.b32 {%0, %1}, [%2];\n}\n"
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %3, 0;\n@p ld.global.cg.v2.b32 {%0, %1}, [%2];\n}\n"
                  : "+r"(x), "+r"(y)
                  : "l"(ptr), "r"((uint32_t)on));
 }
