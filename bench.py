@@ -110,7 +110,10 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm),
+                "sm_mhz_first": sm[0] if sm else None,
+                "window": "timed region plus about a second of the same launches (the timed region alone is "
+                          "shorter than one nvidia-smi sample)"}
 
 
 def cpu_oracle_throughput(cfg, n_pairs, T):

@@ -212,7 +212,12 @@ SFDA_API int sfda_step(const void *q, const void *k, const void *v,
  * Host-buffer forward: the call a user with data in host memory makes.  Copies the
  * inputs from HOST memory (pinned for asynchronous copies) into `arena`, runs
  * sfda_forward there and copies o (and o_im, S_T when not NULL) back to HOST
- * memory, all enqueued on `stream`.  Host pointers: q, k, v, alpha, theta, beta,
+ * memory.  The batch is cut into up to 8 pieces that go up, are computed and come
+ * down overlapped: the kernels run on `stream`, the copies on two streams the
+ * library creates per device on the first such call (the only resources it ever
+ * creates) and chains to `stream` with events; work enqueued on `stream` before the
+ * call precedes all of it, and `stream` is finished only when the last download is.
+ * Host pointers: q, k, v, alpha, theta, beta,
  * S0, o, o_im, S_T.  Device pointer: arena, at least sfda_forward_host_arena_bytes
  * bytes, 256-byte aligned, clobbered.  bytes_h2d / bytes_d2h (host, may be NULL)
  * receive the bytes copied in each direction.

@@ -1,6 +1,8 @@
 // C ABI of the library: argument validation on the host, dispatch to the kernels.
 #include "../../include/sfda.h"
 
+#include <mutex>
+
 #include "sfda_internal.h"
 
 namespace {
@@ -20,6 +22,46 @@ int check_dims(int d_k, int d_v, int chunk, int dtype)
 }
 
 size_t elem_bytes(int dtype) { return dtype == SFDA_BF16 ? 2 : 4; }
+
+// The host-buffer forward overlaps its uploads, kernels and downloads: pieces of the batch go up on one internal
+// stream, are computed on the caller's stream and come down on another internal stream, chained by events.  The two
+// streams and the events are created once per device on first use and kept for the life of the process.
+constexpr int kMaxPieces = 8;
+constexpr int kMaxPipeDevices = 64;
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t up = nullptr, down = nullptr;
+    cudaEvent_t start = nullptr, end = nullptr, uploaded[kMaxPieces] = {}, computed[kMaxPieces] = {};
+};
+std::mutex g_pipe_mutex;
+HostPipe g_pipes[kMaxPipeDevices];
+
+HostPipe *host_pipe()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxPipeDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(g_pipe_mutex);
+    HostPipe &hp = g_pipes[dev];
+    if (!hp.ready) {
+        bool ok = cudaStreamCreateWithFlags(&hp.up, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&hp.down, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp.end, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; ok && i < kMaxPieces; ++i)
+            ok = cudaEventCreateWithFlags(&hp.uploaded[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&hp.computed[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) return nullptr;
+        hp.ready = true;
+    }
+    return &hp;
+}
+
+// batch elements per piece and number of pieces of the host-buffer forward
+void host_pieces(int B, int *per_piece, int *pieces)
+{
+    *per_piece = (B + kMaxPieces - 1) / kMaxPieces;
+    *pieces = (B + *per_piece - 1) / *per_piece;
+}
 
 int validate_forward(const void *q, const void *k, const void *v, const float *alpha, const float *theta,
                      const float *beta, const float *S0, void *o, void *o_im, float *S_T, int B, int T, int H,
@@ -206,7 +248,9 @@ size_t sfda_forward_host_arena_bytes(int B, int T, int H, int d_k, int d_v, int 
     total += 2 * round256(n * m * 4) + round256(n * 4);       // alpha, theta, beta
     total += (want_o_im ? 2 : 1) * round256(n * d_v * eb);    // o, o_im
     if (have_S0 || want_S_T) total += round256((size_t)B * H * d_k * d_v * 4);
-    total += round256(sfda_workspace_bytes(B, T, H, d_k, d_v, chunk, dtype));
+    int per = 1, pieces = 1;
+    host_pieces(B, &per, &pieces);
+    total += (size_t)pieces * round256(sfda_workspace_bytes(per, T, H, d_k, d_v, chunk, dtype));   // one per piece
     return total;
 }
 
@@ -226,50 +270,64 @@ int sfda_forward_host(const void *q, const void *k, const void *v, const float *
     if (reinterpret_cast<uintptr_t>(arena) & 255u) return SFDA_ERR_ALIGN;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    HostPipe *hp = host_pipe();
+    if (!hp) return SFDA_ERR_CUDA;
     const size_t n = (size_t)B * T * H, eb = elem_bytes(dtype), m = d_k / 2;
+    const size_t state_elems = (size_t)H * d_k * d_v;             // per batch element
     char *cur = static_cast<char *>(arena);
     auto take = [&](size_t bytes) { char *p = cur; cur += round256(bytes); return p; };
+    char *dq = take(n * d_k * eb), *dk = take(n * d_k * eb), *dv = take(n * d_v * eb);
+    char *da = take(n * m * 4), *dt = take(n * m * 4), *db = take(n * 4);
+    char *dout = take(n * d_v * eb), *dout_im = o_im ? take(n * d_v * eb) : nullptr;
+    char *dS = (S0 || S_T) ? take((size_t)B * state_elems * 4) : nullptr;
+    int per = 1, pieces = 1;
+    host_pieces(B, &per, &pieces);
+    const size_t ws_bytes = sfda_workspace_bytes(per, T, H, d_k, d_v, chunk, dtype);
+    char *ws0 = take((size_t)pieces * round256(ws_bytes));
+
     size_t h2d = 0, d2h = 0;
     bool ok = true;
-    auto up = [&](const void *src, size_t bytes) {
-        char *dst = take(bytes);
-        ok = ok && cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
-        h2d += bytes;
-        return dst;
+    int launches = 0;
+    auto copy = [&](void *dst, const void *src, size_t bytes, cudaMemcpyKind kind, cudaStream_t st) {
+        ok = ok && cudaMemcpyAsync(dst, src, bytes, kind, st) == cudaSuccess;
+        (kind == cudaMemcpyHostToDevice ? h2d : d2h) += bytes;
     };
-    void *dq = up(q, n * d_k * eb);
-    void *dk = up(k, n * d_k * eb);
-    void *dv = up(v, n * d_v * eb);
-    float *da = reinterpret_cast<float *>(up(alpha, n * m * 4));
-    float *dt = reinterpret_cast<float *>(up(theta, n * m * 4));
-    float *db = reinterpret_cast<float *>(up(beta, n * 4));
-    void *dout = take(n * d_v * eb);
-    void *dout_im = o_im ? take(n * d_v * eb) : nullptr;
-    float *dS = nullptr;
-    const size_t state_bytes = (size_t)B * H * d_k * d_v * 4;
-    if (S0 || S_T) dS = reinterpret_cast<float *>(take(state_bytes));
-    if (S0) {
-        ok = ok && cudaMemcpyAsync(dS, S0, state_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
-        h2d += state_bytes;
+    // everything enqueued on the caller's stream so far comes before the first copy of either direction
+    ok = ok && cudaEventRecord(hp->start, s) == cudaSuccess && cudaStreamWaitEvent(hp->up, hp->start, 0) == cudaSuccess &&
+         cudaStreamWaitEvent(hp->down, hp->start, 0) == cudaSuccess;
+    for (int i = 0; ok && i < pieces; ++i) {
+        const int b0 = i * per, nb = (b0 + per <= B ? per : B - b0);
+        const size_t r0 = (size_t)b0 * T * H, rn = (size_t)nb * T * H;        // (token, head) rows of the piece
+        const char *hq = static_cast<const char *>(q), *hk = static_cast<const char *>(k), *hv = static_cast<const char *>(v);
+        copy(dq + r0 * d_k * eb, hq + r0 * d_k * eb, rn * d_k * eb, cudaMemcpyHostToDevice, hp->up);
+        copy(dk + r0 * d_k * eb, hk + r0 * d_k * eb, rn * d_k * eb, cudaMemcpyHostToDevice, hp->up);
+        copy(dv + r0 * d_v * eb, hv + r0 * d_v * eb, rn * d_v * eb, cudaMemcpyHostToDevice, hp->up);
+        copy(da + r0 * m * 4, alpha + r0 * m, rn * m * 4, cudaMemcpyHostToDevice, hp->up);
+        copy(dt + r0 * m * 4, theta + r0 * m, rn * m * 4, cudaMemcpyHostToDevice, hp->up);
+        copy(db + r0 * 4, beta + r0, rn * 4, cudaMemcpyHostToDevice, hp->up);
+        if (S0) copy(dS + b0 * state_elems * 4, S0 + b0 * state_elems, nb * state_elems * 4, cudaMemcpyHostToDevice, hp->up);
+        ok = ok && cudaEventRecord(hp->uploaded[i], hp->up) == cudaSuccess &&
+             cudaStreamWaitEvent(s, hp->uploaded[i], 0) == cudaSuccess;
+        if (!ok) break;
+        float *dSp = dS ? reinterpret_cast<float *>(dS) + b0 * state_elems : nullptr;
+        const int frc = sfda_forward(dq + r0 * d_k * eb, dk + r0 * d_k * eb, dv + r0 * d_v * eb,
+                                     reinterpret_cast<float *>(da) + r0 * m, reinterpret_cast<float *>(dt) + r0 * m,
+                                     reinterpret_cast<float *>(db) + r0, S0 ? dSp : nullptr, dout + r0 * d_v * eb,
+                                     dout_im ? dout_im + r0 * d_v * eb : nullptr, S_T ? dSp : nullptr, nb, T, H, d_k, d_v,
+                                     chunk, dtype, ws0 + (size_t)i * round256(ws_bytes), ws_bytes, stream);
+        if (frc != SFDA_OK) return frc;
+        launches += g_last_launches;
+        ok = ok && cudaEventRecord(hp->computed[i], s) == cudaSuccess &&
+             cudaStreamWaitEvent(hp->down, hp->computed[i], 0) == cudaSuccess;
+        copy(static_cast<char *>(o) + r0 * d_v * eb, dout + r0 * d_v * eb, rn * d_v * eb, cudaMemcpyDeviceToHost, hp->down);
+        if (o_im)
+            copy(static_cast<char *>(o_im) + r0 * d_v * eb, dout_im + r0 * d_v * eb, rn * d_v * eb, cudaMemcpyDeviceToHost,
+                 hp->down);
+        if (S_T) copy(S_T + b0 * state_elems, dSp, nb * state_elems * 4, cudaMemcpyDeviceToHost, hp->down);
     }
-    const size_t ws_bytes = sfda_workspace_bytes(B, T, H, d_k, d_v, chunk, dtype);
-    void *ws = ws_bytes ? take(ws_bytes) : nullptr;
-    if (!ok) return SFDA_ERR_CUDA;
-
-    const int frc = sfda_forward(dq, dk, dv, da, dt, db, S0 ? dS : nullptr, dout, dout_im, S_T ? dS : nullptr, B, T,
-                                 H, d_k, d_v, chunk, dtype, ws, ws_bytes, stream);
-    if (frc != SFDA_OK) return frc;
-
-    ok = ok && cudaMemcpyAsync(o, dout, n * d_v * eb, cudaMemcpyDeviceToHost, s) == cudaSuccess;
-    d2h += n * d_v * eb;
-    if (o_im) {
-        ok = ok && cudaMemcpyAsync(o_im, dout_im, n * d_v * eb, cudaMemcpyDeviceToHost, s) == cudaSuccess;
-        d2h += n * d_v * eb;
-    }
-    if (S_T) {
-        ok = ok && cudaMemcpyAsync(S_T, dS, state_bytes, cudaMemcpyDeviceToHost, s) == cudaSuccess;
-        d2h += state_bytes;
-    }
+    // the caller's stream is done when the last download is
+    ok = ok && cudaEventRecord(hp->end, hp->down) == cudaSuccess && cudaStreamWaitEvent(s, hp->end, 0) == cudaSuccess;
+    g_last_launches = launches;
     if (bytes_h2d) *bytes_h2d = h2d;
     if (bytes_d2h) *bytes_d2h = d2h;
     return ok ? SFDA_OK : SFDA_ERR_CUDA;
