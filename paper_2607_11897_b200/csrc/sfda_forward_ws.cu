@@ -288,13 +288,17 @@ __device__ __forceinline__ bool test_k_warp(Misc &mi, int bar, int k)
 // the accumulators start from zero.  `b_step`: descriptor advance of B per K = 16 (2 for a K-major tile,
 // 128 for an MN-major one).  The state update uses the same products with conj(E)-side roles swapped, which
 // `swap` selects: Re += x_re b_re, Re -= x_im b_im, Im += x_re b_im, Im += x_im b_re.
+// `part` selects the products of one accumulator: 0 = Re (g = 0, 1), 1 = Im (g = 2, 3), 2 = both.  The two halves
+// touch different accumulator columns, so two threads can issue them side by side (instructions of one thread
+// execute in order, which the accumulation inside a half needs; nothing orders two threads, nor has to).
 template <int kNegG, bool kFresh, bool kSwap, uint32_t kBStep>
 __device__ __forceinline__ void issue_complex(uint32_t d_re, uint32_t d_im, uint32_t a_re, uint32_t a_im, uint32_t b_re,
-                                              uint32_t b_im, uint32_t dhi, uint32_t id)
+                                              uint32_t b_im, uint32_t dhi, uint32_t id, int part)
 {
     if (elect_one()) {
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
+            if (part != 2 && (g >> 1) != part) continue;
             const bool odd = g & 1, mid = g == 1 || g == 2;
             const uint32_t d = g < 2 ? d_re : d_im;
             const uint32_t a = (kSwap ? odd : mid) ? a_im : a_re;
@@ -308,14 +312,38 @@ __device__ __forceinline__ void issue_complex(uint32_t d_re, uint32_t d_im, uint
     __syncwarp();
 }
 
-// The issuing work is split over three warps (they sit on different schedulers):
-//   role 0  the products on the state's dependency chain: D1 (with rho_1), E, the state update
-//   role 1  the output product rho += Aq E and the output stores
-//   role 2  the Gram products (they run ahead of the chain) and the v loads
-__device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint32_t tmem, const CUtensorMap *tm_v,
-                                         const CUtensorMap *tm_o, const CUtensorMap *tm_oim, const Params &p,
-                                         int n_chunks)
+// ---- input prefetch ------------------------------------------------------------------------------------
+// PREP reads q, k, alpha, theta straight from global memory (no shared memory is left to stage them).  So that
+// those loads find their lines in L2 instead of stalling on HBM, the copy engine is asked to bring the four tiles
+// of a chunk into L2 two chunks before PREP gets there: four instructions per chunk.
+__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap *map, int c0, int c1, int c2, int c3)
 {
+    asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(
+                     reinterpret_cast<uint64_t>(map)),
+                 "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+}
+__device__ __forceinline__ void prefetch_chunk(const Maps &maps, const ChunkInfo &ci)
+{
+    if (elect_one()) {
+        tma_prefetch_4d(&maps.al, 0, ci.h, ci.jg * C, ci.b);
+        tma_prefetch_4d(&maps.th, 0, ci.h, ci.jg * C, ci.b);
+        tma_prefetch_4d(&maps.k, 0, ci.h, ci.jg * C, ci.b);
+        tma_prefetch_4d(&maps.q, 0, ci.h, ci.jg * C, ci.b);
+    }
+    __syncwarp();
+}
+
+// The issuing work is split over four warps (they sit on different schedulers):
+//   roles 0, 3  the products on the state's dependency chain: D1, rho_1, E, the state update; role 0 issues the
+//               products into the real accumulators, role 3 those into the imaginary ones (issuing, not the
+//               tensor pipe, is what takes the time: about a hundred cycles per instruction)
+//   role 1      the output product rho += Aq E and the output stores
+//   role 2      the v loads, the Gram products (they run ahead of the chain) and the L2 prefetch of the inputs
+__device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint32_t tmem, const Maps &maps,
+                                         const Params &p, int n_chunks)
+{
+    const CUtensorMap *tm_v = &maps.v, *tm_o = &maps.o, *tm_oim = &maps.oim;
     long long *timing = p.timing;
     const uint64_t dbase = smem_desc(smem_u32(smem));                     // descriptor of byte offset 0
     const uint32_t dlo = (uint32_t)dbase, dhi = (uint32_t)(dbase >> 32);
@@ -325,8 +353,9 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
     const uint32_t x_re = tmem + TM_X16, acc = tmem + TM_ACC;
     const uint32_t m_re = dlo + (OFF_MB >> 4);
 
-    if (role == 0) {
-        SFDA_TDECL((threadIdx.x & 31) == 0);
+    if (role == 0 || role == 3) {
+        const int part = role == 0 ? 0 : 1;      // this warp's accumulator half
+        SFDA_TDECL((threadIdx.x & 31) == 0 && role == 0);
 #pragma unroll 1
         for (int j = 0; j < n_chunks; ++j) {
             const int s = j & 1, u = j >> 1;
@@ -337,11 +366,11 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
             if (!wait_k_warp(mi, B_PREP_FULL0 + s, u)) return;
             tc_fence_after();
             SFDA_T(0);
-            issue_complex<3, true, false, 2>(acc, acc + 128, x_re, x_re + 32, w_re, w_re + 2 * kIm, dhi, I64);
+            issue_complex<3, true, false, 2>(acc, acc + 128, x_re, x_re + 32, w_re, w_re + 2 * kIm, dhi, I64, part);
             if (elect_one()) mma_commit(&bars[B_D1_DONE]);
             if (j > 0 && !wait_k_warp(mi, B_O_STAGED, j - 1)) return;
             tc_fence_after();
-            issue_complex<3, true, false, 2>(acc + 64, acc + 192, x_re, x_re + 32, w_re + kIm, w_re + 3 * kIm, dhi, I64);
+            issue_complex<3, true, false, 2>(acc + 64, acc + 192, x_re, x_re + 32, w_re + kIm, w_re + 3 * kIm, dhi, I64, part);
             if (elect_one()) {
                 mma_commit(&bars[B_O1_DONE]);
                 mma_commit(&bars[B_WQ_FREE0 + s]);
@@ -353,14 +382,14 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
             if (!wait_k_warp(mi, B_MB_FULL, j)) return;
             tc_fence_after();
             SFDA_T(3);
-            issue_complex<1, true, false, 2>(acc, acc + 128, x_re, x_re + 32, m_re, m_re + kIm, dhi, I64);
+            issue_complex<1, true, false, 2>(acc, acc + 128, x_re, x_re + 32, m_re, m_re + kIm, dhi, I64, part);
             if (elect_one()) mma_commit(&bars[B_E_DONE]);
             SFDA_T(4);
             // S += E^T Kc (Kc as MN-major B: rows = tokens)
             if (!wait_k_warp(mi, B_E16_READY, j)) return;
             tc_fence_after();
             SFDA_T(5);
-            issue_complex<1, false, true, 128>(tmem + TM_S32, tmem + TM_S32 + 64, x_re, x_re + 32, k_re, k_re + kIm, dhi, I64M);
+            issue_complex<1, false, true, 128>(tmem + TM_S32, tmem + TM_S32 + 64, x_re, x_re + 32, k_re, k_re + kIm, dhi, I64M, part);
             if (elect_one()) {
                 mma_commit(&bars[B_KC_FREE0 + s]);
                 mma_commit(&bars[B_UPD_DONE]);
@@ -395,7 +424,7 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
             if (!wait_k_warp(mi, B_AQ_FULL0 + (j & 1), j >> 1)) return;
             tc_fence_after();
             const uint32_t a_re = dlo + ((OFF_AQ + (j & 1) * 2 * kTile) >> 4);
-            issue_complex<1, false, false, 2>(acc + 64, acc + 192, x_re, x_re + 32, a_re, a_re + kIm, dhi, I64);
+            issue_complex<1, false, false, 2>(acc + 64, acc + 192, x_re, x_re + 32, a_re, a_re + kIm, dhi, I64, 2);
             if (elect_one()) mma_commit(&bars[B_UPD_DONE]);
         }
     } else {
@@ -403,7 +432,9 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
         // consumed (R of that chunk is built); then the two Gram halves of chunk g, each once its operands are
         // written and the Gram columns have been read out.  Blocking waits: a polling loop here would take issue
         // slots from the warps that do the work.
-        ChunkCursor vcur(p);
+        ChunkCursor vcur(p), pcur(p);            // chunk g below; the chunk whose inputs are prefetched next
+#pragma unroll 1
+        for (int i = 0; i < 2 && i < n_chunks; ++i, pcur.next(p)) prefetch_chunk(maps, pcur.ci);
 #pragma unroll 1
         for (int g = 0; g < n_chunks; ++g) {
             if (g > 0 && !wait_k_warp(mi, B_R16_READY, g - 1)) return;
@@ -436,35 +467,12 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
                 }
                 __syncwarp();
             }
+            // PREP has finished chunk g: time to bring the inputs of chunk g + 2 into L2
+            if (g + 2 < n_chunks) {
+                prefetch_chunk(maps, pcur.ci);
+                pcur.next(p);
+            }
         }
-    }
-}
-
-// ---- input prefetch ------------------------------------------------------------------------------------
-// PREP reads q, k, alpha, theta straight from global memory (no shared memory is left to stage them).  So that
-// those loads find their lines in L2 instead of stalling on HBM, the copy engine is asked to bring the four tiles
-// of a chunk into L2 two chunks before PREP gets there: four instructions per chunk.
-__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap *map, int c0, int c1, int c2, int c3)
-{
-    asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(
-                     reinterpret_cast<uint64_t>(map)),
-                 "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-                 : "memory");
-}
-__device__ __forceinline__ void run_prefetch(Misc &mi, const Params &p, const Maps &maps, int n_chunks)
-{
-    ChunkCursor cur(p);
-#pragma unroll 1
-    for (int j = 0; j < n_chunks; ++j, cur.next(p)) {
-        if (j >= 2 && !wait_k_warp(mi, B_PREP_FULL0 + (j & 1), (j - 2) >> 1)) return;
-        const ChunkInfo ci = cur.ci;
-        if (elect_one()) {
-            tma_prefetch_4d(&maps.al, 0, ci.h, ci.jg * C, ci.b);
-            tma_prefetch_4d(&maps.th, 0, ci.h, ci.jg * C, ci.b);
-            tma_prefetch_4d(&maps.k, 0, ci.h, ci.jg * C, ci.b);
-            tma_prefetch_4d(&maps.q, 0, ci.h, ci.jg * C, ci.b);
-        }
-        __syncwarp();
     }
 }
 
@@ -1104,11 +1112,12 @@ sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
     if (tid == 0) {
         auto init = [&](int bar, uint32_t count) { mbar_init(&mi.bars[bar], count); };
         init(B_PREP_FULL0, kPrepWarps); init(B_PREP_FULL1, kPrepWarps);
-        init(B_WQ_FREE0, 1); init(B_WQ_FREE1, 1); init(B_KC_FREE0, 1); init(B_KC_FREE1, 1);
+        init(B_WQ_FREE0, 2); init(B_WQ_FREE1, 2); init(B_KC_FREE0, 2); init(B_KC_FREE1, 2);   // both issuing warps
         init(B_STORE_DONE0, 1); init(B_STORE_DONE1, 1);
         init(B_GRAM_FULL, 1); init(B_GRAM_DRAINED, kSolveWarps);
         init(B_MB_FULL, kSolveWarps); init(B_AQ_FULL0, kSolveWarps); init(B_AQ_FULL1, kSolveWarps);
-        init(B_D1_DONE, 1); init(B_O1_DONE, 1); init(B_E_DONE, 1); init(B_UPD_DONE, 2);   // state update and rho += Aq E
+        init(B_D1_DONE, 2); init(B_O1_DONE, 2); init(B_E_DONE, 2);
+        init(B_UPD_DONE, 3);   // the two halves of the state update and rho += Aq E
         init(B_S16_READY, kChainWarps); init(B_R16_READY, kChainWarps); init(B_E16_READY, kChainWarps);
         init(B_O_STAGED, kPrepWarps); init(B_V_FULL, 1);
         mi.abort = 0;
@@ -1135,10 +1144,7 @@ sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
     } else {
         regs_dec<kRegsCtrl>();
         const int cw = warp - (kChainWarps + kSolveWarps + kPrepWarps);
-        if (cw == 3)
-            run_prefetch(mi, p, maps, n_chunks);
-        else
-            run_ctrl(cw, smem, mi, tmem, &maps.v, &maps.o, &maps.oim, p, n_chunks);
+        run_ctrl(cw, smem, mi, tmem, maps, p, n_chunks);
     }
 
     tc_fence_before();
