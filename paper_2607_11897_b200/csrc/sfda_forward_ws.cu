@@ -1069,22 +1069,22 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
             const bool sub_v = ph == 0 && half == 0;            // R_re = V - D1_re
             const float sgn = ph == 0 ? -1.f : 1.f;             // R_im = -D1_im
 #pragma unroll 1
-            for (int pc = 0; pc < 4; ++pc) {
-                uint32_t r[16], pk[8];
-                tmem_ld<16>(tlane + TM_ACC + 128 * half + 16 * pc, r);
+            for (int pc = 0; pc < 2; ++pc) {       // 32 columns per tensor-memory round trip
+                uint32_t r[32], pk[16];
+                tmem_ld<32>(tlane + TM_ACC + 128 * half + 32 * pc, r);
                 tc_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
+                for (int i = 0; i < 16; ++i) {
                     float v0 = 0.f, v1 = 0.f;
                     if (sub_v) {
-                        v0 = __uint_as_float((uint32_t)lds16(sv + (16 * pc + 2 * i) * 2 * DV) << 16);
-                        v1 = __uint_as_float((uint32_t)lds16(sv + (16 * pc + 2 * i + 1) * 2 * DV) << 16);
+                        v0 = __uint_as_float((uint32_t)lds16(sv + (32 * pc + 2 * i) * 2 * DV) << 16);
+                        v1 = __uint_as_float((uint32_t)lds16(sv + (32 * pc + 2 * i + 1) * 2 * DV) << 16);
                     }
                     pk[i] = pack_bf16(fmaf(sgn, __uint_as_float(r[2 * i]), v0), fmaf(sgn, __uint_as_float(r[2 * i + 1]), v1));
                 }
                 // R replaces S_0 in the operand columns: rho_1, the last reader of S_0, must be done
                 if (ph == 0 && pc == 0 && !wait_k_warp(mi, B_O1_DONE, j)) return;
-                tmem_st8(tlane + TM_X16 + 32 * half + 8 * pc, pk);
+                tmem_st<16>(tlane + TM_X16 + 32 * half + 16 * pc, pk);
             }
             tc_wait_st();
             tc_fence_before();
