@@ -173,6 +173,34 @@ def test_forward_tensor_core_time_slices():
         assert np.array_equal(x, y)          # slicing only moves the fp32 state through memory: bit-identical
 
 
+def test_forward_tensor_core_optional_outputs_and_zero_state():
+    """Tensor-core path without o_im, without S_T, and with S0 = NULL (zero state)."""
+    cfg = workloads.CONFIGS[1].scaled(name="tc_opt", B=1, T=300, H=2, s0_std=0.0, seed=55)
+    inp = workloads.forward_inputs(cfg)
+    assert inp["S0"] is None or not np.any(inp["S0"])
+    inp["S0"] = None
+    check_forward(cfg, inp, all_pairs(cfg), TOL["bf16"], want_im=False, want_state=False)
+    check_forward(cfg, inp, all_pairs(cfg), TOL["bf16"], want_im=True, want_state=True)
+
+
+def test_forward_tensor_core_large_phases_and_write_extremes():
+    """Phases far outside (-pi, pi] (the kernel's sines and cosines reduce them), beta = 0 and beta = 1 tokens."""
+    cfg = workloads.CONFIGS[1].scaled(name="tc_phase", B=1, T=256, H=2, s0_std=0.3, seed=56)
+    inp = workloads.forward_inputs(cfg)
+    rng = np.random.default_rng(560)
+    inp["theta"] = (inp["theta"] + 2.0 * np.pi * rng.integers(-40, 41, inp["theta"].shape)).astype(np.float32)
+    inp["beta"][:, ::3] = 0.0
+    inp["beta"][:, 1::3] = 1.0
+    check_forward(cfg, inp, all_pairs(cfg), TOL["bf16"])
+
+
+def test_forward_tensor_core_time_slices_with_ragged_tail():
+    """Time slices whose last chunk is a ragged tail (T = 500: eight chunks, the last of 52 tokens)."""
+    cfg = workloads.CONFIGS[1].scaled(name="slices_tail", B=5, T=500, H=40, s0_std=0.05, seed=92)
+    inp = workloads.forward_inputs(cfg)
+    check_forward(cfg, inp, [(0, 0), (4, 39), (2, 20), (3, 7)], TOL["bf16"])
+
+
 def test_forward_tensor_core_matches_cuda_core_path():
     cfg = workloads.CONFIGS[1].scaled(name="tc2", B=1, T=512, H=4, s0_std=0.1, seed=77)
     inp = workloads.forward_inputs(cfg)
