@@ -1,7 +1,10 @@
 // sfda_step: one-token recurrent decode (Section 3, Eq. "sfda" and o_t = S_t^* q_t).
 //
 // HBM-bound: per (batch, head) the d_k x d_v fp32 state is read once and written once; everything
-// else is a few hundred bytes.  One CTA of 128 threads owns one state.  A thread owns four adjacent
+// else is a few hundred bytes.  One CTA of 128 threads owns a block of kColTile value columns of one state (the
+// columns of a state never interact: c = k^* S, the update and o = S^* q are all per column), so that a thread
+// holds few enough registers for four or five CTAs per SM to overlap their loads, arithmetic and stores.
+// A thread owns four adjacent
 // columns (one 16-byte vector per row) of a group of complex rows, so every global access is a
 // coalesced 128-bit load or store, and the whole slice a thread owns stays in registers between the
 // two passes the update needs (first c = k^* (Lambda S), then S += k beta (v - c) and o = S^* q).
@@ -12,6 +15,7 @@ namespace sfda {
 namespace {
 
 constexpr int kStepThreads = 128;
+constexpr int kColTile = 64;   // value columns per CTA
 
 template <int DK, int DV, typename T>
 __global__ void __launch_bounds__(kStepThreads)
@@ -21,20 +25,22 @@ sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__re
                  T *__restrict__ o_im)
 {
     constexpr int M = DK / 2;              // complex rows
-    constexpr int CG = DV / 4;             // threads across one row (float4 each)
+    constexpr int CT = DV < kColTile ? DV : kColTile;   // columns of this CTA
+    constexpr int CG = CT / 4;             // threads across one row (float4 each)
     constexpr int RG = kStepThreads / CG;  // row groups
     constexpr int R = M / RG;              // complex rows per thread
     static_assert(M % RG == 0, "row groups must divide the complex rows");
 
     __shared__ float s_lr[M], s_li[M], s_kr[M], s_ki[M], s_qr[M], s_qi[M];
-    __shared__ float s_v[DV];
-    __shared__ float s_red[RG][2][DV];
+    __shared__ float s_v[CT];
+    __shared__ float s_red[RG][2][CT];
 
     const int tid = threadIdx.x;
     const size_t bh = blockIdx.x;
+    const int c0 = blockIdx.y * CT;        // first column of this CTA
     const int cg = tid % CG, rg = tid / CG;
 
-    float *Sbh = S + bh * (size_t)DK * DV;
+    float *Sbh = S + bh * (size_t)DK * DV + c0;
 
     // Issue the state loads first: they are the long-latency part.
     float4 sre[R], sim[R];
@@ -56,7 +62,7 @@ sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__re
         s_qr[j] = ld_val(q, bh * DK + 2 * j);
         s_qi[j] = ld_val(q, bh * DK + 2 * j + 1);
     }
-    for (int c = tid; c < DV; c += kStepThreads) s_v[c] = ld_val(v, bh * DV + c);
+    for (int c = tid; c < CT; c += kStepThreads) s_v[c] = ld_val(v, bh * DV + c0 + c);
     const float bt = beta[bh];
     __syncthreads();
 
@@ -124,22 +130,22 @@ sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__re
         s_red[rg][1][4 * cg + x] = oim[x];
     }
     __syncthreads();
-    for (int c = tid; c < DV; c += kStepThreads) {
+    for (int c = tid; c < CT; c += kStepThreads) {
         float a = 0.f, b = 0.f;
 #pragma unroll
         for (int g = 0; g < RG; ++g) {
             a += s_red[g][0][c];
             b += s_red[g][1][c];
         }
-        st_val(o, bh * DV + c, a);
-        if (o_im) st_val(o_im, bh * DV + c, b);
+        st_val(o, bh * DV + c0 + c, a);
+        if (o_im) st_val(o_im, bh * DV + c0 + c, b);
     }
 }
 
 template <int DK, int DV, typename T>
 cudaError_t launch_one(const StepArgs &a, cudaStream_t stream)
 {
-    const unsigned grid = (unsigned)a.B * (unsigned)a.H;
+    const dim3 grid((unsigned)a.B * (unsigned)a.H, DV > kColTile ? DV / kColTile : 1);
     sfda_step_kernel<DK, DV, T><<<grid, kStepThreads, 0, stream>>>(
         static_cast<const T *>(a.q), static_cast<const T *>(a.k), static_cast<const T *>(a.v), a.alpha,
         a.theta, a.beta, a.S, static_cast<T *>(a.o), static_cast<T *>(a.o_im));
