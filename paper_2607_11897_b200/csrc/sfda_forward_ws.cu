@@ -711,7 +711,7 @@ __device__ __forceinline__ void cmma_tiles(float (&cr)[NRT][4], float (&ci)[NRT]
     // lane's row address for the A blocks: block m = (rows 0-7 | 8-15) x (k 0-3 | 4-7)
     uint32_t a_addr = lx + (uint32_t)(((a_row0 + r + 8 * (m & 1)) * LS + a_col0 + 8 * s0 + 4 * (m >> 1)) * 4);
     uint32_t b_addr = lx + (uint32_t)(((b_row0 + 8 * s0 + tg) * LS + b_col0 + g) * 4);
-#pragma unroll 2
+#pragma unroll 4
     for (int s = s0; s < s1b; ++s, a_addr += 32, b_addr += 8 * LS * 4) {
         uint32_t br[2], bi[2], nbi[2];
         br[0] = lds32(b_addr);
