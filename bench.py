@@ -171,6 +171,9 @@ def main():
     ap.add_argument("--re-only", action="store_true", help="write o = Re only (default: Re and Im)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--seq-len", type=int, default=0,
+                    help="sweeps only: run the headline shapes with this sequence length (use with --batch; the JSON "
+                         "line then names the changed workload and is not a benchmark value)")
     ap.add_argument("--clock-load-s", type=float, default=1.0,
                     help="seconds of untimed continuation of the same launches under the clock sampler (0: none, "
                          "for profiler runs)")
@@ -205,6 +208,8 @@ def main():
     cfg = workloads.CONFIGS[HEADLINE]
     if args.batch > 0:
         cfg = cfg.scaled(name="%s_batch%d_profiling_only" % (cfg.name, args.batch), B=args.batch)
+    if args.seq_len > 0:
+        cfg = cfg.scaled(name="%s_T%d_sweep_only" % (cfg.name, args.seq_len), T=args.seq_len)
     want_im = not args.re_only
     # every rank draws its own batch: batch elements rank*B .. rank*B + B - 1 of the same recipe
     inp = workloads.forward_inputs(cfg, batch=dp.rank_batch_range(cfg.B, rank))
@@ -340,7 +345,7 @@ def main():
         "tensor_frac": achieved_tf / peaks["bf16_tflops"],
         "roofline_ms": 1e3 * max(hbm_time, tensor_time),
     }
-    if args.batch == 0:
+    if args.batch == 0 and args.seq_len == 0:
         # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this kernel at B = 4 (1.939 GB,
         # profiles/sfda_forward_ws_kernel_batch4_ncu_full.md), scaled by the units processed (traffic grows with B)
         roofline["traffic"] = 1.939e9 * cfg.B / 4
