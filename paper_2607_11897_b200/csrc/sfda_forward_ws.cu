@@ -76,7 +76,8 @@ enum Bar {
     B_GRAM_FULL, B_GRAM_DRAINED,    // commit / SOLVE: one Gram half is in tensor memory / has been read out
     B_MB_FULL, B_AQ_FULL0, B_AQ_FULL1,
     B_D1_DONE, B_O1_DONE, B_E_DONE, B_UPD_DONE,
-    B_S16_READY, B_R16_READY, B_E16_READY, B_O_STAGED,
+    B_S16_A, B_S16_B, B_R16_A, B_R16_B, B_E16_A, B_E16_B,   // first / second half of a bf16 operand is written
+    B_O_STAGED,
     B_V_FULL,
     kNumBars
 };
@@ -291,7 +292,10 @@ __device__ __forceinline__ bool test_k_warp(Misc &mi, int bar, int k)
 // `part` selects the products of one accumulator: 0 = Re (g = 0, 1), 1 = Im (g = 2, 3), 2 = both.  The two halves
 // touch different accumulator columns, so two threads can issue them side by side (instructions of one thread
 // execute in order, which the accumulation inside a half needs; nothing orders two threads, nor has to).
-template <int kNegG, bool kFresh, bool kSwap, uint32_t kBStep>
+// kMask: the K = 16 steps to issue (bit ks); the operands arrive in two halves, and the steps that only need the
+// first half go out while the second is still being written.  With kFresh the lowest step of the mask starts the
+// accumulators from zero (so the call with kFresh has to be the first for its accumulators).
+template <int kNegG, bool kFresh, bool kSwap, uint32_t kBStep, int kMask = 15>
 __device__ __forceinline__ void issue_complex(uint32_t d_re, uint32_t d_im, uint32_t a_re, uint32_t a_im, uint32_t b_re,
                                               uint32_t b_im, uint32_t dhi, uint32_t id, int part)
 {
@@ -304,9 +308,11 @@ __device__ __forceinline__ void issue_complex(uint32_t d_re, uint32_t d_im, uint
             const uint32_t a = (kSwap ? odd : mid) ? a_im : a_re;
             const uint32_t b = (kSwap ? mid : odd) ? b_im : b_re;
             const uint32_t idg = id | (g == kNegG ? 1u << 14 : 0u);
+            constexpr int kFirst = (kMask & 1) ? 0 : (kMask & 2) ? 1 : (kMask & 4) ? 2 : 3;
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
-                mma_ts2(d, a + 8 * ks, b + kBStep * ks, dhi, idg, (!kFresh || odd || ks > 0) ? 1u : 0u);
+                if (kMask >> ks & 1)
+                    mma_ts2(d, a + 8 * ks, b + kBStep * ks, dhi, idg, (!kFresh || odd || ks != kFirst) ? 1u : 0u);
         }
     }
     __syncwarp();
@@ -362,11 +368,15 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
             const uint32_t w_re = dlo + ((OFF_WQ + s * 4 * kTile) >> 4), k_re = dlo + ((OFF_KC + s * 2 * kTile) >> 4);
             // D1 = W^* S_0 as soon as S_0 is there; rho_1 = Qt^* S_0 (the Qt rows follow the W rows in the slot's
             // tiles) once rho of the previous chunk has been read out.  Both read S_0 from the operand columns.
-            if (!wait_k_warp(mi, B_S16_READY, j)) return;
+            // (the state pass writes S_0 in two halves: key coordinates 0-15 and 32-47 = k-steps 0 and 2 first)
+            if (!wait_k_warp(mi, B_S16_A, j)) return;
             if (!wait_k_warp(mi, B_PREP_FULL0 + s, u)) return;
             tc_fence_after();
             SFDA_T(0);
-            issue_complex<3, true, false, 2>(acc, acc + 128, x_re, x_re + 32, w_re, w_re + 2 * kIm, dhi, I64, part);
+            issue_complex<3, true, false, 2, 5>(acc, acc + 128, x_re, x_re + 32, w_re, w_re + 2 * kIm, dhi, I64, part);
+            if (!wait_k_warp(mi, B_S16_B, j)) return;
+            tc_fence_after();
+            issue_complex<3, false, false, 2, 10>(acc, acc + 128, x_re, x_re + 32, w_re, w_re + 2 * kIm, dhi, I64, part);
             if (elect_one()) mma_commit(&bars[B_D1_DONE]);
             if (j > 0 && !wait_k_warp(mi, B_O_STAGED, j - 1)) return;
             tc_fence_after();
@@ -376,20 +386,26 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
                 mma_commit(&bars[B_WQ_FREE0 + s]);
             }
             SFDA_T(1);
-            // E = M_beta R
-            if (!wait_k_warp(mi, B_R16_READY, j)) return;
+            // E = M_beta R (R arrives in two halves of 32 tokens = two k-steps each)
+            if (!wait_k_warp(mi, B_R16_A, j)) return;
             SFDA_T(2);
             if (!wait_k_warp(mi, B_MB_FULL, j)) return;
             tc_fence_after();
             SFDA_T(3);
-            issue_complex<1, true, false, 2>(acc, acc + 128, x_re, x_re + 32, m_re, m_re + kIm, dhi, I64, part);
+            issue_complex<1, true, false, 2, 3>(acc, acc + 128, x_re, x_re + 32, m_re, m_re + kIm, dhi, I64, part);
+            if (!wait_k_warp(mi, B_R16_B, j)) return;
+            tc_fence_after();
+            issue_complex<1, false, false, 2, 12>(acc, acc + 128, x_re, x_re + 32, m_re, m_re + kIm, dhi, I64, part);
             if (elect_one()) mma_commit(&bars[B_E_DONE]);
             SFDA_T(4);
             // S += E^T Kc (Kc as MN-major B: rows = tokens)
-            if (!wait_k_warp(mi, B_E16_READY, j)) return;
+            if (!wait_k_warp(mi, B_E16_A, j)) return;
             tc_fence_after();
             SFDA_T(5);
-            issue_complex<1, false, true, 128>(tmem + TM_S32, tmem + TM_S32 + 64, x_re, x_re + 32, k_re, k_re + kIm, dhi, I64M, part);
+            issue_complex<1, false, true, 128, 3>(tmem + TM_S32, tmem + TM_S32 + 64, x_re, x_re + 32, k_re, k_re + kIm, dhi, I64M, part);
+            if (!wait_k_warp(mi, B_E16_B, j)) return;
+            tc_fence_after();
+            issue_complex<1, false, true, 128, 12>(tmem + TM_S32, tmem + TM_S32 + 64, x_re, x_re + 32, k_re, k_re + kIm, dhi, I64M, part);
             if (elect_one()) {
                 mma_commit(&bars[B_KC_FREE0 + s]);
                 mma_commit(&bars[B_UPD_DONE]);
@@ -420,7 +436,7 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
                 __syncwarp();
                 if (j == n_chunks) break;
             }
-            if (!wait_k_warp(mi, B_E16_READY, j)) return;
+            if (!wait_k_warp(mi, B_E16_B, j)) return;
             if (!wait_k_warp(mi, B_AQ_FULL0 + (j & 1), j >> 1)) return;
             tc_fence_after();
             const uint32_t a_re = dlo + ((OFF_AQ + (j & 1) * 2 * kTile) >> 4);
@@ -437,7 +453,7 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
         for (int i = 0; i < 2 && i < n_chunks; ++i, pcur.next(p)) prefetch_chunk(maps, pcur.ci);
 #pragma unroll 1
         for (int g = 0; g < n_chunks; ++g) {
-            if (g > 0 && !wait_k_warp(mi, B_R16_READY, g - 1)) return;
+            if (g > 0 && !wait_k_warp(mi, B_R16_B, g - 1)) return;
             {
                 const ChunkInfo cv = vcur.ci;
                 vcur.next(p);
@@ -1045,12 +1061,12 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
             tmem_st8(tlane + TM_X16 + 32 + jb / 2, pk);
             tmem_st<16>(tlane + TM_S32 + jb, sre);
             tmem_st<16>(tlane + TM_S32 + 64 + jb, sim);
+            tc_wait_st();
+            tc_fence_before();
+            warp_arrive(&mi.bars[B_S16_A + pc]);   // this half of the operand is complete
         }
         prev_ci = ci;
         cur.next(p);
-        tc_wait_st();
-        tc_fence_before();
-        warp_arrive(&mi.bars[B_S16_READY]);
         SFDA_T(11);
 
         // ---- R = V - D1 (ph 0), then E (ph 1), -> bf16 A operand: 64 fp32 accumulator columns of this warp's half
@@ -1085,10 +1101,10 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
                 // R replaces S_0 in the operand columns: rho_1, the last reader of S_0, must be done
                 if (ph == 0 && pc == 0 && !wait_k_warp(mi, B_O1_DONE, j)) return;
                 tmem_st<16>(tlane + TM_X16 + 32 * half + 16 * pc, pk);
+                tc_wait_st();
+                tc_fence_before();
+                warp_arrive(&mi.bars[(ph == 0 ? B_R16_A : B_E16_A) + pc]);   // this half of the operand is complete
             }
-            tc_wait_st();
-            tc_fence_before();
-            warp_arrive(&mi.bars[ph == 0 ? B_R16_READY : B_E16_READY]);
             SFDA_T(14 + 2 * ph);
         }
     }
@@ -1118,7 +1134,8 @@ sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
         init(B_MB_FULL, kSolveWarps); init(B_AQ_FULL0, kSolveWarps); init(B_AQ_FULL1, kSolveWarps);
         init(B_D1_DONE, 2); init(B_O1_DONE, 2); init(B_E_DONE, 2);
         init(B_UPD_DONE, 3);   // the two halves of the state update and rho += Aq E
-        init(B_S16_READY, kChainWarps); init(B_R16_READY, kChainWarps); init(B_E16_READY, kChainWarps);
+        init(B_S16_A, kChainWarps); init(B_S16_B, kChainWarps); init(B_R16_A, kChainWarps); init(B_R16_B, kChainWarps);
+        init(B_E16_A, kChainWarps); init(B_E16_B, kChainWarps);
         init(B_O_STAGED, kPrepWarps); init(B_V_FULL, 1);
         mi.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
