@@ -9,7 +9,7 @@ import os
 import numpy as np
 import pytest
 
-from oracle import bookkeeping, chunk_wy, recurrence
+from oracle import bookkeeping, chunk_wy, frontend, recurrence
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -473,3 +473,52 @@ def test_chunk_plan():
     assert bookkeeping.chunk_plan(131072, 64) == (2048, 64)
     with pytest.raises(ValueError):
         bookkeeping.chunk_plan(0, 16)
+
+
+# ----------------------------------------------------------------------------
+# stable parameterisation (paragraph "Stable parameterization", Section 3)
+# ----------------------------------------------------------------------------
+def test_parameterisation_special_values_and_ranges():
+    """Values the formulas fix by themselves: sigmoid(0) = 1/2, tanh(0) = 0, the limits, the symmetry of the
+    sigmoid, and a key of norm n mapped to norm n / (n + eps) without changing its direction."""
+    import math
+    z1, z0 = np.zeros((1, 3)), np.zeros(1)
+    k1 = np.array([[3.0, 0.0, 4.0, 0.0]])
+    al, th, be, k = frontend.stable_parameterisation(z1, z1, z0, k1, 0.2, 0.9, 2.5, 1e-3)
+    assert np.allclose(al, 0.55) and np.allclose(th, 0.0) and np.allclose(be, 0.5)
+    assert np.allclose(k, k1 / (5.0 + 1e-3), rtol=0, atol=1e-15)
+    big = np.full((1, 3), 40.0)
+    al, th, be, _ = frontend.stable_parameterisation(big, big, np.full(1, 40.0), k1, 0.2, 0.9, 2.5, 1e-3)
+    assert np.allclose(al, 0.9) and np.allclose(th, 2.5) and np.allclose(be, 1.0)
+    al, th, be, _ = frontend.stable_parameterisation(-big, -big, np.full(1, -40.0), k1, 0.2, 0.9, 2.5, 1e-3)
+    assert np.allclose(al, 0.2) and np.allclose(th, -2.5) and np.allclose(be, 0.0, atol=1e-15)
+    # against the standard library, written with other functions than the oracle uses
+    rng = np.random.default_rng(7)
+    a, b, c = rng.normal(0, 3, (5, 4)), rng.normal(0, 2, (5, 4)), rng.normal(0, 3, 5)
+    kr = rng.normal(0, 1, (5, 8))
+    al, th, be, k = frontend.stable_parameterisation(a, b, c, kr, 0.1, 1.0, math.pi, 1e-6)
+    for i in range(5):
+        for j in range(4):
+            assert math.isclose(al[i, j], 0.1 + 0.9 * 0.5 * (1.0 + math.tanh(0.5 * a[i, j])), rel_tol=1e-12)
+            assert math.isclose(th[i, j], math.pi * math.expm1(2 * b[i, j]) / (math.expm1(2 * b[i, j]) + 2.0), rel_tol=1e-12)
+        assert math.isclose(be[i] + float(frontend.sigmoid(-c[i])), 1.0, rel_tol=1e-14)
+        n = math.sqrt(sum(x * x for x in kr[i]))
+        assert math.isclose(math.sqrt(sum(x * x for x in k[i])), n / (n + 1e-6), rel_tol=1e-12)
+        assert np.allclose(k[i] * kr[i, 0], kr[i] * k[i, 0], rtol=0, atol=1e-14) and np.all(k[i] * kr[i] >= 0)   # same direction
+
+
+def test_parameterisation_gives_the_stability_assumptions():
+    """||Lambda|| <= 1, 0 <= beta ||k||^2 <= 1 (the sentence after Eq. "param-key"), on heavy-tailed raw inputs; and a
+    recurrence driven by them never grows a state beyond the bound of Prop. "Basic numerical stability"."""
+    rng = np.random.default_rng(11)
+    N, T, m, dv = 2, 40, 3, 4
+    a, b, c = rng.standard_cauchy((N, T, m)), rng.standard_cauchy((N, T, m)), rng.standard_cauchy((N, T))
+    kr = rng.standard_cauchy((N, T, 2 * m))
+    al, th, be, k = frontend.stable_parameterisation(a, b, c, kr, 0.0, 1.0, np.pi, 1e-6)
+    assert np.all((al >= 0) & (al <= 1)) and np.all(np.abs(th) <= np.pi) and np.all((be >= 0) & (be <= 1))
+    n2 = np.sum(k * k, axis=-1)
+    assert np.all(n2 <= 1.0) and np.all(be * n2 <= 1.0)
+    q, v = rng.standard_normal((N, T, 2 * m)), rng.standard_normal((N, T, dv))
+    _, _, S_T = recurrence.sfda_recurrence(q, k, v, al, th, be, None)
+    bound = np.sum(np.sqrt(be)[..., None] * np.linalg.norm(v, axis=-1)[..., None], axis=1)   # sum_t sqrt(beta_t) ||v_t||
+    assert np.all(np.linalg.norm(S_T.reshape(N, -1), axis=-1) <= bound[:, 0] + 1e-9)
