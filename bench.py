@@ -18,6 +18,7 @@ on a bounded sample of the same workload.
 """
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -171,6 +172,7 @@ def main():
     ap.add_argument("--re-only", action="store_true", help="write o = Re only (default: Re and Im)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--no-fused", action="store_true", help="skip the leg that times the forward on raw inputs")
     ap.add_argument("--seq-len", type=int, default=0,
                     help="sweeps only: run the headline shapes with this sequence length (use with --batch; the JSON "
                          "line then names the changed workload and is not a benchmark value)")
@@ -288,6 +290,51 @@ def main():
                "d2h_bytes_per_step": int(d2h), "ms_per_step": 1e3 * e2e_s}
         del arena
 
+    # The forward on raw inputs (stable parameterisation fused into the operand preparation) beside the two-step
+    # route it replaces: sfda_frontend writing alpha, theta, beta and the normalised key, then sfda_forward.
+    fused = None
+    if rank == 0 and not args.no_fused:
+        raw = workloads.forward_raw_inputs(cfg)
+        r = {}
+        for key, val in raw.items():
+            t = torch.from_numpy(np.ascontiguousarray(val))
+            r[key] = (t.to(torch.bfloat16) if key in ("q", "k_raw", "v") else t).to(dev)
+        del raw
+        par = (0.0, 1.0, math.pi, 1e-6)
+        al, th = torch.empty_like(r["a_raw"]), torch.empty_like(r["a_raw"])
+        be, kn = torch.empty_like(r["c_raw"]), torch.empty_like(r["k_raw"])
+
+        def timed(fn, n):
+            for _ in range(3):
+                fn()
+            t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            t0.record(stream)
+            for _ in range(n):
+                fn()
+            t1.record(stream)
+            torch.cuda.synchronize()
+            return t0.elapsed_time(t1) / n
+
+        fused_ms = timed(lambda: sfda.sfda_forward_fused(r["q"], r["k_raw"], r["v"], r["a_raw"], r["b_raw"],
+                                                         r["c_raw"], *par, r["S0"], o, o_im, S_T, cfg.chunk, ws,
+                                                         stream), max(args.steps, 5))
+        assert sfda.sfda_workspace_status(ws, stream) == 0
+        front_ms = timed(lambda: sfda.sfda_frontend(r["a_raw"], r["b_raw"], r["c_raw"], r["k_raw"], *par, al, th, be,
+                                                    kn, stream), max(args.steps, 5))
+        two_ms = timed(lambda: (sfda.sfda_frontend(r["a_raw"], r["b_raw"], r["c_raw"], r["k_raw"], *par, al, th, be,
+                                                   kn, stream),
+                                sfda.sfda_forward(r["q"], kn, r["v"], al, th, be, r["S0"], o, o_im, S_T, cfg.chunk,
+                                                  ws, stream)), max(args.steps, 5))
+        rows = cfg.B * cfg.T * cfg.H
+        fbytes = rows * 2 * (2 * cfg.m * 4 + 4 + cfg.d_k * 2)          # every array read once, written once
+        fused = {"workload": cfg.name + " from raw a, b, c, k (alpha in [0,1], theta_max = pi, eps = 1e-6)",
+                 "fused_ms_per_step": fused_ms, "fused_tokens_per_s": cfg.B * cfg.T / (fused_ms * 1e-3),
+                 "frontend_kernel_ms": front_ms, "frontend_bytes": fbytes,
+                 "frontend_achieved_gbs": fbytes / (front_ms * 1e-3) / 1e9,
+                 "two_step_ms_per_step": two_ms, "two_step_tokens_per_s": cfg.B * cfg.T / (two_ms * 1e-3)}
+        del r, al, th, be, kn
+
     # one-token decode (sfda_step) on the decode configuration: HBM-bound, reported beside the headline
     decode = None
     if rank == 0 and not args.no_decode:
@@ -351,6 +398,9 @@ def main():
         roofline["traffic"] = 1.939e9 * cfg.B / 4
         roofline["traffic_source"] = "ncu capture at B=4 scaled to B=%d; Re+Im outputs" % cfg.B
 
+    if fused is not None:
+        fused["frontend_frac"] = fused["frontend_achieved_gbs"] / peaks["hbm_gbs"]
+        fused["peak_source"] = "of " + peaks["source"]
     if decode is not None:
         decode["frac"] = decode["achieved_gbs"] / peaks["hbm_gbs"]
         decode["peak_source"] = "of " + peaks["source"]
@@ -370,7 +420,7 @@ def main():
                    "chunk": cfg.chunk, "outputs": "Re+Im" if want_im else "Re", "state": "fp32", "S0": "N(0,0.02)",
                    "parallelism": "dp%d over (batch, head), no collective" % world,
                    "l2": "inputs+outputs %.2f GB per step, far larger than the 126 MB L2; no flush" % (abytes / 1e9)},
-        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "decode": decode,
+        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "decode": decode, "fused_front_end": fused,
         "gpu_launches": launches_per_step * args.steps, "clocks": clocks.summary(),
     }
     print(json.dumps(line), flush=True)

@@ -63,7 +63,9 @@ typedef enum {
     SFDA_ERR_ALIGN = -4,       /* a pointer is not 16-byte aligned                    */
     SFDA_ERR_WORKSPACE = -5,   /* workspace NULL or smaller than sfda_workspace_bytes */
     SFDA_ERR_CUDA = -6,        /* the CUDA runtime reported an error at launch        */
-    SFDA_ERR_TIMEOUT = -7      /* a bounded device-side wait ran out                  */
+    SFDA_ERR_TIMEOUT = -7,     /* a bounded device-side wait ran out                  */
+    SFDA_ERR_VALUE = -8        /* a scalar of the stable parameterisation is out of   */
+                               /* range (see sfda_frontend)                           */
 } sfda_status;
 
 typedef enum { SFDA_F32 = 0, SFDA_BF16 = 1 } sfda_dtype;
@@ -231,7 +233,56 @@ SFDA_API int sfda_forward_host(const void *q, const void *k, const void *v,
                       void *arena, size_t arena_bytes, void *stream,
                       size_t *bytes_h2d, size_t *bytes_d2h);
 
-/* Number of kernels the last sfda_forward / sfda_step / sfda_chunk_factors call of
+/*
+ * Stable parameterisation (Section 3, paragraph "Stable parameterization", Eqs. "param-alpha", "param-theta",
+ * "param-beta", "param-key"): from unconstrained inputs,
+ *
+ *     alpha = alpha_min + (alpha_max - alpha_min) * sigmoid(a_raw)
+ *     theta = theta_max * tanh(b_raw)
+ *     beta  = sigmoid(c_raw)
+ *     k     = k_raw / (|k_raw|_2 + eps)          (norm over the d_k real channels of a token and head)
+ *
+ * which gives alpha in [alpha_min, alpha_max], |theta| <= theta_max, beta in [0, 1] and |k| <= 1: the
+ * preconditions of Prop. "Basic numerical stability".
+ *
+ *  a_raw, b_raw [B][T][H][m] float     c_raw [B][T][H] float     k_raw [B][T][H][d_k] dtype
+ *  alpha, theta [B][T][H][m] float     beta  [B][T][H] float     k     [B][T][H][d_k] dtype
+ *
+ * Every output may alias the input it is computed from (in-place use).  d_k in {64, 128}.
+ * Scalars: 0 <= alpha_min <= alpha_max <= 1, theta_max >= 0 and finite, eps >= 0 and finite; anything else is
+ * SFDA_ERR_VALUE.  With eps = 0 a zero key stays zero (no 0/0).  fp32 arithmetic.
+ */
+SFDA_API int sfda_frontend(const float *a_raw, const float *b_raw, const float *c_raw, const void *k_raw,
+                           float alpha_min, float alpha_max, float theta_max, float eps,
+                           float *alpha, float *theta, float *beta, void *k,
+                           int B, int T, int H, int d_k, int dtype, void *stream);
+
+/*
+ * sfda_forward on the raw inputs: the stable parameterisation above followed by the chunkwise forward, without
+ * the caller ever holding alpha, theta, beta or the normalised key.
+ *
+ * Arguments as sfda_forward, with a_raw, b_raw, c_raw, k_raw in place of alpha, theta, beta, k, and the four
+ * scalars of sfda_frontend (same ranges, SFDA_ERR_VALUE otherwise).
+ *
+ * On the tensor-core path (bf16, d_k = d_v = 128, chunk = 64) the map is applied inside the kernel and the four
+ * arrays are never written: alpha, theta and beta are transformed in the operand preparation (fast exponential
+ * and reciprocal, 2 ulp each); the key is never divided at all, because the recurrence on k = s k_raw,
+ * s = 1 / (|k_raw| + eps), is the recurrence on k_raw with beta s^2 for beta and v / s for v (Eq. "sfda"), and
+ * |k_raw|^2 is read off the diagonal of the chunk's Gram matrix, i.e. from the bf16 operands (relative error of
+ * s about 2e-4).  |k_raw| + eps below 1e-18 is treated as 1e-18; |k_raw|^2 must be finite in fp32.  The workspace
+ * is the one of sfda_forward.  Other shapes run sfda_frontend into the workspace and the CUDA-core forward from
+ * there.  sfda_forward_fused_workspace_bytes gives the size for full speed in
+ * both cases (the tensor-core path again runs with as little as 256 bytes; the other shapes need it all).
+ */
+SFDA_API size_t sfda_forward_fused_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int dtype);
+SFDA_API int sfda_forward_fused(const void *q, const void *k_raw, const void *v,
+                                const float *a_raw, const float *b_raw, const float *c_raw,
+                                float alpha_min, float alpha_max, float theta_max, float eps,
+                                const float *S0, void *o, void *o_im, float *S_T,
+                                int B, int T, int H, int d_k, int d_v, int chunk, int dtype,
+                                void *workspace, size_t workspace_bytes, void *stream);
+
+/* Number of kernels the last sfda_forward* / sfda_step / sfda_chunk_factors / sfda_frontend call of
  * this thread enqueued (host only; for launch accounting in benchmarks). */
 SFDA_API int sfda_last_launch_count(void);
 

@@ -48,6 +48,11 @@ def load():
     lib.sfda_forward_noalloc.argtypes = [_vp] * 10 + [_ci] * 7 + [_vp]
     lib.sfda_noalloc_status.argtypes = [_vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.sfda_workspace_status.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_uint32)]
+    _cf = ctypes.c_float
+    lib.sfda_frontend.argtypes = [_vp] * 4 + [_cf] * 4 + [_vp] * 4 + [_ci] * 5 + [_vp]
+    lib.sfda_forward_fused_workspace_bytes.restype = _sz
+    lib.sfda_forward_fused_workspace_bytes.argtypes = [_ci] * 7
+    lib.sfda_forward_fused.argtypes = [_vp] * 6 + [_cf] * 4 + [_vp] * 4 + [_ci] * 7 + [_vp, _sz, _vp]
     _LIB = lib
     return lib
 
@@ -215,3 +220,40 @@ def sfda_forward_host(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chunk, aren
 def sfda_forward_host_arena_bytes(B, T, H, d_k, d_v, chunk, dtype, want_o_im, have_S0, want_S_T) -> int:
     return int(load().sfda_forward_host_arena_bytes(B, T, H, d_k, d_v, chunk, dtype, int(want_o_im), int(have_S0),
                                                     int(want_S_T)))
+
+
+def sfda_frontend(a_raw, b_raw, c_raw, k_raw, alpha_min, alpha_max, theta_max, eps, alpha, theta, beta, k,
+                  stream=None):
+    """``sfda_frontend`` of ``include/sfda.h``: the stable parameterisation as a kernel of its own."""
+    B, T, H, d_k = k_raw.shape
+    _check(k_raw, "k_raw")
+    _check(k, "k", k_raw.dtype)
+    for t, n in ((a_raw, "a_raw"), (b_raw, "b_raw"), (c_raw, "c_raw"), (alpha, "alpha"), (theta, "theta"),
+                 (beta, "beta")):
+        _check(t, n, torch.float32)
+    rc = load().sfda_frontend(_ptr(a_raw), _ptr(b_raw), _ptr(c_raw), _ptr(k_raw), alpha_min, alpha_max, theta_max,
+                              eps, _ptr(alpha), _ptr(theta), _ptr(beta), _ptr(k), B, T, H, d_k,
+                              _dtype_code(k_raw), _stream(stream))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_frontend")
+
+
+def sfda_forward_fused_workspace_bytes(B, T, H, d_k, d_v, chunk, dtype) -> int:
+    return int(load().sfda_forward_fused_workspace_bytes(B, T, H, d_k, d_v, chunk, dtype))
+
+
+def sfda_forward_fused(q, k_raw, v, a_raw, b_raw, c_raw, alpha_min, alpha_max, theta_max, eps, S0, o, o_im, S_T,
+                       chunk, workspace=None, stream=None):
+    """``sfda_forward_fused`` of ``include/sfda.h``: the forward on the raw inputs of the stable parameterisation."""
+    B, T, H, d_k = q.shape
+    d_v = v.shape[-1]
+    for t, n in ((q, "q"), (k_raw, "k_raw"), (v, "v"), (o, "o"), (o_im, "o_im")):
+        _check(t, n, q.dtype)
+    for t, n in ((a_raw, "a_raw"), (b_raw, "b_raw"), (c_raw, "c_raw"), (S0, "S0"), (S_T, "S_T")):
+        _check(t, n, torch.float32)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = load().sfda_forward_fused(_ptr(q), _ptr(k_raw), _ptr(v), _ptr(a_raw), _ptr(b_raw), _ptr(c_raw), alpha_min,
+                                   alpha_max, theta_max, eps, _ptr(S0), _ptr(o), _ptr(o_im), _ptr(S_T), B, T, H,
+                                   d_k, d_v, chunk, _dtype_code(q), _ptr(workspace), ws_bytes, _stream(stream))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_forward_fused")

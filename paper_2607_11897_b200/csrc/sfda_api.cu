@@ -90,6 +90,21 @@ sfda::ForwardArgs pack(const void *q, const void *k, const void *v, const float 
 
 size_t round256(size_t x) { return (x + 255u) & ~(size_t)255u; }
 
+// the stable parameterisation's scalars: 0 <= alpha_min <= alpha_max <= 1, theta_max and eps finite and >= 0
+// (comparisons written so that a NaN fails them)
+int check_param_scalars(float alpha_min, float alpha_max, float theta_max, float eps)
+{
+    const bool ok = alpha_min >= 0.f && alpha_min <= alpha_max && alpha_max <= 1.f && theta_max >= 0.f &&
+                    theta_max <= 3.0e38f && eps >= 0.f && eps <= 3.0e38f;
+    return ok ? SFDA_OK : SFDA_ERR_VALUE;
+}
+
+// workspace of sfda_forward_fused on the CUDA-core shapes: alpha, theta, beta and the normalised key
+size_t staged_frontend_bytes(size_t rows, int d_k, int dtype)
+{
+    return 2 * round256(rows * (d_k / 2) * 4) + round256(rows * 4) + round256(rows * d_k * elem_bytes(dtype));
+}
+
 }  // namespace
 
 extern "C" {
@@ -105,6 +120,7 @@ const char *sfda_status_string(int status)
         case SFDA_ERR_WORKSPACE: return "workspace missing or too small";
         case SFDA_ERR_CUDA: return "CUDA runtime error at launch";
         case SFDA_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case SFDA_ERR_VALUE: return "a scalar of the stable parameterisation is out of range";
         default: return "unknown status";
     }
 }
@@ -331,6 +347,73 @@ int sfda_forward_host(const void *q, const void *k, const void *v, const float *
     if (bytes_h2d) *bytes_h2d = h2d;
     if (bytes_d2h) *bytes_d2h = d2h;
     return ok ? SFDA_OK : SFDA_ERR_CUDA;
+}
+
+int sfda_frontend(const float *a_raw, const float *b_raw, const float *c_raw, const void *k_raw, float alpha_min,
+                  float alpha_max, float theta_max, float eps, float *alpha, float *theta, float *beta, void *k,
+                  int B, int T, int H, int d_k, int dtype, void *stream)
+{
+    g_last_launches = 0;
+    if (!a_raw || !b_raw || !c_raw || !k_raw || !alpha || !theta || !beta || !k) return SFDA_ERR_NULL;
+    if (B < 1 || T < 1 || H < 1) return SFDA_ERR_SHAPE;
+    int rc = check_dims(d_k, 64, 64, dtype);
+    if (rc != SFDA_OK) return rc;
+    if ((rc = check_param_scalars(alpha_min, alpha_max, theta_max, eps)) != SFDA_OK) return rc;
+    const void *ptrs[] = {a_raw, b_raw, c_raw, k_raw, alpha, theta, beta, k};
+    for (const void *p : ptrs)
+        if (!aligned16(p)) return SFDA_ERR_ALIGN;
+    sfda::FrontendArgs f;
+    f.a_raw = a_raw; f.b_raw = b_raw; f.c_raw = c_raw; f.k_raw = k_raw;
+    f.alpha = alpha; f.theta = theta; f.beta = beta; f.k = k;
+    f.rows = (long long)B * T * H; f.d_k = d_k; f.dtype = dtype;
+    f.alpha_min = alpha_min; f.alpha_max = alpha_max; f.theta_max = theta_max; f.eps = eps;
+    return sfda::launch_frontend(f, static_cast<cudaStream_t>(stream), &g_last_launches) == cudaSuccess ? SFDA_OK
+                                                                                                         : SFDA_ERR_CUDA;
+}
+
+size_t sfda_forward_fused_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int dtype)
+{
+    if (B < 1 || T < 1 || H < 1 || check_dims(d_k, d_v, chunk, dtype) != SFDA_OK) return 0;
+    sfda::ForwardArgs a{};
+    a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.chunk = chunk; a.dtype = dtype;
+    if (sfda::forward_ws_supported(a)) return sfda::forward_ws_scratch_bytes(B, H);
+    return staged_frontend_bytes((size_t)B * T * H, d_k, dtype);
+}
+
+int sfda_forward_fused(const void *q, const void *k_raw, const void *v, const float *a_raw, const float *b_raw,
+                       const float *c_raw, float alpha_min, float alpha_max, float theta_max, float eps,
+                       const float *S0, void *o, void *o_im, float *S_T, int B, int T, int H, int d_k, int d_v,
+                       int chunk, int dtype, void *workspace, size_t workspace_bytes, void *stream)
+{
+    g_last_launches = 0;
+    int rc = validate_forward(q, k_raw, v, a_raw, b_raw, c_raw, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
+    if (rc != SFDA_OK) return rc;
+    if ((rc = check_param_scalars(alpha_min, alpha_max, theta_max, eps)) != SFDA_OK) return rc;
+    if (workspace && !aligned16(workspace)) return SFDA_ERR_ALIGN;
+    sfda::ForwardArgs a = pack(q, k_raw, v, a_raw, b_raw, c_raw, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (sfda::forward_ws_supported(a)) {
+        if (!workspace || workspace_bytes < sfda::kWsMinScratchBytes) return SFDA_ERR_WORKSPACE;
+        a.fused = 1;
+        a.alpha_min = alpha_min; a.alpha_max = alpha_max; a.theta_max = theta_max; a.eps = eps;
+        return sfda::launch_forward_ws(a, workspace, workspace_bytes, s, &g_last_launches) == cudaSuccess ? SFDA_OK
+                                                                                                          : SFDA_ERR_CUDA;
+    }
+    // other shapes: the parameterisation as a kernel of its own into the workspace, then the CUDA-core forward
+    const size_t rows = (size_t)B * T * H;
+    if (!workspace || workspace_bytes < staged_frontend_bytes(rows, d_k, dtype)) return SFDA_ERR_WORKSPACE;
+    char *w = static_cast<char *>(workspace);
+    sfda::FrontendArgs f;
+    f.a_raw = a_raw; f.b_raw = b_raw; f.c_raw = c_raw; f.k_raw = k_raw;
+    f.alpha = reinterpret_cast<float *>(w);
+    f.theta = reinterpret_cast<float *>(w + round256(rows * (d_k / 2) * 4));
+    f.beta = reinterpret_cast<float *>(w + 2 * round256(rows * (d_k / 2) * 4));
+    f.k = w + 2 * round256(rows * (d_k / 2) * 4) + round256(rows * 4);
+    f.rows = (long long)rows; f.d_k = d_k; f.dtype = dtype;
+    f.alpha_min = alpha_min; f.alpha_max = alpha_max; f.theta_max = theta_max; f.eps = eps;
+    if (sfda::launch_frontend(f, s, &g_last_launches) != cudaSuccess) return SFDA_ERR_CUDA;
+    a.alpha = f.alpha; a.theta = f.theta; a.beta = f.beta; a.k = f.k;
+    return sfda::launch_forward_simt(a, s, &g_last_launches) == cudaSuccess ? SFDA_OK : SFDA_ERR_CUDA;
 }
 
 int sfda_last_launch_count(void) { return g_last_launches; }

@@ -79,6 +79,7 @@ enum Bar {
     B_S16_A, B_S16_B, B_R16_A, B_R16_B, B_E16_A, B_E16_B,   // first / second half of a bf16 operand is written
     B_O_STAGED,
     B_V_FULL,
+    B_NORM_FULL,                    // SOLVE -> CHAIN (fused front end): the chunk's key scales are written
     kNumBars
 };
 
@@ -87,6 +88,8 @@ struct Misc {
     uint32_t part_turns[2][8][M];
     float2 close[4][M];                     // a_C e^{i phi_C} of a ring of four chunks
     float beta[4][C];
+    float kscale[4][C];                     // fused front end: -1 / (|k_raw| + eps) per token, ring of four chunks
+    float ones[C];                          //                  +1: the scale of the passes that apply none
     unsigned long long bars[kNumBars];
     uint32_t tmem_base;
     volatile int abort;
@@ -129,6 +132,9 @@ struct Params {
     int T, H, has_o_im;
     int BH, U, Q, n_units;   // sequences, chunks per work unit, time slices per sequence, Q * BH
     uint32_t magic_BH, magic_H;   // floor(2^32 / d) + 1 (0 for d = 1): quotients by multiplication
+    // fused stable parameterisation (only read by the kFused instantiation): alpha = a_lo + a_range sigmoid(a),
+    // theta = th_max tanh(b), beta = sigmoid(c), k = k_raw / (|k_raw| + eps)
+    float a_lo, a_range, th_max, th_m2, eps;   // th_m2 = -2 th_max
 };
 
 // Tensor maps of the arrays the copy engine touches: [B][T][H][128] bf16 (v, o, o_im, q, k) or [B][T][H][64] fp32
@@ -510,6 +516,33 @@ __device__ __forceinline__ uint32_t turns_f32(float theta)
     return (uint32_t)(unsigned long long)__float2ll_rn(theta * 683565275.6f);
 }
 
+// Stable parameterisation (Section 3, Eqs. "param-alpha", "param-theta", "param-beta") from raw fp32 bits, five
+// instructions each: sigmoid(x) = 1 / (1 + 2^(-x log2 e)), tanh(x) = 1 - 2 / (1 + 2^(2 x log2 e)), with the
+// approximate (2 ulp) exponential and reciprocal of the special-function unit in their flush-to-zero forms, which
+// are single instructions.  Both saturate correctly: the exponential overflows to infinity, whose reciprocal is
+// zero, or flushes to zero.
+__device__ __forceinline__ float rcp1p_ex2(float y)   // 1 / (1 + 2^y)
+{
+    float e, r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(y));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
+    return r;
+}
+__device__ __forceinline__ float alpha_from_raw(const Params &p, uint32_t bits)
+{
+    return fmaf(p.a_range, rcp1p_ex2(__uint_as_float(bits) * -1.4426950408889634f), p.a_lo);
+}
+__device__ __forceinline__ float theta_from_raw(const Params &p, uint32_t bits)
+{
+    return fmaf(p.th_m2, rcp1p_ex2(__uint_as_float(bits) * 2.8853900817779268f), p.th_max);
+}
+
+// kFused: alpha, theta and beta arrive raw and go through the stable parameterisation here, on the way into the
+// operands.  The key is NOT normalised here: with s_t = 1 / (|k_raw,t| + eps), the recurrence on k = s k_raw is the
+// recurrence on k_raw itself with beta s^2 in place of beta and v / s in place of v, so the operands carry the raw
+// key and the scales enter where beta and v do (SOLVE and CHAIN); |k_raw,t|^2 is the diagonal of the chunk's Gram
+// matrix, which the tensor core computes anyway.
+template <bool kFused>
 __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int n_chunks, int pt)
 {
     long long *timing = p.timing;
@@ -601,16 +634,31 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
             // beta of token pt: fetched now, written after the pass below so that its latency is covered
             float beta_t = 0.f;
             if (pt < len) beta_t = __ldg(p.beta + row0 + (size_t)pt * p.H);
+            if (kFused && pt < len) beta_t = rcp1p_ex2(beta_t * -1.4426950408889634f);
             SFDA_T(37);
             {
                 float a0 = 1.f, a1 = 1.f;
                 uint32_t u0 = 0u, u1 = 0u;
+                float rs0 = 0.f, rs1 = 0.f;      // fused: sum of 1 / (1 + e^{2b}) over the octet's real tokens
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
+                    if (kFused) {   // beyond the sequence the defaults are not raw values: skipped, i.e. neutral
+                        if (i < nt) {
+                            a0 *= fmaxf(alpha_from_raw(p, al[i].x), 9.0e-14f);
+                            a1 *= fmaxf(alpha_from_raw(p, al[i].y), 9.0e-14f);
+                            rs0 += rcp1p_ex2(__uint_as_float(th[i].x) * 2.8853900817779268f);
+                            rs1 += rcp1p_ex2(__uint_as_float(th[i].y) * 2.8853900817779268f);
+                        }
+                        continue;
+                    }
                     a0 *= fmaxf(__uint_as_float(al[i].x), 9.0e-14f);           // floor e^-30, as in log_decay
                     a1 *= fmaxf(__uint_as_float(al[i].y), 9.0e-14f);
                     u0 += turns_f32(__uint_as_float(th[i].x));
                     u1 += turns_f32(__uint_as_float(th[i].y));
+                }
+                if (kFused) {   // sum of theta_max tanh(b) = theta_max (n - 2 sum r): at most 8 theta_max, one rounding
+                    u0 = turns_f32(fmaf(p.th_m2, rs0, p.th_max * (float)nt));
+                    u1 = turns_f32(fmaf(p.th_m2, rs1, p.th_max * (float)nt));
                 }
                 *reinterpret_cast<float2 *>(&mi.part_lg[s][tq][2 * jp]) = make_float2(a0, a1);
                 *reinterpret_cast<uint2 *>(&mi.part_turns[s][tq][2 * jp]) = make_uint2(u0, u1);
@@ -674,9 +722,10 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
 #pragma unroll
                 for (int x = 0; x < 2; ++x) {
                     // gamma_t = gamma_{t-1} alpha_t e^{i theta_t}; 1/a_t alongside (capped at e^80)
-                    const float al = fmaxf(__uint_as_float(x ? tk[ii].al.y : tk[ii].al.x), 9.0e-14f);   // floor e^-30
+                    const uint32_t al_bits = x ? tk[ii].al.y : tk[ii].al.x, th_bits = x ? tk[ii].th.y : tk[ii].th.x;
+                    const float al = fmaxf(kFused ? alpha_from_raw(p, al_bits) : __uint_as_float(al_bits), 9.0e-14f);   // floor e^-30
                     float cs, sn;
-                    __sincosf(__uint_as_float(x ? tk[ii].th.y : tk[ii].th.x), &sn, &cs);
+                    __sincosf(kFused ? theta_from_raw(p, th_bits) : __uint_as_float(th_bits), &sn, &cs);
                     float2 &g = x ? g1 : g0;
                     float &ainv = x ? ainv1 : ainv0;
                     const float lr_ = al * cs, li_ = al * sn;
@@ -769,6 +818,11 @@ __device__ __forceinline__ void store_tile_s(const float (&cr)[4], const float (
     sts64(o + kIm + 8 * LS * 4, __float_as_uint(scale * ci[2]), __float_as_uint(scale * ci[3]));
 }
 
+// kFused: the diagonal of the Gram matrix is |k_raw,t|^2 (conj(W) Kc = |k|^2 whatever gamma is); the thread that
+// drains Kt row t turns it into s_t = 1 / (|k_raw,t| + eps), scales its row of L by beta_t s_t^2, and leaves
+// beta_t s_t (the column scale of the M operand, which then maps the normalised R to E / s) and -s_t (for CHAIN's
+// R = v - s W_raw^* S_0) in shared memory.
+template <bool kFused>
 __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int n_chunks, int st)
 {
     long long *timing = p.timing;
@@ -787,23 +841,46 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
         // so the warps that hold them wait for that store first.
         if (row >= 64 && j >= 2 && !dead && !wait_k(mi, B_STORE_DONE0 + s, (j >> 1) - 1)) dead = true;
         // ---- drain the two Gram halves (Re, then Im), 32 columns at a time
+        float bt = 0.f;                           // beta of this thread's Kt row (PREP wrote it before the Gram ran)
 #pragma unroll 1
         for (int im = 0; im < 2; ++im) {
             SFDA_T(20 + 2 * im);
             if (!dead && !wait_k(mi, B_GRAM_FULL, 2 * j + im)) dead = true;
             tc_fence_after();
+            if (im == 0 && row < 64) bt = mi.beta[ring][row];
             SFDA_T(21 + 2 * im);
 #pragma unroll 1
-            for (int hc = 0; hc < 2; ++hc) {
+            for (int it = 0; it < 2; ++it) {
+                // fused: the piece that holds this warp's diagonal entries of Re Kt comes first
+                const bool diag = kFused && im == 0 && it == 0 && row < 64;
+                const int hc = (kFused && im == 0 && w == 1) ? 1 - it : it;
                 uint32_t r[32];
                 tmem_ld<32>(tlane + TM_GRAM + 32 * hc, r);
                 tc_wait_ld();
-                if (hc == 1) {
+                if (it == 1) {
                     tc_fence_before();
                     warp_arrive(&mi.bars[B_GRAM_DRAINED]);
                 }
+                if (diag) {                        // r[lane] by a select tree on the lane's bits
+                    uint32_t d[16];
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) d[x] = (lane & 16) ? r[16 + x] : r[x];
+#pragma unroll
+                    for (int x = 0; x < 8; ++x) d[x] = (lane & 8) ? d[8 + x] : d[x];
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) d[x] = (lane & 4) ? d[4 + x] : d[x];
+#pragma unroll
+                    for (int x = 0; x < 2; ++x) d[x] = (lane & 2) ? d[2 + x] : d[x];
+                    float n = fmaxf(__uint_as_float((lane & 1) ? d[1] : d[0]), 0.f), sc;
+                    asm("sqrt.approx.ftz.f32 %0, %0;" : "+f"(n));
+                    // (|k_raw| + eps below 1e-18 counts as 1e-18: s^2 stays finite, and a zero key stays a zero key)
+                    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(sc) : "f"(fmaxf(n + p.eps, 1.0e-18f)));
+                    mi.kscale[ring][row] = -sc;
+                    mi.beta[ring][row] = bt * sc;
+                    bt = bt * sc * sc;
+                    warp_arrive(&mi.bars[B_NORM_FULL]);
+                }
                 if (row < 64) {                   // L = D_beta Kt, strictly lower
-                    const float bt = mi.beta[ring][row];
                     const uint32_t dst = lx + im * kIm + (uint32_t)((row * LS + 32 * hc) * 4);
                     // no mask: the substitution reads only entries below the diagonal of an 8x8 block and then
                     // overwrites the whole block; the merges read whole blocks strictly below the diagonal
@@ -949,6 +1026,7 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
 }
 
 // ---- CHAIN --------------------------------------------------------------------------------------------
+template <bool kFused>
 __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int n_chunks, int ct)
 {
     long long *timing = p.timing;
@@ -1084,9 +1162,13 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
             SFDA_T(13 + 2 * ph);
             const bool sub_v = ph == 0 && half == 0;            // R_re = V - D1_re
             const float sgn = ph == 0 ? -1.f : 1.f;             // R_im = -D1_im
+            // fused: D1 was formed with the raw key, R = V - s D1; the per-token factor replaces the sign
+            if (kFused && ph == 0 && !wait_k_warp(mi, B_NORM_FULL, j)) return;
+            const uint32_t scp = smem_u32(ph == 0 ? &mi.kscale[(j & 3)][0] : &mi.ones[0]);
 #pragma unroll 1
             for (int pc = 0; pc < 2; ++pc) {       // 32 columns per tensor-memory round trip
                 uint32_t r[32], pk[16];
+                uint4 sc4 = make_uint4(0u, 0u, 0u, 0u);
                 tmem_ld<32>(tlane + TM_ACC + 128 * half + 32 * pc, r);
                 tc_wait_ld();
 #pragma unroll
@@ -1096,7 +1178,13 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
                         v0 = __uint_as_float((uint32_t)lds16(sv + (32 * pc + 2 * i) * 2 * DV) << 16);
                         v1 = __uint_as_float((uint32_t)lds16(sv + (32 * pc + 2 * i + 1) * 2 * DV) << 16);
                     }
-                    pk[i] = pack_bf16(fmaf(sgn, __uint_as_float(r[2 * i]), v0), fmaf(sgn, __uint_as_float(r[2 * i + 1]), v1));
+                    float s0 = sgn, s1 = sgn;
+                    if (kFused) {
+                        if ((i & 1) == 0) sc4 = lds128(scp + (32 * pc + 2 * i) * 4);
+                        s0 = __uint_as_float((i & 1) ? sc4.z : sc4.x);
+                        s1 = __uint_as_float((i & 1) ? sc4.w : sc4.y);
+                    }
+                    pk[i] = pack_bf16(fmaf(s0, __uint_as_float(r[2 * i]), v0), fmaf(s1, __uint_as_float(r[2 * i + 1]), v1));
                 }
                 // R replaces S_0 in the operand columns: rho_1, the last reader of S_0, must be done
                 if (ph == 0 && pc == 0 && !wait_k_warp(mi, B_O1_DONE, j)) return;
@@ -1111,6 +1199,7 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
 }
 
 // ---- the kernel ---------------------------------------------------------------------------------------
+template <bool kFused>
 __global__ void __launch_bounds__(kThreads, 1)
 sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
 {
@@ -1136,10 +1225,11 @@ sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
         init(B_UPD_DONE, 3);   // the two halves of the state update and rho += Aq E
         init(B_S16_A, kChainWarps); init(B_S16_B, kChainWarps); init(B_R16_A, kChainWarps); init(B_R16_B, kChainWarps);
         init(B_E16_A, kChainWarps); init(B_E16_B, kChainWarps);
-        init(B_O_STAGED, kPrepWarps); init(B_V_FULL, 1);
+        init(B_O_STAGED, kPrepWarps); init(B_V_FULL, 1); init(B_NORM_FULL, 2);
         mi.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (kFused && tid < C) mi.ones[tid] = 1.0f;
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&mi.tmem_base)));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
@@ -1151,13 +1241,13 @@ sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
 
     if (warp < kChainWarps) {
         regs_inc<kRegsWork>();
-        run_chain(smem, mi, tmem, p, n_chunks, tid);
+        run_chain<kFused>(smem, mi, tmem, p, n_chunks, tid);
     } else if (warp < kChainWarps + kSolveWarps) {
         regs_inc<kRegsWork>();
-        run_solve(smem, mi, tmem, p, n_chunks, tid - kChainThreads);
+        run_solve<kFused>(smem, mi, tmem, p, n_chunks, tid - kChainThreads);
     } else if (warp < kChainWarps + kSolveWarps + kPrepWarps) {
         regs_inc<kRegsWork>();
-        run_prep(smem, mi, tmem, p, n_chunks, tid - kChainThreads - kSolveThreads);
+        run_prep<kFused>(smem, mi, tmem, p, n_chunks, tid - kChainThreads - kSolveThreads);
     } else {
         regs_dec<kRegsCtrl>();
         const int cw = warp - (kChainWarps + kSolveWarps + kPrepWarps);
@@ -1286,7 +1376,9 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
         !make_map(&maps.k, a.k, a.B, a.T, a.H) || !make_map(&maps.al, a.alpha, a.B, a.T, a.H, true) ||
         !make_map(&maps.th, a.theta, a.B, a.T, a.H, true))
         return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(sfda_forward_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    const bool fused = a.fused != 0;
+    cudaError_t e = fused ? cudaFuncSetAttribute(sfda_forward_ws_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)
+                          : cudaFuncSetAttribute(sfda_forward_ws_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     int dev = 0, n_sm = 0;
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
@@ -1337,7 +1429,15 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
     p.magic_H = a.H > 1 ? (uint32_t)(0x100000000ull / (unsigned)a.H) + 1u : 0u;
     g_ws_last_slices = Q;
     const unsigned grid = (unsigned)(p.n_units < n_sm ? p.n_units : n_sm);
-    sfda_forward_ws_kernel<<<grid, kThreads, kSmemBytes, stream>>>(maps, p);
+    p.a_lo = a.alpha_min;
+    p.a_range = a.alpha_max - a.alpha_min;
+    p.th_max = a.theta_max;
+    p.th_m2 = -2.0f * a.theta_max;
+    p.eps = a.eps;
+    if (fused)
+        sfda_forward_ws_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(maps, p);
+    else
+        sfda_forward_ws_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(maps, p);
     e = cudaGetLastError();
     if (e == cudaSuccess && launches) ++*launches;
     return e;

@@ -12,6 +12,10 @@ struct ForwardArgs {
     void *o, *o_im;
     float *S_T;
     int B, T, H, d_k, d_v, chunk, dtype;
+    // fused == 1 (tensor-core path only): alpha, theta, beta and k hold the raw inputs of the stable
+    // parameterisation, which the kernel applies with these constants on the way in
+    int fused = 0;
+    float alpha_min = 0.f, alpha_max = 1.f, theta_max = 0.f, eps = 0.f;
 };
 
 struct FactorArgs {
@@ -28,6 +32,16 @@ struct StepArgs {
     float *S;
     void *o, *o_im;
     int B, H, d_k, d_v, dtype;
+};
+
+struct FrontendArgs {
+    const float *a_raw, *b_raw, *c_raw;
+    const void *k_raw;
+    float *alpha, *theta, *beta;
+    void *k;
+    long long rows;      // B * T * H
+    int d_k, dtype;
+    float alpha_min, alpha_max, theta_max, eps;
 };
 
 // Each returns a cudaError_t from configuring / launching; *launches is incremented per kernel.
@@ -49,5 +63,7 @@ cudaError_t launch_forward_ws_static(const ForwardArgs &a, cudaStream_t stream, 
 cudaError_t read_static_status(cudaStream_t stream, uint32_t *word);
 cudaError_t launch_chunk_factors(const FactorArgs &a, cudaStream_t stream, int *launches);
 cudaError_t launch_step(const StepArgs &a, cudaStream_t stream, int *launches);
+// Stable parameterisation as a kernel of its own (every supported d_k and dtype).
+cudaError_t launch_frontend(const FrontendArgs &a, cudaStream_t stream, int *launches);
 
 }  // namespace sfda

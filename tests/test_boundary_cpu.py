@@ -41,8 +41,8 @@ def test_plan_matches_integer_bookkeeping(lib):
 
 
 def test_status_strings(lib):
-    seen = {sfda.sfda_status_string(c) for c in range(0, -8, -1)}
-    assert len(seen) == 8 and "ok" in seen
+    seen = {sfda.sfda_status_string(c) for c in range(0, -9, -1)}
+    assert len(seen) == 9 and "ok" in seen
     assert sfda.sfda_status_string(-99) == "unknown status"
 
 
@@ -81,6 +81,61 @@ def test_argument_validation_happens_before_any_launch(lib):
     n = lib.sfda_forward_host_arena_bytes(1, 64, 1, 128, 128, 64, 1, 1, 1, 1)
     assert n >= 64 * (3 * 256 + 2 * 256 + 4 + 2 * 256) + 65536
     assert lib.sfda_forward_host_arena_bytes(1, 64, 1, 100, 128, 64, 1, 1, 1, 1) == 0
+
+
+def test_stable_parameterisation_entry_points_validate_on_the_host(lib):
+    vp, ci, cf = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+    ok = vp(0x1000)
+
+    def front(ptrs, scal, dims):
+        return lib.sfda_frontend(*ptrs[:4], *[cf(x) for x in scal], *ptrs[4:], *[ci(d) for d in dims], None)
+
+    ptrs, scal, dims = [ok] * 8, [0.0, 1.0, 3.0, 1e-6], [1, 8, 1, 128, 1]
+    assert front(ptrs[:3] + [None] + ptrs[4:], scal, dims) == -1
+    assert front(ptrs, scal, [1, 0, 1, 128, 1]) == -2
+    assert front(ptrs, scal, [1, 8, 1, 96, 1]) == -3
+    assert front(ptrs, scal, [1, 8, 1, 128, 5]) == -3
+    assert front([vp(0x1008)] + ptrs[1:], scal, dims) == -4
+    for bad in ([-0.1, 1.0, 3.0, 0.0], [0.6, 0.5, 3.0, 0.0], [0.0, 1.5, 3.0, 0.0], [0.0, 1.0, -1.0, 0.0],
+                [0.0, 1.0, 3.0, -1e-6], [float("nan"), 1.0, 3.0, 0.0], [0.0, 1.0, float("inf"), 0.0],
+                [0.0, 1.0, 3.0, float("nan")]):
+        assert front(ptrs, bad, dims) == -8, bad
+
+    def fused(ptrs, scal, dims, ws=vp(0x2000), ws_bytes=1 << 30):
+        return lib.sfda_forward_fused(*ptrs[:6], *[cf(x) for x in scal], *ptrs[6:], *[ci(d) for d in dims], ws,
+                                      ctypes.c_size_t(ws_bytes), None)
+
+    fptrs, fdims = [ok] * 6 + [None, ok, None, None], [1, 64, 1, 128, 128, 64, 1]
+    assert fused([None] + fptrs[1:], scal, fdims) == -1
+    assert fused(fptrs, scal, [1, 64, 0, 128, 128, 64, 1]) == -2
+    assert fused(fptrs, scal, [1, 64, 1, 128, 96, 64, 1]) == -3
+    assert fused(fptrs, [0.0, 2.0, 3.0, 0.0], fdims) == -8
+    assert fused(fptrs, scal, fdims, ws=None, ws_bytes=0) == -5
+    assert fused(fptrs, scal, [1, 64, 1, 64, 64, 16, 0], ws_bytes=1024) == -5      # staging does not fit
+    # workspace sizes: the tensor-core shape needs what sfda_forward needs; other shapes stage alpha, theta,
+    # beta and the normalised key (each rounded up to 256 bytes)
+    assert sfda.sfda_forward_fused_workspace_bytes(8, 8192, 32, 128, 128, 64, 1) == \
+        sfda.sfda_workspace_bytes(8, 8192, 32, 128, 128, 64, 1)
+    rows = 2 * 70 * 3
+    r256 = lambda x: (x + 255) // 256 * 256
+    assert sfda.sfda_forward_fused_workspace_bytes(2, 70, 3, 64, 64, 16, 0) == \
+        2 * r256(rows * 32 * 4) + r256(rows * 4) + r256(rows * 64 * 4)
+    assert sfda.sfda_forward_fused_workspace_bytes(2, 70, 3, 64, 64, 16, 1) == \
+        2 * r256(rows * 32 * 4) + r256(rows * 4) + r256(rows * 64 * 2)
+    assert sfda.sfda_forward_fused_workspace_bytes(2, 70, 3, 60, 64, 16, 1) == 0
+
+
+def test_raw_input_generator_is_deterministic_and_untransformed():
+    cfg = workloads.CONFIGS[1].scaled(B=2, T=64, H=2, s0_std=0.02)
+    a, b = workloads.forward_raw_inputs(cfg), workloads.forward_raw_inputs(cfg)
+    for key in a:
+        assert np.array_equal(a[key], b[key])
+    assert np.array_equal(workloads.forward_raw_inputs(cfg, batch=[1])["k_raw"][0], a["k_raw"][1])
+    for key in ("q", "k_raw", "v"):
+        assert np.array_equal(workloads.bf16_round(a[key]), a[key])
+    n = np.linalg.norm(a["k_raw"].astype(np.float64), axis=-1)
+    assert n.min() > 1.0 and n.max() / n.min() > 3.0                 # unnormalised, of varying length
+    assert abs(a["a_raw"].mean() - 3.0) < 0.1 and a["b_raw"].std() > 1.3 and (a["c_raw"] < 0).any()
 
 
 def test_missing_library_fails_loudly(monkeypatch):

@@ -12,7 +12,7 @@ import torch
 
 import paper_2607_11897_b200 as sfda
 import workloads
-from oracle import bookkeeping, chunk_wy, recurrence
+from oracle import bookkeeping, chunk_wy, frontend, recurrence
 
 pytestmark = pytest.mark.gpu
 
@@ -421,3 +421,168 @@ def test_argument_errors_launch_nothing():
         sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], None, o[..., 1:].reshape(-1)[1:33],
                           None, None, 16)
     assert e.value.status == -4
+
+
+# ------------------------------------------------------------------------------------------------
+# stable parameterisation: as a kernel of its own, and fused into the forward
+# ------------------------------------------------------------------------------------------------
+PARAM = dict(alpha_min=0.0, alpha_max=1.0, theta_max=float(np.pi), eps=1e-6)
+
+
+def raw_to_dev(raw, cfg):
+    d = {}
+    for key, x in raw.items():
+        if x is None:
+            d[key] = None
+            continue
+        t = torch.from_numpy(np.ascontiguousarray(x)).to(DEV)
+        if key in ("q", "k_raw", "v") and cfg.dtype == "bf16":
+            t = t.to(torch.bfloat16)
+        d[key] = t
+    return d
+
+
+@pytest.mark.parametrize("d_k,dtype,rows", [(128, "bf16", (2, 37, 3)), (64, "bf16", (1, 130, 2)),
+                                            (128, "f32", (1, 65, 5)), (64, "f32", (3, 1, 1))])
+@pytest.mark.parametrize("par", [PARAM, dict(alpha_min=0.25, alpha_max=0.875, theta_max=0.5, eps=0.0)])
+def test_frontend_matches_oracle(d_k, dtype, rows, par):
+    B, T, H = rows
+    cfg = workloads.CONFIGS[0].scaled(name="fe", B=B, T=T, H=H, d_k=d_k, d_v=64, dtype=dtype, seed=40 + d_k)
+    raw = workloads.forward_raw_inputs(cfg)
+    raw["a_raw"][0, 0, 0, :4] = [-100.0, 100.0, -20.0, 20.0]        # saturation of the sigmoid
+    raw["b_raw"][0, 0, 0, :4] = [-50.0, 50.0, 0.0, 1e-4]            # and of tanh; tanh near zero
+    raw["c_raw"][0, 0, 0] = -90.0
+    d = raw_to_dev(raw, cfg)
+    al, th = torch.empty_like(d["a_raw"]), torch.empty_like(d["a_raw"])
+    be, k = torch.empty_like(d["c_raw"]), torch.empty_like(d["k_raw"])
+    sfda.sfda_frontend(d["a_raw"], d["b_raw"], d["c_raw"], d["k_raw"], par["alpha_min"], par["alpha_max"],
+                       par["theta_max"], par["eps"], al, th, be, k)
+    torch.cuda.synchronize()
+    assert sfda.last_launch_count() == 1
+    w_al, w_th, w_be, w_k = frontend.stable_parameterisation(raw["a_raw"], raw["b_raw"], raw["c_raw"], raw["k_raw"],
+                                                             **par)
+    # fp32 evaluation of exp / tanh / sqrt: a few ulp of the result's scale
+    assert np.abs(al.cpu().numpy() - w_al).max() <= 1e-6
+    assert np.abs(th.cpu().numpy() - w_th).max() <= 1e-6 * max(par["theta_max"], 1.0)
+    assert np.abs(be.cpu().numpy() - w_be).max() <= 1e-6
+    k_tol = 2.0 ** -8 if dtype == "bf16" else 1e-6                  # one bf16 rounding of values <= 1
+    assert np.abs(k.float().cpu().numpy() - w_k).max() <= k_tol * np.abs(w_k).max()
+    # in place
+    sfda.sfda_frontend(d["a_raw"], d["b_raw"], d["c_raw"], d["k_raw"], par["alpha_min"], par["alpha_max"],
+                       par["theta_max"], par["eps"], d["a_raw"], d["b_raw"], d["c_raw"], d["k_raw"])
+    torch.cuda.synchronize()
+    assert torch.equal(d["a_raw"], al) and torch.equal(d["b_raw"], th) and torch.equal(d["c_raw"], be)
+    assert torch.equal(d["k_raw"], k)
+
+
+def test_frontend_zero_key_with_zero_eps_stays_zero():
+    cfg = workloads.CONFIGS[0].scaled(name="fe0", B=1, T=8, H=2, d_k=128, dtype="bf16", seed=5)
+    raw = workloads.forward_raw_inputs(cfg)
+    raw["k_raw"][0, 3, 1] = 0.0
+    d = raw_to_dev(raw, cfg)
+    sfda.sfda_frontend(d["a_raw"], d["b_raw"], d["c_raw"], d["k_raw"], 0.0, 1.0, 1.0, 0.0, d["a_raw"], d["b_raw"],
+                       d["c_raw"], d["k_raw"])
+    torch.cuda.synchronize()
+    k = d["k_raw"].float().cpu().numpy()
+    assert np.isfinite(k).all() and np.all(k[0, 3, 1] == 0.0)
+
+
+def run_forward_fused(cfg, raw, par, want_im=True, want_state=True):
+    d = raw_to_dev(raw, cfg)
+    B, T, H = d["q"].shape[:3]
+    o = torch.empty(B, T, H, cfg.d_v, device=DEV, dtype=d["q"].dtype)
+    o_im = torch.empty_like(o) if want_im else None
+    S_T = torch.empty(B, H, cfg.d_k, cfg.d_v, device=DEV, dtype=torch.float32) if want_state else None
+    ws_bytes = sfda.sfda_forward_fused_workspace_bytes(B, T, H, cfg.d_k, cfg.d_v, cfg.chunk,
+                                                       1 if cfg.dtype == "bf16" else 0)
+    assert ws_bytes > 0
+    ws = torch.empty(ws_bytes, device=DEV, dtype=torch.uint8)
+    sfda.sfda_forward_fused(d["q"], d["k_raw"], d["v"], d["a_raw"], d["b_raw"], d["c_raw"], par["alpha_min"],
+                            par["alpha_max"], par["theta_max"], par["eps"], d["S0"], o, o_im, S_T, cfg.chunk, ws)
+    torch.cuda.synchronize()
+    launches = sfda.last_launch_count()
+    return (o.float().cpu().numpy(), None if o_im is None else o_im.float().cpu().numpy(),
+            None if S_T is None else S_T.cpu().numpy(), launches, ws)
+
+
+def oracle_fused_pairs(raw, pairs, par):
+    """The oracle's front end in float64 on the raw inputs, then the token-by-token recurrence."""
+    sel = lambda key: np.stack([raw[key][b, :, h] for b, h in pairs]).astype(np.float64)
+    al, th, be, k = frontend.stable_parameterisation(sel("a_raw"), sel("b_raw"), sel("c_raw"), sel("k_raw"), **par)
+    S0 = None if raw["S0"] is None else np.stack([raw["S0"][b, h] for b, h in pairs]).astype(np.float64)
+    return recurrence.sfda_recurrence(sel("q"), k, sel("v"), al, th, be, S0)
+
+
+def check_forward_fused(cfg, raw, pairs, par, tol, **kw):
+    o, o_im, S_T, launches, ws = run_forward_fused(cfg, raw, par, **kw)
+    w_re, w_im, w_S = oracle_fused_pairs(raw, pairs, par)
+    errs = {"o_re": rel_err(np.stack([o[b, :, h] for b, h in pairs]), w_re)}
+    if o_im is not None:
+        errs["o_im"] = rel_err(np.stack([o_im[b, :, h] for b, h in pairs]), w_im)
+    if S_T is not None:
+        errs["S_T"] = rel_err(np.stack([S_T[b, h] for b, h in pairs]), w_S)
+    for name, e in errs.items():
+        assert e <= tol, "%s: %s rel err %.3e > %.1e (%s)" % (cfg.name, name, e, tol, errs)
+    return launches, ws
+
+
+@pytest.mark.parametrize("B,T,H", [(1, 64, 1), (2, 200, 3), (1, 1, 2), (3, 1029, 2)])
+def test_forward_fused_tensor_core(B, T, H):
+    """One launch: the parameterisation runs inside the tensor-core kernel's operand preparation."""
+    cfg = workloads.CONFIGS[1].scaled(name="fused", B=B, T=T, H=H, s0_std=0.3, seed=60 + T)
+    raw = workloads.forward_raw_inputs(cfg)
+    launches, ws = check_forward_fused(cfg, raw, all_pairs(cfg), PARAM, TOL["bf16"])
+    assert launches == 1
+    assert sfda.sfda_workspace_status(ws) == 0
+
+
+def test_forward_fused_tensor_core_time_slices_and_narrow_ranges():
+    """Enough chunks per sequence for the launcher to cut time slices; alpha in [0.9, 1], small phases."""
+    cfg = workloads.CONFIGS[1].scaled(name="fused_q", B=1, T=4096, H=2, s0_std=0.0, seed=61)
+    raw = workloads.forward_raw_inputs(cfg)
+    raw["a_raw"] -= 3.0                                   # centred logits: alpha spread over the whole range
+    par = dict(alpha_min=0.9, alpha_max=1.0, theta_max=0.3, eps=1e-3)
+    launches, ws = check_forward_fused(cfg, raw, all_pairs(cfg), par, TOL["bf16"])
+    assert launches == 1 and sfda.sfda_workspace_status(ws) == 0
+
+
+def test_forward_fused_tensor_core_saturated_inputs():
+    """Raw inputs far out in the saturating tails, and keys of very different lengths."""
+    cfg = workloads.CONFIGS[1].scaled(name="fused_sat", B=1, T=300, H=2, s0_std=0.2, seed=62)
+    raw = workloads.forward_raw_inputs(cfg)
+    raw["a_raw"][:, ::7] = 60.0                          # alpha = alpha_max
+    raw["a_raw"][:, 3::11, :, ::4] = -60.0               # alpha = alpha_min
+    raw["b_raw"][:, ::5] *= 40.0                         # theta = +-theta_max
+    raw["c_raw"][:, ::3] = 50.0
+    raw["c_raw"][:, 1::3] = -50.0
+    raw["k_raw"][:, ::2] = workloads.bf16_round(raw["k_raw"][:, ::2] * 1e-3)
+    raw["k_raw"][:, 1::4] = workloads.bf16_round(raw["k_raw"][:, 1::4] * 1e3)
+    par = dict(alpha_min=0.5, alpha_max=1.0, theta_max=float(np.pi), eps=1e-6)
+    check_forward_fused(cfg, raw, all_pairs(cfg), par, TOL["bf16"])
+
+
+@pytest.mark.parametrize("d_k,d_v,chunk,dtype", [(64, 64, 16, "f32"), (128, 64, 32, "bf16"), (128, 128, 16, "f32")])
+def test_forward_fused_other_shapes_stage_through_the_workspace(d_k, d_v, chunk, dtype):
+    cfg = workloads.CONFIGS[0].scaled(name="fused_simt", B=2, T=70, H=2, d_k=d_k, d_v=d_v, chunk=chunk,
+                                      dtype=dtype, s0_std=0.4, seed=63)
+    raw = workloads.forward_raw_inputs(cfg)
+    # bf16: the normalised key is rounded to bf16 on its way through the workspace
+    launches, _ = check_forward_fused(cfg, raw, all_pairs(cfg), PARAM, 1e-4 if dtype == "f32" else 1e-2)
+    assert launches >= 2
+
+
+def test_forward_fused_equals_frontend_then_forward_on_fp32_keys():
+    """The fused kernel against the library's own two-step route at matching precision is not expected to be
+    bitwise equal (fast exponentials inside the kernel); both must sit within the bf16 bar of each other."""
+    cfg = workloads.CONFIGS[1].scaled(name="fused_vs", B=2, T=512, H=2, s0_std=0.0, seed=64)
+    raw = workloads.forward_raw_inputs(cfg)
+    o_f, oi_f, S_f, _, _ = run_forward_fused(cfg, raw, PARAM)
+    d = raw_to_dev(raw, cfg)
+    al, th = torch.empty_like(d["a_raw"]), torch.empty_like(d["a_raw"])
+    be, k = torch.empty_like(d["c_raw"]), torch.empty_like(d["k_raw"])
+    sfda.sfda_frontend(d["a_raw"], d["b_raw"], d["c_raw"], d["k_raw"], PARAM["alpha_min"], PARAM["alpha_max"],
+                       PARAM["theta_max"], PARAM["eps"], al, th, be, k)
+    inp = dict(q=raw["q"], k=k.float().cpu().numpy(), v=raw["v"], alpha=al.cpu().numpy(), theta=th.cpu().numpy(),
+               beta=be.cpu().numpy(), S0=None)
+    o_u, oi_u, S_u = run_forward(cfg, inp)
+    assert rel_err(o_f, o_u) <= TOL["bf16"] and rel_err(oi_f, oi_u) <= TOL["bf16"] and rel_err(S_f, S_u) <= TOL["bf16"]

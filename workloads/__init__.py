@@ -13,6 +13,11 @@ Recipe (every stream is ``numpy.random.default_rng([seed, *key])``, PCG64):
   channels (= the complex norm) in float32 *before* bf16 rounding.
 * config 3 draws its per-(head, pair) modulus p from the stream with key
   ``(10**6,)``; p is fixed over time and over the batch.
+* raw inputs of the stable parameterisation (``forward_raw_*``): one stream per batch element with key
+  ``(7 * 10**6 + b,)`` drawn in the order q, k_raw, key scale, v, a_raw, b_raw, c_raw, S0: a_raw ~ N(3, 1)
+  (so that alpha_min = 0, alpha_max = 1 reproduces the "sigmoid(n(3,1))" decay of the forward configs),
+  b_raw ~ N(0, 1.5), c_raw ~ N(0, 1), k_raw = N(0, 1) times a log-normal scale exp(N(0, 0.5)) per token and
+  head (unnormalised keys of varying length).  Nothing is transformed here.
 * decode config: S0 from key ``(2**20,)``; step ``s`` from key ``(s,)`` in the order
   q, k, v, beta, alpha, theta with shape ``[B, H, ...]``.
 """
@@ -151,6 +156,40 @@ def forward_inputs(cfg, batch=None):
             parts = list(pool.map(lambda b: forward_batch_element(cfg, b), bs))
     else:
         parts = [forward_batch_element(cfg, b) for b in bs]
+    out = {}
+    for key in parts[0]:
+        out[key] = None if parts[0][key] is None else np.stack([p[key] for p in parts])
+    return out
+
+
+def forward_raw_batch_element(cfg, b):
+    """Raw (unconstrained) inputs of batch element b: q, k_raw [T,H,d_k], v [T,H,d_v], a_raw, b_raw [T,H,m],
+    c_raw [T,H], S0 or None.  q, k_raw, v hold values exactly representable in cfg.dtype."""
+    rng = np.random.default_rng([cfg.seed, 7 * 10 ** 6 + b])
+    T, H = cfg.T, cfg.H
+    q = _store(cfg, rng.standard_normal((T, H, cfg.d_k), dtype=np.float32))
+    k_raw = rng.standard_normal((T, H, cfg.d_k), dtype=np.float32)
+    scale = np.exp(0.5 * rng.standard_normal((T, H, 1), dtype=np.float32))
+    k_raw = _store(cfg, k_raw * scale)
+    v = _store(cfg, rng.standard_normal((T, H, cfg.d_v), dtype=np.float32))
+    a_raw = (3.0 + rng.standard_normal((T, H, cfg.m), dtype=np.float32)).astype(np.float32)
+    b_raw = (1.5 * rng.standard_normal((T, H, cfg.m), dtype=np.float32)).astype(np.float32)
+    c_raw = rng.standard_normal((T, H), dtype=np.float32)
+    S0 = None
+    if cfg.s0_std > 0:
+        S0 = (cfg.s0_std * rng.standard_normal((H, cfg.d_k, cfg.d_v), dtype=np.float32)).astype(np.float32)
+    return dict(q=q, k_raw=k_raw, v=v, a_raw=a_raw, b_raw=b_raw, c_raw=c_raw, S0=S0)
+
+
+def forward_raw_inputs(cfg, batch=None):
+    """Stack raw batch elements (all of them by default) into [B, T, H, ...] arrays."""
+    bs = list(range(cfg.B) if batch is None else batch)
+    if len(bs) > 1 and cfg.T * cfg.H >= 1 << 16:
+        from concurrent.futures import ThreadPoolExecutor
+        with ThreadPoolExecutor(max_workers=min(len(bs), os.cpu_count() or 1)) as pool:
+            parts = list(pool.map(lambda b: forward_raw_batch_element(cfg, b), bs))
+    else:
+        parts = [forward_raw_batch_element(cfg, b) for b in bs]
     out = {}
     for key in parts[0]:
         out[key] = None if parts[0][key] is None else np.stack([p[key] for p in parts])
