@@ -586,3 +586,25 @@ def test_forward_fused_equals_frontend_then_forward_on_fp32_keys():
                beta=be.cpu().numpy(), S0=None)
     o_u, oi_u, S_u = run_forward(cfg, inp)
     assert rel_err(o_f, o_u) <= TOL["bf16"] and rel_err(oi_f, oi_u) <= TOL["bf16"] and rel_err(S_f, S_u) <= TOL["bf16"]
+
+
+def test_forward_fused_full_size_headline_sampled():
+    """The headline sizes on raw inputs, in the launch configuration bench.py times for the fused forward;
+    the oracle recomputes a sample of (batch, head) sequences end to end.  Also the property that holds for
+    every sequence: ||S_T||_F <= ||S_0||_F + sum_t beta_t ||v_t|| (Prop. "Basic numerical stability",
+    with |k_t| <= 1 from the parameterisation)."""
+    cfg = workloads.CONFIGS[2]
+    raw = workloads.forward_raw_inputs(cfg)
+    pairs = [(0, 0), (cfg.B - 1, cfg.H - 1), (cfg.B // 2, 5), (1, cfg.H // 2)]
+    o, o_im, S_T, launches, ws = run_forward_fused(cfg, raw, PARAM)
+    assert launches == 1 and sfda.sfda_workspace_status(ws) == 0
+    assert np.isfinite(o).all() and np.isfinite(o_im).all() and np.isfinite(S_T).all()
+    w_re, w_im, w_S = oracle_fused_pairs(raw, pairs, PARAM)
+    assert rel_err(np.stack([o[b, :, h] for b, h in pairs]), w_re) <= TOL["bf16"]
+    assert rel_err(np.stack([o_im[b, :, h] for b, h in pairs]), w_im) <= TOL["bf16"]
+    assert rel_err(np.stack([S_T[b, h] for b, h in pairs]), w_S) <= TOL["bf16"]
+    beta = 1.0 / (1.0 + np.exp(-raw["c_raw"].astype(np.float64)))
+    vnorm = np.linalg.norm(raw["v"].astype(np.float64), axis=-1)
+    bound = np.linalg.norm(raw["S0"].astype(np.float64).reshape(cfg.B, cfg.H, -1), axis=-1) \
+        + np.sum(beta * vnorm, axis=1)
+    assert (np.linalg.norm(S_T.astype(np.float64).reshape(cfg.B, cfg.H, -1), axis=-1) <= bound * (1 + 1e-2)).all()
