@@ -172,6 +172,7 @@ def main():
     ap.add_argument("--re-only", action="store_true", help="write o = Re only (default: Re and Im)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--no-factors", action="store_true", help="skip the leg that times sfda_chunk_factors")
     ap.add_argument("--no-fused", action="store_true", help="skip the leg that times the forward on raw inputs")
     ap.add_argument("--seq-len", type=int, default=0,
                     help="sweeps only: run the headline shapes with this sequence length (use with --batch; the JSON "
@@ -335,6 +336,37 @@ def main():
                  "two_step_ms_per_step": two_ms, "two_step_tokens_per_s": cfg.B * cfg.T / (two_ms * 1e-3)}
         del r, al, th, be, kn
 
+    # per-chunk factor export (sfda_chunk_factors) on the headline inputs: Gamma, Y, M, W and the phase turns
+    factors = None
+    if rank == 0 and not args.no_factors:
+        NC = (cfg.T + cfg.chunk - 1) // cfg.chunk
+        G = torch.empty(cfg.B, cfg.H, NC, cfg.m, 2, device=dev)
+        Yf = torch.empty(cfg.B, cfg.H, NC, cfg.m, cfg.chunk, 2, device=dev)
+        Wf = torch.empty_like(Yf)
+        Mf = torch.empty(cfg.B, cfg.H, NC, cfg.chunk, cfg.chunk, 2, device=dev)
+        turns = torch.empty(cfg.B, cfg.T, cfg.H, cfg.m, device=dev, dtype=torch.int32)
+
+        def fstep():
+            sfda.sfda_chunk_factors(d["k"], d["alpha"], d["theta"], d["beta"], G, Yf, Mf, Wf, turns, cfg.chunk, stream)
+
+        for _ in range(2):
+            fstep()
+        nf = 3
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        f0.record(stream)
+        for _ in range(nf):
+            fstep()
+        f1.record(stream)
+        torch.cuda.synchronize()
+        f_ms = f0.elapsed_time(f1) / nf
+        rows = cfg.B * cfg.T * cfg.H
+        fb = rows * (cfg.d_k * 2 + 2 * cfg.m * 4 + 4) + sum(t.numel() * 4 for t in (G, Yf, Wf, Mf, turns))
+        factors = {"workload": cfg.name + " (k, alpha, theta, beta -> Gamma, Y, M, W, phase turns)",
+                   "ms_per_call": f_ms, "chunks_per_s": cfg.B * cfg.H * NC / (f_ms * 1e-3),
+                   "algorithmic_bytes": fb, "achieved_gbs": fb / (f_ms * 1e-3) / 1e9}
+        del G, Yf, Wf, Mf, turns
+
     # one-token decode (sfda_step) on the decode configuration: HBM-bound, reported beside the headline
     decode = None
     if rank == 0 and not args.no_decode:
@@ -398,6 +430,9 @@ def main():
         roofline["traffic"] = 1.939e9 * cfg.B / 4
         roofline["traffic_source"] = "ncu capture at B=4 scaled to B=%d; Re+Im outputs" % cfg.B
 
+    if factors is not None:
+        factors["frac"] = factors["achieved_gbs"] / peaks["hbm_gbs"]
+        factors["peak_source"] = "of " + peaks["source"]
     if fused is not None:
         fused["frontend_frac"] = fused["frontend_achieved_gbs"] / peaks["hbm_gbs"]
         fused["peak_source"] = "of " + peaks["source"]
@@ -420,7 +455,7 @@ def main():
                    "chunk": cfg.chunk, "outputs": "Re+Im" if want_im else "Re", "state": "fp32", "S0": "N(0,0.02)",
                    "parallelism": "dp%d over (batch, head), no collective" % world,
                    "l2": "inputs+outputs %.2f GB per step, far larger than the 126 MB L2; no flush" % (abytes / 1e9)},
-        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "decode": decode, "fused_front_end": fused,
+        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "decode": decode, "fused_front_end": fused, "chunk_factors": factors,
         "gpu_launches": launches_per_step * args.steps, "clocks": clocks.summary(),
     }
     print(json.dumps(line), flush=True)

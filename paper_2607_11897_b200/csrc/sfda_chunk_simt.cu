@@ -1,4 +1,4 @@
-// fp32 CUDA-core chunk-WY forward and per-chunk factor export.
+// fp32 CUDA-core chunk-WY forward.
 //
 // What is computed per chunk (C tokens, one (batch, head) pair, gamma_t = prod_{s<=t} lambda_s inside
 // the chunk, written gamma_t = a_t e^{i phi_t}):
@@ -277,113 +277,6 @@ sfda_forward_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const
 }
 
 // ------------------------------------------------------------------------------------------------
-// factor export
-// ------------------------------------------------------------------------------------------------
-template <int DK, int C>
-constexpr int factor_smem_floats()
-{
-    return ChunkSmem<DK, C>::floats + 4 * C * (C + 1);  // N (re, im), X = (I + N)^{-1} (re, im)
-}
-
-template <int DK, int C, typename T>
-__global__ void __launch_bounds__(kThreads)
-sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alpha,
-                          const float *__restrict__ theta, const float *__restrict__ beta,
-                          float *__restrict__ Gamma, float *__restrict__ Y, float *__restrict__ Mo,
-                          float *__restrict__ W, uint32_t *__restrict__ turns_out, int T_, int H, int NC)
-{
-    constexpr int M = DK / 2;
-    using SM = ChunkSmem<DK, C>;
-    extern __shared__ __align__(16) float smem[];
-    const SM sm(smem);
-    float *Nr = smem + SM::floats;
-    float *Ni = Nr + C * SM::GS;
-    float *Xr = Ni + C * SM::GS;
-    float *Xi = Xr + C * SM::GS;
-
-    const int tid = threadIdx.x;
-    const int ci = blockIdx.x % NC;
-    const int bh = blockIdx.x / NC;
-    const int h = bh % H, b = bh / H;
-    const int t0 = ci * C;
-    const int len = min(C, T_ - t0);
-    const size_t chunk_id = (size_t)bh * NC + ci;
-
-    load_and_rotate<DK, C, T>(sm, k, static_cast<const T *>(nullptr), alpha, theta, beta, turns_out, b, h, T_,
-                              H, t0, len);
-
-    // N[t][i] = beta_i * k_t^* diag(gamma_t / gamma_i) k_i, i < t  (the block-inverse of Eq. "constructive-M").
-    for (int p = tid; p < C * (C + 1) / 2; p += kThreads) {
-        int t, i;
-        tri_decode(p, &t, &i);
-        float ar = 0.f, ai = 0.f;
-        if (i < t) {
-            const float *kt = sm.kp + t * SM::KS, *ki = sm.kp + i * SM::KS;
-            const float *lt = sm.lg + t * SM::LS, *li = sm.lg + i * SM::LS;
-            for (int j = 0; j < M; ++j) {
-                const float w = expf(lt[j] - li[j]);
-                const float br = w * ki[2 * j], bi = w * ki[2 * j + 1];
-                ar += kt[2 * j] * br + kt[2 * j + 1] * bi;
-                ai += kt[2 * j] * bi - kt[2 * j + 1] * br;
-            }
-            ar *= sm.beta[i];
-            ai *= sm.beta[i];
-        }
-        Nr[t * SM::GS + i] = ar;
-        Ni[t * SM::GS + i] = ai;
-    }
-    __syncthreads();
-
-    // M = (I + N)^{-1}: thread c solves column c by forward substitution (it only reads its own column).
-    if (tid < C) {
-        const int c = tid;
-        for (int t = 0; t < C; ++t) {
-            float xr = t == c ? 1.f : 0.f, xi = 0.f;
-            if (t > c) {
-                for (int i = c; i < t; ++i) {
-                    const float nr = Nr[t * SM::GS + i], ni = Ni[t * SM::GS + i];
-                    const float yr = Xr[i * SM::GS + c], yi = Xi[i * SM::GS + c];
-                    xr -= nr * yr - ni * yi;
-                    xi -= nr * yi + ni * yr;
-                }
-            }
-            Xr[t * SM::GS + c] = xr;
-            Xi[t * SM::GS + c] = xi;
-        }
-    }
-    __syncthreads();
-
-    if (Gamma) {
-        for (int j = tid; j < M; j += kThreads) {
-            const float a = expf(sm.lgC[j]);
-            Gamma[(chunk_id * M + j) * 2] = a * sm.gcr[j];
-            Gamma[(chunk_id * M + j) * 2 + 1] = a * sm.gci[j];
-        }
-    }
-    for (int idx = tid; idx < M * C; idx += kThreads) {
-        const int j = idx / C, t = idx % C;
-        const float kr = sm.kp[t * SM::KS + 2 * j], ki = sm.kp[t * SM::KS + 2 * j + 1];
-        if (W) {   // W[:,t] = conj(gamma_t) k_t = a_t k'_t
-            const float a = expf(sm.lg[t * SM::LS + j]);
-            reinterpret_cast<float2 *>(W)[(chunk_id * M + j) * C + t] = make_float2(a * kr, a * ki);
-        }
-        if (Y) {   // Y[:,t] = (gamma_C / gamma_t) beta_t k_t = (a_C / a_t) e^{i phi_C} beta_t k'_t
-            const float w = sm.beta[t] * expf(sm.lgC[j] - sm.lg[t * SM::LS + j]);
-            const float gr = sm.gcr[j], gi = sm.gci[j];
-            reinterpret_cast<float2 *>(Y)[(chunk_id * M + j) * C + t] =
-                make_float2(w * (gr * kr - gi * ki), w * (gr * ki + gi * kr));
-        }
-    }
-    if (Mo) {
-        for (int idx = tid; idx < C * C; idx += kThreads) {
-            const int t = idx / C, i = idx % C;
-            reinterpret_cast<float2 *>(Mo)[chunk_id * C * C + idx] =
-                i <= t ? make_float2(Xr[t * SM::GS + i], Xi[t * SM::GS + i]) : make_float2(0.f, 0.f);
-        }
-    }
-}
-
-// ------------------------------------------------------------------------------------------------
 // launchers
 // ------------------------------------------------------------------------------------------------
 template <int DK, int C, typename T>
@@ -398,20 +291,6 @@ cudaError_t launch_fwd(const ForwardArgs &a, cudaStream_t stream)
                                            static_cast<const T *>(a.v), a.alpha, a.theta, a.beta, a.S0,
                                            static_cast<T *>(a.o), static_cast<T *>(a.o_im), a.S_T, a.T, a.H,
                                            a.d_v);
-    return cudaGetLastError();
-}
-
-template <int DK, int C, typename T>
-cudaError_t launch_fac(const FactorArgs &a, cudaStream_t stream)
-{
-    constexpr size_t smem = sizeof(float) * factor_smem_floats<DK, C>();
-    auto kern = sfda_chunk_factors_kernel<DK, C, T>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    const int NC = (a.T + C - 1) / C;
-    const unsigned grid = (unsigned)a.B * a.H * NC;
-    kern<<<grid, kThreads, smem, stream>>>(static_cast<const T *>(a.k), a.alpha, a.theta, a.beta, a.Gamma, a.Y,
-                                           a.M, a.W, a.phase_turns, a.T, a.H, NC);
     return cudaGetLastError();
 }
 
@@ -437,27 +316,11 @@ cudaError_t dispatch_fwd(const ForwardArgs &a, cudaStream_t s)
         [&] { return launch_fwd<128, 32, T>(a, s); }, [&] { return launch_fwd<128, 64, T>(a, s); });
 }
 
-template <typename T>
-cudaError_t dispatch_fac(const FactorArgs &a, cudaStream_t s)
-{
-    return by_shape<FactorArgs, T>(
-        a, [&] { return launch_fac<64, 16, T>(a, s); }, [&] { return launch_fac<64, 32, T>(a, s); },
-        [&] { return launch_fac<64, 64, T>(a, s); }, [&] { return launch_fac<128, 16, T>(a, s); },
-        [&] { return launch_fac<128, 32, T>(a, s); }, [&] { return launch_fac<128, 64, T>(a, s); });
-}
-
 }  // namespace
 
 cudaError_t launch_forward_simt(const ForwardArgs &a, cudaStream_t stream, int *launches)
 {
     const cudaError_t e = a.dtype == 1 ? dispatch_fwd<__nv_bfloat16>(a, stream) : dispatch_fwd<float>(a, stream);
-    if (e == cudaSuccess && launches) ++*launches;
-    return e;
-}
-
-cudaError_t launch_chunk_factors(const FactorArgs &a, cudaStream_t stream, int *launches)
-{
-    const cudaError_t e = a.dtype == 1 ? dispatch_fac<__nv_bfloat16>(a, stream) : dispatch_fac<float>(a, stream);
     if (e == cudaSuccess && launches) ++*launches;
     return e;
 }

@@ -1,0 +1,364 @@
+// sfda_chunk_factors: per-chunk factors of P = A_C ... A_1 = Gamma - Y M W^* (Theorem "Constructive left-to-right
+// chunk-WY recursion", Cor. "SFDA admits exact constructive block-WY products") in fp32 on the CUDA cores.
+//
+// With gamma_t = prod_{s<=t} lambda_s = a_t e^{i phi_t} inside the chunk and k'_t = e^{-i phi_t} k_t:
+//
+//   Gamma = gamma_C,   W[:,t] = conj(gamma_t) k_t = a_t k'_t,   Y[:,t] = (gamma_C / gamma_t) beta_t k_t
+//   N[t][i] = beta_i k_t^* diag(gamma_t / gamma_i) k_i = beta_i sum_j conj(k'_tj) k'_ij a_tj / a_ij   (i < t)
+//   M = (I + N)^{-1}                                                       (Eq. "constructive-M" unrolled)
+//
+// One CTA of 256 threads per chunk, two CTAs per SM; everything after the loads lives in shared memory:
+//   A  scan:     thread = (coordinate j, group of C/G tokens): log-decay and integer-phase prefix sums, rotated keys
+//   B  export:   Gamma, W, Y (coalesced over t)
+//   C  Gram:     blocks of 8 tokens.  A pair (t, i) of different blocks T > I splits its decay at the last token r
+//                of block I: a_t/a_i = (a_t/a_r)(a_r/a_i), both factors <= 1, so an 4 x 4 tile of pairs needs 8
+//                exponentials per coordinate instead of 16 and nothing overflows whatever alpha is; pairs inside a
+//                block take the ratio directly.  224 tile halves + 32 block quarters = 256 work items at C = 64.
+//   D  inverse:  8 x 8 diagonal blocks by substitution, then X = [[X11, 0], [-X22 N21 X11, X22]] doubling the
+//                block size until it is C.
+// Only ratios <= 1 are ever formed, so any alpha in [0, 1] is safe.
+#include "sfda_common.cuh"
+#include "sfda_internal.h"
+
+namespace sfda {
+namespace {
+
+constexpr int kFacThreads = 256;
+constexpr float kLog2e = 1.4426950408889634f;
+
+__device__ __forceinline__ float ex2f(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// cos / sin of a phase given in 2^-32 turns: the top 23 bits as a fraction of a turn in [-1/2, 1/2), fast sine.
+__device__ __forceinline__ void turns_cos_sin_fast(uint32_t turns, float *c, float *s)
+{
+    float f = __uint_as_float(0x3f800000u | (turns >> 9)) - 1.0f;
+    f -= f >= 0.5f ? 1.0f : 0.0f;
+    __sincosf(f * 6.283185307f, s, c);
+}
+
+template <int DK, int C>
+struct FacSmem {
+    static constexpr int M = DK / 2;
+    static constexpr int KS = M + 1;        // row stride of kp in float2 (odd: rows and columns both conflict-free)
+    static constexpr int LS = M + 1;        // row stride of lg2 in floats
+    static constexpr int NS = C + 1;        // row stride of N / X in float2
+    static constexpr int G = kFacThreads / M;   // token groups of the scan
+    static constexpr int TG = C / G;            // tokens per group
+    static constexpr size_t bytes = (size_t)C * KS * 8 + (size_t)C * LS * 4 + (size_t)C * NS * 8 +
+                                    (size_t)G * M * 8 + (size_t)M * 12 + (size_t)C * 4;
+    float2 *kp;        // [C][KS] rotated keys k'; after the Gram: scratch of the inverse
+    float *lg2;        // [C][LS] log2 of a_t
+    float2 *nx;        // [C][NS] N, inverted in place
+    float *grp_lg;     // [G][M] group totals of the scan
+    uint32_t *grp_tu;  // [G][M]
+    float *gcr, *gci, *lg2C;   // [M] e^{i phi_C}, log2 a_C
+    float *beta;       // [C]
+    __device__ explicit FacSmem(unsigned char *base)
+    {
+        kp = reinterpret_cast<float2 *>(base);
+        lg2 = reinterpret_cast<float *>(kp + C * KS);
+        nx = reinterpret_cast<float2 *>(lg2 + C * LS);
+        grp_lg = reinterpret_cast<float *>(nx + C * NS);
+        grp_tu = reinterpret_cast<uint32_t *>(grp_lg + G * M);
+        gcr = reinterpret_cast<float *>(grp_tu + G * M);
+        gci = gcr + M;
+        lg2C = gci + M;
+        beta = lg2C + M;
+    }
+};
+static_assert(FacSmem<128, 64>::bytes <= 112 * 1024, "two CTAs per SM need at most 113 KB each");
+
+template <int DK, int C, typename T>
+__global__ void __launch_bounds__(kFacThreads, 2)
+sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alpha, const float *__restrict__ theta,
+                          const float *__restrict__ beta, float *__restrict__ Gamma, float *__restrict__ Y,
+                          float *__restrict__ Mo, float *__restrict__ W, uint32_t *__restrict__ turns_out, int T_,
+                          int H, int NC)
+{
+    using S = FacSmem<DK, C>;
+    constexpr int M = S::M, G = S::G, TG = S::TG;
+    static_assert(C % 8 == 0 && C % G == 0 && TG >= 1, "chunk must split into the scan's groups and 8-token blocks");
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const S sm(smem_raw);
+
+    const int tid = threadIdx.x;
+    const int ci = blockIdx.x % NC;
+    const int bh = blockIdx.x / NC;
+    const int h = bh % H, b = bh / H;
+    const int t0 = ci * C;
+    const int len = min(C, T_ - t0);
+    const size_t chunk_id = (size_t)bh * NC + ci;
+
+    // ---- A: loads and scan.  Tokens past `len` are neutral (alpha = 1, theta = 0, beta = 0, k = 0).
+    {
+        const int j = tid % M, g = tid / M;
+        float lgv[TG];
+        uint32_t tu[TG];
+        float2 kv[TG];
+#pragma unroll
+        for (int x = 0; x < TG; ++x) {
+            const int t = g * TG + x;
+            float al = 1.f, th = 0.f;
+            kv[x] = make_float2(0.f, 0.f);
+            if (t < len) {
+                const size_t row = ((size_t)b * T_ + t0 + t) * H + h;
+                al = alpha[row * M + j];
+                th = theta[row * M + j];
+                kv[x] = make_float2(ld_val(k, row * DK + 2 * j), ld_val(k, row * DK + 2 * j + 1));
+            }
+            lgv[x] = al;
+            tu[x] = __float_as_uint(th);
+        }
+        if (tid < C) sm.beta[tid] = tid < len ? beta[((size_t)b * T_ + t0 + tid) * H + h] : 0.f;
+        float acc = 0.f;
+        uint32_t ta = 0u;
+#pragma unroll
+        for (int x = 0; x < TG; ++x) {     // inclusive prefixes inside the group
+            acc += log_decay(lgv[x]) * kLog2e;
+            ta += phase_to_turns(__uint_as_float(tu[x]));
+            lgv[x] = acc;
+            tu[x] = ta;
+        }
+        sm.grp_lg[g * M + j] = acc;
+        sm.grp_tu[g * M + j] = ta;
+        __syncthreads();
+        float base = 0.f;
+        uint32_t tb = 0u;
+        for (int gg = 0; gg < g; ++gg) {
+            base += sm.grp_lg[gg * M + j];
+            tb += sm.grp_tu[gg * M + j];
+        }
+#pragma unroll
+        for (int x = 0; x < TG; ++x) {
+            const int t = g * TG + x;
+            const float l = base + lgv[x];
+            const uint32_t tt = tb + tu[x];
+            if (turns_out && t < len) turns_out[(((size_t)b * T_ + t0 + t) * H + h) * M + j] = tt;
+            float cs, sn;
+            turns_cos_sin_fast(tt, &cs, &sn);
+            sm.lg2[t * S::LS + j] = l;
+            sm.kp[t * S::KS + j] = make_float2(kv[x].x * cs + kv[x].y * sn, kv[x].y * cs - kv[x].x * sn);   // e^{-i phi} k
+            if (t == C - 1) {
+                turns_to_cos_sin(tt, &cs, &sn);    // the exported Gamma takes the accurate sine
+                sm.gcr[j] = cs;
+                sm.gci[j] = sn;
+                sm.lg2C[j] = l;
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- B: Gamma, W, Y
+    if (Gamma) {
+        for (int j = tid; j < M; j += kFacThreads) {
+            const float a = ex2f(sm.lg2C[j]);
+            reinterpret_cast<float2 *>(Gamma)[chunk_id * M + j] = make_float2(a * sm.gcr[j], a * sm.gci[j]);
+        }
+    }
+    if (W || Y) {
+        for (int idx = tid; idx < M * C; idx += kFacThreads) {
+            const int j = idx / C, t = idx % C;
+            const float2 kk = sm.kp[t * S::KS + j];
+            const float l = sm.lg2[t * S::LS + j];
+            if (W) {   // W[:,t] = conj(gamma_t) k_t = a_t k'_t
+                const float a = ex2f(l);
+                reinterpret_cast<float2 *>(W)[(chunk_id * M + j) * C + t] = make_float2(a * kk.x, a * kk.y);
+            }
+            if (Y) {   // Y[:,t] = (gamma_C / gamma_t) beta_t k_t = (a_C / a_t) e^{i phi_C} beta_t k'_t
+                const float w = sm.beta[t] * ex2f(sm.lg2C[j] - l);
+                const float gr = sm.gcr[j], gi = sm.gci[j];
+                reinterpret_cast<float2 *>(Y)[(chunk_id * M + j) * C + t] =
+                    make_float2(w * (gr * kk.x - gi * kk.y), w * (gr * kk.y + gi * kk.x));
+            }
+        }
+    }
+
+    // ---- C: N[t][i] = beta_i sum_j conj(k'_tj) k'_ij a_tj / a_ij,  i < t
+    if (Mo) {
+        constexpr int NB = C / 8;                          // blocks of 8 tokens
+        constexpr int kTileItems = NB * (NB - 1) / 2 * 8;  // block pair T > I: 4 tiles of 4 x 4, two halves of j
+        constexpr int kItems = kTileItems + NB * 4;        // + the diagonal blocks, 7 pairs per item
+        for (int base = 0; base < kItems; base += kFacThreads) {
+            const int item = base + tid;
+            // the two lanes of a tile are neighbours and kTileItems is even: they always take this branch together
+            const unsigned tile_lanes = __ballot_sync(0xffffffffu, item < kTileItems);
+            if (item < kTileItems) {
+                // adjacent lanes hold the two halves of the coordinates of one tile and add up at the end
+                const int half = item & 1, tile = (item >> 1) & 3, bp = item >> 3;
+                int Tb = 1;
+                while (Tb * (Tb + 1) / 2 <= bp) ++Tb;      // bp = Tb (Tb - 1) / 2 + Ib
+                const int Ib = bp - Tb * (Tb - 1) / 2;
+                const int tr = 8 * Tb + 4 * (tile >> 1), ic = 8 * Ib + 4 * (tile & 1), r = 8 * Ib + 7;
+                float ar[4][4], ai[4][4];
+#pragma unroll
+                for (int x = 0; x < 4; ++x)
+#pragma unroll
+                    for (int y = 0; y < 4; ++y) ar[x][y] = ai[x][y] = 0.f;
+#pragma unroll 2
+                for (int jj = 0; jj < M / 2; ++jj) {
+                    const int j = half * (M / 2) + jj;
+                    const float lr = sm.lg2[r * S::LS + j];
+                    float2 a[4], bb[4];
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) {
+                        const float wa = ex2f(sm.lg2[(tr + x) * S::LS + j] - lr);      // a_t / a_r <= 1
+                        const float2 kk = sm.kp[(tr + x) * S::KS + j];
+                        a[x] = make_float2(wa * kk.x, wa * kk.y);
+                        const float wb = ex2f(lr - sm.lg2[(ic + x) * S::LS + j]);      // a_r / a_i <= 1
+                        const float2 kb = sm.kp[(ic + x) * S::KS + j];
+                        bb[x] = make_float2(wb * kb.x, wb * kb.y);
+                    }
+#pragma unroll
+                    for (int x = 0; x < 4; ++x)
+#pragma unroll
+                        for (int y = 0; y < 4; ++y) {      // conj(a) b
+                            ar[x][y] = fmaf(a[x].x, bb[y].x, fmaf(a[x].y, bb[y].y, ar[x][y]));
+                            ai[x][y] = fmaf(a[x].x, bb[y].y, fmaf(-a[x].y, bb[y].x, ai[x][y]));
+                        }
+                }
+#pragma unroll
+                for (int x = 0; x < 4; ++x)
+#pragma unroll
+                    for (int y = 0; y < 4; ++y) {
+                        ar[x][y] += __shfl_xor_sync(tile_lanes, ar[x][y], 1);
+                        ai[x][y] += __shfl_xor_sync(tile_lanes, ai[x][y], 1);
+                    }
+                // each half writes two of the four rows
+#pragma unroll
+                for (int x = 0; x < 4; ++x)
+                    if ((x >> 1) == half)
+#pragma unroll
+                        for (int y = 0; y < 4; ++y) {
+                            const float bt = sm.beta[ic + y];
+                            sm.nx[(tr + x) * S::NS + ic + y] = make_float2(bt * ar[x][y], bt * ai[x][y]);
+                        }
+            } else if (item < kItems) {
+                // pairs inside block blk: quarter qd takes pairs p = qd, qd + 4, ... of the 28 (t, i), i < t
+                const int d = item - kTileItems, blk = d >> 2, qd = d & 3;
+                for (int pidx = qd; pidx < 28; pidx += 4) {
+                    int t = 1;
+                    while (t * (t + 1) / 2 <= pidx) ++t;   // pidx = t (t - 1) / 2 + i
+                    const int i = pidx - t * (t - 1) / 2;
+                    const int tt = 8 * blk + t, ii = 8 * blk + i;
+                    float sr = 0.f, si = 0.f;
+#pragma unroll 4
+                    for (int j = 0; j < M; ++j) {
+                        const float w = ex2f(sm.lg2[tt * S::LS + j] - sm.lg2[ii * S::LS + j]);
+                        const float2 a = sm.kp[tt * S::KS + j], bq = sm.kp[ii * S::KS + j];
+                        sr = fmaf(w, a.x * bq.x + a.y * bq.y, sr);
+                        si = fmaf(w, a.x * bq.y - a.y * bq.x, si);
+                    }
+                    const float bt = sm.beta[ii];
+                    sm.nx[tt * S::NS + ii] = make_float2(bt * sr, bt * si);
+                }
+            }
+        }
+        __syncthreads();
+
+        // ---- D: X = (I + N)^{-1} in place.  Diagonal 8 x 8 blocks: thread = (block, column c), right-looking
+        // substitution of (I + N) x = e_c in registers; everybody reads before anybody writes.
+        {
+            float xr[8], xi[8];
+            const int blk = tid >> 3, c = tid & 7, o = 8 * blk;
+            if (tid < C) {
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    xr[r] = r == c ? 1.f : 0.f;
+                    xi[r] = 0.f;
+                }
+#pragma unroll
+                for (int i = 0; i < 7; ++i) {
+                    const float vr = xr[i], vi = xi[i];
+#pragma unroll
+                    for (int r = i + 1; r < 8; ++r) {
+                        const float2 n = sm.nx[(o + r) * S::NS + o + i];
+                        xr[r] -= n.x * vr - n.y * vi;
+                        xi[r] -= n.x * vi + n.y * vr;
+                    }
+                }
+            }
+            __syncthreads();
+            if (tid < C) {
+#pragma unroll
+                for (int r = 0; r < 8; ++r) sm.nx[(o + r) * S::NS + o + c] = make_float2(xr[r], xi[r]);
+            }
+            __syncthreads();
+        }
+        // merges: blocks of size hs at o (X11) and o + hs (X22), N21 below X11:  X21 = -X22 (N21 X11)
+        float2 *P = sm.kp;                                  // scratch [C / 2 rows of merges][hs x hs], keys are done
+#pragma unroll 1
+        for (int hs = 8; hs < C; hs *= 2) {
+            const int per = hs * hs, total = (C / (2 * hs)) * per;
+            for (int idx = tid; idx < total; idx += kFacThreads) {     // P[r][c] = sum_{k >= c} N21[r][k] X11[k][c]
+                const int mg = idx / per, rc = idx % per, r = rc / hs, c = rc % hs, o = mg * 2 * hs;
+                float pr = 0.f, pi = 0.f;
+                for (int kk = c; kk < hs; ++kk) {
+                    const float2 n = sm.nx[(o + hs + r) * S::NS + o + kk];
+                    const float2 x = sm.nx[(o + kk) * S::NS + o + c];
+                    pr += n.x * x.x - n.y * x.y;
+                    pi += n.x * x.y + n.y * x.x;
+                }
+                P[idx] = make_float2(pr, pi);
+            }
+            __syncthreads();
+            for (int idx = tid; idx < total; idx += kFacThreads) {     // X21[r][c] = -sum_{k <= r} X22[r][k] P[k][c]
+                const int mg = idx / per, rc = idx % per, r = rc / hs, c = rc % hs, o = mg * 2 * hs;
+                float sr = 0.f, si = 0.f;
+                for (int kk = 0; kk <= r; ++kk) {
+                    const float2 x = sm.nx[(o + hs + r) * S::NS + o + hs + kk];
+                    const float2 pp = P[mg * per + kk * hs + c];
+                    sr += x.x * pp.x - x.y * pp.y;
+                    si += x.x * pp.y + x.y * pp.x;
+                }
+                sm.nx[(o + hs + r) * S::NS + o + c] = make_float2(-sr, -si);
+            }
+            __syncthreads();
+        }
+        for (int idx = tid; idx < C * C; idx += kFacThreads) {
+            const int t = idx / C, i = idx % C;
+            reinterpret_cast<float2 *>(Mo)[chunk_id * C * C + idx] = i <= t ? sm.nx[t * S::NS + i] : make_float2(0.f, 0.f);
+        }
+    }
+}
+
+template <int DK, int C, typename T>
+cudaError_t launch_fac(const FactorArgs &a, cudaStream_t stream)
+{
+    constexpr size_t smem = FacSmem<DK, C>::bytes;
+    auto kern = sfda_chunk_factors_kernel<DK, C, T>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const int NC = (a.T + C - 1) / C;
+    const unsigned grid = (unsigned)a.B * a.H * NC;
+    kern<<<grid, kFacThreads, smem, stream>>>(static_cast<const T *>(a.k), a.alpha, a.theta, a.beta, a.Gamma, a.Y, a.M,
+                                              a.W, a.phase_turns, a.T, a.H, NC);
+    return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t dispatch_fac(const FactorArgs &a, cudaStream_t s)
+{
+    if (a.d_k == 64 && a.chunk == 16) return launch_fac<64, 16, T>(a, s);
+    if (a.d_k == 64 && a.chunk == 32) return launch_fac<64, 32, T>(a, s);
+    if (a.d_k == 64 && a.chunk == 64) return launch_fac<64, 64, T>(a, s);
+    if (a.d_k == 128 && a.chunk == 16) return launch_fac<128, 16, T>(a, s);
+    if (a.d_k == 128 && a.chunk == 32) return launch_fac<128, 32, T>(a, s);
+    if (a.d_k == 128 && a.chunk == 64) return launch_fac<128, 64, T>(a, s);
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace
+
+cudaError_t launch_chunk_factors(const FactorArgs &a, cudaStream_t stream, int *launches)
+{
+    const cudaError_t e = a.dtype == 1 ? dispatch_fac<__nv_bfloat16>(a, stream) : dispatch_fac<float>(a, stream);
+    if (e == cudaSuccess && launches) ++*launches;
+    return e;
+}
+
+}  // namespace sfda
