@@ -7,13 +7,14 @@
 //   N[t][i] = beta_i k_t^* diag(gamma_t / gamma_i) k_i = beta_i sum_j conj(k'_tj) k'_ij a_tj / a_ij   (i < t)
 //   M = (I + N)^{-1}                                                       (Eq. "constructive-M" unrolled)
 //
-// One CTA of 256 threads per chunk, two CTAs per SM; everything after the loads lives in shared memory:
+// One CTA of 256 threads per chunk, three CTAs per SM; everything after the loads lives in shared memory (N and its
+// inverse take the place of the rotated keys once the Gram sums are in registers):
 //   A  scan:     thread = (coordinate j, group of C/G tokens): log-decay and integer-phase prefix sums, rotated keys
 //   B  export:   Gamma, W, Y (coalesced over t)
 //   C  Gram:     blocks of 8 tokens.  A pair (t, i) of different blocks T > I splits its decay at the last token r
 //                of block I: a_t/a_i = (a_t/a_r)(a_r/a_i), both factors <= 1, so an 4 x 4 tile of pairs needs 8
 //                exponentials per coordinate instead of 16 and nothing overflows whatever alpha is; pairs inside a
-//                block take the ratio directly.  224 tile halves + 32 block quarters = 256 work items at C = 64.
+//                block take the ratio directly, eight lanes per pair.
 //   D  inverse:  8 x 8 diagonal blocks by substitution, then X = [[X11, 0], [-X22 N21 X11, X22]] doubling the
 //                block size until it is C.
 // Only ratios <= 1 are ever formed, so any alpha in [0, 1] is safe.
@@ -33,6 +34,22 @@ __device__ __forceinline__ float ex2f(float x)
     return y;
 }
 
+// log2 of a decay factor, floored like log_decay (e^-30 = 2^-43.28): one special-function instruction, absolute
+// error about 2^-22.
+__device__ __forceinline__ float log2_decay(float alpha)
+{
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(alpha));
+    return fmaxf(y, -30.0f * kLog2e);
+}
+
+// Two adjacent elements (real and imaginary part of one coordinate) in one load.
+__device__ __forceinline__ float2 ld_pair(const float *p, size_t i) { return *reinterpret_cast<const float2 *>(p + i); }
+__device__ __forceinline__ float2 ld_pair(const __nv_bfloat16 *p, size_t i)
+{
+    return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(p + i));
+}
+
 // cos / sin of a phase given in 2^-32 turns: the top 23 bits as a fraction of a turn in [-1/2, 1/2), fast sine.
 __device__ __forceinline__ void turns_cos_sin_fast(uint32_t turns, float *c, float *s)
 {
@@ -49,32 +66,69 @@ struct FacSmem {
     static constexpr int NS = C + 1;        // row stride of N / X in float2
     static constexpr int G = kFacThreads / M;   // token groups of the scan
     static constexpr int TG = C / G;            // tokens per group
-    static constexpr size_t bytes = (size_t)C * KS * 8 + (size_t)C * LS * 4 + (size_t)C * NS * 8 +
-                                    (size_t)G * M * 8 + (size_t)M * 12 + (size_t)C * 4;
-    float2 *kp;        // [C][KS] rotated keys k'; after the Gram: scratch of the inverse
-    float *lg2;        // [C][LS] log2 of a_t
-    float2 *nx;        // [C][NS] N, inverted in place
-    float *grp_lg;     // [G][M] group totals of the scan
+    static constexpr int kKeyRows = C * (KS > NS ? KS : NS);   // float2: the larger of k' and N
+    static constexpr int kGrpFloats = 2 * G * M > 2 * (C / 8) * 28 ? 2 * G * M : 2 * (C / 8) * 28;
+    static constexpr size_t bytes = (size_t)kKeyRows * 8 + (size_t)C * LS * 4 + (size_t)kGrpFloats * 4 +
+                                    (size_t)M * 12 + (size_t)C * 4;
+    float2 *kp;        // [C][KS] rotated keys k' until the Gram sums are in registers ...
+    float2 *nx;        // ... then [C][NS] N, inverted in place (same memory)
+    float *lg2;        // [C][LS] log2 of a_t; after the Gram: scratch of the inverse's products
+    float *grp_lg;     // [G][M] group totals of the scan; later the Gram sums of the pairs inside 8-token blocks
     uint32_t *grp_tu;  // [G][M]
     float *gcr, *gci, *lg2C;   // [M] e^{i phi_C}, log2 a_C
     float *beta;       // [C]
     __device__ explicit FacSmem(unsigned char *base)
     {
         kp = reinterpret_cast<float2 *>(base);
-        lg2 = reinterpret_cast<float *>(kp + C * KS);
-        nx = reinterpret_cast<float2 *>(lg2 + C * LS);
-        grp_lg = reinterpret_cast<float *>(nx + C * NS);
+        nx = kp;
+        lg2 = reinterpret_cast<float *>(kp + kKeyRows);
+        grp_lg = lg2 + C * LS;
         grp_tu = reinterpret_cast<uint32_t *>(grp_lg + G * M);
-        gcr = reinterpret_cast<float *>(grp_tu + G * M);
+        gcr = grp_lg + kGrpFloats;
         gci = gcr + M;
         lg2C = gci + M;
         beta = lg2C + M;
     }
 };
-static_assert(FacSmem<128, 64>::bytes <= 112 * 1024, "two CTAs per SM need at most 113 KB each");
+static_assert(FacSmem<128, 64>::bytes <= 74 * 1024, "three CTAs per SM need at most 75 KB each");
+
+// One level of the block inverse: every pair of finished diagonal blocks of size HS becomes one of size 2 HS.
+template <typename S, int C, int HS>
+__device__ __forceinline__ void merge_level(const S &sm, int tid)
+{
+    if constexpr (HS < C) {
+        constexpr int per = HS * HS, total = (C / (2 * HS)) * per;
+        float2 *P = reinterpret_cast<float2 *>(sm.lg2);    // scratch [merges of the level][HS x HS]: the decays are done
+        for (int idx = tid; idx < total; idx += kFacThreads) {     // P[r][c] = sum_{k >= c} N21[r][k] X11[k][c]
+            // lanes run over r: one trip count (HS - c) per warp, N21 rows conflict-free, X11 broadcast
+            const int mg = idx / per, rc = idx % per, c = rc / HS, r = rc % HS, o = mg * 2 * HS;
+            float pr = 0.f, pi = 0.f;
+            for (int kk = c; kk < HS; ++kk) {
+                const float2 n = sm.nx[(o + HS + r) * S::NS + o + kk];
+                const float2 x = sm.nx[(o + kk) * S::NS + o + c];
+                pr += n.x * x.x - n.y * x.y;
+                pi += n.x * x.y + n.y * x.x;
+            }
+            P[mg * per + r * HS + c] = make_float2(pr, pi);
+        }
+        __syncthreads();
+        for (int idx = tid; idx < total; idx += kFacThreads) {     // X21[r][c] = -sum_{k <= r} X22[r][k] P[k][c]
+            const int mg = idx / per, rc = idx % per, r = rc / HS, c = rc % HS, o = mg * 2 * HS;
+            float sr = 0.f, si = 0.f;
+            for (int kk = 0; kk <= r; ++kk) {
+                const float2 x = sm.nx[(o + HS + r) * S::NS + o + HS + kk];
+                const float2 pp = P[mg * per + kk * HS + c];
+                sr += x.x * pp.x - x.y * pp.y;
+                si += x.x * pp.y + x.y * pp.x;
+            }
+            sm.nx[(o + HS + r) * S::NS + o + c] = make_float2(-sr, -si);
+        }
+        __syncthreads();
+    }
+}
 
 template <int DK, int C, typename T>
-__global__ void __launch_bounds__(kFacThreads, 2)
+__global__ void __launch_bounds__(kFacThreads, 3)
 sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alpha, const float *__restrict__ theta,
                           const float *__restrict__ beta, float *__restrict__ Gamma, float *__restrict__ Y,
                           float *__restrict__ Mo, float *__restrict__ W, uint32_t *__restrict__ turns_out, int T_,
@@ -83,6 +137,7 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
     using S = FacSmem<DK, C>;
     constexpr int M = S::M, G = S::G, TG = S::TG;
     static_assert(C % 8 == 0 && C % G == 0 && TG >= 1, "chunk must split into the scan's groups and 8-token blocks");
+    static_assert((size_t)C * (C / 4) * 8 <= (size_t)C * S::LS * 4, "the inverse's scratch must fit where lg2 was");
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const S sm(smem_raw);
 
@@ -100,16 +155,19 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
         float lgv[TG];
         uint32_t tu[TG];
         float2 kv[TG];
+        const size_t row0 = ((size_t)b * T_ + t0 + g * TG) * H + h;      // first token of the group
+        const float *ap = alpha + row0 * M + j, *tp = theta + row0 * M + j;
+        const T *kq = k + row0 * DK + 2 * j;
+        const size_t cs = (size_t)H * M;                                  // coordinates from one token to the next
 #pragma unroll
         for (int x = 0; x < TG; ++x) {
             const int t = g * TG + x;
             float al = 1.f, th = 0.f;
             kv[x] = make_float2(0.f, 0.f);
             if (t < len) {
-                const size_t row = ((size_t)b * T_ + t0 + t) * H + h;
-                al = alpha[row * M + j];
-                th = theta[row * M + j];
-                kv[x] = make_float2(ld_val(k, row * DK + 2 * j), ld_val(k, row * DK + 2 * j + 1));
+                al = ap[x * cs];
+                th = tp[x * cs];
+                kv[x] = ld_pair(kq, 2 * x * cs);
             }
             lgv[x] = al;
             tu[x] = __float_as_uint(th);
@@ -119,7 +177,7 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
         uint32_t ta = 0u;
 #pragma unroll
         for (int x = 0; x < TG; ++x) {     // inclusive prefixes inside the group
-            acc += log_decay(lgv[x]) * kLog2e;
+            acc += log2_decay(lgv[x]);
             ta += phase_to_turns(__uint_as_float(tu[x]));
             lgv[x] = acc;
             tu[x] = ta;
@@ -138,7 +196,7 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
             const int t = g * TG + x;
             const float l = base + lgv[x];
             const uint32_t tt = tb + tu[x];
-            if (turns_out && t < len) turns_out[(((size_t)b * T_ + t0 + t) * H + h) * M + j] = tt;
+            if (turns_out && t < len) turns_out[row0 * M + j + x * cs] = tt;
             float cs, sn;
             turns_cos_sin_fast(tt, &cs, &sn);
             sm.lg2[t * S::LS + j] = l;
@@ -161,19 +219,24 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
         }
     }
     if (W || Y) {
-        for (int idx = tid; idx < M * C; idx += kFacThreads) {
-            const int j = idx / C, t = idx % C;
+        // a thread keeps its token and walks over the coordinates: consecutive lanes store consecutive tokens
+        constexpr int JS = kFacThreads / C;                 // coordinates per sweep of the CTA
+        const int t = tid % C;
+        const float bt = sm.beta[t];
+        float2 *Wp = reinterpret_cast<float2 *>(W) + (chunk_id * M + tid / C) * C + t;
+        float2 *Yp = reinterpret_cast<float2 *>(Y) + (chunk_id * M + tid / C) * C + t;
+#pragma unroll 4
+        for (int j = tid / C; j < M; j += JS, Wp += JS * C, Yp += JS * C) {
             const float2 kk = sm.kp[t * S::KS + j];
             const float l = sm.lg2[t * S::LS + j];
             if (W) {   // W[:,t] = conj(gamma_t) k_t = a_t k'_t
                 const float a = ex2f(l);
-                reinterpret_cast<float2 *>(W)[(chunk_id * M + j) * C + t] = make_float2(a * kk.x, a * kk.y);
+                *Wp = make_float2(a * kk.x, a * kk.y);
             }
             if (Y) {   // Y[:,t] = (gamma_C / gamma_t) beta_t k_t = (a_C / a_t) e^{i phi_C} beta_t k'_t
-                const float w = sm.beta[t] * ex2f(sm.lg2C[j] - l);
+                const float w = bt * ex2f(sm.lg2C[j] - l);
                 const float gr = sm.gcr[j], gi = sm.gci[j];
-                reinterpret_cast<float2 *>(Y)[(chunk_id * M + j) * C + t] =
-                    make_float2(w * (gr * kk.x - gi * kk.y), w * (gr * kk.y + gi * kk.x));
+                *Yp = make_float2(w * (gr * kk.x - gi * kk.y), w * (gr * kk.y + gi * kk.x));
             }
         }
     }
@@ -182,81 +245,101 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
     if (Mo) {
         constexpr int NB = C / 8;                          // blocks of 8 tokens
         constexpr int kTileItems = NB * (NB - 1) / 2 * 8;  // block pair T > I: 4 tiles of 4 x 4, two halves of j
-        constexpr int kItems = kTileItems + NB * 4;        // + the diagonal blocks, 7 pairs per item
-        for (int base = 0; base < kItems; base += kFacThreads) {
-            const int item = base + tid;
-            // the two lanes of a tile are neighbours and kTileItems is even: they always take this branch together
-            const unsigned tile_lanes = __ballot_sync(0xffffffffu, item < kTileItems);
-            if (item < kTileItems) {
-                // adjacent lanes hold the two halves of the coordinates of one tile and add up at the end
-                const int half = item & 1, tile = (item >> 1) & 3, bp = item >> 3;
-                int Tb = 1;
-                while (Tb * (Tb + 1) / 2 <= bp) ++Tb;      // bp = Tb (Tb - 1) / 2 + Ib
-                const int Ib = bp - Tb * (Tb - 1) / 2;
-                const int tr = 8 * Tb + 4 * (tile >> 1), ic = 8 * Ib + 4 * (tile & 1), r = 8 * Ib + 7;
-                float ar[4][4], ai[4][4];
+        constexpr int kPairs = NB * 28;                    // pairs (t, i), i < t, inside the blocks
+        static_assert(kTileItems <= kFacThreads && kTileItems % 8 == 0, "one tile half per thread");
+        // Off-diagonal tiles: adjacent lanes hold the two halves of the coordinates of one tile and add up at the
+        // end.  The sums stay in registers: N will overwrite the keys once everybody has read them.
+        const bool has_tile = tid < kTileItems;
+        const unsigned tile_lanes = __ballot_sync(0xffffffffu, has_tile);
+        const int half = tid & 1, tile = (tid >> 1) & 3, bp = tid >> 3;
+        int Tb = 1;
+        while (Tb * (Tb + 1) / 2 <= bp) ++Tb;              // bp = Tb (Tb - 1) / 2 + Ib
+        const int Ib = bp - Tb * (Tb - 1) / 2;
+        const int tr = 8 * Tb + 4 * (tile >> 1), ic = 8 * Ib + 4 * (tile & 1), r = 8 * Ib + 7;
+        float ar[4][4], ai[4][4];
+        if (has_tile) {
 #pragma unroll
-                for (int x = 0; x < 4; ++x)
+            for (int x = 0; x < 4; ++x)
 #pragma unroll
-                    for (int y = 0; y < 4; ++y) ar[x][y] = ai[x][y] = 0.f;
+                for (int y = 0; y < 4; ++y) ar[x][y] = ai[x][y] = 0.f;
 #pragma unroll 2
-                for (int jj = 0; jj < M / 2; ++jj) {
-                    const int j = half * (M / 2) + jj;
-                    const float lr = sm.lg2[r * S::LS + j];
-                    float2 a[4], bb[4];
+            for (int jj = 0; jj < M / 2; ++jj) {
+                const int j = 2 * jj + half;               // the two lanes of a tile read neighbouring banks
+                const float lr = sm.lg2[r * S::LS + j];
+                float2 a[4], bb[4];
 #pragma unroll
-                    for (int x = 0; x < 4; ++x) {
-                        const float wa = ex2f(sm.lg2[(tr + x) * S::LS + j] - lr);      // a_t / a_r <= 1
-                        const float2 kk = sm.kp[(tr + x) * S::KS + j];
-                        a[x] = make_float2(wa * kk.x, wa * kk.y);
-                        const float wb = ex2f(lr - sm.lg2[(ic + x) * S::LS + j]);      // a_r / a_i <= 1
-                        const float2 kb = sm.kp[(ic + x) * S::KS + j];
-                        bb[x] = make_float2(wb * kb.x, wb * kb.y);
-                    }
-#pragma unroll
-                    for (int x = 0; x < 4; ++x)
-#pragma unroll
-                        for (int y = 0; y < 4; ++y) {      // conj(a) b
-                            ar[x][y] = fmaf(a[x].x, bb[y].x, fmaf(a[x].y, bb[y].y, ar[x][y]));
-                            ai[x][y] = fmaf(a[x].x, bb[y].y, fmaf(-a[x].y, bb[y].x, ai[x][y]));
-                        }
+                for (int x = 0; x < 4; ++x) {
+                    const float wa = ex2f(sm.lg2[(tr + x) * S::LS + j] - lr);      // a_t / a_r <= 1
+                    const float2 kk = sm.kp[(tr + x) * S::KS + j];
+                    a[x] = make_float2(wa * kk.x, wa * kk.y);
+                    const float wb = ex2f(lr - sm.lg2[(ic + x) * S::LS + j]);      // a_r / a_i <= 1
+                    const float2 kb = sm.kp[(ic + x) * S::KS + j];
+                    bb[x] = make_float2(wb * kb.x, wb * kb.y);
                 }
 #pragma unroll
                 for (int x = 0; x < 4; ++x)
+#pragma unroll
+                    for (int y = 0; y < 4; ++y) {          // conj(a) b
+                        ar[x][y] = fmaf(a[x].x, bb[y].x, fmaf(a[x].y, bb[y].y, ar[x][y]));
+                        ai[x][y] = fmaf(a[x].x, bb[y].y, fmaf(-a[x].y, bb[y].x, ai[x][y]));
+                    }
+            }
+#pragma unroll
+            for (int x = 0; x < 4; ++x)
+#pragma unroll
+                for (int y = 0; y < 4; ++y) {
+                    ar[x][y] += __shfl_xor_sync(tile_lanes, ar[x][y], 1);
+                    ai[x][y] += __shfl_xor_sync(tile_lanes, ai[x][y], 1);
+                }
+        }
+        // Pairs inside a block take the decay ratio directly.  Eight lanes share a pair (coordinates j = lane, lane +
+        // 8, ...) and add up by shuffles; the sums wait in the scan's group totals, which are no longer needed.
+        float2 *dg = reinterpret_cast<float2 *>(sm.grp_lg);
+        for (int base = 0; base < kPairs * 8; base += kFacThreads) {
+            const int li = base + tid, pr_ = li >> 3, sub = li & 7;
+            const bool on = li < kPairs * 8;
+            const unsigned lanes = __ballot_sync(0xffffffffu, on);     // whole groups of eight lanes
+            if (on) {
+                const int blk = pr_ % NB, pidx = pr_ / NB; // neighbouring groups of lanes work in different blocks
+                int t = 1;
+                while (t * (t + 1) / 2 <= pidx) ++t;       // pidx = t (t - 1) / 2 + i
+                const int i = pidx - t * (t - 1) / 2;
+                const int tt = 8 * blk + t, ii = 8 * blk + i;
+                float sr = 0.f, si = 0.f;
+#pragma unroll 4
+                for (int j = sub; j < M; j += 8) {
+                    const float w = ex2f(sm.lg2[tt * S::LS + j] - sm.lg2[ii * S::LS + j]);
+                    const float2 a = sm.kp[tt * S::KS + j], bq = sm.kp[ii * S::KS + j];
+                    sr = fmaf(w, a.x * bq.x + a.y * bq.y, sr);
+                    si = fmaf(w, a.x * bq.y - a.y * bq.x, si);
+                }
+#pragma unroll
+                for (int dlt = 1; dlt < 8; dlt *= 2) {
+                    sr += __shfl_xor_sync(lanes, sr, dlt);
+                    si += __shfl_xor_sync(lanes, si, dlt);
+                }
+                if (sub == 0) dg[pr_] = make_float2(sr, si);
+            }
+        }
+        __syncthreads();           // every read of the keys is done: N goes where they were
+        if (has_tile) {            // each half writes two of the four rows
+#pragma unroll
+            for (int x = 0; x < 4; ++x)
+                if ((x >> 1) == half)
 #pragma unroll
                     for (int y = 0; y < 4; ++y) {
-                        ar[x][y] += __shfl_xor_sync(tile_lanes, ar[x][y], 1);
-                        ai[x][y] += __shfl_xor_sync(tile_lanes, ai[x][y], 1);
+                        const float bt = sm.beta[ic + y];
+                        sm.nx[(tr + x) * S::NS + ic + y] = make_float2(bt * ar[x][y], bt * ai[x][y]);
                     }
-                // each half writes two of the four rows
-#pragma unroll
-                for (int x = 0; x < 4; ++x)
-                    if ((x >> 1) == half)
-#pragma unroll
-                        for (int y = 0; y < 4; ++y) {
-                            const float bt = sm.beta[ic + y];
-                            sm.nx[(tr + x) * S::NS + ic + y] = make_float2(bt * ar[x][y], bt * ai[x][y]);
-                        }
-            } else if (item < kItems) {
-                // pairs inside block blk: quarter qd takes pairs p = qd, qd + 4, ... of the 28 (t, i), i < t
-                const int d = item - kTileItems, blk = d >> 2, qd = d & 3;
-                for (int pidx = qd; pidx < 28; pidx += 4) {
-                    int t = 1;
-                    while (t * (t + 1) / 2 <= pidx) ++t;   // pidx = t (t - 1) / 2 + i
-                    const int i = pidx - t * (t - 1) / 2;
-                    const int tt = 8 * blk + t, ii = 8 * blk + i;
-                    float sr = 0.f, si = 0.f;
-#pragma unroll 4
-                    for (int j = 0; j < M; ++j) {
-                        const float w = ex2f(sm.lg2[tt * S::LS + j] - sm.lg2[ii * S::LS + j]);
-                        const float2 a = sm.kp[tt * S::KS + j], bq = sm.kp[ii * S::KS + j];
-                        sr = fmaf(w, a.x * bq.x + a.y * bq.y, sr);
-                        si = fmaf(w, a.x * bq.y - a.y * bq.x, si);
-                    }
-                    const float bt = sm.beta[ii];
-                    sm.nx[tt * S::NS + ii] = make_float2(bt * sr, bt * si);
-                }
-            }
+        }
+        for (int pr_ = tid; pr_ < kPairs; pr_ += kFacThreads) {
+            const int blk = pr_ % NB, pidx = pr_ / NB;
+            int t = 1;
+            while (t * (t + 1) / 2 <= pidx) ++t;
+            const int i = pidx - t * (t - 1) / 2;
+            const float2 v = dg[pr_];
+            const float bt = sm.beta[8 * blk + i];
+            sm.nx[(8 * blk + t) * S::NS + 8 * blk + i] = make_float2(bt * v.x, bt * v.y);
         }
         __syncthreads();
 
@@ -289,36 +372,10 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
             }
             __syncthreads();
         }
-        // merges: blocks of size hs at o (X11) and o + hs (X22), N21 below X11:  X21 = -X22 (N21 X11)
-        float2 *P = sm.kp;                                  // scratch [C / 2 rows of merges][hs x hs], keys are done
-#pragma unroll 1
-        for (int hs = 8; hs < C; hs *= 2) {
-            const int per = hs * hs, total = (C / (2 * hs)) * per;
-            for (int idx = tid; idx < total; idx += kFacThreads) {     // P[r][c] = sum_{k >= c} N21[r][k] X11[k][c]
-                const int mg = idx / per, rc = idx % per, r = rc / hs, c = rc % hs, o = mg * 2 * hs;
-                float pr = 0.f, pi = 0.f;
-                for (int kk = c; kk < hs; ++kk) {
-                    const float2 n = sm.nx[(o + hs + r) * S::NS + o + kk];
-                    const float2 x = sm.nx[(o + kk) * S::NS + o + c];
-                    pr += n.x * x.x - n.y * x.y;
-                    pi += n.x * x.y + n.y * x.x;
-                }
-                P[idx] = make_float2(pr, pi);
-            }
-            __syncthreads();
-            for (int idx = tid; idx < total; idx += kFacThreads) {     // X21[r][c] = -sum_{k <= r} X22[r][k] P[k][c]
-                const int mg = idx / per, rc = idx % per, r = rc / hs, c = rc % hs, o = mg * 2 * hs;
-                float sr = 0.f, si = 0.f;
-                for (int kk = 0; kk <= r; ++kk) {
-                    const float2 x = sm.nx[(o + hs + r) * S::NS + o + hs + kk];
-                    const float2 pp = P[mg * per + kk * hs + c];
-                    sr += x.x * pp.x - x.y * pp.y;
-                    si += x.x * pp.y + x.y * pp.x;
-                }
-                sm.nx[(o + hs + r) * S::NS + o + c] = make_float2(-sr, -si);
-            }
-            __syncthreads();
-        }
+        // merges: blocks of size HS at o (X11) and o + HS (X22), N21 below X11:  X21 = -X22 (N21 X11)
+        merge_level<S, C, 8>(sm, tid);
+        merge_level<S, C, 16>(sm, tid);
+        merge_level<S, C, 32>(sm, tid);
         for (int idx = tid; idx < C * C; idx += kFacThreads) {
             const int t = idx / C, i = idx % C;
             reinterpret_cast<float2 *>(Mo)[chunk_id * C * C + idx] = i <= t ? sm.nx[t * S::NS + i] : make_float2(0.f, 0.f);
