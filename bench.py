@@ -399,7 +399,23 @@ def main():
         step_ms = d0.elapsed_time(d1) / nd
         dbytes = dcfg.B * dcfg.H * (2 * dcfg.d_k * dcfg.d_v * 4 + 2 * dcfg.d_k * 2 + dcfg.d_v * 2 + 2 * dcfg.m * 4 + 4
                                      + 2 * dcfg.d_v * 2)
-        decode = {"workload": dcfg.name, "ms_per_step": step_ms, "tokens_per_s": dcfg.B / (step_ms * 1e-3),
+        # the same step on raw inputs of the stable parameterisation (map applied inside the kernel)
+        rawd = workloads.forward_raw_inputs(dcfg)
+        rd = {k: torch.from_numpy(np.ascontiguousarray(v[:, 0])).to(dev) for k, v in rawd.items() if k != "S0"}
+        for k in ("q", "k_raw", "v"):
+            rd[k] = rd[k].to(torch.bfloat16)
+        for _ in range(8):
+            sfda.sfda_step_fused(rd["q"], rd["k_raw"], rd["v"], rd["a_raw"], rd["b_raw"], rd["c_raw"], 0.0, 1.0,
+                                 math.pi, 1e-6, S, od, od_im, stream)
+        torch.cuda.synchronize()
+        d0.record(stream)
+        for _ in range(nd):
+            sfda.sfda_step_fused(rd["q"], rd["k_raw"], rd["v"], rd["a_raw"], rd["b_raw"], rd["c_raw"], 0.0, 1.0,
+                                 math.pi, 1e-6, S, od, od_im, stream)
+        d1.record(stream)
+        torch.cuda.synchronize()
+        fused_step_ms = d0.elapsed_time(d1) / nd
+        decode = {"workload": dcfg.name, "ms_per_step": step_ms, "fused_raw_inputs_ms_per_step": fused_step_ms, "tokens_per_s": dcfg.B / (step_ms * 1e-3),
                   "algorithmic_bytes_per_step": dbytes, "achieved_gbs": dbytes / (step_ms * 1e-3) / 1e9,
                   "state_bytes": int(S.numel() * 4), "note": "state (537 MB) far larger than L2"}
 

@@ -211,6 +211,18 @@ SFDA_API int sfda_step(const void *q, const void *k, const void *v,
               int B, int H, int d_k, int d_v, int dtype, void *stream);
 
 /*
+ * sfda_step on the raw inputs of the stable parameterisation (see sfda_frontend for the map, the scalars'
+ * ranges and SFDA_ERR_VALUE): a_raw, b_raw [B][H][m], c_raw [B][H], k_raw [B][H][d_k] take the place of alpha,
+ * theta, beta, k; the map is applied inside the decode kernel (accurate exp / tanh / sqrt, fp32), nothing else
+ * changes.  With eps = 0 a zero key stays zero.
+ */
+SFDA_API int sfda_step_fused(const void *q, const void *k_raw, const void *v,
+                             const float *a_raw, const float *b_raw, const float *c_raw,
+                             float alpha_min, float alpha_max, float theta_max, float eps,
+                             float *S, void *o, void *o_im,
+                             int B, int H, int d_k, int d_v, int dtype, void *stream);
+
+/*
  * Host-buffer forward: the call a user with data in host memory makes.  Copies the
  * inputs from HOST memory (pinned for asynchronous copies) into `arena`, runs
  * sfda_forward there and copies o (and o_im, S_T when not NULL) back to HOST

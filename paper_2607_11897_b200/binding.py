@@ -53,6 +53,7 @@ def load():
     lib.sfda_forward_fused_workspace_bytes.restype = _sz
     lib.sfda_forward_fused_workspace_bytes.argtypes = [_ci] * 7
     lib.sfda_forward_fused.argtypes = [_vp] * 6 + [_cf] * 4 + [_vp] * 4 + [_ci] * 7 + [_vp, _sz, _vp]
+    lib.sfda_step_fused.argtypes = [_vp] * 6 + [_cf] * 4 + [_vp] * 3 + [_ci] * 5 + [_vp]
     _LIB = lib
     return lib
 
@@ -257,3 +258,18 @@ def sfda_forward_fused(q, k_raw, v, a_raw, b_raw, c_raw, alpha_min, alpha_max, t
                                    d_k, d_v, chunk, _dtype_code(q), _ptr(workspace), ws_bytes, _stream(stream))
     if rc != 0:
         raise SfdaError(rc, "sfda_forward_fused")
+
+
+def sfda_step_fused(q, k_raw, v, a_raw, b_raw, c_raw, alpha_min, alpha_max, theta_max, eps, S, o, o_im, stream=None):
+    """``sfda_step_fused`` of ``include/sfda.h``: one decode step on the raw inputs; S is updated in place."""
+    B, H, d_k = q.shape
+    d_v = v.shape[-1]
+    for t, n in ((q, "q"), (k_raw, "k_raw"), (v, "v"), (o, "o"), (o_im, "o_im")):
+        _check(t, n, q.dtype)
+    for t, n in ((a_raw, "a_raw"), (b_raw, "b_raw"), (c_raw, "c_raw"), (S, "S")):
+        _check(t, n, torch.float32)
+    rc = load().sfda_step_fused(_ptr(q), _ptr(k_raw), _ptr(v), _ptr(a_raw), _ptr(b_raw), _ptr(c_raw), alpha_min,
+                                alpha_max, theta_max, eps, _ptr(S), _ptr(o), _ptr(o_im), B, H, d_k, d_v,
+                                _dtype_code(q), _stream(stream))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_step_fused")

@@ -105,6 +105,27 @@ size_t staged_frontend_bytes(size_t rows, int d_k, int dtype)
     return 2 * round256(rows * (d_k / 2) * 4) + round256(rows * 4) + round256(rows * d_k * elem_bytes(dtype));
 }
 
+int step_common(const void *q, const void *k, const void *v, const float *alpha, const float *theta,
+                const float *beta, float *S, void *o, void *o_im, int B, int H, int d_k, int d_v, int dtype,
+                const sfda::StepParam &par, void *stream)
+{
+    g_last_launches = 0;
+    if (!q || !k || !v || !alpha || !theta || !beta || !S || !o) return SFDA_ERR_NULL;
+    if (B < 1 || H < 1) return SFDA_ERR_SHAPE;
+    const int rc = check_dims(d_k, d_v, 64, dtype);
+    if (rc != SFDA_OK) return rc;
+    const void *ptrs[] = {q, k, v, alpha, theta, beta, S, o, o_im};
+    for (const void *p : ptrs)
+        if (p && !aligned16(p)) return SFDA_ERR_ALIGN;
+    sfda::StepArgs a;
+    a.q = q; a.k = k; a.v = v; a.alpha = alpha; a.theta = theta; a.beta = beta;
+    a.S = S; a.o = o; a.o_im = o_im;
+    a.B = B; a.H = H; a.d_k = d_k; a.d_v = d_v; a.dtype = dtype;
+    a.par = par;
+    return sfda::launch_step(a, static_cast<cudaStream_t>(stream), &g_last_launches) == cudaSuccess ? SFDA_OK
+                                                                                                    : SFDA_ERR_CUDA;
+}
+
 }  // namespace
 
 extern "C" {
@@ -237,20 +258,20 @@ int sfda_step(const void *q, const void *k, const void *v, const float *alpha, c
               const float *beta, float *S, void *o, void *o_im, int B, int H, int d_k, int d_v, int dtype,
               void *stream)
 {
+    return step_common(q, k, v, alpha, theta, beta, S, o, o_im, B, H, d_k, d_v, dtype, sfda::StepParam(), stream);
+}
+
+int sfda_step_fused(const void *q, const void *k_raw, const void *v, const float *a_raw, const float *b_raw,
+                    const float *c_raw, float alpha_min, float alpha_max, float theta_max, float eps, float *S,
+                    void *o, void *o_im, int B, int H, int d_k, int d_v, int dtype, void *stream)
+{
     g_last_launches = 0;
-    if (!q || !k || !v || !alpha || !theta || !beta || !S || !o) return SFDA_ERR_NULL;
-    if (B < 1 || H < 1) return SFDA_ERR_SHAPE;
-    const int rc = check_dims(d_k, d_v, 64, dtype);
+    const int rc = check_param_scalars(alpha_min, alpha_max, theta_max, eps);
     if (rc != SFDA_OK) return rc;
-    const void *ptrs[] = {q, k, v, alpha, theta, beta, S, o, o_im};
-    for (const void *p : ptrs)
-        if (p && !aligned16(p)) return SFDA_ERR_ALIGN;
-    sfda::StepArgs a;
-    a.q = q; a.k = k; a.v = v; a.alpha = alpha; a.theta = theta; a.beta = beta;
-    a.S = S; a.o = o; a.o_im = o_im;
-    a.B = B; a.H = H; a.d_k = d_k; a.d_v = d_v; a.dtype = dtype;
-    return sfda::launch_step(a, static_cast<cudaStream_t>(stream), &g_last_launches) == cudaSuccess ? SFDA_OK
-                                                                                                    : SFDA_ERR_CUDA;
+    sfda::StepParam par;
+    par.fused = 1;
+    par.a_lo = alpha_min; par.a_range = alpha_max - alpha_min; par.th_max = theta_max; par.eps = eps;
+    return step_common(q, k_raw, v, a_raw, b_raw, c_raw, S, o, o_im, B, H, d_k, d_v, dtype, par, stream);
 }
 
 size_t sfda_forward_host_arena_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int dtype, int want_o_im,

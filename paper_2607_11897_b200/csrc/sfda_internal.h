@@ -26,12 +26,19 @@ struct FactorArgs {
     int B, T, H, d_k, chunk, dtype;
 };
 
+// fused != 0: alpha, theta, beta, k hold the raw inputs of the stable parameterisation (decode kernel)
+struct StepParam {
+    int fused = 0;
+    float a_lo = 0.f, a_range = 1.f, th_max = 0.f, eps = 0.f;
+};
+
 struct StepArgs {
     const void *q, *k, *v;
     const float *alpha, *theta, *beta;
     float *S;
     void *o, *o_im;
     int B, H, d_k, d_v, dtype;
+    StepParam par;
 };
 
 struct FrontendArgs {

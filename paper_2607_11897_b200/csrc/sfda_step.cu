@@ -17,12 +17,21 @@ namespace {
 constexpr int kStepThreads = 128;
 constexpr int kColTile = 64;   // value columns per CTA
 
-template <int DK, int DV, typename T>
+// 16-byte load of state that stays where it is written: the loads must be in flight before the (short) preamble
+// runs, whatever else the preamble has to compute.
+__device__ __forceinline__ float4 ld_state(const float *p)
+{
+    float4 v;
+    asm volatile("ld.global.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p) : "memory");
+    return v;
+}
+
+template <int DK, int DV, typename T, bool kFused>
 __global__ void __launch_bounds__(kStepThreads)
 sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v,
                  const float *__restrict__ alpha, const float *__restrict__ theta,
                  const float *__restrict__ beta, float *__restrict__ S, T *__restrict__ o,
-                 T *__restrict__ o_im)
+                 T *__restrict__ o_im, const StepParam par)
 {
     constexpr int M = DK / 2;              // complex rows
     constexpr int CT = DV < kColTile ? DV : kColTile;   // columns of this CTA
@@ -34,6 +43,7 @@ sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__re
     __shared__ float s_lr[M], s_li[M], s_kr[M], s_ki[M], s_qr[M], s_qi[M];
     __shared__ float s_v[CT];
     __shared__ float s_red[RG][2][CT];
+    __shared__ float s_norm[kStepThreads / 32];
 
     const int tid = threadIdx.x;
     const size_t bh = blockIdx.x;
@@ -47,24 +57,64 @@ sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__re
 #pragma unroll
     for (int r = 0; r < R; ++r) {
         const int j = rg * R + r;
-        sre[r] = *reinterpret_cast<const float4 *>(Sbh + (size_t)(2 * j) * DV + 4 * cg);
-        sim[r] = *reinterpret_cast<const float4 *>(Sbh + (size_t)(2 * j + 1) * DV + 4 * cg);
+        sre[r] = ld_state(Sbh + (size_t)(2 * j) * DV + 4 * cg);
+        sim[r] = ld_state(Sbh + (size_t)(2 * j + 1) * DV + 4 * cg);
     }
 
-    for (int j = tid; j < M; j += kStepThreads) {
-        const float a = alpha[bh * M + j];
-        float sn, cs;
-        sincosf(theta[bh * M + j], &sn, &cs);
-        s_lr[j] = a * cs;
-        s_li[j] = a * sn;
-        s_kr[j] = ld_val(k, bh * DK + 2 * j);
-        s_ki[j] = ld_val(k, bh * DK + 2 * j + 1);
-        s_qr[j] = ld_val(q, bh * DK + 2 * j);
-        s_qi[j] = ld_val(q, bh * DK + 2 * j + 1);
+    // kFused: alpha, theta, beta, k arrive raw and go through the stable parameterisation of Section 3 first
+    // (Eqs. "param-alpha", "param-theta", "param-beta", "param-key"); a few hundred values per state, nothing
+    // beside the 128 KB of state traffic.
+    // Every global load of the preamble is issued before anything waits for one of them.
+    static_assert(M <= kStepThreads && CT <= kStepThreads, "one coordinate and one column per thread at most");
+    float a = 1.f, th = 0.f, kr0 = 0.f, ki0 = 0.f, qr0 = 0.f, qi0 = 0.f, v0 = 0.f;
+    if (tid < M) {
+        a = alpha[bh * M + tid];
+        th = theta[bh * M + tid];
+        kr0 = ld_val(k, bh * DK + 2 * tid);
+        ki0 = ld_val(k, bh * DK + 2 * tid + 1);
+        qr0 = ld_val(q, bh * DK + 2 * tid);
+        qi0 = ld_val(q, bh * DK + 2 * tid + 1);
     }
-    for (int c = tid; c < CT; c += kStepThreads) s_v[c] = ld_val(v, bh * DV + c0 + c);
-    const float bt = beta[bh];
+    if (tid < CT) v0 = ld_val(v, bh * DV + c0 + tid);
+    float bt = beta[bh];
+    float ss = 0.f;                        // this thread's share of |k_raw|^2
+    if (tid < M) {
+        if (kFused) {
+            // sigmoid(x) = 1 / (1 + e^-x), tanh(x) = 1 - 2 / (1 + e^2x) with the fast exponential and division
+            // (absolute error about 1e-7; both saturate correctly through infinity and zero)
+            a = fmaf(par.a_range, __fdividef(1.0f, 1.0f + __expf(-a)), par.a_lo);
+            th = fmaf(-2.0f * par.th_max, __fdividef(1.0f, 1.0f + __expf(2.0f * th)), par.th_max);
+            ss = fmaf(kr0, kr0, ki0 * ki0);
+        }
+        float sn, cs;
+        sincosf(th, &sn, &cs);
+        s_lr[tid] = a * cs;
+        s_li[tid] = a * sn;
+        s_kr[tid] = kr0;
+        s_ki[tid] = ki0;
+        s_qr[tid] = qr0;
+        s_qi[tid] = qi0;
+    }
+    if (tid < CT) s_v[tid] = v0;
+    constexpr int kKeyWarps = (M + 31) / 32;       // the warps whose threads read key coordinates above
+    if (kFused) {
+        bt = __fdividef(1.0f, 1.0f + __expf(-bt));
+        if (tid < 32 * kKeyWarps) {                // warp-uniform
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
+            if ((tid & 31) == 0) s_norm[tid >> 5] = ss;
+        }
+    }
     __syncthreads();
+    // s = 1 / (|k_raw| + eps).  The shared key stays raw: with k = s k_raw, c = s (k_raw^* Lambda S) and
+    // S += k e^T = k_raw (s e)^T, so the scale enters twice per column instead of twice per state row.
+    float sk = 1.0f;
+    if (kFused) {
+        float n2 = 0.f;
+#pragma unroll
+        for (int w = 0; w < kKeyWarps; ++w) n2 += s_norm[w];
+        sk = __fdividef(1.0f, fmaxf(__fsqrt_rn(n2) + par.eps, 1.0e-30f));  // a zero key with eps = 0 stays zero
+    }
 
     // S <- Lambda S (2x2 rotation-decay per complex row);  partial c = k^* (Lambda S).
     float cre[4] = {0.f, 0.f, 0.f, 0.f}, cim[4] = {0.f, 0.f, 0.f, 0.f};
@@ -99,8 +149,13 @@ sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__re
             a += s_red[g][0][4 * cg + x];
             b += s_red[g][1][4 * cg + x];
         }
-        ere[x] = bt * (s_v[4 * cg + x] - a);   // e = beta (v - c), v real
-        eim[x] = -bt * b;
+        if (kFused) {                          // c = s c_raw; e -> s e for the raw-key update
+            ere[x] = sk * bt * (s_v[4 * cg + x] - sk * a);
+            eim[x] = -sk * bt * sk * b;
+        } else {
+            ere[x] = bt * (s_v[4 * cg + x] - a);   // e = beta (v - c), v real
+            eim[x] = -bt * b;
+        }
     }
     __syncthreads();   // s_red is reused below
 
@@ -146,9 +201,14 @@ template <int DK, int DV, typename T>
 cudaError_t launch_one(const StepArgs &a, cudaStream_t stream)
 {
     const dim3 grid((unsigned)a.B * (unsigned)a.H, DV > kColTile ? DV / kColTile : 1);
-    sfda_step_kernel<DK, DV, T><<<grid, kStepThreads, 0, stream>>>(
-        static_cast<const T *>(a.q), static_cast<const T *>(a.k), static_cast<const T *>(a.v), a.alpha,
-        a.theta, a.beta, a.S, static_cast<T *>(a.o), static_cast<T *>(a.o_im));
+    if (a.par.fused)
+        sfda_step_kernel<DK, DV, T, true><<<grid, kStepThreads, 0, stream>>>(
+            static_cast<const T *>(a.q), static_cast<const T *>(a.k), static_cast<const T *>(a.v), a.alpha,
+            a.theta, a.beta, a.S, static_cast<T *>(a.o), static_cast<T *>(a.o_im), a.par);
+    else
+        sfda_step_kernel<DK, DV, T, false><<<grid, kStepThreads, 0, stream>>>(
+            static_cast<const T *>(a.q), static_cast<const T *>(a.k), static_cast<const T *>(a.v), a.alpha,
+            a.theta, a.beta, a.S, static_cast<T *>(a.o), static_cast<T *>(a.o_im), a.par);
     return cudaGetLastError();
 }
 

@@ -112,6 +112,15 @@ def test_stable_parameterisation_entry_points_validate_on_the_host(lib):
     assert fused(fptrs, [0.0, 2.0, 3.0, 0.0], fdims) == -8
     assert fused(fptrs, scal, fdims, ws=None, ws_bytes=0) == -5
     assert fused(fptrs, scal, [1, 64, 1, 64, 64, 16, 0], ws_bytes=1024) == -5      # staging does not fit
+    def stepf(ptrs, scal, dims):
+        return lib.sfda_step_fused(*ptrs[:6], *[cf(x) for x in scal], *ptrs[6:], *[ci(d) for d in dims], None)
+
+    sptrs, sdims = [ok] * 8 + [None], [1, 1, 128, 128, 1]
+    assert stepf([None] + sptrs[1:], scal, sdims) == -1
+    assert stepf(sptrs, scal, [0, 1, 128, 128, 1]) == -2
+    assert stepf(sptrs, scal, [1, 1, 128, 32, 1]) == -3
+    assert stepf(sptrs, [0.0, 1.0, float("nan"), 0.0], sdims) == -8
+    assert stepf(sptrs[:1] + [vp(0x1002)] + sptrs[2:], scal, sdims) == -4
     # workspace sizes: the tensor-core shape needs what sfda_forward needs; other shapes stage alpha, theta,
     # beta and the normalised key (each rounded up to 256 bytes)
     assert sfda.sfda_forward_fused_workspace_bytes(8, 8192, 32, 128, 128, 64, 1) == \

@@ -608,3 +608,37 @@ def test_forward_fused_full_size_headline_sampled():
     bound = np.linalg.norm(raw["S0"].astype(np.float64).reshape(cfg.B, cfg.H, -1), axis=-1) \
         + np.sum(beta * vnorm, axis=1)
     assert (np.linalg.norm(S_T.astype(np.float64).reshape(cfg.B, cfg.H, -1), axis=-1) <= bound * (1 + 1e-2)).all()
+
+
+@pytest.mark.parametrize("d_k,d_v,dtype,par", [
+    (128, 128, "bf16", PARAM), (64, 128, "f32", PARAM),
+    (128, 64, "f32", dict(alpha_min=0.25, alpha_max=0.875, theta_max=0.5, eps=0.0))])
+def test_step_fused_iterated_matches_oracle(d_k, d_v, dtype, par):
+    """Decode on raw inputs, token by token, against the oracle's front end followed by its recurrence."""
+    cfg = workloads.CONFIGS[0].scaled(name="stepf", B=2, T=40, H=3, d_k=d_k, d_v=d_v, dtype=dtype, s0_std=0.3,
+                                      seed=70 + d_k)
+    raw = workloads.forward_raw_inputs(cfg)
+    if par["eps"] > 0:
+        raw["k_raw"][0, 5, 1] = 0.0                  # a zero key (0 / (0 + eps) = 0; with eps = 0 the map is 0 / 0)
+    pairs = all_pairs(cfg)
+    w_re, w_im, w_S = oracle_fused_pairs(raw, pairs, par)
+    dt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    S = torch.from_numpy(raw["S0"]).to(DEV)
+    o = torch.empty(cfg.B, cfg.H, cfg.d_v, device=DEV, dtype=dt)
+    o_im = torch.empty_like(o)
+    got_re, got_im = [], []
+    for t in range(cfg.T):
+        d = {k: torch.from_numpy(np.ascontiguousarray(raw[k][:, t])).to(DEV) for k in
+             ("q", "k_raw", "v", "a_raw", "b_raw", "c_raw")}
+        for k in ("q", "k_raw", "v"):
+            d[k] = d[k].to(dt)
+        sfda.sfda_step_fused(d["q"], d["k_raw"], d["v"], d["a_raw"], d["b_raw"], d["c_raw"], par["alpha_min"],
+                             par["alpha_max"], par["theta_max"], par["eps"], S, o, o_im)
+        assert sfda.last_launch_count() == 1
+        got_re.append(o.float().cpu().numpy())
+        got_im.append(o_im.float().cpu().numpy())
+    got_re, got_im = np.stack(got_re, 1), np.stack(got_im, 1)          # [B, T, H, d_v]
+    tol = 5e-3 if dtype == "bf16" else 1e-4                            # bf16: only the stored outputs are rounded
+    assert rel_err(np.stack([got_re[b, :, h] for b, h in pairs]), w_re) <= tol
+    assert rel_err(np.stack([got_im[b, :, h] for b, h in pairs]), w_im) <= tol
+    assert rel_err(np.stack([S[b, h].cpu().numpy() for b, h in pairs]), w_S) <= 1e-4
