@@ -9,7 +9,7 @@ import os
 import numpy as np
 import pytest
 
-from oracle import bookkeeping, chunk_wy, frontend, recurrence
+from oracle import backward, bookkeeping, chunk_wy, frontend, recurrence
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -522,3 +522,92 @@ def test_parameterisation_gives_the_stability_assumptions():
     _, _, S_T = recurrence.sfda_recurrence(q, k, v, al, th, be, None)
     bound = np.sum(np.sqrt(be)[..., None] * np.linalg.norm(v, axis=-1)[..., None], axis=1)   # sum_t sqrt(beta_t) ||v_t||
     assert np.all(np.linalg.norm(S_T.reshape(N, -1), axis=-1) <= bound[:, 0] + 1e-9)
+
+
+# ----------------------------------------------------------------------------
+# backward pass: the gradient of a scalar loss through Eq. "sfda"
+# ----------------------------------------------------------------------------
+def _loss_inputs(seed, N=2, T=7, m=3, dv=4, s0=True):
+    rng = np.random.default_rng(seed)
+    x = dict(q=rng.standard_normal((N, T, 2 * m)), k=0.6 * rng.standard_normal((N, T, 2 * m)),
+             v=rng.standard_normal((N, T, dv)), alpha=rng.uniform(0.5, 1.0, (N, T, m)),
+             theta=rng.uniform(-np.pi, np.pi, (N, T, m)), beta=rng.uniform(0.1, 0.9, (N, T)),
+             S0=(rng.standard_normal((N, 2 * m, dv)) if s0 else None))
+    up = dict(do_re=rng.standard_normal((N, T, dv)), do_im=rng.standard_normal((N, T, dv)),
+              dS_T=rng.standard_normal((N, 2 * m, dv)))
+    return x, up
+
+
+def _loss(x, up):
+    """L = sum do_re . Re o + do_im . Im o + <dS_T, S_T>, evaluated by the forward oracle."""
+    o_re, o_im, S_T = recurrence.sfda_recurrence(x["q"], x["k"], x["v"], x["alpha"], x["theta"], x["beta"], x["S0"])
+    return float(np.sum(up["do_re"] * o_re) + np.sum(up["do_im"] * o_im) + np.sum(up["dS_T"] * S_T))
+
+
+def test_backward_matches_central_differences_of_the_forward_oracle():
+    """Every gradient, entry by entry on a sample, against (L(x + h e) - L(x - h e)) / 2h of the independently
+    written forward oracle (C, per token); also across a segment boundary of the checkpointing."""
+    for seed, seg in ((0, 64), (1, 3)):
+        x, up = _loss_inputs(seed)
+        g = dict(zip(("q", "k", "v", "alpha", "theta", "beta", "S0"),
+                     backward.sfda_backward(x["q"], x["k"], x["v"], x["alpha"], x["theta"], x["beta"], x["S0"],
+                                            up["do_re"], up["do_im"], up["dS_T"], seg=seg)))
+        rng = np.random.default_rng(100 + seed)
+        h = 1e-6
+        for name in g:
+            flat = x[name].reshape(-1)
+            for idx in rng.choice(flat.size, size=min(12, flat.size), replace=False):
+                keep = flat[idx]
+                flat[idx] = keep + h
+                lp = _loss(x, up)
+                flat[idx] = keep - h
+                lm = _loss(x, up)
+                flat[idx] = keep
+                fd = (lp - lm) / (2 * h)
+                assert abs(fd - g[name].reshape(-1)[idx]) <= 2e-7 * max(1.0, abs(fd)), (name, idx, fd, g[name].reshape(-1)[idx])
+
+
+def test_backward_without_writes_is_the_adjoint_of_the_diagonal_scan():
+    """beta = 0: S_t = Gamma_t S_0 and o_t = S_0^* conj(Gamma_t) q_t (Prop. "Interpolation ..."), so
+    dS0 = sum_t conj(Gamma_t)^{-1}... written out: dS0_j = sum_t conj(gamma_tj) (q_tj yb_t^*) + conj(gamma_Tj) dS_T,j,
+    dq_t = Gamma_t S_0 yb_t, and dv = dbeta-free terms vanish (dv = 0)."""
+    x, up = _loss_inputs(3, N=1, T=6)
+    x["beta"][:] = 0.0
+    dq, dk, dv, dal, dth, dbe, dS0 = backward.sfda_backward(x["q"], x["k"], x["v"], x["alpha"], x["theta"],
+                                                             x["beta"], x["S0"], up["do_re"], up["do_im"], up["dS_T"])
+    lam = x["alpha"][0] * np.exp(1j * x["theta"][0])                 # [T, m]
+    gam = np.cumprod(lam, axis=0)
+    S0 = x["S0"][0, 0::2] + 1j * x["S0"][0, 1::2]
+    yb = up["do_re"][0] + 1j * up["do_im"][0]
+    qc = x["q"][0, :, 0::2] + 1j * x["q"][0, :, 1::2]
+    GT = up["dS_T"][0, 0::2] + 1j * up["dS_T"][0, 1::2]
+    want_dS0 = gam[-1].conj()[:, None] * GT + sum(gam[t].conj()[:, None] * np.outer(qc[t], yb[t].conj()) for t in range(6))
+    assert np.allclose(dS0[0, 0::2] + 1j * dS0[0, 1::2], want_dS0, rtol=0, atol=1e-12)
+    for t in range(6):
+        want_dq = (gam[t][:, None] * S0) @ yb[t]
+        assert np.allclose(dq[0, t, 0::2] + 1j * dq[0, t, 1::2], want_dq, rtol=0, atol=1e-12)
+    assert np.all(dv == 0) and np.all(dk == 0)
+
+
+def test_backward_is_linear_in_the_upstream_and_additive_over_a_split():
+    """The cotangents are linear in (do, dS_T); and running the second half first, then feeding its dS0 to the
+    first half as dS_T, gives the gradients of the whole sequence (Theorem "Chunk-bounded exactness", transposed)."""
+    x, up = _loss_inputs(5, N=2, T=9)
+    full = backward.sfda_backward(x["q"], x["k"], x["v"], x["alpha"], x["theta"], x["beta"], x["S0"],
+                                  up["do_re"], up["do_im"], up["dS_T"])
+    twice = backward.sfda_backward(x["q"], x["k"], x["v"], x["alpha"], x["theta"], x["beta"], x["S0"],
+                                   2 * up["do_re"], 2 * up["do_im"], 2 * up["dS_T"])
+    for a, b in zip(full, twice):
+        assert np.allclose(2 * a, b, rtol=1e-13, atol=1e-13)
+    T1 = 4
+    _, _, S_mid = recurrence.sfda_recurrence(x["q"][:, :T1], x["k"][:, :T1], x["v"][:, :T1], x["alpha"][:, :T1],
+                                             x["theta"][:, :T1], x["beta"][:, :T1], x["S0"])
+    second = backward.sfda_backward(x["q"][:, T1:], x["k"][:, T1:], x["v"][:, T1:], x["alpha"][:, T1:],
+                                    x["theta"][:, T1:], x["beta"][:, T1:], S_mid, up["do_re"][:, T1:],
+                                    up["do_im"][:, T1:], up["dS_T"])
+    first = backward.sfda_backward(x["q"][:, :T1], x["k"][:, :T1], x["v"][:, :T1], x["alpha"][:, :T1],
+                                   x["theta"][:, :T1], x["beta"][:, :T1], x["S0"], up["do_re"][:, :T1],
+                                   up["do_im"][:, :T1], second[6])
+    for i in range(6):
+        assert np.allclose(np.concatenate([first[i], second[i]], axis=1), full[i], rtol=1e-12, atol=1e-12)
+    assert np.allclose(first[6], full[6], rtol=1e-12, atol=1e-12)
