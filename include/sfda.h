@@ -294,6 +294,34 @@ SFDA_API int sfda_forward_fused(const void *q, const void *k_raw, const void *v,
                                 int B, int T, int H, int d_k, int d_v, int chunk, int dtype,
                                 void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * Backward pass: the gradients of a real loss L through the recurrence (Eq. "sfda") and o_t = S_t^* q_t, given
+ * the cotangents of the outputs.  (The paper names the backward pass only in its kernel benchmark protocol,
+ * App. E; what it computes is the adjoint of Eq. "sfda".)
+ *
+ *  inputs as sfda_forward:  q, k [B][T][H][d_k] dtype, v [B][T][H][d_v] dtype, alpha, theta [B][T][H][m] float,
+ *                           beta [B][T][H] float, S0 [B][H][d_k][d_v] float or NULL
+ *  cotangents:  d_o    [B][T][H][d_v] dtype   dL/d Re(S_t^* q_t)
+ *               d_o_im same shape or NULL     dL/d Im(S_t^* q_t)  (NULL: zero)
+ *               dS_T   [B][H][d_k][d_v] float or NULL (zero): dL/dS_T in the state's paired-row layout
+ *  gradients:   dq, dk [B][T][H][d_k] dtype (the (Re, Im) pair of a coordinate gets the gradient with respect
+ *               to its two real numbers), dv [B][T][H][d_v] dtype, dalpha, dtheta [B][T][H][m] float,
+ *               dbeta [B][T][H] float, dS0 [B][H][d_k][d_v] float.  All are required and overwritten.
+ *  workspace:   sfda_backward_workspace_bytes(...) bytes of device scratch (the state at the start of every
+ *               64 tokens and the 64 states of one such segment, per (batch, head) pair); clobbered.
+ *
+ * d_k, d_v in {64, 128}; no chunk argument (the derivative does not depend on the chunking).  fp32 arithmetic on
+ * the CUDA cores, token by token, one CTA per (batch, head) pair: a first correct path, not a fast one.  The
+ * result is deterministic (no sum crosses CTAs).
+ */
+SFDA_API size_t sfda_backward_workspace_bytes(int B, int T, int H, int d_k, int d_v, int dtype);
+SFDA_API int sfda_backward(const void *q, const void *k, const void *v,
+                           const float *alpha, const float *theta, const float *beta, const float *S0,
+                           const void *d_o, const void *d_o_im, const float *dS_T,
+                           void *dq, void *dk, void *dv, float *dalpha, float *dtheta, float *dbeta, float *dS0,
+                           int B, int T, int H, int d_k, int d_v, int dtype,
+                           void *workspace, size_t workspace_bytes, void *stream);
+
 /* Number of kernels the last sfda_forward* / sfda_step / sfda_chunk_factors / sfda_frontend call of
  * this thread enqueued (host only; for launch accounting in benchmarks). */
 SFDA_API int sfda_last_launch_count(void);

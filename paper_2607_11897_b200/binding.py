@@ -54,6 +54,9 @@ def load():
     lib.sfda_forward_fused_workspace_bytes.argtypes = [_ci] * 7
     lib.sfda_forward_fused.argtypes = [_vp] * 6 + [_cf] * 4 + [_vp] * 4 + [_ci] * 7 + [_vp, _sz, _vp]
     lib.sfda_step_fused.argtypes = [_vp] * 6 + [_cf] * 4 + [_vp] * 3 + [_ci] * 5 + [_vp]
+    lib.sfda_backward_workspace_bytes.restype = _sz
+    lib.sfda_backward_workspace_bytes.argtypes = [_ci] * 6
+    lib.sfda_backward.argtypes = [_vp] * 17 + [_ci] * 6 + [_vp, _sz, _vp]
     _LIB = lib
     return lib
 
@@ -273,3 +276,27 @@ def sfda_step_fused(q, k_raw, v, a_raw, b_raw, c_raw, alpha_min, alpha_max, thet
                                 _dtype_code(q), _stream(stream))
     if rc != 0:
         raise SfdaError(rc, "sfda_step_fused")
+
+
+def sfda_backward_workspace_bytes(B, T, H, d_k, d_v, dtype) -> int:
+    return int(load().sfda_backward_workspace_bytes(B, T, H, d_k, d_v, dtype))
+
+
+def sfda_backward(q, k, v, alpha, theta, beta, S0, d_o, d_o_im, dS_T, dq, dk, dv, dalpha, dtheta, dbeta, dS0,
+                  workspace, stream=None):
+    """``sfda_backward`` of ``include/sfda.h``: gradients of a real loss through the recurrence."""
+    B, T, H, d_k = q.shape
+    d_v = v.shape[-1]
+    for t, n in ((q, "q"), (k, "k"), (v, "v"), (d_o, "d_o"), (d_o_im, "d_o_im"), (dq, "dq"), (dk, "dk"), (dv, "dv")):
+        _check(t, n, q.dtype)
+    for t, n in ((alpha, "alpha"), (theta, "theta"), (beta, "beta"), (S0, "S0"), (dS_T, "dS_T"), (dalpha, "dalpha"),
+                 (dtheta, "dtheta"), (dbeta, "dbeta"), (dS0, "dS0")):
+        _check(t, n, torch.float32)
+    _check(workspace, "workspace")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = load().sfda_backward(_ptr(q), _ptr(k), _ptr(v), _ptr(alpha), _ptr(theta), _ptr(beta), _ptr(S0), _ptr(d_o),
+                              _ptr(d_o_im), _ptr(dS_T), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dalpha), _ptr(dtheta),
+                              _ptr(dbeta), _ptr(dS0), B, T, H, d_k, d_v, _dtype_code(q), _ptr(workspace), ws_bytes,
+                              _stream(stream))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_backward")

@@ -437,6 +437,39 @@ int sfda_forward_fused(const void *q, const void *k_raw, const void *v, const fl
     return sfda::launch_forward_simt(a, s, &g_last_launches) == cudaSuccess ? SFDA_OK : SFDA_ERR_CUDA;
 }
 
+size_t sfda_backward_workspace_bytes(int B, int T, int H, int d_k, int d_v, int dtype)
+{
+    if (B < 1 || T < 1 || H < 1 || check_dims(d_k, d_v, 64, dtype) != SFDA_OK) return 0;
+    return sfda::backward_workspace_bytes(B, T, H, d_k, d_v);
+}
+
+int sfda_backward(const void *q, const void *k, const void *v, const float *alpha, const float *theta,
+                  const float *beta, const float *S0, const void *d_o, const void *d_o_im, const float *dS_T,
+                  void *dq, void *dk, void *dv, float *dalpha, float *dtheta, float *dbeta, float *dS0, int B, int T,
+                  int H, int d_k, int d_v, int dtype, void *workspace, size_t workspace_bytes, void *stream)
+{
+    g_last_launches = 0;
+    if (!q || !k || !v || !alpha || !theta || !beta || !d_o || !dq || !dk || !dv || !dalpha || !dtheta || !dbeta ||
+        !dS0)
+        return SFDA_ERR_NULL;
+    if (B < 1 || T < 1 || H < 1) return SFDA_ERR_SHAPE;
+    const int rc = check_dims(d_k, d_v, 64, dtype);
+    if (rc != SFDA_OK) return rc;
+    const void *ptrs[] = {q, k, v, alpha, theta, beta, S0, d_o, d_o_im, dS_T, dq, dk, dv, dalpha, dtheta, dbeta, dS0,
+                          workspace};
+    for (const void *p : ptrs)
+        if (p && !aligned16(p)) return SFDA_ERR_ALIGN;
+    if (!workspace || workspace_bytes < sfda::backward_workspace_bytes(B, T, H, d_k, d_v)) return SFDA_ERR_WORKSPACE;
+    sfda::BackwardArgs a;
+    a.q = q; a.k = k; a.v = v; a.d_o = d_o; a.d_o_im = d_o_im;
+    a.alpha = alpha; a.theta = theta; a.beta = beta; a.S0 = S0; a.dS_T = dS_T;
+    a.dq = dq; a.dk = dk; a.dv = dv; a.dalpha = dalpha; a.dtheta = dtheta; a.dbeta = dbeta; a.dS0 = dS0;
+    a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.dtype = dtype;
+    return sfda::launch_backward(a, workspace, static_cast<cudaStream_t>(stream), &g_last_launches) == cudaSuccess
+               ? SFDA_OK
+               : SFDA_ERR_CUDA;
+}
+
 int sfda_last_launch_count(void) { return g_last_launches; }
 
 }  // extern "C"

@@ -1,0 +1,386 @@
+// sfda_backward: reverse-mode derivative of the recurrence of Section 3 (Eq. "sfda") with o_t = S_t^* q_t, token by
+// token in fp32 on the CUDA cores.  (The paper asks for the backward pass only as something to be timed, App. E; what
+// it computes is the adjoint of Eq. "sfda".)  This is the first correct path: one CTA per (batch, head) pair walks
+// the sequence three times --
+//
+//   1. forward, keeping the state at the start of every segment of kSeg tokens (checkpoints in the workspace);
+//   2. per segment, last to first: forward again from the checkpoint, keeping S_{t-1} of every token of the segment;
+//   3. backward through the segment with the cotangent G of the state in shared memory.
+//
+// One backward step, with Z = Lambda_t S_{t-1}, u^T = v_t^T - k_t^* Z (so S_t = Z + beta_t k_t u^T) and
+// yb_t = do_re + i do_im:
+//
+//   G += q yb^*                    p = G^* k                     dv = beta Re p            dbeta = Re(u^T p)
+//   dq = Z yb + beta k (u^T yb)    dk = beta (G conj(u) - Z p)   Zb = G - beta k p^*
+//   lamb_j = sum_c conj(S_{t-1,jc}) Zb_jc      dalpha = Re(conj(lamb) e^{i theta})     dtheta = -Im(conj(lamb) lam)
+//   G <- conj(lam) Zb   (row-wise: the cotangent of S_{t-1})
+//
+// Complex cotangents Xb mean dL = Re sum conj(Xb) dX, i.e. the ordinary gradient with respect to the (Re, Im) pair.
+// No sums cross CTAs, so the result is deterministic.
+#include "sfda_common.cuh"
+#include "sfda_internal.h"
+
+namespace sfda {
+namespace {
+
+constexpr int kBwdThreads = 512;
+constexpr int kSeg = 64;     // tokens between checkpoints
+
+template <int DK, int DV>
+struct BwdSmem {
+    static constexpr int M = DK / 2;
+    static constexpr int RS = DV + 8;            // row stride (floats): rows 8 banks apart, 16-byte aligned
+    static constexpr int NG = kBwdThreads / DV;  // row groups of the column-owner mapping
+    static constexpr int plane = M * RS;
+    // G (re, im), two buffers of S_{t-1} (re, im) and the vectors of one token
+    static constexpr size_t bytes = (size_t)(6 * plane + 6 * M + 2 * M + 8 * DV + NG * 4 * DV + 64) * 4;
+};
+
+__device__ __forceinline__ void cp_async16(float *dst_smem, const float *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst_smem)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
+struct BwdArgsDev {
+    const void *q, *k, *v, *d_o, *d_o_im;
+    const float *alpha, *theta, *beta, *S0, *dS_T;
+    void *dq, *dk, *dv;
+    float *dalpha, *dtheta, *dbeta, *dS0;
+    float *check, *scratch;      // [BH][NS][2][M][DV], [BH][kSeg][2][M][DV]
+    int T, H, NS;
+};
+
+template <int DK, int DV, typename T>
+__global__ void __launch_bounds__(kBwdThreads, 1)
+sfda_backward_kernel(const BwdArgsDev a)
+{
+    using L = BwdSmem<DK, DV>;
+    constexpr int M = L::M, RS = L::RS, NG = L::NG, RA = M / NG;      // RA rows per thread in the column mapping
+    constexpr int TPR = kBwdThreads / M, CPT = DV / TPR;               // threads per row / columns per thread (row mapping)
+    static_assert(M % NG == 0 && DV % TPR == 0 && M + DV + 1 <= kBwdThreads, "thread mappings");
+    extern __shared__ __align__(16) float sm[];
+    float *Gr = sm, *Gi = Gr + L::plane;
+    float *P0 = Gi + L::plane;                              // two S_{t-1} buffers of [re | im] planes
+    auto Pr = [&](int i) { return P0 + i * 2 * L::plane; };
+    auto Pi = [&](int i) { return P0 + i * 2 * L::plane + L::plane; };
+    float *v_lr = P0 + 4 * L::plane, *v_li = v_lr + M, *v_kr = v_li + M, *v_ki = v_kr + M, *v_qr = v_ki + M, *v_qi = v_qr + M;
+    float *v_cs = v_qi + M, *v_sn = v_cs + M;
+    float *v_v = v_sn + M, *v_yr = v_v + DV, *v_yi = v_yr + DV, *v_ur = v_yi + DV, *v_ui = v_ur + DV, *v_pr = v_ui + DV,
+          *v_pi = v_pr + DV, *v_spare = v_pi + DV;
+    float *red = v_spare + DV;                  // [NG][4][DV]
+    float *scal = red + NG * 4 * DV;            // [0] beta, [8 + 4 w + x] partial sums of warp w
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int bh = blockIdx.x, h = bh % a.H, b = bh / a.H;
+    const int T_ = a.T, H = a.H;
+    const T *q = static_cast<const T *>(a.q), *k = static_cast<const T *>(a.k), *v = static_cast<const T *>(a.v);
+    const T *d_o = static_cast<const T *>(a.d_o), *d_oi = static_cast<const T *>(a.d_o_im);
+    float *check = a.check + (size_t)bh * a.NS * 2 * M * DV;
+    float *scratch = a.scratch + (size_t)bh * kSeg * 2 * M * DV;
+
+    // column-owner mapping (A): column c, rows g, g + NG, ...;  row-owner mapping (B): row jb, columns part + TPR n
+    const int c = tid % DV, g = tid / DV;
+    const int jb = tid / TPR, part = tid % TPR;
+
+    // ---- token vectors: registers -> shared memory, one token ahead of the step that uses them
+    float r0 = 0.f, r1 = 0.f, r2 = 0.f, r3 = 0.f, r4 = 0.f, r5 = 0.f;
+    auto load_tok = [&](int t, bool back) {
+        if (t < 0 || t >= T_) return;
+        const size_t row = ((size_t)b * T_ + t) * H + h;
+        if (tid < M) {
+            r0 = a.alpha[row * M + tid];
+            r1 = a.theta[row * M + tid];
+            r2 = ld_val(k, row * DK + 2 * tid);
+            r3 = ld_val(k, row * DK + 2 * tid + 1);
+            if (back) {
+                r4 = ld_val(q, row * DK + 2 * tid);
+                r5 = ld_val(q, row * DK + 2 * tid + 1);
+            }
+        } else if (tid < M + DV) {
+            const int cc = tid - M;
+            r0 = ld_val(v, row * DV + cc);
+            if (back) {
+                r1 = ld_val(d_o, row * DV + cc);
+                r2 = d_oi ? ld_val(d_oi, row * DV + cc) : 0.f;
+            }
+        } else if (tid == M + DV) {
+            r0 = a.beta[row];
+        }
+    };
+    auto stage_tok = [&](bool back) {
+        if (tid < M) {
+            float sn, cs;
+            sincosf(r1, &sn, &cs);
+            v_cs[tid] = cs; v_sn[tid] = sn;
+            v_lr[tid] = r0 * cs; v_li[tid] = r0 * sn;
+            v_kr[tid] = r2; v_ki[tid] = r3;
+            if (back) { v_qr[tid] = r4; v_qi[tid] = r5; }
+        } else if (tid < M + DV) {
+            const int cc = tid - M;
+            v_v[cc] = r0;
+            if (back) { v_yr[cc] = r1; v_yi[cc] = r2; }
+        } else if (tid == M + DV) {
+            scal[0] = r0;
+        }
+    };
+
+    // ---- one forward step on the state in (Sr, Si); the token's vectors are staged and synchronised
+    auto fwd_step = [&](float *Sr, float *Si) {
+        float cr = 0.f, ci = 0.f;
+#pragma unroll
+        for (int r = 0; r < RA; ++r) {
+            const int j = g + NG * r;
+            const float lr = v_lr[j], li = v_li[j], kr = v_kr[j], ki = v_ki[j];
+            const float sr = Sr[j * RS + c], si = Si[j * RS + c];
+            const float zr = lr * sr - li * si, zi = lr * si + li * sr;      // Z = Lambda S
+            Sr[j * RS + c] = zr;
+            Si[j * RS + c] = zi;
+            cr += kr * zr + ki * zi;                                           // conj(k) z
+            ci += kr * zi - ki * zr;
+        }
+        red[(g * 4 + 0) * DV + c] = cr;
+        red[(g * 4 + 1) * DV + c] = ci;
+        __syncthreads();
+        float sr_ = 0.f, si_ = 0.f;
+#pragma unroll
+        for (int gg = 0; gg < NG; ++gg) {
+            sr_ += red[(gg * 4 + 0) * DV + c];
+            si_ += red[(gg * 4 + 1) * DV + c];
+        }
+        const float bt = scal[0];
+        const float er = bt * (v_v[c] - sr_), ei = -bt * si_;                  // e = beta u, u = v - k^* Z
+#pragma unroll
+        for (int r = 0; r < RA; ++r) {
+            const int j = g + NG * r;
+            const float kr = v_kr[j], ki = v_ki[j];
+            Sr[j * RS + c] += kr * er - ki * ei;
+            Si[j * RS + c] += kr * ei + ki * er;
+        }
+        __syncthreads();
+    };
+
+    // ---- state moves between shared and global memory: planes [re | im][M][DV], 16 bytes per access
+    auto store_state = [&](const float *Sr, const float *Si, float *dst) {
+        for (int idx = tid; idx < M * DV / 4; idx += kBwdThreads) {
+            const int j = idx / (DV / 4), c4 = idx % (DV / 4);
+            *reinterpret_cast<float4 *>(dst + (size_t)j * DV + 4 * c4) = *reinterpret_cast<const float4 *>(Sr + j * RS + 4 * c4);
+            *reinterpret_cast<float4 *>(dst + (size_t)(M + j) * DV + 4 * c4) = *reinterpret_cast<const float4 *>(Si + j * RS + 4 * c4);
+        }
+    };
+    auto load_state_async = [&](float *Sr, float *Si, const float *src) {
+        for (int idx = tid; idx < M * DV / 4; idx += kBwdThreads) {
+            const int j = idx / (DV / 4), c4 = idx % (DV / 4);
+            cp_async16(Sr + j * RS + 4 * c4, src + (size_t)j * DV + 4 * c4);
+            cp_async16(Si + j * RS + 4 * c4, src + (size_t)(M + j) * DV + 4 * c4);
+        }
+        cp_async_commit();
+    };
+
+    // ---- sweep 1: forward, checkpoints at the start of every segment (nothing is needed beyond the last one)
+    float *Sr = Pr(0), *Si = Pi(0);
+    for (int idx = tid; idx < M * DV; idx += kBwdThreads) {
+        const int j = idx / DV, cc = idx % DV;
+        Sr[j * RS + cc] = a.S0 ? a.S0[((size_t)bh * DK + 2 * j) * DV + cc] : 0.f;
+        Si[j * RS + cc] = a.S0 ? a.S0[((size_t)bh * DK + 2 * j + 1) * DV + cc] : 0.f;
+    }
+    const int t_last_check = (a.NS - 1) * kSeg;
+    load_tok(0, false);
+    __syncthreads();
+    for (int t = 0; t < t_last_check; ++t) {
+        if (t % kSeg == 0) store_state(Sr, Si, check + (size_t)(t / kSeg) * 2 * M * DV);
+        stage_tok(false);
+        __syncthreads();
+        load_tok(t + 1, false);
+        fwd_step(Sr, Si);
+    }
+    store_state(Sr, Si, check + (size_t)(a.NS - 1) * 2 * M * DV);
+
+    // ---- cotangent of the final state
+    for (int idx = tid; idx < M * DV; idx += kBwdThreads) {
+        const int j = idx / DV, cc = idx % DV;
+        Gr[j * RS + cc] = a.dS_T ? a.dS_T[((size_t)bh * DK + 2 * j) * DV + cc] : 0.f;
+        Gi[j * RS + cc] = a.dS_T ? a.dS_T[((size_t)bh * DK + 2 * j + 1) * DV + cc] : 0.f;
+    }
+    __syncthreads();      // also: every thread's checkpoint stores precede the loads below (same CTA, after a barrier)
+
+    T *dq = static_cast<T *>(a.dq), *dk = static_cast<T *>(a.dk), *dv = static_cast<T *>(a.dv);
+    for (int si = a.NS - 1; si >= 0; --si) {
+        const int t0 = si * kSeg, t1 = min(t0 + kSeg, T_);
+        // ---- sweep 2: forward again from the checkpoint, S_{t-1} of every token to the scratch
+        load_state_async(Sr, Si, check + (size_t)si * 2 * M * DV);
+        load_tok(t0, false);
+        cp_async_wait_all();
+        __syncthreads();
+        for (int t = t0; t < t1; ++t) {
+            store_state(Sr, Si, scratch + (size_t)(t - t0) * 2 * M * DV);
+            stage_tok(false);
+            __syncthreads();
+            load_tok(t + 1 < t1 ? t + 1 : t1 - 1, t + 1 >= t1);     // after the last one: the first backward token
+            if (t + 1 < t1) fwd_step(Sr, Si);                        // the state after the last token is not needed
+        }
+        __syncthreads();      // the scratch stores of this CTA are visible to its own later loads
+
+        // ---- sweep 3: backward through the segment; S_{t-1} arrives one token ahead in the other buffer
+        int buf = 0;
+        load_state_async(Pr(buf), Pi(buf), scratch + (size_t)(t1 - 1 - t0) * 2 * M * DV);
+        for (int t = t1 - 1; t >= t0; --t) {
+            stage_tok(true);
+            cp_async_wait_all();
+            __syncthreads();
+            const float *Qr = Pr(buf), *Qi = Pi(buf);
+            if (t > t0) load_state_async(Pr(buf ^ 1), Pi(buf ^ 1), scratch + (size_t)(t - 1 - t0) * 2 * M * DV);
+            load_tok(t - 1 >= t0 ? t - 1 : t0 - 1, true);           // (a token of the next segment down is reloaded there)
+            const float bt = scal[0];
+            const size_t row = ((size_t)b * T_ + t) * H + h;
+
+            // step 1 (columns): G += q yb^*;  partial p = G^* k and k^* Z
+            {
+                const float yr = v_yr[c], yi = v_yi[c];
+                float pr = 0.f, pi = 0.f, zr_ = 0.f, zi_ = 0.f;
+#pragma unroll
+                for (int r = 0; r < RA; ++r) {
+                    const int j = g + NG * r;
+                    const float qr = v_qr[j], qi = v_qi[j], kr = v_kr[j], ki = v_ki[j], lr = v_lr[j], li = v_li[j];
+                    const float gr = Gr[j * RS + c] + qr * yr + qi * yi;       // q conj(yb)
+                    const float gi = Gi[j * RS + c] + qi * yr - qr * yi;
+                    Gr[j * RS + c] = gr;
+                    Gi[j * RS + c] = gi;
+                    pr += gr * kr + gi * ki;                                    // conj(G) k
+                    pi += gr * ki - gi * kr;
+                    const float sr = Qr[j * RS + c], si_ = Qi[j * RS + c];
+                    const float zr = lr * sr - li * si_, zi = lr * si_ + li * sr;
+                    zr_ += kr * zr + ki * zi;                                   // conj(k) z
+                    zi_ += kr * zi - ki * zr;
+                }
+                red[(g * 4 + 0) * DV + c] = pr;
+                red[(g * 4 + 1) * DV + c] = pi;
+                red[(g * 4 + 2) * DV + c] = zr_;
+                red[(g * 4 + 3) * DV + c] = zi_;
+            }
+            __syncthreads();
+            // step 2: p, u per column; dv; the sums over columns u^T p and u^T yb
+            if (tid < DV) {
+                float pr = 0.f, pi = 0.f, zr = 0.f, zi = 0.f;
+#pragma unroll
+                for (int gg = 0; gg < NG; ++gg) {
+                    pr += red[(gg * 4 + 0) * DV + c];
+                    pi += red[(gg * 4 + 1) * DV + c];
+                    zr += red[(gg * 4 + 2) * DV + c];
+                    zi += red[(gg * 4 + 3) * DV + c];
+                }
+                const float ur = v_v[c] - zr, ui = -zi;
+                v_pr[c] = pr; v_pi[c] = pi; v_ur[c] = ur; v_ui[c] = ui;
+                st_val(dv, row * DV + c, bt * pr);
+                const float yr = v_yr[c], yi = v_yi[c];
+                float s0 = ur * pr - ui * pi;                       // Re(u p)
+                float s1 = ur * yr - ui * yi, s2 = ur * yi + ui * yr;   // u yb
+#pragma unroll
+                for (int d = 16; d >= 1; d >>= 1) {
+                    s0 += __shfl_xor_sync(0xffffffffu, s0, d);
+                    s1 += __shfl_xor_sync(0xffffffffu, s1, d);
+                    s2 += __shfl_xor_sync(0xffffffffu, s2, d);
+                }
+                if (lane == 0) { scal[8 + 4 * warp] = s0; scal[9 + 4 * warp] = s1; scal[10 + 4 * warp] = s2; }
+            }
+            __syncthreads();
+            // step 3 (rows): dq, dk, lamb, and G <- conj(lam) (G - beta k p^*)
+            {
+                float sr_ = 0.f, si_ = 0.f, dbe = 0.f;
+#pragma unroll
+                for (int w = 0; w < DV / 32; ++w) { dbe += scal[8 + 4 * w]; sr_ += scal[9 + 4 * w]; si_ += scal[10 + 4 * w]; }
+                if (tid == 0) a.dbeta[row] = dbe;
+                const int j = jb;
+                const float lr = v_lr[j], li = v_li[j], kr = v_kr[j], ki = v_ki[j];
+                float qzr = 0.f, qzi = 0.f, k1r = 0.f, k1i = 0.f, k2r = 0.f, k2i = 0.f, lbr = 0.f, lbi = 0.f;
+#pragma unroll 4
+                for (int n = 0; n < CPT; ++n) {
+                    const int cc = part + TPR * n;
+                    const float gr = Gr[j * RS + cc], gi = Gi[j * RS + cc], sr = Qr[j * RS + cc], si2 = Qi[j * RS + cc];
+                    const float zr = lr * sr - li * si2, zi = lr * si2 + li * sr;
+                    const float yr = v_yr[cc], yi = v_yi[cc], ur = v_ur[cc], ui = v_ui[cc], pr = v_pr[cc], pi = v_pi[cc];
+                    qzr += zr * yr - zi * yi;  qzi += zr * yi + zi * yr;       // Z yb
+                    k1r += gr * ur + gi * ui;  k1i += gi * ur - gr * ui;       // G conj(u)
+                    k2r += zr * pr - zi * pi;  k2i += zr * pi + zi * pr;       // Z p
+                    // Zb = G - beta k conj(p)
+                    const float br = gr - bt * (kr * pr + ki * pi), bi = gi - bt * (ki * pr - kr * pi);
+                    lbr += sr * br + si2 * bi;  lbi += sr * bi - si2 * br;     // conj(S_{t-1}) Zb
+                    Gr[j * RS + cc] = lr * br + li * bi;                       // conj(lam) Zb
+                    Gi[j * RS + cc] = lr * bi - li * br;
+                }
+#pragma unroll
+                for (int d = TPR / 2; d >= 1; d >>= 1) {
+                    qzr += __shfl_xor_sync(0xffffffffu, qzr, d);  qzi += __shfl_xor_sync(0xffffffffu, qzi, d);
+                    k1r += __shfl_xor_sync(0xffffffffu, k1r, d);  k1i += __shfl_xor_sync(0xffffffffu, k1i, d);
+                    k2r += __shfl_xor_sync(0xffffffffu, k2r, d);  k2i += __shfl_xor_sync(0xffffffffu, k2i, d);
+                    lbr += __shfl_xor_sync(0xffffffffu, lbr, d);  lbi += __shfl_xor_sync(0xffffffffu, lbi, d);
+                }
+                if (part == 0) {
+                    st_val(dq, row * DK + 2 * j, qzr + bt * (kr * sr_ - ki * si_));      // + beta k (u^T yb)
+                    st_val(dq, row * DK + 2 * j + 1, qzi + bt * (kr * si_ + ki * sr_));
+                    st_val(dk, row * DK + 2 * j, bt * (k1r - k2r));
+                    st_val(dk, row * DK + 2 * j + 1, bt * (k1i - k2i));
+                    const float cs = v_cs[j], sn = v_sn[j];
+                    a.dalpha[row * M + j] = lbr * cs + lbi * sn;                          // Re(conj(lamb) e^{i theta})
+                    a.dtheta[row * M + j] = lbi * lr - lbr * li;                          // -Im(conj(lamb) lam)
+                }
+            }
+            __syncthreads();
+            buf ^= 1;
+        }
+        Sr = Pr(0); Si = Pi(0);
+    }
+    for (int idx = tid; idx < M * DV; idx += kBwdThreads) {
+        const int j = idx / DV, cc = idx % DV;
+        a.dS0[((size_t)bh * DK + 2 * j) * DV + cc] = Gr[j * RS + cc];
+        a.dS0[((size_t)bh * DK + 2 * j + 1) * DV + cc] = Gi[j * RS + cc];
+    }
+}
+
+template <int DK, int DV, typename T>
+cudaError_t launch_typed(const BackwardArgs &x, void *workspace, cudaStream_t stream)
+{
+    using L = BwdSmem<DK, DV>;
+    auto kern = sfda_backward_kernel<DK, DV, T>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::bytes);
+    if (e != cudaSuccess) return e;
+    BwdArgsDev a;
+    a.q = x.q; a.k = x.k; a.v = x.v; a.d_o = x.d_o; a.d_o_im = x.d_o_im;
+    a.alpha = x.alpha; a.theta = x.theta; a.beta = x.beta; a.S0 = x.S0; a.dS_T = x.dS_T;
+    a.dq = x.dq; a.dk = x.dk; a.dv = x.dv; a.dalpha = x.dalpha; a.dtheta = x.dtheta; a.dbeta = x.dbeta; a.dS0 = x.dS0;
+    a.T = x.T; a.H = x.H; a.NS = (x.T + kSeg - 1) / kSeg;
+    const size_t bhn = (size_t)x.B * x.H, state = (size_t)DK * DV;
+    a.check = static_cast<float *>(workspace);
+    a.scratch = a.check + bhn * a.NS * state;
+    kern<<<(unsigned)bhn, kBwdThreads, L::bytes, stream>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+size_t backward_workspace_bytes(int B, int T, int H, int d_k, int d_v)
+{
+    const size_t ns = (size_t)(T + kSeg - 1) / kSeg;
+    return (size_t)B * H * (ns + kSeg) * d_k * d_v * sizeof(float);
+}
+
+cudaError_t launch_backward(const BackwardArgs &a, void *workspace, cudaStream_t stream, int *launches)
+{
+    cudaError_t e = cudaErrorInvalidValue;
+    if (a.dtype == 1) {
+        if (a.d_k == 128 && a.d_v == 128) e = launch_typed<128, 128, __nv_bfloat16>(a, workspace, stream);
+        else if (a.d_k == 128 && a.d_v == 64) e = launch_typed<128, 64, __nv_bfloat16>(a, workspace, stream);
+        else if (a.d_k == 64 && a.d_v == 128) e = launch_typed<64, 128, __nv_bfloat16>(a, workspace, stream);
+        else if (a.d_k == 64 && a.d_v == 64) e = launch_typed<64, 64, __nv_bfloat16>(a, workspace, stream);
+    } else {
+        if (a.d_k == 128 && a.d_v == 128) e = launch_typed<128, 128, float>(a, workspace, stream);
+        else if (a.d_k == 128 && a.d_v == 64) e = launch_typed<128, 64, float>(a, workspace, stream);
+        else if (a.d_k == 64 && a.d_v == 128) e = launch_typed<64, 128, float>(a, workspace, stream);
+        else if (a.d_k == 64 && a.d_v == 64) e = launch_typed<64, 64, float>(a, workspace, stream);
+    }
+    if (e == cudaSuccess && launches) ++*launches;
+    return e;
+}
+
+}  // namespace sfda

@@ -51,6 +51,14 @@ struct FrontendArgs {
     float alpha_min, alpha_max, theta_max, eps;
 };
 
+struct BackwardArgs {
+    const void *q, *k, *v, *d_o, *d_o_im;
+    const float *alpha, *theta, *beta, *S0, *dS_T;
+    void *dq, *dk, *dv;
+    float *dalpha, *dtheta, *dbeta, *dS0;
+    int B, T, H, d_k, d_v, dtype;
+};
+
 // Each returns a cudaError_t from configuring / launching; *launches is incremented per kernel.
 cudaError_t launch_forward_simt(const ForwardArgs &a, cudaStream_t stream, int *launches);
 // Tensor-core path (bf16, d_k = d_v = 128, chunk = 64): warp-specialised, chunk-pipelined tcgen05 kernel.
@@ -70,6 +78,10 @@ cudaError_t launch_forward_ws_static(const ForwardArgs &a, cudaStream_t stream, 
 cudaError_t read_static_status(cudaStream_t stream, uint32_t *word);
 cudaError_t launch_chunk_factors(const FactorArgs &a, cudaStream_t stream, int *launches);
 cudaError_t launch_step(const StepArgs &a, cudaStream_t stream, int *launches);
+// Reverse-mode derivative, token by token in fp32 (every supported d_k, d_v and dtype); the workspace holds the
+// checkpointed states.
+size_t backward_workspace_bytes(int B, int T, int H, int d_k, int d_v);
+cudaError_t launch_backward(const BackwardArgs &a, void *workspace, cudaStream_t stream, int *launches);
 // Stable parameterisation as a kernel of its own (every supported d_k and dtype).
 cudaError_t launch_frontend(const FrontendArgs &a, cudaStream_t stream, int *launches);
 

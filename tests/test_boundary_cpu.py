@@ -134,6 +134,29 @@ def test_stable_parameterisation_entry_points_validate_on_the_host(lib):
     assert sfda.sfda_forward_fused_workspace_bytes(2, 70, 3, 60, 64, 16, 1) == 0
 
 
+def test_backward_entry_point_validates_on_the_host(lib):
+    vp, ci = ctypes.c_void_p, ctypes.c_int
+    ok = vp(0x1000)
+
+    def bwd(ptrs, dims, ws=vp(0x2000), ws_bytes=1 << 40):
+        return lib.sfda_backward(*ptrs, *[ci(d) for d in dims], ws, ctypes.c_size_t(ws_bytes), None)
+
+    #       q   k   v   al  th  be  S0    do  do_im dS_T  dq  dk  dv  dal dth dbe dS0
+    ptrs = [ok, ok, ok, ok, ok, ok, None, ok, None, None, ok, ok, ok, ok, ok, ok, ok]
+    dims = [1, 100, 2, 128, 128, 1]
+    assert bwd([None] + ptrs[1:], dims) == -1
+    assert bwd(ptrs[:16] + [None], dims) == -1                       # every gradient is required
+    assert bwd(ptrs, [1, 0, 2, 128, 128, 1]) == -2
+    assert bwd(ptrs, [1, 100, 2, 96, 128, 1]) == -3
+    assert bwd(ptrs, [1, 100, 2, 128, 128, 3]) == -3
+    assert bwd(ptrs[:7] + [vp(0x1004)] + ptrs[8:], dims) == -4
+    need = sfda.sfda_backward_workspace_bytes(1, 100, 2, 128, 128, 1)
+    assert need == 1 * 2 * (2 + 64) * 128 * 128 * 4                  # 2 checkpoints + 64 states per (batch, head)
+    assert bwd(ptrs, dims, ws_bytes=need - 1) == -5
+    assert bwd(ptrs, dims, ws=None, ws_bytes=0) == -5
+    assert sfda.sfda_backward_workspace_bytes(1, 100, 2, 100, 128, 1) == 0
+
+
 def test_raw_input_generator_is_deterministic_and_untransformed():
     cfg = workloads.CONFIGS[1].scaled(B=2, T=64, H=2, s0_std=0.02)
     a, b = workloads.forward_raw_inputs(cfg), workloads.forward_raw_inputs(cfg)

@@ -12,7 +12,7 @@ import torch
 
 import paper_2607_11897_b200 as sfda
 import workloads
-from oracle import bookkeeping, chunk_wy, frontend, recurrence
+from oracle import backward, bookkeeping, chunk_wy, frontend, recurrence
 
 pytestmark = pytest.mark.gpu
 
@@ -642,3 +642,91 @@ def test_step_fused_iterated_matches_oracle(d_k, d_v, dtype, par):
     assert rel_err(np.stack([got_re[b, :, h] for b, h in pairs]), w_re) <= tol
     assert rel_err(np.stack([got_im[b, :, h] for b, h in pairs]), w_im) <= tol
     assert rel_err(np.stack([S[b, h].cpu().numpy() for b, h in pairs]), w_S) <= 1e-4
+
+
+# ------------------------------------------------------------------------------------------------
+# backward pass
+# ------------------------------------------------------------------------------------------------
+def run_backward(cfg, inp, up):
+    d = {k: (None if v is None else to_dev(v, cfg, k)) for k, v in inp.items()}
+    dt = d["q"].dtype
+    B, T, H = d["q"].shape[:3]
+    u = {k: (None if v is None else torch.from_numpy(np.ascontiguousarray(v)).to(DEV)) for k, v in up.items()}
+    for key in ("do_re", "do_im"):
+        if u[key] is not None:
+            u[key] = u[key].to(dt)
+    out = dict(dq=torch.empty_like(d["q"]), dk=torch.empty_like(d["k"]), dv=torch.empty_like(d["v"]),
+               dalpha=torch.empty_like(d["alpha"]), dtheta=torch.empty_like(d["theta"]),
+               dbeta=torch.empty_like(d["beta"]),
+               dS0=torch.empty(B, H, cfg.d_k, cfg.d_v, device=DEV, dtype=torch.float32))
+    n = sfda.sfda_backward_workspace_bytes(B, T, H, cfg.d_k, cfg.d_v, 1 if cfg.dtype == "bf16" else 0)
+    assert n == B * H * ((T + 63) // 64 + 64) * cfg.d_k * cfg.d_v * 4
+    ws = torch.empty(n, device=DEV, dtype=torch.uint8)
+    sfda.sfda_backward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], u["do_re"], u["do_im"],
+                       u["dS_T"], out["dq"], out["dk"], out["dv"], out["dalpha"], out["dtheta"], out["dbeta"],
+                       out["dS0"], ws)
+    torch.cuda.synchronize()
+    assert sfda.last_launch_count() == 1
+    return {k: v.float().cpu().numpy() for k, v in out.items()}
+
+
+def upstream(cfg, seed, want_im=True, want_state=True):
+    """Seeded cotangents on the storage grid of the outputs."""
+    rng = np.random.default_rng([seed, 99])
+    rnd = (lambda x: workloads.bf16_round(x)) if cfg.dtype == "bf16" else (lambda x: x.astype(np.float32))
+    return dict(do_re=rnd(rng.standard_normal((cfg.B, cfg.T, cfg.H, cfg.d_v), dtype=np.float32)),
+                do_im=rnd(rng.standard_normal((cfg.B, cfg.T, cfg.H, cfg.d_v), dtype=np.float32)) if want_im else None,
+                dS_T=rng.standard_normal((cfg.B, cfg.H, cfg.d_k, cfg.d_v), dtype=np.float32) if want_state else None)
+
+
+def check_backward(cfg, inp, up, pairs, tol):
+    got = run_backward(cfg, inp, up)
+    s = workloads.sequences(inp, pairs)
+    sel = lambda x: None if x is None else np.stack([x[b, :, h] for b, h in pairs]).astype(np.float64)
+    dS_T = None if up["dS_T"] is None else np.stack([up["dS_T"][b, h] for b, h in pairs]).astype(np.float64)
+    want = backward.sfda_backward(s["q"], s["k"], s["v"], s["alpha"], s["theta"], s["beta"], s["S0"], sel(up["do_re"]),
+                                  sel(up["do_im"]), dS_T)
+    names = ("dq", "dk", "dv", "dalpha", "dtheta", "dbeta", "dS0")
+    errs = {}
+    for name, w in zip(names, want):
+        g = np.stack([got[name][b, h] for b, h in pairs]) if name == "dS0" else \
+            np.stack([got[name][b, :, h] for b, h in pairs])
+        errs[name] = rel_err(g, w)
+    for name, e in errs.items():
+        assert e <= tol, "%s: %s rel err %.3e > %.1e (%s)" % (cfg.name, name, e, tol, errs)
+    return errs
+
+
+@pytest.mark.parametrize("d_k,d_v,T,dtype", [(128, 128, 150, "f32"), (64, 64, 64, "f32"), (128, 64, 65, "bf16"),
+                                             (64, 128, 1, "f32"), (128, 128, 200, "bf16")])
+def test_backward_matches_oracle(d_k, d_v, T, dtype):
+    cfg = workloads.CONFIGS[0].scaled(name="bwd", B=2, T=T, H=2, d_k=d_k, d_v=d_v, dtype=dtype, s0_std=0.5,
+                                      seed=80 + T)
+    inp = workloads.forward_inputs(cfg)
+    # fp32 arithmetic; bf16 storage rounds the stored dq, dk, dv once (2^-9 relative)
+    check_backward(cfg, inp, upstream(cfg, T), all_pairs(cfg), 1e-4 if dtype == "f32" else 5e-3)
+
+
+def test_backward_optional_cotangents_and_zero_state():
+    cfg = workloads.CONFIGS[0].scaled(name="bwd_opt", B=1, T=130, H=3, d_k=64, d_v=128, s0_std=0.0, seed=81)
+    inp = workloads.forward_inputs(cfg)
+    check_backward(cfg, inp, upstream(cfg, 1, want_im=False, want_state=False), all_pairs(cfg), 1e-4)
+
+
+def test_backward_decay_and_write_extremes():
+    """alpha with exact zeros, beta in {0, 1}: the adjoint needs no division, so nothing degenerates."""
+    cfg = workloads.CONFIGS[0].scaled(name="bwd_edge", B=1, T=96, H=2, d_k=128, d_v=64, alpha="u(0.0,1)",
+                                      beta="bernoulli(0.05)", s0_std=1.0, seed=82)
+    inp = workloads.forward_inputs(cfg)
+    inp["alpha"][:, ::9, :, ::3] = 0.0
+    inp["beta"][:, ::4] = 1.0
+    check_backward(cfg, inp, upstream(cfg, 2), all_pairs(cfg), 1e-4)
+
+
+def test_backward_is_deterministic():
+    cfg = workloads.CONFIGS[1].scaled(name="bwd_det", B=1, T=192, H=2, s0_std=0.1, seed=83)
+    inp, up = workloads.forward_inputs(cfg), None
+    up = upstream(cfg, 3)
+    a, b = run_backward(cfg, inp, up), run_backward(cfg, inp, up)
+    for key in a:
+        assert np.array_equal(a[key], b[key]), key
