@@ -172,6 +172,7 @@ def main():
     ap.add_argument("--re-only", action="store_true", help="write o = Re only (default: Re and Im)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--no-backward", action="store_true", help="skip the leg that times sfda_backward")
     ap.add_argument("--no-factors", action="store_true", help="skip the leg that times sfda_chunk_factors")
     ap.add_argument("--no-fused", action="store_true", help="skip the leg that times the forward on raw inputs")
     ap.add_argument("--seq-len", type=int, default=0,
@@ -336,6 +337,43 @@ def main():
                  "two_step_ms_per_step": two_ms, "two_step_tokens_per_s": cfg.B * cfg.T / (two_ms * 1e-3)}
         del r, al, th, be, kn
 
+    # backward pass (sfda_backward) on the headline inputs: token-level fp32 adjoint, a first correct path
+    bwd = None
+    if rank == 0 and not args.no_backward:
+        g = torch.Generator(device=dev)
+        g.manual_seed(1234)
+        d_o = torch.randn(o.shape, device=dev, generator=g).to(torch.bfloat16)
+        d_oi = torch.randn(o.shape, device=dev, generator=g).to(torch.bfloat16) if want_im else None
+        dS_T = torch.randn(S_T.shape, device=dev, generator=g)
+        dq, dk, dv_ = torch.empty_like(d["q"]), torch.empty_like(d["k"]), torch.empty_like(d["v"])
+        dal, dth, dbe = torch.empty_like(d["alpha"]), torch.empty_like(d["theta"]), torch.empty_like(d["beta"])
+        dS0 = torch.empty_like(S_T)
+        bws = torch.empty(sfda.sfda_backward_workspace_bytes(cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, 1),
+                          dtype=torch.uint8, device=dev)
+
+        def bstep():
+            sfda.sfda_backward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], d_o, d_oi, dS_T,
+                               dq, dk, dv_, dal, dth, dbe, dS0, bws, stream)
+
+        bstep()
+        b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        b0.record(stream)
+        for _ in range(2):
+            bstep()
+        b1.record(stream)
+        torch.cuda.synchronize()
+        b_ms = b0.elapsed_time(b1) / 2
+        rows = cfg.B * cfg.T * cfg.H
+        # inputs and cotangents read once, gradients written once (what an ideal backward moves)
+        bb = rows * ((2 * cfg.d_k + cfg.d_v) * 2 + 2 * cfg.m * 4 + 4) * 2 + rows * cfg.d_v * 2 * (2 if want_im else 1) \
+            + 3 * cfg.B * cfg.H * cfg.d_k * cfg.d_v * 4
+        bwd = {"workload": cfg.name + " (gradients of all inputs)", "ms_per_call": b_ms,
+               "tokens_per_s": cfg.B * cfg.T / (b_ms * 1e-3), "algorithmic_bytes": bb,
+               "achieved_gbs": bb / (b_ms * 1e-3) / 1e9, "workspace_bytes": int(bws.numel()),
+               "note": "token-level adjoint in fp32 on the CUDA cores, one CTA per (batch, head) pair"}
+        del d_o, d_oi, dS_T, dq, dk, dv_, dal, dth, dbe, dS0, bws
+
     # per-chunk factor export (sfda_chunk_factors) on the headline inputs: Gamma, Y, M, W and the phase turns
     factors = None
     if rank == 0 and not args.no_factors:
@@ -446,6 +484,9 @@ def main():
         roofline["traffic"] = 1.939e9 * cfg.B / 4
         roofline["traffic_source"] = "ncu capture at B=4 scaled to B=%d; Re+Im outputs" % cfg.B
 
+    if bwd is not None:
+        bwd["frac"] = bwd["achieved_gbs"] / peaks["hbm_gbs"]
+        bwd["peak_source"] = "of " + peaks["source"]
     if factors is not None:
         factors["frac"] = factors["achieved_gbs"] / peaks["hbm_gbs"]
         factors["peak_source"] = "of " + peaks["source"]
@@ -471,7 +512,7 @@ def main():
                    "chunk": cfg.chunk, "outputs": "Re+Im" if want_im else "Re", "state": "fp32", "S0": "N(0,0.02)",
                    "parallelism": "dp%d over (batch, head), no collective" % world,
                    "l2": "inputs+outputs %.2f GB per step, far larger than the 126 MB L2; no flush" % (abytes / 1e9)},
-        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "decode": decode, "fused_front_end": fused, "chunk_factors": factors,
+        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "decode": decode, "fused_front_end": fused, "chunk_factors": factors, "backward": bwd,
         "gpu_launches": launches_per_step * args.steps, "clocks": clocks.summary(),
     }
     print(json.dumps(line), flush=True)

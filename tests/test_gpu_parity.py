@@ -730,3 +730,12 @@ def test_backward_is_deterministic():
     a, b = run_backward(cfg, inp, up), run_backward(cfg, inp, up)
     for key in a:
         assert np.array_equal(a[key], b[key]), key
+
+
+def test_backward_full_size_headline_sampled():
+    """The headline sizes, in the launch configuration bench.py times; the oracle recomputes the gradients of a
+    sample of (batch, head) sequences end to end.  bf16 storage of dq, dk, dv."""
+    cfg = workloads.CONFIGS[2]
+    inp = workloads.forward_inputs(cfg)
+    pairs = [(0, 0), (cfg.B - 1, cfg.H - 1), (3, 17)]
+    check_backward(cfg, inp, upstream(cfg, 4), pairs, 5e-3)
