@@ -113,8 +113,8 @@ class ClockSampler:
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
                 "reasons": sorted(reasons), "samples": len(sm),
                 "sm_mhz_first": sm[0] if sm else None,
-                "window": "timed region plus about a second of the same launches (the timed region alone is "
-                          "shorter than one nvidia-smi sample)"}
+                "window": "timed region plus about a second of the same launches, longer until five samples are in "
+                          "(the timed region alone is shorter than one nvidia-smi sample)"}
 
 
 def cpu_oracle_throughput(cfg, n_pairs, T):
@@ -258,7 +258,8 @@ def main():
         # The timed region lasts tens of milliseconds, too short for nvidia-smi to see: the same launches go on,
         # untimed, under the sampler until it has had about a second of this load.
         t_load = time.perf_counter()
-        while time.perf_counter() - t_load < args.clock_load_s:
+        while args.clock_load_s > 0 and (time.perf_counter() - t_load < args.clock_load_s or
+                                         (len(clocks.rows) < 5 and time.perf_counter() - t_load < 4.0)):
             for _ in range(20):
                 step()
             torch.cuda.synchronize()
