@@ -57,6 +57,9 @@ def load():
     lib.sfda_backward_workspace_bytes.restype = _sz
     lib.sfda_backward_workspace_bytes.argtypes = [_ci] * 6
     lib.sfda_backward.argtypes = [_vp] * 17 + [_ci] * 6 + [_vp, _sz, _vp]
+    lib.sfda_forward_two_level_workspace_bytes.restype = _sz
+    lib.sfda_forward_two_level_workspace_bytes.argtypes = [_ci] * 8
+    lib.sfda_forward_two_level.argtypes = [_vp] * 10 + [_ci] * 8 + [_vp, _sz, _vp]
     _LIB = lib
     return lib
 
@@ -300,3 +303,23 @@ def sfda_backward(q, k, v, alpha, theta, beta, S0, d_o, d_o_im, dS_T, dq, dk, dv
                               _stream(stream))
     if rc != 0:
         raise SfdaError(rc, "sfda_backward")
+
+
+def sfda_forward_two_level_workspace_bytes(B, T, H, d_k, d_v, chunk, dtype, n_slices=0) -> int:
+    return int(load().sfda_forward_two_level_workspace_bytes(B, T, H, d_k, d_v, chunk, dtype, n_slices))
+
+
+def sfda_forward_two_level(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chunk, n_slices, workspace, stream=None):
+    """``sfda_forward_two_level`` of ``include/sfda.h``: the forward as a two-level scan over time slices."""
+    B, T, H, d_k = q.shape
+    d_v = v.shape[-1]
+    for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o"), (o_im, "o_im")):
+        _check(t, n, q.dtype)
+    for t, n in ((alpha, "alpha"), (theta, "theta"), (beta, "beta"), (S0, "S0"), (S_T, "S_T")):
+        _check(t, n, torch.float32)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = load().sfda_forward_two_level(_ptr(q), _ptr(k), _ptr(v), _ptr(alpha), _ptr(theta), _ptr(beta), _ptr(S0),
+                                       _ptr(o), _ptr(o_im), _ptr(S_T), B, T, H, d_k, d_v, chunk, _dtype_code(q),
+                                       int(n_slices), _ptr(workspace), ws_bytes, _stream(stream))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_forward_two_level")

@@ -105,6 +105,18 @@ size_t staged_frontend_bytes(size_t rows, int d_k, int dtype)
     return 2 * round256(rows * (d_k / 2) * 4) + round256(rows * 4) + round256(rows * d_k * elem_bytes(dtype));
 }
 
+// Time slices of the two-level scan when the caller leaves the choice to the library: the largest power of two that
+// keeps B H n within the SM count of the current device with at least 16 chunks per slice (1: do not slice).
+int auto_slices(int B, int T, int H, int chunk)
+{
+    int dev = 0, n_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return 1;
+    int n = 1;
+    while ((long long)2 * n * B * H <= n_sm && T % (2 * n * chunk) == 0 && T / (2 * n * chunk) >= 16) n *= 2;
+    return n;
+}
+
 int step_common(const void *q, const void *k, const void *v, const float *alpha, const float *theta,
                 const float *beta, float *S, void *o, void *o_im, int B, int H, int d_k, int d_v, int dtype,
                 const sfda::StepParam &par, void *stream)
@@ -196,6 +208,43 @@ int sfda_forward(const void *q, const void *k, const void *v, const float *alpha
                                       &g_last_launches)
             : sfda::launch_forward_simt(a, static_cast<cudaStream_t>(stream), &g_last_launches);
     return e == cudaSuccess ? SFDA_OK : SFDA_ERR_CUDA;
+}
+
+size_t sfda_forward_two_level_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int dtype,
+                                              int n_slices)
+{
+    if (B < 1 || T < 1 || H < 1 || n_slices < 0 || check_dims(d_k, d_v, chunk, dtype) != SFDA_OK) return 0;
+    sfda::ForwardArgs a{};
+    a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.chunk = chunk; a.dtype = dtype;
+    if (!sfda::forward_ws_supported(a)) return 0;
+    const int n = n_slices ? n_slices : auto_slices(B, T, H, chunk);
+    if (n == 1) return sfda::forward_ws_scratch_bytes(B, H);
+    return sfda::forward_two_level_supported(a, n) ? sfda::forward_two_level_bytes(a, n) : 0;
+}
+
+int sfda_forward_two_level(const void *q, const void *k, const void *v, const float *alpha, const float *theta,
+                           const float *beta, const float *S0, void *o, void *o_im, float *S_T, int B, int T, int H,
+                           int d_k, int d_v, int chunk, int dtype, int n_slices, void *workspace,
+                           size_t workspace_bytes, void *stream)
+{
+    g_last_launches = 0;
+    const int rc = validate_forward(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
+    if (rc != SFDA_OK) return rc;
+    if (n_slices < 0 || n_slices == 1) return SFDA_ERR_SHAPE;
+    const sfda::ForwardArgs a = pack(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
+    if (!sfda::forward_ws_supported(a)) return SFDA_ERR_UNSUPPORTED;
+    if (workspace && !aligned16(workspace)) return SFDA_ERR_ALIGN;
+    const int n = n_slices ? n_slices : auto_slices(B, T, H, chunk);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (n == 1) {       // nothing to gain: the plain forward
+        if (!workspace || workspace_bytes < sfda::kWsMinScratchBytes) return SFDA_ERR_WORKSPACE;
+        return sfda::launch_forward_ws(a, workspace, workspace_bytes, s, &g_last_launches) == cudaSuccess ? SFDA_OK
+                                                                                                          : SFDA_ERR_CUDA;
+    }
+    if (!sfda::forward_two_level_supported(a, n)) return SFDA_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < sfda::forward_two_level_bytes(a, n)) return SFDA_ERR_WORKSPACE;
+    return sfda::launch_forward_two_level(a, n, workspace, s, &g_last_launches) == cudaSuccess ? SFDA_OK
+                                                                                                : SFDA_ERR_CUDA;
 }
 
 int sfda_forward_noalloc(const void *q, const void *k, const void *v, const float *alpha, const float *theta,

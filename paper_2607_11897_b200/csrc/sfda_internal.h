@@ -78,6 +78,11 @@ cudaError_t launch_forward_ws_static(const ForwardArgs &a, cudaStream_t stream, 
 cudaError_t read_static_status(cudaStream_t stream, uint32_t *word);
 cudaError_t launch_chunk_factors(const FactorArgs &a, cudaStream_t stream, int *launches);
 cudaError_t launch_step(const StepArgs &a, cudaStream_t stream, int *launches);
+// Two-level scan over n time slices of every sequence (tensor-core shapes, T a multiple of n * chunk): three passes
+// of the chunk forward on the [B n][T / n] view of the same memory plus a small scan kernel.
+bool forward_two_level_supported(const ForwardArgs &a, int n);
+size_t forward_two_level_bytes(const ForwardArgs &a, int n);
+cudaError_t launch_forward_two_level(const ForwardArgs &a, int n, void *workspace, cudaStream_t stream, int *launches);
 // Reverse-mode derivative, token by token in fp32 (every supported d_k, d_v and dtype); the workspace holds the
 // checkpointed states.
 size_t backward_workspace_bytes(int B, int T, int H, int d_k, int d_v);

@@ -134,6 +134,29 @@ def test_stable_parameterisation_entry_points_validate_on_the_host(lib):
     assert sfda.sfda_forward_fused_workspace_bytes(2, 70, 3, 60, 64, 16, 1) == 0
 
 
+def test_two_level_entry_point_validates_on_the_host(lib):
+    vp, ci = ctypes.c_void_p, ctypes.c_int
+    ok = vp(0x1000)
+
+    def two(ptrs, dims, n, ws=vp(0x2000), ws_bytes=1 << 40):
+        return lib.sfda_forward_two_level(*ptrs, *[ci(d) for d in dims], ci(n), ws, ctypes.c_size_t(ws_bytes), None)
+
+    ptrs, dims = [ok] * 6 + [None, ok, None, None], [1, 2048, 2, 128, 128, 64, 1]
+    assert two([None] + ptrs[1:], dims, 2) == -1
+    assert two(ptrs, [1, 0, 2, 128, 128, 64, 1], 2) == -2
+    assert two(ptrs, dims, 1) == -2 and two(ptrs, dims, -3) == -2
+    assert two(ptrs, [1, 2048, 2, 64, 64, 16, 0], 2) == -3            # not a tensor-core shape
+    assert two(ptrs, dims, 3) == -3                                    # 2048 tokens do not split into 3 x k x 64
+    assert two(ptrs, dims, 64) == -3                                   # half a chunk per slice
+    need = sfda.sfda_forward_two_level_workspace_bytes(1, 2048, 2, 128, 128, 64, 1, 2)
+    r256 = lambda x: (x + 255) // 256 * 256
+    states, tokens = 1 * 2 * 2 * 128 * 128 * 4, 1 * 2048 * 2 * 128 * 2
+    assert need == r256(sfda.sfda_workspace_bytes(2, 1024, 2, 128, 128, 64, 1)) + 5 * r256(states) + 2 * r256(tokens)
+    assert two(ptrs, dims, 2, ws_bytes=need - 1) == -5
+    assert sfda.sfda_forward_two_level_workspace_bytes(1, 2048, 2, 128, 128, 64, 1, 3) == 0
+    assert sfda.sfda_forward_two_level_workspace_bytes(1, 2048, 2, 64, 64, 16, 0, 2) == 0
+
+
 def test_backward_entry_point_validates_on_the_host(lib):
     vp, ci = ctypes.c_void_p, ctypes.c_int
     ok = vp(0x1000)

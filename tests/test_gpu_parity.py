@@ -739,3 +739,62 @@ def test_backward_full_size_headline_sampled():
     inp = workloads.forward_inputs(cfg)
     pairs = [(0, 0), (cfg.B - 1, cfg.H - 1), (3, 17)]
     check_backward(cfg, inp, upstream(cfg, 4), pairs, 5e-3)
+
+
+# ------------------------------------------------------------------------------------------------
+# two-level scan over time slices
+# ------------------------------------------------------------------------------------------------
+def run_two_level(cfg, inp, n_slices, want_im=True, want_state=True):
+    d = {k: (None if v is None else to_dev(v, cfg, k)) for k, v in inp.items()}
+    B, T, H = d["q"].shape[:3]
+    o = torch.empty(B, T, H, cfg.d_v, device=DEV, dtype=d["q"].dtype)
+    o_im = torch.empty_like(o) if want_im else None
+    S_T = torch.empty(B, H, cfg.d_k, cfg.d_v, device=DEV, dtype=torch.float32) if want_state else None
+    n = sfda.sfda_forward_two_level_workspace_bytes(B, T, H, cfg.d_k, cfg.d_v, cfg.chunk, 1, n_slices)
+    assert n > 0
+    ws = torch.empty(n, device=DEV, dtype=torch.uint8)
+    sfda.sfda_forward_two_level(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im, S_T,
+                                cfg.chunk, n_slices, ws)
+    torch.cuda.synchronize()
+    launches = sfda.last_launch_count()
+    assert sfda.sfda_workspace_status(ws) == 0
+    return (o.float().cpu().numpy(), None if o_im is None else o_im.float().cpu().numpy(),
+            None if S_T is None else S_T.cpu().numpy(), launches)
+
+
+@pytest.mark.parametrize("B,T,H,n_slices,s0", [(1, 2048, 2, 2, 0.3), (2, 2048, 1, 4, 0.0), (1, 4096, 3, 8, 0.3),
+                                               (1, 2048, 2, 0, 0.3)])
+def test_forward_two_level_matches_oracle(B, T, H, n_slices, s0):
+    cfg = workloads.CONFIGS[1].scaled(name="two_level", B=B, T=T, H=H, s0_std=s0, seed=90 + n_slices)
+    inp = workloads.forward_inputs(cfg)
+    pairs = all_pairs(cfg)
+    o, o_im, S_T, launches = run_two_level(cfg, inp, n_slices)
+    w_re, w_im, w_S = oracle_pairs(inp, pairs)
+    assert rel_err(np.stack([o[b, :, h] for b, h in pairs]), w_re) <= TOL["bf16"]
+    assert rel_err(np.stack([o_im[b, :, h] for b, h in pairs]), w_im) <= TOL["bf16"]
+    assert rel_err(np.stack([S_T[b, h] for b, h in pairs]), w_S) <= TOL["bf16"]
+    assert launches == 6          # two fills, three forward passes, one scan (n_slices = 0 picks 2 slices here)
+
+
+def test_forward_two_level_optional_outputs_and_agreement_with_the_plain_forward():
+    cfg = workloads.CONFIGS[1].scaled(name="two_level_opt", B=1, T=4096, H=2, s0_std=0.1, seed=95)
+    inp = workloads.forward_inputs(cfg)
+    o2, none_im, none_S, _ = run_two_level(cfg, inp, 4, want_im=False, want_state=False)
+    assert none_im is None and none_S is None
+    o1, _, _ = run_forward(cfg, inp)
+    assert rel_err(o2, o1) <= TOL["bf16"]
+
+
+def test_forward_two_level_long_context_sampled():
+    """Configuration 3 (B=1, T=131072, H=16: 16 sequences on 148 SMs) with the library's own choice of slices;
+    the oracle recomputes sampled heads end to end."""
+    cfg = workloads.CONFIGS[3]
+    inp = workloads.forward_inputs(cfg)
+    pairs = [(0, 0), (0, 9)]
+    o, o_im, S_T, launches = run_two_level(cfg, inp, 0)
+    assert launches == 6
+    assert np.isfinite(o).all() and np.isfinite(o_im).all() and np.isfinite(S_T).all()
+    w_re, w_im, w_S = oracle_pairs(inp, pairs)
+    assert rel_err(np.stack([o[b, :, h] for b, h in pairs]), w_re) <= TOL["bf16"]
+    assert rel_err(np.stack([o_im[b, :, h] for b, h in pairs]), w_im) <= TOL["bf16"]
+    assert rel_err(np.stack([S_T[b, h] for b, h in pairs]), w_S) <= TOL["bf16"]
