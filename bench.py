@@ -172,6 +172,8 @@ def main():
     ap.add_argument("--re-only", action="store_true", help="write o = Re only (default: Re and Im)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--no-long-context", action="store_true",
+                    help="skip the leg that times configuration 3 with and without the two-level scan")
     ap.add_argument("--no-backward", action="store_true", help="skip the leg that times sfda_backward")
     ap.add_argument("--no-factors", action="store_true", help="skip the leg that times sfda_chunk_factors")
     ap.add_argument("--no-fused", action="store_true", help="skip the leg that times the forward on raw inputs")
@@ -337,6 +339,49 @@ def main():
                  "frontend_achieved_gbs": fbytes / (front_ms * 1e-3) / 1e9,
                  "two_step_ms_per_step": two_ms, "two_step_tokens_per_s": cfg.B * cfg.T / (two_ms * 1e-3)}
         del r, al, th, be, kn
+
+    # few, long sequences (configuration 3: 16 sequences of 131072 tokens): the plain forward, one serial chain per
+    # sequence, beside the two-level scan over time slices
+    longctx = None
+    if rank == 0 and not args.no_long_context:
+        lcfg = workloads.CONFIGS[3]
+        linp = workloads.forward_inputs(lcfg)
+        ld = {}
+        for key, val in linp.items():
+            if val is None:
+                ld[key] = None
+                continue
+            t = torch.from_numpy(np.ascontiguousarray(val))
+            ld[key] = (t.to(torch.bfloat16) if key in ("q", "k", "v") else t).to(dev)
+        del linp
+        lo = torch.empty(lcfg.B, lcfg.T, lcfg.H, lcfg.d_v, device=dev, dtype=torch.bfloat16)
+        lo_im = torch.empty_like(lo)
+        lS = torch.empty(lcfg.B, lcfg.H, lcfg.d_k, lcfg.d_v, device=dev)
+        lws = torch.empty(sfda.sfda_forward_two_level_workspace_bytes(lcfg.B, lcfg.T, lcfg.H, lcfg.d_k, lcfg.d_v,
+                                                                      lcfg.chunk, 1, 0), dtype=torch.uint8, device=dev)
+
+        def timed3(fn):
+            fn()
+            t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            t0.record(stream)
+            for _ in range(3):
+                fn()
+            t1.record(stream)
+            torch.cuda.synchronize()
+            return t0.elapsed_time(t1) / 3
+
+        plain_ms = timed3(lambda: sfda.sfda_forward(ld["q"], ld["k"], ld["v"], ld["alpha"], ld["theta"], ld["beta"],
+                                                    ld["S0"], lo, lo_im, lS, lcfg.chunk, lws, stream))
+        two_ms = timed3(lambda: sfda.sfda_forward_two_level(ld["q"], ld["k"], ld["v"], ld["alpha"], ld["theta"],
+                                                            ld["beta"], ld["S0"], lo, lo_im, lS, lcfg.chunk, 0, lws,
+                                                            stream))
+        assert sfda.sfda_workspace_status(lws, stream) == 0
+        longctx = {"workload": lcfg.name + " (B=1, T=131072, H=16)", "plain_ms_per_step": plain_ms,
+                   "plain_tokens_per_s": lcfg.B * lcfg.T / (plain_ms * 1e-3), "two_level_ms_per_step": two_ms,
+                   "two_level_tokens_per_s": lcfg.B * lcfg.T / (two_ms * 1e-3),
+                   "two_level_launches": sfda.last_launch_count(), "workspace_bytes": int(lws.numel())}
+        del ld, lo, lo_im, lS, lws
 
     # backward pass (sfda_backward) on the headline inputs: token-level fp32 adjoint, a first correct path
     bwd = None
@@ -513,7 +558,7 @@ def main():
                    "chunk": cfg.chunk, "outputs": "Re+Im" if want_im else "Re", "state": "fp32", "S0": "N(0,0.02)",
                    "parallelism": "dp%d over (batch, head), no collective" % world,
                    "l2": "inputs+outputs %.2f GB per step, far larger than the 126 MB L2; no flush" % (abytes / 1e9)},
-        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "decode": decode, "fused_front_end": fused, "chunk_factors": factors, "backward": bwd,
+        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "decode": decode, "fused_front_end": fused, "chunk_factors": factors, "backward": bwd, "long_context": longctx,
         "gpu_launches": launches_per_step * args.steps, "clocks": clocks.summary(),
     }
     print(json.dumps(line), flush=True)

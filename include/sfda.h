@@ -130,7 +130,7 @@ SFDA_API int sfda_forward(const void *q, const void *k, const void *v,
  *
  * Arguments, layouts and results as sfda_forward.  n_slices >= 2 must divide T into multiples of chunk;
  * n_slices = 0 lets the library choose (the largest power of two with B H n_slices <= the device's SM count and at
- * least 16 chunks per slice; if that is 1, the call is sfda_forward).  Only the shapes of the tensor-core path
+ * least 16 chunks per slice; below 4 slices the three passes cannot pay and the call is sfda_forward).  Only the shapes of the tensor-core path
  * (bf16, d_k = d_v = 128, chunk = 64) -> SFDA_ERR_UNSUPPORTED otherwise, also for an n_slices that does not divide.
  * workspace: sfda_forward_two_level_workspace_bytes(...) bytes (the forward's own scratch, five sets of
  * B n_slices H states, a zero v and an unread output of the size of v); all of it is required.

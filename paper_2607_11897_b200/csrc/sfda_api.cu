@@ -106,7 +106,8 @@ size_t staged_frontend_bytes(size_t rows, int d_k, int dtype)
 }
 
 // Time slices of the two-level scan when the caller leaves the choice to the library: the largest power of two that
-// keeps B H n within the SM count of the current device with at least 16 chunks per slice (1: do not slice).
+// keeps B H n within the SM count of the current device with at least 16 chunks per slice; 1 (do not slice) unless
+// that is at least 4.
 int auto_slices(int B, int T, int H, int chunk)
 {
     int dev = 0, n_sm = 0;
@@ -114,7 +115,7 @@ int auto_slices(int B, int T, int H, int chunk)
         return 1;
     int n = 1;
     while ((long long)2 * n * B * H <= n_sm && T % (2 * n * chunk) == 0 && T / (2 * n * chunk) >= 16) n *= 2;
-    return n;
+    return n >= 4 ? n : 1;      // three passes of T / n tokens each: fewer than four slices cannot pay
 }
 
 int step_common(const void *q, const void *k, const void *v, const float *alpha, const float *theta,

@@ -773,7 +773,9 @@ def test_forward_two_level_matches_oracle(B, T, H, n_slices, s0):
     assert rel_err(np.stack([o[b, :, h] for b, h in pairs]), w_re) <= TOL["bf16"]
     assert rel_err(np.stack([o_im[b, :, h] for b, h in pairs]), w_im) <= TOL["bf16"]
     assert rel_err(np.stack([S_T[b, h] for b, h in pairs]), w_S) <= TOL["bf16"]
-    assert launches == 6          # two fills, three forward passes, one scan (n_slices = 0 picks 2 slices here)
+    # two fills, three forward passes, one scan; left to itself the library does not slice two sequences of 32
+    # chunks (fewer than four slices cannot pay) and runs the plain forward
+    assert launches == (6 if n_slices else 1)
 
 
 def test_forward_two_level_optional_outputs_and_agreement_with_the_plain_forward():
