@@ -172,6 +172,8 @@ def main():
     ap.add_argument("--re-only", action="store_true", help="write o = Re only (default: Re and Im)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--two-level", action="store_true",
+                    help="sweeps only: time sfda_forward_two_level (slices chosen by the library) instead of sfda_forward")
     ap.add_argument("--no-long-context", action="store_true",
                     help="skip the leg that times configuration 3 with and without the two-level scan")
     ap.add_argument("--no-backward", action="store_true", help="skip the leg that times sfda_backward")
@@ -229,13 +231,20 @@ def main():
     o = torch.empty(cfg.B, cfg.T, cfg.H, cfg.d_v, device=dev, dtype=torch.bfloat16)
     o_im = torch.empty_like(o) if want_im else None
     S_T = torch.empty(cfg.B, cfg.H, cfg.d_k, cfg.d_v, device=dev)
-    ws = torch.empty(max(sfda.sfda_workspace_bytes(cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk, 1), 256),
-                     dtype=torch.uint8, device=dev)
+    ws_bytes = sfda.sfda_workspace_bytes(cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk, 1)
+    if args.two_level:
+        ws_bytes = max(ws_bytes, sfda.sfda_forward_two_level_workspace_bytes(cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v,
+                                                                              cfg.chunk, 1, 0))
+    ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
 
     def step():
-        sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im, S_T,
-                          cfg.chunk, ws, stream)
+        if args.two_level:      # sweeps only: the library slices the time axis when that pays (few, long sequences)
+            sfda.sfda_forward_two_level(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im,
+                                        S_T, cfg.chunk, 0, ws, stream)
+        else:
+            sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im, S_T,
+                              cfg.chunk, ws, stream)
 
     def barrier():
         if world > 1:
