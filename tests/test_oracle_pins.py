@@ -611,3 +611,59 @@ def test_backward_is_linear_in_the_upstream_and_additive_over_a_split():
     for i in range(6):
         assert np.allclose(np.concatenate([first[i], second[i]], axis=1), full[i], rtol=1e-12, atol=1e-12)
     assert np.allclose(first[6], full[6], rtol=1e-12, atol=1e-12)
+
+
+# ----------------------------------------------------------------------------
+# identities the CUDA path leans on, checked on the oracle alone
+# ----------------------------------------------------------------------------
+def test_key_normalisation_is_a_rescaling_of_beta_and_v():
+    """Eq. "sfda" with k = s k_raw equals Eq. "sfda" with k_raw, beta s^2 in place of beta and v / s in place of v
+    (erase term beta s^2 k_raw k_raw^*, write term (beta s^2) k_raw (v / s)^*): states and outputs agree.  The fused
+    forward never divides the key and relies on exactly this."""
+    rng = np.random.default_rng(21)
+    N, T, m, dv = 2, 30, 4, 5
+    q = rng.standard_normal((N, T, 2 * m))
+    k_raw = rng.standard_normal((N, T, 2 * m)) * np.exp(rng.standard_normal((N, T, 1)))
+    v = rng.standard_normal((N, T, dv))
+    alpha, theta = rng.uniform(0.6, 1.0, (N, T, m)), rng.uniform(-np.pi, np.pi, (N, T, m))
+    beta = rng.uniform(0.0, 1.0, (N, T))
+    S0 = rng.standard_normal((N, 2 * m, dv))
+    s = 1.0 / (np.linalg.norm(k_raw, axis=-1) + 1e-6)
+    a = recurrence.sfda_recurrence(q, k_raw * s[..., None], v, alpha, theta, beta, S0)
+    b = recurrence.sfda_recurrence(q, k_raw, v / s[..., None], alpha, theta, beta * s * s, S0)
+    for x, y in zip(a, b):
+        assert np.allclose(x, y, rtol=1e-11, atol=1e-11)
+
+
+def test_time_slice_transfer_from_the_identity_state_and_the_zero_state():
+    """Over a time slice S_out = P S_in + B (Theorem "Exact affine chunk transfer"): B is what the slice reaches from
+    a zero state, and P is read off the first m columns of what it reaches with v = 0 from the state [I | 0].
+    Scanning S_{i+1} = P_i S_i + B_i over the slices reproduces the states of the whole sequence, and the outputs of
+    every slice from its scanned state are those of the whole sequence: the two-level scan is exact."""
+    rng = np.random.default_rng(22)
+    N, T, m, dv, n = 2, 24, 3, 4, 4
+    q, k = rng.standard_normal((N, T, 2 * m)), 0.7 * rng.standard_normal((N, T, 2 * m))
+    v = rng.standard_normal((N, T, dv))
+    alpha, theta = rng.uniform(0.6, 1.0, (N, T, m)), rng.uniform(-np.pi, np.pi, (N, T, m))
+    beta = rng.uniform(0.0, 1.0, (N, T))
+    S0 = rng.standard_normal((N, 2 * m, dv))
+    o_re, o_im, S_T = recurrence.sfda_recurrence(q, k, v, alpha, theta, beta, S0)
+    L = T // n
+    ident = np.zeros((N, 2 * m, m))                    # complex identity in paired rows: Re row 2j, column j
+    for j in range(m):
+        ident[:, 2 * j, j] = 1.0
+    S = S0[:, 0::2] + 1j * S0[:, 1::2]
+    for i in range(n):
+        sl = slice(i * L, (i + 1) * L)
+        S_in = np.empty((N, 2 * m, dv))
+        S_in[:, 0::2], S_in[:, 1::2] = S.real, S.imag
+        got_re, got_im, _ = recurrence.sfda_recurrence(q[:, sl], k[:, sl], v[:, sl], alpha[:, sl], theta[:, sl],
+                                                       beta[:, sl], S_in)
+        assert np.allclose(got_re, o_re[:, sl], atol=1e-11) and np.allclose(got_im, o_im[:, sl], atol=1e-11)
+        _, _, Bp = recurrence.sfda_recurrence(q[:, sl], k[:, sl], v[:, sl], alpha[:, sl], theta[:, sl], beta[:, sl], None)
+        _, _, Pp = recurrence.sfda_recurrence(q[:, sl], k[:, sl], np.zeros((N, L, m)), alpha[:, sl], theta[:, sl],
+                                              beta[:, sl], ident)
+        P = Pp[:, 0::2] + 1j * Pp[:, 1::2]            # [N, m, m]
+        Bc = Bp[:, 0::2] + 1j * Bp[:, 1::2]
+        S = np.einsum("njl,nlc->njc", P, S) + Bc
+    assert np.allclose(S.real, S_T[:, 0::2], atol=1e-11) and np.allclose(S.imag, S_T[:, 1::2], atol=1e-11)
