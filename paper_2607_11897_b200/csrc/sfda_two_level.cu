@@ -20,7 +20,7 @@
 namespace sfda {
 namespace {
 
-constexpr int kScanThreads = 256;
+constexpr int kScanThreads = 1024;
 
 // S0 of pass 1b: the complex identity in the first M columns, zero elsewhere (paired rows: row 2j is Re of coordinate j).
 __global__ void two_level_identity_kernel(float *__restrict__ S, int d_k, int d_v, size_t n_states)
