@@ -33,7 +33,7 @@ struct BwdSmem {
     static constexpr int NG = kBwdThreads / DV;  // row groups of the column-owner mapping
     static constexpr int plane = M * RS;
     // G (re, im), two buffers of S_{t-1} (re, im) and the vectors of one token
-    static constexpr size_t bytes = (size_t)(6 * plane + 6 * M + 2 * M + 8 * DV + NG * 4 * DV + 64) * 4;
+    static constexpr size_t bytes = (size_t)(6 * plane + 8 * M + 7 * DV + NG * 4 * DV + 64) * 4;
 };
 
 __device__ __forceinline__ void cp_async16(float *dst_smem, const float *src)
@@ -65,11 +65,15 @@ sfda_backward_kernel(const BwdArgsDev a)
     float *P0 = Gi + L::plane;                              // two S_{t-1} buffers of [re | im] planes
     auto Pr = [&](int i) { return P0 + i * 2 * L::plane; };
     auto Pi = [&](int i) { return P0 + i * 2 * L::plane + L::plane; };
-    float *v_lr = P0 + 4 * L::plane, *v_li = v_lr + M, *v_kr = v_li + M, *v_ki = v_kr + M, *v_qr = v_ki + M, *v_qi = v_qr + M;
-    float *v_cs = v_qi + M, *v_sn = v_cs + M;
-    float *v_v = v_sn + M, *v_yr = v_v + DV, *v_yi = v_yr + DV, *v_ur = v_yi + DV, *v_ui = v_ur + DV, *v_pr = v_ui + DV,
-          *v_pi = v_pr + DV, *v_spare = v_pi + DV;
-    float *red = v_spare + DV;                  // [NG][4][DV]
+    // per-row vectors of the token, packed so that one (broadcast) load fetches all a step needs of a row:
+    // (lam re, lam im, k re, k im), (q re, q im, cos theta, sin theta); per-column vectors likewise:
+    // (yb re, yb im, u re, u im), (p re, p im), v
+    float4 *v_lk = reinterpret_cast<float4 *>(P0 + 4 * L::plane);
+    float4 *v_qc = v_lk + M;
+    float4 *v_yu = v_qc + M;
+    float2 *v_p = reinterpret_cast<float2 *>(v_yu + DV);
+    float *v_v = reinterpret_cast<float *>(v_p + DV);
+    float *red = v_v + DV;                      // [NG][4][DV]
     float *scal = red + NG * 4 * DV;            // [0] beta, [8 + 4 w + x] partial sums of warp w
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -113,14 +117,12 @@ sfda_backward_kernel(const BwdArgsDev a)
         if (tid < M) {
             float sn, cs;
             sincosf(r1, &sn, &cs);
-            v_cs[tid] = cs; v_sn[tid] = sn;
-            v_lr[tid] = r0 * cs; v_li[tid] = r0 * sn;
-            v_kr[tid] = r2; v_ki[tid] = r3;
-            if (back) { v_qr[tid] = r4; v_qi[tid] = r5; }
+            v_lk[tid] = make_float4(r0 * cs, r0 * sn, r2, r3);
+            if (back) v_qc[tid] = make_float4(r4, r5, cs, sn);
         } else if (tid < M + DV) {
             const int cc = tid - M;
             v_v[cc] = r0;
-            if (back) { v_yr[cc] = r1; v_yi[cc] = r2; }
+            if (back) v_yu[cc] = make_float4(r1, r2, 0.f, 0.f);
         } else if (tid == M + DV) {
             scal[0] = r0;
         }
@@ -128,17 +130,16 @@ sfda_backward_kernel(const BwdArgsDev a)
 
     // ---- one forward step on the state in (Sr, Si); the token's vectors are staged and synchronised
     auto fwd_step = [&](float *Sr, float *Si) {
-        float cr = 0.f, ci = 0.f;
+        float cr = 0.f, ci = 0.f, zr[RA], zi[RA];
 #pragma unroll
         for (int r = 0; r < RA; ++r) {
             const int j = g + NG * r;
-            const float lr = v_lr[j], li = v_li[j], kr = v_kr[j], ki = v_ki[j];
+            const float4 lk = v_lk[j];
             const float sr = Sr[j * RS + c], si = Si[j * RS + c];
-            const float zr = lr * sr - li * si, zi = lr * si + li * sr;      // Z = Lambda S
-            Sr[j * RS + c] = zr;
-            Si[j * RS + c] = zi;
-            cr += kr * zr + ki * zi;                                           // conj(k) z
-            ci += kr * zi - ki * zr;
+            zr[r] = lk.x * sr - lk.y * si;                                     // Z = Lambda S
+            zi[r] = lk.x * si + lk.y * sr;
+            cr += lk.z * zr[r] + lk.w * zi[r];                                 // conj(k) z
+            ci += lk.z * zi[r] - lk.w * zr[r];
         }
         red[(g * 4 + 0) * DV + c] = cr;
         red[(g * 4 + 1) * DV + c] = ci;
@@ -154,9 +155,9 @@ sfda_backward_kernel(const BwdArgsDev a)
 #pragma unroll
         for (int r = 0; r < RA; ++r) {
             const int j = g + NG * r;
-            const float kr = v_kr[j], ki = v_ki[j];
-            Sr[j * RS + c] += kr * er - ki * ei;
-            Si[j * RS + c] += kr * ei + ki * er;
+            const float4 lk = v_lk[j];
+            Sr[j * RS + c] = zr[r] + lk.z * er - lk.w * ei;
+            Si[j * RS + c] = zi[r] + lk.z * ei + lk.w * er;
         }
         __syncthreads();
     };
@@ -235,24 +236,23 @@ sfda_backward_kernel(const BwdArgsDev a)
             const float bt = scal[0];
             const size_t row = ((size_t)b * T_ + t) * H + h;
 
-            // step 1 (columns): G += q yb^*;  partial p = G^* k and k^* Z
+            // step 1 (columns): partial p = (G + q yb^*)^* k and k^* Z  (G itself is updated in step 3)
             {
-                const float yr = v_yr[c], yi = v_yi[c];
+                const float4 yu = v_yu[c];
+                const float yr = yu.x, yi = yu.y;
                 float pr = 0.f, pi = 0.f, zr_ = 0.f, zi_ = 0.f;
 #pragma unroll
                 for (int r = 0; r < RA; ++r) {
                     const int j = g + NG * r;
-                    const float qr = v_qr[j], qi = v_qi[j], kr = v_kr[j], ki = v_ki[j], lr = v_lr[j], li = v_li[j];
-                    const float gr = Gr[j * RS + c] + qr * yr + qi * yi;       // q conj(yb)
-                    const float gi = Gi[j * RS + c] + qi * yr - qr * yi;
-                    Gr[j * RS + c] = gr;
-                    Gi[j * RS + c] = gi;
-                    pr += gr * kr + gi * ki;                                    // conj(G) k
-                    pi += gr * ki - gi * kr;
+                    const float4 lk = v_lk[j], qc = v_qc[j];
+                    const float gr = Gr[j * RS + c] + qc.x * yr + qc.y * yi;   // G + q conj(yb)
+                    const float gi = Gi[j * RS + c] + qc.y * yr - qc.x * yi;
+                    pr += gr * lk.z + gi * lk.w;                                // conj(G) k
+                    pi += gr * lk.w - gi * lk.z;
                     const float sr = Qr[j * RS + c], si_ = Qi[j * RS + c];
-                    const float zr = lr * sr - li * si_, zi = lr * si_ + li * sr;
-                    zr_ += kr * zr + ki * zi;                                   // conj(k) z
-                    zi_ += kr * zi - ki * zr;
+                    const float zr = lk.x * sr - lk.y * si_, zi = lk.x * si_ + lk.y * sr;
+                    zr_ += lk.z * zr + lk.w * zi;                               // conj(k) z
+                    zi_ += lk.z * zi - lk.w * zr;
                 }
                 red[(g * 4 + 0) * DV + c] = pr;
                 red[(g * 4 + 1) * DV + c] = pi;
@@ -271,9 +271,11 @@ sfda_backward_kernel(const BwdArgsDev a)
                     zi += red[(gg * 4 + 3) * DV + c];
                 }
                 const float ur = v_v[c] - zr, ui = -zi;
-                v_pr[c] = pr; v_pi[c] = pi; v_ur[c] = ur; v_ui[c] = ui;
+                const float4 yu = v_yu[c];
+                const float yr = yu.x, yi = yu.y;
+                v_p[c] = make_float2(pr, pi);
+                v_yu[c] = make_float4(yr, yi, ur, ui);
                 st_val(dv, row * DV + c, bt * pr);
-                const float yr = v_yr[c], yi = v_yi[c];
                 float s0 = ur * pr - ui * pi;                       // Re(u p)
                 float s1 = ur * yr - ui * yi, s2 = ur * yi + ui * yr;   // u yb
 #pragma unroll
@@ -292,14 +294,19 @@ sfda_backward_kernel(const BwdArgsDev a)
                 for (int w = 0; w < DV / 32; ++w) { dbe += scal[8 + 4 * w]; sr_ += scal[9 + 4 * w]; si_ += scal[10 + 4 * w]; }
                 if (tid == 0) a.dbeta[row] = dbe;
                 const int j = jb;
-                const float lr = v_lr[j], li = v_li[j], kr = v_kr[j], ki = v_ki[j];
+                const float4 lk = v_lk[j], qc = v_qc[j];
+                const float lr = lk.x, li = lk.y, kr = lk.z, ki = lk.w;
                 float qzr = 0.f, qzi = 0.f, k1r = 0.f, k1i = 0.f, k2r = 0.f, k2i = 0.f, lbr = 0.f, lbi = 0.f;
 #pragma unroll 4
                 for (int n = 0; n < CPT; ++n) {
                     const int cc = part + TPR * n;
-                    const float gr = Gr[j * RS + cc], gi = Gi[j * RS + cc], sr = Qr[j * RS + cc], si2 = Qi[j * RS + cc];
+                    const float4 yu = v_yu[cc];
+                    const float2 pp = v_p[cc];
+                    const float yr = yu.x, yi = yu.y, ur = yu.z, ui = yu.w, pr = pp.x, pi = pp.y;
+                    const float gr = Gr[j * RS + cc] + qc.x * yr + qc.y * yi;  // G + q conj(yb)
+                    const float gi = Gi[j * RS + cc] + qc.y * yr - qc.x * yi;
+                    const float sr = Qr[j * RS + cc], si2 = Qi[j * RS + cc];
                     const float zr = lr * sr - li * si2, zi = lr * si2 + li * sr;
-                    const float yr = v_yr[cc], yi = v_yi[cc], ur = v_ur[cc], ui = v_ui[cc], pr = v_pr[cc], pi = v_pi[cc];
                     qzr += zr * yr - zi * yi;  qzi += zr * yi + zi * yr;       // Z yb
                     k1r += gr * ur + gi * ui;  k1i += gi * ur - gr * ui;       // G conj(u)
                     k2r += zr * pr - zi * pi;  k2i += zr * pi + zi * pr;       // Z p
@@ -321,7 +328,7 @@ sfda_backward_kernel(const BwdArgsDev a)
                     st_val(dq, row * DK + 2 * j + 1, qzi + bt * (kr * si_ + ki * sr_));
                     st_val(dk, row * DK + 2 * j, bt * (k1r - k2r));
                     st_val(dk, row * DK + 2 * j + 1, bt * (k1i - k2i));
-                    const float cs = v_cs[j], sn = v_sn[j];
+                    const float cs = qc.z, sn = qc.w;
                     a.dalpha[row * M + j] = lbr * cs + lbi * sn;                          // Re(conj(lamb) e^{i theta})
                     a.dtheta[row * M + j] = lbi * lr - lbr * li;                          // -Im(conj(lamb) lam)
                 }
