@@ -29,10 +29,10 @@ constexpr int kSeg = 64;     // tokens between checkpoints
 template <int DK, int DV>
 struct BwdSmem {
     static constexpr int M = DK / 2;
-    static constexpr int RS = DV + 8;            // row stride (floats): rows 8 banks apart, 16-byte aligned
+    static constexpr int RS = DV + 8;            // row stride in complex (float2) elements: rows 16 banks apart
     static constexpr int NG = kBwdThreads / DV;  // row groups of the column-owner mapping
-    static constexpr int plane = M * RS;
-    // G (re, im), two buffers of S_{t-1} (re, im) and the vectors of one token
+    static constexpr int plane = M * RS;         // floats in half a state buffer
+    // G and two buffers of S_{t-1} as interleaved complex [M][RS], and the vectors of one token
     static constexpr size_t bytes = (size_t)(6 * plane + 8 * M + 7 * DV + NG * 4 * DV + 64) * 4;
 };
 
@@ -48,7 +48,7 @@ struct BwdArgsDev {
     const float *alpha, *theta, *beta, *S0, *dS_T;
     void *dq, *dk, *dv;
     float *dalpha, *dtheta, *dbeta, *dS0;
-    float *check, *scratch;      // [BH][NS][2][M][DV], [BH][kSeg][2][M][DV]
+    float *check, *scratch;      // [BH][NS][M][DV][2], [BH][kSeg][M][DV][2] (interleaved complex)
     int T, H, NS;
 };
 
@@ -61,10 +61,9 @@ sfda_backward_kernel(const BwdArgsDev a)
     constexpr int TPR = kBwdThreads / M, CPT = DV / TPR;               // threads per row / columns per thread (row mapping)
     static_assert(M % NG == 0 && DV % TPR == 0 && M + DV + 1 <= kBwdThreads, "thread mappings");
     extern __shared__ __align__(16) float sm[];
-    float *Gr = sm, *Gi = Gr + L::plane;
-    float *P0 = Gi + L::plane;                              // two S_{t-1} buffers of [re | im] planes
-    auto Pr = [&](int i) { return P0 + i * 2 * L::plane; };
-    auto Pi = [&](int i) { return P0 + i * 2 * L::plane + L::plane; };
+    float2 *G = reinterpret_cast<float2 *>(sm);            // cotangent of the state, complex [M][RS]
+    float *P0 = sm + 2 * L::plane;                          // two buffers of the same shape for S / S_{t-1}
+    auto Pb = [&](int i) { return reinterpret_cast<float2 *>(P0 + i * 2 * L::plane); };
     // per-row vectors of the token, packed so that one (broadcast) load fetches all a step needs of a row:
     // (lam re, lam im, k re, k im), (q re, q im, cos theta, sin theta); per-column vectors likewise:
     // (yb re, yb im, u re, u im), (p re, p im), v
@@ -128,16 +127,16 @@ sfda_backward_kernel(const BwdArgsDev a)
         }
     };
 
-    // ---- one forward step on the state in (Sr, Si); the token's vectors are staged and synchronised
-    auto fwd_step = [&](float *Sr, float *Si) {
+    // ---- one forward step on the state S; the token's vectors are staged and synchronised
+    auto fwd_step = [&](float2 *S) {
         float cr = 0.f, ci = 0.f, zr[RA], zi[RA];
 #pragma unroll
         for (int r = 0; r < RA; ++r) {
             const int j = g + NG * r;
             const float4 lk = v_lk[j];
-            const float sr = Sr[j * RS + c], si = Si[j * RS + c];
-            zr[r] = lk.x * sr - lk.y * si;                                     // Z = Lambda S
-            zi[r] = lk.x * si + lk.y * sr;
+            const float2 sv = S[j * RS + c];
+            zr[r] = lk.x * sv.x - lk.y * sv.y;                                 // Z = Lambda S
+            zi[r] = lk.x * sv.y + lk.y * sv.x;
             cr += lk.z * zr[r] + lk.w * zi[r];                                 // conj(k) z
             ci += lk.z * zi[r] - lk.w * zr[r];
         }
@@ -156,53 +155,51 @@ sfda_backward_kernel(const BwdArgsDev a)
         for (int r = 0; r < RA; ++r) {
             const int j = g + NG * r;
             const float4 lk = v_lk[j];
-            Sr[j * RS + c] = zr[r] + lk.z * er - lk.w * ei;
-            Si[j * RS + c] = zi[r] + lk.z * ei + lk.w * er;
+            S[j * RS + c] = make_float2(zr[r] + lk.z * er - lk.w * ei, zi[r] + lk.z * ei + lk.w * er);
         }
         __syncthreads();
     };
 
-    // ---- state moves between shared and global memory: planes [re | im][M][DV], 16 bytes per access
-    auto store_state = [&](const float *Sr, const float *Si, float *dst) {
-        for (int idx = tid; idx < M * DV / 4; idx += kBwdThreads) {
-            const int j = idx / (DV / 4), c4 = idx % (DV / 4);
-            *reinterpret_cast<float4 *>(dst + (size_t)j * DV + 4 * c4) = *reinterpret_cast<const float4 *>(Sr + j * RS + 4 * c4);
-            *reinterpret_cast<float4 *>(dst + (size_t)(M + j) * DV + 4 * c4) = *reinterpret_cast<const float4 *>(Si + j * RS + 4 * c4);
+    // ---- state moves between shared and global memory (workspace format: interleaved complex [M][DV]), 16 bytes
+    // = two elements per access
+    auto store_state = [&](const float2 *S, float *dst) {
+        for (int idx = tid; idx < M * DV / 2; idx += kBwdThreads) {
+            const int j = idx / (DV / 2), c2 = idx % (DV / 2);
+            *reinterpret_cast<float4 *>(dst + ((size_t)j * DV + 2 * c2) * 2) = *reinterpret_cast<const float4 *>(S + j * RS + 2 * c2);
         }
     };
-    auto load_state_async = [&](float *Sr, float *Si, const float *src) {
-        for (int idx = tid; idx < M * DV / 4; idx += kBwdThreads) {
-            const int j = idx / (DV / 4), c4 = idx % (DV / 4);
-            cp_async16(Sr + j * RS + 4 * c4, src + (size_t)j * DV + 4 * c4);
-            cp_async16(Si + j * RS + 4 * c4, src + (size_t)(M + j) * DV + 4 * c4);
+    auto load_state_async = [&](float2 *S, const float *src) {
+        for (int idx = tid; idx < M * DV / 2; idx += kBwdThreads) {
+            const int j = idx / (DV / 2), c2 = idx % (DV / 2);
+            cp_async16(reinterpret_cast<float *>(S + j * RS + 2 * c2), src + ((size_t)j * DV + 2 * c2) * 2);
         }
         cp_async_commit();
     };
 
     // ---- sweep 1: forward, checkpoints at the start of every segment (nothing is needed beyond the last one)
-    float *Sr = Pr(0), *Si = Pi(0);
+    float2 *S = Pb(0);
     for (int idx = tid; idx < M * DV; idx += kBwdThreads) {
         const int j = idx / DV, cc = idx % DV;
-        Sr[j * RS + cc] = a.S0 ? a.S0[((size_t)bh * DK + 2 * j) * DV + cc] : 0.f;
-        Si[j * RS + cc] = a.S0 ? a.S0[((size_t)bh * DK + 2 * j + 1) * DV + cc] : 0.f;
+        S[j * RS + cc] = a.S0 ? make_float2(a.S0[((size_t)bh * DK + 2 * j) * DV + cc], a.S0[((size_t)bh * DK + 2 * j + 1) * DV + cc])
+                              : make_float2(0.f, 0.f);
     }
     const int t_last_check = (a.NS - 1) * kSeg;
     load_tok(0, false);
     __syncthreads();
     for (int t = 0; t < t_last_check; ++t) {
-        if (t % kSeg == 0) store_state(Sr, Si, check + (size_t)(t / kSeg) * 2 * M * DV);
+        if (t % kSeg == 0) store_state(S, check + (size_t)(t / kSeg) * 2 * M * DV);
         stage_tok(false);
         __syncthreads();
         load_tok(t + 1, false);
-        fwd_step(Sr, Si);
+        fwd_step(S);
     }
-    store_state(Sr, Si, check + (size_t)(a.NS - 1) * 2 * M * DV);
+    store_state(S, check + (size_t)(a.NS - 1) * 2 * M * DV);
 
     // ---- cotangent of the final state
     for (int idx = tid; idx < M * DV; idx += kBwdThreads) {
         const int j = idx / DV, cc = idx % DV;
-        Gr[j * RS + cc] = a.dS_T ? a.dS_T[((size_t)bh * DK + 2 * j) * DV + cc] : 0.f;
-        Gi[j * RS + cc] = a.dS_T ? a.dS_T[((size_t)bh * DK + 2 * j + 1) * DV + cc] : 0.f;
+        G[j * RS + cc] = a.dS_T ? make_float2(a.dS_T[((size_t)bh * DK + 2 * j) * DV + cc], a.dS_T[((size_t)bh * DK + 2 * j + 1) * DV + cc])
+                                : make_float2(0.f, 0.f);
     }
     __syncthreads();      // also: every thread's checkpoint stores precede the loads below (same CTA, after a barrier)
 
@@ -210,28 +207,28 @@ sfda_backward_kernel(const BwdArgsDev a)
     for (int si = a.NS - 1; si >= 0; --si) {
         const int t0 = si * kSeg, t1 = min(t0 + kSeg, T_);
         // ---- sweep 2: forward again from the checkpoint, S_{t-1} of every token to the scratch
-        load_state_async(Sr, Si, check + (size_t)si * 2 * M * DV);
+        load_state_async(S, check + (size_t)si * 2 * M * DV);
         load_tok(t0, false);
         cp_async_wait_all();
         __syncthreads();
         for (int t = t0; t < t1; ++t) {
-            store_state(Sr, Si, scratch + (size_t)(t - t0) * 2 * M * DV);
+            store_state(S, scratch + (size_t)(t - t0) * 2 * M * DV);
             stage_tok(false);
             __syncthreads();
             load_tok(t + 1 < t1 ? t + 1 : t1 - 1, t + 1 >= t1);     // after the last one: the first backward token
-            if (t + 1 < t1) fwd_step(Sr, Si);                        // the state after the last token is not needed
+            if (t + 1 < t1) fwd_step(S);                        // the state after the last token is not needed
         }
         __syncthreads();      // the scratch stores of this CTA are visible to its own later loads
 
         // ---- sweep 3: backward through the segment; S_{t-1} arrives one token ahead in the other buffer
         int buf = 0;
-        load_state_async(Pr(buf), Pi(buf), scratch + (size_t)(t1 - 1 - t0) * 2 * M * DV);
+        load_state_async(Pb(buf), scratch + (size_t)(t1 - 1 - t0) * 2 * M * DV);
         for (int t = t1 - 1; t >= t0; --t) {
             stage_tok(true);
             cp_async_wait_all();
             __syncthreads();
-            const float *Qr = Pr(buf), *Qi = Pi(buf);
-            if (t > t0) load_state_async(Pr(buf ^ 1), Pi(buf ^ 1), scratch + (size_t)(t - 1 - t0) * 2 * M * DV);
+            const float2 *Q = Pb(buf);
+            if (t > t0) load_state_async(Pb(buf ^ 1), scratch + (size_t)(t - 1 - t0) * 2 * M * DV);
             load_tok(t - 1 >= t0 ? t - 1 : t0 - 1, true);           // (a token of the next segment down is reloaded there)
             const float bt = scal[0];
             const size_t row = ((size_t)b * T_ + t) * H + h;
@@ -245,12 +242,13 @@ sfda_backward_kernel(const BwdArgsDev a)
                 for (int r = 0; r < RA; ++r) {
                     const int j = g + NG * r;
                     const float4 lk = v_lk[j], qc = v_qc[j];
-                    const float gr = Gr[j * RS + c] + qc.x * yr + qc.y * yi;   // G + q conj(yb)
-                    const float gi = Gi[j * RS + c] + qc.y * yr - qc.x * yi;
+                    const float2 gv = G[j * RS + c];
+                    const float gr = gv.x + qc.x * yr + qc.y * yi;              // G + q conj(yb)
+                    const float gi = gv.y + qc.y * yr - qc.x * yi;
                     pr += gr * lk.z + gi * lk.w;                                // conj(G) k
                     pi += gr * lk.w - gi * lk.z;
-                    const float sr = Qr[j * RS + c], si_ = Qi[j * RS + c];
-                    const float zr = lk.x * sr - lk.y * si_, zi = lk.x * si_ + lk.y * sr;
+                    const float2 sv = Q[j * RS + c];
+                    const float zr = lk.x * sv.x - lk.y * sv.y, zi = lk.x * sv.y + lk.y * sv.x;
                     zr_ += lk.z * zr + lk.w * zi;                               // conj(k) z
                     zi_ += lk.z * zi - lk.w * zr;
                 }
@@ -303,9 +301,10 @@ sfda_backward_kernel(const BwdArgsDev a)
                     const float4 yu = v_yu[cc];
                     const float2 pp = v_p[cc];
                     const float yr = yu.x, yi = yu.y, ur = yu.z, ui = yu.w, pr = pp.x, pi = pp.y;
-                    const float gr = Gr[j * RS + cc] + qc.x * yr + qc.y * yi;  // G + q conj(yb)
-                    const float gi = Gi[j * RS + cc] + qc.y * yr - qc.x * yi;
-                    const float sr = Qr[j * RS + cc], si2 = Qi[j * RS + cc];
+                    const float2 gv = G[j * RS + cc], sv = Q[j * RS + cc];
+                    const float gr = gv.x + qc.x * yr + qc.y * yi;             // G + q conj(yb)
+                    const float gi = gv.y + qc.y * yr - qc.x * yi;
+                    const float sr = sv.x, si2 = sv.y;
                     const float zr = lr * sr - li * si2, zi = lr * si2 + li * sr;
                     qzr += zr * yr - zi * yi;  qzi += zr * yi + zi * yr;       // Z yb
                     k1r += gr * ur + gi * ui;  k1i += gi * ur - gr * ui;       // G conj(u)
@@ -313,8 +312,7 @@ sfda_backward_kernel(const BwdArgsDev a)
                     // Zb = G - beta k conj(p)
                     const float br = gr - bt * (kr * pr + ki * pi), bi = gi - bt * (ki * pr - kr * pi);
                     lbr += sr * br + si2 * bi;  lbi += sr * bi - si2 * br;     // conj(S_{t-1}) Zb
-                    Gr[j * RS + cc] = lr * br + li * bi;                       // conj(lam) Zb
-                    Gi[j * RS + cc] = lr * bi - li * br;
+                    G[j * RS + cc] = make_float2(lr * br + li * bi, lr * bi - li * br);   // conj(lam) Zb
                 }
 #pragma unroll
                 for (int d = TPR / 2; d >= 1; d >>= 1) {
@@ -336,12 +334,12 @@ sfda_backward_kernel(const BwdArgsDev a)
             __syncthreads();
             buf ^= 1;
         }
-        Sr = Pr(0); Si = Pi(0);
+        S = Pb(0);
     }
     for (int idx = tid; idx < M * DV; idx += kBwdThreads) {
         const int j = idx / DV, cc = idx % DV;
-        a.dS0[((size_t)bh * DK + 2 * j) * DV + cc] = Gr[j * RS + cc];
-        a.dS0[((size_t)bh * DK + 2 * j + 1) * DV + cc] = Gi[j * RS + cc];
+        a.dS0[((size_t)bh * DK + 2 * j) * DV + cc] = G[j * RS + cc].x;
+        a.dS0[((size_t)bh * DK + 2 * j + 1) * DV + cc] = G[j * RS + cc].y;
     }
 }
 
