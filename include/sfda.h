@@ -124,17 +124,19 @@ SFDA_API int sfda_forward(const void *q, const void *k, const void *v,
  * sfda_forward for few, long sequences: a two-level scan over the time axis.  A sequence is one serial chain of
  * chunks, so with fewer (batch, head) pairs than SMs most of the GPU idles.  By Theorem "Exact affine chunk
  * transfer" a time slice maps its initial state affinely, S_out = P S_in + B; so every sequence is cut into
- * n_slices slices that run as independent sequences: once from a zero state (B), once with v = 0 from [I | 0] (P),
- * then a small scan S_{i+1} = P_i S_i + B_i gives every slice its true initial state and a last pass the outputs.
- * Three passes over the data, each n_slices times as parallel; exact up to the forward's own rounding.
+ * n_slices slices that run as independent sequences: once from a zero state (B and the outputs o^(0)), once with
+ * v = 0 from [I | 0] (P, and g_t = P_t^* q_t in the first d_k / 2 channels of its outputs); a small scan
+ * S_{i+1} = P_i S_i + B_i gives every slice its true initial state S_in, and o_t = o_t^(0) + S_in^* g_t is added in
+ * place by a tensor-core product.  Two chain passes, each n_slices times as parallel, and a memory-bound epilogue;
+ * exact algebra, with P, B, g and S_in carrying the forward's bf16 rounding once more.
  *
  * Arguments, layouts and results as sfda_forward.  n_slices >= 2 must divide T into multiples of chunk;
  * n_slices = 0 lets the library choose (the largest power of two with B H n_slices <= the device's SM count and at
- * least 16 chunks per slice; below 4 slices the three passes cannot pay and the call is sfda_forward).  Only the shapes of the tensor-core path
+ * least 16 chunks per slice; below 4 slices the call is sfda_forward).  Only the shapes of the tensor-core path
  * (bf16, d_k = d_v = 128, chunk = 64) -> SFDA_ERR_UNSUPPORTED otherwise, also for an n_slices that does not divide.
  * workspace: sfda_forward_two_level_workspace_bytes(...) bytes (the forward's own scratch, five sets of
- * B n_slices H states, a zero v and an unread output of the size of v); all of it is required.
- * sfda_workspace_status on this workspace reports the last of the three passes.
+ * B n_slices H states, a zero v and the two outputs of the second pass, each of the size of v); all of it is
+ * required.  sfda_workspace_status on this workspace reports the last of the two chain passes.
  */
 SFDA_API size_t sfda_forward_two_level_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int dtype,
                                                        int n_slices);

@@ -151,7 +151,7 @@ def test_two_level_entry_point_validates_on_the_host(lib):
     need = sfda.sfda_forward_two_level_workspace_bytes(1, 2048, 2, 128, 128, 64, 1, 2)
     r256 = lambda x: (x + 255) // 256 * 256
     states, tokens = 1 * 2 * 2 * 128 * 128 * 4, 1 * 2048 * 2 * 128 * 2
-    assert need == r256(sfda.sfda_workspace_bytes(2, 1024, 2, 128, 128, 64, 1)) + 5 * r256(states) + 2 * r256(tokens)
+    assert need == r256(sfda.sfda_workspace_bytes(2, 1024, 2, 128, 128, 64, 1)) + 5 * r256(states) + 3 * r256(tokens)
     assert two(ptrs, dims, 2, ws_bytes=need - 1) == -5
     assert sfda.sfda_forward_two_level_workspace_bytes(1, 2048, 2, 128, 128, 64, 1, 3) == 0
     assert sfda.sfda_forward_two_level_workspace_bytes(1, 2048, 2, 64, 64, 16, 0, 2) == 0
