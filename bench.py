@@ -282,6 +282,37 @@ def main():
     value = dp.whole_job_throughput(cfg.B * cfg.T, world, ms_per_step * 1e-3)
     assert sfda.sfda_workspace_status(ws, stream) == 0      # no bounded device-side wait ran out
 
+    # The other output mode beside the quoted one (Re + Im is the paper-literal o; Re only is what a real readout
+    # uses).  By now the GPU has run for a second and sits at its power-capped clock, so both modes are timed again,
+    # back to back, under the same conditions.
+    other_mode = None
+    if rank == 0:
+        alt_im = None if want_im else torch.empty_like(o)
+
+        def timed_mode(im):
+            for _ in range(3):
+                sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, im, S_T,
+                                  cfg.chunk, ws, stream)
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a0.record(stream)
+            for _ in range(max(args.steps, 10)):
+                sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, im, S_T,
+                                  cfg.chunk, ws, stream)
+            a1.record(stream)
+            torch.cuda.synchronize()
+            return a0.elapsed_time(a1) / max(args.steps, 10)
+
+        quoted_ms = timed_mode(o_im)
+        alt_ms = timed_mode(alt_im)
+        alt_bytes = algorithmic_bytes(cfg, not want_im)
+        other_mode = {"outputs": "Re" if want_im else "Re+Im", "ms_per_step": alt_ms,
+                      "tokens_per_s": cfg.B * cfg.T / (alt_ms * 1e-3), "algorithmic_bytes": alt_bytes,
+                      "achieved_gbs": alt_bytes / (alt_ms * 1e-3) / 1e9,
+                      "quoted_mode_ms_per_step_same_conditions": quoted_ms,
+                      "note": "both modes timed back to back after about a second of load (power-capped clock)"}
+        del alt_im
+
     # end to end through the host-buffer entry point: H2D of the inputs and D2H of the results inside the timing
     e2e = None
     if args.e2e_steps > 0:
@@ -539,6 +570,8 @@ def main():
         roofline["traffic"] = 1.939e9 * cfg.B / 4
         roofline["traffic_source"] = "ncu capture at B=4 scaled to B=%d; Re+Im outputs" % cfg.B
 
+    if other_mode is not None:
+        other_mode["frac"] = other_mode["achieved_gbs"] / peaks["hbm_gbs"]
     if bwd is not None:
         bwd["frac"] = bwd["achieved_gbs"] / peaks["hbm_gbs"]
         bwd["peak_source"] = "of " + peaks["source"]
@@ -567,7 +600,7 @@ def main():
                    "chunk": cfg.chunk, "outputs": "Re+Im" if want_im else "Re", "state": "fp32", "S0": "N(0,0.02)",
                    "parallelism": "dp%d over (batch, head), no collective" % world,
                    "l2": "inputs+outputs %.2f GB per step, far larger than the 126 MB L2; no flush" % (abytes / 1e9)},
-        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "decode": decode, "fused_front_end": fused, "chunk_factors": factors, "backward": bwd, "long_context": longctx,
+        "roofline": roofline, "cpu_baseline": cpu, "other_output_mode": other_mode, "e2e": e2e, "decode": decode, "fused_front_end": fused, "chunk_factors": factors, "backward": bwd, "long_context": longctx,
         "gpu_launches": launches_per_step * args.steps, "clocks": clocks.summary(),
     }
     print(json.dumps(line), flush=True)
