@@ -559,7 +559,8 @@ def main():
     roofline = {
         "bound": "hbm", "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
         "frac": achieved_gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": "of " + peaks["source"],
-        "kernel": "sfda_forward chunk kernel (1 launch per step)", "kernel_ms": k_ms,
+        "kernel": "sfda_forward chunk kernel (1 launch per step)", "kernel_ms": k_ms, "kernel_ms_median": float(statistics.median(kernel_ms)),
+        "kernel_ms_best": float(min(kernel_ms)),
         "algorithmic_bytes": abytes, "algorithmic_flops": aflops, "achieved_tflops": achieved_tf,
         "tensor_frac": achieved_tf / peaks["bf16_tflops"],
         "roofline_ms": 1e3 * max(hbm_time, tensor_time),
