@@ -225,9 +225,6 @@ __device__ __forceinline__ void role_sync(int id, int nthreads)
     asm volatile("barrier.cta.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
-// Waits are bounded in ticks of the SM's own clock counter, which is cheap to read.
-__device__ __forceinline__ unsigned long long now_ticks() { return (unsigned long long)clock64(); }
-constexpr unsigned long long kWaitLimitTicks = 4000000000ull;   // about 2 s at the maximum SM clock
 #ifdef SFDA_WS_TIMING
 __device__ __forceinline__ unsigned long long now_ns()
 {
@@ -237,16 +234,6 @@ __device__ __forceinline__ unsigned long long now_ns()
 }
 #endif
 
-// Non-blocking test of completion number k (0-based) of a barrier.
-__device__ __forceinline__ bool test_k(Misc &mi, int bar, int k)
-{
-    uint32_t ok;
-    asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
-                 : "=r"(ok)
-                 : "r"(smem_u32(&mi.bars[bar])), "r"((uint32_t)k & 1u)
-                 : "memory");
-    return ok != 0;
-}
 // Wait for completion number k of a barrier; gives up after about a second (2^31 ticks of the SM clock) and
 // raises the abort flag.  try_wait parks the thread in hardware for up to the hinted time, so waiting warps do
 // not compete with working ones for issue slots.  Kept to a handful of instructions: it is inlined at every
@@ -282,10 +269,6 @@ __device__ __forceinline__ bool elect_one()
 __device__ __forceinline__ bool wait_k_warp(Misc &mi, int bar, int k)
 {
     return __all_sync(0xffffffffu, wait_k(mi, bar, k) ? 1 : 0) != 0;
-}
-__device__ __forceinline__ bool test_k_warp(Misc &mi, int bar, int k)
-{
-    return __all_sync(0xffffffffu, test_k(mi, bar, k) ? 1 : 0) != 0;
 }
 
 // One complex product as four real ones (g = 0..3), each of four K = 16 instructions:
@@ -356,11 +339,11 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
                                          const Params &p, int n_chunks)
 {
     const CUtensorMap *tm_v = &maps.v, *tm_o = &maps.o, *tm_oim = &maps.oim;
-    long long *timing = p.timing;
+    [[maybe_unused]] long long *timing = p.timing;
     const uint64_t dbase = smem_desc(smem_u32(smem));                     // descriptor of byte offset 0
     const uint32_t dlo = (uint32_t)dbase, dhi = (uint32_t)(dbase >> 32);
     unsigned long long *bars = mi.bars;
-    constexpr uint32_t I64 = idesc(64, 0), I128 = idesc(128, 0), I64M = idesc(64, 0) | (1u << 16);   // M: B MN-major
+    constexpr uint32_t I64 = idesc(64, 0), I64M = idesc(64, 0) | (1u << 16);   // M: B MN-major
     constexpr uint32_t kIm = kTile >> 4;                                  // re -> im tile, in descriptor units
     const uint32_t x_re = tmem + TM_X16, acc = tmem + TM_ACC;
     const uint32_t m_re = dlo + (OFF_MB >> 4);
@@ -545,7 +528,7 @@ __device__ __forceinline__ float theta_from_raw(const Params &p, uint32_t bits)
 template <bool kFused>
 __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int n_chunks, int pt)
 {
-    long long *timing = p.timing;
+    [[maybe_unused]] long long *timing = p.timing;
     const int jp = pt & 31, tq = pt >> 5;   // channel pair (channels 2jp, 2jp+1), token octet (8 tokens)
     bool dead = false;
     // this role also reads the finished outputs out of tensor memory (its warps cover the four lane quadrants
@@ -825,7 +808,7 @@ __device__ __forceinline__ void store_tile_s(const float (&cr)[4], const float (
 template <bool kFused>
 __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int n_chunks, int st)
 {
-    long long *timing = p.timing;
+    [[maybe_unused]] long long *timing = p.timing;
     const int lane = st & 31, w = st >> 5;    // w = TMEM lane quadrant of this warp
     constexpr uint32_t kIm = 64 * LS * 4;     // Re -> Im in the scratch
     const uint32_t sbase = smem_u32(smem), lx = sbase + OFF_LX;
@@ -1029,7 +1012,7 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
 template <bool kFused>
 __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int n_chunks, int ct)
 {
-    long long *timing = p.timing;
+    [[maybe_unused]] long long *timing = p.timing;
     const int lane = ct & 31, warp = ct >> 5;
     const int quad = warp & 3, half = warp >> 2;
     const int c = quad * 32 + lane;            // value channel = TMEM lane
