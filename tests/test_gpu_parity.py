@@ -800,3 +800,40 @@ def test_forward_two_level_long_context_sampled():
     assert rel_err(np.stack([o[b, :, h] for b, h in pairs]), w_re) <= TOL["bf16"]
     assert rel_err(np.stack([o_im[b, :, h] for b, h in pairs]), w_im) <= TOL["bf16"]
     assert rel_err(np.stack([S_T[b, h] for b, h in pairs]), w_S) <= TOL["bf16"]
+
+
+def test_chunk_factors_full_size_headline_sampled():
+    """The factor export at the headline sizes, in the launch configuration bench.py times; the oracle recomputes
+    sampled chunks (first, middle, last of sampled sequences), and the phase turns are compared on whole sequences."""
+    cfg = workloads.CONFIGS[2]
+    inp = workloads.forward_inputs(cfg)
+    B, H, m, C, T = cfg.B, cfg.H, cfg.m, cfg.chunk, cfg.T
+    NC = T // C
+    G = torch.empty(B, H, NC, m, 2, device=DEV)
+    Y = torch.empty(B, H, NC, m, C, 2, device=DEV)
+    W = torch.empty_like(Y)
+    M = torch.empty(B, H, NC, C, C, 2, device=DEV)
+    turns = torch.empty(B, T, H, m, device=DEV, dtype=torch.int32)
+    sfda.sfda_chunk_factors(to_dev(inp["k"], cfg, "k"), to_dev(inp["alpha"], cfg, "alpha"),
+                            to_dev(inp["theta"], cfg, "theta"), to_dev(inp["beta"], cfg, "beta"), G, Y, M, W, turns, C)
+    torch.cuda.synchronize()
+    assert sfda.last_launch_count() == 1
+    cx = lambda t: t.cpu().numpy().astype(np.float64)[..., 0] + 1j * t.cpu().numpy().astype(np.float64)[..., 1]
+    worst = 0.0
+    for b, h in [(0, 0), (B - 1, H - 1), (3, 17)]:
+        kc = chunk_wy.pair(inp["k"][b, :, h])
+        for c in (0, NC // 2, NC - 1):
+            sl = slice(c * C, (c + 1) * C)
+            g, y, w, mm = chunk_wy.chunk_factors(kc[sl], inp["alpha"][b, sl, h].astype(np.float64),
+                                                 inp["theta"][b, sl, h].astype(np.float64),
+                                                 inp["beta"][b, sl, h].astype(np.float64))
+            Gc, Yc, Wc, Mc = cx(G[b, h, c]), cx(Y[b, h, c]), cx(W[b, h, c]), cx(M[b, h, c])
+            worst = max(worst, rel_err(Gc.view(np.float64), g.view(np.float64)),
+                        rel_err(Yc.copy().view(np.float64), y.copy().view(np.float64)),
+                        rel_err(Wc.copy().view(np.float64), w.copy().view(np.float64)),
+                        rel_err(Mc.copy().view(np.float64), mm.copy().view(np.float64)))
+            assert np.abs((np.diag(Gc) - Yc @ Mc @ Wc.conj().T) - (np.diag(g) - y @ mm @ w.conj().T)).max() < 2e-5
+        got = turns[b, :, h].cpu().numpy().view(np.uint32)
+        want = bookkeeping.cumulative_phase_turns(inp["theta"][b, :, h], C)
+        assert np.array_equal(got, want)
+    assert worst < 1e-4, worst
