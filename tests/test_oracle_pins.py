@@ -667,3 +667,64 @@ def test_time_slice_transfer_from_the_identity_state_and_the_zero_state():
         Bc = Bp[:, 0::2] + 1j * Bp[:, 1::2]
         S = np.einsum("njl,nlc->njc", P, S) + Bc
     assert np.allclose(S.real, S_T[:, 0::2], atol=1e-11) and np.allclose(S.imag, S_T[:, 1::2], atol=1e-11)
+
+
+# ----------------------------------------------------------------------------
+# write-decoupled variant (Eq. "sfda-decoupled-main")
+# ----------------------------------------------------------------------------
+def _decoupled_inputs(seed, N=2, T=12, m=3, dv=4):
+    rng = np.random.default_rng(seed)
+    return dict(q=rng.standard_normal((N, T, 2 * m)), k=0.6 * rng.standard_normal((N, T, 2 * m)),
+                r=0.6 * rng.standard_normal((N, T, 2 * m)), v=rng.standard_normal((N, T, dv)),
+                alpha=rng.uniform(0.5, 1.0, (N, T, m)), theta=rng.uniform(-np.pi, np.pi, (N, T, m)),
+                eta=rng.uniform(0.1, 0.9, (N, T)), beta=rng.uniform(0.1, 0.9, (N, T)),
+                S0=rng.standard_normal((N, 2 * m, dv)))
+
+
+def test_decoupled_variant_reduces_to_the_tied_model():
+    """r = k and eta = beta is Eq. "sfda" (checked against the C oracle); r = k with eta != beta is Eq. "sfda" with
+    beta := eta and v := (beta / eta) v."""
+    from oracle import variants
+    x = _decoupled_inputs(31)
+    a = variants.sfda_decoupled_recurrence(x["q"], x["k"], x["k"], x["v"], x["alpha"], x["theta"], x["beta"], x["beta"], x["S0"])
+    b = recurrence.sfda_recurrence(x["q"], x["k"], x["v"], x["alpha"], x["theta"], x["beta"], x["S0"])
+    for u, w in zip(a, b):
+        assert np.allclose(u, w, rtol=1e-12, atol=1e-12)
+    a = variants.sfda_decoupled_recurrence(x["q"], x["k"], x["k"], x["v"], x["alpha"], x["theta"], x["eta"], x["beta"], x["S0"])
+    b = recurrence.sfda_recurrence(x["q"], x["k"], x["v"] * (x["beta"] / x["eta"])[..., None], x["alpha"], x["theta"],
+                                   x["eta"], x["S0"])
+    for u, w in zip(a, b):
+        assert np.allclose(u, w, rtol=1e-12, atol=1e-12)
+
+
+def test_decoupled_variant_against_explicit_matrices_and_limits():
+    """Dense brute force S_t = A_t S_{t-1} + B_t with explicit m x m matrices; eta = 0 leaves a decayed sum of the
+    writes, S_T = Gamma_T S_0 + sum_t (Gamma_T / Gamma_t) beta_t r_t v_t^T; beta = 0 never increases the Frobenius
+    norm when eta |k|^2 <= 1 (the erase factor is a contraction, Prop. "Basic numerical stability")."""
+    from oracle import variants
+    x = _decoupled_inputs(32, N=1, T=7)
+    o_re, o_im, S_T = variants.sfda_decoupled_recurrence(**x)
+    m = 3
+    kc, rc, qc = (x[n][0, :, 0::2] + 1j * x[n][0, :, 1::2] for n in ("k", "r", "q"))
+    lam = x["alpha"][0] * np.exp(1j * x["theta"][0])
+    S = x["S0"][0, 0::2] + 1j * x["S0"][0, 1::2]
+    for t in range(7):
+        A = (np.eye(m) - x["eta"][0, t] * np.outer(kc[t], kc[t].conj())) @ np.diag(lam[t])
+        S = A @ S + x["beta"][0, t] * np.outer(rc[t], x["v"][0, t])
+        assert np.allclose(S.conj().T @ qc[t], o_re[0, t] + 1j * o_im[0, t], atol=1e-12)
+    assert np.allclose(S, S_T[0, 0::2] + 1j * S_T[0, 1::2], atol=1e-12)
+    # eta = 0
+    y = dict(x, eta=np.zeros_like(x["eta"]))
+    _, _, S_T0 = variants.sfda_decoupled_recurrence(**y)
+    gam = np.cumprod(lam, axis=0)
+    want = gam[-1][:, None] * (x["S0"][0, 0::2] + 1j * x["S0"][0, 1::2]) + sum(
+        (gam[-1] / gam[t])[:, None] * x["beta"][0, t] * np.outer(rc[t], x["v"][0, t]) for t in range(7))
+    assert np.allclose(S_T0[0, 0::2] + 1j * S_T0[0, 1::2], want, atol=1e-12)
+    # beta = 0, eta |k|^2 <= 1
+    z = dict(x, beta=np.zeros_like(x["beta"]))
+    z["k"] = z["k"] / np.linalg.norm(z["k"], axis=-1, keepdims=True)
+    norms = [np.linalg.norm(x["S0"][0])]
+    for T_ in range(1, 8):
+        _, _, S_p = variants.sfda_decoupled_recurrence(**{n: (v if n == "S0" else v[:, :T_]) for n, v in z.items()})
+        norms.append(np.linalg.norm(S_p[0]))
+    assert all(b <= a + 1e-12 for a, b in zip(norms[:-1], norms[1:]))
