@@ -539,7 +539,26 @@ def main():
         d1.record(stream)
         torch.cuda.synchronize()
         fused_step_ms = d0.elapsed_time(d1) / nd
-        decode = {"workload": dcfg.name, "ms_per_step": step_ms, "fused_raw_inputs_ms_per_step": fused_step_ms, "tokens_per_s": dcfg.B / (step_ms * 1e-3),
+        # and one step of the write-decoupled variant (separate write direction r and erase strength eta)
+        gd = torch.Generator(device=dev)
+        gd.manual_seed(4321)
+        r_dec = (0.1 * torch.randn(dcfg.B, dcfg.H, dcfg.d_k, device=dev, generator=gd)).to(torch.bfloat16)
+        eta_dec = torch.rand(dcfg.B, dcfg.H, device=dev, generator=gd)
+        x0 = ring[0]
+        for _ in range(8):
+            sfda.sfda_step_decoupled(x0["q"], x0["k"], r_dec, x0["v"], x0["alpha"], x0["theta"], eta_dec, x0["beta"], S,
+                                     od, od_im, stream)
+        torch.cuda.synchronize()
+        d0.record(stream)
+        for i in range(nd):
+            x = ring[i % len(ring)]
+            sfda.sfda_step_decoupled(x["q"], x["k"], r_dec, x["v"], x["alpha"], x["theta"], eta_dec, x["beta"], S, od,
+                                     od_im, stream)
+        d1.record(stream)
+        torch.cuda.synchronize()
+        dec_step_ms = d0.elapsed_time(d1) / nd
+        decode = {"workload": dcfg.name, "ms_per_step": step_ms, "fused_raw_inputs_ms_per_step": fused_step_ms,
+                  "write_decoupled_ms_per_step": dec_step_ms, "tokens_per_s": dcfg.B / (step_ms * 1e-3),
                   "algorithmic_bytes_per_step": dbytes, "achieved_gbs": dbytes / (step_ms * 1e-3) / 1e9,
                   "state_bytes": int(S.numel() * 4), "note": "state (537 MB) far larger than L2"}
 

@@ -249,6 +249,21 @@ SFDA_API int sfda_step_fused(const void *q, const void *k_raw, const void *v,
                              int B, int H, int d_k, int d_v, int dtype, void *stream);
 
 /*
+ * One decode step of the write-decoupled variant (Section 3, paragraph "Write-decoupled variant",
+ * Eq. "sfda-decoupled-main"):
+ *
+ *     S <- (I - eta k k^*) Lambda S + beta r v^*,        o = S^* q,
+ *
+ * erase direction and strength (k, eta) separate from write direction and strength (r, beta); r = k, eta = beta is
+ * sfda_step.  Arguments as sfda_step plus r [B][H][d_k] dtype and eta [B][H] float.  (The chunk kernels of this
+ * library compute the tied model only: the variant needs a second operand tile per chunk.)
+ */
+SFDA_API int sfda_step_decoupled(const void *q, const void *k, const void *r, const void *v,
+                                 const float *alpha, const float *theta, const float *eta, const float *beta,
+                                 float *S, void *o, void *o_im,
+                                 int B, int H, int d_k, int d_v, int dtype, void *stream);
+
+/*
  * Host-buffer forward: the call a user with data in host memory makes.  Copies the
  * inputs from HOST memory (pinned for asynchronous copies) into `arena`, runs
  * sfda_forward there and copies o (and o_im, S_T when not NULL) back to HOST

@@ -60,6 +60,7 @@ def load():
     lib.sfda_forward_two_level_workspace_bytes.restype = _sz
     lib.sfda_forward_two_level_workspace_bytes.argtypes = [_ci] * 8
     lib.sfda_forward_two_level.argtypes = [_vp] * 10 + [_ci] * 8 + [_vp, _sz, _vp]
+    lib.sfda_step_decoupled.argtypes = [_vp] * 11 + [_ci] * 5 + [_vp]
     _LIB = lib
     return lib
 
@@ -323,3 +324,18 @@ def sfda_forward_two_level(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chunk,
                                        int(n_slices), _ptr(workspace), ws_bytes, _stream(stream))
     if rc != 0:
         raise SfdaError(rc, "sfda_forward_two_level")
+
+
+def sfda_step_decoupled(q, k, r, v, alpha, theta, eta, beta, S, o, o_im, stream=None):
+    """``sfda_step_decoupled`` of ``include/sfda.h``: one decode step of the write-decoupled variant."""
+    B, H, d_k = q.shape
+    d_v = v.shape[-1]
+    for t, n in ((q, "q"), (k, "k"), (r, "r"), (v, "v"), (o, "o"), (o_im, "o_im")):
+        _check(t, n, q.dtype)
+    for t, n in ((alpha, "alpha"), (theta, "theta"), (eta, "eta"), (beta, "beta"), (S, "S")):
+        _check(t, n, torch.float32)
+    rc = load().sfda_step_decoupled(_ptr(q), _ptr(k), _ptr(r), _ptr(v), _ptr(alpha), _ptr(theta), _ptr(eta),
+                                    _ptr(beta), _ptr(S), _ptr(o), _ptr(o_im), B, H, d_k, d_v, _dtype_code(q),
+                                    _stream(stream))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_step_decoupled")

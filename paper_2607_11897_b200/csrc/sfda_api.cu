@@ -311,6 +311,19 @@ int sfda_step(const void *q, const void *k, const void *v, const float *alpha, c
     return step_common(q, k, v, alpha, theta, beta, S, o, o_im, B, H, d_k, d_v, dtype, sfda::StepParam(), stream);
 }
 
+int sfda_step_decoupled(const void *q, const void *k, const void *r, const void *v, const float *alpha,
+                        const float *theta, const float *eta, const float *beta, float *S, void *o, void *o_im, int B,
+                        int H, int d_k, int d_v, int dtype, void *stream)
+{
+    g_last_launches = 0;
+    if (!r || !eta) return SFDA_ERR_NULL;
+    if (!aligned16(r) || !aligned16(eta)) return SFDA_ERR_ALIGN;
+    sfda::StepParam par;
+    par.r = r;
+    par.eta = eta;
+    return step_common(q, k, v, alpha, theta, beta, S, o, o_im, B, H, d_k, d_v, dtype, par, stream);
+}
+
 int sfda_step_fused(const void *q, const void *k_raw, const void *v, const float *a_raw, const float *b_raw,
                     const float *c_raw, float alpha_min, float alpha_max, float theta_max, float eps, float *S,
                     void *o, void *o_im, int B, int H, int d_k, int d_v, int dtype, void *stream)

@@ -30,6 +30,9 @@ struct FactorArgs {
 struct StepParam {
     int fused = 0;
     float a_lo = 0.f, a_range = 1.f, th_max = 0.f, eps = 0.f;
+    // write-decoupled variant (r != nullptr): write direction r [B][H][d_k] in the dtype of q, erase strength eta [B][H]
+    const void *r = nullptr;
+    const float *eta = nullptr;
 };
 
 struct StepArgs {

@@ -26,13 +26,16 @@ __device__ __forceinline__ float4 ld_state(const float *p)
     return v;
 }
 
-template <int DK, int DV, typename T, bool kFused>
+// kMode: 0 the tied recurrence; 1 the same on raw inputs of the stable parameterisation; 2 the write-decoupled
+// variant S_t = (I - eta k k^*) Lambda S_{t-1} + beta r v^* (Section 3, Eq. "sfda-decoupled-main").
+template <int DK, int DV, typename T, int kMode>
 __global__ void __launch_bounds__(kStepThreads)
 sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v,
                  const float *__restrict__ alpha, const float *__restrict__ theta,
                  const float *__restrict__ beta, float *__restrict__ S, T *__restrict__ o,
                  T *__restrict__ o_im, const StepParam par)
 {
+    constexpr bool kFused = kMode == 1, kDec = kMode == 2;
     constexpr int M = DK / 2;              // complex rows
     constexpr int CT = DV < kColTile ? DV : kColTile;   // columns of this CTA
     constexpr int CG = CT / 4;             // threads across one row (float4 each)
@@ -44,6 +47,7 @@ sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__re
     __shared__ float s_v[CT];
     __shared__ float s_red[RG][2][CT];
     __shared__ float s_norm[kStepThreads / 32];
+    __shared__ float s_rr[kDec ? M : 1], s_ri[kDec ? M : 1];      // write direction r of the decoupled variant
 
     const int tid = threadIdx.x;
     const size_t bh = blockIdx.x;
@@ -66,7 +70,12 @@ sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__re
     // beside the 128 KB of state traffic.
     // Every global load of the preamble is issued before anything waits for one of them.
     static_assert(M <= kStepThreads && CT <= kStepThreads, "one coordinate and one column per thread at most");
-    float a = 1.f, th = 0.f, kr0 = 0.f, ki0 = 0.f, qr0 = 0.f, qi0 = 0.f, v0 = 0.f;
+    float a = 1.f, th = 0.f, kr0 = 0.f, ki0 = 0.f, qr0 = 0.f, qi0 = 0.f, v0 = 0.f, rr0 = 0.f, ri0 = 0.f;
+    const float eta = kDec ? par.eta[bh] : 0.f;
+    if (kDec && tid < M) {
+        rr0 = ld_val(static_cast<const T *>(par.r), bh * DK + 2 * tid);
+        ri0 = ld_val(static_cast<const T *>(par.r), bh * DK + 2 * tid + 1);
+    }
     if (tid < M) {
         a = alpha[bh * M + tid];
         th = theta[bh * M + tid];
@@ -94,6 +103,10 @@ sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__re
         s_ki[tid] = ki0;
         s_qr[tid] = qr0;
         s_qi[tid] = qi0;
+        if (kDec) {
+            s_rr[tid] = rr0;
+            s_ri[tid] = ri0;
+        }
     }
     if (tid < CT) s_v[tid] = v0;
     constexpr int kKeyWarps = (M + 31) / 32;       // the warps whose threads read key coordinates above
@@ -149,7 +162,10 @@ sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__re
             a += s_red[g][0][4 * cg + x];
             b += s_red[g][1][4 * cg + x];
         }
-        if (kFused) {                          // c = s c_raw; e -> s e for the raw-key update
+        if (kDec) {                            // erase part -eta c along k; the write beta v goes along r below
+            ere[x] = -eta * a;
+            eim[x] = -eta * b;
+        } else if (kFused) {                   // c = s c_raw; e -> s e for the raw-key update
             ere[x] = sk * bt * (s_v[4 * cg + x] - sk * a);
             eim[x] = -sk * bt * sk * b;
         } else {
@@ -165,12 +181,17 @@ sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__re
     for (int r = 0; r < R; ++r) {
         const int j = rg * R + r;
         const float kr = s_kr[j], ki = s_ki[j], qr = s_qr[j], qi = s_qi[j];
+        const float wr = kDec ? bt * s_rr[j] : 0.f, wi = kDec ? bt * s_ri[j] : 0.f;     // beta r
         float *pr = reinterpret_cast<float *>(&sre[r]);
         float *pi = reinterpret_cast<float *>(&sim[r]);
 #pragma unroll
         for (int x = 0; x < 4; ++x) {
-            const float nr = pr[x] + kr * ere[x] - ki * eim[x];
-            const float ni = pi[x] + kr * eim[x] + ki * ere[x];
+            float nr = pr[x] + kr * ere[x] - ki * eim[x];
+            float ni = pi[x] + kr * eim[x] + ki * ere[x];
+            if (kDec) {                        // + beta r v^T (v real)
+                nr = fmaf(wr, s_v[4 * cg + x], nr);
+                ni = fmaf(wi, s_v[4 * cg + x], ni);
+            }
             pr[x] = nr;
             pi[x] = ni;
             ore[x] += nr * qr + ni * qi;   // conj(s) * q
@@ -201,12 +222,16 @@ template <int DK, int DV, typename T>
 cudaError_t launch_one(const StepArgs &a, cudaStream_t stream)
 {
     const dim3 grid((unsigned)a.B * (unsigned)a.H, DV > kColTile ? DV / kColTile : 1);
-    if (a.par.fused)
-        sfda_step_kernel<DK, DV, T, true><<<grid, kStepThreads, 0, stream>>>(
+    if (a.par.r)
+        sfda_step_kernel<DK, DV, T, 2><<<grid, kStepThreads, 0, stream>>>(
+            static_cast<const T *>(a.q), static_cast<const T *>(a.k), static_cast<const T *>(a.v), a.alpha,
+            a.theta, a.beta, a.S, static_cast<T *>(a.o), static_cast<T *>(a.o_im), a.par);
+    else if (a.par.fused)
+        sfda_step_kernel<DK, DV, T, 1><<<grid, kStepThreads, 0, stream>>>(
             static_cast<const T *>(a.q), static_cast<const T *>(a.k), static_cast<const T *>(a.v), a.alpha,
             a.theta, a.beta, a.S, static_cast<T *>(a.o), static_cast<T *>(a.o_im), a.par);
     else
-        sfda_step_kernel<DK, DV, T, false><<<grid, kStepThreads, 0, stream>>>(
+        sfda_step_kernel<DK, DV, T, 0><<<grid, kStepThreads, 0, stream>>>(
             static_cast<const T *>(a.q), static_cast<const T *>(a.k), static_cast<const T *>(a.v), a.alpha,
             a.theta, a.beta, a.S, static_cast<T *>(a.o), static_cast<T *>(a.o_im), a.par);
     return cudaGetLastError();

@@ -121,6 +121,16 @@ def test_stable_parameterisation_entry_points_validate_on_the_host(lib):
     assert stepf(sptrs, scal, [1, 1, 128, 32, 1]) == -3
     assert stepf(sptrs, [0.0, 1.0, float("nan"), 0.0], sdims) == -8
     assert stepf(sptrs[:1] + [vp(0x1002)] + sptrs[2:], scal, sdims) == -4
+    def stepd(ptrs, dims):
+        return lib.sfda_step_decoupled(*ptrs, *[ci(d) for d in dims], None)
+
+    #        q   k   r   v   al  th  eta be  S   o   o_im
+    dptrs = [ok, ok, ok, ok, ok, ok, ok, ok, ok, ok, None]
+    assert stepd(dptrs[:2] + [None] + dptrs[3:], sdims) == -1
+    assert stepd(dptrs[:6] + [None] + dptrs[7:], sdims) == -1
+    assert stepd(dptrs, [1, 0, 128, 128, 1]) == -2
+    assert stepd(dptrs, [1, 1, 128, 48, 1]) == -3
+    assert stepd(dptrs[:2] + [vp(0x1002)] + dptrs[3:], sdims) == -4
     # workspace sizes: the tensor-core shape needs what sfda_forward needs; other shapes stage alpha, theta,
     # beta and the normalised key (each rounded up to 256 bytes)
     assert sfda.sfda_forward_fused_workspace_bytes(8, 8192, 32, 128, 128, 64, 1) == \

@@ -837,3 +837,49 @@ def test_chunk_factors_full_size_headline_sampled():
         want = bookkeeping.cumulative_phase_turns(inp["theta"][b, :, h], C)
         assert np.array_equal(got, want)
     assert worst < 1e-4, worst
+
+
+@pytest.mark.parametrize("d_k,d_v,dtype", [(128, 128, "bf16"), (64, 128, "f32"), (128, 64, "f32")])
+def test_step_decoupled_iterated_matches_oracle(d_k, d_v, dtype):
+    """The write-decoupled variant, token by token, against its oracle (Eq. "sfda-decoupled-main"); with r = k and
+    eta = beta the kernel reproduces sfda_step bit for bit."""
+    from oracle import variants
+    cfg = workloads.CONFIGS[0].scaled(name="stepd", B=2, T=40, H=3, d_k=d_k, d_v=d_v, dtype=dtype, s0_std=0.3,
+                                      seed=120 + d_k)
+    inp = workloads.forward_inputs(cfg)
+    rng = np.random.default_rng([cfg.seed, 5])
+    rnd = (lambda x: workloads.bf16_round(x)) if dtype == "bf16" else (lambda x: x.astype(np.float32))
+    r = rnd(0.1 * rng.standard_normal((cfg.B, cfg.T, cfg.H, d_k), dtype=np.float32))
+    eta = rng.uniform(0.0, 1.0, (cfg.B, cfg.T, cfg.H)).astype(np.float32)
+    eta[:, ::7] = 0.0                                   # no erase at all on some tokens
+    pairs = all_pairs(cfg)
+    sel = lambda x: np.stack([x[b, :, h] for b, h in pairs]).astype(np.float64)
+    S0 = np.stack([inp["S0"][b, h] for b, h in pairs]).astype(np.float64)
+    w_re, w_im, w_S = variants.sfda_decoupled_recurrence(sel(inp["q"]), sel(inp["k"]), sel(r), sel(inp["v"]),
+                                                         sel(inp["alpha"]), sel(inp["theta"]), sel(eta),
+                                                         sel(inp["beta"]), S0)
+    dt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    S = torch.from_numpy(inp["S0"]).to(DEV)
+    S_tied = S.clone()
+    o = torch.empty(cfg.B, cfg.H, cfg.d_v, device=DEV, dtype=dt)
+    o_im, o2, o2_im = torch.empty_like(o), torch.empty_like(o), torch.empty_like(o)
+    got_re, got_im = [], []
+    for t in range(cfg.T):
+        d = {k: to_dev(np.ascontiguousarray(inp[k][:, t]), cfg, k) for k in ("q", "k", "v", "alpha", "theta", "beta")}
+        rt = torch.from_numpy(np.ascontiguousarray(r[:, t])).to(DEV).to(dt)
+        et = torch.from_numpy(np.ascontiguousarray(eta[:, t])).to(DEV)
+        sfda.sfda_step_decoupled(d["q"], d["k"], rt, d["v"], d["alpha"], d["theta"], et, d["beta"], S, o, o_im)
+        assert sfda.last_launch_count() == 1
+        got_re.append(o.float().cpu().numpy())
+        got_im.append(o_im.float().cpu().numpy())
+        # r = k, eta = beta: the tied step
+        S_a = S_tied.clone()
+        sfda.sfda_step_decoupled(d["q"], d["k"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["beta"], S_a, o2,
+                                 o2_im)
+        sfda.sfda_step(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], S_tied, o, o_im)
+        assert rel_err(S_a.cpu().numpy(), S_tied.cpu().numpy()) < 1e-6 and rel_err(o2.float().cpu().numpy(), o.float().cpu().numpy()) < 1e-2
+    got_re, got_im = np.stack(got_re, 1), np.stack(got_im, 1)
+    tol = 5e-3 if dtype == "bf16" else 1e-4
+    assert rel_err(np.stack([got_re[b, :, h] for b, h in pairs]), w_re) <= tol
+    assert rel_err(np.stack([got_im[b, :, h] for b, h in pairs]), w_im) <= tol
+    assert rel_err(np.stack([S[b, h].cpu().numpy() for b, h in pairs]), w_S) <= 1e-4
