@@ -176,6 +176,7 @@ def main():
                     help="sweeps only: time sfda_forward_two_level (slices chosen by the library) instead of sfda_forward")
     ap.add_argument("--no-long-context", action="store_true",
                     help="skip the leg that times configuration 3 with and without the two-level scan")
+    ap.add_argument("--no-variants", action="store_true", help="skip the leg that times the write-decoupled forward")
     ap.add_argument("--no-backward", action="store_true", help="skip the leg that times sfda_backward")
     ap.add_argument("--no-factors", action="store_true", help="skip the leg that times sfda_chunk_factors")
     ap.add_argument("--no-fused", action="store_true", help="skip the leg that times the forward on raw inputs")
@@ -460,6 +461,32 @@ def main():
                "note": "token-level adjoint in fp32 on the CUDA cores, one CTA per (batch, head) pair"}
         del d_o, d_oi, dS_T, dq, dk, dv_, dal, dth, dbe, dS0, bws
 
+    # forward of the write-decoupled variant (token-level fp32 reference path) on the headline inputs
+    variant = None
+    if rank == 0 and not args.no_variants:
+        gv = torch.Generator(device=dev)
+        gv.manual_seed(99)
+        r_w = (0.1 * torch.randn(d["k"].shape, device=dev, generator=gv)).to(torch.bfloat16)
+        eta_w = torch.rand(d["beta"].shape, device=dev, generator=gv)
+
+        def vstep():
+            sfda.sfda_forward_decoupled(d["q"], d["k"], r_w, d["v"], d["alpha"], d["theta"], eta_w, d["beta"], d["S0"],
+                                        o, o_im, S_T, stream)
+
+        vstep()
+        v0, v1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        v0.record(stream)
+        for _ in range(2):
+            vstep()
+        v1.record(stream)
+        torch.cuda.synchronize()
+        v_ms = v0.elapsed_time(v1) / 2
+        variant = {"workload": cfg.name + " with a separate write direction r and erase strength eta",
+                   "ms_per_step": v_ms, "tokens_per_s": cfg.B * cfg.T / (v_ms * 1e-3),
+                   "note": "token-level fp32 reference path; the chunk kernels compute the tied model only"}
+        del r_w, eta_w
+
     # per-chunk factor export (sfda_chunk_factors) on the headline inputs: Gamma, Y, M, W and the phase turns
     factors = None
     if rank == 0 and not args.no_factors:
@@ -620,7 +647,7 @@ def main():
                    "chunk": cfg.chunk, "outputs": "Re+Im" if want_im else "Re", "state": "fp32", "S0": "N(0,0.02)",
                    "parallelism": "dp%d over (batch, head), no collective" % world,
                    "l2": "inputs+outputs %.2f GB per step, far larger than the 126 MB L2; no flush" % (abytes / 1e9)},
-        "roofline": roofline, "cpu_baseline": cpu, "other_output_mode": other_mode, "e2e": e2e, "decode": decode, "fused_front_end": fused, "chunk_factors": factors, "backward": bwd, "long_context": longctx,
+        "roofline": roofline, "cpu_baseline": cpu, "other_output_mode": other_mode, "e2e": e2e, "decode": decode, "fused_front_end": fused, "chunk_factors": factors, "backward": bwd, "write_decoupled_forward": variant, "long_context": longctx,
         "gpu_launches": launches_per_step * args.steps, "clocks": clocks.summary(),
     }
     print(json.dumps(line), flush=True)

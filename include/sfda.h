@@ -255,9 +255,18 @@ SFDA_API int sfda_step_fused(const void *q, const void *k_raw, const void *v,
  *     S <- (I - eta k k^*) Lambda S + beta r v^*,        o = S^* q,
  *
  * erase direction and strength (k, eta) separate from write direction and strength (r, beta); r = k, eta = beta is
- * sfda_step.  Arguments as sfda_step plus r [B][H][d_k] dtype and eta [B][H] float.  (The chunk kernels of this
- * library compute the tied model only: the variant needs a second operand tile per chunk.)
+ * sfda_step.  Arguments as sfda_step plus r [B][H][d_k] dtype and eta [B][H] float.
+ *
+ * sfda_forward_decoupled runs the same variant over whole sequences: arguments, layouts and results as
+ * sfda_forward (no chunk, no workspace) plus r [B][T][H][d_k] dtype and eta [B][T][H] float; token by token in
+ * fp32 on the CUDA cores, a reference path.  (The chunk-WY kernels of this library compute the tied model only:
+ * with a separate write direction a chunk needs a second rotated operand tile, two more Gram blocks and one more
+ * product.)
  */
+SFDA_API int sfda_forward_decoupled(const void *q, const void *k, const void *r, const void *v,
+                                    const float *alpha, const float *theta, const float *eta, const float *beta,
+                                    const float *S0, void *o, void *o_im, float *S_T,
+                                    int B, int T, int H, int d_k, int d_v, int dtype, void *stream);
 SFDA_API int sfda_step_decoupled(const void *q, const void *k, const void *r, const void *v,
                                  const float *alpha, const float *theta, const float *eta, const float *beta,
                                  float *S, void *o, void *o_im,

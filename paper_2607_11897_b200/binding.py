@@ -61,6 +61,7 @@ def load():
     lib.sfda_forward_two_level_workspace_bytes.argtypes = [_ci] * 8
     lib.sfda_forward_two_level.argtypes = [_vp] * 10 + [_ci] * 8 + [_vp, _sz, _vp]
     lib.sfda_step_decoupled.argtypes = [_vp] * 11 + [_ci] * 5 + [_vp]
+    lib.sfda_forward_decoupled.argtypes = [_vp] * 12 + [_ci] * 6 + [_vp]
     _LIB = lib
     return lib
 
@@ -339,3 +340,18 @@ def sfda_step_decoupled(q, k, r, v, alpha, theta, eta, beta, S, o, o_im, stream=
                                     _stream(stream))
     if rc != 0:
         raise SfdaError(rc, "sfda_step_decoupled")
+
+
+def sfda_forward_decoupled(q, k, r, v, alpha, theta, eta, beta, S0, o, o_im, S_T, stream=None):
+    """``sfda_forward_decoupled`` of ``include/sfda.h``: the write-decoupled variant over whole sequences."""
+    B, T, H, d_k = q.shape
+    d_v = v.shape[-1]
+    for t, n in ((q, "q"), (k, "k"), (r, "r"), (v, "v"), (o, "o"), (o_im, "o_im")):
+        _check(t, n, q.dtype)
+    for t, n in ((alpha, "alpha"), (theta, "theta"), (eta, "eta"), (beta, "beta"), (S0, "S0"), (S_T, "S_T")):
+        _check(t, n, torch.float32)
+    rc = load().sfda_forward_decoupled(_ptr(q), _ptr(k), _ptr(r), _ptr(v), _ptr(alpha), _ptr(theta), _ptr(eta),
+                                       _ptr(beta), _ptr(S0), _ptr(o), _ptr(o_im), _ptr(S_T), B, T, H, d_k, d_v,
+                                       _dtype_code(q), _stream(stream))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_forward_decoupled")

@@ -62,6 +62,14 @@ struct BackwardArgs {
     int B, T, H, d_k, d_v, dtype;
 };
 
+struct DecoupledArgs {
+    const void *q, *k, *r, *v;
+    const float *alpha, *theta, *eta, *beta, *S0;
+    void *o, *o_im;
+    float *S_T;
+    int B, T, H, d_k, d_v, dtype;
+};
+
 // Each returns a cudaError_t from configuring / launching; *launches is incremented per kernel.
 cudaError_t launch_forward_simt(const ForwardArgs &a, cudaStream_t stream, int *launches);
 // Tensor-core path (bf16, d_k = d_v = 128, chunk = 64): warp-specialised, chunk-pipelined tcgen05 kernel.
@@ -90,6 +98,8 @@ cudaError_t launch_forward_two_level(const ForwardArgs &a, int n, void *workspac
 // checkpointed states.
 size_t backward_workspace_bytes(int B, int T, int H, int d_k, int d_v);
 cudaError_t launch_backward(const BackwardArgs &a, void *workspace, cudaStream_t stream, int *launches);
+// Forward of the write-decoupled variant, token by token in fp32 (every supported d_k, d_v and dtype).
+cudaError_t launch_forward_decoupled(const DecoupledArgs &a, cudaStream_t stream, int *launches);
 // Stable parameterisation as a kernel of its own (every supported d_k and dtype).
 cudaError_t launch_frontend(const FrontendArgs &a, cudaStream_t stream, int *launches);
 

@@ -131,6 +131,17 @@ def test_stable_parameterisation_entry_points_validate_on_the_host(lib):
     assert stepd(dptrs, [1, 0, 128, 128, 1]) == -2
     assert stepd(dptrs, [1, 1, 128, 48, 1]) == -3
     assert stepd(dptrs[:2] + [vp(0x1002)] + dptrs[3:], sdims) == -4
+    def fwdd(ptrs, dims):
+        return lib.sfda_forward_decoupled(*ptrs, *[ci(d) for d in dims], None)
+
+    #         q   k   r   v   al  th  eta be  S0    o   o_im  S_T
+    fdptrs = [ok, ok, ok, ok, ok, ok, ok, ok, None, ok, None, None]
+    fddims = [1, 10, 2, 128, 64, 0]
+    assert fwdd(fdptrs[:2] + [None] + fdptrs[3:], fddims) == -1
+    assert fwdd(fdptrs[:6] + [None] + fdptrs[7:], fddims) == -1
+    assert fwdd(fdptrs, [1, 0, 2, 128, 64, 0]) == -2
+    assert fwdd(fdptrs, [1, 10, 2, 100, 64, 0]) == -3
+    assert fwdd(fdptrs[:9] + [vp(0x1004)] + fdptrs[10:], fddims) == -4
     # workspace sizes: the tensor-core shape needs what sfda_forward needs; other shapes stage alpha, theta,
     # beta and the normalised key (each rounded up to 256 bytes)
     assert sfda.sfda_forward_fused_workspace_bytes(8, 8192, 32, 128, 128, 64, 1) == \

@@ -883,3 +883,44 @@ def test_step_decoupled_iterated_matches_oracle(d_k, d_v, dtype):
     assert rel_err(np.stack([got_re[b, :, h] for b, h in pairs]), w_re) <= tol
     assert rel_err(np.stack([got_im[b, :, h] for b, h in pairs]), w_im) <= tol
     assert rel_err(np.stack([S[b, h].cpu().numpy() for b, h in pairs]), w_S) <= 1e-4
+
+
+@pytest.mark.parametrize("d_k,d_v,T,dtype", [(128, 128, 150, "f32"), (64, 64, 33, "f32"), (128, 64, 200, "bf16"),
+                                             (64, 128, 1, "f32")])
+def test_forward_decoupled_matches_oracle(d_k, d_v, T, dtype):
+    """The write-decoupled variant over whole sequences against its oracle; with r = k and eta = beta it agrees with
+    the tied forward of the library."""
+    from oracle import variants
+    cfg = workloads.CONFIGS[0].scaled(name="fwdd", B=2, T=T, H=2, d_k=d_k, d_v=d_v, dtype=dtype, s0_std=0.4,
+                                      seed=130 + T)
+    inp = workloads.forward_inputs(cfg)
+    rng = np.random.default_rng([cfg.seed, 6])
+    rnd = (lambda x: workloads.bf16_round(x)) if dtype == "bf16" else (lambda x: x.astype(np.float32))
+    r = rnd(0.1 * rng.standard_normal((cfg.B, T, cfg.H, d_k), dtype=np.float32))
+    eta = rng.uniform(0.0, 1.0, (cfg.B, T, cfg.H)).astype(np.float32)
+    d = {k: (None if v is None else to_dev(v, cfg, k)) for k, v in inp.items()}
+    dt = d["q"].dtype
+    rt, et = torch.from_numpy(r).to(DEV).to(dt), torch.from_numpy(eta).to(DEV)
+    o = torch.empty(cfg.B, T, cfg.H, d_v, device=DEV, dtype=dt)
+    o_im = torch.empty_like(o)
+    S_T = torch.empty(cfg.B, cfg.H, d_k, d_v, device=DEV)
+    sfda.sfda_forward_decoupled(d["q"], d["k"], rt, d["v"], d["alpha"], d["theta"], et, d["beta"], d["S0"], o, o_im, S_T)
+    torch.cuda.synchronize()
+    assert sfda.last_launch_count() == 1
+    pairs = all_pairs(cfg)
+    sel = lambda x: np.stack([x[b, :, h] for b, h in pairs]).astype(np.float64)
+    S0 = np.stack([inp["S0"][b, h] for b, h in pairs]).astype(np.float64)
+    w_re, w_im, w_S = variants.sfda_decoupled_recurrence(sel(inp["q"]), sel(inp["k"]), sel(r), sel(inp["v"]),
+                                                         sel(inp["alpha"]), sel(inp["theta"]), sel(eta),
+                                                         sel(inp["beta"]), S0)
+    tol = 5e-3 if dtype == "bf16" else 1e-4
+    on, oin, Sn = o.float().cpu().numpy(), o_im.float().cpu().numpy(), S_T.cpu().numpy()
+    assert rel_err(np.stack([on[b, :, h] for b, h in pairs]), w_re) <= tol
+    assert rel_err(np.stack([oin[b, :, h] for b, h in pairs]), w_im) <= tol
+    assert rel_err(np.stack([Sn[b, h] for b, h in pairs]), w_S) <= 1e-4
+    # tied special case against the library's own forward
+    sfda.sfda_forward_decoupled(d["q"], d["k"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["beta"], d["S0"],
+                                o, None, S_T)
+    torch.cuda.synchronize()
+    o_t, _, S_t = run_forward(cfg, inp, simt=True)
+    assert rel_err(o.float().cpu().numpy(), o_t) <= tol and rel_err(S_T.cpu().numpy(), S_t) <= 1e-4
