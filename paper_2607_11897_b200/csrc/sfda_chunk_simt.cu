@@ -38,7 +38,7 @@ struct ChunkSmem {
     static constexpr int KS = DK + 2;  // row stride of kp / qp (floats): spreads rows over banks
     static constexpr int LS = M + 1;   // row stride of lg
     static constexpr int GS = C + 1;   // row stride of the Gram matrices
-    float *kp, *qp, *lg, *gcr, *gci, *lgC, *beta;
+    float *kp, *qp, *lg, *gcr, *gci, *lgC, *beta, *scan;
     __device__ explicit ChunkSmem(float *base)
     {
         kp = base;
@@ -48,8 +48,9 @@ struct ChunkSmem {
         gci = gcr + M;
         lgC = gci + M;
         beta = lgC + M;
+        scan = beta + C;                                   // [2][kThreads]: group totals of the scan
     }
-    static constexpr int floats = 2 * C * KS + C * LS + 3 * M + C;
+    static constexpr int floats = 2 * C * KS + C * LS + 3 * M + C + 2 * kThreads;
 };
 
 // Loads one chunk of k (and q when given), alpha, theta, beta; leaves in shared memory the rotated
@@ -64,44 +65,72 @@ __device__ void load_and_rotate(const ChunkSmem<DK, C> &sm, const T *__restrict_
 {
     constexpr int M = DK / 2;
     using S = ChunkSmem<DK, C>;
+    // thread = (coordinate j, group g of TG consecutive tokens): every global load of the thread is issued before the
+    // first one is used; the prefix sums run inside a group first and the groups are chained through shared memory
+    constexpr int G = kThreads / M, TG = C / G;
+    static_assert(kThreads % M == 0 && C % G == 0, "the scan's groups must tile the chunk");
     const int tid = threadIdx.x;
-    for (int idx = tid; idx < C * DK; idx += kThreads) {
-        const int t = idx / DK, x = idx % DK;
-        float kv = 0.f, qv = 0.f;
+    const int j = tid % M, g = tid / M;
+    float lgv[TG], kr[TG], ki[TG], qr[TG], qi[TG];
+    uint32_t tu[TG];
+#pragma unroll
+    for (int x = 0; x < TG; ++x) {
+        const int t = g * TG + x;
+        float al = 1.f, th = 0.f;
+        kr[x] = ki[x] = qr[x] = qi[x] = 0.f;
         if (t < len) {
-            const size_t g = (((size_t)b * T_ + t0 + t) * H + h) * DK + x;
-            kv = ld_val(k, g);
-            if (q) qv = ld_val(q, g);
+            const size_t row = ((size_t)b * T_ + t0 + t) * H + h;
+            al = alpha[row * M + j];
+            th = theta[row * M + j];
+            kr[x] = ld_val(k, row * DK + 2 * j);
+            ki[x] = ld_val(k, row * DK + 2 * j + 1);
+            if (q) {
+                qr[x] = ld_val(q, row * DK + 2 * j);
+                qi[x] = ld_val(q, row * DK + 2 * j + 1);
+            }
         }
-        sm.kp[t * S::KS + x] = kv;
-        sm.qp[t * S::KS + x] = qv;
+        lgv[x] = al;
+        tu[x] = __float_as_uint(th);
     }
     if (tid < C) sm.beta[tid] = tid < len ? beta[((size_t)b * T_ + t0 + tid) * H + h] : 0.f;
+    float acc = 0.f;
+    uint32_t ta = 0u;
+#pragma unroll
+    for (int x = 0; x < TG; ++x) {
+        acc += log_decay(lgv[x]);
+        ta += phase_to_turns(__uint_as_float(tu[x]));
+        lgv[x] = acc;
+        tu[x] = ta;
+    }
+    float *grp_lg = sm.scan;                                        // [G][M]
+    uint32_t *grp_tu = reinterpret_cast<uint32_t *>(sm.scan + G * M);
+    grp_lg[g * M + j] = acc;
+    grp_tu[g * M + j] = ta;
     __syncthreads();
-    if (tid < M) {
-        const int j = tid;
-        float acc = 0.f, cs = 1.f, sn = 0.f;
-        uint32_t turns = 0u;
-#pragma unroll 4
-        for (int t = 0; t < C; ++t) {
-            if (t < len) {
-                const size_t g = (((size_t)b * T_ + t0 + t) * H + h) * M + j;
-                acc += log_decay(alpha[g]);
-                turns += phase_to_turns(theta[g]);
-                if (turns_out) turns_out[g] = turns;
-            }
-            sm.lg[t * S::LS + j] = acc;
-            turns_to_cos_sin(turns, &cs, &sn);
-            const float kr = sm.kp[t * S::KS + 2 * j], ki = sm.kp[t * S::KS + 2 * j + 1];
-            sm.kp[t * S::KS + 2 * j] = kr * cs + ki * sn;      // e^{-i phi} (kr + i ki)
-            sm.kp[t * S::KS + 2 * j + 1] = ki * cs - kr * sn;
-            const float qr = sm.qp[t * S::KS + 2 * j], qi = sm.qp[t * S::KS + 2 * j + 1];
-            sm.qp[t * S::KS + 2 * j] = qr * cs + qi * sn;
-            sm.qp[t * S::KS + 2 * j + 1] = qi * cs - qr * sn;
+    float base = 0.f;
+    uint32_t tb = 0u;
+    for (int gg = 0; gg < g; ++gg) {
+        base += grp_lg[gg * M + j];
+        tb += grp_tu[gg * M + j];
+    }
+#pragma unroll
+    for (int x = 0; x < TG; ++x) {
+        const int t = g * TG + x;
+        const float l = base + lgv[x];
+        const uint32_t tt = tb + tu[x];
+        if (turns_out && t < len) turns_out[(((size_t)b * T_ + t0 + t) * H + h) * M + j] = tt;
+        float cs, sn;
+        turns_to_cos_sin(tt, &cs, &sn);
+        sm.lg[t * S::LS + j] = l;
+        sm.kp[t * S::KS + 2 * j] = kr[x] * cs + ki[x] * sn;         // e^{-i phi} (kr + i ki)
+        sm.kp[t * S::KS + 2 * j + 1] = ki[x] * cs - kr[x] * sn;
+        sm.qp[t * S::KS + 2 * j] = qr[x] * cs + qi[x] * sn;
+        sm.qp[t * S::KS + 2 * j + 1] = qi[x] * cs - qr[x] * sn;
+        if (t == C - 1) {
+            sm.gcr[j] = cs;
+            sm.gci[j] = sn;
+            sm.lgC[j] = l;
         }
-        sm.gcr[j] = cs;
-        sm.gci[j] = sn;
-        sm.lgC[j] = acc;
     }
     __syncthreads();
 }
@@ -114,7 +143,8 @@ constexpr int forward_smem_floats()
 {
     return ChunkSmem<DK, C>::floats + 2 * (DK / 2) * kSlice  // state (re, im)
            + 4 * C * (C + 1)                                  // Kt, Aq (re, im)
-           + 2 * C * kSlice;                                  // E (re, im)
+           + 2 * C * kSlice                                   // E (re, im)
+           + 2 * C * (DK / 2 + 1);                            // a_t and a_C / a_t of the chunk
 }
 
 template <int DK, int C, typename T>
@@ -136,6 +166,8 @@ sfda_forward_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const
     float *Aqi = Aqr + C * SM::GS;
     float *Er = Aqi + C * SM::GS;
     float *Ei = Er + C * kSlice;
+    float *aw = Ei + C * kSlice;          // [C][LS]  a_t = exp(lg_t)           (<= 1)
+    float *yw = aw + C * SM::LS;          // [C][LS]  a_C / a_t = exp(lg_C - lg_t)  (<= 1)
 
     const int tid = threadIdx.x, lane = tid % 32, wid = tid / 32;
     const int nsl = dv / kSlice;
@@ -156,6 +188,14 @@ sfda_forward_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const
         const int len = min(C, T_ - t0);
         __syncthreads();
         load_and_rotate<DK, C, T>(sm, k, q, alpha, theta, beta, nullptr, b, h, T_, H, t0, len);
+        // the two decay weights every product with the state needs, once per chunk instead of once per use
+        for (int idx = tid; idx < C * M; idx += kThreads) {
+            const int t = idx / M, j = idx % M;
+            const float l = sm.lg[t * SM::LS + j];
+            aw[t * SM::LS + j] = expf(l);
+            yw[t * SM::LS + j] = expf(sm.lgC[j] - l);
+        }
+        __syncthreads();
 
         // Gram blocks Kt (i < t) and Aq (i <= t).
         for (int p = tid; p < C * (C + 1) / 2; p += kThreads) {
@@ -184,9 +224,9 @@ sfda_forward_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const
         for (int t = wid; t < C; t += kThreads / 32) {
             float rr = 0.f, ri = 0.f;
             if (t < len) rr = ld_val(v, (((size_t)b * T_ + t0 + t) * H + h) * dv + c0 + lane);
-            const float *kt = sm.kp + t * SM::KS, *lt = sm.lg + t * SM::LS;
+            const float *kt = sm.kp + t * SM::KS, *at = aw + t * SM::LS;
             for (int j = 0; j < M; ++j) {
-                const float w = expf(lt[j]);
+                const float w = at[j];
                 const float wr = w * kt[2 * j], wi = w * kt[2 * j + 1];
                 const float sr = Sre[j * kSlice + lane], si = Sim[j * kSlice + lane];
                 rr -= wr * sr + wi * si;   // conj(w) * s
@@ -230,9 +270,9 @@ sfda_forward_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const
         // Outputs: o_t^* = (conj(gamma_t) q_t)^* S_0 + sum_{i<=t} Aq[t][i] e_i^T ; o = conj of that row.
         for (int t = wid; t < len; t += kThreads / 32) {
             float rr = 0.f, ri = 0.f;
-            const float *qt = sm.qp + t * SM::KS, *lt = sm.lg + t * SM::LS;
+            const float *qt = sm.qp + t * SM::KS, *at = aw + t * SM::LS;
             for (int j = 0; j < M; ++j) {
-                const float w = expf(lt[j]);
+                const float w = at[j];
                 const float wr = w * qt[2 * j], wi = w * qt[2 * j + 1];
                 const float sr = Sre[j * kSlice + lane], si = Sim[j * kSlice + lane];
                 rr += wr * sr + wi * si;
@@ -255,7 +295,7 @@ sfda_forward_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const
             const float aC = expf(sm.lgC[j]);
             float nr = aC * Sre[j * kSlice + lane], ni = aC * Sim[j * kSlice + lane];
             for (int t = 0; t < C; ++t) {
-                const float w = expf(sm.lgC[j] - sm.lg[t * SM::LS + j]);
+                const float w = yw[t * SM::LS + j];
                 const float yr = w * sm.kp[t * SM::KS + 2 * j], yi = w * sm.kp[t * SM::KS + 2 * j + 1];
                 const float er = Er[t * kSlice + lane], ei = Ei[t * kSlice + lane];
                 nr += yr * er - yi * ei;
