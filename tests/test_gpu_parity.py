@@ -924,3 +924,26 @@ def test_forward_decoupled_matches_oracle(d_k, d_v, T, dtype):
     torch.cuda.synchronize()
     o_t, _, S_t = run_forward(cfg, inp, simt=True)
     assert rel_err(o.float().cpu().numpy(), o_t) <= tol and rel_err(S_T.cpu().numpy(), S_t) <= 1e-4
+
+
+def test_final_state_may_alias_the_initial_state():
+    """S_T == S0 (the same buffer) is allowed: the plain tensor-core forward and the two-level scan."""
+    cfg = workloads.CONFIGS[1].scaled(name="alias", B=2, T=2048, H=2, s0_std=0.3, seed=140)
+    inp = workloads.forward_inputs(cfg)
+    pairs = all_pairs(cfg)
+    _, _, w_S = oracle_pairs(inp, pairs)
+    d = {k: to_dev(v, cfg, k) for k, v in inp.items()}
+    o = torch.empty(cfg.B, cfg.T, cfg.H, cfg.d_v, device=DEV, dtype=torch.bfloat16)
+    for two_level in (False, True):
+        S = d["S0"].clone()
+        if two_level:
+            ws = torch.empty(sfda.sfda_forward_two_level_workspace_bytes(cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk,
+                                                                         1, 4), device=DEV, dtype=torch.uint8)
+            sfda.sfda_forward_two_level(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], S, o, None, S,
+                                        cfg.chunk, 4, ws)
+        else:
+            ws = torch.empty(sfda.sfda_workspace_bytes(cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk, 1),
+                             device=DEV, dtype=torch.uint8)
+            sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], S, o, None, S, cfg.chunk, ws)
+        torch.cuda.synchronize()
+        assert rel_err(np.stack([S.cpu().numpy()[b, h] for b, h in pairs]), w_S) <= TOL["bf16"]
