@@ -418,11 +418,30 @@ def main():
                                                             ld["beta"], ld["S0"], lo, lo_im, lS, lcfg.chunk, 0, lws,
                                                             stream))
         assert sfda.sfda_workspace_status(lws, stream) == 0
+        two_launches = sfda.last_launch_count()
+        # the backward pass on the same few sequences: the value columns are split over 4 CTAs per sequence
+        lg = [torch.empty_like(ld[key]) for key in ("q", "k", "v", "alpha", "theta", "beta")] + [torch.empty_like(lS)]
+        lbws = torch.empty(sfda.sfda_backward_workspace_bytes(lcfg.B, lcfg.T, lcfg.H, lcfg.d_k, lcfg.d_v, 1),
+                           dtype=torch.uint8, device=dev)
+
+        def lbstep():
+            sfda.sfda_backward(ld["q"], ld["k"], ld["v"], ld["alpha"], ld["theta"], ld["beta"], ld["S0"], lo, lo_im, lS,
+                               *lg, lbws, stream)
+
+        lbstep()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        t0.record(stream)
+        lbstep()
+        t1.record(stream)
+        torch.cuda.synchronize()
+        lb_ms = t0.elapsed_time(t1)
         longctx = {"workload": lcfg.name + " (B=1, T=131072, H=16)", "plain_ms_per_step": plain_ms,
                    "plain_tokens_per_s": lcfg.B * lcfg.T / (plain_ms * 1e-3), "two_level_ms_per_step": two_ms,
                    "two_level_tokens_per_s": lcfg.B * lcfg.T / (two_ms * 1e-3),
-                   "two_level_launches": sfda.last_launch_count(), "workspace_bytes": int(lws.numel())}
-        del ld, lo, lo_im, lS, lws
+                   "two_level_launches": two_launches, "workspace_bytes": int(lws.numel()),
+                   "backward_ms_per_call": lb_ms, "backward_launches": sfda.last_launch_count()}
+        del ld, lo, lo_im, lS, lws, lg, lbws
 
     # backward pass (sfda_backward) on the headline inputs: token-level fp32 adjoint, a first correct path
     bwd = None

@@ -357,12 +357,15 @@ SFDA_API int sfda_forward_fused(const void *q, const void *k_raw, const void *v,
  *  gradients:   dq, dk [B][T][H][d_k] dtype (the (Re, Im) pair of a coordinate gets the gradient with respect
  *               to its two real numbers), dv [B][T][H][d_v] dtype, dalpha, dtheta [B][T][H][m] float,
  *               dbeta [B][T][H] float, dS0 [B][H][d_k][d_v] float.  All are required and overwritten.
- *  workspace:   sfda_backward_workspace_bytes(...) bytes of device scratch (the state at the start of every
- *               64 tokens and the 64 states of one such segment, per (batch, head) pair); clobbered.
+ *  workspace:   sfda_backward_workspace_bytes(...) bytes of device scratch (per (batch, head) pair the state at the
+ *               start of every 64 tokens and the 64 states of one such segment; with few sequences also fp32
+ *               shares of dq, dk, dalpha, dtheta, dbeta per block of value columns); clobbered.
  *
  * d_k, d_v in {64, 128}; no chunk argument (the derivative does not depend on the chunking).  fp32 arithmetic on
- * the CUDA cores, token by token, one CTA per (batch, head) pair: a first correct path, not a fast one.  The
- * result is deterministic (no sum crosses CTAs).
+ * the CUDA cores, token by token: a first correct path, not a fast one.  One CTA per (batch, head) pair; when
+ * B * H is at most half (a quarter) of the 148 SMs of a B200, the value columns -- which never interact -- are split
+ * into blocks of 64 (32) with a CTA each, and a second kernel adds the blocks' shares of the sums over the
+ * columns in a fixed order.  The result is deterministic either way.
  */
 SFDA_API size_t sfda_backward_workspace_bytes(int B, int T, int H, int d_k, int d_v, int dtype);
 SFDA_API int sfda_backward(const void *q, const void *k, const void *v,

@@ -1,7 +1,8 @@
 // sfda_backward: reverse-mode derivative of the recurrence of Section 3 (Eq. "sfda") with o_t = S_t^* q_t, token by
 // token in fp32 on the CUDA cores.  (The paper asks for the backward pass only as something to be timed, App. E; what
-// it computes is the adjoint of Eq. "sfda".)  This is the first correct path: one CTA per (batch, head) pair walks
-// the sequence three times --
+// it computes is the adjoint of Eq. "sfda".)  This is the first correct path: one CTA per (batch, head) pair and
+// block of value columns (the columns of the state and of its cotangent never interact; with many sequences a block
+// is all d_v columns, with few it is 64 or 32 of them so that every SM has work) walks the sequence three times --
 //
 //   1. forward, keeping the state at the start of every segment of kSeg tokens (checkpoints in the workspace);
 //   2. per segment, last to first: forward again from the checkpoint, keeping S_{t-1} of every token of the segment;
@@ -16,7 +17,9 @@
 //   G <- conj(lam) Zb   (row-wise: the cotangent of S_{t-1})
 //
 // Complex cotangents Xb mean dL = Re sum conj(Xb) dX, i.e. the ordinary gradient with respect to the (Re, Im) pair.
-// No sums cross CTAs, so the result is deterministic.
+// dq, dk, dalpha, dtheta, dbeta are sums over the value columns: with more than one column block every block writes
+// its share as fp32 to the workspace and a second kernel adds the shares in a fixed order, so the result is
+// deterministic either way.
 #include "sfda_common.cuh"
 #include "sfda_internal.h"
 
@@ -48,14 +51,19 @@ struct BwdArgsDev {
     const float *alpha, *theta, *beta, *S0, *dS_T;
     void *dq, *dk, *dv;
     float *dalpha, *dtheta, *dbeta, *dS0;
-    float *check, *scratch;      // [BH][NS][M][DV][2], [BH][kSeg][M][DV][2] (interleaved complex)
+    float *dq_p, *dk_p, *dalpha_p, *dtheta_p, *dbeta_p;   // shares of the column blocks: [blocks][rows][...] fp32
+    float *check, *scratch;      // [BH][blocks][NS][M][cols][2], [BH][blocks][kSeg][M][cols][2] (interleaved complex)
+    size_t rows;                 // B * T * H
     int T, H, NS;
 };
 
-template <int DK, int DV, typename T>
+// DVT value columns per state, DV of them per CTA
+template <int DK, int DVT, int DV, typename T>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 sfda_backward_kernel(const BwdArgsDev a)
 {
+    constexpr int NSL = DVT / DV;                  // column blocks per state
+    static_assert(DVT % DV == 0 && DV % 32 == 0, "the value columns split into blocks of whole warps");
     using L = BwdSmem<DK, DV>;
     constexpr int M = L::M, RS = L::RS, NG = L::NG, RA = M / NG;      // RA rows per thread in the column mapping
     constexpr int TPR = kBwdThreads / M, CPT = DV / TPR;               // threads per row / columns per thread (row mapping)
@@ -76,12 +84,12 @@ sfda_backward_kernel(const BwdArgsDev a)
     float *scal = red + NG * 4 * DV;            // [0] beta, [8 + 4 w + x] partial sums of warp w
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int bh = blockIdx.x, h = bh % a.H, b = bh / a.H;
+    const int bh = blockIdx.x, h = bh % a.H, b = bh / a.H, slice = blockIdx.y, c0 = slice * DV;
     const int T_ = a.T, H = a.H;
     const T *q = static_cast<const T *>(a.q), *k = static_cast<const T *>(a.k), *v = static_cast<const T *>(a.v);
     const T *d_o = static_cast<const T *>(a.d_o), *d_oi = static_cast<const T *>(a.d_o_im);
-    float *check = a.check + (size_t)bh * a.NS * 2 * M * DV;
-    float *scratch = a.scratch + (size_t)bh * kSeg * 2 * M * DV;
+    float *check = a.check + ((size_t)bh * NSL + slice) * a.NS * 2 * M * DV;
+    float *scratch = a.scratch + ((size_t)bh * NSL + slice) * kSeg * 2 * M * DV;
 
     // column-owner mapping (A): column c, rows g, g + NG, ...;  row-owner mapping (B): row jb, columns part + TPR n
     const int c = tid % DV, g = tid / DV;
@@ -103,10 +111,10 @@ sfda_backward_kernel(const BwdArgsDev a)
             }
         } else if (tid < M + DV) {
             const int cc = tid - M;
-            r0 = ld_val(v, row * DV + cc);
+            r0 = ld_val(v, row * DVT + c0 + cc);
             if (back) {
-                r1 = ld_val(d_o, row * DV + cc);
-                r2 = d_oi ? ld_val(d_oi, row * DV + cc) : 0.f;
+                r1 = ld_val(d_o, row * DVT + c0 + cc);
+                r2 = d_oi ? ld_val(d_oi, row * DVT + c0 + cc) : 0.f;
             }
         } else if (tid == M + DV) {
             r0 = a.beta[row];
@@ -180,7 +188,7 @@ sfda_backward_kernel(const BwdArgsDev a)
     float2 *S = Pb(0);
     for (int idx = tid; idx < M * DV; idx += kBwdThreads) {
         const int j = idx / DV, cc = idx % DV;
-        S[j * RS + cc] = a.S0 ? make_float2(a.S0[((size_t)bh * DK + 2 * j) * DV + cc], a.S0[((size_t)bh * DK + 2 * j + 1) * DV + cc])
+        S[j * RS + cc] = a.S0 ? make_float2(a.S0[((size_t)bh * DK + 2 * j) * DVT + c0 + cc], a.S0[((size_t)bh * DK + 2 * j + 1) * DVT + c0 + cc])
                               : make_float2(0.f, 0.f);
     }
     const int t_last_check = (a.NS - 1) * kSeg;
@@ -198,12 +206,15 @@ sfda_backward_kernel(const BwdArgsDev a)
     // ---- cotangent of the final state
     for (int idx = tid; idx < M * DV; idx += kBwdThreads) {
         const int j = idx / DV, cc = idx % DV;
-        G[j * RS + cc] = a.dS_T ? make_float2(a.dS_T[((size_t)bh * DK + 2 * j) * DV + cc], a.dS_T[((size_t)bh * DK + 2 * j + 1) * DV + cc])
+        G[j * RS + cc] = a.dS_T ? make_float2(a.dS_T[((size_t)bh * DK + 2 * j) * DVT + c0 + cc], a.dS_T[((size_t)bh * DK + 2 * j + 1) * DVT + c0 + cc])
                                 : make_float2(0.f, 0.f);
     }
     __syncthreads();      // also: every thread's checkpoint stores precede the loads below (same CTA, after a barrier)
 
     T *dq = static_cast<T *>(a.dq), *dk = static_cast<T *>(a.dk), *dv = static_cast<T *>(a.dv);
+    float *dq_p = a.dq_p + (size_t)slice * a.rows * DK, *dk_p = a.dk_p + (size_t)slice * a.rows * DK;
+    float *dal_p = a.dalpha_p + (size_t)slice * a.rows * M, *dth_p = a.dtheta_p + (size_t)slice * a.rows * M;
+    float *dbe_p = a.dbeta_p + (size_t)slice * a.rows;
     for (int si = a.NS - 1; si >= 0; --si) {
         const int t0 = si * kSeg, t1 = min(t0 + kSeg, T_);
         // ---- sweep 2: forward again from the checkpoint, S_{t-1} of every token to the scratch
@@ -273,7 +284,7 @@ sfda_backward_kernel(const BwdArgsDev a)
                 const float yr = yu.x, yi = yu.y;
                 v_p[c] = make_float2(pr, pi);
                 v_yu[c] = make_float4(yr, yi, ur, ui);
-                st_val(dv, row * DV + c, bt * pr);
+                st_val(dv, row * DVT + c0 + c, bt * pr);
                 float s0 = ur * pr - ui * pi;                       // Re(u p)
                 float s1 = ur * yr - ui * yi, s2 = ur * yi + ui * yr;   // u yb
 #pragma unroll
@@ -290,7 +301,7 @@ sfda_backward_kernel(const BwdArgsDev a)
                 float sr_ = 0.f, si_ = 0.f, dbe = 0.f;
 #pragma unroll
                 for (int w = 0; w < DV / 32; ++w) { dbe += scal[8 + 4 * w]; sr_ += scal[9 + 4 * w]; si_ += scal[10 + 4 * w]; }
-                if (tid == 0) a.dbeta[row] = dbe;
+                if (tid == 0) (NSL == 1 ? a.dbeta : dbe_p)[row] = dbe;
                 const int j = jb;
                 const float4 lk = v_lk[j], qc = v_qc[j];
                 const float lr = lk.x, li = lk.y, kr = lk.z, ki = lk.w;
@@ -322,13 +333,24 @@ sfda_backward_kernel(const BwdArgsDev a)
                     lbr += __shfl_xor_sync(0xffffffffu, lbr, d);  lbi += __shfl_xor_sync(0xffffffffu, lbi, d);
                 }
                 if (part == 0) {
-                    st_val(dq, row * DK + 2 * j, qzr + bt * (kr * sr_ - ki * si_));      // + beta k (u^T yb)
-                    st_val(dq, row * DK + 2 * j + 1, qzi + bt * (kr * si_ + ki * sr_));
-                    st_val(dk, row * DK + 2 * j, bt * (k1r - k2r));
-                    st_val(dk, row * DK + 2 * j + 1, bt * (k1i - k2i));
+                    const float dqr = qzr + bt * (kr * sr_ - ki * si_), dqi = qzi + bt * (kr * si_ + ki * sr_);   // + beta k (u^T yb)
+                    const float dkr = bt * (k1r - k2r), dki = bt * (k1i - k2i);
                     const float cs = qc.z, sn = qc.w;
-                    a.dalpha[row * M + j] = lbr * cs + lbi * sn;                          // Re(conj(lamb) e^{i theta})
-                    a.dtheta[row * M + j] = lbi * lr - lbr * li;                          // -Im(conj(lamb) lam)
+                    const float dal = lbr * cs + lbi * sn;                                // Re(conj(lamb) e^{i theta})
+                    const float dth = lbi * lr - lbr * li;                                // -Im(conj(lamb) lam)
+                    if constexpr (NSL == 1) {
+                        st_val(dq, row * DK + 2 * j, dqr);
+                        st_val(dq, row * DK + 2 * j + 1, dqi);
+                        st_val(dk, row * DK + 2 * j, dkr);
+                        st_val(dk, row * DK + 2 * j + 1, dki);
+                        a.dalpha[row * M + j] = dal;
+                        a.dtheta[row * M + j] = dth;
+                    } else {      // this column block's share of the sums over the columns
+                        *reinterpret_cast<float2 *>(dq_p + row * DK + 2 * j) = make_float2(dqr, dqi);
+                        *reinterpret_cast<float2 *>(dk_p + row * DK + 2 * j) = make_float2(dkr, dki);
+                        dal_p[row * M + j] = dal;
+                        dth_p[row * M + j] = dth;
+                    }
                 }
             }
             __syncthreads();
@@ -338,53 +360,163 @@ sfda_backward_kernel(const BwdArgsDev a)
     }
     for (int idx = tid; idx < M * DV; idx += kBwdThreads) {
         const int j = idx / DV, cc = idx % DV;
-        a.dS0[((size_t)bh * DK + 2 * j) * DV + cc] = G[j * RS + cc].x;
-        a.dS0[((size_t)bh * DK + 2 * j + 1) * DV + cc] = G[j * RS + cc].y;
+        a.dS0[((size_t)bh * DK + 2 * j) * DVT + c0 + cc] = G[j * RS + cc].x;
+        a.dS0[((size_t)bh * DK + 2 * j + 1) * DVT + c0 + cc] = G[j * RS + cc].y;
     }
 }
 
-template <int DK, int DV, typename T>
-cudaError_t launch_typed(const BackwardArgs &x, void *workspace, cudaStream_t stream)
+// ---- the sums over the column blocks: out[i] = share_0[i] + share_1[i] + ... in that order, one thread per four
+// consecutive elements.  HBM-bound and small beside the sweeps.
+constexpr int kSumThreads = 256;
+
+__device__ __forceinline__ void st_val4(float *p, float4 x) { *reinterpret_cast<float4 *>(p) = x; }
+__device__ __forceinline__ void st_val4(__nv_bfloat16 *p, float4 x)
+{
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(x.x, x.y), hi = __floats2bfloat162_rn(x.z, x.w);
+    *reinterpret_cast<uint2 *>(p) = make_uint2(*reinterpret_cast<const uint32_t *>(&lo), *reinterpret_cast<const uint32_t *>(&hi));
+}
+
+template <int NSL, typename T>
+__global__ void __launch_bounds__(kSumThreads)
+sfda_backward_sum_kernel(const float *__restrict__ dq_p, const float *__restrict__ dk_p, const float *__restrict__ dal_p,
+                         const float *__restrict__ dth_p, const float *__restrict__ dbe_p, T *__restrict__ dq,
+                         T *__restrict__ dk, float *__restrict__ dalpha, float *__restrict__ dtheta,
+                         float *__restrict__ dbeta, size_t n_key, size_t n_coord, size_t rows)
+{
+    // work items in float4 units: [dq | dk | dalpha | dtheta] then dbeta one by one
+    const size_t q4 = n_key / 4, c4 = n_coord / 4, total = 2 * q4 + 2 * c4 + rows;
+    for (size_t i = (size_t)blockIdx.x * kSumThreads + threadIdx.x; i < total; i += (size_t)gridDim.x * kSumThreads) {
+        if (i < 2 * q4 + 2 * c4) {
+            const float *src;
+            size_t n, at;
+            int which;
+            if (i < q4) { src = dq_p; n = n_key; at = i; which = 0; }
+            else if (i < 2 * q4) { src = dk_p; n = n_key; at = i - q4; which = 1; }
+            else if (i < 2 * q4 + c4) { src = dal_p; n = n_coord; at = i - 2 * q4; which = 2; }
+            else { src = dth_p; n = n_coord; at = i - 2 * q4 - c4; which = 3; }
+            float4 acc = *reinterpret_cast<const float4 *>(src + 4 * at);
+#pragma unroll
+            for (int sl = 1; sl < NSL; ++sl) {
+                const float4 x = *reinterpret_cast<const float4 *>(src + (size_t)sl * n + 4 * at);
+                acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+            }
+            if (which >= 2) {
+                *reinterpret_cast<float4 *>((which == 2 ? dalpha : dtheta) + 4 * at) = acc;
+            } else {
+                st_val4((which == 0 ? dq : dk) + 4 * at, acc);
+            }
+        } else {
+            const size_t at = i - 2 * q4 - 2 * c4;
+            float acc = dbe_p[at];
+#pragma unroll
+            for (int sl = 1; sl < NSL; ++sl) acc += dbe_p[(size_t)sl * rows + at];
+            dbeta[at] = acc;
+        }
+    }
+}
+
+// Value columns per CTA: all of them while the (batch, head) pairs alone fill the SMs; halved (down to 32) while the
+// grid still fits the SMs of a B200, so that few sequences use the whole device.  (A fixed count rather than the
+// device's: the workspace size must not depend on where it is asked for.)
+constexpr int kBwdTargetCtas = 148;
+
+int bwd_cols(int B, int H, int d_v)
+{
+    int cols = d_v;
+    while (cols > 32 && (long long)B * H * (d_v / (cols / 2)) <= kBwdTargetCtas) cols /= 2;
+    return cols;
+}
+
+// workspace: checkpoints, the S_{t-1} of one segment, then (more than one column block only) the blocks' shares of
+// dq, dk, dalpha, dtheta, dbeta
+struct BwdWorkspace {
+    size_t check, scratch, dq, dk, dalpha, dtheta, dbeta, total;   // offsets and size in floats
+};
+
+BwdWorkspace bwd_workspace(int B, int T, int H, int d_k, int d_v)
+{
+    const size_t bhn = (size_t)B * H, ns = (size_t)(T + kSeg - 1) / kSeg, state = (size_t)d_k * d_v;
+    const size_t rows = bhn * T, nsl = (size_t)(d_v / bwd_cols(B, H, d_v)), shares = nsl > 1 ? nsl * rows : 0;
+    BwdWorkspace w;
+    w.check = 0;
+    w.scratch = w.check + bhn * ns * state;
+    w.dq = w.scratch + bhn * kSeg * state;
+    w.dk = w.dq + shares * d_k;
+    w.dalpha = w.dk + shares * d_k;
+    w.dtheta = w.dalpha + shares * (d_k / 2);
+    w.dbeta = w.dtheta + shares * (d_k / 2);
+    w.total = w.dbeta + ((shares + 3) & ~(size_t)3);
+    return w;
+}
+
+template <int DK, int DVT, int DV, typename T>
+cudaError_t launch_cols(const BackwardArgs &x, void *workspace, cudaStream_t stream, int *launches)
 {
     using L = BwdSmem<DK, DV>;
-    auto kern = sfda_backward_kernel<DK, DV, T>;
+    constexpr int NSL = DVT / DV;
+    auto kern = sfda_backward_kernel<DK, DVT, DV, T>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::bytes);
     if (e != cudaSuccess) return e;
+    const BwdWorkspace w = bwd_workspace(x.B, x.T, x.H, DK, DVT);
+    float *ws = static_cast<float *>(workspace);
     BwdArgsDev a;
     a.q = x.q; a.k = x.k; a.v = x.v; a.d_o = x.d_o; a.d_o_im = x.d_o_im;
     a.alpha = x.alpha; a.theta = x.theta; a.beta = x.beta; a.S0 = x.S0; a.dS_T = x.dS_T;
     a.dq = x.dq; a.dk = x.dk; a.dv = x.dv; a.dalpha = x.dalpha; a.dtheta = x.dtheta; a.dbeta = x.dbeta; a.dS0 = x.dS0;
     a.T = x.T; a.H = x.H; a.NS = (x.T + kSeg - 1) / kSeg;
-    const size_t bhn = (size_t)x.B * x.H, state = (size_t)DK * DV;
-    a.check = static_cast<float *>(workspace);
-    a.scratch = a.check + bhn * a.NS * state;
-    kern<<<(unsigned)bhn, kBwdThreads, L::bytes, stream>>>(a);
-    return cudaGetLastError();
+    const size_t bhn = (size_t)x.B * x.H;
+    a.rows = bhn * x.T;
+    a.check = ws + w.check; a.scratch = ws + w.scratch;
+    a.dq_p = ws + w.dq; a.dk_p = ws + w.dk; a.dalpha_p = ws + w.dalpha; a.dtheta_p = ws + w.dtheta; a.dbeta_p = ws + w.dbeta;
+    kern<<<dim3((unsigned)bhn, NSL), kBwdThreads, L::bytes, stream>>>(a);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if (launches) ++*launches;
+    if constexpr (NSL > 1) {
+        const size_t n_key = a.rows * DK, n_coord = a.rows * (DK / 2);
+        const size_t items = n_key / 2 + n_coord / 2 + a.rows;
+        size_t blocks = (items + kSumThreads - 1) / kSumThreads;
+        if (blocks > 148 * 8 * 8) blocks = 148 * 8 * 8;
+        sfda_backward_sum_kernel<NSL, T><<<(unsigned)blocks, kSumThreads, 0, stream>>>(
+            a.dq_p, a.dk_p, a.dalpha_p, a.dtheta_p, a.dbeta_p, static_cast<T *>(x.dq), static_cast<T *>(x.dk), x.dalpha,
+            x.dtheta, x.dbeta, n_key, n_coord, a.rows);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        if (launches) ++*launches;
+    }
+    return cudaSuccess;
+}
+
+template <int DK, int DV, typename T>
+cudaError_t launch_typed(const BackwardArgs &x, void *workspace, cudaStream_t stream, int *launches)
+{
+    const int cols = bwd_cols(x.B, x.H, DV);
+    if (cols == DV) return launch_cols<DK, DV, DV, T>(x, workspace, stream, launches);
+    if constexpr (DV > 64) {
+        if (cols == 64) return launch_cols<DK, DV, 64, T>(x, workspace, stream, launches);
+    }
+    return launch_cols<DK, DV, 32, T>(x, workspace, stream, launches);
 }
 
 }  // namespace
 
 size_t backward_workspace_bytes(int B, int T, int H, int d_k, int d_v)
 {
-    const size_t ns = (size_t)(T + kSeg - 1) / kSeg;
-    return (size_t)B * H * (ns + kSeg) * d_k * d_v * sizeof(float);
+    return bwd_workspace(B, T, H, d_k, d_v).total * sizeof(float);
 }
 
 cudaError_t launch_backward(const BackwardArgs &a, void *workspace, cudaStream_t stream, int *launches)
 {
     cudaError_t e = cudaErrorInvalidValue;
     if (a.dtype == 1) {
-        if (a.d_k == 128 && a.d_v == 128) e = launch_typed<128, 128, __nv_bfloat16>(a, workspace, stream);
-        else if (a.d_k == 128 && a.d_v == 64) e = launch_typed<128, 64, __nv_bfloat16>(a, workspace, stream);
-        else if (a.d_k == 64 && a.d_v == 128) e = launch_typed<64, 128, __nv_bfloat16>(a, workspace, stream);
-        else if (a.d_k == 64 && a.d_v == 64) e = launch_typed<64, 64, __nv_bfloat16>(a, workspace, stream);
+        if (a.d_k == 128 && a.d_v == 128) e = launch_typed<128, 128, __nv_bfloat16>(a, workspace, stream, launches);
+        else if (a.d_k == 128 && a.d_v == 64) e = launch_typed<128, 64, __nv_bfloat16>(a, workspace, stream, launches);
+        else if (a.d_k == 64 && a.d_v == 128) e = launch_typed<64, 128, __nv_bfloat16>(a, workspace, stream, launches);
+        else if (a.d_k == 64 && a.d_v == 64) e = launch_typed<64, 64, __nv_bfloat16>(a, workspace, stream, launches);
     } else {
-        if (a.d_k == 128 && a.d_v == 128) e = launch_typed<128, 128, float>(a, workspace, stream);
-        else if (a.d_k == 128 && a.d_v == 64) e = launch_typed<128, 64, float>(a, workspace, stream);
-        else if (a.d_k == 64 && a.d_v == 128) e = launch_typed<64, 128, float>(a, workspace, stream);
-        else if (a.d_k == 64 && a.d_v == 64) e = launch_typed<64, 64, float>(a, workspace, stream);
+        if (a.d_k == 128 && a.d_v == 128) e = launch_typed<128, 128, float>(a, workspace, stream, launches);
+        else if (a.d_k == 128 && a.d_v == 64) e = launch_typed<128, 64, float>(a, workspace, stream, launches);
+        else if (a.d_k == 64 && a.d_v == 128) e = launch_typed<64, 128, float>(a, workspace, stream, launches);
+        else if (a.d_k == 64 && a.d_v == 64) e = launch_typed<64, 64, float>(a, workspace, stream, launches);
     }
-    if (e == cudaSuccess && launches) ++*launches;
     return e;
 }
 

@@ -195,7 +195,11 @@ def test_backward_entry_point_validates_on_the_host(lib):
     assert bwd(ptrs, [1, 100, 2, 128, 128, 3]) == -3
     assert bwd(ptrs[:7] + [vp(0x1004)] + ptrs[8:], dims) == -4
     need = sfda.sfda_backward_workspace_bytes(1, 100, 2, 128, 128, 1)
-    assert need == 1 * 2 * (2 + 64) * 128 * 128 * 4                  # 2 checkpoints + 64 states per (batch, head)
+    # 2 checkpoints + 64 states per (batch, head); two sequences split the columns into 4 blocks of 32, each with
+    # its shares of dq, dk (128 each), dalpha, dtheta (64 each) and dbeta of the 200 (token, head) rows
+    assert need == (1 * 2 * (2 + 64) * 128 * 128 + 4 * 200 * (3 * 128 + 1)) * 4
+    # many sequences: one block, no shares
+    assert sfda.sfda_backward_workspace_bytes(8, 128, 32, 128, 128, 1) == 8 * 32 * (2 + 64) * 128 * 128 * 4
     assert bwd(ptrs, dims, ws_bytes=need - 1) == -5
     assert bwd(ptrs, dims, ws=None, ws_bytes=0) == -5
     assert sfda.sfda_backward_workspace_bytes(1, 100, 2, 100, 128, 1) == 0

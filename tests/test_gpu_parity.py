@@ -660,14 +660,24 @@ def run_backward(cfg, inp, up):
                dbeta=torch.empty_like(d["beta"]),
                dS0=torch.empty(B, H, cfg.d_k, cfg.d_v, device=DEV, dtype=torch.float32))
     n = sfda.sfda_backward_workspace_bytes(B, T, H, cfg.d_k, cfg.d_v, 1 if cfg.dtype == "bf16" else 0)
-    assert n == B * H * ((T + 63) // 64 + 64) * cfg.d_k * cfg.d_v * 4
+    blocks = backward_column_blocks(B, H, cfg.d_v)
+    shares = blocks * B * T * H if blocks > 1 else 0
+    assert n == (B * H * ((T + 63) // 64 + 64) * cfg.d_k * cfg.d_v + shares * 3 * cfg.d_k + (shares + 3) // 4 * 4) * 4
     ws = torch.empty(n, device=DEV, dtype=torch.uint8)
     sfda.sfda_backward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], u["do_re"], u["do_im"],
                        u["dS_T"], out["dq"], out["dk"], out["dv"], out["dalpha"], out["dtheta"], out["dbeta"],
                        out["dS0"], ws)
     torch.cuda.synchronize()
-    assert sfda.last_launch_count() == 1
+    assert sfda.last_launch_count() == (2 if blocks > 1 else 1)   # the sweeps, then the sum of the blocks' shares
     return {k: v.float().cpu().numpy() for k, v in out.items()}
+
+
+def backward_column_blocks(B, H, d_v):
+    """Column blocks per state: the value columns are halved (down to 32 per CTA) while the grid fits 148 SMs."""
+    cols = d_v
+    while cols > 32 and B * H * (d_v // (cols // 2)) <= 148:
+        cols //= 2
+    return d_v // cols
 
 
 def upstream(cfg, seed, want_im=True, want_state=True):
@@ -705,6 +715,16 @@ def test_backward_matches_oracle(d_k, d_v, T, dtype):
     inp = workloads.forward_inputs(cfg)
     # fp32 arithmetic; bf16 storage rounds the stored dq, dk, dv once (2^-9 relative)
     check_backward(cfg, inp, upstream(cfg, T), all_pairs(cfg), 1e-4 if dtype == "f32" else 5e-3)
+
+
+@pytest.mark.parametrize("B,H,d_v,blocks", [(5, 8, 128, 2), (19, 8, 128, 1), (10, 8, 64, 1), (3, 3, 64, 2)])
+def test_backward_column_blocks(B, H, d_v, blocks):
+    """Few sequences split the value columns over more CTAs (shares summed by a second kernel); many do not."""
+    assert backward_column_blocks(B, H, d_v) == blocks
+    cfg = workloads.CONFIGS[0].scaled(name="bwd_blocks", B=B, T=70, H=H, d_k=64, d_v=d_v, dtype="bf16", s0_std=0.5,
+                                      seed=85 + B)
+    inp = workloads.forward_inputs(cfg)
+    check_backward(cfg, inp, upstream(cfg, B), [(0, 0), (B - 1, H - 1), (B // 2, 1)], 5e-3)
 
 
 def test_backward_optional_cotangents_and_zero_state():
