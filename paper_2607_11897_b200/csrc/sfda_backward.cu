@@ -6,7 +6,10 @@
 //
 //   1. forward, keeping the state at the start of every segment of kSeg tokens (checkpoints in the workspace);
 //   2. per segment, last to first: forward again from the checkpoint, keeping S_{t-1} of every token of the segment;
-//   3. backward through the segment with the cotangent G of the state in shared memory.
+//   3. backward through the segment.
+//
+// The state (sweeps 1, 2) and its cotangent G (sweep 3) live in registers, a tile of rows x columns per thread;
+// S_{t-1} of the backward step arrives from the scratch by cp.async, one token ahead.
 //
 // One backward step, with Z = Lambda_t S_{t-1}, u^T = v_t^T - k_t^* Z (so S_t = Z + beta_t k_t u^T) and
 // yb_t = do_re + i do_im:
@@ -29,14 +32,20 @@ namespace {
 constexpr int kBwdThreads = 512;
 constexpr int kSeg = 64;     // tokens between checkpoints
 
+// Thread mapping: warp w owns TR consecutive rows of the (complex) state, lane l owns TC consecutive value columns,
+// so a thread keeps a TR x TC tile of the cotangent G -- and of the state, while a step needs it -- in registers.
+// Sums over rows (per column) cross the warps through shared memory; sums over columns (per row) stay inside a warp.
 template <int DK, int DV>
 struct BwdSmem {
-    static constexpr int M = DK / 2;
-    static constexpr int RS = DV + 8;            // row stride in complex (float2) elements: rows 16 banks apart
-    static constexpr int NG = kBwdThreads / DV;  // row groups of the column-owner mapping
-    static constexpr int plane = M * RS;         // floats in half a state buffer
-    // G and two buffers of S_{t-1} as interleaved complex [M][RS], and the vectors of one token
-    static constexpr size_t bytes = (size_t)(6 * plane + 8 * M + 7 * DV + NG * 4 * DV + 64) * 4;
+    static constexpr int M = DK / 2, NW = kBwdThreads / 32;
+    static constexpr int TR = M / NW, TC = DV / 32;
+    static_assert(M % NW == 0 && DV % 32 == 0 && (TC == 1 || TC == 2 || TC == 4), "tile shape");
+    // two buffers of S_{t-1} (interleaved complex [M][DV]), the warps' partial column sums [NW][DV] float4, two
+    // sets of token vectors (row vectors 2 float4 [M], column vectors float2 + float [DV], beta), and the
+    // per-column results of a step (p, u / e: 2 float2 [DV]) with the warps' scalar sums
+    static constexpr int state = M * DV * 2;                           // floats
+    static constexpr int tokvec = 8 * M + 3 * DV + 4;                  // floats, one set
+    static constexpr size_t bytes = (size_t)(2 * state + NW * DV * 4 + 2 * tokvec + 4 * DV + 64) * 4;
 };
 
 __device__ __forceinline__ void cp_async16(float *dst_smem, const float *src)
@@ -45,6 +54,33 @@ __device__ __forceinline__ void cp_async16(float *dst_smem, const float *src)
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
+// N consecutive float2 (N = 1, 2, 4) with the widest accesses; p is aligned to 8 N bytes (16 for N = 4)
+template <int N>
+__device__ __forceinline__ void ld_row(const float2 *p, float2 (&x)[N])
+{
+    if constexpr (N == 1) {
+        x[0] = *p;
+    } else {
+#pragma unroll
+        for (int i = 0; i < N / 2; ++i) {
+            const float4 t = reinterpret_cast<const float4 *>(p)[i];
+            x[2 * i] = make_float2(t.x, t.y);
+            x[2 * i + 1] = make_float2(t.z, t.w);
+        }
+    }
+}
+template <int N>
+__device__ __forceinline__ void st_row(float2 *p, const float2 (&x)[N])
+{
+    if constexpr (N == 1) {
+        *p = x[0];
+    } else {
+#pragma unroll
+        for (int i = 0; i < N / 2; ++i)
+            reinterpret_cast<float4 *>(p)[i] = make_float4(x[2 * i].x, x[2 * i].y, x[2 * i + 1].x, x[2 * i + 1].y);
+    }
+}
 
 struct BwdArgsDev {
     const void *q, *k, *v, *d_o, *d_o_im;
@@ -63,25 +99,25 @@ __global__ void __launch_bounds__(kBwdThreads, 1)
 sfda_backward_kernel(const BwdArgsDev a)
 {
     constexpr int NSL = DVT / DV;                  // column blocks per state
-    static_assert(DVT % DV == 0 && DV % 32 == 0, "the value columns split into blocks of whole warps");
+    static_assert(DVT % DV == 0, "the value columns split into equal blocks");
     using L = BwdSmem<DK, DV>;
-    constexpr int M = L::M, RS = L::RS, NG = L::NG, RA = M / NG;      // RA rows per thread in the column mapping
-    constexpr int TPR = kBwdThreads / M, CPT = DV / TPR;               // threads per row / columns per thread (row mapping)
-    static_assert(M % NG == 0 && DV % TPR == 0 && M + DV + 1 <= kBwdThreads, "thread mappings");
+    constexpr int M = L::M, NW = L::NW, TR = L::TR, TC = L::TC;
+    static_assert(M + DV + 1 <= kBwdThreads, "one thread per staged value");
     extern __shared__ __align__(16) float sm[];
-    float2 *G = reinterpret_cast<float2 *>(sm);            // cotangent of the state, complex [M][RS]
-    float *P0 = sm + 2 * L::plane;                          // two buffers of the same shape for S / S_{t-1}
-    auto Pb = [&](int i) { return reinterpret_cast<float2 *>(P0 + i * 2 * L::plane); };
-    // per-row vectors of the token, packed so that one (broadcast) load fetches all a step needs of a row:
-    // (lam re, lam im, k re, k im), (q re, q im, cos theta, sin theta); per-column vectors likewise:
-    // (yb re, yb im, u re, u im), (p re, p im), v
-    float4 *v_lk = reinterpret_cast<float4 *>(P0 + 4 * L::plane);
-    float4 *v_qc = v_lk + M;
-    float4 *v_yu = v_qc + M;
-    float2 *v_p = reinterpret_cast<float2 *>(v_yu + DV);
-    float *v_v = reinterpret_cast<float *>(v_p + DV);
-    float *red = v_v + DV;                      // [NG][4][DV]
-    float *scal = red + NG * 4 * DV;            // [0] beta, [8 + 4 w + x] partial sums of warp w
+    float2 *const Sbuf0 = reinterpret_cast<float2 *>(sm);                        // S_{t-1}, two buffers [M][DV]
+    float4 *const red = reinterpret_cast<float4 *>(sm + 2 * L::state);           // [NW][DV] partial column sums
+    float *const tok0 = sm + 2 * L::state + NW * DV * 4;                         // two sets of token vectors
+    float2 *const v_p = reinterpret_cast<float2 *>(tok0 + 2 * L::tokvec);        // p per column (backward)
+    float2 *const v_u = v_p + DV;                                                // u (backward) / e = beta u (forward)
+    float *const scal = reinterpret_cast<float *>(v_u + DV);                     // [4 w + x]: scalar sums of warp w
+    auto Sbuf = [&](int i) { return Sbuf0 + i * (M * DV); };
+    // token vectors of set i: per row (lam re, lam im, k re, k im), (q re, q im, cos theta, sin theta); per column
+    // yb (re, im) and v; beta
+    auto t_lk = [&](int i) { return reinterpret_cast<float4 *>(tok0 + i * L::tokvec); };
+    auto t_qc = [&](int i) { return reinterpret_cast<float4 *>(tok0 + i * L::tokvec) + M; };
+    auto t_y = [&](int i) { return reinterpret_cast<float2 *>(tok0 + i * L::tokvec + 8 * M); };
+    auto t_v = [&](int i) { return tok0 + i * L::tokvec + 8 * M + 2 * DV; };
+    auto t_beta = [&](int i) { return tok0 + i * L::tokvec + 8 * M + 3 * DV; };
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bh = blockIdx.x, h = bh % a.H, b = bh / a.H, slice = blockIdx.y, c0 = slice * DV;
@@ -90,126 +126,143 @@ sfda_backward_kernel(const BwdArgsDev a)
     const T *d_o = static_cast<const T *>(a.d_o), *d_oi = static_cast<const T *>(a.d_o_im);
     float *check = a.check + ((size_t)bh * NSL + slice) * a.NS * 2 * M * DV;
     float *scratch = a.scratch + ((size_t)bh * NSL + slice) * kSeg * 2 * M * DV;
+    const int j0 = warp * TR, cl = lane * TC;      // this thread's tile: rows j0 + r, columns cl + x
 
-    // column-owner mapping (A): column c, rows g, g + NG, ...;  row-owner mapping (B): row jb, columns part + TPR n
-    const int c = tid % DV, g = tid / DV;
-    const int jb = tid / TPR, part = tid % TPR;
-
-    // ---- token vectors: registers -> shared memory, one token ahead of the step that uses them
+    // ---- token vectors: global -> registers (issued a step ahead) -> one of the two sets in shared memory
+    // (staged by the last M + DV + 1 threads: the first DV are the ones that reduce the column sums meanwhile)
+    const int sid = kBwdThreads - 1 - tid;
     float r0 = 0.f, r1 = 0.f, r2 = 0.f, r3 = 0.f, r4 = 0.f, r5 = 0.f;
     auto load_tok = [&](int t, bool back) {
         if (t < 0 || t >= T_) return;
         const size_t row = ((size_t)b * T_ + t) * H + h;
-        if (tid < M) {
-            r0 = a.alpha[row * M + tid];
-            r1 = a.theta[row * M + tid];
-            r2 = ld_val(k, row * DK + 2 * tid);
-            r3 = ld_val(k, row * DK + 2 * tid + 1);
+        if (sid < M) {
+            r0 = a.alpha[row * M + sid];
+            r1 = a.theta[row * M + sid];
+            r2 = ld_val(k, row * DK + 2 * sid);
+            r3 = ld_val(k, row * DK + 2 * sid + 1);
             if (back) {
-                r4 = ld_val(q, row * DK + 2 * tid);
-                r5 = ld_val(q, row * DK + 2 * tid + 1);
+                r4 = ld_val(q, row * DK + 2 * sid);
+                r5 = ld_val(q, row * DK + 2 * sid + 1);
             }
-        } else if (tid < M + DV) {
-            const int cc = tid - M;
+        } else if (sid < M + DV) {
+            const int cc = sid - M;
             r0 = ld_val(v, row * DVT + c0 + cc);
             if (back) {
                 r1 = ld_val(d_o, row * DVT + c0 + cc);
                 r2 = d_oi ? ld_val(d_oi, row * DVT + c0 + cc) : 0.f;
             }
-        } else if (tid == M + DV) {
+        } else if (sid == M + DV) {
             r0 = a.beta[row];
         }
     };
-    auto stage_tok = [&](bool back) {
-        if (tid < M) {
+    auto stage_tok = [&](int set, bool back) {
+        if (sid < M) {
             float sn, cs;
             sincosf(r1, &sn, &cs);
-            v_lk[tid] = make_float4(r0 * cs, r0 * sn, r2, r3);
-            if (back) v_qc[tid] = make_float4(r4, r5, cs, sn);
-        } else if (tid < M + DV) {
-            const int cc = tid - M;
-            v_v[cc] = r0;
-            if (back) v_yu[cc] = make_float4(r1, r2, 0.f, 0.f);
-        } else if (tid == M + DV) {
-            scal[0] = r0;
+            t_lk(set)[sid] = make_float4(r0 * cs, r0 * sn, r2, r3);
+            if (back) t_qc(set)[sid] = make_float4(r4, r5, cs, sn);
+        } else if (sid < M + DV) {
+            const int cc = sid - M;
+            t_v(set)[cc] = r0;
+            if (back) t_y(set)[cc] = make_float2(r1, r2);
+        } else if (sid == M + DV) {
+            t_beta(set)[0] = r0;
         }
     };
 
-    // ---- one forward step on the state S; the token's vectors are staged and synchronised
-    auto fwd_step = [&](float2 *S) {
-        float cr = 0.f, ci = 0.f, zr[RA], zi[RA];
+    // ---- one forward step on the tile s (registers).  Set `set` holds the token's vectors (visible to all); the
+    // next token's vectors, already in registers, are staged into the other set on the way.
+    auto fwd_step = [&](float2 (&s)[TR][TC], int set, bool stage_next) {
+        const float4 *lkv = t_lk(set);
+        float2 kz[TC];
 #pragma unroll
-        for (int r = 0; r < RA; ++r) {
-            const int j = g + NG * r;
-            const float4 lk = v_lk[j];
-            const float2 sv = S[j * RS + c];
-            zr[r] = lk.x * sv.x - lk.y * sv.y;                                 // Z = Lambda S
-            zi[r] = lk.x * sv.y + lk.y * sv.x;
-            cr += lk.z * zr[r] + lk.w * zi[r];                                 // conj(k) z
-            ci += lk.z * zi[r] - lk.w * zr[r];
+        for (int x = 0; x < TC; ++x) kz[x] = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int r = 0; r < TR; ++r) {
+            const float4 lk = lkv[j0 + r];
+#pragma unroll
+            for (int x = 0; x < TC; ++x) {
+                const float zr = lk.x * s[r][x].x - lk.y * s[r][x].y, zi = lk.x * s[r][x].y + lk.y * s[r][x].x;   // Z = Lambda S
+                s[r][x] = make_float2(zr, zi);
+                kz[x].x += lk.z * zr + lk.w * zi;                                  // conj(k) z
+                kz[x].y += lk.z * zi - lk.w * zr;
+            }
         }
-        red[(g * 4 + 0) * DV + c] = cr;
-        red[(g * 4 + 1) * DV + c] = ci;
+#pragma unroll
+        for (int x = 0; x < TC; ++x) reinterpret_cast<float2 *>(red)[(warp * TC + x) * 32 + lane] = kz[x];
         __syncthreads();
-        float sr_ = 0.f, si_ = 0.f;
+        if (tid < DV) {                     // warp x' of these sums column x' of every lane's tile
+            const int c = lane * TC + warp;
+            float sr_ = 0.f, si_ = 0.f;
 #pragma unroll
-        for (int gg = 0; gg < NG; ++gg) {
-            sr_ += red[(gg * 4 + 0) * DV + c];
-            si_ += red[(gg * 4 + 1) * DV + c];
+            for (int w = 0; w < NW; ++w) {
+                const float2 x = reinterpret_cast<const float2 *>(red)[(w * TC + warp) * 32 + lane];
+                sr_ += x.x;
+                si_ += x.y;
+            }
+            const float bt = t_beta(set)[0];
+            v_u[c] = make_float2(bt * (t_v(set)[c] - sr_), -bt * si_);              // e = beta u, u = v - k^* Z
         }
-        const float bt = scal[0];
-        const float er = bt * (v_v[c] - sr_), ei = -bt * si_;                  // e = beta u, u = v - k^* Z
-#pragma unroll
-        for (int r = 0; r < RA; ++r) {
-            const int j = g + NG * r;
-            const float4 lk = v_lk[j];
-            S[j * RS + c] = make_float2(zr[r] + lk.z * er - lk.w * ei, zi[r] + lk.z * ei + lk.w * er);
-        }
+        if (stage_next) stage_tok(set ^ 1, false);
         __syncthreads();
+        float2 e[TC];
+        ld_row<TC>(v_u + cl, e);
+#pragma unroll
+        for (int r = 0; r < TR; ++r) {
+            const float4 lk = lkv[j0 + r];
+#pragma unroll
+            for (int x = 0; x < TC; ++x) {
+                s[r][x].x += lk.z * e[x].x - lk.w * e[x].y;
+                s[r][x].y += lk.z * e[x].y + lk.w * e[x].x;
+            }
+        }
     };
 
-    // ---- state moves between shared and global memory (workspace format: interleaved complex [M][DV]), 16 bytes
-    // = two elements per access
-    auto store_state = [&](const float2 *S, float *dst) {
-        for (int idx = tid; idx < M * DV / 2; idx += kBwdThreads) {
-            const int j = idx / (DV / 2), c2 = idx % (DV / 2);
-            *reinterpret_cast<float4 *>(dst + ((size_t)j * DV + 2 * c2) * 2) = *reinterpret_cast<const float4 *>(S + j * RS + 2 * c2);
-        }
+    // ---- a tile between registers and global memory (workspace format: interleaved complex [M][DV])
+    auto store_tile = [&](const float2 (&s)[TR][TC], float *dst) {
+#pragma unroll
+        for (int r = 0; r < TR; ++r) st_row<TC>(reinterpret_cast<float2 *>(dst) + (size_t)(j0 + r) * DV + cl, s[r]);
+    };
+    auto load_tile = [&](float2 (&s)[TR][TC], const float *src) {
+#pragma unroll
+        for (int r = 0; r < TR; ++r) ld_row<TC>(reinterpret_cast<const float2 *>(src) + (size_t)(j0 + r) * DV + cl, s[r]);
     };
     auto load_state_async = [&](float2 *S, const float *src) {
-        for (int idx = tid; idx < M * DV / 2; idx += kBwdThreads) {
-            const int j = idx / (DV / 2), c2 = idx % (DV / 2);
-            cp_async16(reinterpret_cast<float *>(S + j * RS + 2 * c2), src + ((size_t)j * DV + 2 * c2) * 2);
-        }
+        for (int idx = tid; idx < M * DV / 2; idx += kBwdThreads) cp_async16(reinterpret_cast<float *>(S) + 4 * idx, src + 4 * idx);
         cp_async_commit();
     };
 
     // ---- sweep 1: forward, checkpoints at the start of every segment (nothing is needed beyond the last one)
-    float2 *S = Pb(0);
-    for (int idx = tid; idx < M * DV; idx += kBwdThreads) {
-        const int j = idx / DV, cc = idx % DV;
-        S[j * RS + cc] = a.S0 ? make_float2(a.S0[((size_t)bh * DK + 2 * j) * DVT + c0 + cc], a.S0[((size_t)bh * DK + 2 * j + 1) * DVT + c0 + cc])
-                              : make_float2(0.f, 0.f);
-    }
+    float2 s[TR][TC];
+#pragma unroll
+    for (int r = 0; r < TR; ++r)
+#pragma unroll
+        for (int x = 0; x < TC; ++x) {
+            const size_t at = ((size_t)bh * DK + 2 * (j0 + r)) * DVT + c0 + cl + x;
+            s[r][x] = a.S0 ? make_float2(a.S0[at], a.S0[at + DVT]) : make_float2(0.f, 0.f);
+        }
     const int t_last_check = (a.NS - 1) * kSeg;
+    int set = 0;
     load_tok(0, false);
+    stage_tok(set, false);
     __syncthreads();
     for (int t = 0; t < t_last_check; ++t) {
-        if (t % kSeg == 0) store_state(S, check + (size_t)(t / kSeg) * 2 * M * DV);
-        stage_tok(false);
-        __syncthreads();
+        if (t % kSeg == 0) store_tile(s, check + (size_t)(t / kSeg) * 2 * M * DV);
         load_tok(t + 1, false);
-        fwd_step(S);
+        fwd_step(s, set, true);
+        set ^= 1;
     }
-    store_state(S, check + (size_t)(a.NS - 1) * 2 * M * DV);
+    store_tile(s, check + (size_t)(a.NS - 1) * 2 * M * DV);
 
     // ---- cotangent of the final state
-    for (int idx = tid; idx < M * DV; idx += kBwdThreads) {
-        const int j = idx / DV, cc = idx % DV;
-        G[j * RS + cc] = a.dS_T ? make_float2(a.dS_T[((size_t)bh * DK + 2 * j) * DVT + c0 + cc], a.dS_T[((size_t)bh * DK + 2 * j + 1) * DVT + c0 + cc])
-                                : make_float2(0.f, 0.f);
-    }
-    __syncthreads();      // also: every thread's checkpoint stores precede the loads below (same CTA, after a barrier)
+    float2 G[TR][TC];
+#pragma unroll
+    for (int r = 0; r < TR; ++r)
+#pragma unroll
+        for (int x = 0; x < TC; ++x) {
+            const size_t at = ((size_t)bh * DK + 2 * (j0 + r)) * DVT + c0 + cl + x;
+            G[r][x] = a.dS_T ? make_float2(a.dS_T[at], a.dS_T[at + DVT]) : make_float2(0.f, 0.f);
+        }
 
     T *dq = static_cast<T *>(a.dq), *dk = static_cast<T *>(a.dk), *dv = static_cast<T *>(a.dv);
     float *dq_p = a.dq_p + (size_t)slice * a.rows * DK, *dk_p = a.dk_p + (size_t)slice * a.rows * DK;
@@ -217,152 +270,188 @@ sfda_backward_kernel(const BwdArgsDev a)
     float *dbe_p = a.dbeta_p + (size_t)slice * a.rows;
     for (int si = a.NS - 1; si >= 0; --si) {
         const int t0 = si * kSeg, t1 = min(t0 + kSeg, T_);
-        // ---- sweep 2: forward again from the checkpoint, S_{t-1} of every token to the scratch
-        load_state_async(S, check + (size_t)si * 2 * M * DV);
+        // ---- sweep 2: forward again from the checkpoint (this thread wrote the tile it reads), S_{t-1} of every
+        // token to the scratch
+        __syncthreads();                  // every reader of the token vectors and of v_u is done
+        load_tile(s, check + (size_t)si * 2 * M * DV);
+        set = 0;
         load_tok(t0, false);
-        cp_async_wait_all();
+        stage_tok(set, false);
         __syncthreads();
         for (int t = t0; t < t1; ++t) {
-            store_state(S, scratch + (size_t)(t - t0) * 2 * M * DV);
-            stage_tok(false);
-            __syncthreads();
-            load_tok(t + 1 < t1 ? t + 1 : t1 - 1, t + 1 >= t1);     // after the last one: the first backward token
-            if (t + 1 < t1) fwd_step(S);                        // the state after the last token is not needed
+            store_tile(s, scratch + (size_t)(t - t0) * 2 * M * DV);
+            if (t + 1 < t1) {                                   // the state after the last token is not needed
+                load_tok(t + 1, false);
+                fwd_step(s, set, true);
+                set ^= 1;
+            }
         }
         __syncthreads();      // the scratch stores of this CTA are visible to its own later loads
 
         // ---- sweep 3: backward through the segment; S_{t-1} arrives one token ahead in the other buffer
         int buf = 0;
-        load_state_async(Pb(buf), scratch + (size_t)(t1 - 1 - t0) * 2 * M * DV);
+        set = 0;
+        load_state_async(Sbuf(buf), scratch + (size_t)(t1 - 1 - t0) * 2 * M * DV);
+        load_tok(t1 - 1, true);
+        stage_tok(set, true);
+        cp_async_wait_all();
+        __syncthreads();
         for (int t = t1 - 1; t >= t0; --t) {
-            stage_tok(true);
-            cp_async_wait_all();
-            __syncthreads();
-            const float2 *Q = Pb(buf);
-            if (t > t0) load_state_async(Pb(buf ^ 1), scratch + (size_t)(t - 1 - t0) * 2 * M * DV);
-            load_tok(t - 1 >= t0 ? t - 1 : t0 - 1, true);           // (a token of the next segment down is reloaded there)
-            const float bt = scal[0];
+            if (t > t0) {
+                load_state_async(Sbuf(buf ^ 1), scratch + (size_t)(t - 1 - t0) * 2 * M * DV);
+                load_tok(t - 1, true);
+            }
+            const float4 *lkv = t_lk(set), *qcv = t_qc(set);
+            const float bt = t_beta(set)[0];
             const size_t row = ((size_t)b * T_ + t) * H + h;
+            float2 y[TC];
+            ld_row<TC>(t_y(set) + cl, y);
 
-            // step 1 (columns): partial p = (G + q yb^*)^* k and k^* Z  (G itself is updated in step 3)
+            // step 1: G += q yb^*; partial sums over this warp's rows of p = G^* k and k^* Z
             {
-                const float4 yu = v_yu[c];
-                const float yr = yu.x, yi = yu.y;
-                float pr = 0.f, pi = 0.f, zr_ = 0.f, zi_ = 0.f;
+                float4 acc[TC];
 #pragma unroll
-                for (int r = 0; r < RA; ++r) {
-                    const int j = g + NG * r;
-                    const float4 lk = v_lk[j], qc = v_qc[j];
-                    const float2 gv = G[j * RS + c];
-                    const float gr = gv.x + qc.x * yr + qc.y * yi;              // G + q conj(yb)
-                    const float gi = gv.y + qc.y * yr - qc.x * yi;
-                    pr += gr * lk.z + gi * lk.w;                                // conj(G) k
-                    pi += gr * lk.w - gi * lk.z;
-                    const float2 sv = Q[j * RS + c];
-                    const float zr = lk.x * sv.x - lk.y * sv.y, zi = lk.x * sv.y + lk.y * sv.x;
-                    zr_ += lk.z * zr + lk.w * zi;                               // conj(k) z
-                    zi_ += lk.z * zi - lk.w * zr;
+                for (int x = 0; x < TC; ++x) acc[x] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int r = 0; r < TR; ++r) {
+                    const float4 lk = lkv[j0 + r], qc = qcv[j0 + r];
+                    ld_row<TC>(Sbuf(buf) + (j0 + r) * DV + cl, s[r]);
+#pragma unroll
+                    for (int x = 0; x < TC; ++x) {
+                        const float gr = G[r][x].x + qc.x * y[x].x + qc.y * y[x].y;          // G + q conj(yb)
+                        const float gi = G[r][x].y + qc.y * y[x].x - qc.x * y[x].y;
+                        G[r][x] = make_float2(gr, gi);
+                        acc[x].x += gr * lk.z + gi * lk.w;                                  // conj(G) k
+                        acc[x].y += gr * lk.w - gi * lk.z;
+                        const float zr = lk.x * s[r][x].x - lk.y * s[r][x].y, zi = lk.x * s[r][x].y + lk.y * s[r][x].x;
+                        acc[x].z += lk.z * zr + lk.w * zi;                                  // conj(k) z
+                        acc[x].w += lk.z * zi - lk.w * zr;
+                    }
                 }
-                red[(g * 4 + 0) * DV + c] = pr;
-                red[(g * 4 + 1) * DV + c] = pi;
-                red[(g * 4 + 2) * DV + c] = zr_;
-                red[(g * 4 + 3) * DV + c] = zi_;
+#pragma unroll
+                for (int x = 0; x < TC; ++x) red[(warp * TC + x) * 32 + lane] = acc[x];     // [warp][x][lane]: no bank conflicts
             }
             __syncthreads();
-            // step 2: p, u per column; dv; the sums over columns u^T p and u^T yb
-            if (tid < DV) {
+            // step 2: p, u per column; dv; the sums over columns u^T p and u^T yb (one set per warp of columns)
+            if (tid < DV) {                 // warp x' of these sums column x' of every lane's tile
+                const int c = lane * TC + warp;
                 float pr = 0.f, pi = 0.f, zr = 0.f, zi = 0.f;
 #pragma unroll
-                for (int gg = 0; gg < NG; ++gg) {
-                    pr += red[(gg * 4 + 0) * DV + c];
-                    pi += red[(gg * 4 + 1) * DV + c];
-                    zr += red[(gg * 4 + 2) * DV + c];
-                    zi += red[(gg * 4 + 3) * DV + c];
+                for (int w = 0; w < NW; ++w) {
+                    const float4 x = red[(w * TC + warp) * 32 + lane];
+                    pr += x.x;  pi += x.y;  zr += x.z;  zi += x.w;
                 }
-                const float ur = v_v[c] - zr, ui = -zi;
-                const float4 yu = v_yu[c];
-                const float yr = yu.x, yi = yu.y;
+                const float ur = t_v(set)[c] - zr, ui = -zi;
+                const float2 yy = t_y(set)[c];
                 v_p[c] = make_float2(pr, pi);
-                v_yu[c] = make_float4(yr, yi, ur, ui);
+                v_u[c] = make_float2(ur, ui);
                 st_val(dv, row * DVT + c0 + c, bt * pr);
-                float s0 = ur * pr - ui * pi;                       // Re(u p)
-                float s1 = ur * yr - ui * yi, s2 = ur * yi + ui * yr;   // u yb
+                float s0 = ur * pr - ui * pi;                                   // Re(u p)
+                float s1 = ur * yy.x - ui * yy.y, s2 = ur * yy.y + ui * yy.x;   // u yb
 #pragma unroll
                 for (int d = 16; d >= 1; d >>= 1) {
                     s0 += __shfl_xor_sync(0xffffffffu, s0, d);
                     s1 += __shfl_xor_sync(0xffffffffu, s1, d);
                     s2 += __shfl_xor_sync(0xffffffffu, s2, d);
                 }
-                if (lane == 0) { scal[8 + 4 * warp] = s0; scal[9 + 4 * warp] = s1; scal[10 + 4 * warp] = s2; }
+                if (lane == 0) { scal[4 * warp] = s0; scal[4 * warp + 1] = s1; scal[4 * warp + 2] = s2; }
             }
+            if (t > t0) stage_tok(set ^ 1, true);
+            cp_async_wait_all();
             __syncthreads();
-            // step 3 (rows): dq, dk, lamb, and G <- conj(lam) (G - beta k p^*)
+            // step 3: this warp's rows: shares of dq, dk, dalpha, dtheta; G <- conj(lam) (G - beta k p^*)
             {
-                float sr_ = 0.f, si_ = 0.f, dbe = 0.f;
+                float uy_r = 0.f, uy_i = 0.f, dbe = 0.f;
 #pragma unroll
-                for (int w = 0; w < DV / 32; ++w) { dbe += scal[8 + 4 * w]; sr_ += scal[9 + 4 * w]; si_ += scal[10 + 4 * w]; }
+                for (int w = 0; w < DV / 32; ++w) { dbe += scal[4 * w]; uy_r += scal[4 * w + 1]; uy_i += scal[4 * w + 2]; }
                 if (tid == 0) (NSL == 1 ? a.dbeta : dbe_p)[row] = dbe;
-                const int j = jb;
-                const float4 lk = v_lk[j], qc = v_qc[j];
-                const float lr = lk.x, li = lk.y, kr = lk.z, ki = lk.w;
-                float qzr = 0.f, qzi = 0.f, k1r = 0.f, k1i = 0.f, k2r = 0.f, k2i = 0.f, lbr = 0.f, lbi = 0.f;
-#pragma unroll 4
-                for (int n = 0; n < CPT; ++n) {
-                    const int cc = part + TPR * n;
-                    const float4 yu = v_yu[cc];
-                    const float2 pp = v_p[cc];
-                    const float yr = yu.x, yi = yu.y, ur = yu.z, ui = yu.w, pr = pp.x, pi = pp.y;
-                    const float2 gv = G[j * RS + cc], sv = Q[j * RS + cc];
-                    const float gr = gv.x + qc.x * yr + qc.y * yi;             // G + q conj(yb)
-                    const float gi = gv.y + qc.y * yr - qc.x * yi;
-                    const float sr = sv.x, si2 = sv.y;
-                    const float zr = lr * sr - li * si2, zi = lr * si2 + li * sr;
-                    qzr += zr * yr - zi * yi;  qzi += zr * yi + zi * yr;       // Z yb
-                    k1r += gr * ur + gi * ui;  k1i += gi * ur - gr * ui;       // G conj(u)
-                    k2r += zr * pr - zi * pi;  k2i += zr * pi + zi * pr;       // Z p
-                    // Zb = G - beta k conj(p)
-                    const float br = gr - bt * (kr * pr + ki * pi), bi = gi - bt * (ki * pr - kr * pi);
-                    lbr += sr * br + si2 * bi;  lbi += sr * bi - si2 * br;     // conj(S_{t-1}) Zb
-                    G[j * RS + cc] = make_float2(lr * br + li * bi, lr * bi - li * br);   // conj(lam) Zb
-                }
+                float2 pp[TC], uu[TC];
+                ld_row<TC>(v_p + cl, pp);
+                ld_row<TC>(v_u + cl, uu);
+                // per row: dq re, im; dk re, im (before the factor beta); dalpha; dtheta; two unused
+                constexpr int NV = 8 * TR;
+                float val[NV];
 #pragma unroll
-                for (int d = TPR / 2; d >= 1; d >>= 1) {
-                    qzr += __shfl_xor_sync(0xffffffffu, qzr, d);  qzi += __shfl_xor_sync(0xffffffffu, qzi, d);
-                    k1r += __shfl_xor_sync(0xffffffffu, k1r, d);  k1i += __shfl_xor_sync(0xffffffffu, k1i, d);
-                    k2r += __shfl_xor_sync(0xffffffffu, k2r, d);  k2i += __shfl_xor_sync(0xffffffffu, k2i, d);
-                    lbr += __shfl_xor_sync(0xffffffffu, lbr, d);  lbi += __shfl_xor_sync(0xffffffffu, lbi, d);
+                for (int r = 0; r < TR; ++r) {
+                    const float4 lk = lkv[j0 + r], qc = qcv[j0 + r];
+                    const float lr = lk.x, li = lk.y, kr = lk.z, ki = lk.w;
+                    float qzr = 0.f, qzi = 0.f, dkr = 0.f, dki = 0.f, lbr = 0.f, lbi = 0.f;
+#pragma unroll
+                    for (int x = 0; x < TC; ++x) {
+                        const float gr = G[r][x].x, gi = G[r][x].y, sr = s[r][x].x, si2 = s[r][x].y;
+                        const float yr = y[x].x, yi = y[x].y, ur = uu[x].x, ui = uu[x].y, pr = pp[x].x, pi = pp[x].y;
+                        const float zr = lr * sr - li * si2, zi = lr * si2 + li * sr;
+                        qzr += zr * yr - zi * yi;  qzi += zr * yi + zi * yr;                 // Z yb
+                        dkr += gr * ur + gi * ui - (zr * pr - zi * pi);                      // G conj(u) - Z p
+                        dki += gi * ur - gr * ui - (zr * pi + zi * pr);
+                        // Zb = G - beta k conj(p)
+                        const float br = gr - bt * (kr * pr + ki * pi), bi = gi - bt * (ki * pr - kr * pi);
+                        lbr += sr * br + si2 * bi;  lbi += sr * bi - si2 * br;               // conj(S_{t-1}) Zb
+                        G[r][x] = make_float2(lr * br + li * bi, lr * bi - li * br);         // conj(lam) Zb
+                    }
+                    val[8 * r + 0] = qzr;
+                    val[8 * r + 1] = qzi;
+                    val[8 * r + 2] = bt * dkr;
+                    val[8 * r + 3] = bt * dki;
+                    val[8 * r + 4] = lbr * qc.z + lbi * qc.w;                                // Re(conj(lamb) e^{i theta})
+                    val[8 * r + 5] = lbi * lr - lbr * li;                                    // -Im(conj(lamb) lam)
+                    val[8 * r + 6] = 0.f;
+                    val[8 * r + 7] = 0.f;
                 }
-                if (part == 0) {
-                    const float dqr = qzr + bt * (kr * sr_ - ki * si_), dqi = qzi + bt * (kr * si_ + ki * sr_);   // + beta k (u^T yb)
-                    const float dkr = bt * (k1r - k2r), dki = bt * (k1i - k2i);
-                    const float cs = qc.z, sn = qc.w;
-                    const float dal = lbr * cs + lbi * sn;                                // Re(conj(lamb) e^{i theta})
-                    const float dth = lbi * lr - lbr * li;                                // -Im(conj(lamb) lam)
+                // sums over the warp's lanes (= columns): every exchange halves the values a lane still carries, so
+                // that lane l ends with the total of value l (NV = 32) or l / 2 (NV = 16)
+                int n = NV;
+#pragma unroll
+                for (int d = 16; d >= 1; d >>= 1) {
+                    if (n > 1) {
+                        const int half = n / 2;
+                        const bool up = (lane & d) != 0;
+#pragma unroll
+                        for (int i = 0; i < NV / 2; ++i) {
+                            if (i < half) {
+                                const float send = up ? val[i] : val[i + half];
+                                const float keep = up ? val[i + half] : val[i];
+                                val[i] = keep + __shfl_xor_sync(0xffffffffu, send, d);
+                            }
+                        }
+                        n = half;
+                    } else {
+                        val[0] += __shfl_xor_sync(0xffffffffu, val[0], d);
+                    }
+                }
+                const int vi = NV == 32 ? lane : lane >> 1;
+                const int rr = vi >> 3, qq = vi & 7, j = j0 + rr;
+                if (qq < 6 && (NV == 32 || !(lane & 1))) {
+                    float out = val[0];
+                    if (qq < 2) {
+                        const float4 lk = lkv[j];
+                        out += qq == 0 ? bt * (lk.z * uy_r - lk.w * uy_i) : bt * (lk.z * uy_i + lk.w * uy_r);   // + beta k (u^T yb)
+                    }
                     if constexpr (NSL == 1) {
-                        st_val(dq, row * DK + 2 * j, dqr);
-                        st_val(dq, row * DK + 2 * j + 1, dqi);
-                        st_val(dk, row * DK + 2 * j, dkr);
-                        st_val(dk, row * DK + 2 * j + 1, dki);
-                        a.dalpha[row * M + j] = dal;
-                        a.dtheta[row * M + j] = dth;
+                        if (qq < 2) st_val(dq, row * DK + 2 * j + qq, out);
+                        else if (qq < 4) st_val(dk, row * DK + 2 * j + qq - 2, out);
+                        else if (qq == 4) a.dalpha[row * M + j] = out;
+                        else a.dtheta[row * M + j] = out;
                     } else {      // this column block's share of the sums over the columns
-                        *reinterpret_cast<float2 *>(dq_p + row * DK + 2 * j) = make_float2(dqr, dqi);
-                        *reinterpret_cast<float2 *>(dk_p + row * DK + 2 * j) = make_float2(dkr, dki);
-                        dal_p[row * M + j] = dal;
-                        dth_p[row * M + j] = dth;
+                        if (qq < 2) dq_p[row * DK + 2 * j + qq] = out;
+                        else if (qq < 4) dk_p[row * DK + 2 * j + qq - 2] = out;
+                        else if (qq == 4) dal_p[row * M + j] = out;
+                        else dth_p[row * M + j] = out;
                     }
                 }
             }
-            __syncthreads();
             buf ^= 1;
+            set ^= 1;
         }
-        S = Pb(0);
     }
-    for (int idx = tid; idx < M * DV; idx += kBwdThreads) {
-        const int j = idx / DV, cc = idx % DV;
-        a.dS0[((size_t)bh * DK + 2 * j) * DVT + c0 + cc] = G[j * RS + cc].x;
-        a.dS0[((size_t)bh * DK + 2 * j + 1) * DVT + c0 + cc] = G[j * RS + cc].y;
-    }
+#pragma unroll
+    for (int r = 0; r < TR; ++r)
+#pragma unroll
+        for (int x = 0; x < TC; ++x) {
+            const size_t at = ((size_t)bh * DK + 2 * (j0 + r)) * DVT + c0 + cl + x;
+            a.dS0[at] = G[r][x].x;
+            a.dS0[at + DVT] = G[r][x].y;
+        }
 }
 
 // ---- the sums over the column blocks: out[i] = share_0[i] + share_1[i] + ... in that order, one thread per four
