@@ -176,6 +176,8 @@ def main():
                     help="sweeps only: time sfda_forward_two_level (slices chosen by the library) instead of sfda_forward")
     ap.add_argument("--no-long-context", action="store_true",
                     help="skip the leg that times configuration 3 with and without the two-level scan")
+    ap.add_argument("--no-t-sweep", action="store_true",
+                    help="skip the leg that times forward and backward at T = 4k, 16k, 64k, 128k")
     ap.add_argument("--no-variants", action="store_true", help="skip the leg that times the write-decoupled forward")
     ap.add_argument("--no-backward", action="store_true", help="skip the leg that times sfda_backward")
     ap.add_argument("--no-factors", action="store_true", help="skip the leg that times sfda_chunk_factors")
@@ -443,6 +445,54 @@ def main():
                    "backward_ms_per_call": lb_ms, "backward_launches": sfda.last_launch_count()}
         del ld, lo, lo_im, lS, lws, lg, lbws
 
+    # sequence-length sweep of the kernel benchmark protocol (App. E): T = 4k, 16k, 64k, 128k at d_k = d_v = 128,
+    # C = 64, H = 32, with B chosen for the headline's 65536 tokens per head (one sequence at 128k: twice that).
+    # Inputs drawn on the device with the distributions of configuration 1.
+    t_sweep = None
+    if rank == 0 and not args.no_t_sweep and args.batch == 0 and args.seq_len == 0:
+        t_sweep = []
+        for Ts in (4096, 16384, 65536, 131072):
+            Bs, Hs, dk, dv, ch = max(1, 65536 // Ts), cfg.H, cfg.d_k, cfg.d_v, cfg.chunk
+            gs = torch.Generator(device=dev)
+            gs.manual_seed(Ts)
+            rn = lambda *shape: torch.randn(*shape, device=dev, generator=gs)
+            sq, sv = rn(Bs, Ts, Hs, dk).to(torch.bfloat16), rn(Bs, Ts, Hs, dv).to(torch.bfloat16)
+            sk = torch.nn.functional.normalize(rn(Bs, Ts, Hs, dk), dim=-1).to(torch.bfloat16)
+            sal = torch.sigmoid(3.0 + rn(Bs, Ts, Hs, dk // 2))
+            sth = (torch.rand(Bs, Ts, Hs, dk // 2, device=dev, generator=gs) * 2.0 - 1.0) * math.pi
+            sbe = torch.sigmoid(rn(Bs, Ts, Hs))
+            so, so_im = torch.empty_like(sv), torch.empty_like(sv)
+            sS = torch.empty(Bs, Hs, dk, dv, device=dev)
+            sws = torch.empty(sfda.sfda_forward_two_level_workspace_bytes(Bs, Ts, Hs, dk, dv, ch, 1, 0),
+                              dtype=torch.uint8, device=dev)
+
+            def timed(fn, reps):
+                fn()
+                t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                t0.record(stream)
+                for _ in range(reps):
+                    fn()
+                t1.record(stream)
+                torch.cuda.synchronize()
+                return t0.elapsed_time(t1) / reps
+
+            f_ms = timed(lambda: sfda.sfda_forward(sq, sk, sv, sal, sth, sbe, None, so, so_im, sS, ch, sws, stream), 3)
+            assert sfda.sfda_workspace_status(sws, stream) == 0
+            # slices chosen by the library: with enough sequences this is the same single launch
+            f2_ms = timed(lambda: sfda.sfda_forward_two_level(sq, sk, sv, sal, sth, sbe, None, so, so_im, sS, ch, 0, sws,
+                                                              stream), 3)
+            f2_launches = sfda.last_launch_count()
+            assert sfda.sfda_workspace_status(sws, stream) == 0
+            sg = [torch.empty_like(x) for x in (sq, sk, sv, sal, sth, sbe)] + [torch.empty_like(sS)]
+            sbws = torch.empty(sfda.sfda_backward_workspace_bytes(Bs, Ts, Hs, dk, dv, 1), dtype=torch.uint8, device=dev)
+            b_ms = timed(lambda: sfda.sfda_backward(sq, sk, sv, sal, sth, sbe, None, so, so_im, sS, *sg, sbws, stream), 1)
+            t_sweep.append({"T": Ts, "B": Bs, "H": Hs, "forward_ms": f_ms, "forward_two_level_auto_ms": f2_ms,
+                            "two_level_launches": f2_launches, "backward_ms": b_ms,
+                            "forward_tokens_per_s": Bs * Ts / (min(f_ms, f2_ms) * 1e-3),
+                            "backward_tokens_per_s": Bs * Ts / (b_ms * 1e-3)})
+            del sq, sk, sv, sal, sth, sbe, so, so_im, sS, sws, sg, sbws
+
     # backward pass (sfda_backward) on the headline inputs: token-level fp32 adjoint, a first correct path
     bwd = None
     if rank == 0 and not args.no_backward:
@@ -666,7 +716,7 @@ def main():
                    "chunk": cfg.chunk, "outputs": "Re+Im" if want_im else "Re", "state": "fp32", "S0": "N(0,0.02)",
                    "parallelism": "dp%d over (batch, head), no collective" % world,
                    "l2": "inputs+outputs %.2f GB per step, far larger than the 126 MB L2; no flush" % (abytes / 1e9)},
-        "roofline": roofline, "cpu_baseline": cpu, "other_output_mode": other_mode, "e2e": e2e, "decode": decode, "fused_front_end": fused, "chunk_factors": factors, "backward": bwd, "write_decoupled_forward": variant, "long_context": longctx,
+        "roofline": roofline, "cpu_baseline": cpu, "other_output_mode": other_mode, "e2e": e2e, "decode": decode, "fused_front_end": fused, "chunk_factors": factors, "backward": bwd, "write_decoupled_forward": variant, "long_context": longctx, "t_sweep": t_sweep,
         "gpu_launches": launches_per_step * args.steps, "clocks": clocks.summary(),
     }
     print(json.dumps(line), flush=True)
