@@ -9,7 +9,7 @@ import os
 import numpy as np
 import pytest
 
-from oracle import backward, bookkeeping, chunk_wy, frontend, recurrence
+from oracle import backward, backward_chunk, bookkeeping, chunk_wy, frontend, recurrence
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -611,6 +611,36 @@ def test_backward_is_linear_in_the_upstream_and_additive_over_a_split():
     for i in range(6):
         assert np.allclose(np.concatenate([first[i], second[i]], axis=1), full[i], rtol=1e-12, atol=1e-12)
     assert np.allclose(first[6], full[6], rtol=1e-12, atol=1e-12)
+
+
+@pytest.mark.parametrize("chunk,T", [(1, 5), (4, 12), (8, 8), (6, 18)])
+def test_chunked_backward_equals_the_token_level_adjoint(chunk, T):
+    """The chunk form of the backward pass (triangular solves with the forward's Gram matrix, state-sized products
+    with S_0 and with the cotangent of S_C, C x C couplings) against the adjoint taken token by token -- and, for two
+    of the gradients, directly against central differences of the forward oracle.  Includes beta = 0 and beta = 1
+    tokens, a missing initial state, a missing Im cotangent and a missing final-state cotangent."""
+    x, up = _loss_inputs(40 + chunk, N=2, T=T)
+    x["beta"][0, 1] = 0.0
+    x["beta"][1, 2] = 1.0
+    args = (x["q"], x["k"], x["v"], x["alpha"], x["theta"], x["beta"])
+    want = backward.sfda_backward(*args, x["S0"], up["do_re"], up["do_im"], up["dS_T"])
+    got = backward_chunk.sfda_backward_chunked(*args, x["S0"], up["do_re"], up["do_im"], up["dS_T"], chunk)
+    for name, a, b in zip(("dq", "dk", "dv", "dalpha", "dtheta", "dbeta", "dS0"), got, want):
+        assert np.allclose(a, b, rtol=1e-10, atol=1e-10), name
+    want = backward.sfda_backward(*args, None, up["do_re"], None, None)
+    got = backward_chunk.sfda_backward_chunked(*args, None, up["do_re"], None, None, chunk)
+    for name, a, b in zip(("dq", "dk", "dv", "dalpha", "dtheta", "dbeta", "dS0"), got, want):
+        assert np.allclose(a, b, rtol=1e-10, atol=1e-10), name
+    # independent of the token-level adjoint: finite differences of the forward oracle
+    g = dict(zip(("q", "k", "v", "alpha", "theta", "beta", "S0"),
+                 backward_chunk.sfda_backward_chunked(*args, x["S0"], up["do_re"], up["do_im"], up["dS_T"], chunk)))
+    h = 1e-6
+    for key, idx in (("theta", (1, T - 2, 1)), ("k", (0, 0, 3)), ("alpha", (0, T // 2, 0))):
+        xp, xm = {n: np.array(a, copy=True) for n, a in x.items()}, {n: np.array(a, copy=True) for n, a in x.items()}
+        xp[key][idx] += h
+        xm[key][idx] -= h
+        fd = (_loss(xp, up) - _loss(xm, up)) / (2 * h)
+        assert abs(fd - g[key][idx]) <= 1e-6 * max(1.0, abs(fd)), (key, fd, g[key][idx])
 
 
 # ----------------------------------------------------------------------------
