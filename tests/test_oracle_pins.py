@@ -758,3 +758,112 @@ def test_decoupled_variant_against_explicit_matrices_and_limits():
         _, _, S_p = variants.sfda_decoupled_recurrence(**{n: (v if n == "S0" else v[:, :T_]) for n, v in z.items()})
         norms.append(np.linalg.norm(S_p[0]))
     assert all(b <= a + 1e-12 for a, b in zip(norms[:-1], norms[1:]))
+
+
+# ----------------------------------------------------------------------------
+# real-coordinate model with 2 x 2 orthogonal control blocks (rotations, reflections) and a real rank-one erase
+# ----------------------------------------------------------------------------
+def test_block_controls_without_reflections_are_the_complex_model():
+    """Lemma "Real-to-complex phase equivalence": with rotation blocks only and the realified complex erase, the
+    real-coordinate recurrence (dense real matrices) is the complex write-decoupled recurrence."""
+    from oracle import variants
+    x = _decoupled_inputs(50, N=2, T=9)
+    a = variants.sfda_decoupled_recurrence(**x)
+    b = variants.sfda_block_control_recurrence(x["q"], x["k"], x["r"], x["v"], x["alpha"], x["theta"], None, x["eta"],
+                                               x["beta"], x["S0"])
+    for u, w in zip(a, b):
+        assert np.allclose(u, w, rtol=1e-12, atol=1e-12)
+
+
+def test_reflection_block_is_complex_conjugation():
+    """F = diag(1, -1) on a row pair is z -> conj(z): a token whose blocks are alpha R(theta) F maps the complex row
+    S_j to alpha e^{i theta} conj(S_j) (then the same erase and write as before)."""
+    from oracle import variants
+    x = _decoupled_inputs(51, N=1, T=6)
+    rng = np.random.default_rng(51)
+    flip = rng.integers(0, 2, (1, 6, 3))
+    flip[0, 0] = 1
+    o_re, o_im, S_T = variants.sfda_block_control_recurrence(x["q"], x["k"], x["r"], x["v"], x["alpha"], x["theta"],
+                                                             flip, x["eta"], x["beta"], x["S0"])
+    kc, rc, qc = (x[n][0, :, 0::2] + 1j * x[n][0, :, 1::2] for n in ("k", "r", "q"))
+    lam = x["alpha"][0] * np.exp(1j * x["theta"][0])
+    S = x["S0"][0, 0::2] + 1j * x["S0"][0, 1::2]
+    for t in range(6):
+        Z = lam[t][:, None] * np.where(flip[0, t][:, None] == 1, S.conj(), S)
+        S = Z - x["eta"][0, t] * np.outer(kc[t], kc[t].conj() @ Z) + x["beta"][0, t] * np.outer(rc[t], x["v"][0, t])
+        assert np.allclose(S.conj().T @ qc[t], o_re[0, t] + 1j * o_im[0, t], atol=1e-12)
+    assert np.allclose(S, S_T[0, 0::2] + 1j * S_T[0, 1::2], atol=1e-12)
+
+
+def test_dihedral_group_is_tracked_exactly():
+    """Theorem "Dihedral phase-orientation memory": beta = 0, one row pair, d_v = 2, S_0 = I; the symbols R (rotation
+    by 2 pi / n), F (reflection) and RF drive S_t = rho(sigma_t ... sigma_1).  The expected matrix comes from integer
+    arithmetic in D_n, (R^a F^f)(R^b F^g) = R^{a + (-1)^f b} F^{f + g}; also F^2 = I and F R F = R^{-1}."""
+    from oracle import variants
+    n, T = 7, 40
+    rng = np.random.default_rng(52)
+    sym = rng.integers(0, 3, T)                       # 0: R, 1: F, 2: R F
+    theta = np.where(sym == 1, 0.0, 2 * np.pi / n)[None, :, None]
+    flip = (sym >= 1).astype(np.int64)[None, :, None]
+    one, zero = np.ones((1, T)), np.zeros((1, T))
+    zq = np.zeros((1, T, 2))
+    _, _, S_T = variants.sfda_block_control_recurrence(zq, zq, zq, np.zeros((1, T, 2)), np.ones((1, T, 1)), theta, flip,
+                                                       zero, zero, np.eye(2)[None])
+    a, f = 0, 0                                       # group element R^a F^f, multiplied from the left
+    for s in sym:
+        b, g = (1, 0) if s == 0 else (0, 1) if s == 1 else (1, 1)
+        a, f = (b + (-1) ** g * a) % n, (g + f) % 2   # (R^b F^g)(R^a F^f)
+    ang = 2 * np.pi * a / n
+    R = np.array([[np.cos(ang), -np.sin(ang)], [np.sin(ang), np.cos(ang)]])
+    want = R @ (np.diag([1.0, -1.0]) if f else np.eye(2))
+    assert np.allclose(S_T[0], want, atol=1e-12)
+    assert abs(np.linalg.norm(S_T[0], 2) - 1.0) < 1e-12          # orthogonal: bounded norm
+
+    def run(symbols):
+        th = np.array([0.0 if s == 1 else 2 * np.pi / n for s in symbols])[None, :, None]
+        fl = np.array([1 if s >= 1 else 0 for s in symbols])[None, :, None]
+        L = len(symbols)
+        z = np.zeros((1, L, 2))
+        return variants.sfda_block_control_recurrence(z, z, z, z, np.ones((1, L, 1)), th, fl, np.zeros((1, L)),
+                                                      np.zeros((1, L)), np.eye(2)[None])[2][0]
+    assert np.allclose(run([1, 1]), np.eye(2), atol=1e-15)                        # F^2 = I
+    assert np.allclose(run([1, 0, 1]) @ run([0]), np.eye(2), atol=1e-12)          # F R F = R^{-1}
+
+
+def test_real_rank_one_erase_is_the_real_delta_rule():
+    """With the erase k k^T on R^{2m} (Eq. "intro-sfda-real" read literally): theta = 0 and no reflections give the
+    textbook real gated delta rule S <- (I - beta k k^T) Diag(a) S + beta k v^T of dimension 2m (Prop. "KDA is a
+    special case"); a unit key with beta = 1 stores its value exactly, k_t^T S_t = v_t^T; and the real and the
+    complex erase differ by exactly eta (Jk)(Jk)^T applied to the controlled state."""
+    from oracle import variants
+    x = _decoupled_inputs(53, N=1, T=8)
+    x["k"] = x["k"] / np.linalg.norm(x["k"], axis=-1, keepdims=True)
+    zero_th = np.zeros_like(x["theta"])
+    o_re, _, S_T = variants.sfda_block_control_recurrence(x["q"], x["k"], x["k"], x["v"], x["alpha"], zero_th, None,
+                                                          x["beta"], x["beta"], x["S0"], real_erase=True)
+    S = x["S0"][0].copy()
+    for t in range(8):
+        a = np.repeat(x["alpha"][0, t], 2)
+        kk, b = x["k"][0, t], x["beta"][0, t]
+        S = a[:, None] * S
+        S = S - b * np.outer(kk, kk @ S) + b * np.outer(kk, x["v"][0, t])
+        assert np.allclose(S.T @ x["q"][0, t], o_re[0, t], atol=1e-12)
+    assert np.allclose(S, S_T[0], atol=1e-12)
+    # exact storage
+    ones = np.ones_like(x["beta"])
+    for T_ in (1, 5, 8):
+        _, _, S_p = variants.sfda_block_control_recurrence(x["q"][:, :T_], x["k"][:, :T_], x["k"][:, :T_], x["v"][:, :T_],
+                                                           x["alpha"][:, :T_], x["theta"][:, :T_], None, ones[:, :T_],
+                                                           ones[:, :T_], x["S0"], real_erase=True)
+        assert np.allclose(x["k"][0, T_ - 1] @ S_p[0], x["v"][0, T_ - 1], atol=1e-12)
+    # one step: the two erase terms differ by eta (Jk)(Jk)^T Z
+    args = [x[n][:, :1] for n in ("q", "k", "r", "v", "alpha", "theta")] + [None, x["eta"][:, :1], x["beta"][:, :1], x["S0"]]
+    S_c = variants.sfda_block_control_recurrence(*args)[2][0]
+    S_r = variants.sfda_block_control_recurrence(*args, real_erase=True)[2][0]
+    lam = x["alpha"][0, 0] * np.exp(1j * x["theta"][0, 0])
+    Zc = lam[:, None] * (x["S0"][0, 0::2] + 1j * x["S0"][0, 1::2])
+    Z = np.empty_like(x["S0"][0])
+    Z[0::2], Z[1::2] = Zc.real, Zc.imag
+    Jk = np.empty(6)
+    Jk[0::2], Jk[1::2] = -x["k"][0, 0, 1::2], x["k"][0, 0, 0::2]
+    assert np.allclose(S_r - S_c, x["eta"][0, 0] * np.outer(Jk, Jk @ Z), atol=1e-12)
