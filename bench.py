@@ -551,10 +551,26 @@ def main():
         v1.record(stream)
         torch.cuda.synchronize()
         v_ms = v0.elapsed_time(v1) / 2
+        # the same with 2 x 2 rotation / reflection control blocks and the real rank-one erase
+        flip_w = (torch.rand(d["alpha"].shape, device=dev, generator=gv) < 0.3).to(torch.uint8)
+
+        def bstep_():
+            sfda.sfda_forward_blocks(d["q"], d["k"], r_w, d["v"], d["alpha"], d["theta"], flip_w, eta_w, d["beta"],
+                                     d["S0"], o, o_im, S_T, sfda.ERASE_REAL, stream)
+
+        bstep_()
+        torch.cuda.synchronize()
+        v0.record(stream)
+        for _ in range(2):
+            bstep_()
+        v1.record(stream)
+        torch.cuda.synchronize()
+        vb_ms = v0.elapsed_time(v1) / 2
         variant = {"workload": cfg.name + " with a separate write direction r and erase strength eta",
                    "ms_per_step": v_ms, "tokens_per_s": cfg.B * cfg.T / (v_ms * 1e-3),
+                   "reflection_blocks_real_erase_ms_per_step": vb_ms,
                    "note": "token-level fp32 reference path; the chunk kernels compute the tied model only"}
-        del r_w, eta_w
+        del r_w, eta_w, flip_w
 
     # per-chunk factor export (sfda_chunk_factors) on the headline inputs: Gamma, Y, M, W and the phase turns
     factors = None
@@ -653,8 +669,23 @@ def main():
         d1.record(stream)
         torch.cuda.synchronize()
         dec_step_ms = d0.elapsed_time(d1) / nd
+        # and with 2 x 2 rotation / reflection control blocks and the real rank-one erase
+        flip_dec = (torch.rand(dcfg.B, dcfg.H, dcfg.d_k // 2, device=dev, generator=gd) < 0.3).to(torch.uint8)
+        for _ in range(8):
+            sfda.sfda_step_blocks(x0["q"], x0["k"], r_dec, x0["v"], x0["alpha"], x0["theta"], flip_dec, eta_dec,
+                                  x0["beta"], S, od, od_im, sfda.ERASE_REAL, stream)
+        torch.cuda.synchronize()
+        d0.record(stream)
+        for i in range(nd):
+            x = ring[i % len(ring)]
+            sfda.sfda_step_blocks(x["q"], x["k"], r_dec, x["v"], x["alpha"], x["theta"], flip_dec, eta_dec, x["beta"], S,
+                                  od, od_im, sfda.ERASE_REAL, stream)
+        d1.record(stream)
+        torch.cuda.synchronize()
+        blk_step_ms = d0.elapsed_time(d1) / nd
         decode = {"workload": dcfg.name, "ms_per_step": step_ms, "fused_raw_inputs_ms_per_step": fused_step_ms,
-                  "write_decoupled_ms_per_step": dec_step_ms, "tokens_per_s": dcfg.B / (step_ms * 1e-3),
+                  "write_decoupled_ms_per_step": dec_step_ms, "reflection_blocks_real_erase_ms_per_step": blk_step_ms,
+                  "tokens_per_s": dcfg.B / (step_ms * 1e-3),
                   "algorithmic_bytes_per_step": dbytes, "achieved_gbs": dbytes / (step_ms * 1e-3) / 1e9,
                   "state_bytes": int(S.numel() * 4), "note": "state (537 MB) far larger than L2"}
 

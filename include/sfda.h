@@ -273,6 +273,32 @@ SFDA_API int sfda_step_decoupled(const void *q, const void *k, const void *r, co
                                  int B, int H, int d_k, int d_v, int dtype, void *stream);
 
 /*
+ * The layer in real coordinates with aligned 2 x 2 orthogonal control blocks (Eq. "intro-sfda-real"; Theorem
+ * "Dihedral phase-orientation memory" and the remark after it):
+ *
+ *     S <- (I - eta P) U D S + beta r v^T,   U D = direct sum of alpha_j R(theta_j) F^{flip_j},   F = diag(1, -1),
+ *
+ * on the row pairs (2j, 2j+1) of S.  flip [B][T][H][m] (sfda_step_blocks: [B][H][m]) holds one byte per block,
+ * zero = rotation only, non-zero = reflect then rotate; NULL means no reflections.  erase selects P:
+ * SFDA_ERASE_COMPLEX, the realification k k^T + (Jk)(Jk)^T of the complex k k^* (with flip = NULL this is
+ * sfda_forward_decoupled), or SFDA_ERASE_REAL, the real rank-one k k^T on R^{2m} that Eq. "intro-sfda-real"
+ * writes.  o = S^T q and o_im = -S^T (Jq), J(x, y) = (-y, x) per pair (Re and Im of S^* q).  Other arguments,
+ * layouts, dtypes and errors as sfda_forward_decoupled / sfda_step_decoupled; erase outside the two values gives
+ * SFDA_ERR_VALUE.  Token by token in fp32 on the CUDA cores: reference paths, as for the write-decoupled variant.
+ */
+enum { SFDA_ERASE_COMPLEX = 0, SFDA_ERASE_REAL = 1 };
+SFDA_API int sfda_forward_blocks(const void *q, const void *k, const void *r, const void *v,
+                                 const float *alpha, const float *theta, const uint8_t *flip,
+                                 const float *eta, const float *beta,
+                                 const float *S0, void *o, void *o_im, float *S_T,
+                                 int B, int T, int H, int d_k, int d_v, int dtype, int erase, void *stream);
+SFDA_API int sfda_step_blocks(const void *q, const void *k, const void *r, const void *v,
+                              const float *alpha, const float *theta, const uint8_t *flip,
+                              const float *eta, const float *beta,
+                              float *S, void *o, void *o_im,
+                              int B, int H, int d_k, int d_v, int dtype, int erase, void *stream);
+
+/*
  * Host-buffer forward: the call a user with data in host memory makes.  Copies the
  * inputs from HOST memory (pinned for asynchronous copies) into `arena`, runs
  * sfda_forward there and copies o (and o_im, S_T when not NULL) back to HOST

@@ -62,6 +62,8 @@ def load():
     lib.sfda_forward_two_level.argtypes = [_vp] * 10 + [_ci] * 8 + [_vp, _sz, _vp]
     lib.sfda_step_decoupled.argtypes = [_vp] * 11 + [_ci] * 5 + [_vp]
     lib.sfda_forward_decoupled.argtypes = [_vp] * 12 + [_ci] * 6 + [_vp]
+    lib.sfda_step_blocks.argtypes = [_vp] * 12 + [_ci] * 6 + [_vp]
+    lib.sfda_forward_blocks.argtypes = [_vp] * 13 + [_ci] * 7 + [_vp]
     _LIB = lib
     return lib
 
@@ -355,3 +357,40 @@ def sfda_forward_decoupled(q, k, r, v, alpha, theta, eta, beta, S0, o, o_im, S_T
                                        _dtype_code(q), _stream(stream))
     if rc != 0:
         raise SfdaError(rc, "sfda_forward_decoupled")
+
+
+ERASE_COMPLEX, ERASE_REAL = 0, 1
+
+
+def sfda_step_blocks(q, k, r, v, alpha, theta, flip, eta, beta, S, o, o_im, erase=ERASE_COMPLEX, stream=None):
+    """``sfda_step_blocks`` of ``include/sfda.h``: one decode step with 2 x 2 rotation / reflection control blocks
+    (``flip``: uint8 [B, H, m] or None) and the complex or the real rank-one erase."""
+    B, H, d_k = q.shape
+    d_v = v.shape[-1]
+    for t, n in ((q, "q"), (k, "k"), (r, "r"), (v, "v"), (o, "o"), (o_im, "o_im")):
+        _check(t, n, q.dtype)
+    for t, n in ((alpha, "alpha"), (theta, "theta"), (eta, "eta"), (beta, "beta"), (S, "S")):
+        _check(t, n, torch.float32)
+    _check(flip, "flip", torch.uint8)
+    rc = load().sfda_step_blocks(_ptr(q), _ptr(k), _ptr(r), _ptr(v), _ptr(alpha), _ptr(theta), _ptr(flip), _ptr(eta),
+                                 _ptr(beta), _ptr(S), _ptr(o), _ptr(o_im), B, H, d_k, d_v, _dtype_code(q), int(erase),
+                                 _stream(stream))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_step_blocks")
+
+
+def sfda_forward_blocks(q, k, r, v, alpha, theta, flip, eta, beta, S0, o, o_im, S_T, erase=ERASE_COMPLEX, stream=None):
+    """``sfda_forward_blocks`` of ``include/sfda.h``: whole sequences with 2 x 2 rotation / reflection control
+    blocks (``flip``: uint8 [B, T, H, m] or None) and the complex or the real rank-one erase."""
+    B, T, H, d_k = q.shape
+    d_v = v.shape[-1]
+    for t, n in ((q, "q"), (k, "k"), (r, "r"), (v, "v"), (o, "o"), (o_im, "o_im")):
+        _check(t, n, q.dtype)
+    for t, n in ((alpha, "alpha"), (theta, "theta"), (eta, "eta"), (beta, "beta"), (S0, "S0"), (S_T, "S_T")):
+        _check(t, n, torch.float32)
+    _check(flip, "flip", torch.uint8)
+    rc = load().sfda_forward_blocks(_ptr(q), _ptr(k), _ptr(r), _ptr(v), _ptr(alpha), _ptr(theta), _ptr(flip),
+                                    _ptr(eta), _ptr(beta), _ptr(S0), _ptr(o), _ptr(o_im), _ptr(S_T), B, T, H, d_k, d_v,
+                                    _dtype_code(q), int(erase), _stream(stream))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_forward_blocks")

@@ -342,6 +342,42 @@ int sfda_step_decoupled(const void *q, const void *k, const void *r, const void 
     return step_common(q, k, v, alpha, theta, beta, S, o, o_im, B, H, d_k, d_v, dtype, par, stream);
 }
 
+int sfda_forward_blocks(const void *q, const void *k, const void *r, const void *v, const float *alpha,
+                        const float *theta, const uint8_t *flip, const float *eta, const float *beta, const float *S0,
+                        void *o, void *o_im, float *S_T, int B, int T, int H, int d_k, int d_v, int dtype, int erase,
+                        void *stream)
+{
+    g_last_launches = 0;
+    if (!r || !eta) return SFDA_ERR_NULL;
+    const int rc = validate_forward(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, 64, dtype);
+    if (rc != SFDA_OK) return rc;
+    if (erase != SFDA_ERASE_COMPLEX && erase != SFDA_ERASE_REAL) return SFDA_ERR_VALUE;
+    if (!aligned16(r) || !aligned16(eta) || (flip && !aligned16(flip))) return SFDA_ERR_ALIGN;
+    sfda::DecoupledArgs a;
+    a.q = q; a.k = k; a.r = r; a.v = v; a.alpha = alpha; a.theta = theta; a.eta = eta; a.beta = beta; a.S0 = S0;
+    a.o = o; a.o_im = o_im; a.S_T = S_T;
+    a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.dtype = dtype;
+    a.blocks = 1; a.real_erase = erase == SFDA_ERASE_REAL; a.flip = flip;
+    return sfda::launch_forward_decoupled(a, static_cast<cudaStream_t>(stream), &g_last_launches) == cudaSuccess
+               ? SFDA_OK
+               : SFDA_ERR_CUDA;
+}
+
+int sfda_step_blocks(const void *q, const void *k, const void *r, const void *v, const float *alpha,
+                     const float *theta, const uint8_t *flip, const float *eta, const float *beta, float *S, void *o,
+                     void *o_im, int B, int H, int d_k, int d_v, int dtype, int erase, void *stream)
+{
+    g_last_launches = 0;
+    if (!r || !eta) return SFDA_ERR_NULL;
+    if (erase != SFDA_ERASE_COMPLEX && erase != SFDA_ERASE_REAL) return SFDA_ERR_VALUE;
+    if (!aligned16(r) || !aligned16(eta) || (flip && !aligned16(flip))) return SFDA_ERR_ALIGN;
+    sfda::StepParam par;
+    par.r = r;
+    par.eta = eta;
+    par.blocks = 1; par.real_erase = erase == SFDA_ERASE_REAL; par.flip = flip;
+    return step_common(q, k, v, alpha, theta, beta, S, o, o_im, B, H, d_k, d_v, dtype, par, stream);
+}
+
 int sfda_step_fused(const void *q, const void *k_raw, const void *v, const float *a_raw, const float *b_raw,
                     const float *c_raw, float alpha_min, float alpha_max, float theta_max, float eps, float *S,
                     void *o, void *o_im, int B, int H, int d_k, int d_v, int dtype, void *stream)

@@ -33,6 +33,10 @@ struct StepParam {
     // write-decoupled variant (r != nullptr): write direction r [B][H][d_k] in the dtype of q, erase strength eta [B][H]
     const void *r = nullptr;
     const float *eta = nullptr;
+    // 2 x 2 orthogonal control blocks (blocks != 0, with r and eta): flip [B][H][m] bytes or nullptr (no reflections),
+    // real_erase != 0: the erase term is the real rank-one k k^T on R^{2m} instead of the complex k k^*
+    int blocks = 0, real_erase = 0;
+    const uint8_t *flip = nullptr;
 };
 
 struct StepArgs {
@@ -68,6 +72,9 @@ struct DecoupledArgs {
     void *o, *o_im;
     float *S_T;
     int B, T, H, d_k, d_v, dtype;
+    // 2 x 2 orthogonal control blocks: see StepParam; flip is [B][T][H][m] here
+    int blocks = 0, real_erase = 0;
+    const uint8_t *flip = nullptr;
 };
 
 // Each returns a cudaError_t from configuring / launching; *launches is incremented per kernel.

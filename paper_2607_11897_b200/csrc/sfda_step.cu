@@ -27,7 +27,9 @@ __device__ __forceinline__ float4 ld_state(const float *p)
 }
 
 // kMode: 0 the tied recurrence; 1 the same on raw inputs of the stable parameterisation; 2 the write-decoupled
-// variant S_t = (I - eta k k^*) Lambda S_{t-1} + beta r v^* (Section 3, Eq. "sfda-decoupled-main").
+// variant S_t = (I - eta k k^*) Lambda S_{t-1} + beta r v^* (Section 3, Eq. "sfda-decoupled-main"); 3 the same with
+// 2 x 2 orthogonal control blocks alpha R(theta) F^flip (a reflecting block conjugates the complex row first) and
+// the choice of the real rank-one erase k k^T on R^{2m} (Eq. "intro-sfda-real"), which takes Re(k^* Z) only.
 template <int DK, int DV, typename T, int kMode>
 __global__ void __launch_bounds__(kStepThreads)
 sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v,
@@ -35,7 +37,7 @@ sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__re
                  const float *__restrict__ beta, float *__restrict__ S, T *__restrict__ o,
                  T *__restrict__ o_im, const StepParam par)
 {
-    constexpr bool kFused = kMode == 1, kDec = kMode == 2;
+    constexpr bool kFused = kMode == 1, kDec = kMode >= 2, kBlk = kMode == 3;
     constexpr int M = DK / 2;              // complex rows
     constexpr int CT = DV < kColTile ? DV : kColTile;   // columns of this CTA
     constexpr int CG = CT / 4;             // threads across one row (float4 each)
@@ -48,6 +50,7 @@ sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__re
     __shared__ float s_red[RG][2][CT];
     __shared__ float s_norm[kStepThreads / 32];
     __shared__ float s_rr[kDec ? M : 1], s_ri[kDec ? M : 1];      // write direction r of the decoupled variant
+    __shared__ float s_sg[kBlk ? M : 1];                          // -1 where the block reflects, else 1
 
     const int tid = threadIdx.x;
     const size_t bh = blockIdx.x;
@@ -72,9 +75,11 @@ sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__re
     static_assert(M <= kStepThreads && CT <= kStepThreads, "one coordinate and one column per thread at most");
     float a = 1.f, th = 0.f, kr0 = 0.f, ki0 = 0.f, qr0 = 0.f, qi0 = 0.f, v0 = 0.f, rr0 = 0.f, ri0 = 0.f;
     const float eta = kDec ? par.eta[bh] : 0.f;
+    float sg0 = 1.f;
     if (kDec && tid < M) {
         rr0 = ld_val(static_cast<const T *>(par.r), bh * DK + 2 * tid);
         ri0 = ld_val(static_cast<const T *>(par.r), bh * DK + 2 * tid + 1);
+        if (kBlk && par.flip) sg0 = par.flip[bh * M + tid] ? -1.f : 1.f;
     }
     if (tid < M) {
         a = alpha[bh * M + tid];
@@ -107,6 +112,7 @@ sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__re
             s_rr[tid] = rr0;
             s_ri[tid] = ri0;
         }
+        if (kBlk) s_sg[tid] = sg0;
     }
     if (tid < CT) s_v[tid] = v0;
     constexpr int kKeyWarps = (M + 31) / 32;       // the warps whose threads read key coordinates above
@@ -137,10 +143,12 @@ sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__re
         const float lr = s_lr[j], li = s_li[j], kr = s_kr[j], ki = s_ki[j];
         float *pr = reinterpret_cast<float *>(&sre[r]);
         float *pi = reinterpret_cast<float *>(&sim[r]);
+        const float sg = kBlk ? s_sg[j] : 1.f;
 #pragma unroll
         for (int x = 0; x < 4; ++x) {
-            const float nr = lr * pr[x] - li * pi[x];
-            const float ni = lr * pi[x] + li * pr[x];
+            const float si = kBlk ? sg * pi[x] : pi[x];
+            const float nr = lr * pr[x] - li * si;
+            const float ni = lr * si + li * pr[x];
             pr[x] = nr;
             pi[x] = ni;
             cre[x] += kr * nr + ki * ni;   // conj(k) * s
@@ -164,7 +172,7 @@ sfda_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__re
         }
         if (kDec) {                            // erase part -eta c along k; the write beta v goes along r below
             ere[x] = -eta * a;
-            eim[x] = -eta * b;
+            eim[x] = kBlk && par.real_erase ? 0.f : -eta * b;
         } else if (kFused) {                   // c = s c_raw; e -> s e for the raw-key update
             ere[x] = sk * bt * (s_v[4 * cg + x] - sk * a);
             eim[x] = -sk * bt * sk * b;
@@ -222,7 +230,11 @@ template <int DK, int DV, typename T>
 cudaError_t launch_one(const StepArgs &a, cudaStream_t stream)
 {
     const dim3 grid((unsigned)a.B * (unsigned)a.H, DV > kColTile ? DV / kColTile : 1);
-    if (a.par.r)
+    if (a.par.r && a.par.blocks)
+        sfda_step_kernel<DK, DV, T, 3><<<grid, kStepThreads, 0, stream>>>(
+            static_cast<const T *>(a.q), static_cast<const T *>(a.k), static_cast<const T *>(a.v), a.alpha,
+            a.theta, a.beta, a.S, static_cast<T *>(a.o), static_cast<T *>(a.o_im), a.par);
+    else if (a.par.r)
         sfda_step_kernel<DK, DV, T, 2><<<grid, kStepThreads, 0, stream>>>(
             static_cast<const T *>(a.q), static_cast<const T *>(a.k), static_cast<const T *>(a.v), a.alpha,
             a.theta, a.beta, a.S, static_cast<T *>(a.o), static_cast<T *>(a.o_im), a.par);

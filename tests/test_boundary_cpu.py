@@ -205,6 +205,33 @@ def test_backward_entry_point_validates_on_the_host(lib):
     assert sfda.sfda_backward_workspace_bytes(1, 100, 2, 100, 128, 1) == 0
 
 
+def test_block_control_entry_points_validate_on_the_host(lib):
+    """sfda_forward_blocks / sfda_step_blocks: NULL, erase selector and alignment are refused before any launch."""
+    import ctypes
+    vp, ci = ctypes.c_void_p, ctypes.c_int
+    fake = [vp(0x1000 + 0x100 * i) for i in range(13)]           # q k r v alpha theta flip eta beta S0 o o_im S_T
+    lib.sfda_forward_blocks.restype = ci
+    lib.sfda_step_blocks.restype = ci
+
+    def fwd(ptrs, erase=0, dims=(1, 8, 2, 128, 128, 1)):
+        return lib.sfda_forward_blocks(*ptrs, *[ci(x) for x in dims], ci(erase), None)
+
+    assert fwd(fake[:2] + [None] + fake[3:]) == -1               # r
+    assert fwd(fake[:7] + [None] + fake[8:]) == -1               # eta
+    assert fwd(fake, erase=2) == -8
+    assert fwd(fake[:6] + [vp(0x1004)] + fake[7:]) == -4         # flip
+    assert fwd(fake, dims=(1, 8, 2, 96, 128, 1)) == -3
+    step = [vp(0x1000 + 0x100 * i) for i in range(12)]           # q k r v alpha theta flip eta beta S o o_im
+
+    def stp(ptrs, erase=0):
+        return lib.sfda_step_blocks(*ptrs, ci(1), ci(2), ci(128), ci(128), ci(1), ci(erase), None)
+
+    assert stp(step[:2] + [None] + step[3:]) == -1
+    assert stp(step, erase=-1) == -8
+    assert stp(step[:6] + [vp(0x1001)] + step[7:]) == -4
+    assert stp(step[:9] + [None] + step[10:]) == -1              # S
+
+
 def test_raw_input_generator_is_deterministic_and_untransformed():
     cfg = workloads.CONFIGS[1].scaled(B=2, T=64, H=2, s0_std=0.02)
     a, b = workloads.forward_raw_inputs(cfg), workloads.forward_raw_inputs(cfg)

@@ -946,6 +946,132 @@ def test_forward_decoupled_matches_oracle(d_k, d_v, T, dtype):
     assert rel_err(o.float().cpu().numpy(), o_t) <= tol and rel_err(S_T.cpu().numpy(), S_t) <= 1e-4
 
 
+def _block_case(cfg, seed, flips=True):
+    """Write direction, erase strength and reflection flags for the block-control variant."""
+    rng = np.random.default_rng([cfg.seed, seed])
+    rnd = (lambda x: workloads.bf16_round(x)) if cfg.dtype == "bf16" else (lambda x: x.astype(np.float32))
+    r = rnd(0.1 * rng.standard_normal((cfg.B, cfg.T, cfg.H, cfg.d_k), dtype=np.float32))
+    eta = rng.uniform(0.0, 1.0, (cfg.B, cfg.T, cfg.H)).astype(np.float32)
+    flip = (rng.uniform(size=(cfg.B, cfg.T, cfg.H, cfg.d_k // 2)) < 0.3).astype(np.uint8) if flips else None
+    return r, eta, flip
+
+
+@pytest.mark.parametrize("d_k,d_v,T,dtype,erase", [(128, 128, 90, "f32", 1), (64, 64, 33, "f32", 0),
+                                                   (128, 64, 120, "bf16", 1), (64, 128, 1, "f32", 0)])
+def test_forward_blocks_matches_oracle(d_k, d_v, T, dtype, erase):
+    """2 x 2 rotation / reflection control blocks with the complex or the real rank-one erase (Eq. "intro-sfda-real")
+    against the dense real-matrix oracle; without reflections and with the complex erase the kernel reproduces
+    sfda_forward_decoupled bit for bit."""
+    from oracle import variants
+    cfg = workloads.CONFIGS[0].scaled(name="fwdb", B=2, T=T, H=2, d_k=d_k, d_v=d_v, dtype=dtype, s0_std=0.4,
+                                      seed=140 + T)
+    inp = workloads.forward_inputs(cfg)
+    r, eta, flip = _block_case(cfg, 7)
+    d = {k: (None if v is None else to_dev(v, cfg, k)) for k, v in inp.items()}
+    dt = d["q"].dtype
+    rt, et, ft = torch.from_numpy(r).to(DEV).to(dt), torch.from_numpy(eta).to(DEV), torch.from_numpy(flip).to(DEV)
+    o = torch.empty(cfg.B, T, cfg.H, d_v, device=DEV, dtype=dt)
+    o_im = torch.empty_like(o)
+    S_T = torch.empty(cfg.B, cfg.H, d_k, d_v, device=DEV)
+    sfda.sfda_forward_blocks(d["q"], d["k"], rt, d["v"], d["alpha"], d["theta"], ft, et, d["beta"], d["S0"], o, o_im,
+                             S_T, erase)
+    torch.cuda.synchronize()
+    assert sfda.last_launch_count() == 1
+    pairs = all_pairs(cfg)
+    sel = lambda x: np.stack([x[b, :, h] for b, h in pairs]).astype(np.float64)
+    S0 = np.stack([inp["S0"][b, h] for b, h in pairs]).astype(np.float64)
+    w_re, w_im, w_S = variants.sfda_block_control_recurrence(sel(inp["q"]), sel(inp["k"]), sel(r), sel(inp["v"]),
+                                                             sel(inp["alpha"]), sel(inp["theta"]), sel(flip), sel(eta),
+                                                             sel(inp["beta"]), S0, real_erase=bool(erase))
+    tol = 5e-3 if dtype == "bf16" else 1e-4
+    on, oin, Sn = o.float().cpu().numpy(), o_im.float().cpu().numpy(), S_T.cpu().numpy()
+    assert rel_err(np.stack([on[b, :, h] for b, h in pairs]), w_re) <= tol
+    assert rel_err(np.stack([oin[b, :, h] for b, h in pairs]), w_im) <= tol
+    assert rel_err(np.stack([Sn[b, h] for b, h in pairs]), w_S) <= 1e-4
+    # no reflections, complex erase: the write-decoupled forward
+    o2, o2_im, S2 = torch.empty_like(o), torch.empty_like(o), torch.empty_like(S_T)
+    sfda.sfda_forward_blocks(d["q"], d["k"], rt, d["v"], d["alpha"], d["theta"], None, et, d["beta"], d["S0"], o, o_im,
+                             S_T, sfda.ERASE_COMPLEX)
+    sfda.sfda_forward_decoupled(d["q"], d["k"], rt, d["v"], d["alpha"], d["theta"], et, d["beta"], d["S0"], o2, o2_im, S2)
+    torch.cuda.synchronize()
+    assert torch.equal(o, o2) and torch.equal(o_im, o2_im) and torch.equal(S_T, S2)
+
+
+@pytest.mark.parametrize("d_k,d_v,dtype,erase", [(128, 128, "bf16", 1), (64, 128, "f32", 0), (128, 64, "f32", 1)])
+def test_step_blocks_iterated_matches_oracle(d_k, d_v, dtype, erase):
+    """The decode step of the block-control variant, token by token, against the dense real-matrix oracle."""
+    from oracle import variants
+    cfg = workloads.CONFIGS[0].scaled(name="stepb", B=2, T=24, H=3, d_k=d_k, d_v=d_v, dtype=dtype, s0_std=0.3,
+                                      seed=150 + d_k)
+    inp = workloads.forward_inputs(cfg)
+    r, eta, flip = _block_case(cfg, 8)
+    pairs = all_pairs(cfg)
+    sel = lambda x: np.stack([x[b, :, h] for b, h in pairs]).astype(np.float64)
+    S0 = np.stack([inp["S0"][b, h] for b, h in pairs]).astype(np.float64)
+    w_re, w_im, w_S = variants.sfda_block_control_recurrence(sel(inp["q"]), sel(inp["k"]), sel(r), sel(inp["v"]),
+                                                             sel(inp["alpha"]), sel(inp["theta"]), sel(flip), sel(eta),
+                                                             sel(inp["beta"]), S0, real_erase=bool(erase))
+    dt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    S = torch.from_numpy(inp["S0"]).to(DEV)
+    o = torch.empty(cfg.B, cfg.H, cfg.d_v, device=DEV, dtype=dt)
+    o_im = torch.empty_like(o)
+    got_re, got_im = [], []
+    for t in range(cfg.T):
+        d = {k: to_dev(np.ascontiguousarray(inp[k][:, t]), cfg, k) for k in ("q", "k", "v", "alpha", "theta", "beta")}
+        rt = torch.from_numpy(np.ascontiguousarray(r[:, t])).to(DEV).to(dt)
+        et = torch.from_numpy(np.ascontiguousarray(eta[:, t])).to(DEV)
+        ft = torch.from_numpy(np.ascontiguousarray(flip[:, t])).to(DEV)
+        sfda.sfda_step_blocks(d["q"], d["k"], rt, d["v"], d["alpha"], d["theta"], ft, et, d["beta"], S, o, o_im, erase)
+        assert sfda.last_launch_count() == 1
+        got_re.append(o.float().cpu().numpy())
+        got_im.append(o_im.float().cpu().numpy())
+    got_re, got_im = np.stack(got_re, 1), np.stack(got_im, 1)
+    tol = 5e-3 if dtype == "bf16" else 1e-4
+    assert rel_err(np.stack([got_re[b, :, h] for b, h in pairs]), w_re) <= tol
+    assert rel_err(np.stack([got_im[b, :, h] for b, h in pairs]), w_im) <= tol
+    assert rel_err(np.stack([S[b, h].cpu().numpy() for b, h in pairs]), w_S) <= 1e-4
+
+
+def test_blocks_track_dihedral_groups_exactly():
+    """Theorem "Dihedral phase-orientation memory" on the device: beta = eta = 0, alpha = 1, every row pair j of a
+    state starts as the 2 x 2 identity in columns (2j, 2j+1) and is driven by its own random word in R (rotation by
+    2 pi / 7), F (reflection), RF; the final block is rho of the product, which integer arithmetic in D_7 gives."""
+    n, T, B, H, d_k, d_v = 7, 50, 1, 2, 64, 64
+    m = d_k // 2
+    rng = np.random.default_rng(160)
+    sym = rng.integers(0, 3, (B, T, H, m))
+    theta = np.where(sym == 1, 0.0, 2 * np.pi / n).astype(np.float32)
+    flip = (sym >= 1).astype(np.uint8)
+    S0 = np.zeros((B, H, d_k, d_v), np.float32)
+    for j in range(m):
+        S0[:, :, 2 * j, 2 * j] = 1.0
+        S0[:, :, 2 * j + 1, 2 * j + 1] = 1.0
+    z = lambda *shape: torch.zeros(*shape, device=DEV)
+    o, o_im = z(B, T, H, d_v), z(B, T, H, d_v)
+    S_T = torch.empty(B, H, d_k, d_v, device=DEV)
+    sfda.sfda_forward_blocks(z(B, T, H, d_k), z(B, T, H, d_k), z(B, T, H, d_k), z(B, T, H, d_v),
+                             torch.ones(B, T, H, m, device=DEV), torch.from_numpy(theta).to(DEV),
+                             torch.from_numpy(flip).to(DEV), z(B, T, H), z(B, T, H), torch.from_numpy(S0).to(DEV), o,
+                             o_im, S_T, sfda.ERASE_REAL)
+    torch.cuda.synchronize()
+    got = S_T.cpu().numpy().astype(np.float64)
+    want = np.zeros_like(got)
+    for h in range(H):
+        for j in range(m):
+            a, f = 0, 0
+            for s in sym[0, :, h, j]:
+                b_, g = (1, 0) if s == 0 else (0, 1) if s == 1 else (1, 1)
+                a, f = (b_ + (-1) ** g * a) % n, (g + f) % 2
+            ang = 2 * np.pi * a / n
+            R = np.array([[np.cos(ang), -np.sin(ang)], [np.sin(ang), np.cos(ang)]])
+            want[0, h, 2 * j:2 * j + 2, 2 * j:2 * j + 2] = R @ (np.diag([1.0, -1.0]) if f else np.eye(2))
+    assert np.abs(got - want).max() < 2e-5
+    off = np.ones((d_k, d_v), bool)
+    for j in range(m):
+        off[2 * j:2 * j + 2, 2 * j:2 * j + 2] = False
+    assert np.count_nonzero(got[:, :, off]) == 0             # nothing leaks out of a pair's own block
+
+
 def test_final_state_may_alias_the_initial_state():
     """S_T == S0 (the same buffer) is allowed: the plain tensor-core forward and the two-level scan."""
     cfg = workloads.CONFIGS[1].scaled(name="alias", B=2, T=2048, H=2, s0_std=0.3, seed=140)
