@@ -422,28 +422,33 @@ def main():
         assert sfda.sfda_workspace_status(lws, stream) == 0
         two_launches = sfda.last_launch_count()
         # the backward pass on the same few sequences: the value columns are split over 4 CTAs per sequence
-        lg = [torch.empty_like(ld[key]) for key in ("q", "k", "v", "alpha", "theta", "beta")] + [torch.empty_like(lS)]
-        lbws = torch.empty(sfda.sfda_backward_workspace_bytes(lcfg.B, lcfg.T, lcfg.H, lcfg.d_k, lcfg.d_v, 1),
-                           dtype=torch.uint8, device=dev)
+        lb_ms, lb_launches = None, None
+        try:
+            lg = [torch.empty_like(ld[key]) for key in ("q", "k", "v", "alpha", "theta", "beta")] + [torch.empty_like(lS)]
+            lbws = torch.empty(sfda.sfda_backward_workspace_bytes(lcfg.B, lcfg.T, lcfg.H, lcfg.d_k, lcfg.d_v, 1),
+                               dtype=torch.uint8, device=dev)
 
-        def lbstep():
-            sfda.sfda_backward(ld["q"], ld["k"], ld["v"], ld["alpha"], ld["theta"], ld["beta"], ld["S0"], lo, lo_im, lS,
-                               *lg, lbws, stream)
+            def lbstep():
+                sfda.sfda_backward(ld["q"], ld["k"], ld["v"], ld["alpha"], ld["theta"], ld["beta"], ld["S0"], lo, lo_im,
+                                   lS, *lg, lbws, stream)
 
-        lbstep()
-        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        t0.record(stream)
-        lbstep()
-        t1.record(stream)
-        torch.cuda.synchronize()
-        lb_ms = t0.elapsed_time(t1)
+            lbstep()
+            t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            t0.record(stream)
+            lbstep()
+            t1.record(stream)
+            torch.cuda.synchronize()
+            lb_ms, lb_launches = t0.elapsed_time(t1), sfda.last_launch_count()
+            del lg, lbws
+        except torch.cuda.OutOfMemoryError:
+            pass                                      # reported as null: not enough free device memory
         longctx = {"workload": lcfg.name + " (B=1, T=131072, H=16)", "plain_ms_per_step": plain_ms,
                    "plain_tokens_per_s": lcfg.B * lcfg.T / (plain_ms * 1e-3), "two_level_ms_per_step": two_ms,
                    "two_level_tokens_per_s": lcfg.B * lcfg.T / (two_ms * 1e-3),
                    "two_level_launches": two_launches, "workspace_bytes": int(lws.numel()),
-                   "backward_ms_per_call": lb_ms, "backward_launches": sfda.last_launch_count()}
-        del ld, lo, lo_im, lS, lws, lg, lbws
+                   "backward_ms_per_call": lb_ms, "backward_launches": lb_launches}
+        del ld, lo, lo_im, lS, lws
 
     # sequence-length sweep of the kernel benchmark protocol (App. E): T = 4k, 16k, 64k, 128k at d_k = d_v = 128,
     # C = 64, H = 32, with B chosen for the headline's 65536 tokens per head (one sequence at 128k: twice that).
@@ -451,7 +456,8 @@ def main():
     t_sweep = None
     if rank == 0 and not args.no_t_sweep and args.batch == 0 and args.seq_len == 0:
         t_sweep = []
-        for Ts in (4096, 16384, 65536, 131072):
+
+        def sweep_point(Ts):
             Bs, Hs, dk, dv, ch = max(1, 65536 // Ts), cfg.H, cfg.d_k, cfg.d_v, cfg.chunk
             gs = torch.Generator(device=dev)
             gs.manual_seed(Ts)
@@ -487,11 +493,17 @@ def main():
             sg = [torch.empty_like(x) for x in (sq, sk, sv, sal, sth, sbe)] + [torch.empty_like(sS)]
             sbws = torch.empty(sfda.sfda_backward_workspace_bytes(Bs, Ts, Hs, dk, dv, 1), dtype=torch.uint8, device=dev)
             b_ms = timed(lambda: sfda.sfda_backward(sq, sk, sv, sal, sth, sbe, None, so, so_im, sS, *sg, sbws, stream), 1)
-            t_sweep.append({"T": Ts, "B": Bs, "H": Hs, "forward_ms": f_ms, "forward_two_level_auto_ms": f2_ms,
-                            "two_level_launches": f2_launches, "backward_ms": b_ms,
-                            "forward_tokens_per_s": Bs * Ts / (min(f_ms, f2_ms) * 1e-3),
-                            "backward_tokens_per_s": Bs * Ts / (b_ms * 1e-3)})
-            del sq, sk, sv, sal, sth, sbe, so, so_im, sS, sws, sg, sbws
+            return {"T": Ts, "B": Bs, "H": Hs, "forward_ms": f_ms, "forward_two_level_auto_ms": f2_ms,
+                    "two_level_launches": f2_launches, "backward_ms": b_ms,
+                    "forward_tokens_per_s": Bs * Ts / (min(f_ms, f2_ms) * 1e-3),
+                    "backward_tokens_per_s": Bs * Ts / (b_ms * 1e-3)}
+
+        for Ts in (4096, 16384, 65536, 131072):      # (a point's buffers are released when its function returns)
+            try:
+                t_sweep.append(sweep_point(Ts))
+            except torch.cuda.OutOfMemoryError:
+                t_sweep.append({"T": Ts, "skipped": "not enough free device memory for this point"})
+            torch.cuda.empty_cache()
 
     # backward pass (sfda_backward) on the headline inputs: token-level fp32 adjoint, a first correct path
     bwd = None
