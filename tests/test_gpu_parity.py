@@ -1093,3 +1093,58 @@ def test_final_state_may_alias_the_initial_state():
             sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], S, o, None, S, cfg.chunk, ws)
         torch.cuda.synchronize()
         assert rel_err(np.stack([S.cpu().numpy()[b, h] for b, h in pairs]), w_S) <= TOL["bf16"]
+
+
+def test_more_than_2_to_the_31_elements_per_array():
+    """B = 72 at the headline shapes: q, k, v, o hold 2.4e9 elements each, so any 32-bit index arithmetic would
+    wrap.  The kernels are deterministic and sequences independent, so the last two batch elements computed inside
+    the big batch must equal, bit for bit, the same ones computed alone (forward and fused forward on the tensor
+    cores, the backward pass)."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 120e9:
+        pytest.skip("needs about 110 GB of free device memory")
+    B, T, H, d = 72, 8192, 32, 128
+    g = torch.Generator(device=DEV)
+    g.manual_seed(7)
+    rn = lambda *s: torch.randn(*s, device=DEV, generator=g)
+    q, v = rn(B, T, H, d).to(torch.bfloat16), rn(B, T, H, d).to(torch.bfloat16)
+    k = rn(B, T, H, d)
+    k = (k / k.norm(dim=-1, keepdim=True)).to(torch.bfloat16)
+    alpha = torch.sigmoid(3.0 + rn(B, T, H, d // 2))
+    theta = (torch.rand(B, T, H, d // 2, device=DEV, generator=g) * 2 - 1) * np.pi
+    beta = torch.sigmoid(rn(B, T, H))
+    S0 = 0.02 * rn(B, H, d, d)
+    ins = (q, k, v, alpha, theta, beta, S0)
+    tail = tuple(x[B - 2:].contiguous() for x in ins)
+
+    def forward(x, fused):
+        b = x[0].shape[0]
+        o = torch.empty(b, T, H, d, device=DEV, dtype=torch.bfloat16)
+        o_im, S_T = torch.empty_like(o), torch.empty(b, H, d, d, device=DEV)
+        if fused:      # the same arrays read as raw inputs of the stable parameterisation
+            ws = torch.empty(sfda.sfda_forward_fused_workspace_bytes(b, T, H, d, d, 64, 1), dtype=torch.uint8, device=DEV)
+            sfda.sfda_forward_fused(x[0], x[1], x[2], x[3], x[4], x[5], 0.0, 1.0, float(np.pi), 1e-6, x[6], o, o_im, S_T,
+                                    64, ws)
+        else:
+            ws = torch.empty(sfda.sfda_workspace_bytes(b, T, H, d, d, 64, 1), dtype=torch.uint8, device=DEV)
+            sfda.sfda_forward(*x, o, o_im, S_T, 64, ws)
+        torch.cuda.synchronize()
+        assert sfda.sfda_workspace_status(ws) == 0
+        return o, o_im, S_T
+
+    for fused in (False, True):
+        big, small = forward(ins, fused), forward(tail, fused)
+        for a, b_ in zip(big, small):
+            assert torch.equal(a[B - 2:], b_), "fused" if fused else "plain"
+        del big, small
+    # backward: cotangents = the inputs themselves (any values do)
+    def backward_(x):
+        b = x[0].shape[0]
+        out = [torch.empty_like(t) for t in x]
+        ws = torch.empty(sfda.sfda_backward_workspace_bytes(b, T, H, d, d, 1), dtype=torch.uint8, device=DEV)
+        sfda.sfda_backward(*x, x[2], x[0], x[6], *out, ws)
+        torch.cuda.synchronize()
+        return out
+    big, small = backward_(ins), backward_(tuple(x[B - 4:].contiguous() for x in ins))
+    for a, b_ in zip(big, small):
+        assert torch.equal(a[B - 4:], b_)
