@@ -1100,6 +1100,9 @@ def test_more_than_2_to_the_31_elements_per_array():
     wrap.  The kernels are deterministic and sequences independent, so the last two batch elements computed inside
     the big batch must equal, bit for bit, the same ones computed alone (forward and fused forward on the tensor
     cores, the backward pass)."""
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()                       # earlier tests' cached blocks count as used otherwise
     free, _ = torch.cuda.mem_get_info()
     if free < 120e9:
         pytest.skip("needs about 110 GB of free device memory")
@@ -1148,3 +1151,102 @@ def test_more_than_2_to_the_31_elements_per_array():
     big, small = backward_(ins), backward_(tuple(x[B - 4:].contiguous() for x in ins))
     for a, b_ in zip(big, small):
         assert torch.equal(a[B - 4:], b_)
+
+
+def test_more_than_2_to_the_31_elements_other_kernels():
+    """The same check for the other kernels: stand-alone parameterisation, factor export, write-decoupled forward
+    (B = 72 at the headline shapes), the decode step on 163840 states (2.7e9 state elements) and the two-level scan on
+    one batch element of 2^20 tokens, each against the same computation on a small part of the data."""
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()                       # earlier tests' cached blocks count as used otherwise
+    free, _ = torch.cuda.mem_get_info()
+    if free < 120e9:
+        pytest.skip("needs about 100 GB of free device memory")
+    B, T, H, d = 72, 8192, 32, 128
+    g = torch.Generator(device=DEV)
+    g.manual_seed(8)
+    rn = lambda *s: torch.randn(*s, device=DEV, generator=g)
+    k = rn(B, T, H, d).to(torch.bfloat16)
+    a, b, c = 3.0 + rn(B, T, H, d // 2), rn(B, T, H, d // 2), rn(B, T, H)
+
+    def frontend(x):
+        outs = (torch.empty_like(x[0]), torch.empty_like(x[1]), torch.empty_like(x[2]), torch.empty_like(x[3]))
+        sfda.sfda_frontend(x[0], x[1], x[2], x[3], 0.0, 1.0, float(np.pi), 1e-6, *outs)
+        torch.cuda.synchronize()
+        return outs
+    big = frontend((a, b, c, k))
+    small = frontend(tuple(x[B - 2:].contiguous() for x in (a, b, c, k)))
+    for x, y in zip(big, small):
+        assert torch.equal(x[B - 2:], y)
+    alpha, theta, beta, kn = big
+    del a, b, c, small
+
+    def factors(x):
+        bb, NC = x[0].shape[0], T // 64
+        Gm = torch.empty(bb, H, NC, d // 2, 2, device=DEV)
+        Y = torch.empty(bb, H, NC, d // 2, 64, 2, device=DEV)
+        W, M = torch.empty_like(Y), torch.empty(bb, H, NC, 64, 64, 2, device=DEV)
+        turns = torch.empty(bb, T, H, d // 2, device=DEV, dtype=torch.int32)
+        sfda.sfda_chunk_factors(x[0], x[1], x[2], x[3], Gm, Y, M, W, turns, 64)
+        torch.cuda.synchronize()
+        return Gm, Y, M, W, turns
+    big = factors((kn, alpha, theta, beta))
+    small = factors(tuple(x[B - 1:].contiguous() for x in (kn, alpha, theta, beta)))
+    for x, y in zip(big, small):
+        assert torch.equal(x[B - 1:], y)
+    del big, small
+
+    q, v = rn(B, T, H, d).to(torch.bfloat16), rn(B, T, H, d).to(torch.bfloat16)
+    r, eta = (0.1 * rn(B, T, H, d)).to(torch.bfloat16), torch.rand(B, T, H, device=DEV, generator=g)
+
+    def decoupled(x):
+        bb = x[0].shape[0]
+        o = torch.empty(bb, T, H, d, device=DEV, dtype=torch.bfloat16)
+        o_im, S_T = torch.empty_like(o), torch.empty(bb, H, d, d, device=DEV)
+        sfda.sfda_forward_decoupled(*x, None, o, o_im, S_T)
+        torch.cuda.synchronize()
+        return o, o_im, S_T
+    ins = (q, kn, r, v, alpha, theta, eta, beta)
+    big, small = decoupled(ins), decoupled(tuple(x[B - 1:].contiguous() for x in ins))
+    for x, y in zip(big, small):
+        assert torch.equal(x[B - 1:], y)
+    del big, small, ins, q, v, r, eta, kn, alpha, theta, beta, k
+
+    # decode: 4096 x 40 states
+    Bd, Hd = 4096, 40
+    S = 0.02 * rn(Bd, Hd, d, d)
+    qd, vd = rn(Bd, Hd, d).to(torch.bfloat16), rn(Bd, Hd, d).to(torch.bfloat16)
+    kd = rn(Bd, Hd, d)
+    kd = (kd / kd.norm(dim=-1, keepdim=True)).to(torch.bfloat16)
+    ad, td, bd = torch.sigmoid(3.0 + rn(Bd, Hd, d // 2)), rn(Bd, Hd, d // 2), torch.sigmoid(rn(Bd, Hd))
+    S_small = S[Bd - 3:].clone()
+    o, o_im = torch.empty_like(vd), torch.empty_like(vd)
+    sfda.sfda_step(qd, kd, vd, ad, td, bd, S, o, o_im)
+    o_s, o_im_s = torch.empty_like(vd[Bd - 3:]), torch.empty_like(vd[Bd - 3:])
+    sfda.sfda_step(*(x[Bd - 3:].contiguous() for x in (qd, kd, vd, ad, td, bd)), S_small, o_s, o_im_s)
+    torch.cuda.synchronize()
+    assert torch.equal(S[Bd - 3:], S_small) and torch.equal(o[Bd - 3:], o_s) and torch.equal(o_im[Bd - 3:], o_im_s)
+    del S, S_small, qd, kd, vd, ad, td, bd
+
+    # two-level scan: one batch element, 16 heads, 2^20 tokens (2^31 elements in q); head 15 alone for comparison
+    Tl, Hl = 1 << 20, 16
+    ql, vl = rn(1, Tl, Hl, d).to(torch.bfloat16), rn(1, Tl, Hl, d).to(torch.bfloat16)
+    kl = rn(1, Tl, Hl, d)
+    kl = (kl / kl.norm(dim=-1, keepdim=True)).to(torch.bfloat16)
+    al, tl, bl = torch.sigmoid(3.0 + rn(1, Tl, Hl, d // 2)), rn(1, Tl, Hl, d // 2), torch.sigmoid(rn(1, Tl, Hl))
+
+    def two_level(x):
+        hh = x[0].shape[2]
+        o = torch.empty(1, Tl, hh, d, device=DEV, dtype=torch.bfloat16)
+        o_im, S_T = torch.empty_like(o), torch.empty(1, hh, d, d, device=DEV)
+        ws = torch.empty(sfda.sfda_forward_two_level_workspace_bytes(1, Tl, hh, d, d, 64, 1, 8), dtype=torch.uint8,
+                         device=DEV)
+        sfda.sfda_forward_two_level(*x, None, o, o_im, S_T, 64, 8, ws)
+        torch.cuda.synchronize()
+        assert sfda.sfda_workspace_status(ws) == 0
+        return o, o_im, S_T
+    ins = (ql, kl, vl, al, tl, bl)
+    big, small = two_level(ins), two_level(tuple(x[:, :, Hl - 1:].contiguous() for x in ins))
+    assert torch.equal(big[0][:, :, Hl - 1:], small[0]) and torch.equal(big[1][:, :, Hl - 1:], small[1])
+    assert torch.equal(big[2][:, Hl - 1:], small[2])
