@@ -1148,12 +1148,17 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
             // fused: D1 was formed with the raw key, R = V - s D1; the per-token factor replaces the sign
             if (kFused && ph == 0 && !wait_k_warp(mi, B_NORM_FULL, j)) return;
             const uint32_t scp = smem_u32(ph == 0 ? &mi.kscale[(j & 3)][0] : &mi.ones[0]);
+            // The second half of the accumulator is read into registers before the first half of the operand is
+            // announced: the product which that announcement releases (E = M_beta R goes out in two halves of its K
+            // dimension) starts these very accumulator columns from zero, all 64 of them, so a warp that fetched
+            // columns 32..63 only after announcing columns 0..31 could find E's partial sums where D1 was.
+            uint32_t r[32];
+            tmem_ld<32>(tlane + TM_ACC + 128 * half, r);
+            tc_wait_ld();
 #pragma unroll 1
             for (int pc = 0; pc < 2; ++pc) {       // 32 columns per tensor-memory round trip
-                uint32_t r[32], pk[16];
+                uint32_t pk[16];
                 uint4 sc4 = make_uint4(0u, 0u, 0u, 0u);
-                tmem_ld<32>(tlane + TM_ACC + 128 * half + 32 * pc, r);
-                tc_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     float v0 = 0.f, v1 = 0.f;
@@ -1168,6 +1173,10 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
                         s1 = __uint_as_float((i & 1) ? sc4.w : sc4.y);
                     }
                     pk[i] = pack_bf16(fmaf(s0, __uint_as_float(r[2 * i]), v0), fmaf(s1, __uint_as_float(r[2 * i + 1]), v1));
+                }
+                if (pc == 0) {
+                    tmem_ld<32>(tlane + TM_ACC + 128 * half + 32, r);
+                    tc_wait_ld();
                 }
                 // R replaces S_0 in the operand columns: rho_1, the last reader of S_0, must be done
                 if (ph == 0 && pc == 0 && !wait_k_warp(mi, B_O1_DONE, j)) return;

@@ -211,6 +211,43 @@ def test_forward_tensor_core_is_deterministic():
         assert np.array_equal(x, y)
 
 
+def test_forward_tensor_core_is_deterministic_at_the_headline_sizes():
+    """Five launches of the plain and of the fused forward at B = 8, T = 8192, H = 32: every bit of o, o_im and S_T
+    the same.  (32768 chunks per launch: enough for a rare ordering hazard between the roles of the kernel to show;
+    a product released by the first half of an operand once overwrote accumulator columns whose second half a slow
+    warp had not read yet, in about one chunk per million.)"""
+    B, T, H, d = 8, 8192, 32, 128
+    g = torch.Generator(device=DEV)
+    g.manual_seed(94)
+    rn = lambda *s: torch.randn(*s, device=DEV, generator=g)
+    q, v = rn(B, T, H, d).to(torch.bfloat16), rn(B, T, H, d).to(torch.bfloat16)
+    k = rn(B, T, H, d)
+    k = (k / k.norm(dim=-1, keepdim=True)).to(torch.bfloat16)
+    a = torch.sigmoid(3.0 + rn(B, T, H, d // 2))
+    b = (torch.rand(B, T, H, d // 2, device=DEV, generator=g) * 2 - 1) * np.pi
+    c, S0 = torch.sigmoid(rn(B, T, H)), 0.02 * rn(B, H, d, d)
+
+    def run(fused):
+        o = torch.empty(B, T, H, d, device=DEV, dtype=torch.bfloat16)
+        o_im, S_T = torch.empty_like(o), torch.empty(B, H, d, d, device=DEV)
+        if fused:      # the same arrays read as raw inputs of the stable parameterisation
+            ws = torch.empty(sfda.sfda_forward_fused_workspace_bytes(B, T, H, d, d, 64, 1), dtype=torch.uint8, device=DEV)
+            sfda.sfda_forward_fused(q, k, v, a, b, c, 0.0, 1.0, float(np.pi), 1e-6, S0, o, o_im, S_T, 64, ws)
+        else:
+            ws = torch.empty(sfda.sfda_workspace_bytes(B, T, H, d, d, 64, 1), dtype=torch.uint8, device=DEV)
+            sfda.sfda_forward(q, k, v, a, b, c, S0, o, o_im, S_T, 64, ws)
+        torch.cuda.synchronize()
+        assert sfda.sfda_workspace_status(ws) == 0
+        return o, o_im, S_T
+
+    for fused in (False, True):
+        first = run(fused)
+        for _ in range(4):
+            again = run(fused)
+            for x, y in zip(first, again):
+                assert torch.equal(x, y), "fused" if fused else "plain"
+
+
 def test_forward_tensor_core_matches_cuda_core_path():
     cfg = workloads.CONFIGS[1].scaled(name="tc2", B=1, T=512, H=4, s0_std=0.1, seed=77)
     inp = workloads.forward_inputs(cfg)
