@@ -188,6 +188,19 @@ struct ChunkCursor {
     }
 };
 
+// Development builds only (-DSFDA_WS_CHAOS): a pseudo-random pause of 0.1 to 1.1 us after one in eight barrier
+// arrivals and completed waits.  The results do not depend on timing, so a build with the pauses must reproduce
+// the plain build bit for bit; an ordering hazard between the roles shows as a difference.
+#ifdef SFDA_WS_CHAOS
+__device__ __forceinline__ void chaos(uint32_t salt)
+{
+    uint32_t x = (uint32_t)clock() * 2654435761u + salt * 40503u + (threadIdx.x >> 5) * 9176u;
+    x ^= x >> 13; x *= 0x5bd1e995u; x ^= x >> 15;
+    if ((x & 7u) == 0u) __nanosleep(100u + ((x >> 8) & 1023u));
+}
+#else
+__device__ __forceinline__ void chaos(uint32_t) {}
+#endif
 __device__ __forceinline__ void mbar_arrive(unsigned long long *bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -198,6 +211,11 @@ __device__ __forceinline__ void warp_arrive(unsigned long long *bar)
 {
     __syncwarp();
     if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
+#ifdef SFDA_WS_CHAOS
+    __syncwarp();
+    chaos((uint32_t)(size_t)bar);
+    __syncwarp();
+#endif
 }
 template <int N>
 __device__ __forceinline__ void regs_inc()
@@ -249,7 +267,10 @@ __device__ __forceinline__ bool wait_k(Misc &mi, int bar, int k)
             : "=r"(ok)
             : "r"(addr), "r"(parity), "r"(20000u)
             : "memory");
-        if (ok) return true;
+        if (ok) {
+            chaos(addr + 77u);
+            return true;
+        }
     } while ((uint32_t)clock() - t0 < 0x80000000u);
     mi.abort = 1;
     return false;
