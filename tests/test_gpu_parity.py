@@ -1287,3 +1287,54 @@ def test_more_than_2_to_the_31_elements_other_kernels():
     big, small = two_level(ins), two_level(tuple(x[:, :, Hl - 1:].contiguous() for x in ins))
     assert torch.equal(big[0][:, :, Hl - 1:], small[0]) and torch.equal(big[1][:, :, Hl - 1:], small[1])
     assert torch.equal(big[2][:, Hl - 1:], small[2])
+
+
+def test_calls_can_be_captured_in_a_cuda_graph():
+    """The library only enqueues on the caller's stream (no allocation, no synchronisation), so its calls can be
+    recorded into a CUDA graph and replayed: eight decode steps, a forward, a fused forward, a two-level forward and
+    a backward pass give the same bits replayed as run directly."""
+    cfg = workloads.CONFIGS[1].scaled(name="graph", B=1, T=4096, H=4, s0_std=0.05, seed=97)
+    inp = workloads.forward_inputs(cfg)
+    d = {k: to_dev(v, cfg, k) for k, v in inp.items()}
+    B, T, H, dk, dv = cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v
+    new = lambda *s, dt=torch.bfloat16: torch.empty(*s, device=DEV, dtype=dt)
+    o, o_im, S_T = new(B, T, H, dv), new(B, T, H, dv), new(B, H, dk, dv, dt=torch.float32)
+    o2, o2_im, S2 = new(B, T, H, dv), new(B, T, H, dv), new(B, H, dk, dv, dt=torch.float32)
+    o3, o3_im, S3 = new(B, T, H, dv), new(B, T, H, dv), new(B, H, dk, dv, dt=torch.float32)
+    ws = torch.empty(sfda.sfda_forward_two_level_workspace_bytes(B, T, H, dk, dv, 64, 1, 4), dtype=torch.uint8, device=DEV)
+    ws2 = torch.empty_like(ws)
+    ws3 = torch.empty_like(ws)
+    grads = [torch.empty_like(d[k]) for k in ("q", "k", "v", "alpha", "theta", "beta")] + [torch.empty_like(S_T)]
+    bws = torch.empty(sfda.sfda_backward_workspace_bytes(B, T, H, dk, dv, 1), dtype=torch.uint8, device=DEV)
+    S_dec = d["S0"].clone()
+    od, od_im = new(B, H, dv), new(B, H, dv)
+    step_in = [{k: d[k][:, t].clone() for k in ("q", "k", "v", "alpha", "theta", "beta")} for t in range(8)]
+
+    def work():
+        sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im, S_T, 64, ws)
+        sfda.sfda_forward_fused(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], 0.0, 1.0, float(np.pi), 1e-6,
+                                d["S0"], o2, o2_im, S2, 64, ws2)
+        sfda.sfda_forward_two_level(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o3, o3_im, S3,
+                                    64, 4, ws3)
+        sfda.sfda_backward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im, S_T, *grads, bws)
+        for x in step_in:
+            sfda.sfda_step(x["q"], x["k"], x["v"], x["alpha"], x["theta"], x["beta"], S_dec, od, od_im)
+
+    outs = [o, o_im, S_T, o2, o2_im, S2, o3, o3_im, S3, S_dec, od, od_im] + grads
+    work()
+    torch.cuda.synchronize()
+    want = [x.clone() for x in outs]
+    for x in outs:
+        x.zero_()
+    S_dec.copy_(d["S0"])
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        work()
+    for x in outs:                      # capturing runs nothing
+        x.zero_()
+    S_dec.copy_(d["S0"])
+    graph.replay()
+    torch.cuda.synchronize()
+    assert sfda.sfda_workspace_status(ws) == 0 and sfda.sfda_workspace_status(ws2) == 0
+    for got, w in zip(outs, want):
+        assert torch.equal(got, w)
