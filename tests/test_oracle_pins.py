@@ -524,6 +524,38 @@ def test_parameterisation_gives_the_stability_assumptions():
     assert np.all(np.linalg.norm(S_T.reshape(N, -1), axis=-1) <= bound[:, 0] + 1e-9)
 
 
+def test_parameterisation_backward_matches_central_differences():
+    """The gradients with respect to the raw inputs against (L(x + h e) - L(x - h e)) / 2h of the forward
+    parameterisation, L = <dalpha, alpha> + <dtheta, theta> + <dbeta, beta> + <dk, k>, entry by entry; a zero key
+    passes s dk through; and the key's gradient is orthogonal to the key when eps = 0 (k does not depend on the
+    length of k_raw then)."""
+    rng = np.random.default_rng(61)
+    a, b, c = rng.normal(0, 2, (3, 4)), rng.normal(0, 1.5, (3, 4)), rng.normal(0, 2, 3)
+    kr = rng.normal(0, 1, (3, 8))
+    up = [rng.normal(size=x.shape) for x in (a, b, c, kr)]
+    par = (0.1, 0.95, 2.0, 1e-3)
+
+    def loss(a_, b_, c_, k_):
+        out = frontend.stable_parameterisation(a_, b_, c_, k_, *par)
+        return float(sum(np.sum(u * o) for u, o in zip(up, out)))
+
+    got = frontend.stable_parameterisation_backward(a, b, c, kr, *par, *up)
+    h = 1e-6
+    for idx_arr, (x, g) in enumerate(zip((a, b, c, kr), got)):
+        for idx in np.ndindex(x.shape):
+            args_p, args_m = [a.copy(), b.copy(), c.copy(), kr.copy()], [a.copy(), b.copy(), c.copy(), kr.copy()]
+            args_p[idx_arr][idx] += h
+            args_m[idx_arr][idx] -= h
+            fd = (loss(*args_p) - loss(*args_m)) / (2 * h)
+            assert abs(fd - g[idx]) <= 1e-7 * max(1.0, abs(fd)), (idx_arr, idx, fd, g[idx])
+    z = np.zeros((1, 8))
+    dk = rng.normal(size=(1, 8))
+    g0 = frontend.stable_parameterisation_backward(a[:1], b[:1], c[:1], z, *par, up[0][:1], up[1][:1], up[2][:1], dk)[3]
+    assert np.allclose(g0, dk / 1e-3)
+    g1 = frontend.stable_parameterisation_backward(a, b, c, kr, 0.1, 0.95, 2.0, 0.0, *up)[3]
+    assert np.allclose(np.sum(g1 * kr, axis=-1), 0.0, atol=1e-12)
+
+
 # ----------------------------------------------------------------------------
 # backward pass: the gradient of a scalar loss through Eq. "sfda"
 # ----------------------------------------------------------------------------
