@@ -374,12 +374,17 @@ def main():
                                                    kn, stream),
                                 sfda.sfda_forward(r["q"], kn, r["v"], al, th, be, r["S0"], o, o_im, S_T, cfg.chunk,
                                                   ws, stream)), max(args.steps, 5))
+        # the derivative of the parameterisation (gradients in place: al, th, be, kn serve as incoming gradients)
+        fb_ms = timed(lambda: sfda.sfda_frontend_backward(r["a_raw"], r["b_raw"], r["c_raw"], r["k_raw"], *par, al, th, be,
+                                                          kn, al, th, be, kn, stream), max(args.steps, 5))
         rows = cfg.B * cfg.T * cfg.H
         fbytes = rows * 2 * (2 * cfg.m * 4 + 4 + cfg.d_k * 2)          # every array read once, written once
         fused = {"workload": cfg.name + " from raw a, b, c, k (alpha in [0,1], theta_max = pi, eps = 1e-6)",
                  "fused_ms_per_step": fused_ms, "fused_tokens_per_s": cfg.B * cfg.T / (fused_ms * 1e-3),
                  "frontend_kernel_ms": front_ms, "frontend_bytes": fbytes,
                  "frontend_achieved_gbs": fbytes / (front_ms * 1e-3) / 1e9,
+                 "frontend_backward_kernel_ms": fb_ms, "frontend_backward_bytes": fbytes * 3 // 2,
+                 "frontend_backward_achieved_gbs": fbytes * 1.5 / (fb_ms * 1e-3) / 1e9,
                  "two_step_ms_per_step": two_ms, "two_step_tokens_per_s": cfg.B * cfg.T / (two_ms * 1e-3)}
         del r, al, th, be, kn
 

@@ -346,6 +346,24 @@ SFDA_API int sfda_frontend(const float *a_raw, const float *b_raw, const float *
                            int B, int T, int H, int d_k, int dtype, void *stream);
 
 /*
+ * The derivative of sfda_frontend: with the gradients of a loss with respect to alpha, theta, beta, k (for instance
+ * dalpha, dtheta, dbeta, dk of sfda_backward), its gradients with respect to the raw inputs,
+ *
+ *     da = dalpha (alpha_max - alpha_min) sigmoid(a_raw) (1 - sigmoid(a_raw))
+ *     db = dtheta theta_max (1 - tanh(b_raw)^2)
+ *     dc = dbeta sigmoid(c_raw) (1 - sigmoid(c_raw))
+ *     dk_raw = s dk - s^2 (dk . k_raw) k_raw / |k_raw|,     s = 1 / (|k_raw| + eps)      (a zero key: s dk)
+ *
+ * Layouts, dtypes, scalars and errors as sfda_frontend; dalpha, dtheta, da, db like alpha; dbeta, dc like beta;
+ * dk, dk_raw like k.  Every output may alias the gradient it is computed from.  fp32 arithmetic, one launch.
+ */
+SFDA_API int sfda_frontend_backward(const float *a_raw, const float *b_raw, const float *c_raw, const void *k_raw,
+                                    float alpha_min, float alpha_max, float theta_max, float eps,
+                                    const float *dalpha, const float *dtheta, const float *dbeta, const void *dk,
+                                    float *da, float *db, float *dc, void *dk_raw,
+                                    int B, int T, int H, int d_k, int dtype, void *stream);
+
+/*
  * sfda_forward on the raw inputs: the stable parameterisation above followed by the chunkwise forward, without
  * the caller ever holding alpha, theta, beta or the normalised key.
  *

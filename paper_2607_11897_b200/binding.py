@@ -62,6 +62,7 @@ def load():
     lib.sfda_forward_two_level.argtypes = [_vp] * 10 + [_ci] * 8 + [_vp, _sz, _vp]
     lib.sfda_step_decoupled.argtypes = [_vp] * 11 + [_ci] * 5 + [_vp]
     lib.sfda_forward_decoupled.argtypes = [_vp] * 12 + [_ci] * 6 + [_vp]
+    lib.sfda_frontend_backward.argtypes = [_vp] * 4 + [_cf] * 4 + [_vp] * 8 + [_ci] * 5 + [_vp]
     lib.sfda_step_blocks.argtypes = [_vp] * 12 + [_ci] * 6 + [_vp]
     lib.sfda_forward_blocks.argtypes = [_vp] * 13 + [_ci] * 7 + [_vp]
     _LIB = lib
@@ -394,3 +395,22 @@ def sfda_forward_blocks(q, k, r, v, alpha, theta, flip, eta, beta, S0, o, o_im, 
                                     _dtype_code(q), int(erase), _stream(stream))
     if rc != 0:
         raise SfdaError(rc, "sfda_forward_blocks")
+
+
+def sfda_frontend_backward(a_raw, b_raw, c_raw, k_raw, alpha_min, alpha_max, theta_max, eps, dalpha, dtheta, dbeta, dk,
+                           da, db, dc, dk_raw, stream=None):
+    """``sfda_frontend_backward`` of ``include/sfda.h``: gradients with respect to the raw inputs of the stable
+    parameterisation from the gradients with respect to alpha, theta, beta and the normalised key."""
+    B, T, H, d_k = k_raw.shape
+    _check(k_raw, "k_raw")
+    for t, n in ((dk, "dk"), (dk_raw, "dk_raw")):
+        _check(t, n, k_raw.dtype)
+    for t, n in ((a_raw, "a_raw"), (b_raw, "b_raw"), (c_raw, "c_raw"), (dalpha, "dalpha"), (dtheta, "dtheta"),
+                 (dbeta, "dbeta"), (da, "da"), (db, "db"), (dc, "dc")):
+        _check(t, n, torch.float32)
+    rc = load().sfda_frontend_backward(_ptr(a_raw), _ptr(b_raw), _ptr(c_raw), _ptr(k_raw), alpha_min, alpha_max,
+                                       theta_max, eps, _ptr(dalpha), _ptr(dtheta), _ptr(dbeta), _ptr(dk), _ptr(da),
+                                       _ptr(db), _ptr(dc), _ptr(dk_raw), B, T, H, d_k, _dtype_code(k_raw),
+                                       _stream(stream))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_frontend_backward")

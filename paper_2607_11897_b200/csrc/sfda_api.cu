@@ -509,6 +509,31 @@ int sfda_frontend(const float *a_raw, const float *b_raw, const float *c_raw, co
                                                                                                          : SFDA_ERR_CUDA;
 }
 
+int sfda_frontend_backward(const float *a_raw, const float *b_raw, const float *c_raw, const void *k_raw,
+                           float alpha_min, float alpha_max, float theta_max, float eps, const float *dalpha,
+                           const float *dtheta, const float *dbeta, const void *dk, float *da, float *db, float *dc,
+                           void *dk_raw, int B, int T, int H, int d_k, int dtype, void *stream)
+{
+    g_last_launches = 0;
+    if (!a_raw || !b_raw || !c_raw || !k_raw || !dalpha || !dtheta || !dbeta || !dk || !da || !db || !dc || !dk_raw)
+        return SFDA_ERR_NULL;
+    if (B < 1 || T < 1 || H < 1) return SFDA_ERR_SHAPE;
+    int rc = check_dims(d_k, 64, 64, dtype);
+    if (rc != SFDA_OK) return rc;
+    if ((rc = check_param_scalars(alpha_min, alpha_max, theta_max, eps)) != SFDA_OK) return rc;
+    const void *ptrs[] = {a_raw, b_raw, c_raw, k_raw, dalpha, dtheta, dbeta, dk, da, db, dc, dk_raw};
+    for (const void *p : ptrs)
+        if (!aligned16(p)) return SFDA_ERR_ALIGN;
+    sfda::FrontendArgs f;
+    f.a_raw = a_raw; f.b_raw = b_raw; f.c_raw = c_raw; f.k_raw = k_raw;
+    f.alpha = da; f.theta = db; f.beta = dc; f.k = dk_raw;
+    f.rows = (long long)B * T * H; f.d_k = d_k; f.dtype = dtype;
+    f.alpha_min = alpha_min; f.alpha_max = alpha_max; f.theta_max = theta_max; f.eps = eps;
+    f.backward = 1; f.dalpha = dalpha; f.dtheta = dtheta; f.dbeta = dbeta; f.dk = dk;
+    return sfda::launch_frontend(f, static_cast<cudaStream_t>(stream), &g_last_launches) == cudaSuccess ? SFDA_OK
+                                                                                                         : SFDA_ERR_CUDA;
+}
+
 size_t sfda_forward_fused_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int dtype)
 {
     if (B < 1 || T < 1 || H < 1 || check_dims(d_k, d_v, chunk, dtype) != SFDA_OK) return 0;

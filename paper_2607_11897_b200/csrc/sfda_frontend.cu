@@ -85,6 +85,90 @@ sfda_frontend_kernel(const float *__restrict__ a_raw, const float *__restrict__ 
     }
 }
 
+// The derivative of the same map: gradients with respect to alpha, theta, beta, k in, gradients with respect to the
+// raw inputs out,
+//
+//     da = dalpha (alpha_max - alpha_min) sigmoid(a) (1 - sigmoid(a))      db = dtheta theta_max (1 - tanh(b)^2)
+//     dc = dbeta sigmoid(c) (1 - sigmoid(c))       dk_raw = s dk - s^2 (dk . k_raw) k_raw / |k_raw|,  s = 1 / (|k_raw| + eps)
+//
+// (a zero key passes s dk through).  Same mapping of warps to rows; HBM-bound: two reads and one write of the
+// forward's arrays.
+template <int DK, typename T>
+__global__ void __launch_bounds__(kFrontThreads)
+sfda_frontend_backward_kernel(const float *__restrict__ a_raw, const float *__restrict__ b_raw,
+                              const float *__restrict__ c_raw, const T *__restrict__ k_raw,
+                              const float *__restrict__ dalpha, const float *__restrict__ dtheta,
+                              const float *__restrict__ dbeta, const T *__restrict__ dk, float *__restrict__ da,
+                              float *__restrict__ db, float *__restrict__ dc, T *__restrict__ dk_raw, long long rows,
+                              float a_range, float th_max, float eps)
+{
+    constexpr int CPL = DK / 32, MPL = CPL / 2;
+    using KV = Vec<T, CPL>;
+    using FV = Vec<float, MPL>;
+    constexpr int kRows = 2;          // rows in flight per warp (four were slower: 1.27 ms against 0.97 ms)
+    const int lane = threadIdx.x & 31;
+    const long long warp = (long long)blockIdx.x * (kFrontThreads / 32) + (threadIdx.x >> 5);
+    const long long n_warps = (long long)gridDim.x * (kFrontThreads / 32);
+    for (long long r0 = warp * kRows; r0 < rows; r0 += n_warps * kRows) {
+        KV kv[kRows], gv[kRows];
+        FV av[kRows], bv[kRows], gav[kRows], gbv[kRows];
+        float cv[kRows], gcv[kRows];
+#pragma unroll
+        for (int i = 0; i < kRows; ++i) {
+            const long long r = r0 + i;
+            if (r < rows) {
+                kv[i] = reinterpret_cast<const KV *>(k_raw + r * DK)[lane];
+                gv[i] = reinterpret_cast<const KV *>(dk + r * DK)[lane];
+                av[i] = reinterpret_cast<const FV *>(a_raw + r * (DK / 2))[lane];
+                bv[i] = reinterpret_cast<const FV *>(b_raw + r * (DK / 2))[lane];
+                gav[i] = reinterpret_cast<const FV *>(dalpha + r * (DK / 2))[lane];
+                gbv[i] = reinterpret_cast<const FV *>(dtheta + r * (DK / 2))[lane];
+                cv[i] = c_raw[r];
+                gcv[i] = dbeta[r];
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < kRows; ++i) {
+            const long long r = r0 + i;
+            if (r >= rows) break;                    // uniform over the warp
+            float kf[CPL], gf[CPL], ss = 0.f, dot = 0.f;
+#pragma unroll
+            for (int x = 0; x < CPL; ++x) {
+                kf[x] = ld_val(kv[i].x, x);
+                gf[x] = ld_val(gv[i].x, x);
+                ss = fmaf(kf[x], kf[x], ss);
+                dot = fmaf(gf[x], kf[x], dot);
+            }
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) {
+                ss += __shfl_xor_sync(0xffffffffu, ss, d);
+                dot += __shfl_xor_sync(0xffffffffu, dot, d);
+            }
+            const float n = sqrtf(ss);
+            const float s = 1.0f / fmaxf(n + eps, 1.0e-30f);
+            const float w = n > 0.f ? s * s * dot / n : 0.f;
+            KV ko;
+            FV ao, bo;
+#pragma unroll
+            for (int x = 0; x < CPL; ++x) st_val(ko.x, x, fmaf(s, gf[x], -w * kf[x]));
+#pragma unroll
+            for (int x = 0; x < MPL; ++x) {
+                const float sg = 1.0f / (1.0f + expf(-av[i].x[x]));
+                const float th = tanhf(bv[i].x[x]);
+                ao.x[x] = gav[i].x[x] * a_range * sg * (1.0f - sg);
+                bo.x[x] = gbv[i].x[x] * th_max * (1.0f - th * th);
+            }
+            reinterpret_cast<KV *>(dk_raw + r * DK)[lane] = ko;
+            reinterpret_cast<FV *>(da + r * (DK / 2))[lane] = ao;
+            reinterpret_cast<FV *>(db + r * (DK / 2))[lane] = bo;
+            if (lane == 0) {
+                const float sg = 1.0f / (1.0f + expf(-cv[i]));
+                dc[r] = gcv[i] * sg * (1.0f - sg);
+            }
+        }
+    }
+}
+
 template <int DK, typename T>
 cudaError_t launch_typed(const FrontendArgs &a, cudaStream_t stream, int *launches)
 {
@@ -96,9 +180,15 @@ cudaError_t launch_typed(const FrontendArgs &a, cudaStream_t stream, int *launch
     if ((e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     const long long cap = (long long)n_sm * 8 * 4;      // a few waves of resident blocks, then the grid strides
     if (blocks > cap) blocks = cap;
-    sfda_frontend_kernel<DK, T><<<(unsigned)blocks, kFrontThreads, 0, stream>>>(
-        a.a_raw, a.b_raw, a.c_raw, static_cast<const T *>(a.k_raw), a.alpha, a.theta, a.beta, static_cast<T *>(a.k),
-        a.rows, a.alpha_min, a.alpha_max - a.alpha_min, a.theta_max, a.eps);
+    if (a.backward)
+        sfda_frontend_backward_kernel<DK, T><<<(unsigned)blocks, kFrontThreads, 0, stream>>>(
+            a.a_raw, a.b_raw, a.c_raw, static_cast<const T *>(a.k_raw), a.dalpha, a.dtheta, a.dbeta,
+            static_cast<const T *>(a.dk), a.alpha, a.theta, a.beta, static_cast<T *>(a.k), a.rows,
+            a.alpha_max - a.alpha_min, a.theta_max, a.eps);
+    else
+        sfda_frontend_kernel<DK, T><<<(unsigned)blocks, kFrontThreads, 0, stream>>>(
+            a.a_raw, a.b_raw, a.c_raw, static_cast<const T *>(a.k_raw), a.alpha, a.theta, a.beta, static_cast<T *>(a.k),
+            a.rows, a.alpha_min, a.alpha_max - a.alpha_min, a.theta_max, a.eps);
     e = cudaGetLastError();
     if (e == cudaSuccess && launches) ++*launches;
     return e;

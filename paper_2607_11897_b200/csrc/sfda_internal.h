@@ -56,6 +56,11 @@ struct FrontendArgs {
     long long rows;      // B * T * H
     int d_k, dtype;
     float alpha_min, alpha_max, theta_max, eps;
+    // backward != 0: the derivative of the map; dalpha, dtheta, dbeta, dk are the incoming gradients and the four
+    // output fields above receive da, db, dc, dk_raw
+    int backward = 0;
+    const float *dalpha = nullptr, *dtheta = nullptr, *dbeta = nullptr;
+    const void *dk = nullptr;
 };
 
 struct BackwardArgs {

@@ -91,6 +91,17 @@ def test_stable_parameterisation_entry_points_validate_on_the_host(lib):
         return lib.sfda_frontend(*ptrs[:4], *[cf(x) for x in scal], *ptrs[4:], *[ci(d) for d in dims], None)
 
     ptrs, scal, dims = [ok] * 8, [0.0, 1.0, 3.0, 1e-6], [1, 8, 1, 128, 1]
+
+    def front_bwd(ptrs12, scal, dims):
+        return lib.sfda_frontend_backward(*ptrs12[:4], *[cf(x) for x in scal], *ptrs12[4:], *[ci(d) for d in dims], None)
+
+    lib.sfda_frontend_backward.restype = ci
+    p12 = [ok] * 12                     # a, b, c, k_raw | dalpha, dtheta, dbeta, dk | da, db, dc, dk_raw
+    assert front_bwd(p12[:7] + [None] + p12[8:], scal, dims) == -1          # dk
+    assert front_bwd(p12[:11] + [None], scal, dims) == -1                     # dk_raw
+    assert front_bwd(p12, scal, [1, 8, 1, 96, 1]) == -3
+    assert front_bwd(p12[:4] + [vp(0x1004)] + p12[5:], scal, dims) == -4
+    assert front_bwd(p12, [0.6, 0.5, 3.0, 0.0], dims) == -8
     assert front(ptrs[:3] + [None] + ptrs[4:], scal, dims) == -1
     assert front(ptrs, scal, [1, 0, 1, 128, 1]) == -2
     assert front(ptrs, scal, [1, 8, 1, 96, 1]) == -3

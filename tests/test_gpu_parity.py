@@ -512,6 +512,86 @@ def test_frontend_matches_oracle(d_k, dtype, rows, par):
     assert torch.equal(d["k_raw"], k)
 
 
+@pytest.mark.parametrize("d_k,dtype,rows", [(128, "bf16", (2, 37, 3)), (64, "f32", (1, 130, 2)), (128, "f32", (1, 65, 5))])
+@pytest.mark.parametrize("par", [PARAM, dict(alpha_min=0.25, alpha_max=0.875, theta_max=0.5, eps=1e-3)])
+def test_frontend_backward_matches_oracle(d_k, dtype, rows, par):
+    """Gradients with respect to the raw inputs of the stable parameterisation; a zero key passes s dk through; the
+    outputs may alias the incoming gradients."""
+    B, T, H = rows
+    cfg = workloads.CONFIGS[0].scaled(name="feb", B=B, T=T, H=H, d_k=d_k, d_v=64, dtype=dtype, seed=45 + d_k)
+    raw = workloads.forward_raw_inputs(cfg)
+    raw["a_raw"][0, 0, 0, :4] = [-100.0, 100.0, -20.0, 20.0]
+    raw["b_raw"][0, 0, 0, :4] = [-50.0, 50.0, 0.0, 1e-4]
+    raw["k_raw"][0, 1, 0] = 0.0
+    rng = np.random.default_rng([cfg.seed, 3])
+    rnd = (lambda x: workloads.bf16_round(x)) if dtype == "bf16" else (lambda x: x.astype(np.float32))
+    g_al = rng.standard_normal(raw["a_raw"].shape, dtype=np.float32)
+    g_th = rng.standard_normal(raw["a_raw"].shape, dtype=np.float32)
+    g_be = rng.standard_normal(raw["c_raw"].shape, dtype=np.float32)
+    g_k = rnd(rng.standard_normal(raw["k_raw"].shape, dtype=np.float32))
+    d = raw_to_dev(raw, cfg)
+    dt = d["k_raw"].dtype
+    t = lambda x, ty=torch.float32: torch.from_numpy(np.ascontiguousarray(x)).to(DEV).to(ty)
+    ga, gt, gb, gk = t(g_al), t(g_th), t(g_be), t(g_k, dt)
+    da, db, dc, dkr = torch.empty_like(ga), torch.empty_like(gt), torch.empty_like(gb), torch.empty_like(gk)
+    sfda.sfda_frontend_backward(d["a_raw"], d["b_raw"], d["c_raw"], d["k_raw"], par["alpha_min"], par["alpha_max"],
+                                par["theta_max"], par["eps"], ga, gt, gb, gk, da, db, dc, dkr)
+    torch.cuda.synchronize()
+    assert sfda.last_launch_count() == 1
+    w = frontend.stable_parameterisation_backward(raw["a_raw"], raw["b_raw"], raw["c_raw"], raw["k_raw"],
+                                                  par["alpha_min"], par["alpha_max"], par["theta_max"], par["eps"],
+                                                  g_al, g_th, g_be, g_k)
+    for got, want, tol in ((da, w[0], 1e-5), (db, w[1], 1e-5), (dc, w[2], 1e-5),
+                           (dkr, w[3], 2.0 ** -8 if dtype == "bf16" else 1e-5)):
+        assert rel_err(got.float().cpu().numpy(), want) <= tol
+    # in place
+    sfda.sfda_frontend_backward(d["a_raw"], d["b_raw"], d["c_raw"], d["k_raw"], par["alpha_min"], par["alpha_max"],
+                                par["theta_max"], par["eps"], ga, gt, gb, gk, ga, gt, gb, gk)
+    torch.cuda.synchronize()
+    assert torch.equal(ga, da) and torch.equal(gt, db) and torch.equal(gb, dc) and torch.equal(gk, dkr)
+
+
+def test_gradients_with_respect_to_raw_inputs_end_to_end():
+    """A training step's backward on raw inputs: sfda_frontend, then sfda_backward on its outputs, then
+    sfda_frontend_backward -- against the oracle's composition of the same three maps."""
+    cfg = workloads.CONFIGS[0].scaled(name="e2eb", B=1, T=96, H=2, d_k=128, d_v=128, dtype="f32", s0_std=0.3, seed=46)
+    raw = workloads.forward_raw_inputs(cfg)
+    inp = workloads.forward_inputs(cfg)            # q, v, S0 of the same shapes
+    par = PARAM
+    d = raw_to_dev(raw, cfg)
+    q, v, S0 = (to_dev(inp[k], cfg, k) for k in ("q", "v", "S0"))
+    al, th = torch.empty_like(d["a_raw"]), torch.empty_like(d["a_raw"])
+    be, k = torch.empty_like(d["c_raw"]), torch.empty_like(d["k_raw"])
+    sfda.sfda_frontend(d["a_raw"], d["b_raw"], d["c_raw"], d["k_raw"], par["alpha_min"], par["alpha_max"],
+                       par["theta_max"], par["eps"], al, th, be, k)
+    up = upstream(cfg, 9)
+    g = dict(dq=torch.empty_like(q), dk=torch.empty_like(k), dv=torch.empty_like(v), dalpha=torch.empty_like(al),
+             dtheta=torch.empty_like(th), dbeta=torch.empty_like(be), dS0=torch.empty_like(S0))
+    ws = torch.empty(sfda.sfda_backward_workspace_bytes(cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, 0), dtype=torch.uint8,
+                     device=DEV)
+    tdev = lambda x: torch.from_numpy(np.ascontiguousarray(x)).to(DEV)
+    sfda.sfda_backward(q, k, v, al, th, be, S0, tdev(up["do_re"]), tdev(up["do_im"]), tdev(up["dS_T"]), g["dq"], g["dk"],
+                       g["dv"], g["dalpha"], g["dtheta"], g["dbeta"], g["dS0"], ws)
+    da, db, dc, dkr = (torch.empty_like(x) for x in (al, th, be, k))
+    sfda.sfda_frontend_backward(d["a_raw"], d["b_raw"], d["c_raw"], d["k_raw"], par["alpha_min"], par["alpha_max"],
+                                par["theta_max"], par["eps"], g["dalpha"], g["dtheta"], g["dbeta"], g["dk"], da, db, dc,
+                                dkr)
+    torch.cuda.synchronize()
+    w_al, w_th, w_be, w_k = frontend.stable_parameterisation(raw["a_raw"], raw["b_raw"], raw["c_raw"], raw["k_raw"], **par)
+    pairs = all_pairs(cfg)
+    sel = lambda x: np.stack([x[b, :, h] for b, h in pairs]).astype(np.float64)
+    S0n = np.stack([inp["S0"][b, h] for b, h in pairs]).astype(np.float64)
+    dST = np.stack([up["dS_T"][b, h] for b, h in pairs]).astype(np.float64)
+    wb = backward.sfda_backward(sel(inp["q"]), sel(w_k), sel(inp["v"]), sel(w_al), sel(w_th), sel(w_be), S0n,
+                                sel(up["do_re"]), sel(up["do_im"]), dST)
+    unsel = lambda x, like: np.stack([x[i] for i in range(len(pairs))]).reshape(cfg.B, cfg.H, *x.shape[1:]).swapaxes(1, 2)
+    wr = frontend.stable_parameterisation_backward(raw["a_raw"], raw["b_raw"], raw["c_raw"], raw["k_raw"], par["alpha_min"],
+                                                   par["alpha_max"], par["theta_max"], par["eps"], unsel(wb[3], None),
+                                                   unsel(wb[4], None), unsel(wb[5], None), unsel(wb[1], None))
+    for got, want in zip((da, db, dc, dkr), wr):
+        assert rel_err(got.float().cpu().numpy(), want) <= 2e-4
+
+
 def test_frontend_zero_key_with_zero_eps_stays_zero():
     cfg = workloads.CONFIGS[0].scaled(name="fe0", B=1, T=8, H=2, d_k=128, dtype="bf16", seed=5)
     raw = workloads.forward_raw_inputs(cfg)
