@@ -1418,3 +1418,55 @@ def test_calls_can_be_captured_in_a_cuda_graph():
     assert sfda.sfda_workspace_status(ws) == 0 and sfda.sfda_workspace_status(ws2) == 0
     for got, w in zip(outs, want):
         assert torch.equal(got, w)
+
+
+def test_concurrent_calls_from_host_threads():
+    """Four host threads, each with its own stream, buffers and workspace, call the tensor-core forward 20 times
+    at once (the binding releases the interpreter lock during a call): every result equals the serial one bit for
+    bit, and no bounded device-side wait runs out although the persistent kernels compete for the SMs."""
+    import threading
+    d = 128
+
+    def make(seed, B, T, H):
+        g = torch.Generator(device=DEV)
+        g.manual_seed(seed)
+        rn = lambda *s: torch.randn(*s, device=DEV, generator=g)
+        q, v = rn(B, T, H, d).to(torch.bfloat16), rn(B, T, H, d).to(torch.bfloat16)
+        k = rn(B, T, H, d)
+        k = (k / k.norm(dim=-1, keepdim=True)).to(torch.bfloat16)
+        a = torch.sigmoid(3.0 + rn(B, T, H, d // 2))
+        b = (torch.rand(B, T, H, d // 2, device=DEV, generator=g) * 2 - 1) * np.pi
+        return (q, k, v, a, b, torch.sigmoid(rn(B, T, H)), 0.02 * rn(B, H, d, d))
+
+    def run(x, reps):
+        B, T, H = x[0].shape[:3]
+        stream, outs = torch.cuda.Stream(), []
+        with torch.cuda.stream(stream):
+            for _ in range(reps):
+                o = torch.empty(B, T, H, d, device=DEV, dtype=torch.bfloat16)
+                o_im, S_T = torch.empty_like(o), torch.empty(B, H, d, d, device=DEV)
+                ws = torch.empty(sfda.sfda_workspace_bytes(B, T, H, d, d, 64, 1), dtype=torch.uint8, device=DEV)
+                sfda.sfda_forward(*x, o, o_im, S_T, 64, ws, stream)
+                outs.append((o, o_im, S_T, ws))
+            stream.synchronize()
+        return outs
+
+    torch.cuda.synchronize()
+    xs = [make(1, 2, 2048, 16), make(2, 1, 4096, 40), make(3, 4, 1024, 8), make(4, 3, 1536 + 7, 11)]
+    serial = [run(x, 1)[0] for x in xs]
+    res = [None] * len(xs)
+
+    def worker(i):
+        res[i] = run(xs[i], 20)
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(len(xs))]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    for i in range(len(xs)):
+        assert res[i] is not None
+        for out in res[i]:
+            assert sfda.sfda_workspace_status(out[3]) == 0
+            for a, b in zip(out[:3], serial[i][:3]):
+                assert torch.equal(a, b)
