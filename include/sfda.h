@@ -88,7 +88,15 @@ SFDA_API int sfda_plan(int T, int chunk, int *n_chunks, int *tail_len);
  * needs none).  The tensor-core path keeps a 256-byte status block there and, when it
  * gets the full size (256 + 4*B*H rounded up to 256 + B*H*d_k*d_v*4 bytes), also the
  * boundary states of the time slices it may cut long sequences into to keep every SM
- * busy; with at least 256 bytes it still runs, one (batch, head) pair per CTA at a time.  Returns 0 for invalid sizes as well; sfda_forward reports those.
+ * busy; with at least 256 bytes it still runs, one (batch, head) pair per CTA at a time.  Returns 0 for invalid
+ * sizes as well; sfda_forward reports those.
+ *
+ * Concurrency: calls may come from several host threads and streams, each with its own buffers and workspace.
+ * With time slices, a CTA of the persistent kernel waits (bounded: about a second, then SFDA_ERR_TIMEOUT through
+ * sfda_workspace_status) for the CTA that runs the previous slice of its sequence; this assumes that all CTAs of one
+ * launch become resident before those of a launch enqueued later on another stream take the SMs they need, which
+ * is how grids are dispatched today.  A caller that cannot rely on that gives the concurrent calls 256-byte
+ * workspaces (no time slices) or keeps them on one stream.
  */
 SFDA_API size_t sfda_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int dtype);
 
