@@ -93,10 +93,11 @@ SFDA_API int sfda_plan(int T, int chunk, int *n_chunks, int *tail_len);
  *
  * Concurrency: calls may come from several host threads and streams, each with its own buffers and workspace.
  * With time slices, a CTA of the persistent kernel waits (bounded: about a second, then SFDA_ERR_TIMEOUT through
- * sfda_workspace_status) for the CTA that runs the previous slice of its sequence; this assumes that all CTAs of one
- * launch become resident before those of a launch enqueued later on another stream take the SMs they need, which
- * is how grids are dispatched today.  A caller that cannot rely on that gives the concurrent calls 256-byte
- * workspaces (no time slices) or keeps them on one stream.
+ * sfda_workspace_status) for the CTA that runs the previous slice of its sequence, so all CTAs of one launch have to
+ * be resident together.  Time-sliced launches are therefore cooperative launches (at most one CTA per SM): the
+ * driver starts such a grid only when all of it fits beside whatever other streams are running, and the call
+ * returns the CUDA error instead of launching when the grid can never fit (a context limited to fewer SMs than the
+ * device has).
  */
 SFDA_API size_t sfda_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int dtype);
 

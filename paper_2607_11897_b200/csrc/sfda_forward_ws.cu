@@ -1447,10 +1447,24 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
     p.th_max = a.theta_max;
     p.th_m2 = -2.0f * a.theta_max;
     p.eps = a.eps;
+    // With time slices a CTA waits for the CTA that runs the previous slice of its sequence, so all CTAs of the
+    // launch have to be resident together: a cooperative launch makes the driver guarantee just that, whatever else
+    // is running on other streams.  (Never more CTAs than SMs, one per SM: the grid always fits.)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = Q > 1 ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     if (fused)
-        sfda_forward_ws_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(maps, p);
+        e = cudaLaunchKernelEx(&cfg, sfda_forward_ws_kernel<true>, maps, p);
     else
-        sfda_forward_ws_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(maps, p);
+        e = cudaLaunchKernelEx(&cfg, sfda_forward_ws_kernel<false>, maps, p);
+    if (e != cudaSuccess) return e;
     e = cudaGetLastError();
     if (e == cudaSuccess && launches) ++*launches;
     return e;
