@@ -92,9 +92,11 @@ SFDA_API int sfda_plan(int T, int chunk, int *n_chunks, int *tail_len);
  * sizes as well; sfda_forward reports those.
  *
  * Concurrency: calls may come from several host threads and streams, each with its own buffers and workspace.
- * With time slices, a CTA of the persistent kernel waits (bounded: about a second, then SFDA_ERR_TIMEOUT through
- * sfda_workspace_status) for the CTA that runs the previous slice of its sequence, so all CTAs of one launch have to
- * be resident together.  Time-sliced launches are therefore cooperative launches (at most one CTA per SM): the
+ * When sequences are cut (time slices, or, with at least as many sequences as SMs and a chunk count that does
+ * not halve, one contiguous range of chunks per CTA), a CTA of the persistent kernel waits (bounded: about a
+ * second, then SFDA_ERR_TIMEOUT through sfda_workspace_status) for the CTA that runs the previous piece of its
+ * sequence, so all CTAs of one launch have to
+ * be resident together.  Such launches are therefore cooperative launches (at most one CTA per SM): the
  * driver starts such a grid only when all of it fits beside whatever other streams are running, and the call
  * returns the CUDA error instead of launching when the grid can never fit (a context limited to fewer SMs than the
  * device has).

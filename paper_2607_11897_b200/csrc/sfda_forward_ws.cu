@@ -127,11 +127,12 @@ struct Params {
     const float *alpha, *theta, *beta, *S0;
     float *S_T;
     uint32_t *status;
-    uint32_t *flags;     // [B*H] progress counters of the time slices (only used when Q > 1)
-    float *handoff;      // [B*H][d_k][d_v] boundary states between time slices (only used when Q > 1)
+    uint32_t *flags;     // [B*H] arrival counters of the pieces of a cut sequence (only used when sequences are cut)
+    float *handoff;      // [B*H][d_k][d_v] boundary states between the pieces (only used when sequences are cut)
     int T, H, has_o_im;
     int BH, U, Q, n_units;   // sequences, chunks per work unit, time slices per sequence, Q * BH
-    uint32_t magic_BH, magic_H;   // floor(2^32 / d) + 1 (0 for d = 1): quotients by multiplication
+    int bal, NC, bal_base, bal_rem;   // balanced partition: on / off, chunks per sequence, BH * NC = grid * base + rem
+    uint32_t magic_BH, magic_H, magic_NC;   // floor(2^32 / d) + 1 (0 for d = 1): quotients by multiplication
     // fused stable parameterisation (only read by the kFused instantiation): alpha = a_lo + a_range sigmoid(a),
     // theta = th_max tanh(b), beta = sigmoid(c), k = k_raw / (|k_raw| + eps)
     float a_lo, a_range, th_max, th_m2, eps;   // th_m2 = -2 th_max
@@ -143,48 +144,90 @@ struct Maps {
     CUtensorMap v, o, oim, q, k, al, th;
 };
 
-// Work units.  A sequence is cut into Q time slices of U chunks; unit u = slice * BH + sequence.  CTA c works
-// through units c, c + gridDim, ... as ONE stream of chunks, so its pipeline never drains between units; only
-// the state pass notices a unit boundary (it writes the finished state out and takes the next one in).  A slice
-// q > 0 starts from the boundary state slice q - 1 left in `handoff`; its CTA waits for that (bounded).  Units
-// are handed out in increasing order and every CTA is resident, so the unit a CTA waits for is always already
+// Work units, in one of two partitions chosen by the launcher.
+// Sliced: a sequence is cut into Q time slices of U chunks; unit u = slice * BH + sequence; CTA c works through
+// units c, c + gridDim, ...  Units are handed out in increasing order, so the unit a CTA waits for is always already
 // running or done.
+// Balanced (only with at least as many sequences as CTAs): the B*H*NC chunks of all sequences, laid end to end,
+// are cut into gridDim contiguous ranges of equal length (to within one chunk), so a range holds whole sequences
+// plus the tail of one sequence at its start and the head of another at its end, and a sequence is cut at most
+// once.  A CTA takes the pieces of its range in DESCENDING sequence order: the head piece first, which the next
+// CTA needs only for the piece it takes last.
+// Either way a CTA's pieces form ONE stream of chunks, so its pipeline never drains between them; only the state
+// pass notices a boundary (it writes the finished state out and takes the next one in).  A piece that does not
+// start its sequence begins from the boundary state its predecessor left in `handoff`; its CTA waits for that
+// (bounded).  All CTAs are resident (cooperative launch).
 struct ChunkInfo {
-    int b, h, bh, jg, q;   // sequence, chunk index inside the sequence, time slice
-    bool first, last;      // first / last chunk of its unit
+    int b, h, bh, jg;           // sequence, chunk index inside the sequence
+    uint32_t want;              // arrivals at the sequence's counter that the piece waits for (unless seq_first)
+    bool first;                 // first chunk of its piece
+    bool seq_first, seq_last;   // the piece starts / ends its sequence
 };
-// Walks the stream chunk by chunk; the divisions happen once per unit, not once per chunk.
+// Walks the stream chunk by chunk; the quotients are taken once per piece, not once per chunk.
 struct ChunkCursor {
     ChunkInfo ci;
-    int jl, u;
+    int j_end, u;   // chunk index at which the piece ends; unit index (sliced) or first chunk of the range (balanced)
     // n / d for n * d < 2^32 from the precomputed floor(2^32 / d) + 1 (d = 1 is flagged by 0)
     static __device__ __forceinline__ int quot(int n, uint32_t magic) { return magic ? (int)__umulhi((uint32_t)n, magic) : n; }
-    __device__ __forceinline__ void set_unit(const Params &p)
+    // this CTA's range of the balanced partition: [lo, lo + n)
+    static __device__ __forceinline__ void range(const Params &p, int &lo, int &n)
     {
-        ci.q = quot(u, p.magic_BH);
-        ci.bh = u - ci.q * p.BH;
+        const int c = (int)blockIdx.x;
+        lo = c * p.bal_base + min(c, p.bal_rem);
+        n = p.bal_base + (c < p.bal_rem ? 1 : 0);
+    }
+    static __device__ __forceinline__ int stream_chunks(const Params &p)
+    {
+        if (p.bal) {
+            int lo, n;
+            range(p, lo, n);
+            return n;
+        }
+        return ((p.n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * p.U;
+    }
+    __device__ __forceinline__ void set_piece(const Params &p)
+    {
+        if (p.bal) {
+            ci.jg = max(u - ci.bh * p.NC, 0);
+            ci.seq_first = ci.jg == 0;
+            ci.want = 8u;
+        } else {
+            const int q = quot(u, p.magic_BH);
+            ci.bh = u - q * p.BH;
+            ci.jg = q * p.U;
+            j_end = ci.jg + p.U;
+            ci.seq_first = q == 0;
+            ci.seq_last = q == p.Q - 1;
+            ci.want = 8u * (uint32_t)q;
+        }
         ci.b = quot(ci.bh, p.magic_H);
         ci.h = ci.bh - ci.b * p.H;
+        ci.first = true;
     }
-    __device__ __forceinline__ void refresh(const Params &p)
+    __device__ __forceinline__ explicit ChunkCursor(const Params &p) : u((int)blockIdx.x)
     {
-        ci.jg = ci.q * p.U + jl;
-        ci.first = jl == 0;
-        ci.last = jl == p.U - 1;
-    }
-    __device__ __forceinline__ explicit ChunkCursor(const Params &p) : jl(0), u((int)blockIdx.x)
-    {
-        set_unit(p);
-        refresh(p);
+        if (p.bal) {
+            int n;
+            range(p, u, n);
+            ci.bh = quot(u + n - 1, p.magic_NC);
+            j_end = u + n - ci.bh * p.NC;
+            ci.seq_last = j_end == p.NC;
+        }
+        set_piece(p);
     }
     __device__ __forceinline__ void next(const Params &p)
     {
-        if (++jl == p.U) {
-            jl = 0;
-            u += (int)gridDim.x;
-            set_unit(p);
+        ci.first = false;
+        if (++ci.jg == j_end) {
+            if (p.bal) {
+                --ci.bh;
+                j_end = p.NC;
+                ci.seq_last = true;
+            } else {
+                u += (int)gridDim.x;
+            }
+            set_piece(p);
         }
-        refresh(p);
     }
 };
 
@@ -1060,7 +1103,7 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
             // A unit ends (chunk j - 1 was its last): its final state e^{i phi_C} a_C S goes to S_T (last time
             // slice) or to the hand-off buffer, where the CTA that runs the next slice is told about it.
             if (j > 0) {
-                float *dst = prev_ci.q == p.Q - 1 ? p.S_T : p.handoff;
+                float *dst = prev_ci.seq_last ? p.S_T : p.handoff;
                 if (dst) {
                     dst += (size_t)prev_ci.bh * DK * DV + c;
 #pragma unroll 1
@@ -1079,7 +1122,7 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
                         }
                     }
                 }
-                if (prev_ci.q < p.Q - 1) {     // one count per warp: slice q + 1 may start once all eight have arrived
+                if (!prev_ci.seq_last) {     // one count per warp: the next piece may start once all eight have arrived
                     __threadfence();
                     __syncwarp();
                     if (lane == 0) atomicAdd(p.flags + prev_ci.bh, 1u);
@@ -1089,14 +1132,14 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
 #endif
             }
             if (fin) break;
-            if (ci.q == 0) {
+            if (ci.seq_first) {
                 src = p.S0 ? p.S0 + (size_t)ci.bh * DK * DV + c : nullptr;
             } else {
                 // the boundary state of this sequence's previous time slice must have been written (eight warp
                 // counts per slice); bounded like every other wait, warp-uniform result
                 int ok = 1;
                 if (lane == 0) {
-                    const uint32_t want = 8u * (uint32_t)ci.q, t0 = (uint32_t)clock();
+                    const uint32_t want = ci.want, t0 = (uint32_t)clock();
                     uint32_t seen;
                     do {
                         asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(p.flags + ci.bh) : "memory");
@@ -1221,8 +1264,7 @@ sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
     Misc &mi = *reinterpret_cast<Misc *>(smem + OFF_MISC);
 
     const int tid = threadIdx.x, warp = tid >> 5;
-    // this CTA's stream: units blockIdx, blockIdx + gridDim, ... of U chunks each
-    const int n_chunks = ((p.n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * p.U;
+    const int n_chunks = ChunkCursor::stream_chunks(p);   // length of this CTA's stream of chunks
 
 #ifdef SFDA_WS_TIMING
     if (tid == 0 && p.timing) { p.timing[64 + 2 * blockIdx.x] = (long long)now_ns(); if (blockIdx.x == 0) p.timing[400] = clock64(); unsigned sm; asm volatile("mov.u32 %0, %smid;" : "=r"(sm)); p.timing[700 + blockIdx.x] = sm; }
@@ -1401,8 +1443,15 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
     // slices even out the last round (256 sequences on 148 SMs: two rounds of 128 chunks, or seven rounds of
     // 32); every unit boundary costs about one chunk period (the state goes through global memory and the next
     // slice waits for it).  The smallest Q within 3 % of the cheapest is taken.
+    // With at least as many sequences as SMs the balanced partition (equal contiguous ranges of the chunks of all
+    // sequences, see ChunkCursor) has no last round at all and two boundaries per CTA at most.  Its chunks are
+    // slower, though: measured per-CTA timelines show the two SMs of a TPC finishing together to the microsecond
+    // and the kernel, bound by instruction fetch, running 5 to 23 % slower per chunk once the CTAs reach their
+    // boundaries at different times and stop executing the same code in step (equal-sized slices keep them in
+    // step).  So it is taken only when its chunk count, weighted by 1.25, is still the smaller: shapes the slices
+    // cannot even out (odd chunk counts, short sequences), where it measured 21 to 22 % faster.
     const int BH = a.B * a.H, NC = (a.T + C - 1) / C;
-    int Q = 1;
+    int Q = 1, bal = 0;
     if (scratch_bytes >= forward_ws_scratch_bytes(a.B, a.H)) {
         double best = 0.0;
         for (int q = 1; q <= 8; q *= 2) {
@@ -1411,12 +1460,18 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
             const double cost = (double)((units + n_sm - 1) / n_sm) * (NC / q + 1.0);
             if (q == 1 || cost < 0.97 * best) { best = cost; Q = q; }
         }
+        const long long N = (long long)BH * NC;
+        if (BH >= n_sm && NC >= 4 && N * NC < 0x100000000ll && 1.25 * ((double)((N + n_sm - 1) / n_sm) + 2.0) < best) {
+            bal = 1;
+            Q = 1;
+        }
     }
 #ifdef SFDA_WS_TIMING
-    if (g_ws_force_q) Q = g_ws_force_q;
+    if (g_ws_force_q) { Q = g_ws_force_q; bal = 0; }
     if (g_ws_grid_cap && g_ws_grid_cap < n_sm) n_sm = g_ws_grid_cap;
 #endif
-    const size_t header = kWsMinScratchBytes + (Q > 1 ? (((size_t)BH * 4 + 255) & ~(size_t)255) : 0);
+    const bool pieces = Q > 1 || bal;   // sequences are cut: counters and boundary states in use, CTAs wait on one another
+    const size_t header = kWsMinScratchBytes + (pieces ? (((size_t)BH * 4 + 255) & ~(size_t)255) : 0);
     e = cudaMemsetAsync(scratch, 0, header, stream);
     if (e != cudaSuccess) return e;
     Params p;
@@ -1442,6 +1497,11 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
     p.magic_H = a.H > 1 ? (uint32_t)(0x100000000ull / (unsigned)a.H) + 1u : 0u;
     g_ws_last_slices = Q;
     const unsigned grid = (unsigned)(p.n_units < n_sm ? p.n_units : n_sm);
+    p.bal = bal;
+    p.NC = NC;
+    p.bal_base = (int)((long long)BH * NC / grid);
+    p.bal_rem = (int)((long long)BH * NC % grid);
+    p.magic_NC = NC > 1 ? (uint32_t)(0x100000000ull / (unsigned)NC) + 1u : 0u;
     p.a_lo = a.alpha_min;
     p.a_range = a.alpha_max - a.alpha_min;
     p.th_max = a.theta_max;
@@ -1457,7 +1517,7 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeCooperative;
-    attr[0].val.cooperative = Q > 1 ? 1 : 0;
+    attr[0].val.cooperative = pieces ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     if (fused)

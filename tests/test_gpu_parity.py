@@ -173,6 +173,30 @@ def test_forward_tensor_core_time_slices():
         assert np.array_equal(x, y)          # slicing only moves the fp32 state through memory: bit-identical
 
 
+def test_forward_tensor_core_balanced_partition():
+    """304 sequences of nine chunks (an odd count, which time slices cannot halve; the last chunk a ragged tail
+    of 63 tokens): the launcher cuts the chunks of all sequences, laid end to end, into one contiguous range per
+    CTA, so most sequences are cut once, at different places, and continue on a neighbouring CTA through the
+    workspace.  Checked against the oracle on sequences cut early, late and not at all, and bit for bit against
+    the same call with only the status block as workspace (no cuts)."""
+    cfg = workloads.CONFIGS[1].scaled(name="balanced", B=16, T=575, H=19, s0_std=0.05, seed=93)
+    inp = workloads.forward_inputs(cfg)
+    pairs = [(0, 0), (0, 1), (0, 2), (7, 9), (8, 0), (15, 17), (15, 18)]
+    check_forward(cfg, inp, pairs, TOL["bf16"])
+    d = {k: (None if v is None else to_dev(v, cfg, k)) for k, v in inp.items()}
+    outs = []
+    for nbytes in (sfda.sfda_workspace_bytes(cfg.B, cfg.T, cfg.H, 128, 128, 64, 1), 256):
+        o = torch.empty(cfg.B, cfg.T, cfg.H, cfg.d_v, device=DEV, dtype=torch.bfloat16)
+        o_im, S_T = torch.empty_like(o), torch.empty(cfg.B, cfg.H, 128, 128, device=DEV)
+        ws = torch.empty(nbytes, device=DEV, dtype=torch.uint8)
+        for _ in range(2):          # the second call finds the first call's counters in the workspace
+            sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im, S_T, 64, ws)
+            assert sfda.sfda_workspace_status(ws) == 0
+        outs.append((o.float().cpu().numpy(), o_im.float().cpu().numpy(), S_T.cpu().numpy()))
+    for x, y in zip(*outs):
+        assert np.array_equal(x, y)
+
+
 def test_forward_tensor_core_optional_outputs_and_zero_state():
     """Tensor-core path without o_im, without S_T, and with S0 = NULL (zero state)."""
     cfg = workloads.CONFIGS[1].scaled(name="tc_opt", B=1, T=300, H=2, s0_std=0.0, seed=55)
