@@ -1456,8 +1456,9 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
         double best = 0.0;
         for (int q = 1; q <= 8; q *= 2) {
             if (NC % q != 0 || NC / q < 4) break;
-            const long units = (long)BH * q;
-            const double cost = (double)((units + n_sm - 1) / n_sm) * (NC / q + 1.0);
+            // the q slices of one sequence run one after another: never fewer than q unit times
+            const long units = (long)BH * q, rounds = (units + n_sm - 1) / n_sm;
+            const double cost = (double)(rounds > q ? rounds : q) * (NC / q + 1.0);
             if (q == 1 || cost < 0.97 * best) { best = cost; Q = q; }
         }
         const long long N = (long long)BH * NC;
