@@ -729,9 +729,9 @@ def main():
         "roofline_ms": 1e3 * max(hbm_time, tensor_time),
     }
     if args.batch == 0 and args.seq_len == 0:
-        # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this kernel at B = 4 (1.940 GB,
+        # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this kernel at B = 4 (1.867 GB,
         # profiles/sfda_forward_ws_kernel_batch4_ncu_full.md), scaled by the units processed (traffic grows with B)
-        roofline["traffic"] = 1.940e9 * cfg.B / 4
+        roofline["traffic"] = 1.867e9 * cfg.B / 4
         roofline["traffic_source"] = "ncu capture at B=4 scaled to B=%d; Re+Im outputs" % cfg.B
 
     if other_mode is not None:
