@@ -11,10 +11,10 @@
 // inverse take the place of the rotated keys once the Gram sums are in registers):
 //   A  scan:     thread = (coordinate j, group of C/G tokens): log-decay and integer-phase prefix sums, rotated keys
 //   B  export:   Gamma, W, Y (coalesced over t)
-//   C  Gram:     blocks of 8 tokens.  A pair (t, i) of different blocks T > I splits its decay at the last token r
-//                of block I: a_t/a_i = (a_t/a_r)(a_r/a_i), both factors <= 1, so an 4 x 4 tile of pairs needs 8
-//                exponentials per coordinate instead of 16 and nothing overflows whatever alpha is; pairs inside a
-//                block take the ratio directly, eight lanes per pair.
+//   C  Gram:     pairs (t, i) of different 8-token blocks on the tensor cores (mma.sync, 3 x TF32), level by level
+//                of a binary split of the chunk, the decay split at the last token r of the lower half:
+//                a_t/a_i = (a_t/a_r)(a_r/a_i), both factors <= 1, so nothing overflows whatever alpha is; pairs
+//                inside a block take the ratio directly, eight lanes per pair.
 //   D  inverse:  8 x 8 diagonal blocks by substitution, then X = [[X11, 0], [-X22 N21 X11, X22]] doubling the
 //                block size until it is C.
 // Only ratios <= 1 are ever formed, so any alpha in [0, 1] is safe.
@@ -58,6 +58,28 @@ __device__ __forceinline__ void turns_cos_sin_fast(uint32_t turns, float *c, flo
     __sincosf(f * 6.283185307f, s, c);
 }
 
+// x = head + tail, both representable in TF32 (10 mantissa bits), to within 2^-22 |x|
+__device__ __forceinline__ void split_tf32(float x, uint32_t &head, uint32_t &tail)
+{
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(head) : "f"(x));
+    const float rest = x - __uint_as_float(head);
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(tail) : "f"(rest));
+}
+__device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], const uint32_t (&b)[2])
+{
+    asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+// d += a b^T with fp32-like accuracy: the small products first
+__device__ __forceinline__ void mma3_tf32(float (&d)[4], const uint32_t (&ah)[4], const uint32_t (&al)[4],
+                                          const uint32_t (&bh)[2], const uint32_t (&bl)[2])
+{
+    mma_tf32(d, al, bh);
+    mma_tf32(d, ah, bl);
+    mma_tf32(d, ah, bh);
+}
 template <int DK, int C>
 struct FacSmem {
     static constexpr int M = DK / 2;
@@ -244,53 +266,72 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
     // ---- C: N[t][i] = beta_i sum_j conj(k'_tj) k'_ij a_tj / a_ij,  i < t
     if (Mo) {
         constexpr int NB = C / 8;                          // blocks of 8 tokens
-        constexpr int kTileItems = NB * (NB - 1) / 2 * 8;  // block pair T > I: 4 tiles of 4 x 4, two halves of j
         constexpr int kPairs = NB * 28;                    // pairs (t, i), i < t, inside the blocks
-        static_assert(kTileItems <= kFacThreads && kTileItems % 8 == 0, "one tile half per thread");
-        // Off-diagonal tiles: adjacent lanes hold the two halves of the coordinates of one tile and add up at the
-        // end.  The sums stay in registers: N will overwrite the keys once everybody has read them.
-        const bool has_tile = tid < kTileItems;
-        const unsigned tile_lanes = __ballot_sync(0xffffffffu, has_tile);
-        const int half = tid & 1, tile = (tid >> 1) & 3, bp = tid >> 3;
-        int Tb = 1;
-        while (Tb * (Tb + 1) / 2 <= bp) ++Tb;              // bp = Tb (Tb - 1) / 2 + Ib
-        const int Ib = bp - Tb * (Tb - 1) / 2;
-        const int tr = 8 * Tb + 4 * (tile >> 1), ic = 8 * Ib + 4 * (tile & 1), r = 8 * Ib + 7;
-        float ar[4][4], ai[4][4];
-        if (has_tile) {
+        // Pairs of different blocks, on the tensor cores (mma.sync m16n8k8, 3 x TF32: every operand is split into
+        // a TF32 head and a TF32 tail and the three significant products are added in fp32, which keeps the sums
+        // at fp32 accuracy).  The pairs are taken level by level of a binary split of the chunk: rows of the upper
+        // half of a span of 16, 32 or 64 tokens against the columns of its lower half, with the decay split at the
+        // last token r of the lower half, a_t / a_i = (a_t / a_r)(a_r / a_i), both factors <= 1.  Job = a tile of
+        // 16 rows x 8 columns with its r; rows of the tile that do not lie past r are computed (decay clamped to
+        // 1) and dropped.  A warp has at most two jobs, which share their row operand when tile and r agree.
+        // The sums stay in registers: N will overwrite the keys once everybody has read them.
+        const int warp = tid >> 5, lane = tid & 31, fg = lane >> 2, ft = lane & 3;
+        int jm[2] = {-1, -1}, jc[2] = {0, 0}, jr[2] = {0, 0};   // row tile, first column, split token of the jobs
+        if (C == 64) {
+            if (warp < 4) { jm[0] = jm[1] = 2 + (warp >> 1); jc[0] = 16 * (warp & 1); jc[1] = jc[0] + 8; jr[0] = jr[1] = 31; }
+            else if (warp < 6) { jm[0] = jm[1] = 2 * warp - 7; jc[0] = 32 * (warp - 4); jc[1] = jc[0] + 8; jr[0] = jr[1] = jc[0] + 15; }
+            else { jm[0] = 2 * (warp - 6); jm[1] = jm[0] + 1; jc[0] = 16 * jm[0]; jc[1] = 16 * jm[1]; jr[0] = jc[0] + 7; jr[1] = jc[1] + 7; }
+        } else if (C == 32) {
+            if (warp == 0) { jm[0] = jm[1] = 1; jc[0] = 0; jc[1] = 8; jr[0] = jr[1] = 15; }
+            else if (warp < 3) { jm[0] = warp - 1; jc[0] = 16 * jm[0]; jr[0] = jc[0] + 7; }
+        } else {
+            if (warp == 0) { jm[0] = 0; jc[0] = 0; jr[0] = 7; }
+        }
+        const bool share = jm[1] == jm[0] && jr[1] == jr[0];
+        float acc[2][3][4];                                // per job: Re, and the two parts of Im = sum ar bi - sum ai br
 #pragma unroll
-            for (int x = 0; x < 4; ++x)
+        for (int n = 0; n < 2; ++n)
 #pragma unroll
-                for (int y = 0; y < 4; ++y) ar[x][y] = ai[x][y] = 0.f;
-#pragma unroll 2
-            for (int jj = 0; jj < M / 2; ++jj) {
-                const int j = 2 * jj + half;               // the two lanes of a tile read neighbouring banks
-                const float lr = sm.lg2[r * S::LS + j];
-                float2 a[4], bb[4];
+            for (int x = 0; x < 3; ++x)
 #pragma unroll
-                for (int x = 0; x < 4; ++x) {
-                    const float wa = ex2f(sm.lg2[(tr + x) * S::LS + j] - lr);      // a_t / a_r <= 1
-                    const float2 kk = sm.kp[(tr + x) * S::KS + j];
-                    a[x] = make_float2(wa * kk.x, wa * kk.y);
-                    const float wb = ex2f(lr - sm.lg2[(ic + x) * S::LS + j]);      // a_r / a_i <= 1
-                    const float2 kb = sm.kp[(ic + x) * S::KS + j];
-                    bb[x] = make_float2(wb * kb.x, wb * kb.y);
-                }
+                for (int y = 0; y < 4; ++y) acc[n][x][y] = 0.f;
+        if (jm[0] >= 0) {
+#pragma unroll 1
+            for (int ks = 0; ks < M / 8; ++ks) {
+                // the 8 coordinates of this step, chosen so that the 64-bit loads of a half-warp hit 16 different
+                // banks: fragment column c <-> coordinate jb + 4 (c % 4) + c / 4
+                const int jb = 16 * (ks >> 1) + 2 * (ks & 1) + 4 * ft;
+                uint32_t ah[2][4], al[2][4], bh_[2][2], bl[2][2];   // [re / im][fragment element], heads and tails
 #pragma unroll
-                for (int x = 0; x < 4; ++x)
+                for (int n = 0; n < 2; ++n) {
+                    if (n == 1 && jm[1] < 0) break;
+                    const int r = jr[n];
+                    if (n == 0 || !share) {
+                        const int rowA = 16 * jm[n] + fg;
 #pragma unroll
-                    for (int y = 0; y < 4; ++y) {          // conj(a) b
-                        ar[x][y] = fmaf(a[x].x, bb[y].x, fmaf(a[x].y, bb[y].y, ar[x][y]));
-                        ai[x][y] = fmaf(a[x].x, bb[y].y, fmaf(-a[x].y, bb[y].x, ai[x][y]));
+                        for (int e = 0; e < 4; ++e) {      // a0 (g, c), a1 (g + 8, c), a2 (g, c + 4), a3 (g + 8, c + 4)
+                            const int row = rowA + 8 * (e & 1), j = jb + (e >> 1);
+                            const float w = ex2f(fminf(sm.lg2[row * S::LS + j] - sm.lg2[r * S::LS + j], 0.f));
+                            const float2 kk = sm.kp[row * S::KS + j];
+                            split_tf32(w * kk.x, ah[0][e], al[0][e]);
+                            split_tf32(w * kk.y, ah[1][e], al[1][e]);
+                        }
                     }
-            }
+                    const int rowB = jc[n] + fg;
 #pragma unroll
-            for (int x = 0; x < 4; ++x)
-#pragma unroll
-                for (int y = 0; y < 4; ++y) {
-                    ar[x][y] += __shfl_xor_sync(tile_lanes, ar[x][y], 1);
-                    ai[x][y] += __shfl_xor_sync(tile_lanes, ai[x][y], 1);
+                    for (int e = 0; e < 2; ++e) {          // b0 (k = c, n = g), b1 (k = c + 4, n = g)
+                        const int j = jb + e;
+                        const float w = ex2f(sm.lg2[r * S::LS + j] - sm.lg2[rowB * S::LS + j]);   // a_r / a_i <= 1
+                        const float2 kk = sm.kp[rowB * S::KS + j];
+                        split_tf32(w * kk.x, bh_[0][e], bl[0][e]);
+                        split_tf32(w * kk.y, bh_[1][e], bl[1][e]);
+                    }
+                    mma3_tf32(acc[n][0], ah[0], al[0], bh_[0], bl[0]);   // ar br
+                    mma3_tf32(acc[n][0], ah[1], al[1], bh_[1], bl[1]);   // ai bi
+                    mma3_tf32(acc[n][1], ah[0], al[0], bh_[1], bl[1]);   // ar bi
+                    mma3_tf32(acc[n][2], ah[1], al[1], bh_[0], bl[0]);   // ai br
                 }
+            }
         }
         // Pairs inside a block take the decay ratio directly.  Eight lanes share a pair (coordinates j = lane, lane +
         // 8, ...) and add up by shuffles; the sums wait in the scan's group totals, which are no longer needed.
@@ -322,15 +363,17 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
             }
         }
         __syncthreads();           // every read of the keys is done: N goes where they were
-        if (has_tile) {            // each half writes two of the four rows
 #pragma unroll
-            for (int x = 0; x < 4; ++x)
-                if ((x >> 1) == half)
+        for (int n = 0; n < 2; ++n) {
+            if (jm[n] < 0) continue;
 #pragma unroll
-                    for (int y = 0; y < 4; ++y) {
-                        const float bt = sm.beta[ic + y];
-                        sm.nx[(tr + x) * S::NS + ic + y] = make_float2(bt * ar[x][y], bt * ai[x][y]);
-                    }
+            for (int e = 0; e < 4; ++e) {                  // c0 (g, 2c), c1 (g, 2c + 1), c2 (g + 8, 2c), c3 (g + 8, 2c + 1)
+                const int row = 16 * jm[n] + fg + 8 * (e >> 1), i = jc[n] + 2 * ft + (e & 1);
+                if (row > jr[n]) {
+                    const float bt = sm.beta[i];
+                    sm.nx[row * S::NS + i] = make_float2(bt * acc[n][0][e], bt * (acc[n][1][e] - acc[n][2][e]));
+                }
+            }
         }
         for (int pr_ = tid; pr_ < kPairs; pr_ += kFacThreads) {
             const int blk = pr_ % NB, pidx = pr_ / NB;
