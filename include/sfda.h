@@ -104,6 +104,19 @@ SFDA_API int sfda_plan(int T, int chunk, int *n_chunks, int *tail_len);
 SFDA_API size_t sfda_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int dtype);
 
 /*
+ * How sfda_forward would spread these sizes over a device of n_sm multiprocessors when given workspace_bytes of
+ * scratch (host only, integer arithmetic, nothing is launched; Section "chunkwise form": every (batch, head) pair
+ * is one serial chain of chunks, so only whole sequences or consecutive pieces of them can be shared out).
+ * Writes: slices, the number of equal time slices per sequence (1 = uncut); balanced, 1 when the chunks of
+ * all sequences, laid end to end, are instead cut into one contiguous range per CTA (ranges differ by at most one
+ * chunk; CTA c starts at chunk c*(N/ctas) + min(c, N%ctas) of the N = B*H*ceil(T/chunk)); ctas, the number of
+ * persistent CTAs.  Shapes that the tensor-core path does not take (see sfda_forward) report slices = 1,
+ * balanced = 0, ctas = 0.  Returns SFDA_ERR_NULL / SFDA_ERR_SHAPE for bad arguments.
+ */
+SFDA_API int sfda_forward_partition(int B, int T, int H, int d_k, int d_v, int chunk, int dtype,
+                                    size_t workspace_bytes, int n_sm, int *slices, int *balanced, int *ctas);
+
+/*
  * Chunkwise forward: o_t for every token and the final state, by Algorithm 1
  * ("Constructive SFDA-WY chunk summary"), Eq. "apply-transfer" and Theorem "Prefix
  * outputs inside a chunk", scanning boundary states over the chunks of every

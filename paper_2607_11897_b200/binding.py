@@ -36,6 +36,7 @@ def load():
     lib.sfda_plan.argtypes = [_ci, _ci, ctypes.POINTER(_ci), ctypes.POINTER(_ci)]
     lib.sfda_workspace_bytes.restype = _sz
     lib.sfda_workspace_bytes.argtypes = [_ci] * 7
+    lib.sfda_forward_partition.argtypes = [_ci] * 7 + [_sz, _ci] + [ctypes.POINTER(_ci)] * 3
     lib.sfda_forward.argtypes = [_vp] * 10 + [_ci] * 7 + [_vp, _sz, _vp]
     lib.sfda_forward_simt.argtypes = [_vp] * 10 + [_ci] * 7 + [_vp]
     lib.sfda_chunk_factors.argtypes = [_vp] * 9 + [_ci] * 6 + [_vp]
@@ -87,6 +88,16 @@ def sfda_plan(T: int, chunk: int):
 
 def sfda_workspace_bytes(B, T, H, d_k, d_v, chunk, dtype) -> int:
     return int(load().sfda_workspace_bytes(B, T, H, d_k, d_v, chunk, dtype))
+
+
+def sfda_forward_partition(B, T, H, d_k, d_v, chunk, dtype, workspace_bytes, n_sm):
+    """(slices, balanced, ctas) that sfda_forward would use on a device of n_sm multiprocessors (host only)."""
+    q, b, c = _ci(), _ci(), _ci()
+    rc = load().sfda_forward_partition(B, T, H, d_k, d_v, chunk, dtype, workspace_bytes, n_sm, ctypes.byref(q),
+                                       ctypes.byref(b), ctypes.byref(c))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_forward_partition")
+    return q.value, b.value, c.value
 
 
 def _ptr(t):

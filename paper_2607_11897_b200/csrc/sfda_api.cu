@@ -178,6 +178,26 @@ size_t sfda_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, in
     return sfda::forward_ws_supported(a) ? sfda::forward_ws_scratch_bytes(B, H) : 0;
 }
 
+int sfda_forward_partition(int B, int T, int H, int d_k, int d_v, int chunk, int dtype, size_t workspace_bytes,
+                           int n_sm, int *slices, int *balanced, int *ctas)
+{
+    if (!slices || !balanced || !ctas) return SFDA_ERR_NULL;
+    if (B < 1 || T < 1 || H < 1 || n_sm < 1) return SFDA_ERR_SHAPE;
+    const int rc = check_dims(d_k, d_v, chunk, dtype);
+    if (rc != SFDA_OK) return rc;
+    *slices = 1;
+    *balanced = 0;
+    *ctas = 0;
+    sfda::ForwardArgs a{};
+    a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.chunk = chunk; a.dtype = dtype;
+    if (!sfda::forward_ws_supported(a) || workspace_bytes < 256) return SFDA_OK;
+    const int BH = B * H, NC = (T + chunk - 1) / chunk;
+    sfda::forward_ws_partition(BH, NC, n_sm, workspace_bytes >= sfda::forward_ws_scratch_bytes(B, H), slices, balanced);
+    const long long units = (long long)BH * *slices;
+    *ctas = (int)(units < n_sm ? units : n_sm);
+    return SFDA_OK;
+}
+
 int sfda_forward_simt(const void *q, const void *k, const void *v, const float *alpha, const float *theta,
                       const float *beta, const float *S0, void *o, void *o_im, float *S_T, int B, int T, int H,
                       int d_k, int d_v, int chunk, int dtype, void *stream)

@@ -1423,6 +1423,40 @@ size_t forward_ws_scratch_bytes(int B, int H)
     return kWsMinScratchBytes + ((bh * 4 + 255) & ~(size_t)255) + bh * DK * DV * 4;
 }
 
+// How the launcher cuts BH sequences of NC chunks for a device of n_sm SMs (pure host arithmetic).
+void forward_ws_partition(int BH, int NC, int n_sm, bool cuts_allowed, int *slices, int *balanced)
+{
+    // Time slices per sequence: one CTA per SM works through ceil(units / SMs) units of NC / Q chunks.  More
+    // slices even out the last round (256 sequences on 148 SMs: two rounds of 128 chunks, or seven rounds of
+    // 32); every unit boundary costs about one chunk period (the state goes through global memory and the next
+    // slice waits for it).  The smallest Q within 3 % of the cheapest is taken.
+    // With at least as many sequences as SMs the balanced partition (equal contiguous ranges of the chunks of all
+    // sequences, see ChunkCursor) has no last round at all and two boundaries per CTA at most.  Its chunks are
+    // slower, though: measured per-CTA timelines show the two SMs of a TPC finishing together to the microsecond
+    // and the kernel, bound by instruction fetch, running 5 to 23 % slower per chunk once the CTAs reach their
+    // boundaries at different times and stop executing the same code in step (equal-sized slices keep them in
+    // step).  So it is taken only when its chunk count, weighted by 1.25, is still the smaller: shapes the slices
+    // cannot even out (odd chunk counts, short sequences), where it measured 21 to 22 % faster.
+    int Q = 1, bal = 0;
+    if (cuts_allowed) {
+        double best = 0.0;
+        for (int q = 1; q <= 8; q *= 2) {
+            if (NC % q != 0 || NC / q < 4) break;
+            // the q slices of one sequence run one after another: never fewer than q unit times
+            const long units = (long)BH * q, rounds = (units + n_sm - 1) / n_sm;
+            const double cost = (double)(rounds > q ? rounds : q) * (NC / q + 1.0);
+            if (q == 1 || cost < 0.97 * best) { best = cost; Q = q; }
+        }
+        const long long N = (long long)BH * NC;
+        if (BH >= n_sm && NC >= 4 && N * NC < 0x100000000ll && 1.25 * ((double)((N + n_sm - 1) / n_sm) + 2.0) < best) {
+            bal = 1;
+            Q = 1;
+        }
+    }
+    *slices = Q;
+    *balanced = bal;
+}
+
 cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratch_bytes, cudaStream_t stream, int *launches)
 {
     Maps maps;
@@ -1439,34 +1473,9 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
     if ((e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
 
-    // Time slices per sequence: one CTA per SM works through ceil(units / SMs) units of NC / Q chunks.  More
-    // slices even out the last round (256 sequences on 148 SMs: two rounds of 128 chunks, or seven rounds of
-    // 32); every unit boundary costs about one chunk period (the state goes through global memory and the next
-    // slice waits for it).  The smallest Q within 3 % of the cheapest is taken.
-    // With at least as many sequences as SMs the balanced partition (equal contiguous ranges of the chunks of all
-    // sequences, see ChunkCursor) has no last round at all and two boundaries per CTA at most.  Its chunks are
-    // slower, though: measured per-CTA timelines show the two SMs of a TPC finishing together to the microsecond
-    // and the kernel, bound by instruction fetch, running 5 to 23 % slower per chunk once the CTAs reach their
-    // boundaries at different times and stop executing the same code in step (equal-sized slices keep them in
-    // step).  So it is taken only when its chunk count, weighted by 1.25, is still the smaller: shapes the slices
-    // cannot even out (odd chunk counts, short sequences), where it measured 21 to 22 % faster.
     const int BH = a.B * a.H, NC = (a.T + C - 1) / C;
     int Q = 1, bal = 0;
-    if (scratch_bytes >= forward_ws_scratch_bytes(a.B, a.H)) {
-        double best = 0.0;
-        for (int q = 1; q <= 8; q *= 2) {
-            if (NC % q != 0 || NC / q < 4) break;
-            // the q slices of one sequence run one after another: never fewer than q unit times
-            const long units = (long)BH * q, rounds = (units + n_sm - 1) / n_sm;
-            const double cost = (double)(rounds > q ? rounds : q) * (NC / q + 1.0);
-            if (q == 1 || cost < 0.97 * best) { best = cost; Q = q; }
-        }
-        const long long N = (long long)BH * NC;
-        if (BH >= n_sm && NC >= 4 && N * NC < 0x100000000ll && 1.25 * ((double)((N + n_sm - 1) / n_sm) + 2.0) < best) {
-            bal = 1;
-            Q = 1;
-        }
-    }
+    forward_ws_partition(BH, NC, n_sm, scratch_bytes >= forward_ws_scratch_bytes(a.B, a.H), &Q, &bal);
 #ifdef SFDA_WS_TIMING
     if (g_ws_force_q) { Q = g_ws_force_q; bal = 0; }
     if (g_ws_grid_cap && g_ws_grid_cap < n_sm) n_sm = g_ws_grid_cap;

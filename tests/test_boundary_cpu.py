@@ -328,3 +328,57 @@ def test_two_process_sharding_needs_no_collective(tmp_path):
     assert np.array_equal(got, want)                              # shards simply concatenate
     assert list(dp.rank_batch_range(8, 3)) == list(range(24, 32))
     assert [len(dp.split_batch(7, 3, r)) for r in range(3)] == [3, 2, 2]
+
+
+def test_forward_partition_rules():
+    """How the forward spreads sequences over the SMs (host arithmetic of the launcher): time slices only when they
+    shorten the schedule, none with fewer sequences than SMs (a sequence's slices run one after another), the
+    balanced ranges only for shapes the slices cannot even out, nothing cut without the full workspace."""
+    full = lambda B, H: sfda.sfda_workspace_bytes(B, 8192, H, 128, 128, 64, 1)
+    part = lambda B, T, H, ws, sm=148: sfda.sfda_forward_partition(B, T, H, 128, 128, 64, 1, ws, sm)
+    assert part(8, 8192, 32, full(8, 32)) == (4, 0, 148)          # headline: 1024 units, 7 rounds of 32 chunks
+    assert part(8, 8192, 32, 256) == (1, 0, 148)                  # status block only: whole sequences
+    assert part(4, 16384, 32, full(4, 32)) == (1, 0, 128)         # 128 sequences < 148 SMs: slicing buys nothing
+    assert part(1, 131072, 16, full(1, 16)) == (1, 0, 16)
+    assert part(16, 575, 19, full(16, 19)) == (1, 1, 148)         # 304 sequences of 9 chunks: balanced ranges
+    assert part(4, 4113, 50, full(4, 50)) == (1, 1, 148)          # 200 sequences of 65 chunks
+    assert part(5, 512, 40, full(5, 40)) == (2, 0, 148)           # 200 sequences of 8 chunks: two slices suffice
+    assert part(8, 8192, 32, full(8, 32), sm=64) == (1, 0, 64)    # 256 sequences on 64 SMs: four even rounds
+    assert sfda.sfda_forward_partition(1, 256, 2, 64, 64, 16, 0, 1 << 20, 148) == (1, 0, 0)   # CUDA-core path
+    with pytest.raises(sfda.SfdaError):
+        part(0, 64, 1, 256)
+
+
+def test_balanced_ranges_cover_every_chunk_once():
+    """The contiguous ranges the header defines for the balanced partition (CTA c starts at c*(N/ctas) +
+    min(c, N % ctas)), walked the way the kernel walks them (last sequence of the range first): every chunk of
+    every sequence exactly once, a sequence cut at most once, the head piece before anything else on its CTA and
+    the tail piece last, so that no CTA waits for a piece that has not been started."""
+    for B, T, H, sm in ((16, 575, 19, 148), (4, 4113, 50, 148), (1, 256, 149, 148), (3, 960, 60, 148), (1, 320, 101, 100)):
+        slices, balanced, ctas = sfda.sfda_forward_partition(B, T, H, 128, 128, 64, 1,
+                                                             sfda.sfda_workspace_bytes(B, T, H, 128, 128, 64, 1), sm)
+        assert (slices, balanced, ctas) == (1, 1, sm)
+        BH, NC = B * H, (T + 63) // 64
+        N = BH * NC
+        base, rem = divmod(N, ctas)
+        seen, cuts = set(), {}
+        for c in range(ctas):
+            lo = c * base + min(c, rem)
+            hi = lo + base + (1 if c < rem else 0)
+            pieces = []
+            bh = (hi - 1) // NC
+            while bh * NC + NC > lo and bh >= 0:
+                j0, j1 = max(lo - bh * NC, 0), min(hi - bh * NC, NC)
+                pieces.append((bh, j0, j1))
+                bh -= 1
+            for n, (s, j0, j1) in enumerate(pieces):
+                assert j0 < j1
+                for j in range(j0, j1):
+                    assert (s, j) not in seen
+                    seen.add((s, j))
+                if j1 < NC:                    # a head piece: first on its CTA
+                    assert n == 0 and j0 == 0
+                    cuts[s] = cuts.get(s, 0) + 1
+                if j0 > 0:                     # a tail piece: last on its CTA
+                    assert n == len(pieces) - 1 and j1 == NC
+        assert len(seen) == N and all(v == 1 for v in cuts.values())

@@ -180,6 +180,10 @@ def test_forward_tensor_core_balanced_partition():
     workspace.  Checked against the oracle on sequences cut early, late and not at all, and bit for bit against
     the same call with only the status block as workspace (no cuts)."""
     cfg = workloads.CONFIGS[1].scaled(name="balanced", B=16, T=575, H=19, s0_std=0.05, seed=93)
+    n_sm = torch.cuda.get_device_properties(0).multi_processor_count
+    full = sfda.sfda_workspace_bytes(cfg.B, cfg.T, cfg.H, 128, 128, 64, 1)
+    assert sfda.sfda_forward_partition(cfg.B, cfg.T, cfg.H, 128, 128, 64, 1, full, n_sm)[:2] == (1, 1)
+    assert sfda.sfda_forward_partition(cfg.B, cfg.T, cfg.H, 128, 128, 64, 1, 256, n_sm)[:2] == (1, 0)
     inp = workloads.forward_inputs(cfg)
     pairs = [(0, 0), (0, 1), (0, 2), (7, 9), (8, 0), (15, 17), (15, 18)]
     check_forward(cfg, inp, pairs, TOL["bf16"])
