@@ -115,6 +115,16 @@ int auto_slices(int B, int T, int H, int chunk)
         return 1;
     int n = 1;
     while ((long long)2 * n * B * H <= n_sm && T % (2 * n * chunk) == 0 && T / (2 * n * chunk) >= 16) n *= 2;
+    // One more doubling puts more slices than SMs on the machine; the chunk forward then cuts them into time slices
+    // of its own and fills the SMs that n slices left idle.  Taken when its schedule is at least 8 % shorter (the
+    // scan and the correction grow a little with n): 128 slices of 256 chunks -> 256 of 128 measured 4.00 -> 3.81 ms.
+    if (n >= 4 && T % (2 * n * chunk) == 0 && T / (2 * n * chunk) >= 16) {
+        int q = 1, bal = 0;
+        double now = 0.0, then = 0.0;
+        sfda::forward_ws_partition(n * B * H, T / (n * chunk), n_sm, true, &q, &bal, &now);
+        sfda::forward_ws_partition(2 * n * B * H, T / (2 * n * chunk), n_sm, true, &q, &bal, &then);
+        if (then < 0.92 * now) n *= 2;
+    }
     return n >= 4 ? n : 1;      // three passes of T / n tokens each: fewer than four slices cannot pay
 }
 
@@ -192,7 +202,7 @@ int sfda_forward_partition(int B, int T, int H, int d_k, int d_v, int chunk, int
     a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.chunk = chunk; a.dtype = dtype;
     if (!sfda::forward_ws_supported(a) || workspace_bytes < 256) return SFDA_OK;
     const int BH = B * H, NC = (T + chunk - 1) / chunk;
-    sfda::forward_ws_partition(BH, NC, n_sm, workspace_bytes >= sfda::forward_ws_scratch_bytes(B, H), slices, balanced);
+    sfda::forward_ws_partition(BH, NC, n_sm, workspace_bytes >= sfda::forward_ws_scratch_bytes(B, H), slices, balanced, nullptr);
     const long long units = (long long)BH * *slices;
     *ctas = (int)(units < n_sm ? units : n_sm);
     return SFDA_OK;

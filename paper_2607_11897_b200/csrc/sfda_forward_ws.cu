@@ -1424,7 +1424,7 @@ size_t forward_ws_scratch_bytes(int B, int H)
 }
 
 // How the launcher cuts BH sequences of NC chunks for a device of n_sm SMs (pure host arithmetic).
-void forward_ws_partition(int BH, int NC, int n_sm, bool cuts_allowed, int *slices, int *balanced)
+void forward_ws_partition(int BH, int NC, int n_sm, bool cuts_allowed, int *slices, int *balanced, double *periods)
 {
     // Time slices per sequence: one CTA per SM works through ceil(units / SMs) units of NC / Q chunks.  More
     // slices even out the last round (256 sequences on 148 SMs: two rounds of 128 chunks, or seven rounds of
@@ -1438,8 +1438,8 @@ void forward_ws_partition(int BH, int NC, int n_sm, bool cuts_allowed, int *slic
     // step).  So it is taken only when its chunk count, weighted by 1.25, is still the smaller: shapes the slices
     // cannot even out (odd chunk counts, short sequences), where it measured 21 to 22 % faster.
     int Q = 1, bal = 0;
+    double best = (double)((BH + n_sm - 1) / n_sm) * (NC + 1.0);   // uncut: whole sequences, round after round
     if (cuts_allowed) {
-        double best = 0.0;
         for (int q = 1; q <= 8; q *= 2) {
             if (NC % q != 0 || NC / q < 4) break;
             // the q slices of one sequence run one after another: never fewer than q unit times
@@ -1451,10 +1451,12 @@ void forward_ws_partition(int BH, int NC, int n_sm, bool cuts_allowed, int *slic
         if (BH >= n_sm && NC >= 4 && N * NC < 0x100000000ll && 1.25 * ((double)((N + n_sm - 1) / n_sm) + 2.0) < best) {
             bal = 1;
             Q = 1;
+            best = (double)((N + n_sm - 1) / n_sm) + 2.0;
         }
     }
     *slices = Q;
     *balanced = bal;
+    if (periods) *periods = best;      // the schedule's length in chunk periods (what the choice was made on)
 }
 
 cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratch_bytes, cudaStream_t stream, int *launches)
@@ -1475,7 +1477,7 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
 
     const int BH = a.B * a.H, NC = (a.T + C - 1) / C;
     int Q = 1, bal = 0;
-    forward_ws_partition(BH, NC, n_sm, scratch_bytes >= forward_ws_scratch_bytes(a.B, a.H), &Q, &bal);
+    forward_ws_partition(BH, NC, n_sm, scratch_bytes >= forward_ws_scratch_bytes(a.B, a.H), &Q, &bal, nullptr);
 #ifdef SFDA_WS_TIMING
     if (g_ws_force_q) { Q = g_ws_force_q; bal = 0; }
     if (g_ws_grid_cap && g_ws_grid_cap < n_sm) n_sm = g_ws_grid_cap;

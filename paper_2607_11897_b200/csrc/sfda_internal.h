@@ -92,7 +92,7 @@ bool forward_ws_supported(const ForwardArgs &a);
 // launcher may also cut every sequence into time slices that hand their boundary state over through the scratch.
 constexpr size_t kWsMinScratchBytes = 256;
 size_t forward_ws_scratch_bytes(int B, int H);
-void forward_ws_partition(int BH, int NC, int n_sm, bool cuts_allowed, int *slices, int *balanced);
+void forward_ws_partition(int BH, int NC, int n_sm, bool cuts_allowed, int *slices, int *balanced, double *periods);
 cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratch_bytes, cudaStream_t stream,
                               int *launches);
 // The same kernel on the library's own statically allocated scratch block (kStaticScratchBytes), and a read of

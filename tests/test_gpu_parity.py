@@ -927,7 +927,7 @@ def run_two_level(cfg, inp, n_slices, want_im=True, want_state=True):
             None if S_T is None else S_T.cpu().numpy(), launches)
 
 
-@pytest.mark.parametrize("B,T,H,n_slices,s0", [(1, 2048, 2, 2, 0.3), (2, 2048, 1, 4, 0.0), (1, 4096, 3, 8, 0.3),
+@pytest.mark.parametrize("B,T,H,n_slices,s0", [(1, 2048, 2, 2, 0.3), (2, 2048, 1, 4, 0.0), (1, 4096, 3, 8, 0.3), (1, 4096, 2, 16, 0.3),
                                                (1, 2048, 2, 0, 0.3)])
 def test_forward_two_level_matches_oracle(B, T, H, n_slices, s0):
     cfg = workloads.CONFIGS[1].scaled(name="two_level", B=B, T=T, H=H, s0_std=s0, seed=90 + n_slices)
