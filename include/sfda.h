@@ -145,6 +145,28 @@ SFDA_API int sfda_forward(const void *q, const void *k, const void *v,
                  void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * sfda_forward on the tensor-core shapes (bf16, d_k = d_v = 128, chunk = 64; SFDA_ERR_UNSUPPORTED otherwise) that
+ * also writes the integer bookkeeping of the cumulative phase (Eq. "constructive-Gamma"; App. "Kernel sketch",
+ * Stage 1: phases kept as integers):
+ *
+ *  phase_turns [B][H][NC][m] uint32 (device, 16-byte aligned, NC = ceil(T / chunk)): for every chunk and complex
+ *         coordinate the phase the chunk closes with, in 2^-32 turns: the sum, modulo 2^32, over the chunk's tokens of
+ *         (uint32)(int64)rint(theta * 683565275.6f), the product taken in single precision (one IEEE multiply,
+ *         round to nearest even) and rounded to the nearest integer (ties to even).  Tokens beyond T count as 0.
+ *
+ * The kernel forms exactly these integers (per group of eight tokens, then summed; integer addition is
+ * associative, so the grouping does not show) and takes the chunk's closing rotation and every group's starting
+ * angle from them; inside a group of eight tokens gamma_t is a running single-precision complex product.  The
+ * conversion differs from sfda_chunk_factors' double-precision one by at most 2^-24 of the angle per token.
+ * All other arguments, results and errors as sfda_forward.
+ */
+SFDA_API int sfda_forward_phase(const void *q, const void *k, const void *v,
+                 const float *alpha, const float *theta, const float *beta,
+                 const float *S0, void *o, void *o_im, float *S_T, uint32_t *phase_turns,
+                 int B, int T, int H, int d_k, int d_v, int chunk, int dtype,
+                 void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * sfda_forward for few, long sequences: a two-level scan over the time axis.  A sequence is one serial chain of
  * chunks, so with fewer (batch, head) pairs than SMs most of the GPU idles.  By Theorem "Exact affine chunk
  * transfer" a time slice maps its initial state affinely, S_out = P S_in + B; so every sequence is cut into
@@ -235,8 +257,9 @@ SFDA_API int sfda_forward_simt(const void *q, const void *k, const void *v,
  *  M     [B][H][NC][C][C][2]    unit lower triangular
  *  W     [B][H][NC][m][C][2]    W[:,t] = conj(gamma_t) k_t
  *  phase_turns [B][T][H][m] uint32, or NULL: the chunk-local inclusive prefix sum,
- *         modulo 2^32, of  rint((double)theta * 2^32 / (2 pi))  -- the integer
- *         cumulative phase every kernel of this library derives gamma's angle from.
+ *         modulo 2^32, of  rint((double)theta * 2^32 / (2 pi)).  This kernel and the
+ *         fp32 forward derive gamma's angle from these integers; the tensor-core
+ *         forward sums a single-precision conversion instead (see sfda_forward_phase).
  *
  * NC = ceil(T / chunk), C = chunk.  Columns (and rows of M) of padded tail tokens
  * are those of neutral tokens (zero columns in Y and W, identity rows in M).

@@ -44,3 +44,35 @@ def cumulative_phase_turns(theta, chunk: int):
         acc = np.cumsum(u[..., start:stop, :], axis=-2, dtype=np.uint64)
         out[..., start:stop, :] = (acc & 0xFFFFFFFF).astype(np.uint32)
     return out
+
+
+# The same constant rounded to single precision (the nearest float32 to 683565275.57...), for the
+# single-precision variant of the conversion.
+TURNS_PER_RADIAN_F32 = np.float32(683565275.6)
+
+
+def phase_to_turns_f32(theta):
+    """Single-precision variant: the product theta * 2**32/(2 pi) is ONE float32 multiply (round to
+    nearest even), then rounded to the nearest integer (ties to even) and wrapped modulo 2**32."""
+    th = np.asarray(theta, dtype=np.float32)
+    prod = th * TURNS_PER_RADIAN_F32                       # float32 * float32 -> float32, IEEE
+    assert prod.dtype == np.float32
+    r = np.rint(prod.astype(np.float64))                   # exact widening, then ties-to-even rounding
+    return (r.astype(np.int64) & 0xFFFFFFFF).astype(np.uint32)
+
+
+def chunk_closing_turns_f32(theta, chunk: int):
+    """Phase every chunk closes with (Eq. "constructive-Gamma" at t = C, unit-modulus part), in 2**-32 turns:
+    the sum modulo 2**32 of phase_to_turns_f32 over the chunk's tokens.
+
+    theta: [..., T, m]  ->  [..., NC, m] uint32 with NC = ceil(T / chunk); a short last chunk sums
+    the tokens it has (missing tokens are neutral: phase 0).
+    """
+    u = phase_to_turns_f32(theta).astype(np.uint64)
+    T = u.shape[-2]
+    n_chunks, _ = chunk_plan(T, chunk)
+    out = np.empty(u.shape[:-2] + (n_chunks, u.shape[-1]), np.uint32)
+    for c in range(n_chunks):
+        seg = u[..., c * chunk:min((c + 1) * chunk, T), :]
+        out[..., c, :] = (seg.sum(axis=-2, dtype=np.uint64) & 0xFFFFFFFF).astype(np.uint32)
+    return out

@@ -39,6 +39,7 @@ def load():
     lib.sfda_forward_partition.argtypes = [_ci] * 7 + [_sz, _ci] + [ctypes.POINTER(_ci)] * 3
     lib.sfda_forward.argtypes = [_vp] * 10 + [_ci] * 7 + [_vp, _sz, _vp]
     lib.sfda_forward_simt.argtypes = [_vp] * 10 + [_ci] * 7 + [_vp]
+    lib.sfda_forward_phase.argtypes = [_vp] * 11 + [_ci] * 7 + [_vp, _sz, _vp]
     lib.sfda_chunk_factors.argtypes = [_vp] * 9 + [_ci] * 6 + [_vp]
     lib.sfda_step.argtypes = [_vp] * 9 + [_ci] * 5 + [_vp]
     lib.sfda_forward_host_arena_bytes.restype = _sz
@@ -155,6 +156,25 @@ def _forward_common(fn_name, q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chun
 def sfda_forward(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chunk, workspace=None, stream=None):
     """``sfda_forward`` of ``include/sfda.h``; tensors are CUDA tensors the caller allocated."""
     _forward_common("sfda_forward", q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chunk, workspace, stream)
+
+
+def sfda_forward_phase(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, phase_turns, chunk, workspace, stream=None):
+    """``sfda_forward_phase`` of ``include/sfda.h``: the tensor-core forward that also writes the chunk-closing
+    integer phase ``phase_turns`` ([B][H][NC][m], int32 tensor holding the uint32 bit patterns)."""
+    lib = load()
+    B, T, H, d_k = q.shape
+    d_v = v.shape[-1]
+    for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o"), (o_im, "o_im")):
+        _check(t, n, q.dtype)
+    for t, n in ((alpha, "alpha"), (theta, "theta"), (beta, "beta"), (S0, "S0"), (S_T, "S_T")):
+        _check(t, n, torch.float32)
+    _check(phase_turns, "phase_turns", torch.int32)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib.sfda_forward_phase(_ptr(q), _ptr(k), _ptr(v), _ptr(alpha), _ptr(theta), _ptr(beta), _ptr(S0), _ptr(o),
+                                _ptr(o_im), _ptr(S_T), _ptr(phase_turns), B, T, H, d_k, d_v, chunk, _dtype_code(q),
+                                _ptr(workspace), ws_bytes, _stream(stream))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_forward_phase")
 
 
 def sfda_workspace_status(workspace, stream=None) -> int:

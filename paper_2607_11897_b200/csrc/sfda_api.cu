@@ -241,6 +241,27 @@ int sfda_forward(const void *q, const void *k, const void *v, const float *alpha
     return e == cudaSuccess ? SFDA_OK : SFDA_ERR_CUDA;
 }
 
+int sfda_forward_phase(const void *q, const void *k, const void *v, const float *alpha, const float *theta,
+                       const float *beta, const float *S0, void *o, void *o_im, float *S_T, uint32_t *phase_turns,
+                       int B, int T, int H, int d_k, int d_v, int chunk, int dtype, void *workspace,
+                       size_t workspace_bytes, void *stream)
+{
+    g_last_launches = 0;
+    const int rc = validate_forward(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
+    if (rc != SFDA_OK) return rc;
+    if (!phase_turns) return SFDA_ERR_NULL;
+    if (!aligned16(phase_turns)) return SFDA_ERR_ALIGN;
+    sfda::ForwardArgs a = pack(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
+    if (!sfda::forward_ws_supported(a)) return SFDA_ERR_UNSUPPORTED;     // the export belongs to the tensor-core kernel
+    if (!workspace || workspace_bytes < sfda::kWsMinScratchBytes) return SFDA_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return SFDA_ERR_ALIGN;
+    a.phase_turns = phase_turns;
+    return sfda::launch_forward_ws(a, workspace, workspace_bytes, static_cast<cudaStream_t>(stream), &g_last_launches) ==
+                   cudaSuccess
+               ? SFDA_OK
+               : SFDA_ERR_CUDA;
+}
+
 size_t sfda_forward_two_level_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int dtype,
                                               int n_slices)
 {

@@ -126,6 +126,7 @@ struct Params {
     const __nv_bfloat16 *q, *k;
     const float *alpha, *theta, *beta, *S0;
     float *S_T;
+    uint32_t *phase_out; // [B*H][NC][64] chunk-closing phase in 2^-32 turns, or nullptr (plain instantiation only)
     uint32_t *status;
     uint32_t *flags;     // [B*H] arrival counters of the pieces of a cut sequence (only used when sequences are cut)
     float *handoff;      // [B*H][d_k][d_v] boundary states between the pieces (only used when sequences are cut)
@@ -476,8 +477,12 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
                 prev.next(p);
                 if (elect_one()) {
                     tma_store_4d(tm_o, smem + OFF_OST, 0, pc.h, pc.jg * C, pc.b);
-                    if (p.has_o_im)
-                        tma_store_4d(tm_oim, smem + OFF_AQ + ((j - 1) & 1) * 2 * kTile, 0, pc.h, pc.jg * C, pc.b);
+                    tma_store_4d(tm_o, smem + OFF_OST + kTile, 64, pc.h, pc.jg * C, pc.b);
+                    if (p.has_o_im) {
+                        const uint8_t *src = smem + OFF_AQ + ((j - 1) & 1) * 2 * kTile;
+                        tma_store_4d(tm_oim, src, 0, pc.h, pc.jg * C, pc.b);
+                        tma_store_4d(tm_oim, src + kTile, 64, pc.h, pc.jg * C, pc.b);
+                    }
                     tma_store_commit();
                     if (j < n_chunks) {
                         tma_store_wait_read();
@@ -606,20 +611,30 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
         if (jd >= 1 && !dead && !wait_k(mi, B_STORE_DONE0 + ((jd - 1) & 1), (jd - 1) >> 1)) dead = true;
         tc_fence_after();
         if (half == 0 || p.has_o_im) {
-            __nv_bfloat16 *stage =
-                reinterpret_cast<__nv_bfloat16 *>(smem + (half ? OFF_AQ + (jd & 1) * 2 * kTile : OFF_OST)) + c;
+            // Tensor memory is read in the 16-lane x 256-bit fragment shape (thread T: channel rows T / 4 and T / 4 + 8,
+            // token pairs 2 (T % 4) of every block of eight tokens), whose bf16 pairs are exactly the fragments of a
+            // transposing 8 x 8 matrix store: four matrices (one block of eight tokens x four groups of eight
+            // channels) per instruction instead of one 2-byte store per value.  The staging tiles hold 64 channels
+            // per 128-byte row in the copy engine's 128-byte swizzle, so the 32 row pieces of one store fall into
+            // different banks.
             const uint32_t flip = half ? 0x80008000u : 0u;   // o = conj(rho)
-            const uint32_t st = smem_u32(stage);
+            const int r8 = lane & 7, chunk = (quad & 1) * 4 + (lane >> 3);
+            uint32_t st = smem_u32(smem + (half ? OFF_AQ + (jd & 1) * 2 * kTile : OFF_OST)) + (quad >> 1) * kTile +
+                          (uint32_t)(r8 * 128 + ((chunk ^ r8) << 4));
+            uint32_t ta = tlane + TM_ACC + 64 + 128 * half;
 #pragma unroll 1
-            for (int pc = 0; pc < 2; ++pc) {
-                uint32_t r[32];
-                tmem_ld<32>(tlane + TM_ACC + 64 + 128 * half + 32 * pc, r);
+            for (int ch = 0; ch < 2; ++ch, st += 4 * 1024, ta += 32) {
+                uint32_t ra[16], rb[16];
+                tmem_ld_16x256b_x4(ta, ra);
+                tmem_ld_16x256b_x4(ta + (16u << 16), rb);
                 tc_wait_ld();
 #pragma unroll
-                for (int t = 0; t < 32; t += 2) {
-                    const uint32_t pk = pack_bf16(__uint_as_float(r[t]), __uint_as_float(r[t + 1])) ^ flip;
-                    sts16(st + (32 * pc + t) * 2 * DV, (uint16_t)pk);
-                    sts16(st + (32 * pc + t + 1) * 2 * DV, (uint16_t)(pk >> 16));
+                for (int i = 0; i < 4; ++i) {
+                    stmatrix_x4_trans(st + i * 1024,
+                                      pack_bf16(__uint_as_float(ra[4 * i]), __uint_as_float(ra[4 * i + 1])) ^ flip,
+                                      pack_bf16(__uint_as_float(ra[4 * i + 2]), __uint_as_float(ra[4 * i + 3])) ^ flip,
+                                      pack_bf16(__uint_as_float(rb[4 * i]), __uint_as_float(rb[4 * i + 1])) ^ flip,
+                                      pack_bf16(__uint_as_float(rb[4 * i + 2]), __uint_as_float(rb[4 * i + 3])) ^ flip);
                 }
             }
         }
@@ -733,6 +748,10 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
                 turns_sincos(tb1, &sn, &cs);
                 g1 = make_float2(base1 * cs, base1 * sn);
                 if (tq == 0) {
+                    // the integer phase the chunk closes with: what the operands' angles are derived from, exported
+                    // on request so that it can be compared bit for bit
+                    if (!kFused && p.phase_out)
+                        *reinterpret_cast<uint2 *>(p.phase_out + ((size_t)ci.bh * p.NC + ci.jg) * M + 2 * jp) = make_uint2(tb0, tb1);
                     mi.close[ring][2 * jp] = g0;
                     mi.close[ring][2 * jp + 1] = g1;
                     g0 = make_float2(1.f, 0.f); g1 = g0; base0 = 1.f; base1 = 1.f;
@@ -1343,17 +1362,19 @@ EncodeTiledFn encode_fn()
 }
 
 // [B][T][H][inner] tensor of bf16 (inner = 128) or fp32 (inner = 64), box = 64 tokens of one head.
-bool make_map(CUtensorMap *map, const void *base, int B, int T, int H, bool f32 = false)
+bool make_map(CUtensorMap *map, const void *base, int B, int T, int H, bool f32 = false, bool half_swizzled = false)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t inner = f32 ? M : DV, row = 256;      // elements, bytes per (token, head)
     const cuuint64_t dims[4] = {inner, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)B};
     const cuuint64_t strides[3] = {row, (cuuint64_t)H * row, (cuuint64_t)T * H * row};
-    const cuuint32_t box[4] = {(cuuint32_t)inner, 1, (cuuint32_t)C, 1};
+    // half_swizzled (outputs): a box is 64 tokens x 64 channels (128-byte rows) in the 128-byte swizzle
+    const cuuint32_t box[4] = {(cuuint32_t)(half_swizzled ? inner / 2 : inner), 1, (cuuint32_t)C, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     return fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base),
-              dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+              dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              half_swizzled ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -1462,8 +1483,8 @@ void forward_ws_partition(int BH, int NC, int n_sm, bool cuts_allowed, int *slic
 cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratch_bytes, cudaStream_t stream, int *launches)
 {
     Maps maps;
-    if (!make_map(&maps.v, a.v, a.B, a.T, a.H) || !make_map(&maps.o, a.o, a.B, a.T, a.H) ||
-        !make_map(&maps.oim, a.o_im ? a.o_im : a.o, a.B, a.T, a.H) || !make_map(&maps.q, a.q, a.B, a.T, a.H) ||
+    if (!make_map(&maps.v, a.v, a.B, a.T, a.H) || !make_map(&maps.o, a.o, a.B, a.T, a.H, false, true) ||
+        !make_map(&maps.oim, a.o_im ? a.o_im : a.o, a.B, a.T, a.H, false, true) || !make_map(&maps.q, a.q, a.B, a.T, a.H) ||
         !make_map(&maps.k, a.k, a.B, a.T, a.H) || !make_map(&maps.al, a.alpha, a.B, a.T, a.H, true) ||
         !make_map(&maps.th, a.theta, a.B, a.T, a.H, true))
         return cudaErrorInvalidValue;
@@ -1495,6 +1516,7 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
     p.beta = a.beta;
     p.S0 = a.S0;
     p.S_T = a.S_T;
+    p.phase_out = a.phase_turns;
     p.status = static_cast<uint32_t *>(scratch);
     p.flags = reinterpret_cast<uint32_t *>(static_cast<char *>(scratch) + kWsMinScratchBytes);
     p.handoff = reinterpret_cast<float *>(static_cast<char *>(scratch) + header);

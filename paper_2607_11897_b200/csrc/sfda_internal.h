@@ -16,6 +16,8 @@ struct ForwardArgs {
     // parameterisation, which the kernel applies with these constants on the way in
     int fused = 0;
     float alpha_min = 0.f, alpha_max = 1.f, theta_max = 0.f, eps = 0.f;
+    // tensor-core path, plain inputs only: [B][H][NC][m] chunk-closing integer phase, or nullptr
+    uint32_t *phase_turns = nullptr;
 };
 
 struct FactorArgs {

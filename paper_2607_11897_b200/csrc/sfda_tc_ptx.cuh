@@ -161,6 +161,31 @@ __device__ __forceinline__ void tmem_ld8(uint32_t addr, uint32_t *r)
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
                  : "r"(addr));
 }
+// 16 lanes x 64 columns of 32-bit tensor memory in the 16x256b fragment shape: for column block i (8 columns),
+// thread T receives r[4i], r[4i+1] = (lane T / 4, columns 8i + 2 (T % 4), + 1) and r[4i+2], r[4i+3] = the same
+// columns of lane T / 4 + 8 (the accumulator-fragment layout of the warp-level MMA).
+__device__ __forceinline__ void tmem_ld_16x256b_x8(uint32_t addr, uint32_t *r)
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : SFDA_R32(r, 0), SFDA_R32(r, 16)
+        : "r"(addr));
+}
+__device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t addr, uint32_t *r)
+{
+    asm volatile("tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : SFDA_R32(r, 0)
+                 : "r"(addr));
+}
+// Four 8 x 8 matrices of 16-bit elements, stored transposed: lane l gives the address of (transposed) row l % 8 of
+// matrix l / 8; register k of thread T holds elements (row T / 4, columns 2 (T % 4), + 1) of matrix k.
+__device__ __forceinline__ void stmatrix_x4_trans(uint32_t saddr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("stmatrix.sync.aligned.m8n8.x4.trans.shared.b16 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(a), "r"(b),
+                 "r"(c), "r"(d)
+                 : "memory");
+}
 __device__ __forceinline__ uint16_t lds16(uint32_t saddr)
 {
     uint16_t v;

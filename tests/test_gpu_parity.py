@@ -326,6 +326,37 @@ def test_forward_long_context_stability():
 # ------------------------------------------------------------------------------------------------
 # factor export
 # ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name,B,T,H,full_ws", [("cfg1", 2, 4096, 16, True), ("cfg1_ragged", 1, 1029, 3, False),
+                                                ("cfg3", 1, 131072, 16, True), ("cfg2_slices", 8, 2048, 32, True)])
+def test_tensor_core_forward_phase_bookkeeping_is_bit_exact(name, B, T, H, full_ws):
+    """The integer cumulative phase of the tensor-core kernel (what its rotations are derived from), chunk by chunk,
+    against the oracle's emulation of the same single-precision conversion: every bit, with the sequences cut into
+    time slices (full workspace) and uncut (256-byte workspace), on uniform and on quantised phases."""
+    base = workloads.CONFIGS[3] if name == "cfg3" else workloads.CONFIGS[2 if name == "cfg2_slices" else 1]
+    cfg = base.scaled(B=B, T=T, H=H)
+    inp = workloads.forward_inputs(cfg)
+    d = {k: (None if v is None else to_dev(v, cfg, k)) for k, v in inp.items()}
+    NC = (T + 63) // 64
+    o = torch.empty(B, T, H, 128, device=DEV, dtype=torch.bfloat16)
+    S_T = torch.empty(B, H, 128, 128, device=DEV)
+    ph = torch.full((B, H, NC, 64), -1, device=DEV, dtype=torch.int32)
+    nws = sfda.sfda_workspace_bytes(B, T, H, 128, 128, 64, 1) if full_ws else 256
+    ws = torch.empty(nws, device=DEV, dtype=torch.uint8)
+    sfda.sfda_forward_phase(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, None, S_T, ph, 64, ws)
+    torch.cuda.synchronize()
+    assert sfda.sfda_workspace_status(ws) == 0
+    got = ph.cpu().numpy().view(np.uint32)                                   # [B][H][NC][m]
+    want = bookkeeping.chunk_closing_turns_f32(np.moveaxis(inp["theta"], 2, 1), 64)   # theta [B][T][H][m] -> [B][H][T][m]
+    assert got.shape == want.shape
+    assert np.array_equal(got, want)
+    # the same launch still computes the forward: same bits as the plain entry point
+    o2 = torch.empty_like(o)
+    S2 = torch.empty_like(S_T)
+    sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o2, None, S2, 64, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(o, o2) and torch.equal(S_T, S2)
+
+
 @pytest.mark.parametrize("d_k,chunk,T,dtype", [(64, 16, 50, "f32"), (128, 64, 150, "f32"), (128, 32, 64, "bf16"),
                                                (64, 64, 64, "f32")])
 def test_chunk_factors_match_constructive_recursion(d_k, chunk, T, dtype):

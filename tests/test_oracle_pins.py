@@ -466,6 +466,70 @@ def test_cumulative_turns_are_chunk_local_integer_sums():
         == (2 * int(bookkeeping.phase_to_turns(np.float32(np.pi)))) % 2 ** 32
 
 
+def test_single_precision_phase_turns_match_exact_rational_arithmetic():
+    """phase_to_turns_f32 against its definition in exact arithmetic: the float32 nearest to the exact product of
+    the two float32 factors (ties to even), then the nearest integer (ties to even), modulo 2**32."""
+    from fractions import Fraction
+    rng = np.random.default_rng(27)
+    th = np.concatenate([rng.uniform(-np.pi, np.pi, 3000), rng.uniform(-40.0, 40.0, 500),
+                         [0.0, np.pi, -np.pi, 1e-9, -1e-9, 100.0, -7.5, 2 * np.pi / 3, 2 * np.pi / 7]]).astype(np.float32)
+    got = bookkeeping.phase_to_turns_f32(th)
+    c = Fraction(float(bookkeeping.TURNS_PER_RADIAN_F32))
+    assert abs(float(c) - 2 ** 32 / (2 * np.pi)) <= 32.0           # float32 spacing there is 64
+
+    def round_to_f32(x):            # nearest float32 (24-bit significand) to the rational x, ties to even
+        if x == 0:
+            return Fraction(0)
+        sign, a = (-1 if x < 0 else 1), abs(x)
+        e = 0
+        while a >= 2 ** 24:
+            a /= 2
+            e += 1
+        while a < 2 ** 23:
+            a *= 2
+            e -= 1
+        n = a.numerator // a.denominator
+        rem = a - n
+        if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and n % 2 == 1):
+            n += 1
+        return sign * Fraction(n) * Fraction(2) ** e
+
+    def round_half_even(x):
+        n = x.numerator // x.denominator
+        rem = x - n
+        if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and n % 2 == 1):
+            n += 1
+        return n
+
+    for x, g in zip(th, got):
+        want = round_half_even(round_to_f32(Fraction(float(x)) * c)) % 2 ** 32
+        assert int(g) == want
+    # odd symmetry, and closeness to the double-precision conversion: within 2^-24 of the angle (plus one unit)
+    assert np.array_equal(bookkeeping.phase_to_turns_f32(-th), (-got.astype(np.int64) & 0xFFFFFFFF).astype(np.uint32))
+    d = (got.astype(np.int64) - bookkeeping.phase_to_turns(th).astype(np.int64) + 2 ** 31) % 2 ** 32 - 2 ** 31
+    assert np.all(np.abs(d) <= np.abs(th.astype(np.float64)) * bookkeeping.TURNS_PER_RADIAN * 2.0 ** -23 + 1)
+
+
+def test_chunk_closing_turns_are_integer_sums_over_each_chunk():
+    rng = np.random.default_rng(28)
+    T, m, C = 150, 3, 64
+    th = rng.uniform(-np.pi, np.pi, (2, T, m)).astype(np.float32)
+    u = bookkeeping.phase_to_turns_f32(th)
+    close = bookkeeping.chunk_closing_turns_f32(th, C)
+    assert close.shape == (2, 3, m) and close.dtype == np.uint32
+    for n in range(2):
+        for j in range(m):
+            for c in range(3):
+                acc = 0
+                for t in range(c * C, min((c + 1) * C, T)):
+                    acc = (acc + int(u[n, t, j])) % 2 ** 32
+                assert int(close[n, c, j]) == acc
+    # p steps of 2 pi / p close a chunk within p rounding units of a whole turn
+    for p_ in (2, 3, 5, 7):
+        last = int(bookkeeping.chunk_closing_turns_f32(np.full((1, p_, 1), 2 * np.pi / p_, np.float32), 64)[0, 0, 0])
+        assert min(last, 2 ** 32 - last) <= 2 ** 32 * 2.0 ** -23 * p_
+
+
 def test_chunk_plan():
     assert bookkeeping.chunk_plan(256, 16) == (16, 16)
     assert bookkeeping.chunk_plan(257, 16) == (17, 1)
