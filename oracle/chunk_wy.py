@@ -1,7 +1,7 @@
 """Naive chunked SFDA path in numpy complex128 (test infrastructure only).
 
 It takes the steps of the paper in the paper's order and notation, one token at
-a time, with no blocking or fusion:
+a time, with no blocking or fusion (written from the theorems' equations):
 
 * Algorithm 1 ("Constructive SFDA-WY chunk summary") / Theorem "Constructive
   left-to-right chunk-WY recursion": the factors (Gamma, Y, W, M) of
@@ -40,32 +40,39 @@ def pair_rows(S):
 
 
 def chunk_factor_steps(k, alpha, theta, beta):
-    """Run the recursion of Theorem "Constructive left-to-right chunk-WY recursion".
+    """Factors of P_t = A_t ... A_1 = Gamma_t - Y_t M_t W_t^* for t = 1..C, from the four equations of Theorem
+    "Constructive left-to-right chunk-WY recursion" (u_t = beta_t k_t, r_t = Lambda_t^* k_t):
 
-    k: [C, m] complex; alpha, theta: [C, m]; beta: [C].
-    Yields, after each token t = 1..C, the tuple (Gamma_t, Y_t, W_t, M_t) with
-    Gamma_t the diagonal as a vector [m], Y_t, W_t: [m, t], M_t: [t, t].
+      Gamma_t = Lambda_t Gamma_{t-1}                         Eq. "constructive-Gamma"
+      Y_t     = [Lambda_t Y_{t-1} | u_t]                     Eq. "constructive-Y"
+      W_t     = [W_{t-1} | Gamma_{t-1}^* r_t]                Eq. "constructive-W"
+      M_t     = [[M_{t-1}, 0], [-r_t^* Y_{t-1} M_{t-1}, 1]]  Eq. "constructive-M"
+
+    k: [C, m] complex; alpha, theta: [C, m]; beta: [C].  Yields (Gamma_t [m], Y_t [m, t], W_t [m, t], M_t [t, t])
+    after every token.  The factors live in arrays of the chunk's full size that grow by one column (and one row of
+    M) per token; W_t and M_t are leading blocks of the final ones, Y_t is not (its old columns are multiplied by
+    Lambda_t every step), so what is yielded are copies of the current leading blocks.
     """
+    k = np.asarray(k, dtype=np.complex128)
     C, m = k.shape
-    Gamma = np.ones(m, np.complex128)
-    Y = np.zeros((m, 0), np.complex128)
-    W = np.zeros((m, 0), np.complex128)
-    M = np.zeros((0, 0), np.complex128)
+    lam = np.asarray(alpha, np.float64) * np.exp(1j * np.asarray(theta, np.float64))     # diagonal of Lambda_t, [C, m]
+    u_all = np.asarray(beta, np.float64)[:, None] * k                                   # rows u_t
+    r_all = np.conj(lam) * k                                                            # rows r_t
+    gamma = np.cumprod(lam, axis=0)                                                     # rows diag(Gamma_t)
+    Y = np.zeros((m, C), np.complex128)
+    W = np.zeros((m, C), np.complex128)
+    M = np.eye(C, dtype=np.complex128)
     for t in range(C):
-        lam = alpha[t] * np.exp(1j * theta[t])          # Lambda_t (diagonal)
-        u = beta[t] * k[t]                              # u_t = beta_t k_t
-        r = np.conj(lam) * k[t]                         # r_t = Lambda_t^* k_t
-        Gamma_old, Y_old, W_old, M_old = Gamma, Y, W, M
-        Gamma = lam * Gamma_old                         # Eq. constructive-Gamma
-        Y = np.concatenate([lam[:, None] * Y_old, u[:, None]], axis=1)      # Eq. constructive-Y
-        W = np.concatenate([W_old, (np.conj(Gamma_old) * r)[:, None]], axis=1)  # Eq. constructive-W
-        row = -(np.conj(r)[None, :] @ Y_old) @ M_old    # -r_t^* Y_{t-1} M_{t-1}
-        n = M_old.shape[0]
-        M = np.zeros((n + 1, n + 1), np.complex128)     # Eq. constructive-M
-        M[:n, :n] = M_old
-        M[n, :n] = row[0]
-        M[n, n] = 1.0
-        yield Gamma, Y, W, M
+        if t > 0:
+            # row t of M first: it needs Y_{t-1} and M_{t-1}, both still untouched by this step
+            M[t, :t] = -(np.conj(r_all[t]) @ Y[:, :t]) @ M[:t, :t]
+            Y[:, :t] *= lam[t][:, None]
+            W[:, t] = np.conj(gamma[t - 1]) * r_all[t]
+        else:
+            W[:, 0] = r_all[0]                            # Gamma_0 = I
+        Y[:, t] = u_all[t]
+        n = t + 1
+        yield gamma[t].copy(), Y[:, :n].copy(), W[:, :n].copy(), M[:n, :n].copy()
 
 
 def chunk_factors(k, alpha, theta, beta):
