@@ -450,11 +450,14 @@ size_t sfda_forward_host_arena_bytes(int B, int T, int H, int d_k, int d_v, int 
     size_t total = 0;
     total += 2 * round256(n * d_k * eb);                      // q, k
     total += round256(n * d_v * eb);                          // v
-    total += 2 * round256(n * m * 4) + round256(n * 4);       // alpha, theta, beta
+    total += 2 * round256(n * m * 4);                         // alpha, theta
     total += (want_o_im ? 2 : 1) * round256(n * d_v * eb);    // o, o_im
     if (have_S0 || want_S_T) total += round256((size_t)B * H * d_k * d_v * 4);
     int per = 1, pieces = 1;
     host_pieces(B, &per, &pieces);
+    // beta has 4 bytes per (token, head): a piece's share of one contiguous array would start on a 16-byte boundary
+    // only when per * T * H is a multiple of four, so every piece gets a region of its own
+    total += (size_t)pieces * round256((size_t)per * T * H * 4);
     total += (size_t)pieces * round256(sfda_workspace_bytes(per, T, H, d_k, d_v, chunk, dtype));   // one per piece
     return total;
 }
@@ -482,17 +485,19 @@ int sfda_forward_host(const void *q, const void *k, const void *v, const float *
     char *cur = static_cast<char *>(arena);
     auto take = [&](size_t bytes) { char *p = cur; cur += round256(bytes); return p; };
     char *dq = take(n * d_k * eb), *dk = take(n * d_k * eb), *dv = take(n * d_v * eb);
-    char *da = take(n * m * 4), *dt = take(n * m * 4), *db = take(n * 4);
+    char *da = take(n * m * 4), *dt = take(n * m * 4);
     char *dout = take(n * d_v * eb), *dout_im = o_im ? take(n * d_v * eb) : nullptr;
     char *dS = (S0 || S_T) ? take((size_t)B * state_elems * 4) : nullptr;
     int per = 1, pieces = 1;
     host_pieces(B, &per, &pieces);
+    const size_t beta_stride = round256((size_t)per * T * H * 4);   // one 256-byte-aligned beta region per piece
+    char *db = take((size_t)pieces * beta_stride);
     const size_t ws_bytes = sfda_workspace_bytes(per, T, H, d_k, d_v, chunk, dtype);
     char *ws0 = take((size_t)pieces * round256(ws_bytes));
 
     size_t h2d = 0, d2h = 0;
     bool ok = true;
-    int launches = 0;
+    int launches = 0, status = SFDA_OK;
     auto copy = [&](void *dst, const void *src, size_t bytes, cudaMemcpyKind kind, cudaStream_t st) {
         ok = ok && cudaMemcpyAsync(dst, src, bytes, kind, st) == cudaSuccess;
         (kind == cudaMemcpyHostToDevice ? h2d : d2h) += bytes;
@@ -509,7 +514,7 @@ int sfda_forward_host(const void *q, const void *k, const void *v, const float *
         copy(dv + r0 * d_v * eb, hv + r0 * d_v * eb, rn * d_v * eb, cudaMemcpyHostToDevice, hp->up);
         copy(da + r0 * m * 4, alpha + r0 * m, rn * m * 4, cudaMemcpyHostToDevice, hp->up);
         copy(dt + r0 * m * 4, theta + r0 * m, rn * m * 4, cudaMemcpyHostToDevice, hp->up);
-        copy(db + r0 * 4, beta + r0, rn * 4, cudaMemcpyHostToDevice, hp->up);
+        copy(db + (size_t)i * beta_stride, beta + r0, rn * 4, cudaMemcpyHostToDevice, hp->up);
         if (S0) copy(dS + b0 * state_elems * 4, S0 + b0 * state_elems, nb * state_elems * 4, cudaMemcpyHostToDevice, hp->up);
         ok = ok && cudaEventRecord(hp->uploaded[i], hp->up) == cudaSuccess &&
              cudaStreamWaitEvent(s, hp->uploaded[i], 0) == cudaSuccess;
@@ -517,10 +522,13 @@ int sfda_forward_host(const void *q, const void *k, const void *v, const float *
         float *dSp = dS ? reinterpret_cast<float *>(dS) + b0 * state_elems : nullptr;
         const int frc = sfda_forward(dq + r0 * d_k * eb, dk + r0 * d_k * eb, dv + r0 * d_v * eb,
                                      reinterpret_cast<float *>(da) + r0 * m, reinterpret_cast<float *>(dt) + r0 * m,
-                                     reinterpret_cast<float *>(db) + r0, S0 ? dSp : nullptr, dout + r0 * d_v * eb,
+                                     reinterpret_cast<float *>(db + (size_t)i * beta_stride), S0 ? dSp : nullptr, dout + r0 * d_v * eb,
                                      dout_im ? dout_im + r0 * d_v * eb : nullptr, S_T ? dSp : nullptr, nb, T, H, d_k, d_v,
                                      chunk, dtype, ws0 + (size_t)i * round256(ws_bytes), ws_bytes, stream);
-        if (frc != SFDA_OK) return frc;
+        if (frc != SFDA_OK) {      // nothing of this piece was launched; what is already queued still has to be joined below
+            status = frc;
+            break;
+        }
         launches += g_last_launches;
         ok = ok && cudaEventRecord(hp->computed[i], s) == cudaSuccess &&
              cudaStreamWaitEvent(hp->down, hp->computed[i], 0) == cudaSuccess;
@@ -530,12 +538,15 @@ int sfda_forward_host(const void *q, const void *k, const void *v, const float *
                  hp->down);
         if (S_T) copy(S_T + b0 * state_elems, dSp, nb * state_elems * 4, cudaMemcpyDeviceToHost, hp->down);
     }
-    // the caller's stream is done when the last download is
-    ok = ok && cudaEventRecord(hp->end, hp->down) == cudaSuccess && cudaStreamWaitEvent(s, hp->end, 0) == cudaSuccess;
+    // The caller's stream is done when the last download is -- and, also after an error, only when every upload
+    // already queued on the internal stream is: otherwise a reuse of the arena could race those copies.
+    const bool joined = cudaEventRecord(hp->end, hp->down) == cudaSuccess && cudaStreamWaitEvent(s, hp->end, 0) == cudaSuccess &&
+                        cudaEventRecord(hp->start, hp->up) == cudaSuccess && cudaStreamWaitEvent(s, hp->start, 0) == cudaSuccess;
     g_last_launches = launches;
     if (bytes_h2d) *bytes_h2d = h2d;
     if (bytes_d2h) *bytes_d2h = d2h;
-    return ok ? SFDA_OK : SFDA_ERR_CUDA;
+    if (status != SFDA_OK) return status;
+    return ok && joined ? SFDA_OK : SFDA_ERR_CUDA;
 }
 
 int sfda_frontend(const float *a_raw, const float *b_raw, const float *c_raw, const void *k_raw, float alpha_min,

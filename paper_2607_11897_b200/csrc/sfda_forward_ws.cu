@@ -1480,7 +1480,8 @@ void forward_ws_partition(int BH, int NC, int n_sm, bool cuts_allowed, int *slic
     if (periods) *periods = best;      // the schedule's length in chunk periods (what the choice was made on)
 }
 
-cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratch_bytes, cudaStream_t stream, int *launches)
+cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratch_bytes, cudaStream_t stream, int *launches,
+                              bool clear_status)
 {
     Maps maps;
     if (!make_map(&maps.v, a.v, a.B, a.T, a.H) || !make_map(&maps.o, a.o, a.B, a.T, a.H, false, true) ||
@@ -1505,7 +1506,12 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
 #endif
     const bool pieces = Q > 1 || bal;   // sequences are cut: counters and boundary states in use, CTAs wait on one another
     const size_t header = kWsMinScratchBytes + (pieces ? (((size_t)BH * 4 + 255) & ~(size_t)255) : 0);
-    e = cudaMemsetAsync(scratch, 0, header, stream);
+    // The status word is only ever set by the kernel, never cleared: a caller that runs several launches on one
+    // scratch block and reads the word once at the end clears it with the first launch only.
+    if (clear_status)
+        e = cudaMemsetAsync(scratch, 0, header, stream);
+    else if (header > kWsMinScratchBytes)
+        e = cudaMemsetAsync(static_cast<char *>(scratch) + kWsMinScratchBytes, 0, header - kWsMinScratchBytes, stream);
     if (e != cudaSuccess) return e;
     Params p;
     p.timing = g_ws_timing;

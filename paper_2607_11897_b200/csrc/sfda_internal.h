@@ -95,8 +95,9 @@ bool forward_ws_supported(const ForwardArgs &a);
 constexpr size_t kWsMinScratchBytes = 256;
 size_t forward_ws_scratch_bytes(int B, int H);
 void forward_ws_partition(int BH, int NC, int n_sm, bool cuts_allowed, int *slices, int *balanced, double *periods);
+// clear_status = false keeps what an earlier launch on the same scratch block left in the status word.
 cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratch_bytes, cudaStream_t stream,
-                              int *launches);
+                              int *launches, bool clear_status = true);
 // The same kernel on the library's own statically allocated scratch block (kStaticScratchBytes), and a read of
 // the status word kept there (synchronises the stream).  Neither allocates.
 constexpr size_t kStaticScratchBytes = 256;

@@ -328,8 +328,9 @@ cudaError_t launch_forward_two_level(const ForwardArgs &a, int n, void *workspac
     s.S0 = S_a; s.S_T = B_st;
     if ((e = launch_forward_ws(s, fwd_ws, fwd_bytes, stream, launches)) != cudaSuccess) return e;
     // pass 1b: P of every slice, and g_t = P_t^* q_t in the first d_k / 2 channels of its outputs
+    // (same scratch block: the status word keeps a timeout of pass 1a, so that the caller's one read sees either)
     s.v = v_zero; s.S0 = S_id; s.S_T = P_st; s.o = g_re; s.o_im = g_im;
-    if ((e = launch_forward_ws(s, fwd_ws, fwd_bytes, stream, launches)) != cudaSuccess) return e;
+    if ((e = launch_forward_ws(s, fwd_ws, fwd_bytes, stream, launches, false)) != cudaSuccess) return e;
     // scan over the slices
     two_level_scan_kernel<128, 128><<<dim3((unsigned)(a.B * a.H), 128 / kScanCols), kScanThreads, 0, stream>>>(
         B_st, P_st, a.S0, S_in, a.S_T, n, a.H);

@@ -54,6 +54,22 @@ def test_workspace_bytes(lib):
     assert sfda.sfda_workspace_bytes(0, 256, 2, 128, 128, 64, sfda.SFDA_BF16) == 0
 
 
+def test_host_arena_gives_every_piece_of_the_batch_an_aligned_beta_region(lib):
+    """sfda_forward_host cuts the batch into at most eight pieces; beta has four bytes per (token, head), so a
+    piece's share of one contiguous device array would leave the 16-byte grid whenever per * T * H is not a
+    multiple of four.  The arena therefore reserves one 256-byte-rounded beta region per piece (host arithmetic)."""
+    r256 = lambda x: (x + 255) // 256 * 256
+    for B, T, H in ((2, 5, 1), (3, 130, 3), (9, 67, 1), (8, 64, 2), (17, 33, 5)):
+        n, eb, d, m = B * T * H, 2, 128, 64
+        per = (B + 7) // 8
+        pieces = (B + per - 1) // per
+        want = 2 * r256(n * d * eb) + r256(n * d * eb) + 2 * r256(n * m * 4) + 2 * r256(n * d * eb) \
+            + r256(B * H * d * d * 4) + pieces * r256(per * T * H * 4) \
+            + pieces * r256(sfda.sfda_workspace_bytes(per, T, H, d, d, 64, sfda.SFDA_BF16))
+        assert sfda.sfda_forward_host_arena_bytes(B, T, H, d, d, 64, sfda.SFDA_BF16, True, True, True) == want
+        assert (per * T * H * 4) % 16 != 0 or (B, T, H) in ((8, 64, 2),)      # the cases above do leave the grid
+
+
 def test_argument_validation_happens_before_any_launch(lib):
     """Every error below is found on the host; nothing touches a device (there is none here)."""
     vp, ci = ctypes.c_void_p, ctypes.c_int

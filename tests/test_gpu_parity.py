@@ -481,8 +481,12 @@ def test_iterated_step_equals_forward():
 # ------------------------------------------------------------------------------------------------
 # host-buffer entry point and argument errors
 # ------------------------------------------------------------------------------------------------
-def test_forward_host_matches_device_call():
-    cfg = workloads.CONFIGS[1].scaled(name="host", B=2, T=256, H=2, s0_std=0.1)
+@pytest.mark.parametrize("B,T,H", [(2, 256, 2), (2, 5, 1), (3, 130, 3), (9, 67, 1)])
+def test_forward_host_matches_device_call(B, T, H):
+    """Host buffers in, host buffers out, against the device-pointer call: also where a piece of the batch holds a
+    number of (token, head) rows that is not a multiple of four (beta then starts off a 16-byte boundary in the
+    caller's array) and where the last piece is shorter than the others."""
+    cfg = workloads.CONFIGS[1].scaled(name="host", B=B, T=T, H=H, s0_std=0.1)
     inp = workloads.forward_inputs(cfg)
     o_d, o_im_d, S_d = run_forward(cfg, inp)
     h = {}
