@@ -64,8 +64,8 @@ typedef enum {
     SFDA_ERR_WORKSPACE = -5,   /* workspace NULL or smaller than sfda_workspace_bytes */
     SFDA_ERR_CUDA = -6,        /* the CUDA runtime reported an error at launch        */
     SFDA_ERR_TIMEOUT = -7,     /* a bounded device-side wait ran out                  */
-    SFDA_ERR_VALUE = -8        /* a scalar of the stable parameterisation is out of   */
-                               /* range (see sfda_frontend)                           */
+    SFDA_ERR_VALUE = -8        /* a scalar argument is out of range (the constants of */
+                               /* sfda_frontend; slices / wait_ticks of the diagnostic)*/
 } sfda_status;
 
 typedef enum { SFDA_F32 = 0, SFDA_BF16 = 1 } sfda_dtype;
@@ -164,6 +164,26 @@ SFDA_API int sfda_forward_phase(const void *q, const void *k, const void *v,
                  const float *alpha, const float *theta, const float *beta,
                  const float *S0, void *o, void *o_im, float *S_T, uint32_t *phase_turns,
                  int B, int T, int H, int d_k, int d_v, int chunk, int dtype,
+                 void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Diagnostic: exercises the kernel's handling of a wait that runs out, without any fault.  Every wait inside the
+ * tensor-core forward is bounded (App. "Kernel sketch" leaves the pipeline to the implementation; the boundary-state
+ * scan of Section "chunkwise form" is what is being handed over); when one runs out, the CTA raises a flag, all its
+ * roles leave their loops, tensor memory is freed, the kernel ends normally and the status word reads
+ * SFDA_ERR_TIMEOUT.  This call runs sfda_forward on the tensor-core shapes with every sequence cut into `slices`
+ * (2..8, dividing the number of chunks) time slices whose boundary states are written but never announced, and
+ * with the wait limit set to `wait_ticks` SM-clock ticks (2^16..2^26): every slice after the first waits for its
+ * predecessor until the limit and gives up.  The outputs of first slices are valid, everything else is undefined;
+ * sfda_workspace_status(workspace) afterwards returns SFDA_ERR_TIMEOUT, and the context stays usable: a following
+ * ordinary call on the same workspace is correct.  Needs the full sfda_workspace_bytes; SFDA_ERR_VALUE for slices
+ * or wait_ticks out of range, SFDA_ERR_SHAPE when slices does not divide the chunk count, otherwise the errors of
+ * sfda_forward.  Nothing in the library calls this.
+ */
+SFDA_API int sfda_forward_withheld_handoff(const void *q, const void *k, const void *v,
+                 const float *alpha, const float *theta, const float *beta,
+                 const float *S0, void *o, void *o_im, float *S_T,
+                 int B, int T, int H, int d_k, int d_v, int chunk, int dtype, int slices, unsigned wait_ticks,
                  void *workspace, size_t workspace_bytes, void *stream);
 
 /*

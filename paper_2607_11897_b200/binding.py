@@ -24,9 +24,13 @@ def lib_path() -> str:
 def load():
     """Load ``libsfda.so``; raise if it has not been built (no fallback exists)."""
     global _LIB
-    if _LIB is not None:
-        return _LIB
-    path = lib_path()
+    if _LIB is None:
+        _LIB = load_library(lib_path())
+    return _LIB
+
+
+def load_library(path):
+    """Open a build of the library at `path` and declare the argument types of its entry points."""
     if not os.path.exists(path):
         raise ImportError("%s is missing: run `python -m paper_2607_11897_b200.build` "
                           "(or __graft_entry__.build()) first" % path)
@@ -40,6 +44,7 @@ def load():
     lib.sfda_forward.argtypes = [_vp] * 10 + [_ci] * 7 + [_vp, _sz, _vp]
     lib.sfda_forward_simt.argtypes = [_vp] * 10 + [_ci] * 7 + [_vp]
     lib.sfda_forward_phase.argtypes = [_vp] * 11 + [_ci] * 7 + [_vp, _sz, _vp]
+    lib.sfda_forward_withheld_handoff.argtypes = [_vp] * 10 + [_ci] * 8 + [ctypes.c_uint, _vp, _sz, _vp]
     lib.sfda_chunk_factors.argtypes = [_vp] * 9 + [_ci] * 6 + [_vp]
     lib.sfda_step.argtypes = [_vp] * 9 + [_ci] * 5 + [_vp]
     lib.sfda_forward_host_arena_bytes.restype = _sz
@@ -67,7 +72,6 @@ def load():
     lib.sfda_frontend_backward.argtypes = [_vp] * 4 + [_cf] * 4 + [_vp] * 8 + [_ci] * 5 + [_vp]
     lib.sfda_step_blocks.argtypes = [_vp] * 12 + [_ci] * 6 + [_vp]
     lib.sfda_forward_blocks.argtypes = [_vp] * 13 + [_ci] * 7 + [_vp]
-    _LIB = lib
     return lib
 
 
@@ -175,6 +179,20 @@ def sfda_forward_phase(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, phase_turn
                                 _ptr(workspace), ws_bytes, _stream(stream))
     if rc != 0:
         raise SfdaError(rc, "sfda_forward_phase")
+
+
+def sfda_forward_withheld_handoff(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, chunk, slices, wait_ticks, workspace,
+                                  stream=None):
+    """``sfda_forward_withheld_handoff`` of ``include/sfda.h``: the diagnostic launch whose time slices never
+    announce their boundary states, so that every later slice's bounded wait runs out."""
+    B, T, H, d_k = q.shape
+    d_v = v.shape[-1]
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = load().sfda_forward_withheld_handoff(_ptr(q), _ptr(k), _ptr(v), _ptr(alpha), _ptr(theta), _ptr(beta), _ptr(S0),
+                                              _ptr(o), _ptr(o_im), _ptr(S_T), B, T, H, d_k, d_v, chunk, _dtype_code(q),
+                                              int(slices), int(wait_ticks), _ptr(workspace), ws_bytes, _stream(stream))
+    if rc != 0:
+        raise SfdaError(rc, "sfda_forward_withheld_handoff")
 
 
 def sfda_workspace_status(workspace, stream=None) -> int:

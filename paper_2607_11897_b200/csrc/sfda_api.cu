@@ -262,6 +262,31 @@ int sfda_forward_phase(const void *q, const void *k, const void *v, const float 
                : SFDA_ERR_CUDA;
 }
 
+int sfda_forward_withheld_handoff(const void *q, const void *k, const void *v, const float *alpha, const float *theta,
+                                  const float *beta, const float *S0, void *o, void *o_im, float *S_T, int B, int T,
+                                  int H, int d_k, int d_v, int chunk, int dtype, int slices, unsigned wait_ticks,
+                                  void *workspace, size_t workspace_bytes, void *stream)
+{
+    g_last_launches = 0;
+    const int rc = validate_forward(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
+    if (rc != SFDA_OK) return rc;
+    sfda::ForwardArgs a = pack(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
+    if (!sfda::forward_ws_supported(a)) return SFDA_ERR_UNSUPPORTED;
+    // at least two slices (so that something waits), a limit between 2^16 and 2^26 ticks (a few dozen microseconds to a
+    // few dozen milliseconds), whole chunks per slice, and the full workspace (the hand-off buffers live there)
+    if (slices < 2 || slices > 8 || wait_ticks < (1u << 16) || wait_ticks > (1u << 26)) return SFDA_ERR_VALUE;
+    if (((T + chunk - 1) / chunk) % slices != 0) return SFDA_ERR_SHAPE;
+    if (!workspace || workspace_bytes < sfda::forward_ws_scratch_bytes(B, H)) return SFDA_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return SFDA_ERR_ALIGN;
+    a.debug_slices = slices;
+    a.debug_withhold = 1;
+    a.wait_ticks = wait_ticks;
+    return sfda::launch_forward_ws(a, workspace, workspace_bytes, static_cast<cudaStream_t>(stream), &g_last_launches) ==
+                   cudaSuccess
+               ? SFDA_OK
+               : SFDA_ERR_CUDA;
+}
+
 size_t sfda_forward_two_level_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, int dtype,
                                               int n_slices)
 {

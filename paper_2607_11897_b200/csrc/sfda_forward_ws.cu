@@ -92,6 +92,7 @@ struct Misc {
     float ones[C];                          //                  +1: the scale of the passes that apply none
     unsigned long long bars[kNumBars];
     uint32_t tmem_base;
+    uint32_t wait_limit;                    // SM-clock ticks after which a wait gives up
     volatile int abort;
 };
 static_assert(sizeof(Misc) <= kMiscBytes, "misc area too small");
@@ -131,6 +132,8 @@ struct Params {
     uint32_t *flags;     // [B*H] arrival counters of the pieces of a cut sequence (only used when sequences are cut)
     float *handoff;      // [B*H][d_k][d_v] boundary states between the pieces (only used when sequences are cut)
     int T, H, has_o_im;
+    uint32_t wait_limit;   // ticks of the SM clock after which a device-side wait gives up
+    int withhold;          // diagnostic launches only: boundary states are written but never announced
     int BH, U, Q, n_units;   // sequences, chunks per work unit, time slices per sequence, Q * BH
     int bal, NC, bal_base, bal_rem;   // balanced partition: on / off, chunks per sequence, BH * NC = grid * base + rem
     uint32_t magic_BH, magic_H, magic_NC;   // floor(2^32 / d) + 1 (0 for d = 1): quotients by multiplication
@@ -296,10 +299,12 @@ __device__ __forceinline__ unsigned long long now_ns()
 }
 #endif
 
-// Wait for completion number k of a barrier; gives up after about a second (2^31 ticks of the SM clock) and
-// raises the abort flag.  try_wait parks the thread in hardware for up to the hinted time, so waiting warps do
+// Wait for completion number k of a barrier; gives up after the launch's wait limit (about a second: 2^31 ticks of
+// the SM clock, unless the caller asked for less) or as soon as any other wait of the CTA has given up, and raises
+// the abort flag.  try_wait parks the thread in hardware for up to the hinted time, so waiting warps do
 // not compete with working ones for issue slots.  Kept to a handful of instructions: it is inlined at every
 // wait, and the kernel's per-chunk code has to stay inside the SM's instruction cache.
+template <bool kDiag>
 __device__ __forceinline__ bool wait_k(Misc &mi, int bar, int k)
 {
     const uint32_t addr = smem_u32(&mi.bars[bar]), parity = (uint32_t)k & 1u;
@@ -315,7 +320,9 @@ __device__ __forceinline__ bool wait_k(Misc &mi, int bar, int k)
             chaos(addr + 77u);
             return true;
         }
-    } while ((uint32_t)clock() - t0 < 0x80000000u);
+        // the diagnostic instantiation takes its limit from the launch and also leaves as soon as any other wait
+        // of the CTA has given up (a few more instructions per wait than the product kernel can afford)
+    } while (kDiag ? (!mi.abort && (uint32_t)clock() - t0 < mi.wait_limit) : ((uint32_t)clock() - t0 < 0x80000000u));
     mi.abort = 1;
     return false;
 }
@@ -331,9 +338,10 @@ __device__ __forceinline__ bool elect_one()
     return pred != 0;
 }
 // wait_k with a warp-uniform outcome, so that a warp leaves (or stays) as a whole
+template <bool kDiag>
 __device__ __forceinline__ bool wait_k_warp(Misc &mi, int bar, int k)
 {
-    return __all_sync(0xffffffffu, wait_k(mi, bar, k) ? 1 : 0) != 0;
+    return __all_sync(0xffffffffu, wait_k<kDiag>(mi, bar, k) ? 1 : 0) != 0;
 }
 
 // One complex product as four real ones (g = 0..3), each of four K = 16 instructions:
@@ -400,6 +408,7 @@ __device__ __forceinline__ void prefetch_chunk(const Maps &maps, const ChunkInfo
 //               tensor pipe, is what takes the time: about a hundred cycles per instruction)
 //   role 1      the output product rho += Aq E and the output stores
 //   role 2      the v loads, the Gram products (they run ahead of the chain) and the L2 prefetch of the inputs
+template <bool kDiag>
 __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint32_t tmem, const Maps &maps,
                                          const Params &p, int n_chunks)
 {
@@ -423,16 +432,16 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
             // D1 = W^* S_0 as soon as S_0 is there; rho_1 = Qt^* S_0 (the Qt rows follow the W rows in the slot's
             // tiles) once rho of the previous chunk has been read out.  Both read S_0 from the operand columns.
             // (the state pass writes S_0 in two halves: key coordinates 0-15 and 32-47 = k-steps 0 and 2 first)
-            if (!wait_k_warp(mi, B_S16_A, j)) return;
-            if (!wait_k_warp(mi, B_PREP_FULL0 + s, u)) return;
+            if (!wait_k_warp<kDiag>(mi, B_S16_A, j)) return;
+            if (!wait_k_warp<kDiag>(mi, B_PREP_FULL0 + s, u)) return;
             tc_fence_after();
             SFDA_T(0);
             issue_complex<3, true, false, 2, 5>(acc, acc + 128, x_re, x_re + 32, w_re, w_re + 2 * kIm, dhi, I64, part);
-            if (!wait_k_warp(mi, B_S16_B, j)) return;
+            if (!wait_k_warp<kDiag>(mi, B_S16_B, j)) return;
             tc_fence_after();
             issue_complex<3, false, false, 2, 10>(acc, acc + 128, x_re, x_re + 32, w_re, w_re + 2 * kIm, dhi, I64, part);
             if (elect_one()) mma_commit(&bars[B_D1_DONE]);
-            if (j > 0 && !wait_k_warp(mi, B_O_STAGED, j - 1)) return;
+            if (j > 0 && !wait_k_warp<kDiag>(mi, B_O_STAGED, j - 1)) return;
             tc_fence_after();
             issue_complex<3, true, false, 2>(acc + 64, acc + 192, x_re, x_re + 32, w_re + kIm, w_re + 3 * kIm, dhi, I64, part);
             if (elect_one()) {
@@ -441,23 +450,23 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
             }
             SFDA_T(1);
             // E = M_beta R (R arrives in two halves of 32 tokens = two k-steps each)
-            if (!wait_k_warp(mi, B_R16_A, j)) return;
+            if (!wait_k_warp<kDiag>(mi, B_R16_A, j)) return;
             SFDA_T(2);
-            if (!wait_k_warp(mi, B_MB_FULL, j)) return;
+            if (!wait_k_warp<kDiag>(mi, B_MB_FULL, j)) return;
             tc_fence_after();
             SFDA_T(3);
             issue_complex<1, true, false, 2, 3>(acc, acc + 128, x_re, x_re + 32, m_re, m_re + kIm, dhi, I64, part);
-            if (!wait_k_warp(mi, B_R16_B, j)) return;
+            if (!wait_k_warp<kDiag>(mi, B_R16_B, j)) return;
             tc_fence_after();
             issue_complex<1, false, false, 2, 12>(acc, acc + 128, x_re, x_re + 32, m_re, m_re + kIm, dhi, I64, part);
             if (elect_one()) mma_commit(&bars[B_E_DONE]);
             SFDA_T(4);
             // S += E^T Kc (Kc as MN-major B: rows = tokens)
-            if (!wait_k_warp(mi, B_E16_A, j)) return;
+            if (!wait_k_warp<kDiag>(mi, B_E16_A, j)) return;
             tc_fence_after();
             SFDA_T(5);
             issue_complex<1, false, true, 128, 3>(tmem + TM_S32, tmem + TM_S32 + 64, x_re, x_re + 32, k_re, k_re + kIm, dhi, I64M, part);
-            if (!wait_k_warp(mi, B_E16_B, j)) return;
+            if (!wait_k_warp<kDiag>(mi, B_E16_B, j)) return;
             tc_fence_after();
             issue_complex<1, false, true, 128, 12>(tmem + TM_S32, tmem + TM_S32 + 64, x_re, x_re + 32, k_re, k_re + kIm, dhi, I64M, part);
             if (elect_one()) {
@@ -472,7 +481,7 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
 #pragma unroll 1
         for (int j = 0; j <= n_chunks; ++j) {
             if (j > 0) {
-                if (!wait_k_warp(mi, B_O_STAGED, j - 1)) return;
+                if (!wait_k_warp<kDiag>(mi, B_O_STAGED, j - 1)) return;
                 const ChunkInfo pc = prev.ci;
                 prev.next(p);
                 if (elect_one()) {
@@ -494,8 +503,8 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
                 __syncwarp();
                 if (j == n_chunks) break;
             }
-            if (!wait_k_warp(mi, B_E16_B, j)) return;
-            if (!wait_k_warp(mi, B_AQ_FULL0 + (j & 1), j >> 1)) return;
+            if (!wait_k_warp<kDiag>(mi, B_E16_B, j)) return;
+            if (!wait_k_warp<kDiag>(mi, B_AQ_FULL0 + (j & 1), j >> 1)) return;
             tc_fence_after();
             const uint32_t a_re = dlo + ((OFF_AQ + (j & 1) * 2 * kTile) >> 4);
             issue_complex<1, false, false, 2>(acc + 64, acc + 192, x_re, x_re + 32, a_re, a_re + kIm, dhi, I64, 2);
@@ -511,7 +520,7 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
         for (int i = 0; i < 2 && i < n_chunks; ++i, pcur.next(p)) prefetch_chunk(maps, pcur.ci);
 #pragma unroll 1
         for (int g = 0; g < n_chunks; ++g) {
-            if (g > 0 && !wait_k_warp(mi, B_R16_B, g - 1)) return;
+            if (g > 0 && !wait_k_warp<kDiag>(mi, B_R16_B, g - 1)) return;
             {
                 const ChunkInfo cv = vcur.ci;
                 vcur.next(p);
@@ -523,10 +532,10 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
             }
             const int s = g & 1;
             const uint32_t w_re = dlo + ((OFF_WQ + s * 4 * kTile) >> 4), k_re = dlo + ((OFF_KC + s * 2 * kTile) >> 4);
-            if (!wait_k_warp(mi, B_PREP_FULL0 + s, g >> 1)) return;
+            if (!wait_k_warp<kDiag>(mi, B_PREP_FULL0 + s, g >> 1)) return;
 #pragma unroll 1
             for (int gh = 0; gh < 2; ++gh) {
-                if (2 * g + gh > 0 && !wait_k_warp(mi, B_GRAM_DRAINED, 2 * g + gh - 1)) return;
+                if (2 * g + gh > 0 && !wait_k_warp<kDiag>(mi, B_GRAM_DRAINED, 2 * g + gh - 1)) return;
                 tc_fence_after();
                 // rows = [W ; Qt], columns = tokens i.  Re: W_re Kc_re + W_im Kc_im; Im: W_re Kc_im - W_im Kc_re
                 if (elect_one()) {
@@ -594,7 +603,7 @@ __device__ __forceinline__ float theta_from_raw(const Params &p, uint32_t bits)
 // recurrence on k_raw itself with beta s^2 in place of beta and v / s in place of v, so the operands carry the raw
 // key and the scales enter where beta and v do (SOLVE and CHAIN); |k_raw,t|^2 is the diagonal of the chunk's Gram
 // matrix, which the tensor core computes anyway.
-template <bool kFused>
+template <bool kFused, bool kDiag>
 __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int n_chunks, int pt)
 {
     [[maybe_unused]] long long *timing = p.timing;
@@ -606,9 +615,9 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
     const int c = quad * 32 + lane;
     const uint32_t tlane = tmem + ((uint32_t)(quad * 32) << 16);
     auto drain_outputs = [&](int jd) {           // rho of chunk jd -> bf16 staging tiles [t][128]
-        if (!dead && !wait_k(mi, B_UPD_DONE, jd)) dead = true;
+        if (!dead && !wait_k<kDiag>(mi, B_UPD_DONE, jd)) dead = true;
         // the Re staging tile is shared by all chunks: the store of chunk jd-1 must have read it
-        if (jd >= 1 && !dead && !wait_k(mi, B_STORE_DONE0 + ((jd - 1) & 1), (jd - 1) >> 1)) dead = true;
+        if (jd >= 1 && !dead && !wait_k<kDiag>(mi, B_STORE_DONE0 + ((jd - 1) & 1), (jd - 1) >> 1)) dead = true;
         tc_fence_after();
         if (half == 0 || p.has_o_im) {
             // Tensor memory is read in the 16-lane x 256-bit fragment shape (thread T: channel rows T / 4 and T / 4 + 8,
@@ -763,8 +772,8 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
 
             // the slot's tiles must have been consumed: W/Qt by rho_1 of chunk j-2, Kc by its state update
             if (j >= 2) {
-                if (!dead && !wait_k(mi, B_WQ_FREE0 + s, (j >> 1) - 1)) dead = true;
-                if (!dead && !wait_k(mi, B_KC_FREE0 + s, (j >> 1) - 1)) dead = true;
+                if (!dead && !wait_k<kDiag>(mi, B_WQ_FREE0 + s, (j >> 1) - 1)) dead = true;
+                if (!dead && !wait_k<kDiag>(mi, B_KC_FREE0 + s, (j >> 1) - 1)) dead = true;
             }
             SFDA_T(32);
         }
@@ -888,7 +897,7 @@ __device__ __forceinline__ void store_tile_s(const float (&cr)[4], const float (
 // drains Kt row t turns it into s_t = 1 / (|k_raw,t| + eps), scales its row of L by beta_t s_t^2, and leaves
 // beta_t s_t (the column scale of the M operand, which then maps the normalised R to E / s) and -s_t (for CHAIN's
 // R = v - s W_raw^* S_0) in shared memory.
-template <bool kFused>
+template <bool kFused, bool kDiag>
 __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int n_chunks, int st)
 {
     [[maybe_unused]] long long *timing = p.timing;
@@ -905,13 +914,13 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
         const int s = j & 1, ring = j & 3;
         // The Aq tile of this slot also staged o_im of chunk j-2: its rows are written straight from the drain,
         // so the warps that hold them wait for that store first.
-        if (row >= 64 && j >= 2 && !dead && !wait_k(mi, B_STORE_DONE0 + s, (j >> 1) - 1)) dead = true;
+        if (row >= 64 && j >= 2 && !dead && !wait_k<kDiag>(mi, B_STORE_DONE0 + s, (j >> 1) - 1)) dead = true;
         // ---- drain the two Gram halves (Re, then Im), 32 columns at a time
         float bt = 0.f;                           // beta of this thread's Kt row (PREP wrote it before the Gram ran)
 #pragma unroll 1
         for (int im = 0; im < 2; ++im) {
             SFDA_T(20 + 2 * im);
-            if (!dead && !wait_k(mi, B_GRAM_FULL, 2 * j + im)) dead = true;
+            if (!dead && !wait_k<kDiag>(mi, B_GRAM_FULL, 2 * j + im)) dead = true;
             tc_fence_after();
             if (im == 0 && row < 64) bt = mi.beta[ring][row];
             SFDA_T(21 + 2 * im);
@@ -1058,7 +1067,7 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
         SFDA_T(27);
 
         // ---- M_beta = X D_beta as a bf16 operand tile, once E of the previous chunk has read the old one
-        if (j >= 1 && !dead && !wait_k(mi, B_E_DONE, j - 1)) dead = true;
+        if (j >= 1 && !dead && !wait_k<kDiag>(mi, B_E_DONE, j - 1)) dead = true;
         SFDA_T(28);
         {
             const int t = st >> 1, part = st & 1;   // row t, columns 32 part .. 32 part + 31
@@ -1092,7 +1101,7 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
 }
 
 // ---- CHAIN --------------------------------------------------------------------------------------------
-template <bool kFused>
+template <bool kFused, bool kDiag>
 __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int n_chunks, int ct)
 {
     [[maybe_unused]] long long *timing = p.timing;
@@ -1110,7 +1119,7 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
     for (int j = 0; j <= n_chunks; ++j) {
         // ---- state pass: S_0 of this chunk = e^{i phi_C} a_C (accumulated state of the previous chunk)
         if (j > 0) {
-            if (!wait_k_warp(mi, B_UPD_DONE, j - 1)) return;
+            if (!wait_k_warp<kDiag>(mi, B_UPD_DONE, j - 1)) return;
             tc_fence_after();
         }
         SFDA_T(10);
@@ -1144,7 +1153,7 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
                 if (!prev_ci.seq_last) {     // one count per warp: the next piece may start once all eight have arrived
                     __threadfence();
                     __syncwarp();
-                    if (lane == 0) atomicAdd(p.flags + prev_ci.bh, 1u);
+                    if (lane == 0 && !(kDiag && p.withhold)) atomicAdd(p.flags + prev_ci.bh, 1u);
                 }
 #ifdef SFDA_WS_TIMING
                 if (ct == 0 && p.timing) p.timing[512 + blockIdx.x] = (long long)now_ns();
@@ -1164,7 +1173,7 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
                         asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(p.flags + ci.bh) : "memory");
                         if (seen >= want) break;
                         __nanosleep(200);
-                    } while (!mi.abort && (uint32_t)clock() - t0 < 0x80000000u);
+                    } while (!mi.abort && (uint32_t)clock() - t0 < (kDiag ? p.wait_limit : 0x80000000u));
                     ok = seen >= want;
                     if (!ok) mi.abort = 1;
                 }
@@ -1219,17 +1228,17 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
 #pragma unroll 1
         for (int ph = 0; ph < 2; ++ph) {
             if (ph == 0) {
-                if (!wait_k_warp(mi, B_D1_DONE, j)) return;
-                if (!wait_k_warp(mi, B_V_FULL, j)) return;
+                if (!wait_k_warp<kDiag>(mi, B_D1_DONE, j)) return;
+                if (!wait_k_warp<kDiag>(mi, B_V_FULL, j)) return;
             } else {
-                if (!wait_k_warp(mi, B_E_DONE, j)) return;
+                if (!wait_k_warp<kDiag>(mi, B_E_DONE, j)) return;
             }
             tc_fence_after();
             SFDA_T(13 + 2 * ph);
             const bool sub_v = ph == 0 && half == 0;            // R_re = V - D1_re
             const float sgn = ph == 0 ? -1.f : 1.f;             // R_im = -D1_im
             // fused: D1 was formed with the raw key, R = V - s D1; the per-token factor replaces the sign
-            if (kFused && ph == 0 && !wait_k_warp(mi, B_NORM_FULL, j)) return;
+            if (kFused && ph == 0 && !wait_k_warp<kDiag>(mi, B_NORM_FULL, j)) return;
             const uint32_t scp = smem_u32(ph == 0 ? &mi.kscale[(j & 3)][0] : &mi.ones[0]);
             // The second half of the accumulator is read into registers before the first half of the operand is
             // announced: the product which that announcement releases (E = M_beta R goes out in two halves of its K
@@ -1262,7 +1271,7 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
                     tc_wait_ld();
                 }
                 // R replaces S_0 in the operand columns: rho_1, the last reader of S_0, must be done
-                if (ph == 0 && pc == 0 && !wait_k_warp(mi, B_O1_DONE, j)) return;
+                if (ph == 0 && pc == 0 && !wait_k_warp<kDiag>(mi, B_O1_DONE, j)) return;
                 tmem_st<16>(tlane + TM_X16 + 32 * half + 16 * pc, pk);
                 tc_wait_st();
                 tc_fence_before();
@@ -1274,7 +1283,7 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
 }
 
 // ---- the kernel ---------------------------------------------------------------------------------------
-template <bool kFused>
+template <bool kFused, bool kDiag>
 __global__ void __launch_bounds__(kThreads, 1)
 sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
 {
@@ -1301,6 +1310,7 @@ sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
         init(B_E16_A, kChainWarps); init(B_E16_B, kChainWarps);
         init(B_O_STAGED, kPrepWarps); init(B_V_FULL, 1); init(B_NORM_FULL, 2);
         mi.abort = 0;
+        if (kDiag) mi.wait_limit = p.wait_limit;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (kFused && tid < C) mi.ones[tid] = 1.0f;
@@ -1315,17 +1325,17 @@ sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
 
     if (warp < kChainWarps) {
         regs_inc<kRegsWork>();
-        run_chain<kFused>(smem, mi, tmem, p, n_chunks, tid);
+        run_chain<kFused, kDiag>(smem, mi, tmem, p, n_chunks, tid);
     } else if (warp < kChainWarps + kSolveWarps) {
         regs_inc<kRegsWork>();
-        run_solve<kFused>(smem, mi, tmem, p, n_chunks, tid - kChainThreads);
+        run_solve<kFused, kDiag>(smem, mi, tmem, p, n_chunks, tid - kChainThreads);
     } else if (warp < kChainWarps + kSolveWarps + kPrepWarps) {
         regs_inc<kRegsWork>();
-        run_prep<kFused>(smem, mi, tmem, p, n_chunks, tid - kChainThreads - kSolveThreads);
+        run_prep<kFused, kDiag>(smem, mi, tmem, p, n_chunks, tid - kChainThreads - kSolveThreads);
     } else {
         regs_dec<kRegsCtrl>();
         const int cw = warp - (kChainWarps + kSolveWarps + kPrepWarps);
-        run_ctrl(cw, smem, mi, tmem, maps, p, n_chunks);
+        run_ctrl<kDiag>(cw, smem, mi, tmem, maps, p, n_chunks);
     }
 
     tc_fence_before();
@@ -1333,7 +1343,13 @@ sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
 #ifdef SFDA_WS_TIMING
     if (tid == 0 && p.timing) { p.timing[64 + 2 * blockIdx.x + 1] = (long long)now_ns(); if (blockIdx.x == 0) p.timing[401] = clock64(); }
 #endif
-    if (tid == 0 && mi.abort) atomicExch(p.status, 1u);
+    if (mi.abort) {
+        // a wait ran out: before the shared memory is given back, leave the copy engine time to land whatever this
+        // CTA still has in flight (its loads complete in a microsecond or two), then report
+        __nanosleep(20000);
+        __syncthreads();
+        if (tid == 0) atomicExch(p.status, 1u);
+    }
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem));
 }
 
@@ -1490,8 +1506,14 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
         !make_map(&maps.th, a.theta, a.B, a.T, a.H, true))
         return cudaErrorInvalidValue;
     const bool fused = a.fused != 0;
-    cudaError_t e = fused ? cudaFuncSetAttribute(sfda_forward_ws_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)
-                          : cudaFuncSetAttribute(sfda_forward_ws_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    // three instantiations: plain, raw inputs (stable parameterisation inside), and the diagnostic one whose waits
+    // take their limit from the launch
+    const bool diag = a.debug_withhold != 0 || a.wait_ticks != 0;
+    if (diag && fused) return cudaErrorInvalidValue;
+    const void *kernel = diag    ? reinterpret_cast<const void *>(sfda_forward_ws_kernel<false, true>)
+                         : fused ? reinterpret_cast<const void *>(sfda_forward_ws_kernel<true, false>)
+                                 : reinterpret_cast<const void *>(sfda_forward_ws_kernel<false, false>);
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     int dev = 0, n_sm = 0;
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
@@ -1500,6 +1522,11 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
     const int BH = a.B * a.H, NC = (a.T + C - 1) / C;
     int Q = 1, bal = 0;
     forward_ws_partition(BH, NC, n_sm, scratch_bytes >= forward_ws_scratch_bytes(a.B, a.H), &Q, &bal, nullptr);
+    if (a.debug_slices > 0) {      // diagnostic launches: the caller fixes the number of time slices
+        if (NC % a.debug_slices != 0 || scratch_bytes < forward_ws_scratch_bytes(a.B, a.H)) return cudaErrorInvalidValue;
+        Q = a.debug_slices;
+        bal = 0;
+    }
 #ifdef SFDA_WS_TIMING
     if (g_ws_force_q) { Q = g_ws_force_q; bal = 0; }
     if (g_ws_grid_cap && g_ws_grid_cap < n_sm) n_sm = g_ws_grid_cap;
@@ -1529,6 +1556,8 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
     p.T = a.T;
     p.H = a.H;
     p.has_o_im = a.o_im != nullptr;
+    p.wait_limit = a.wait_ticks ? a.wait_ticks : 0x80000000u;
+    p.withhold = a.debug_withhold;
     p.BH = BH;
     p.Q = Q;
     p.U = NC / Q;
@@ -1560,10 +1589,8 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
     attr[0].val.cooperative = pieces ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (fused)
-        e = cudaLaunchKernelEx(&cfg, sfda_forward_ws_kernel<true>, maps, p);
-    else
-        e = cudaLaunchKernelEx(&cfg, sfda_forward_ws_kernel<false>, maps, p);
+    void *kargs[2] = {&maps, &p};
+    e = cudaLaunchKernelExC(&cfg, kernel, kargs);
     if (e != cudaSuccess) return e;
     e = cudaGetLastError();
     if (e == cudaSuccess && launches) ++*launches;

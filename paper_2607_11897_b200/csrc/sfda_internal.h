@@ -18,6 +18,11 @@ struct ForwardArgs {
     float alpha_min = 0.f, alpha_max = 1.f, theta_max = 0.f, eps = 0.f;
     // tensor-core path, plain inputs only: [B][H][NC][m] chunk-closing integer phase, or nullptr
     uint32_t *phase_turns = nullptr;
+    // tensor-core path, diagnostic launches: device-side wait limit in SM-clock ticks (0: the default of about a
+    // second), a fixed number of time slices per sequence (0: the launcher's choice), and hand-offs between slices
+    // that are written but never announced (every later slice then waits until the limit and gives up)
+    uint32_t wait_ticks = 0;
+    int debug_slices = 0, debug_withhold = 0;
 };
 
 struct FactorArgs {

@@ -79,6 +79,63 @@ def all_pairs(cfg):
     return [(b, h) for b in range(cfg.B) for h in range(cfg.H)]
 
 
+# Regression guards of the bf16 tensor-core forward, beside the pass / fail bar TOL["bf16"] = 2e-2 of the task: the
+# measured errors are 5e-3 to 8e-3 (maximum) and 4.4e-3 to 4.6e-3 (root mean square, relative) on every
+# configuration; 1.5 times that must not be passed without somebody looking.
+GUARD_MAX, GUARD_RMS = 1.2e-2, 7.0e-3
+
+
+class ErrAcc:
+    """max |x - y| / max |y| and rms(x - y) / rms(y) of one output tensor, accumulated over batches of sequences."""
+
+    def __init__(self):
+        self.dmax = self.ymax = self.d2 = self.y2 = 0.0
+        self.n = 0
+
+    def add(self, got, want):
+        got = np.asarray(got, np.float64)
+        assert np.isfinite(got).all(), "non-finite GPU output"
+        d = got - want
+        self.dmax = max(self.dmax, float(np.abs(d).max()))
+        self.ymax = max(self.ymax, float(np.abs(want).max()))
+        self.d2 += float((d * d).sum())
+        self.y2 += float((want * want).sum())
+        self.n += d.size
+
+    @property
+    def max_rel(self):
+        return self.dmax / max(self.ymax, 1e-30)
+
+    @property
+    def rms_rel(self):
+        return float(np.sqrt(self.d2 / max(self.y2, 1e-300)))
+
+
+def check_all_sequences(name, pairs, oracle_batch, outputs, tol, guard=True, batch=64):
+    """Every sequence of `pairs` against the oracle, `batch` sequences at a time (what host memory holds);
+    `oracle_batch(sub_pairs)` returns the oracle's (o_re, o_im, S_T) of those sequences, `outputs` the GPU's
+    (o [B,T,H,dv], o_im or None, S_T [B,H,dk,dv] or None).  Prints and checks both error figures per tensor."""
+    o, o_im, S_T = outputs
+    acc = {"o_re": ErrAcc(), "o_im": ErrAcc(), "S_T": ErrAcc()}
+    for i in range(0, len(pairs), batch):
+        sub = pairs[i:i + batch]
+        w_re, w_im, w_S = oracle_batch(sub)
+        acc["o_re"].add(np.stack([o[b, :, h] for b, h in sub]), w_re)
+        if o_im is not None:
+            acc["o_im"].add(np.stack([o_im[b, :, h] for b, h in sub]), w_im)
+        if S_T is not None:
+            acc["S_T"].add(np.stack([S_T[b, h] for b, h in sub]), w_S)
+    report = {k: (a.max_rel, a.rms_rel) for k, a in acc.items() if a.n}
+    print("%s: %d sequences; max rel / rms rel: %s" % (
+        name, len(pairs), ", ".join("%s %.2e / %.2e" % (k, m, r) for k, (m, r) in report.items())))
+    for k, (m, r) in report.items():
+        assert m <= tol, "%s: %s max rel err %.3e above the bar %.1e" % (name, k, m, tol)
+        if guard:
+            assert m <= GUARD_MAX, "%s: %s max rel err %.3e above the regression guard %.1e" % (name, k, m, GUARD_MAX)
+            assert r <= GUARD_RMS, "%s: %s rms rel err %.3e above the regression guard %.1e" % (name, k, r, GUARD_RMS)
+    return report
+
+
 # ------------------------------------------------------------------------------------------------
 # forward
 # ------------------------------------------------------------------------------------------------
@@ -201,6 +258,48 @@ def test_forward_tensor_core_balanced_partition():
         assert np.array_equal(x, y)
 
 
+@pytest.mark.parametrize("case", ["product_exactly_e-80", "product_e-77", "product_e-40_uneven"])
+def test_forward_tensor_core_at_the_documented_decay_edge(case):
+    """The tensor-core path forms 1 / |gamma_t| inside a chunk and documents prod_chunk alpha >= e^-80 per coordinate
+    as its precondition.  Parity must hold up to that edge: a constant alpha = e^-1.25 (product over 64 tokens
+    e^-80), e^-1.2 (e^-76.8), and an uneven case (a third of the tokens at e^-1.8, the rest near 1)."""
+    cfg = workloads.CONFIGS[1].scaled(name="edge_" + case, B=1, T=256, H=3, s0_std=0.5, seed=321)
+    inp = dict(workloads.forward_inputs(cfg))
+    rng = np.random.default_rng(99)
+    if case == "product_exactly_e-80":
+        inp["alpha"] = np.full(inp["alpha"].shape, np.exp(-1.25), np.float32)
+    elif case == "product_e-77":
+        inp["alpha"] = np.full(inp["alpha"].shape, np.exp(-1.2), np.float32)
+    else:
+        strong = rng.uniform(0, 1, inp["alpha"].shape) < 1.0 / 3.0
+        inp["alpha"] = np.where(strong, np.exp(-1.8), rng.uniform(0.98, 1.0, inp["alpha"].shape)).astype(np.float32)
+    check_forward(cfg, inp, all_pairs(cfg), TOL["bf16"])
+
+
+@pytest.mark.parametrize("case", ["some_alpha_zero", "all_alpha_tiny", "alpha_u(0,1)"])
+def test_forward_tensor_core_beyond_the_decay_edge_stays_finite(case):
+    """Beyond the documented precondition (alpha = 0 is admissible in the recurrence, Section 3; Prop. "Basic
+    numerical stability") the tensor-core path promises finite results, not accuracy: every output and the final
+    state must be finite numbers, and the status must stay clean."""
+    cfg = workloads.CONFIGS[1].scaled(name="beyond_" + case, B=2, T=200, H=2, s0_std=0.5, seed=322)
+    inp = dict(workloads.forward_inputs(cfg))
+    rng = np.random.default_rng(98)
+    if case == "some_alpha_zero":
+        a = inp["alpha"].copy()
+        a[rng.uniform(0, 1, a.shape) < 0.1] = 0.0
+        inp["alpha"] = a
+    elif case == "all_alpha_tiny":
+        inp["alpha"] = np.full(inp["alpha"].shape, 1e-20, np.float32)
+    else:
+        inp["alpha"] = rng.uniform(0.0, 1.0, inp["alpha"].shape).astype(np.float32)
+    o, o_im, S_T = run_forward(cfg, inp)            # run_forward checks the status word
+    assert np.isfinite(o).all() and np.isfinite(o_im).all() and np.isfinite(S_T).all()
+    # the same inputs on the fp32 path, which has no such precondition, agree with the oracle
+    w = oracle_pairs(inp, all_pairs(cfg))
+    a = run_forward(cfg, inp, simt=True)
+    assert rel_err(np.stack([a[0][b, :, h] for b, h in all_pairs(cfg)]), w[0]) <= 5e-3
+
+
 def test_forward_tensor_core_optional_outputs_and_zero_state():
     """Tensor-core path without o_im, without S_T, and with S0 = NULL (zero state)."""
     cfg = workloads.CONFIGS[1].scaled(name="tc_opt", B=1, T=300, H=2, s0_std=0.0, seed=55)
@@ -286,27 +385,24 @@ def test_forward_tensor_core_matches_cuda_core_path():
 
 
 @pytest.mark.parametrize("idx", [1, 2])
-def test_forward_full_size_bf16_configs_sampled(idx):
-    """Configurations 1 and 2 at full size, in the launch configuration bench.py times;
-    the oracle recomputes a sample of (batch, head) sequences end to end."""
+def test_forward_full_size_bf16_configs_all_sequences(idx):
+    """Configurations 1 and 2 at full size, in the launch configuration bench.py times (configuration 2: 148
+    persistent CTAs, every sequence cut into time slices that hand their state over): EVERY (batch, head) sequence
+    against the oracle, element by element, so that a fault tied to a CTA, a slice boundary or a hand-off shows."""
     cfg = workloads.CONFIGS[idx]
     inp = workloads.forward_inputs(cfg)
-    pairs = [(0, 0), (cfg.B - 1, cfg.H - 1), (cfg.B // 2, 5), (1, cfg.H // 2)]
-    check_forward(cfg, inp, pairs, TOL["bf16"])
+    out = run_forward(cfg, inp)
+    check_all_sequences(cfg.name, all_pairs(cfg), lambda sub: oracle_pairs(inp, sub), out, TOL["bf16"])
 
 
 def test_forward_long_context_stability():
-    """Configuration 3 (T = 131072): parity on sampled heads, finite outputs, the Frobenius
+    """Configuration 3 (T = 131072): parity on all 16 sequences, finite outputs, the Frobenius
     bound of Prop. "Basic numerical stability", bit-exact cumulative phase turns."""
     cfg = workloads.CONFIGS[3]
     inp = workloads.forward_inputs(cfg)
-    pairs = [(0, 0), (0, 9)]
     o, o_im, S_T = run_forward(cfg, inp)
     assert np.isfinite(o).all() and np.isfinite(o_im).all() and np.isfinite(S_T).all()
-    w_re, w_im, w_S = oracle_pairs(inp, pairs)
-    assert rel_err(np.stack([o[b, :, h] for b, h in pairs]), w_re) <= TOL["bf16"]
-    assert rel_err(np.stack([o_im[b, :, h] for b, h in pairs]), w_im) <= TOL["bf16"]
-    assert rel_err(np.stack([S_T[b, h] for b, h in pairs]), w_S) <= TOL["bf16"]
+    check_all_sequences(cfg.name, all_pairs(cfg), lambda sub: oracle_pairs(inp, sub), (o, o_im, S_T), TOL["bf16"], batch=8)
     # ||S_T||_F <= ||S_0||_F + sum beta |k| |v|
     for h in range(cfg.H):
         bound = np.sum(inp["beta"][0, :, h].astype(np.float64)
@@ -420,13 +516,14 @@ def run_decode(cfg, steps, pairs):
     out_im = torch.empty_like(out)
     keys = ("q", "k", "v", "alpha", "theta", "beta")
     sampled = {k: [] for k in keys}
+    bsel, hsel = np.array([p[0] for p in pairs]), np.array([p[1] for p in pairs])
     window = 32
     with ThreadPoolExecutor(max_workers=8) as pool:
         for s0 in range(0, steps, window):
             batch = list(pool.map(lambda s: workloads.decode_step_inputs(cfg, s), range(s0, min(s0 + window, steps))))
             for i, x in enumerate(batch):
                 for k in keys:
-                    sampled[k].append(np.stack([x[k][b, h] for b, h in pairs]))
+                    sampled[k].append(x[k][bsel, hsel])
                 d = {k: to_dev(v, cfg, k) for k, v in x.items()}
                 sfda.sfda_step(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], S, o, o_im)
                 out[s0 + i] = o[bi, hi].float()
@@ -456,10 +553,13 @@ def test_step_small(d_k, d_v, dtype):
 
 
 def test_step_full_size_decode_config():
-    """Configuration 4: B = 256 sequences, H = 32, 1024 consecutive steps; the oracle follows a
-    sample of (batch, head) states through all steps."""
+    """Configuration 4: B = 256 sequences, H = 32, 1024 consecutive steps; the oracle follows 256
+    (batch, head) states through all steps."""
     cfg = workloads.CONFIGS[4]
-    check_decode(cfg, [(0, 0), (255, 31), (100, 7), (31, 16)], TOL["bf16"], 1e-4)
+    # 256 of the 8192 states, spread evenly (one in 32: state index 32 i + (i mod 32) visits every head and, with two
+    # CTAs per state and four resident CTAs per SM, every SM of every wave)
+    pairs = [divmod(32 * i + (i % 32), cfg.H) for i in range(256)]
+    check_decode(cfg, pairs, TOL["bf16"], 1e-4)
 
 
 def test_iterated_step_equals_forward():
@@ -768,21 +868,18 @@ def test_forward_fused_equals_frontend_then_forward_on_fp32_keys():
     assert rel_err(o_f, o_u) <= TOL["bf16"] and rel_err(oi_f, oi_u) <= TOL["bf16"] and rel_err(S_f, S_u) <= TOL["bf16"]
 
 
-def test_forward_fused_full_size_headline_sampled():
+def test_forward_fused_full_size_headline_all_sequences():
     """The headline sizes on raw inputs, in the launch configuration bench.py times for the fused forward;
-    the oracle recomputes a sample of (batch, head) sequences end to end.  Also the property that holds for
-    every sequence: ||S_T||_F <= ||S_0||_F + sum_t beta_t ||v_t|| (Prop. "Basic numerical stability",
+    the oracle recomputes every (batch, head) sequence end to end.  Also the bound
+    ||S_T||_F <= ||S_0||_F + sum_t beta_t ||v_t|| (Prop. "Basic numerical stability",
     with |k_t| <= 1 from the parameterisation)."""
     cfg = workloads.CONFIGS[2]
     raw = workloads.forward_raw_inputs(cfg)
-    pairs = [(0, 0), (cfg.B - 1, cfg.H - 1), (cfg.B // 2, 5), (1, cfg.H // 2)]
     o, o_im, S_T, launches, ws = run_forward_fused(cfg, raw, PARAM)
     assert launches == 1 and sfda.sfda_workspace_status(ws) == 0
     assert np.isfinite(o).all() and np.isfinite(o_im).all() and np.isfinite(S_T).all()
-    w_re, w_im, w_S = oracle_fused_pairs(raw, pairs, PARAM)
-    assert rel_err(np.stack([o[b, :, h] for b, h in pairs]), w_re) <= TOL["bf16"]
-    assert rel_err(np.stack([o_im[b, :, h] for b, h in pairs]), w_im) <= TOL["bf16"]
-    assert rel_err(np.stack([S_T[b, h] for b, h in pairs]), w_S) <= TOL["bf16"]
+    check_all_sequences("fused " + cfg.name, all_pairs(cfg), lambda sub: oracle_fused_pairs(raw, sub, PARAM),
+                        (o, o_im, S_T), TOL["bf16"])
     beta = 1.0 / (1.0 + np.exp(-raw["c_raw"].astype(np.float64)))
     vnorm = np.linalg.norm(raw["v"].astype(np.float64), axis=-1)
     bound = np.linalg.norm(raw["S0"].astype(np.float64).reshape(cfg.B, cfg.H, -1), axis=-1) \
@@ -1533,3 +1630,120 @@ def test_concurrent_calls_from_host_threads():
             assert sfda.sfda_workspace_status(out[3]) == 0
             for a, b in zip(out[:3], serial[i][:3]):
                 assert torch.equal(a, b)
+
+
+# ------------------------------------------------------------------------------------------------
+# timing perturbation: a build whose roles pause at random must reproduce the plain build bit for bit
+# ------------------------------------------------------------------------------------------------
+def test_forward_results_do_not_depend_on_the_timing_of_the_roles():
+    """The tensor-core forward hands tiles between four concurrently running roles through barriers.  No result
+    may depend on how fast a role runs; a development build of the library (-DSFDA_WS_CHAOS) pauses every role for
+    0.1 to 1.1 microseconds after one in eight barrier arrivals and completed waits.  A missing or misplaced
+    synchronisation (a tile announced before it is complete, an accumulator read after the next product has
+    started it from zero) shows as a bit difference between that build and the plain one.  Shapes: a ragged tail,
+    time slices with hand-off between CTAs, the balanced partition, raw inputs, the two-level scan."""
+    from paper_2607_11897_b200 import binding, build as cuda_build
+    chaos = binding.load_library(cuda_build.build_variant("chaos", ["-DSFDA_WS_CHAOS"]))
+    plain = binding.load()
+
+    def with_lib(lib, fn):
+        binding._LIB = lib
+        try:
+            return fn()
+        finally:
+            binding._LIB = plain
+
+    def forward_case(B, T, H, s0, want_im, cut):
+        cfg = workloads.CONFIGS[2].scaled(name="chaos", B=B, T=T, H=H, s0_std=s0, seed=900 + B + T + H)
+        inp = workloads.forward_inputs(cfg)
+        d = {k: (None if v is None else to_dev(v, cfg, k)) for k, v in inp.items()}
+        nws = sfda.sfda_workspace_bytes(B, T, H, 128, 128, 64, 1) if cut else 256
+
+        def run():
+            o = torch.empty(B, T, H, 128, device=DEV, dtype=torch.bfloat16)
+            o_im = torch.empty_like(o) if want_im else None
+            S_T = torch.empty(B, H, 128, 128, device=DEV)
+            ws = torch.empty(nws, device=DEV, dtype=torch.uint8)
+            sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im, S_T, 64, ws)
+            torch.cuda.synchronize()
+            assert sfda.sfda_workspace_status(ws) == 0
+            return [o, S_T] + ([o_im] if want_im else [])
+        return run
+
+    def fused_case(B, T, H):
+        cfg = workloads.CONFIGS[2].scaled(name="chaosf", B=B, T=T, H=H, s0_std=0.02, seed=950 + T)
+        raw = workloads.forward_raw_inputs(cfg)
+        return lambda: [torch.from_numpy(x) for x in run_forward_fused(cfg, raw, PARAM)[:3]]
+
+    def two_level_case(B, T, H, n):
+        cfg = workloads.CONFIGS[3].scaled(name="chaos2", B=B, T=T, H=H, s0_std=0.3, seed=970)
+        inp = workloads.forward_inputs(cfg)
+        d = {k: (None if v is None else to_dev(v, cfg, k)) for k, v in inp.items()}
+
+        def run():
+            o = torch.empty(B, T, H, 128, device=DEV, dtype=torch.bfloat16)
+            o_im = torch.empty_like(o)
+            S_T = torch.empty(B, H, 128, 128, device=DEV)
+            ws = torch.empty(sfda.sfda_forward_two_level_workspace_bytes(B, T, H, 128, 128, 64, 1, n), device=DEV,
+                             dtype=torch.uint8)
+            sfda.sfda_forward_two_level(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im, S_T,
+                                        64, n, ws)
+            torch.cuda.synchronize()
+            return [o, o_im, S_T]
+        return run
+
+    cases = {
+        "ragged tail, B = 4": forward_case(4, 1029, 8, 0.02, True, True),
+        "time slices with hand-off (150 sequences of 64 chunks)": forward_case(1, 4096, 150, 0.02, True, True),
+        "balanced partition (149 sequences of 4 chunks)": forward_case(1, 256, 149, 0.0, False, True),
+        "uncut, one head": forward_case(2, 2048, 1, 0.02, True, False),
+        "raw inputs": fused_case(3, 1029, 2),
+        "raw inputs, time slices": fused_case(1, 2048, 150),
+        "two-level scan": two_level_case(1, 4096, 3, 8),
+    }
+    for name, run in cases.items():
+        want = with_lib(plain, run)
+        for rep in range(3):
+            got = with_lib(chaos, run)
+            for x, y in zip(got, want):
+                assert torch.equal(x, y), "%s: the build with random pauses differs from the plain build (launch %d)" % (name, rep)
+
+
+# ------------------------------------------------------------------------------------------------
+# a bounded device-side wait that runs out (no fault: the kernel gives up, reports, and ends)
+# ------------------------------------------------------------------------------------------------
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    """Two sequences of eight chunks, each cut into two time slices on four CTAs; the diagnostic launch writes the
+    boundary states but never announces them, with the wait limit at 2^20 ticks of the SM clock (about half a
+    millisecond).  The two CTAs that run second slices wait for their predecessors until the limit, give up, all
+    their roles leave, tensor memory is freed and the kernel ends; the status word reads SFDA_ERR_TIMEOUT.  The first
+    slices' outputs are still right, and an ordinary call on the same workspace afterwards is right everywhere."""
+    cfg = workloads.CONFIGS[1].scaled(name="timeout", B=1, T=512, H=2, s0_std=0.1, seed=611)
+    inp = workloads.forward_inputs(cfg)
+    d = {k: (None if v is None else to_dev(v, cfg, k)) for k, v in inp.items()}
+    o = torch.zeros(cfg.B, cfg.T, cfg.H, 128, device=DEV, dtype=torch.bfloat16)
+    o_im = torch.zeros_like(o)
+    S_T = torch.zeros(cfg.B, cfg.H, 128, 128, device=DEV)
+    ws = torch.empty(sfda.sfda_workspace_bytes(cfg.B, cfg.T, cfg.H, 128, 128, 64, 1), device=DEV, dtype=torch.uint8)
+    w_re, w_im, w_S = oracle_pairs(inp, all_pairs(cfg))
+    sfda.sfda_forward_withheld_handoff(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im, S_T,
+                                       64, 2, 1 << 20, ws)
+    with pytest.raises(sfda.SfdaError) as e:
+        sfda.sfda_workspace_status(ws)
+    assert e.value.status == -7
+    half = cfg.T // 2                                    # first slices: tokens 0 .. T/2 - 1 of both sequences
+    got = np.stack([o.float().cpu().numpy()[0, :half, h] for h in range(cfg.H)])
+    assert rel_err(got, w_re[:, :half]) <= TOL["bf16"]
+    # argument checks of the diagnostic itself
+    for slices, ticks, code in ((1, 1 << 20, -8), (2, 1 << 10, -8), (2, 1 << 30, -8), (3, 1 << 20, -2)):
+        with pytest.raises(sfda.SfdaError) as e:
+            sfda.sfda_forward_withheld_handoff(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im,
+                                               S_T, 64, slices, ticks, ws)
+        assert e.value.status == code
+    # the context is intact: the ordinary call, on the very same workspace
+    sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im, S_T, 64, ws)
+    assert sfda.sfda_workspace_status(ws) == 0
+    on, oin, Sn = o.float().cpu().numpy(), o_im.float().cpu().numpy(), S_T.cpu().numpy()
+    assert rel_err(np.stack([on[0, :, h] for h in range(cfg.H)]), w_re) <= TOL["bf16"]
+    assert rel_err(np.stack([oin[0, :, h] for h in range(cfg.H)]), w_im) <= TOL["bf16"]
+    assert rel_err(np.stack([Sn[0, h] for h in range(cfg.H)]), w_S) <= TOL["bf16"]
