@@ -70,8 +70,6 @@ static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA exceeded");
 
 enum Bar {
     B_PREP_FULL0, B_PREP_FULL1,     // PREP -> CTRL: W/Qt/Kc tiles of the slot are written
-    B_WQ_FREE0, B_WQ_FREE1,         // commit: rho_1 (last reader of the slot's W/Qt tiles) has run
-    B_KC_FREE0, B_KC_FREE1,         // commit: the state update (last reader of the slot's Kc tile) has run
     B_STORE_DONE0, B_STORE_DONE1,   // CTRL: the output store of a chunk of this parity has read its staging
     B_GRAM_FULL, B_GRAM_DRAINED,    // commit / SOLVE: one Gram half is in tensor memory / has been read out
     B_MB_FULL, B_AQ_FULL0, B_AQ_FULL1,
@@ -83,6 +81,18 @@ enum Bar {
     kNumBars
 };
 
+// One chunk of a CTA's stream of chunks (see ChunkCursor below).
+struct __align__(16) ChunkInfo {
+    int b, h, bh, jg;           // sequence, chunk index inside the sequence
+    uint32_t want;              // arrivals at the sequence's counter that the piece waits for (unless seq_first)
+    bool first;                 // first chunk of its piece
+    bool seq_first, seq_last;   // the piece starts / ends its sequence
+    bool pad_;
+    int pad2_[2];
+};
+static_assert(sizeof(ChunkInfo) == 32, "ring entries are copied as two 16-byte words");
+constexpr int kRing = 8;        // chunks whose description is kept (the roles are at most a few chunks apart)
+
 struct Misc {
     float part_lg[2][8][M];                 // per-group partial products / phase sums, two chunks deep
     uint32_t part_turns[2][8][M];
@@ -90,6 +100,8 @@ struct Misc {
     float beta[4][C];
     float kscale[4][C];                     // fused front end: -1 / (|k_raw| + eps) per token, ring of four chunks
     float ones[C];                          //                  +1: the scale of the passes that apply none
+    uint4 cursor_raw[3];                    // the prologue's cursor (a ChunkCursor), taken over by PREP
+    ChunkInfo ring[kRing];                  // description of chunk j at ring[j % kRing], published by PREP two chunks ahead
     unsigned long long bars[kNumBars];
     uint32_t tmem_base;
     uint32_t wait_limit;                    // SM-clock ticks after which a wait gives up
@@ -161,12 +173,6 @@ struct Maps {
 // pass notices a boundary (it writes the finished state out and takes the next one in).  A piece that does not
 // start its sequence begins from the boundary state its predecessor left in `handoff`; its CTA waits for that
 // (bounded).  All CTAs are resident (cooperative launch).
-struct ChunkInfo {
-    int b, h, bh, jg;           // sequence, chunk index inside the sequence
-    uint32_t want;              // arrivals at the sequence's counter that the piece waits for (unless seq_first)
-    bool first;                 // first chunk of its piece
-    bool seq_first, seq_last;   // the piece starts / ends its sequence
-};
 // Walks the stream chunk by chunk; the quotients are taken once per piece, not once per chunk.
 struct ChunkCursor {
     ChunkInfo ci;
@@ -208,6 +214,20 @@ struct ChunkCursor {
         ci.h = ci.bh - ci.b * p.H;
         ci.first = true;
     }
+    ChunkCursor() = default;
+    // hand-over through shared memory (three 16-byte words)
+    __device__ __forceinline__ void store(uint4 *dst) const
+    {
+        const uint4 *src = reinterpret_cast<const uint4 *>(this);
+        dst[0] = src[0]; dst[1] = src[1]; dst[2] = src[2];
+    }
+    static __device__ __forceinline__ ChunkCursor load(const uint4 *src)
+    {
+        ChunkCursor c;
+        uint4 *dst = reinterpret_cast<uint4 *>(&c);
+        dst[0] = src[0]; dst[1] = src[1]; dst[2] = src[2];
+        return c;
+    }
     __device__ __forceinline__ explicit ChunkCursor(const Params &p) : u((int)blockIdx.x)
     {
         if (p.bal) {
@@ -234,6 +254,28 @@ struct ChunkCursor {
         }
     }
 };
+
+// The chunks' descriptions go through a small ring in shared memory: ONE thread (of PREP) walks the cursor, two
+// chunks ahead of PREP's own work, and every role reads chunk j's entry after an event that is ordered behind its
+// publication (the start of the kernel for chunks 0 and 1; for chunk j >= 2 the tiles of chunk j - 2, which PREP
+// announces after publishing).  That keeps the cursor's code out of the other roles' loops.
+__device__ __forceinline__ void ring_put(Misc &mi, int j, const ChunkInfo &ci)
+{
+    const uint4 *src = reinterpret_cast<const uint4 *>(&ci);
+    uint4 *dst = reinterpret_cast<uint4 *>(&mi.ring[j & (kRing - 1)]);
+    dst[0] = src[0];
+    dst[1] = src[1];
+}
+__device__ __forceinline__ ChunkInfo ring_get(const Misc &mi, int j)
+{
+    ChunkInfo ci;
+    const uint4 *src = reinterpret_cast<const uint4 *>(&mi.ring[j & (kRing - 1)]);
+    reinterpret_cast<uint4 *>(&ci)[0] = src[0];
+    reinterpret_cast<uint4 *>(&ci)[1] = src[1];
+    return ci;
+}
+
+static_assert(sizeof(ChunkCursor) == 48, "the cursor is handed over as three 16-byte words");
 
 // Development builds only (-DSFDA_WS_CHAOS): a pseudo-random pause of 0.1 to 1.1 us after one in eight barrier
 // arrivals and completed waits.  The results do not depend on timing, so a build with the pauses must reproduce
@@ -391,15 +433,12 @@ __device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap *map, int c0, 
                  "r"(c0), "r"(c1), "r"(c2), "r"(c3)
                  : "memory");
 }
-__device__ __forceinline__ void prefetch_chunk(const Maps &maps, const ChunkInfo &ci)
+__device__ __forceinline__ void prefetch_chunk(const Maps &maps, const ChunkInfo &ci)   // one thread
 {
-    if (elect_one()) {
-        tma_prefetch_4d(&maps.al, 0, ci.h, ci.jg * C, ci.b);
-        tma_prefetch_4d(&maps.th, 0, ci.h, ci.jg * C, ci.b);
-        tma_prefetch_4d(&maps.k, 0, ci.h, ci.jg * C, ci.b);
-        tma_prefetch_4d(&maps.q, 0, ci.h, ci.jg * C, ci.b);
-    }
-    __syncwarp();
+    tma_prefetch_4d(&maps.al, 0, ci.h, ci.jg * C, ci.b);
+    tma_prefetch_4d(&maps.th, 0, ci.h, ci.jg * C, ci.b);
+    tma_prefetch_4d(&maps.k, 0, ci.h, ci.jg * C, ci.b);
+    tma_prefetch_4d(&maps.q, 0, ci.h, ci.jg * C, ci.b);
 }
 
 // The issuing work is split over four warps (they sit on different schedulers):
@@ -446,7 +485,6 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
             issue_complex<3, true, false, 2>(acc + 64, acc + 192, x_re, x_re + 32, w_re + kIm, w_re + 3 * kIm, dhi, I64, part);
             if (elect_one()) {
                 mma_commit(&bars[B_O1_DONE]);
-                mma_commit(&bars[B_WQ_FREE0 + s]);
             }
             SFDA_T(1);
             // E = M_beta R (R arrives in two halves of 32 tokens = two k-steps each)
@@ -470,20 +508,17 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
             tc_fence_after();
             issue_complex<1, false, true, 128, 12>(tmem + TM_S32, tmem + TM_S32 + 64, x_re, x_re + 32, k_re, k_re + kIm, dhi, I64M, part);
             if (elect_one()) {
-                mma_commit(&bars[B_KC_FREE0 + s]);
                 mma_commit(&bars[B_UPD_DONE]);
             }
             SFDA_T(6);
         }
     } else if (role == 1) {
-        ChunkCursor prev(p);             // the chunk whose outputs are stored next
         // iteration j: store the outputs of chunk j - 1 (once staged), then issue rho += Aq E of chunk j
 #pragma unroll 1
         for (int j = 0; j <= n_chunks; ++j) {
             if (j > 0) {
                 if (!wait_k_warp<kDiag>(mi, B_O_STAGED, j - 1)) return;
-                const ChunkInfo pc = prev.ci;
-                prev.next(p);
+                const ChunkInfo pc = ring_get(mi, j - 1);
                 if (elect_one()) {
                     tma_store_4d(tm_o, smem + OFF_OST, 0, pc.h, pc.jg * C, pc.b);
                     tma_store_4d(tm_o, smem + OFF_OST + kTile, 64, pc.h, pc.jg * C, pc.b);
@@ -515,15 +550,11 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
         // consumed (R of that chunk is built); then the two Gram halves of chunk g, each once its operands are
         // written and the Gram columns have been read out.  Blocking waits: a polling loop here would take issue
         // slots from the warps that do the work.
-        ChunkCursor vcur(p), pcur(p);            // chunk g below; the chunk whose inputs are prefetched next
-#pragma unroll 1
-        for (int i = 0; i < 2 && i < n_chunks; ++i, pcur.next(p)) prefetch_chunk(maps, pcur.ci);
 #pragma unroll 1
         for (int g = 0; g < n_chunks; ++g) {
             if (g > 0 && !wait_k_warp<kDiag>(mi, B_R16_B, g - 1)) return;
             {
-                const ChunkInfo cv = vcur.ci;
-                vcur.next(p);
+                const ChunkInfo cv = ring_get(mi, g);
                 if (elect_one()) {
                     mbar_expect_tx(&bars[B_V_FULL], 16384);
                     tma_load_4d(smem + OFF_V, tm_v, &bars[B_V_FULL], 0, cv.h, cv.jg * C, cv.b);
@@ -550,10 +581,11 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
                 }
                 __syncwarp();
             }
-            // PREP has finished chunk g: time to bring the inputs of chunk g + 2 into L2
+            // PREP has finished chunk g and, before that, described chunk g + 2: time to bring its inputs into L2
             if (g + 2 < n_chunks) {
-                prefetch_chunk(maps, pcur.ci);
-                pcur.next(p);
+                const ChunkInfo cp = ring_get(mi, g + 2);
+                if (elect_one()) prefetch_chunk(maps, cp);
+                __syncwarp();
             }
         }
     }
@@ -604,7 +636,8 @@ __device__ __forceinline__ float theta_from_raw(const Params &p, uint32_t bits)
 // key and the scales enter where beta and v do (SOLVE and CHAIN); |k_raw,t|^2 is the diagonal of the chunk's Gram
 // matrix, which the tensor core computes anyway.
 template <bool kFused, bool kDiag>
-__device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int n_chunks, int pt)
+__device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem, const Maps &maps, const Params &p,
+                                         int n_chunks, int pt)
 {
     [[maybe_unused]] long long *timing = p.timing;
     const int jp = pt & 31, tq = pt >> 5;   // channel pair (channels 2jp, 2jp+1), token octet (8 tokens)
@@ -652,7 +685,7 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
         warp_arrive(&mi.bars[B_O_STAGED]);
     };
     SFDA_TDECL(pt == 0);
-    ChunkCursor cur(p);
+    ChunkCursor cur = ChunkCursor::load(mi.cursor_raw);   // at chunk 2: chunks 0 and 1 were published before the roles started
 #pragma unroll 1
     for (int j = 0; j < n_chunks + 2; ++j) {
         const bool live = j < n_chunks;          // after the last chunk only the outputs of two chunks are left
@@ -681,8 +714,13 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
             tk[ii].k = make_uint2(0u, 0u); tk[ii].q = make_uint2(0u, 0u);
         }
         if (live) {
-            const ChunkInfo ci = cur.ci;
-            cur.next(p);
+            // chunk j + 2: its description for the other roles (the warp that issues the Gram products reads it once this
+            // chunk's tiles are announced, and asks for that chunk's q, k, alpha, theta tiles to be brought into L2)
+            if (j + 2 < n_chunks) {
+                if (pt == 0) ring_put(mi, j + 2, cur.ci);
+                cur.next(p);
+            }
+            const ChunkInfo ci = ring_get(mi, j);
             const int t0 = ci.jg * C, len = min(C, p.T - t0);
             const size_t row0 = ((size_t)ci.b * p.T + t0) * p.H + ci.h;   // token t of this head: row0 + t * H
             nt = min(8, max(0, len - tq * 8));
@@ -770,11 +808,8 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
             }
             SFDA_T(31);
 
-            // the slot's tiles must have been consumed: W/Qt by rho_1 of chunk j-2, Kc by its state update
-            if (j >= 2) {
-                if (!dead && !wait_k<kDiag>(mi, B_WQ_FREE0 + s, (j >> 1) - 1)) dead = true;
-                if (!dead && !wait_k<kDiag>(mi, B_KC_FREE0 + s, (j >> 1) - 1)) dead = true;
-            }
+            // (the slot's tiles, last read by the state update of chunk j-2, are free once that chunk's products are
+            // complete, which the read-out of its outputs below waits for)
             SFDA_T(32);
         }
         // the state update of chunk j-2 has just finished (it freed Kc above): read out that chunk's outputs,
@@ -1113,8 +1148,7 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
     const uint32_t sv = smem_u32(smem) + OFF_V + 2 * c;   // v[t][c], rows of 256 bytes
 
     SFDA_TDECL(ct == 0);
-    ChunkCursor cur(p);
-    ChunkInfo prev_ci = cur.ci;
+    ChunkInfo prev_ci = ring_get(mi, 0);
 #pragma unroll 1
     for (int j = 0; j <= n_chunks; ++j) {
         // ---- state pass: S_0 of this chunk = e^{i phi_C} a_C (accumulated state of the previous chunk)
@@ -1123,8 +1157,8 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
             tc_fence_after();
         }
         SFDA_T(10);
-        const ChunkInfo ci = cur.ci;
         const bool fin = j == n_chunks;
+        const ChunkInfo ci = fin ? prev_ci : ring_get(mi, j);
         const float2 *close = mi.close[(j - 1) & 3];
         const float *src = nullptr;
         if (fin || ci.first) {
@@ -1219,7 +1253,6 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
             warp_arrive(&mi.bars[B_S16_A + pc]);   // this half of the operand is complete
         }
         prev_ci = ci;
-        cur.next(p);
         SFDA_T(11);
 
         // ---- R = V - D1 (ph 0), then E (ph 1), -> bf16 A operand: 64 fp32 accumulator columns of this warp's half
@@ -1300,7 +1333,6 @@ sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
     if (tid == 0) {
         auto init = [&](int bar, uint32_t count) { mbar_init(&mi.bars[bar], count); };
         init(B_PREP_FULL0, kPrepWarps); init(B_PREP_FULL1, kPrepWarps);
-        init(B_WQ_FREE0, 2); init(B_WQ_FREE1, 2); init(B_KC_FREE0, 2); init(B_KC_FREE1, 2);   // both issuing warps
         init(B_STORE_DONE0, 1); init(B_STORE_DONE1, 1);
         init(B_GRAM_FULL, 1); init(B_GRAM_DRAINED, kSolveWarps);
         init(B_MB_FULL, kSolveWarps); init(B_AQ_FULL0, kSolveWarps); init(B_AQ_FULL1, kSolveWarps);
@@ -1314,6 +1346,18 @@ sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (kFused && tid < C) mi.ones[tid] = 1.0f;
+    if (tid == kChainThreads + kSolveThreads) {
+        // PREP's first thread walks the stream of chunks for everybody: chunks 0 and 1 are described (and their inputs
+        // requested into L2) before the roles start; it goes on from there inside PREP, two chunks ahead
+        ChunkCursor cur(p);
+#pragma unroll 1
+        for (int i = 0; i < 2 && i < n_chunks; ++i) {
+            ring_put(mi, i, cur.ci);
+            prefetch_chunk(maps, cur.ci);
+            cur.next(p);
+        }
+        cur.store(mi.cursor_raw);
+    }
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&mi.tmem_base)));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
@@ -1331,7 +1375,7 @@ sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
         run_solve<kFused, kDiag>(smem, mi, tmem, p, n_chunks, tid - kChainThreads);
     } else if (warp < kChainWarps + kSolveWarps + kPrepWarps) {
         regs_inc<kRegsWork>();
-        run_prep<kFused, kDiag>(smem, mi, tmem, p, n_chunks, tid - kChainThreads - kSolveThreads);
+        run_prep<kFused, kDiag>(smem, mi, tmem, maps, p, n_chunks, tid - kChainThreads - kSolveThreads);
     } else {
         regs_dec<kRegsCtrl>();
         const int cw = warp - (kChainWarps + kSolveWarps + kPrepWarps);
