@@ -96,7 +96,7 @@ constexpr int kRing = 8;        // chunks whose description is kept (the roles a
 struct Misc {
     float part_lg[2][8][M];                 // per-group partial products / phase sums, two chunks deep
     uint32_t part_turns[2][8][M];
-    float2 close[4][M];                     // a_C e^{i phi_C} of a ring of four chunks
+    float close_re[4][M], close_im[4][M];   // a_C e^{i phi_C} of a ring of four chunks, real and imaginary parts
     float beta[4][C];
     float kscale[4][C];                     // fused front end: -1 / (|k_raw| + eps) per token, ring of four chunks
     float ones[C];                          //                  +1: the scale of the passes that apply none
@@ -716,7 +716,7 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
         if (live) {
             // chunk j + 2: its description for the other roles (the warp that issues the Gram products reads it once this
             // chunk's tiles are announced, and asks for that chunk's q, k, alpha, theta tiles to be brought into L2)
-            if (j + 2 < n_chunks) {
+            if (tq == 0 && j + 2 < n_chunks) {       // (the first warp alone walks the cursor)
                 if (pt == 0) ring_put(mi, j + 2, cur.ci);
                 cur.next(p);
             }
@@ -799,8 +799,8 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
                     // on request so that it can be compared bit for bit
                     if (!kFused && p.phase_out)
                         *reinterpret_cast<uint2 *>(p.phase_out + ((size_t)ci.bh * p.NC + ci.jg) * M + 2 * jp) = make_uint2(tb0, tb1);
-                    mi.close[ring][2 * jp] = g0;
-                    mi.close[ring][2 * jp + 1] = g1;
+                    *reinterpret_cast<float2 *>(&mi.close_re[ring][2 * jp]) = make_float2(g0.x, g1.x);
+                    *reinterpret_cast<float2 *>(&mi.close_im[ring][2 * jp]) = make_float2(g0.y, g1.y);
                     g0 = make_float2(1.f, 0.f); g1 = g0; base0 = 1.f; base1 = 1.f;
                 }
                 ainv0 = fminf(__fdividef(1.0f, base0), 5.5e34f);          // 1/a, capped at e^80
@@ -823,39 +823,47 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
         // registers of the token kTB places before it as soon as that one has been worked on.
         const uint32_t wq_re = smem_u32(smem) + OFF_WQ + s * 4 * kTile + tq * 1024 + (jp & 3) * 4;   // + row, swizzle
         const uint32_t kc_re = smem_u32(smem) + OFF_KC + s * 2 * kTile + tq * 1024 + (jp & 3) * 4;
+        // The thread's two coordinates go through the arithmetic side by side as packed pairs (one instruction for both):
+        // this role is short of issue slots, not of floating-point throughput.
+        float2 gx2 = make_float2(g0.x, g1.x), gy2 = make_float2(g0.y, g1.y), ainv2 = make_float2(ainv0, ainv1);
 #pragma unroll 1
         for (int h = 0; h < 8 / kTB; ++h) {
 #pragma unroll
             for (int ii = 0; ii < kTB; ++ii) {
                 const int i = h * kTB + ii;
-                float wr[2], wi[2], cr_[2], ci_[2], qr_[2], qi_[2];
-#pragma unroll
-                for (int x = 0; x < 2; ++x) {
-                    // gamma_t = gamma_{t-1} alpha_t e^{i theta_t}; 1/a_t alongside (capped at e^80)
-                    const uint32_t al_bits = x ? tk[ii].al.y : tk[ii].al.x, th_bits = x ? tk[ii].th.y : tk[ii].th.x;
-                    const float al = fmaxf(kFused ? alpha_from_raw(p, al_bits) : __uint_as_float(al_bits), 9.0e-14f);   // floor e^-30
-                    float cs, sn;
-                    __sincosf(kFused ? theta_from_raw(p, th_bits) : __uint_as_float(th_bits), &sn, &cs);
-                    float2 &g = x ? g1 : g0;
-                    float &ainv = x ? ainv1 : ainv0;
-                    const float lr_ = al * cs, li_ = al * sn;
-                    g = make_float2(g.x * lr_ - g.y * li_, g.x * li_ + g.y * lr_);
-                    ainv = fminf(ainv * __fdividef(1.0f, al), 5.5e34f);
-                    const uint32_t kx = x ? tk[ii].k.y : tk[ii].k.x, qx = x ? tk[ii].q.y : tk[ii].q.x;
-                    const float kr = __uint_as_float(kx << 16), ki = __uint_as_float(kx & 0xffff0000u);
-                    const float qr = __uint_as_float(qx << 16), qi = __uint_as_float(qx & 0xffff0000u);
-                    wr[x] = g.x * kr + g.y * ki; wi[x] = g.x * ki - g.y * kr;          // W = conj(gamma) k
-                    qr_[x] = g.x * qr + g.y * qi; qi_[x] = g.x * qi - g.y * qr;        // Qt = conj(gamma) q
-                    cr_[x] = (wr[x] * ainv) * ainv; ci_[x] = (wi[x] * ainv) * ainv;    // Kc = k / gamma = W / a^2
-                }
+                // gamma_t = gamma_{t-1} alpha_t e^{i theta_t}; 1/a_t alongside (capped at e^80)
+                const float2 al2 = make_float2(
+                    fmaxf(kFused ? alpha_from_raw(p, tk[ii].al.x) : __uint_as_float(tk[ii].al.x), 9.0e-14f),   // floor e^-30
+                    fmaxf(kFused ? alpha_from_raw(p, tk[ii].al.y) : __uint_as_float(tk[ii].al.y), 9.0e-14f));
+                float2 cs2, sn2;
+                __sincosf(kFused ? theta_from_raw(p, tk[ii].th.x) : __uint_as_float(tk[ii].th.x), &sn2.x, &cs2.x);
+                __sincosf(kFused ? theta_from_raw(p, tk[ii].th.y) : __uint_as_float(tk[ii].th.y), &sn2.y, &cs2.y);
+                const float2 lr2 = __fmul2_rn(al2, cs2), li2 = __fmul2_rn(al2, sn2);
+                const float2 gxn = __ffma2_rn(gy2, make_float2(-li2.x, -li2.y), __fmul2_rn(gx2, lr2));
+                gy2 = __ffma2_rn(gy2, lr2, __fmul2_rn(gx2, li2));
+                gx2 = gxn;
+                ainv2 = __fmul2_rn(ainv2, make_float2(__fdividef(1.0f, al2.x), __fdividef(1.0f, al2.y)));
+                ainv2 = make_float2(fminf(ainv2.x, 5.5e34f), fminf(ainv2.y, 5.5e34f));
+                const uint32_t k0 = tk[ii].k.x, k1 = tk[ii].k.y, q0 = tk[ii].q.x, q1 = tk[ii].q.y;
+                const float2 kr2 = make_float2(__uint_as_float(k0 << 16), __uint_as_float(k1 << 16));
+                const float2 ki2 = make_float2(__uint_as_float(k0 & 0xffff0000u), __uint_as_float(k1 & 0xffff0000u));
+                const float2 qr2 = make_float2(__uint_as_float(q0 << 16), __uint_as_float(q1 << 16));
+                const float2 qi2 = make_float2(__uint_as_float(q0 & 0xffff0000u), __uint_as_float(q1 & 0xffff0000u));
+                const float2 ngy2 = make_float2(-gy2.x, -gy2.y);
+                const float2 wr2 = __ffma2_rn(gy2, ki2, __fmul2_rn(gx2, kr2));     // W = conj(gamma) k
+                const float2 wi2 = __ffma2_rn(ngy2, kr2, __fmul2_rn(gx2, ki2));
+                const float2 tr2 = __ffma2_rn(gy2, qi2, __fmul2_rn(gx2, qr2));     // Qt = conj(gamma) q
+                const float2 ti2 = __ffma2_rn(ngy2, qr2, __fmul2_rn(gx2, qi2));
+                const float2 cr2 = __fmul2_rn(__fmul2_rn(wr2, ainv2), ainv2);      // Kc = k / gamma = W / a^2
+                const float2 ci2 = __fmul2_rn(__fmul2_rn(wi2, ainv2), ainv2);
                 load_token(tk[ii], i + kTB);
                 const int o1 = i * 128 + ((((jp >> 2) ^ i) & 7) << 4);      // row i of the octet's 8-row swizzle atom
-                sts32(wq_re + o1, pack_bf16(wr[0], wr[1]));
-                sts32(wq_re + 2 * kTile + o1, pack_bf16(wi[0], wi[1]));
-                sts32(wq_re + kTile + o1, pack_bf16(qr_[0], qr_[1]));
-                sts32(wq_re + 3 * kTile + o1, pack_bf16(qi_[0], qi_[1]));
-                sts32(kc_re + o1, pack_bf16(cr_[0], cr_[1]));
-                sts32(kc_re + kTile + o1, pack_bf16(ci_[0], ci_[1]));
+                sts32(wq_re + o1, pack_bf16(wr2.x, wr2.y));
+                sts32(wq_re + 2 * kTile + o1, pack_bf16(wi2.x, wi2.y));
+                sts32(wq_re + kTile + o1, pack_bf16(tr2.x, tr2.y));
+                sts32(wq_re + 3 * kTile + o1, pack_bf16(ti2.x, ti2.y));
+                sts32(kc_re + o1, pack_bf16(cr2.x, cr2.y));
+                sts32(kc_re + kTile + o1, pack_bf16(ci2.x, ci2.y));
             }
         }
         fence_async_smem();
@@ -995,11 +1003,12 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
                     // no mask: the substitution reads only entries below the diagonal of an 8x8 block and then
                     // overwrites the whole block; the merges read whole blocks strictly below the diagonal
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4)
-                        sts128(dst + 4 * i, __float_as_uint(bt * __uint_as_float(r[i])),
-                               __float_as_uint(bt * __uint_as_float(r[i + 1])),
-                               __float_as_uint(bt * __uint_as_float(r[i + 2])),
-                               __float_as_uint(bt * __uint_as_float(r[i + 3])));
+                    for (int i = 0; i < 32; i += 4) {
+                        const float2 bt2 = make_float2(bt, bt);
+                        const float2 lo = __fmul2_rn(bt2, make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])));
+                        const float2 hi = __fmul2_rn(bt2, make_float2(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])));
+                        sts128(dst + 4 * i, __float_as_uint(lo.x), __float_as_uint(lo.y), __float_as_uint(hi.x), __float_as_uint(hi.y));
+                    }
                 } else {                          // Aq, lower incl. diagonal, as a bf16 operand tile
                     const int t = row - 64;
                     const uint32_t tile = sbase + OFF_AQ + (s * 2 + im) * kTile;
@@ -1159,7 +1168,7 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
         SFDA_T(10);
         const bool fin = j == n_chunks;
         const ChunkInfo ci = fin ? prev_ci : ring_get(mi, j);
-        const float2 *close = mi.close[(j - 1) & 3];
+        const float *close_re = mi.close_re[(j - 1) & 3], *close_im = mi.close_im[(j - 1) & 3];
         const float *src = nullptr;
         if (fin || ci.first) {
             // A unit ends (chunk j - 1 was its last): its final state e^{i phi_C} a_C S goes to S_T (last time
@@ -1177,10 +1186,12 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
                         tc_wait_ld();
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
-                            const float2 cl = close[jb + i];
+                            const float clx = close_re[jb + i], cly = close_im[jb + i];
                             const float xr = __uint_as_float(sre[i]), xi = __uint_as_float(sim[i]);
-                            __stcg(dst + (size_t)(2 * (jb + i)) * DV, cl.x * xr - cl.y * xi);
-                            __stcg(dst + (size_t)(2 * (jb + i) + 1) * DV, cl.x * xi + cl.y * xr);
+                            // (the same roundings as the state pass, so that a state handed over through memory
+                            // continues with the very bits an uncut sequence carries on chip)
+                            __stcg(dst + (size_t)(2 * (jb + i)) * DV, __fmaf_rn(-cly, xi, __fmul_rn(clx, xr)));
+                            __stcg(dst + (size_t)(2 * (jb + i) + 1) * DV, __fmaf_rn(cly, xr, __fmul_rn(clx, xi)));
                         }
                     }
                 }
@@ -1232,12 +1243,22 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
                 tmem_ld<16>(tlane + TM_S32 + jb, sre);
                 tmem_ld<16>(tlane + TM_S32 + 64 + jb, sim);
                 tc_wait_ld();
+                // two rows per instruction (packed pairs): (re, im) <- (c_re re - c_im im, c_re im + c_im re)
+                const uint32_t cre = smem_u32(close_re + jb), cim = smem_u32(close_im + jb);
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float2 cl = close[jb + i];
-                    const float xr = __uint_as_float(sre[i]), xi = __uint_as_float(sim[i]);
-                    sre[i] = __float_as_uint(cl.x * xr - cl.y * xi);
-                    sim[i] = __float_as_uint(cl.x * xi + cl.y * xr);
+                for (int i = 0; i < 16; i += 4) {
+                    const uint4 c4 = lds128(cre + 4 * i), d4 = lds128(cim + 4 * i);
+#pragma unroll
+                    for (int x = 0; x < 4; x += 2) {
+                        const float2 cr2 = make_float2(__uint_as_float(x ? c4.z : c4.x), __uint_as_float(x ? c4.w : c4.y));
+                        const float2 ci2 = make_float2(__uint_as_float(x ? d4.z : d4.x), __uint_as_float(x ? d4.w : d4.y));
+                        const float2 xr2 = make_float2(__uint_as_float(sre[i + x]), __uint_as_float(sre[i + x + 1]));
+                        const float2 xi2 = make_float2(__uint_as_float(sim[i + x]), __uint_as_float(sim[i + x + 1]));
+                        const float2 nr2 = __ffma2_rn(make_float2(-ci2.x, -ci2.y), xi2, __fmul2_rn(cr2, xr2));
+                        const float2 ni2 = __ffma2_rn(ci2, xr2, __fmul2_rn(cr2, xi2));
+                        sre[i + x] = __float_as_uint(nr2.x); sre[i + x + 1] = __float_as_uint(nr2.y);
+                        sim[i + x] = __float_as_uint(ni2.x); sim[i + x + 1] = __float_as_uint(ni2.y);
+                    }
                 }
             }
 #pragma unroll
