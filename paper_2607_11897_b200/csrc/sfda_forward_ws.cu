@@ -98,8 +98,7 @@ struct Misc {
     uint32_t part_turns[2][8][M];
     float close_re[4][M], close_im[4][M];   // a_C e^{i phi_C} of a ring of four chunks, real and imaginary parts
     float beta[4][C];
-    float kscale[4][C];                     // fused front end: -1 / (|k_raw| + eps) per token, ring of four chunks
-    float ones[C];                          //                  +1: the scale of the passes that apply none
+    float kscale[4][C];                     // fused front end: 1 / (|k_raw| + eps) per token, ring of four chunks
     uint4 cursor_raw[3];                    // the prologue's cursor (a ChunkCursor), taken over by PREP
     ChunkInfo ring[kRing];                  // description of chunk j at ring[j % kRing], published by PREP two chunks ahead
     unsigned long long bars[kNumBars];
@@ -115,27 +114,7 @@ constexpr uint32_t TM_X16 = 128;    // bf16 A operand: S_0, then R, then E (64 p
 constexpr uint32_t TM_GRAM = 192;   // Gram half (Re, then Im): lanes 0..63 Kt rows, 64..127 Aq rows
 constexpr uint32_t TM_ACC = 256;    // [D1/E re | rho re | D1/E im | rho im], 64 columns each
 
-// Optional per-role cycle accounting of CTA 0 (development builds only, -DSFDA_WS_TIMING): each role's first
-// thread adds the cycles since its previous mark to slot i.
-#ifdef SFDA_WS_TIMING
-#define SFDA_TDECL(cond) long long tmark_ = clock64(); const bool ton_ = blockIdx.x == 0 && timing != nullptr && (cond)
-#define SFDA_T(i)                                   \
-    do {                                            \
-        if (ton_) {                                 \
-            const long long now_ = clock64();       \
-            timing[i] += now_ - tmark_;             \
-            tmark_ = now_;                          \
-        }                                           \
-    } while (0)
-#else
-#define SFDA_TDECL(cond)
-#define SFDA_T(i) \
-    do {          \
-    } while (0)
-#endif
-
 struct Params {
-    long long *timing;
     const __nv_bfloat16 *q, *k;
     const float *alpha, *theta, *beta, *S0;
     float *S_T;
@@ -332,14 +311,6 @@ __device__ __forceinline__ void role_sync(int id, int nthreads)
     asm volatile("barrier.cta.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
-#ifdef SFDA_WS_TIMING
-__device__ __forceinline__ unsigned long long now_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-#endif
 
 // Wait for completion number k of a barrier; gives up after the launch's wait limit (about a second: 2^31 ticks of
 // the SM clock, unless the caller asked for less) or as soon as any other wait of the CTA has given up, and raises
@@ -389,7 +360,7 @@ __device__ __forceinline__ bool wait_k_warp(Misc &mi, int bar, int k)
 // One complex product as four real ones (g = 0..3), each of four K = 16 instructions:
 //   Re += x_re b_re,  Re -+= x_im b_im,  Im += x_im b_re,  Im +-= x_re b_im
 // A (x) is the bf16 operand in tensor memory (or, for the Gram, tiles in shared memory); `a_im`, `b_im`, `d_im`
-// are the imaginary parts' addresses; `neg_g` is the g whose product is subtracted; `fresh`:
+// are the imaginary parts' addresses; kNegMask has bit g set for the products that are subtracted; `fresh`:
 // the accumulators start from zero.  `b_step`: descriptor advance of B per K = 16 (2 for a K-major tile,
 // 128 for an MN-major one).  The state update uses the same products with conj(E)-side roles swapped, which
 // `swap` selects: Re += x_re b_re, Re -= x_im b_im, Im += x_re b_im, Im += x_im b_re.
@@ -399,7 +370,7 @@ __device__ __forceinline__ bool wait_k_warp(Misc &mi, int bar, int k)
 // kMask: the K = 16 steps to issue (bit ks); the operands arrive in two halves, and the steps that only need the
 // first half go out while the second is still being written.  With kFresh the lowest step of the mask starts the
 // accumulators from zero (so the call with kFresh has to be the first for its accumulators).
-template <int kNegG, bool kFresh, bool kSwap, uint32_t kBStep, int kMask = 15>
+template <int kNegMask, bool kFresh, bool kSwap, uint32_t kBStep, int kMask = 15>
 __device__ __forceinline__ void issue_complex(uint32_t d_re, uint32_t d_im, uint32_t a_re, uint32_t a_im, uint32_t b_re,
                                               uint32_t b_im, uint32_t dhi, uint32_t id, int part)
 {
@@ -411,7 +382,7 @@ __device__ __forceinline__ void issue_complex(uint32_t d_re, uint32_t d_im, uint
             const uint32_t d = g < 2 ? d_re : d_im;
             const uint32_t a = (kSwap ? odd : mid) ? a_im : a_re;
             const uint32_t b = (kSwap ? mid : odd) ? b_im : b_re;
-            const uint32_t idg = id | (g == kNegG ? 1u << 14 : 0u);
+            const uint32_t idg = id | ((kNegMask >> g & 1) ? 1u << 14 : 0u);
             constexpr int kFirst = (kMask & 1) ? 0 : (kMask & 2) ? 1 : (kMask & 4) ? 2 : 3;
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
@@ -452,7 +423,6 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
                                          const Params &p, int n_chunks)
 {
     const CUtensorMap *tm_v = &maps.v, *tm_o = &maps.o, *tm_oim = &maps.oim;
-    [[maybe_unused]] long long *timing = p.timing;
     const uint64_t dbase = smem_desc(smem_u32(smem));                     // descriptor of byte offset 0
     const uint32_t dlo = (uint32_t)dbase, dhi = (uint32_t)(dbase >> 32);
     unsigned long long *bars = mi.bars;
@@ -463,54 +433,47 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
 
     if (role == 0 || role == 3) {
         const int part = role == 0 ? 0 : 1;      // this warp's accumulator half
-        SFDA_TDECL((threadIdx.x & 31) == 0 && role == 0);
 #pragma unroll 1
         for (int j = 0; j < n_chunks; ++j) {
             const int s = j & 1, u = j >> 1;
             const uint32_t w_re = dlo + ((OFF_WQ + s * 4 * kTile) >> 4), k_re = dlo + ((OFF_KC + s * 2 * kTile) >> 4);
-            // D1 = W^* S_0 as soon as S_0 is there; rho_1 = Qt^* S_0 (the Qt rows follow the W rows in the slot's
+            // -D1 = -W^* S_0 (all four real products with the opposite sign, so that R = V + (-D1) needs no multiplication
+            // on the way to the operand columns) as soon as S_0 is there; rho_1 = Qt^* S_0 (the Qt rows follow the W rows in the slot's
             // tiles) once rho of the previous chunk has been read out.  Both read S_0 from the operand columns.
             // (the state pass writes S_0 in two halves: key coordinates 0-15 and 32-47 = k-steps 0 and 2 first)
             if (!wait_k_warp<kDiag>(mi, B_S16_A, j)) return;
             if (!wait_k_warp<kDiag>(mi, B_PREP_FULL0 + s, u)) return;
             tc_fence_after();
-            SFDA_T(0);
-            issue_complex<3, true, false, 2, 5>(acc, acc + 128, x_re, x_re + 32, w_re, w_re + 2 * kIm, dhi, I64, part);
+            issue_complex<7, true, false, 2, 5>(acc, acc + 128, x_re, x_re + 32, w_re, w_re + 2 * kIm, dhi, I64, part);
             if (!wait_k_warp<kDiag>(mi, B_S16_B, j)) return;
             tc_fence_after();
-            issue_complex<3, false, false, 2, 10>(acc, acc + 128, x_re, x_re + 32, w_re, w_re + 2 * kIm, dhi, I64, part);
+            issue_complex<7, false, false, 2, 10>(acc, acc + 128, x_re, x_re + 32, w_re, w_re + 2 * kIm, dhi, I64, part);
             if (elect_one()) mma_commit(&bars[B_D1_DONE]);
             if (j > 0 && !wait_k_warp<kDiag>(mi, B_O_STAGED, j - 1)) return;
             tc_fence_after();
-            issue_complex<3, true, false, 2>(acc + 64, acc + 192, x_re, x_re + 32, w_re + kIm, w_re + 3 * kIm, dhi, I64, part);
+            issue_complex<8, true, false, 2>(acc + 64, acc + 192, x_re, x_re + 32, w_re + kIm, w_re + 3 * kIm, dhi, I64, part);
             if (elect_one()) {
                 mma_commit(&bars[B_O1_DONE]);
             }
-            SFDA_T(1);
             // E = M_beta R (R arrives in two halves of 32 tokens = two k-steps each)
             if (!wait_k_warp<kDiag>(mi, B_R16_A, j)) return;
-            SFDA_T(2);
             if (!wait_k_warp<kDiag>(mi, B_MB_FULL, j)) return;
             tc_fence_after();
-            SFDA_T(3);
-            issue_complex<1, true, false, 2, 3>(acc, acc + 128, x_re, x_re + 32, m_re, m_re + kIm, dhi, I64, part);
+            issue_complex<2, true, false, 2, 3>(acc, acc + 128, x_re, x_re + 32, m_re, m_re + kIm, dhi, I64, part);
             if (!wait_k_warp<kDiag>(mi, B_R16_B, j)) return;
             tc_fence_after();
-            issue_complex<1, false, false, 2, 12>(acc, acc + 128, x_re, x_re + 32, m_re, m_re + kIm, dhi, I64, part);
+            issue_complex<2, false, false, 2, 12>(acc, acc + 128, x_re, x_re + 32, m_re, m_re + kIm, dhi, I64, part);
             if (elect_one()) mma_commit(&bars[B_E_DONE]);
-            SFDA_T(4);
             // S += E^T Kc (Kc as MN-major B: rows = tokens)
             if (!wait_k_warp<kDiag>(mi, B_E16_A, j)) return;
             tc_fence_after();
-            SFDA_T(5);
-            issue_complex<1, false, true, 128, 3>(tmem + TM_S32, tmem + TM_S32 + 64, x_re, x_re + 32, k_re, k_re + kIm, dhi, I64M, part);
+            issue_complex<2, false, true, 128, 3>(tmem + TM_S32, tmem + TM_S32 + 64, x_re, x_re + 32, k_re, k_re + kIm, dhi, I64M, part);
             if (!wait_k_warp<kDiag>(mi, B_E16_B, j)) return;
             tc_fence_after();
-            issue_complex<1, false, true, 128, 12>(tmem + TM_S32, tmem + TM_S32 + 64, x_re, x_re + 32, k_re, k_re + kIm, dhi, I64M, part);
+            issue_complex<2, false, true, 128, 12>(tmem + TM_S32, tmem + TM_S32 + 64, x_re, x_re + 32, k_re, k_re + kIm, dhi, I64M, part);
             if (elect_one()) {
                 mma_commit(&bars[B_UPD_DONE]);
             }
-            SFDA_T(6);
         }
     } else if (role == 1) {
         // iteration j: store the outputs of chunk j - 1 (once staged), then issue rho += Aq E of chunk j
@@ -542,7 +505,7 @@ __device__ __forceinline__ void run_ctrl(int role, uint8_t *smem, Misc &mi, uint
             if (!wait_k_warp<kDiag>(mi, B_AQ_FULL0 + (j & 1), j >> 1)) return;
             tc_fence_after();
             const uint32_t a_re = dlo + ((OFF_AQ + (j & 1) * 2 * kTile) >> 4);
-            issue_complex<1, false, false, 2>(acc + 64, acc + 192, x_re, x_re + 32, a_re, a_re + kIm, dhi, I64, 2);
+            issue_complex<2, false, false, 2>(acc + 64, acc + 192, x_re, x_re + 32, a_re, a_re + kIm, dhi, I64, 2);
             if (elect_one()) mma_commit(&bars[B_UPD_DONE]);
         }
     } else {
@@ -639,7 +602,6 @@ template <bool kFused, bool kDiag>
 __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem, const Maps &maps, const Params &p,
                                          int n_chunks, int pt)
 {
-    [[maybe_unused]] long long *timing = p.timing;
     const int jp = pt & 31, tq = pt >> 5;   // channel pair (channels 2jp, 2jp+1), token octet (8 tokens)
     bool dead = false;
     // this role also reads the finished outputs out of tensor memory (its warps cover the four lane quadrants
@@ -684,7 +646,6 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
         tc_fence_before();
         warp_arrive(&mi.bars[B_O_STAGED]);
     };
-    SFDA_TDECL(pt == 0);
     ChunkCursor cur = ChunkCursor::load(mi.cursor_raw);   // at chunk 2: chunks 0 and 1 were published before the roles started
 #pragma unroll 1
     for (int j = 0; j < n_chunks + 2; ++j) {
@@ -727,7 +688,6 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
             // all four arrays have 256 bytes per (token, head): the same byte offset serves them all
             step = (size_t)p.H * 256;
             off = (row0 + (size_t)(tq * 8) * p.H) * 256 + 8 * jp;
-            SFDA_T(35);
 
             // pass 1: this thread's product of alpha (fp32 products of at most 64 factors: relative error far
             // below bf16's) and sum of the integer phase over its 8 tokens
@@ -739,12 +699,10 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
                 ldg64_if(al[i].x, al[i].y, reinterpret_cast<const char *>(p.alpha) + off + i * step, i < nt);
                 ldg64_if(th[i].x, th[i].y, reinterpret_cast<const char *>(p.theta) + off + i * step, i < nt);
             }
-            SFDA_T(36);
             // beta of token pt: fetched now, written after the pass below so that its latency is covered
             float beta_t = 0.f;
             if (pt < len) beta_t = __ldg(p.beta + row0 + (size_t)pt * p.H);
             if (kFused && pt < len) beta_t = rcp1p_ex2(beta_t * -1.4426950408889634f);
-            SFDA_T(37);
             {
                 float a0 = 1.f, a1 = 1.f;
                 uint32_t u0 = 0u, u1 = 0u;
@@ -773,7 +731,6 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
                 *reinterpret_cast<uint2 *>(&mi.part_turns[s][tq][2 * jp]) = make_uint2(u0, u1);
             }
             if (pt < C) mi.beta[ring][pt] = beta_t;
-            SFDA_T(30);
 #pragma unroll
             for (int ii = 0; ii < kTB; ++ii) load_token(tk[ii], ii);
             // The only barrier of the role.  The partial sums are kept two chunks deep: a warp that runs ahead
@@ -806,16 +763,13 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
                 ainv0 = fminf(__fdividef(1.0f, base0), 5.5e34f);          // 1/a, capped at e^80
                 ainv1 = fminf(__fdividef(1.0f, base1), 5.5e34f);
             }
-            SFDA_T(31);
 
             // (the slot's tiles, last read by the state update of chunk j-2, are free once that chunk's products are
             // complete, which the read-out of its outputs below waits for)
-            SFDA_T(32);
         }
         // the state update of chunk j-2 has just finished (it freed Kc above): read out that chunk's outputs,
         // so that rho is free when the next chunk's first product is issued
         if (j >= 2) drain_outputs(j - 2);
-        SFDA_T(34);
         if (!live) continue;
 
         // pass 2: rotated / decayed operands.  A rolled loop over groups of kTB tokens keeps the code small; each
@@ -868,7 +822,6 @@ __device__ __forceinline__ void run_prep(uint8_t *smem, Misc &mi, uint32_t tmem,
         }
         fence_async_smem();
         warp_arrive(&mi.bars[B_PREP_FULL0 + s]);
-        SFDA_T(33);
     }
 }
 
@@ -943,14 +896,12 @@ __device__ __forceinline__ void store_tile_s(const float (&cr)[4], const float (
 template <bool kFused, bool kDiag>
 __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int n_chunks, int st)
 {
-    [[maybe_unused]] long long *timing = p.timing;
     const int lane = st & 31, w = st >> 5;    // w = TMEM lane quadrant of this warp
     constexpr uint32_t kIm = 64 * LS * 4;     // Re -> Im in the scratch
     const uint32_t sbase = smem_u32(smem), lx = sbase + OFF_LX;
     const uint32_t tlane = tmem + ((uint32_t)(w * 32) << 16);
     const int row = w * 32 + lane;            // Gram row held by this thread: < 64 -> Kt row, else Aq row
     bool dead = false;
-    SFDA_TDECL(st == 0);
 #pragma unroll 1
     for (int j = 0; j < n_chunks; ++j) {
         if (role_sync_or(1, kSolveThreads, dead || mi.abort)) break;   // also: scratch of the last chunk is free
@@ -962,11 +913,9 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
         float bt = 0.f;                           // beta of this thread's Kt row (PREP wrote it before the Gram ran)
 #pragma unroll 1
         for (int im = 0; im < 2; ++im) {
-            SFDA_T(20 + 2 * im);
             if (!dead && !wait_k<kDiag>(mi, B_GRAM_FULL, 2 * j + im)) dead = true;
             tc_fence_after();
             if (im == 0 && row < 64) bt = mi.beta[ring][row];
-            SFDA_T(21 + 2 * im);
 #pragma unroll 1
             for (int it = 0; it < 2; ++it) {
                 // fused: the piece that holds this warp's diagonal entries of Re Kt comes first
@@ -993,7 +942,7 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
                     asm("sqrt.approx.ftz.f32 %0, %0;" : "+f"(n));
                     // (|k_raw| + eps below 1e-18 counts as 1e-18: s^2 stays finite, and a zero key stays a zero key)
                     asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(sc) : "f"(fmaxf(n + p.eps, 1.0e-18f)));
-                    mi.kscale[ring][row] = -sc;
+                    mi.kscale[ring][row] = sc;
                     mi.beta[ring][row] = bt * sc;
                     bt = bt * sc * sc;
                     warp_arrive(&mi.bars[B_NORM_FULL]);
@@ -1029,7 +978,6 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
         fence_async_smem();
         warp_arrive(&mi.bars[B_AQ_FULL0 + s]);
         role_sync(1, kSolveThreads);
-        SFDA_T(24);
 
         // ---- X = (I + L)^{-1} in place.  Diagonal 8x8 blocks: lane = column c of block blk solves
         // (I + L) x = e_c right-looking (after x_i is final every later row is updated at once).
@@ -1083,7 +1031,6 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
             sts64(tpos + kIm, 0u, 0u);
         }
         role_sync(1, kSolveThreads);
-        SFDA_T(25);
         {   // level 1: 16 -> 32.  Warp pair pr merges 32-block pr; warp's column tile nt of the 16 columns
             const int pr = w >> 1, nt = w & 1;
             const int r0 = 32 * pr + 16, c0 = 32 * pr;
@@ -1095,7 +1042,6 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
             store_tile_s(cr[0], ci[0], -1.f, lx, r0, c0 + 8 * nt, lane);
         }
         role_sync(1, kSolveThreads);
-        SFDA_T(26);
         {   // level 2: 32 -> 64.  T in the top-right quadrant; warp w owns column tile w of the 32 columns
             const int nt = w;
             float cr[2][4], ci[2][4];
@@ -1108,11 +1054,9 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
             store_tile_s(cr[1], ci[1], -1.f, lx, 48, 8 * nt, lane);
         }
         role_sync(1, kSolveThreads);
-        SFDA_T(27);
 
         // ---- M_beta = X D_beta as a bf16 operand tile, once E of the previous chunk has read the old one
         if (j >= 1 && !dead && !wait_k<kDiag>(mi, B_E_DONE, j - 1)) dead = true;
-        SFDA_T(28);
         {
             const int t = st >> 1, part = st & 1;   // row t, columns 32 part .. 32 part + 31
             const uint32_t src = lx + (uint32_t)((t * LS + 32 * part) * 4);
@@ -1140,7 +1084,6 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
         }
         fence_async_smem();
         warp_arrive(&mi.bars[B_MB_FULL]);
-        SFDA_T(29);
     }
 }
 
@@ -1148,7 +1091,6 @@ __device__ __forceinline__ void run_solve(uint8_t *smem, Misc &mi, uint32_t tmem
 template <bool kFused, bool kDiag>
 __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem, const Params &p, int n_chunks, int ct)
 {
-    [[maybe_unused]] long long *timing = p.timing;
     const int lane = ct & 31, warp = ct >> 5;
     const int quad = warp & 3, half = warp >> 2;
     const int c = quad * 32 + lane;            // value channel = TMEM lane
@@ -1156,7 +1098,6 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
     const uint32_t tlane = tmem + ((uint32_t)(quad * 32) << 16);
     const uint32_t sv = smem_u32(smem) + OFF_V + 2 * c;   // v[t][c], rows of 256 bytes
 
-    SFDA_TDECL(ct == 0);
     ChunkInfo prev_ci = ring_get(mi, 0);
 #pragma unroll 1
     for (int j = 0; j <= n_chunks; ++j) {
@@ -1165,7 +1106,6 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
             if (!wait_k_warp<kDiag>(mi, B_UPD_DONE, j - 1)) return;
             tc_fence_after();
         }
-        SFDA_T(10);
         const bool fin = j == n_chunks;
         const ChunkInfo ci = fin ? prev_ci : ring_get(mi, j);
         const float *close_re = mi.close_re[(j - 1) & 3], *close_im = mi.close_im[(j - 1) & 3];
@@ -1200,9 +1140,6 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
                     __syncwarp();
                     if (lane == 0 && !(kDiag && p.withhold)) atomicAdd(p.flags + prev_ci.bh, 1u);
                 }
-#ifdef SFDA_WS_TIMING
-                if (ct == 0 && p.timing) p.timing[512 + blockIdx.x] = (long long)now_ns();
-#endif
             }
             if (fin) break;
             if (ci.seq_first) {
@@ -1274,7 +1211,6 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
             warp_arrive(&mi.bars[B_S16_A + pc]);   // this half of the operand is complete
         }
         prev_ci = ci;
-        SFDA_T(11);
 
         // ---- R = V - D1 (ph 0), then E (ph 1), -> bf16 A operand: 64 fp32 accumulator columns of this warp's half
         // (Re for the first four warps, Im for the others), 16 at a time.  D1 and rho_1, which read S_0 from the
@@ -1288,12 +1224,12 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
                 if (!wait_k_warp<kDiag>(mi, B_E_DONE, j)) return;
             }
             tc_fence_after();
-            SFDA_T(13 + 2 * ph);
-            const bool sub_v = ph == 0 && half == 0;            // R_re = V - D1_re
-            const float sgn = ph == 0 ? -1.f : 1.f;             // R_im = -D1_im
-            // fused: D1 was formed with the raw key, R = V - s D1; the per-token factor replaces the sign
+            // The accumulators hold -D1 (ph 0) or E (ph 1): R_re = V + (-D1)_re, R_im = (-D1)_im, E as it is -- only the
+            // four warps of the real half add anything, and only in ph 0.
+            const bool sub_v = ph == 0 && half == 0;
+            // fused: D1 was formed with the raw key, R = V - s D1: the per-token factor s multiplies -D1
             if (kFused && ph == 0 && !wait_k_warp<kDiag>(mi, B_NORM_FULL, j)) return;
-            const uint32_t scp = smem_u32(ph == 0 ? &mi.kscale[(j & 3)][0] : &mi.ones[0]);
+            [[maybe_unused]] const uint32_t scp = smem_u32(&mi.kscale[(j & 3)][0]);
             // The second half of the accumulator is read into registers before the first half of the operand is
             // announced: the product which that announcement releases (E = M_beta R goes out in two halves of its K
             // dimension) starts these very accumulator columns from zero, all 64 of them, so a warp that fetched
@@ -1304,21 +1240,26 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
 #pragma unroll 1
             for (int pc = 0; pc < 2; ++pc) {       // 32 columns per tensor-memory round trip
                 uint32_t pk[16];
-                uint4 sc4 = make_uint4(0u, 0u, 0u, 0u);
+                if (kFused && ph == 0) {
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    float v0 = 0.f, v1 = 0.f;
-                    if (sub_v) {
-                        v0 = __uint_as_float((uint32_t)lds16(sv + (32 * pc + 2 * i) * 2 * DV) << 16);
-                        v1 = __uint_as_float((uint32_t)lds16(sv + (32 * pc + 2 * i + 1) * 2 * DV) << 16);
+                    for (int i = 0; i < 16; i += 2) {
+                        const uint4 sc4 = lds128(scp + (32 * pc + 2 * i) * 4);
+                        r[2 * i] = __float_as_uint(__uint_as_float(sc4.x) * __uint_as_float(r[2 * i]));
+                        r[2 * i + 1] = __float_as_uint(__uint_as_float(sc4.y) * __uint_as_float(r[2 * i + 1]));
+                        r[2 * i + 2] = __float_as_uint(__uint_as_float(sc4.z) * __uint_as_float(r[2 * i + 2]));
+                        r[2 * i + 3] = __float_as_uint(__uint_as_float(sc4.w) * __uint_as_float(r[2 * i + 3]));
                     }
-                    float s0 = sgn, s1 = sgn;
-                    if (kFused) {
-                        if ((i & 1) == 0) sc4 = lds128(scp + (32 * pc + 2 * i) * 4);
-                        s0 = __uint_as_float((i & 1) ? sc4.z : sc4.x);
-                        s1 = __uint_as_float((i & 1) ? sc4.w : sc4.y);
+                }
+                if (sub_v) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float v0 = __uint_as_float((uint32_t)lds16(sv + (32 * pc + 2 * i) * 2 * DV) << 16);
+                        const float v1 = __uint_as_float((uint32_t)lds16(sv + (32 * pc + 2 * i + 1) * 2 * DV) << 16);
+                        pk[i] = pack_bf16(__uint_as_float(r[2 * i]) + v0, __uint_as_float(r[2 * i + 1]) + v1);
                     }
-                    pk[i] = pack_bf16(fmaf(s0, __uint_as_float(r[2 * i]), v0), fmaf(s1, __uint_as_float(r[2 * i + 1]), v1));
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
                 }
                 if (pc == 0) {
                     tmem_ld<32>(tlane + TM_ACC + 128 * half + 32, r);
@@ -1331,7 +1272,6 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
                 tc_fence_before();
                 warp_arrive(&mi.bars[(ph == 0 ? B_R16_A : B_E16_A) + pc]);   // this half of the operand is complete
             }
-            SFDA_T(14 + 2 * ph);
         }
     }
 }
@@ -1348,9 +1288,6 @@ sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
     const int tid = threadIdx.x, warp = tid >> 5;
     const int n_chunks = ChunkCursor::stream_chunks(p);   // length of this CTA's stream of chunks
 
-#ifdef SFDA_WS_TIMING
-    if (tid == 0 && p.timing) { p.timing[64 + 2 * blockIdx.x] = (long long)now_ns(); if (blockIdx.x == 0) p.timing[400] = clock64(); unsigned sm; asm volatile("mov.u32 %0, %smid;" : "=r"(sm)); p.timing[700 + blockIdx.x] = sm; }
-#endif
     if (tid == 0) {
         auto init = [&](int bar, uint32_t count) { mbar_init(&mi.bars[bar], count); };
         init(B_PREP_FULL0, kPrepWarps); init(B_PREP_FULL1, kPrepWarps);
@@ -1366,7 +1303,6 @@ sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
         if (kDiag) mi.wait_limit = p.wait_limit;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (kFused && tid < C) mi.ones[tid] = 1.0f;
     if (tid == kChainThreads + kSolveThreads) {
         // PREP's first thread walks the stream of chunks for everybody: chunks 0 and 1 are described (and their inputs
         // requested into L2) before the roles start; it goes on from there inside PREP, two chunks ahead
@@ -1405,9 +1341,6 @@ sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
 
     tc_fence_before();
     __syncthreads();
-#ifdef SFDA_WS_TIMING
-    if (tid == 0 && p.timing) { p.timing[64 + 2 * blockIdx.x + 1] = (long long)now_ns(); if (blockIdx.x == 0) p.timing[401] = clock64(); }
-#endif
     if (mi.abort) {
         // a wait ran out: before the shared memory is given back, leave the copy engine time to land whatever this
         // CTA still has in flight (its loads complete in a microsecond or two), then report
@@ -1419,11 +1352,6 @@ sfda_forward_ws_kernel(const __grid_constant__ Maps maps, const Params p)
 }
 
 // ---- host side ----------------------------------------------------------------------------------------
-long long *g_ws_timing = nullptr;   // set by development probes built with -DSFDA_WS_TIMING
-int g_ws_last_slices = 0;           // time slices chosen by the last launch (read by development probes)
-#ifdef SFDA_WS_TIMING
-int g_ws_grid_cap = 0, g_ws_force_q = 0;   // development probes only
-#endif
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -1592,10 +1520,6 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
         Q = a.debug_slices;
         bal = 0;
     }
-#ifdef SFDA_WS_TIMING
-    if (g_ws_force_q) { Q = g_ws_force_q; bal = 0; }
-    if (g_ws_grid_cap && g_ws_grid_cap < n_sm) n_sm = g_ws_grid_cap;
-#endif
     const bool pieces = Q > 1 || bal;   // sequences are cut: counters and boundary states in use, CTAs wait on one another
     const size_t header = kWsMinScratchBytes + (pieces ? (((size_t)BH * 4 + 255) & ~(size_t)255) : 0);
     // The status word is only ever set by the kernel, never cleared: a caller that runs several launches on one
@@ -1606,7 +1530,6 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
         e = cudaMemsetAsync(static_cast<char *>(scratch) + kWsMinScratchBytes, 0, header - kWsMinScratchBytes, stream);
     if (e != cudaSuccess) return e;
     Params p;
-    p.timing = g_ws_timing;
     p.q = static_cast<const __nv_bfloat16 *>(a.q);
     p.k = static_cast<const __nv_bfloat16 *>(a.k);
     p.alpha = a.alpha;
@@ -1629,7 +1552,6 @@ cudaError_t launch_forward_ws(const ForwardArgs &a, void *scratch, size_t scratc
     p.n_units = BH * Q;
     p.magic_BH = BH > 1 ? (uint32_t)(0x100000000ull / (unsigned)BH) + 1u : 0u;
     p.magic_H = a.H > 1 ? (uint32_t)(0x100000000ull / (unsigned)a.H) + 1u : 0u;
-    g_ws_last_slices = Q;
     const unsigned grid = (unsigned)(p.n_units < n_sm ? p.n_units : n_sm);
     p.bal = bal;
     p.NC = NC;
