@@ -14,10 +14,12 @@
 //   C  Gram:     pairs (t, i) of different 8-token blocks on the tensor cores (mma.sync, 3 x TF32), level by level
 //                of a binary split of the chunk, the decay split at the last token r of the lower half:
 //                a_t/a_i = (a_t/a_r)(a_r/a_i), both factors <= 1, so nothing overflows whatever alpha is; pairs
-//                inside a block take the ratio directly, eight lanes per pair.
+//                inside a block take the ratio directly: one warp per block, the block's tokens in registers,
+//                packed two-lane arithmetic, sums over the lanes through a small scratch.
 //   D  inverse:  8 x 8 diagonal blocks by substitution, then X = [[X11, 0], [-X22 N21 X11, X22]] doubling the
-//                block size until it is C.
-// Only ratios <= 1 are ever formed, so any alpha in [0, 1] is safe.
+//                block size until it is C, both products of a level as 16 x 8 tiles on the tensor cores (3 x TF32).
+// Only ratios <= 1 are ever formed, so any alpha in [0, 1] is safe.  Offsets inside a chunk are 32-bit: with 64-bit
+// offsets the unrolled loads and stores of the scan spent more instructions on addresses than on data.
 #include "sfda_common.cuh"
 #include "sfda_internal.h"
 
@@ -58,12 +60,12 @@ __device__ __forceinline__ void turns_cos_sin_fast(uint32_t turns, float *c, flo
     __sincosf(f * 6.283185307f, s, c);
 }
 
-// x = head + tail, both representable in TF32 (10 mantissa bits), to within 2^-22 |x|
+// x = head + tail to within 2^-20 |x|: the head is x cut to TF32's ten mantissa bits, the tail the exact rest, of which
+// the tensor core in turn reads the leading bits (it ignores the low 13 bits of a TF32 operand).  Two instructions.
 __device__ __forceinline__ void split_tf32(float x, uint32_t &head, uint32_t &tail)
 {
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(head) : "f"(x));
-    const float rest = x - __uint_as_float(head);
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(tail) : "f"(rest));
+    head = __float_as_uint(x) & 0xffffe000u;
+    tail = __float_as_uint(x - __uint_as_float(head));
 }
 __device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], const uint32_t (&b)[2])
 {
@@ -85,13 +87,14 @@ struct FacSmem {
     static constexpr int M = DK / 2;
     static constexpr int KS = M + 1;        // row stride of kp in float2 (odd: rows and columns both conflict-free)
     static constexpr int LS = M + 1;        // row stride of lg2 in floats
-    static constexpr int NS = C + 1;        // row stride of N / X in float2
+    static constexpr int NS = C + 4;        // row stride of N / X in float2 (4 mod 16: the tensor-core tiles' 64-bit loads
+                                            // of a half-warp, rows g and columns c or rows c and columns g, hit 16 different slots)
     static constexpr int G = kFacThreads / M;   // token groups of the scan
     static constexpr int TG = C / G;            // tokens per group
     static constexpr int kKeyRows = C * (KS > NS ? KS : NS);   // float2: the larger of k' and N
     static constexpr int kGrpFloats = 2 * G * M > 2 * (C / 8) * 28 ? 2 * G * M : 2 * (C / 8) * 28;
     static constexpr size_t bytes = (size_t)kKeyRows * 8 + (size_t)C * LS * 4 + (size_t)kGrpFloats * 4 +
-                                    (size_t)M * 12 + (size_t)C * 4;
+                                    (size_t)M * 12 + (size_t)C * 4 + (size_t)(kFacThreads / 32) * 14 * 33 * 4;
     float2 *kp;        // [C][KS] rotated keys k' until the Gram sums are in registers ...
     float2 *nx;        // ... then [C][NS] N, inverted in place (same memory)
     float *lg2;        // [C][LS] log2 of a_t; after the Gram: scratch of the inverse's products
@@ -99,6 +102,7 @@ struct FacSmem {
     uint32_t *grp_tu;  // [G][M]
     float *gcr, *gci, *lg2C;   // [M] e^{i phi_C}, log2 a_C
     float *beta;       // [C]
+    float *red;        // [warp][14][33] terms of seven pairs inside a block, lane by lane
     __device__ explicit FacSmem(unsigned char *base)
     {
         kp = reinterpret_cast<float2 *>(base);
@@ -110,40 +114,90 @@ struct FacSmem {
         gci = gcr + M;
         lg2C = gci + M;
         beta = lg2C + M;
+        red = beta + C;
     }
 };
 static_assert(FacSmem<128, 64>::bytes <= 74 * 1024, "three CTAs per SM need at most 75 KB each");
 
-// One level of the block inverse: every pair of finished diagonal blocks of size HS becomes one of size 2 HS.
+// One 8-wide step of a complex 16 x 8 tile product on the tensor cores with fp32-like accuracy (3 x TF32 per real
+// product).  `a` points at element (row g, column c) of the A tile's columns of this step, `b` at element
+// (row c, column g) of the B tile's rows (g = lane / 4, c = lane % 4); strides in float2.  The four real products
+// keep their own accumulators: Re = acc[0] - acc[1], Im = acc[2] + acc[3].
+__device__ __forceinline__ void cmma3_step(float (&acc)[4][4], const float2 *a, int as, const float2 *b, int bs)
+{
+    uint32_t arh[4], arl[4], aih[4], ail[4], brh[2], brl[2], bih[2], bil[2];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {          // a0 (g, c), a1 (g + 8, c), a2 (g, c + 4), a3 (g + 8, c + 4)
+        const float2 v = a[(e & 1) * 8 * as + (e >> 1) * 4];
+        split_tf32(v.x, arh[e], arl[e]);
+        split_tf32(v.y, aih[e], ail[e]);
+    }
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {          // b0 (k = c, n = g), b1 (k = c + 4, n = g)
+        const float2 v = b[e * 4 * bs];
+        split_tf32(v.x, brh[e], brl[e]);
+        split_tf32(v.y, bih[e], bil[e]);
+    }
+    mma3_tf32(acc[0], arh, arl, brh, brl);
+    mma3_tf32(acc[1], aih, ail, bih, bil);
+    mma3_tf32(acc[2], arh, arl, bih, bil);
+    mma3_tf32(acc[3], aih, ail, brh, brl);
+}
+
+// One level of the block inverse: every pair of finished diagonal blocks of size HS (X11 at o, X22 at o + HS, N21
+// below X11) becomes one of size 2 HS: X21 = -X22 (N21 X11), both products as 16 x 8 tiles on the tensor cores, one
+// tile per warp and round.  Whole 8 x 8 blocks are read: the blocks on the diagonal hold zeros above it, the block
+// right of the upper diagonal block of every 16 rows was zeroed, and the ranges of the sums leave out every other
+// block above the diagonal.  With HS = 8 the tile lies on the whole 16-row block and its lower eight rows count.
 template <typename S, int C, int HS>
 __device__ __forceinline__ void merge_level(const S &sm, int tid)
 {
     if constexpr (HS < C) {
-        constexpr int per = HS * HS, total = (C / (2 * HS)) * per;
-        float2 *P = reinterpret_cast<float2 *>(sm.lg2);    // scratch [merges of the level][HS x HS]: the decays are done
-        for (int idx = tid; idx < total; idx += kFacThreads) {     // P[r][c] = sum_{k >= c} N21[r][k] X11[k][c]
-            // lanes run over r: one trip count (HS - c) per warp, N21 rows conflict-free, X11 broadcast
-            const int mg = idx / per, rc = idx % per, c = rc / HS, r = rc % HS, o = mg * 2 * HS;
-            float pr = 0.f, pi = 0.f;
-            for (int kk = c; kk < HS; ++kk) {
-                const float2 n = sm.nx[(o + HS + r) * S::NS + o + kk];
-                const float2 x = sm.nx[(o + kk) * S::NS + o + c];
-                pr += n.x * x.x - n.y * x.y;
-                pi += n.x * x.y + n.y * x.x;
-            }
-            P[mg * per + r * HS + c] = make_float2(pr, pi);
+        constexpr int PS = 36;                              // row stride of the scratch (float2): conflict-free 64-bit loads
+        constexpr int MT = HS >= 16 ? HS / 16 : 1, NT = HS / 8, kTiles = (C / (2 * HS)) * MT * NT;
+        static_assert((C / 2) * PS * 8 <= (C * S::LS + S::kGrpFloats) * 4, "the products' scratch must fit where lg2 and the group sums were");
+        float2 *P = reinterpret_cast<float2 *>(sm.lg2);    // [merge][HS][PS]: N21 X11 (the decays and the group sums after them are done)
+        const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, c = lane & 3;
+        for (int tile = warp; tile < kTiles; tile += kFacThreads / 32) {
+            const int mg = tile / (MT * NT), mt = (tile % (MT * NT)) / NT, nt = tile % NT, o = mg * 2 * HS;
+            const int arow = HS >= 16 ? o + HS + 16 * mt : o;
+            float acc[4][4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x)
+#pragma unroll
+                for (int y = 0; y < 4; ++y) acc[x][y] = 0.f;
+            const float2 *a = sm.nx + (arow + g) * S::NS + o + c;
+            const float2 *b = sm.nx + (o + c) * S::NS + o + 8 * nt + g;
+#pragma unroll 1
+            for (int ks = nt; ks < NT; ++ks)                // X11[k][col] = 0 for k-blocks above the column's
+                cmma3_step(acc, a + 8 * ks, S::NS, b + 8 * ks * S::NS, S::NS);
+            float2 *dst = P + (mg * HS + 16 * mt + g) * PS + 8 * nt + 2 * c;
+            if (HS >= 16)
+                *reinterpret_cast<float4 *>(dst) = make_float4(acc[0][0] - acc[1][0], acc[2][0] + acc[3][0],
+                                                               acc[0][1] - acc[1][1], acc[2][1] + acc[3][1]);
+            *reinterpret_cast<float4 *>(dst + (HS >= 16 ? 8 * PS : 0)) =
+                make_float4(acc[0][2] - acc[1][2], acc[2][2] + acc[3][2], acc[0][3] - acc[1][3], acc[2][3] + acc[3][3]);
         }
         __syncthreads();
-        for (int idx = tid; idx < total; idx += kFacThreads) {     // X21[r][c] = -sum_{k <= r} X22[r][k] P[k][c]
-            const int mg = idx / per, rc = idx % per, r = rc / HS, c = rc % HS, o = mg * 2 * HS;
-            float sr = 0.f, si = 0.f;
-            for (int kk = 0; kk <= r; ++kk) {
-                const float2 x = sm.nx[(o + HS + r) * S::NS + o + HS + kk];
-                const float2 pp = P[mg * per + kk * HS + c];
-                sr += x.x * pp.x - x.y * pp.y;
-                si += x.x * pp.y + x.y * pp.x;
-            }
-            sm.nx[(o + HS + r) * S::NS + o + c] = make_float2(-sr, -si);
+        for (int tile = warp; tile < kTiles; tile += kFacThreads / 32) {
+            const int mg = tile / (MT * NT), mt = (tile % (MT * NT)) / NT, nt = tile % NT, o = mg * 2 * HS;
+            const int arow = HS >= 16 ? o + HS + 16 * mt : o;
+            float acc[4][4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x)
+#pragma unroll
+                for (int y = 0; y < 4; ++y) acc[x][y] = 0.f;
+            const float2 *a = sm.nx + (arow + g) * S::NS + o + HS + c;
+            const float2 *b = P + (mg * HS + c) * PS + 8 * nt + g;
+            const int nks = HS >= 16 ? 2 * mt + 2 : 1;      // X22[row][k] = 0 for k-blocks beyond the tile's rows
+#pragma unroll 1
+            for (int ks = 0; ks < nks; ++ks) cmma3_step(acc, a + 8 * ks, S::NS, b + 8 * ks * PS, PS);
+            float2 *dst = sm.nx + (o + HS + 16 * mt + g) * S::NS + o + 8 * nt + 2 * c;
+            if (HS >= 16)
+                *reinterpret_cast<float4 *>(dst) = make_float4(acc[1][0] - acc[0][0], -acc[2][0] - acc[3][0],
+                                                               acc[1][1] - acc[0][1], -acc[2][1] - acc[3][1]);
+            *reinterpret_cast<float4 *>(dst + (HS >= 16 ? 8 * S::NS : 0)) =
+                make_float4(acc[1][2] - acc[0][2], -acc[2][2] - acc[3][2], acc[1][3] - acc[0][3], -acc[2][3] - acc[3][3]);
         }
         __syncthreads();
     }
@@ -159,7 +213,6 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
     using S = FacSmem<DK, C>;
     constexpr int M = S::M, G = S::G, TG = S::TG;
     static_assert(C % 8 == 0 && C % G == 0 && TG >= 1, "chunk must split into the scan's groups and 8-token blocks");
-    static_assert((size_t)C * (C / 4) * 8 <= (size_t)C * S::LS * 4, "the inverse's scratch must fit where lg2 was");
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const S sm(smem_raw);
 
@@ -180,7 +233,10 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
         const size_t row0 = ((size_t)b * T_ + t0 + g * TG) * H + h;      // first token of the group
         const float *ap = alpha + row0 * M + j, *tp = theta + row0 * M + j;
         const T *kq = k + row0 * DK + 2 * j;
-        const size_t cs = (size_t)H * M;                                  // coordinates from one token to the next
+        // coordinates from one token to the next; offsets inside a chunk stay below 2^32, and 32-bit offsets keep
+        // the address arithmetic of the unrolled loads to one instruction each
+        const unsigned cs = (unsigned)H * M;
+        uint32_t *tpo = turns_out ? turns_out + row0 * M + j : nullptr;
 #pragma unroll
         for (int x = 0; x < TG; ++x) {
             const int t = g * TG + x;
@@ -189,7 +245,7 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
             if (t < len) {
                 al = ap[x * cs];
                 th = tp[x * cs];
-                kv[x] = ld_pair(kq, 2 * x * cs);
+                kv[x] = ld_pair(kq, (size_t)(2u * x * cs));
             }
             lgv[x] = al;
             tu[x] = __float_as_uint(th);
@@ -218,7 +274,7 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
             const int t = g * TG + x;
             const float l = base + lgv[x];
             const uint32_t tt = tb + tu[x];
-            if (turns_out && t < len) turns_out[row0 * M + j + x * cs] = tt;
+            if (tpo && t < len) tpo[x * cs] = tt;
             float cs, sn;
             turns_cos_sin_fast(tt, &cs, &sn);
             sm.lg2[t * S::LS + j] = l;
@@ -276,6 +332,57 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
         // 1) and dropped.  A warp has at most two jobs, which share their row operand when tile and r agree.
         // The sums stay in registers: N will overwrite the keys once everybody has read them.
         const int warp = tid >> 5, lane = tid & 31, fg = lane >> 2, ft = lane & 3;
+        // Pairs inside a block take the decay ratio directly: a_t / a_i <= 1 for i < t.  One warp per block; a lane keeps
+        // the eight tokens' rotated keys and log-decays of its coordinates (lane and lane + 32) in registers and forms
+        // the 28 pairs' terms with packed two-lane arithmetic; the sums over the lanes go through a small scratch,
+        // seven pairs at a time.  The results wait in the scan's group totals, which are no longer needed.
+        float2 *dg = reinterpret_cast<float2 *>(sm.grp_lg);
+        for (int blk = warp; blk < NB; blk += kFacThreads / 32) {
+            float2 kx[8], ky[8], lg[8];                    // .x: coordinate `lane`, .y: coordinate `lane + 32`
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+                const float2 k0 = sm.kp[(8 * blk + r) * S::KS + lane];
+                float2 k1 = make_float2(0.f, 0.f);
+                float l1 = 0.f;
+                if (M > 32) {
+                    k1 = sm.kp[(8 * blk + r) * S::KS + (M > 32 ? lane + 32 : lane)];
+                    l1 = sm.lg2[(8 * blk + r) * S::LS + (M > 32 ? lane + 32 : lane)];
+                }
+                kx[r] = make_float2(k0.x, k1.x);
+                ky[r] = make_float2(k0.y, k1.y);
+                lg[r] = make_float2(sm.lg2[(8 * blk + r) * S::LS + lane], l1);
+            }
+            float *red = sm.red + warp * (14 * 33);
+#pragma unroll
+            for (int t = 1; t < 8; ++t) {
+                const float2 nky = make_float2(-ky[t].x, -ky[t].y);
+#pragma unroll
+                for (int i = 0; i < t; ++i) {
+                    const int pidx = t * (t - 1) / 2 + i, v = 2 * (pidx % 7);   // compile-time
+                    const float2 d = __fadd2_rn(lg[t], make_float2(-lg[i].x, -lg[i].y));
+                    const float2 w = make_float2(ex2f(d.x), ex2f(d.y));
+                    const float2 pr = __ffma2_rn(ky[t], ky[i], __fmul2_rn(kx[t], kx[i]));      // Re conj(k'_t) k'_i
+                    const float2 pi = __ffma2_rn(nky, kx[i], __fmul2_rn(kx[t], ky[i]));        // Im conj(k'_t) k'_i
+                    const float2 sr = __fmul2_rn(w, pr), si = __fmul2_rn(w, pi);
+                    red[v * 33 + lane] = sr.x + sr.y;
+                    red[(v + 1) * 33 + lane] = si.x + si.y;
+                    if (pidx % 7 == 6) {                   // seven pairs are in: add up over the lanes
+                        __syncwarp();
+                        // lanes 2 v and 2 v + 1 add the two halves of value v's 32 terms
+                        float acc = 0.f;
+                        const float *src = red + (lane >> 1) * 33 + 16 * (lane & 1);
+                        if (lane < 28) {
+#pragma unroll
+                            for (int x = 0; x < 16; ++x) acc += src[x];
+                        }
+                        acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+                        const float im = __shfl_xor_sync(0xffffffffu, acc, 2);
+                        if ((lane & 3) == 0 && lane < 28) dg[(pidx - 6 + (lane >> 2)) * NB + blk] = make_float2(acc, im);
+                        __syncwarp();
+                    }
+                }
+            }
+        }
         int jm[2] = {-1, -1}, jc[2] = {0, 0}, jr[2] = {0, 0};   // row tile, first column, split token of the jobs
         if (C == 64) {
             if (warp < 4) { jm[0] = jm[1] = 2 + (warp >> 1); jc[0] = 16 * (warp & 1); jc[1] = jc[0] + 8; jr[0] = jr[1] = 31; }
@@ -333,36 +440,10 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
                 }
             }
         }
-        // Pairs inside a block take the decay ratio directly.  Eight lanes share a pair (coordinates j = lane, lane +
-        // 8, ...) and add up by shuffles; the sums wait in the scan's group totals, which are no longer needed.
-        float2 *dg = reinterpret_cast<float2 *>(sm.grp_lg);
-        for (int base = 0; base < kPairs * 8; base += kFacThreads) {
-            const int li = base + tid, pr_ = li >> 3, sub = li & 7;
-            const bool on = li < kPairs * 8;
-            const unsigned lanes = __ballot_sync(0xffffffffu, on);     // whole groups of eight lanes
-            if (on) {
-                const int blk = pr_ % NB, pidx = pr_ / NB; // neighbouring groups of lanes work in different blocks
-                int t = 1;
-                while (t * (t + 1) / 2 <= pidx) ++t;       // pidx = t (t - 1) / 2 + i
-                const int i = pidx - t * (t - 1) / 2;
-                const int tt = 8 * blk + t, ii = 8 * blk + i;
-                float sr = 0.f, si = 0.f;
-#pragma unroll 4
-                for (int j = sub; j < M; j += 8) {
-                    const float w = ex2f(sm.lg2[tt * S::LS + j] - sm.lg2[ii * S::LS + j]);
-                    const float2 a = sm.kp[tt * S::KS + j], bq = sm.kp[ii * S::KS + j];
-                    sr = fmaf(w, a.x * bq.x + a.y * bq.y, sr);
-                    si = fmaf(w, a.x * bq.y - a.y * bq.x, si);
-                }
-#pragma unroll
-                for (int dlt = 1; dlt < 8; dlt *= 2) {
-                    sr += __shfl_xor_sync(lanes, sr, dlt);
-                    si += __shfl_xor_sync(lanes, si, dlt);
-                }
-                if (sub == 0) dg[pr_] = make_float2(sr, si);
-            }
-        }
         __syncthreads();           // every read of the keys is done: N goes where they were
+        // the 8 x 8 block right of the upper diagonal block of every 16 rows: read as zeros by the inverse's tiles
+        for (int idx = tid; idx < (C / 16) * 64; idx += kFacThreads)
+            sm.nx[(16 * (idx >> 6) + ((idx >> 3) & 7)) * S::NS + 16 * (idx >> 6) + 8 + (idx & 7)] = make_float2(0.f, 0.f);
 #pragma unroll
         for (int n = 0; n < 2; ++n) {
             if (jm[n] < 0) continue;
