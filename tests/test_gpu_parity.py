@@ -499,6 +499,66 @@ def test_chunk_factors_match_constructive_recursion(d_k, chunk, T, dtype):
     assert worst < 1e-4, worst
 
 
+@pytest.mark.parametrize("case", ["zeros_and_tiny", "all_one", "strong_everywhere", "one_dead_coordinate"])
+@pytest.mark.parametrize("d_k,chunk", [(128, 64), (64, 32)])
+def test_chunk_factors_decay_and_write_extremes(case, d_k, chunk):
+    """The factor export forms only decay ratios a_t / a_i <= 1 (split at the level boundaries on the tensor cores,
+    direct inside the 8-token blocks), so every alpha in [0, 1] is admissible (Section 3 admits alpha = 0): chunks
+    with exact zeros, with factors of 1e-6, with alpha = 1 throughout and with strong decay everywhere, beta in
+    {0, 1} mixed in and phases far outside (-pi, pi], against the constructive recursion at the usual bar."""
+    T, B, H = 2 * chunk + 5, 1, 2
+    cfg = workloads.CONFIGS[0].scaled(name="facx", B=B, T=T, H=H, d_k=d_k, chunk=chunk, dtype="bf16", seed=77)
+    inp = workloads.forward_inputs(cfg)
+    rng = np.random.default_rng([cfg.seed, len(case)])
+    m, C = cfg.m, chunk
+    alpha = inp["alpha"].copy()
+    if case == "zeros_and_tiny":
+        pick = rng.random(alpha.shape)
+        alpha[pick < 0.05] = 0.0
+        alpha[(pick >= 0.05) & (pick < 0.15)] = 1e-6
+        alpha[(pick >= 0.15) & (pick < 0.30)] = 1.0
+    elif case == "all_one":
+        alpha[:] = 1.0
+    elif case == "strong_everywhere":
+        alpha[:] = (1e-3 * (1.0 + rng.random(alpha.shape))).astype(np.float32)
+    else:
+        alpha[..., 3] = 0.0                               # one coordinate forgets everything at every token
+    beta = inp["beta"].copy()
+    pick = rng.random(beta.shape)
+    beta[pick < 0.2] = 0.0
+    beta[pick > 0.8] = 1.0
+    theta = (inp["theta"] * 16.0).astype(np.float32)      # up to about +-50 rad
+    NC = -(-T // C)
+    G = torch.full((B, H, NC, m, 2), float("nan"), device=DEV)
+    Y = torch.full((B, H, NC, m, C, 2), float("nan"), device=DEV)
+    M = torch.full((B, H, NC, C, C, 2), float("nan"), device=DEV)
+    W = torch.full((B, H, NC, m, C, 2), float("nan"), device=DEV)
+    turns = torch.zeros(B, T, H, m, device=DEV, dtype=torch.int32)
+    sfda.sfda_chunk_factors(to_dev(inp["k"], cfg, "k"), to_dev(alpha, cfg, "alpha"), to_dev(theta, cfg, "theta"),
+                            to_dev(beta, cfg, "beta"), G, Y, M, W, turns, chunk)
+    torch.cuda.synchronize()
+    cx = lambda t: t.cpu().numpy().astype(np.float64)[..., 0] + 1j * t.cpu().numpy().astype(np.float64)[..., 1]
+    G, Y, M, W = cx(G), cx(Y), cx(M), cx(W)
+    assert np.isfinite(G).all() and np.isfinite(Y).all() and np.isfinite(M).all() and np.isfinite(W).all()
+    want_turns = np.moveaxis(bookkeeping.cumulative_phase_turns(np.moveaxis(theta, 1, 2), chunk), 2, 1)
+    assert np.array_equal(turns.cpu().numpy().view(np.uint32), want_turns)
+    worst = 0.0
+    for h in range(H):
+        kc = chunk_wy.pair(inp["k"][0, :, h])
+        for c in range(NC):
+            sl = slice(c * C, min((c + 1) * C, T))
+            L = sl.stop - sl.start
+            g, y, w, mm = chunk_wy.chunk_factors(kc[sl], alpha[0, sl, h].astype(np.float64),
+                                                 theta[0, sl, h].astype(np.float64), beta[0, sl, h].astype(np.float64))
+            # absolute bars: the keys have unit norm, so every factor is O(1) at most and a column that decays to
+            # nothing has nothing to be relative to
+            worst = max(worst, np.abs(G[0, h, c] - g).max(), np.abs(Y[0, h, c][:, :L] - y).max(),
+                        np.abs(W[0, h, c][:, :L] - w).max(), np.abs(M[0, h, c][:L, :L] - mm).max())
+            P_gpu = np.diag(G[0, h, c]) - Y[0, h, c] @ M[0, h, c] @ W[0, h, c].conj().T
+            assert np.abs(P_gpu - (np.diag(g) - y @ mm @ w.conj().T)).max() < 2e-5
+    assert worst < 1e-4, worst
+
+
 # ------------------------------------------------------------------------------------------------
 # decode
 # ------------------------------------------------------------------------------------------------
