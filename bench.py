@@ -618,7 +618,43 @@ def main():
         factors = {"workload": cfg.name + " (k, alpha, theta, beta -> Gamma, Y, M, W, phase turns)",
                    "ms_per_call": f_ms, "chunks_per_s": cfg.B * cfg.H * NC / (f_ms * 1e-3),
                    "algorithmic_bytes": fb, "achieved_gbs": fb / (f_ms * 1e-3) / 1e9}
-        del G, Yf, Wf, Mf, turns
+        del G, Yf, Wf, Mf
+        # the kernel-benchmark protocol's other chunk size (App. E: C in {64, 128}): the forward runs a 128-token chunk as
+        # an exact superchunk of two 64-token tiles (same launch, timed for the record), the factor export composes the
+        # 128-token factors out of the tiles' (two launches)
+        if cfg.T % 128 == 0:
+            NC2 = cfg.T // 128
+            G2 = torch.empty(cfg.B, cfg.H, NC2, cfg.m, 2, device=dev)
+            Y2 = torch.empty(cfg.B, cfg.H, NC2, cfg.m, 128, 2, device=dev)
+            W2 = torch.empty_like(Y2)
+            M2 = torch.empty(cfg.B, cfg.H, NC2, 128, 128, 2, device=dev)
+
+            def timed_n(fn, n):
+                for _ in range(2):
+                    fn()
+                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                g0.record(stream)
+                for _ in range(n):
+                    fn()
+                g1.record(stream)
+                torch.cuda.synchronize()
+                return g0.elapsed_time(g1) / n
+
+            f128_ms = timed_n(lambda: sfda.sfda_chunk_factors(d["k"], d["alpha"], d["theta"], d["beta"], G2, Y2, M2, W2,
+                                                              turns, 128, stream), 3)
+            fw128_ms = timed_n(lambda: sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"],
+                                                         d["S0"], o, o_im, S_T, 128, ws, stream), max(args.steps, 5))
+            fb2 = rows * (cfg.d_k * 2 + 2 * cfg.m * 4 + 4) + sum(t.numel() * 4 for t in (G2, Y2, W2, M2, turns))
+            factors["chunk_128"] = {"factors_ms_per_call": f128_ms, "factors_launches": 2,
+                                    "factors_algorithmic_bytes": fb2,
+                                    "factors_achieved_gbs": fb2 / (f128_ms * 1e-3) / 1e9,
+                                    "forward_ms_per_step": fw128_ms,
+                                    "forward_tokens_per_s": cfg.B * cfg.T / (fw128_ms * 1e-3),
+                                    "note": "forward: exact superchunk of two 64-token tiles, the kernel and launch of "
+                                            "chunk = 64; factors: tile kernel plus composition kernel"}
+            del G2, Y2, W2, M2
+        del turns
 
     # one-token decode (sfda_step) on the decode configuration: HBM-bound, reported beside the headline
     decode = None

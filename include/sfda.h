@@ -58,7 +58,7 @@ typedef enum {
     SFDA_OK = 0,
     SFDA_ERR_NULL = -1,        /* a required pointer is NULL                          */
     SFDA_ERR_SHAPE = -2,       /* B, T, H < 1, odd d_k, non-positive chunk            */
-    SFDA_ERR_UNSUPPORTED = -3, /* d_k, d_v not in {64,128}; chunk not in {16,32,64};  */
+    SFDA_ERR_UNSUPPORTED = -3, /* d_k, d_v not in {64,128}; chunk not in {16,...,256}; */
                                /* unknown dtype                                       */
     SFDA_ERR_ALIGN = -4,       /* a pointer is not 16-byte aligned                    */
     SFDA_ERR_WORKSPACE = -5,   /* workspace NULL or smaller than sfda_workspace_bytes */
@@ -131,8 +131,13 @@ SFDA_API int sfda_forward_partition(int B, int T, int H, int d_k, int d_v, int c
  *             NULL when that is 0; the tensor-core path needs at least 256 bytes);
  *             contents are clobbered.
  *
- * Supported: d_k, d_v in {64, 128}; chunk in {16, 32, 64}.
- * bf16 inputs with d_k = d_v = 128 and chunk = 64 take the tensor-core path
+ * Supported: d_k, d_v in {64, 128}; chunk in {16, 32, 64, 128, 256}.  The kernels' tile
+ * is at most 64 tokens: chunk = 128 or 256 runs as an exact superchunk of two or four
+ * 64-token tiles (Section 6, "superchunks": chunk transfers compose exactly; the state
+ * is carried on chip from tile to tile), so outputs and final state are those of the
+ * chunk size named (they do not depend on where a sequence is cut) at the cost per
+ * token of chunk = 64; workspace, partition and slicing rules are those of chunk = 64.
+ * bf16 inputs with d_k = d_v = 128 and chunk >= 64 take the tensor-core path
  * (bf16 operands, fp32 accumulation and state); everything else runs in fp32 on
  * the CUDA cores.  The tensor-core path forms 1/gamma_t inside a chunk and so
  * additionally assumes prod_{t in chunk} alpha_{t,j} >= exp(-80) for every
@@ -145,7 +150,7 @@ SFDA_API int sfda_forward(const void *q, const void *k, const void *v,
                  void *workspace, size_t workspace_bytes, void *stream);
 
 /*
- * sfda_forward on the tensor-core shapes (bf16, d_k = d_v = 128, chunk = 64; SFDA_ERR_UNSUPPORTED otherwise) that
+ * sfda_forward on the tensor-core shapes (bf16, d_k = d_v = 128, chunk = 64 exactly; SFDA_ERR_UNSUPPORTED otherwise) that
  * also writes the integer bookkeeping of the cumulative phase (Eq. "constructive-Gamma"; App. "Kernel sketch",
  * Stage 1: phases kept as integers):
  *
@@ -284,6 +289,13 @@ SFDA_API int sfda_forward_simt(const void *q, const void *k, const void *v,
  * NC = ceil(T / chunk), C = chunk.  Columns (and rows of M) of padded tail tokens
  * are those of neutral tokens (zero columns in Y and W, identity rows in M).
  * Any of Gamma, Y, M, W may be NULL to skip that output.  fp32 arithmetic.
+ *
+ * chunk in {16, 32, 64, 128}.  The factors of a 128-token chunk are composed exactly out
+ * of those of its two 64-token tiles (block form of Eq. "constructive-M": Gamma =
+ * Gamma_2 Gamma_1, Y = [Gamma_2 Y_1 | Y_2], W = [W_1 | Gamma_1^* W_2], lower left block of
+ * M = -M_2 (W_2^* Y_1) M_1) by a second kernel; the tiles' Gamma wait inside M meanwhile,
+ * so with chunk = 128 all of Gamma, Y, M, W are required (SFDA_ERR_NULL otherwise).
+ * chunk = 256 -> SFDA_ERR_UNSUPPORTED.
  */
 SFDA_API int sfda_chunk_factors(const void *k, const float *alpha, const float *theta, const float *beta,
                        float *Gamma, float *Y, float *M, float *W, uint32_t *phase_turns,

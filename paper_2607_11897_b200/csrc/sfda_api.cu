@@ -16,12 +16,18 @@ int check_dims(int d_k, int d_v, int chunk, int dtype)
     if (d_k < 2 || (d_k & 1) || d_v < 1 || chunk < 1) return SFDA_ERR_SHAPE;
     if (d_k != 64 && d_k != 128) return SFDA_ERR_UNSUPPORTED;
     if (d_v != 64 && d_v != 128) return SFDA_ERR_UNSUPPORTED;
-    if (chunk != 16 && chunk != 32 && chunk != 64) return SFDA_ERR_UNSUPPORTED;
+    if (chunk != 16 && chunk != 32 && chunk != 64 && chunk != 128 && chunk != 256) return SFDA_ERR_UNSUPPORTED;
     if (dtype != SFDA_F32 && dtype != SFDA_BF16) return SFDA_ERR_UNSUPPORTED;
     return SFDA_OK;
 }
 
 size_t elem_bytes(int dtype) { return dtype == SFDA_BF16 ? 2 : 4; }
+
+// The kernels' tile is at most 64 tokens (tensor memory and shared memory are full at 64).  A chunk of 128 or 256
+// tokens is run as an exact superchunk of two or four tiles (Section 6, "superchunks": chunk transfers compose
+// exactly): the state is carried on chip from tile to tile, and since the recurrence's result does not depend on
+// where a sequence is cut, outputs and final state are those of the chunk size the caller named.
+int tile_chunk(int chunk) { return chunk > 64 ? 64 : chunk; }
 
 // The host-buffer forward overlaps its uploads, kernels and downloads: pieces of the batch go up on one internal
 // stream, are computed on the caller's stream and come down on another internal stream, chained by events.  The two
@@ -84,7 +90,7 @@ sfda::ForwardArgs pack(const void *q, const void *k, const void *v, const float 
     sfda::ForwardArgs a;
     a.q = q; a.k = k; a.v = v; a.alpha = alpha; a.theta = theta; a.beta = beta; a.S0 = S0;
     a.o = o; a.o_im = o_im; a.S_T = S_T;
-    a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.chunk = chunk; a.dtype = dtype;
+    a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.chunk = tile_chunk(chunk); a.dtype = dtype;
     return a;
 }
 
@@ -183,7 +189,7 @@ size_t sfda_workspace_bytes(int B, int T, int H, int d_k, int d_v, int chunk, in
 {
     if (B < 1 || T < 1 || H < 1 || check_dims(d_k, d_v, chunk, dtype) != SFDA_OK) return 0;
     sfda::ForwardArgs a{};
-    a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.chunk = chunk; a.dtype = dtype;
+    a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.chunk = tile_chunk(chunk); a.dtype = dtype;
     // the tensor-core path keeps a status word there, and the boundary states of its time slices
     return sfda::forward_ws_supported(a) ? sfda::forward_ws_scratch_bytes(B, H) : 0;
 }
@@ -199,9 +205,9 @@ int sfda_forward_partition(int B, int T, int H, int d_k, int d_v, int chunk, int
     *balanced = 0;
     *ctas = 0;
     sfda::ForwardArgs a{};
-    a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.chunk = chunk; a.dtype = dtype;
+    a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.chunk = tile_chunk(chunk); a.dtype = dtype;
     if (!sfda::forward_ws_supported(a) || workspace_bytes < 256) return SFDA_OK;
-    const int BH = B * H, NC = (T + chunk - 1) / chunk;
+    const int BH = B * H, NC = (T + a.chunk - 1) / a.chunk;
     sfda::forward_ws_partition(BH, NC, n_sm, workspace_bytes >= sfda::forward_ws_scratch_bytes(B, H), slices, balanced, nullptr);
     const long long units = (long long)BH * *slices;
     *ctas = (int)(units < n_sm ? units : n_sm);
@@ -251,6 +257,7 @@ int sfda_forward_phase(const void *q, const void *k, const void *v, const float 
     if (rc != SFDA_OK) return rc;
     if (!phase_turns) return SFDA_ERR_NULL;
     if (!aligned16(phase_turns)) return SFDA_ERR_ALIGN;
+    if (chunk > 64) return SFDA_ERR_UNSUPPORTED;                         // one phase per 64-token tile is what is exported
     sfda::ForwardArgs a = pack(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
     if (!sfda::forward_ws_supported(a)) return SFDA_ERR_UNSUPPORTED;     // the export belongs to the tensor-core kernel
     if (!workspace || workspace_bytes < sfda::kWsMinScratchBytes) return SFDA_ERR_WORKSPACE;
@@ -275,7 +282,7 @@ int sfda_forward_withheld_handoff(const void *q, const void *k, const void *v, c
     // at least two slices (so that something waits), a limit between 2^16 and 2^26 ticks (a few dozen microseconds to a
     // few dozen milliseconds), whole chunks per slice, and the full workspace (the hand-off buffers live there)
     if (slices < 2 || slices > 8 || wait_ticks < (1u << 16) || wait_ticks > (1u << 26)) return SFDA_ERR_VALUE;
-    if (((T + chunk - 1) / chunk) % slices != 0) return SFDA_ERR_SHAPE;
+    if (((T + a.chunk - 1) / a.chunk) % slices != 0) return SFDA_ERR_SHAPE;
     if (!workspace || workspace_bytes < sfda::forward_ws_scratch_bytes(B, H)) return SFDA_ERR_WORKSPACE;
     if (!aligned16(workspace)) return SFDA_ERR_ALIGN;
     a.debug_slices = slices;
@@ -292,9 +299,9 @@ size_t sfda_forward_two_level_workspace_bytes(int B, int T, int H, int d_k, int 
 {
     if (B < 1 || T < 1 || H < 1 || n_slices < 0 || check_dims(d_k, d_v, chunk, dtype) != SFDA_OK) return 0;
     sfda::ForwardArgs a{};
-    a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.chunk = chunk; a.dtype = dtype;
+    a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.chunk = tile_chunk(chunk); a.dtype = dtype;
     if (!sfda::forward_ws_supported(a)) return 0;
-    const int n = n_slices ? n_slices : auto_slices(B, T, H, chunk);
+    const int n = n_slices ? n_slices : auto_slices(B, T, H, tile_chunk(chunk));
     if (n == 1) return sfda::forward_ws_scratch_bytes(B, H);
     return sfda::forward_two_level_supported(a, n) ? sfda::forward_two_level_bytes(a, n) : 0;
 }
@@ -311,7 +318,7 @@ int sfda_forward_two_level(const void *q, const void *k, const void *v, const fl
     const sfda::ForwardArgs a = pack(q, k, v, alpha, theta, beta, S0, o, o_im, S_T, B, T, H, d_k, d_v, chunk, dtype);
     if (!sfda::forward_ws_supported(a)) return SFDA_ERR_UNSUPPORTED;
     if (workspace && !aligned16(workspace)) return SFDA_ERR_ALIGN;
-    const int n = n_slices ? n_slices : auto_slices(B, T, H, chunk);
+    const int n = n_slices ? n_slices : auto_slices(B, T, H, tile_chunk(chunk));
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (n == 1) {       // nothing to gain: the plain forward
         if (!workspace || workspace_bytes < sfda::kWsMinScratchBytes) return SFDA_ERR_WORKSPACE;
@@ -368,6 +375,9 @@ int sfda_chunk_factors(const void *k, const float *alpha, const float *theta, co
     if (B < 1 || T < 1 || H < 1) return SFDA_ERR_SHAPE;
     const int rc = check_dims(d_k, 64, chunk, dtype);
     if (rc != SFDA_OK) return rc;
+    // 128-token chunks are composed of two 64-token tiles, whose Gamma wait inside M: all four factor arrays are needed
+    if (chunk > 128) return SFDA_ERR_UNSUPPORTED;
+    if (chunk == 128 && (!Gamma || !Y || !M || !W)) return SFDA_ERR_NULL;
     const void *ptrs[] = {k, alpha, theta, beta, Gamma, Y, M, W, phase_turns};
     for (const void *p : ptrs)
         if (p && !aligned16(p)) return SFDA_ERR_ALIGN;
@@ -625,7 +635,7 @@ size_t sfda_forward_fused_workspace_bytes(int B, int T, int H, int d_k, int d_v,
 {
     if (B < 1 || T < 1 || H < 1 || check_dims(d_k, d_v, chunk, dtype) != SFDA_OK) return 0;
     sfda::ForwardArgs a{};
-    a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.chunk = chunk; a.dtype = dtype;
+    a.B = B; a.T = T; a.H = H; a.d_k = d_k; a.d_v = d_v; a.chunk = tile_chunk(chunk); a.dtype = dtype;
     if (sfda::forward_ws_supported(a)) return sfda::forward_ws_scratch_bytes(B, H);
     return staged_frontend_bytes((size_t)B * T * H, d_k, dtype);
 }

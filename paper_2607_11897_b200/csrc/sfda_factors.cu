@@ -208,7 +208,7 @@ __global__ void __launch_bounds__(kFacThreads, 3)
 sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alpha, const float *__restrict__ theta,
                           const float *__restrict__ beta, float *__restrict__ Gamma, float *__restrict__ Y,
                           float *__restrict__ Mo, float *__restrict__ W, uint32_t *__restrict__ turns_out, int T_,
-                          int H, int NC)
+                          int H, int NC, int sup)
 {
     using S = FacSmem<DK, C>;
     constexpr int M = S::M, G = S::G, TG = S::TG;
@@ -222,7 +222,10 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
     const int h = bh % H, b = bh / H;
     const int t0 = ci * C;
     const int len = min(C, T_ - t0);
-    const size_t chunk_id = (size_t)bh * NC + ci;
+    // The factors of chunk `ci` go to tile `part` of output chunk `sc`, which spans `sup` tiles (sup = 1: the chunk is
+    // the tile; sup = 2: a 128-token chunk out of two tiles, completed by sfda_compose_factors_kernel).
+    const int sc = ci / sup, part = ci - sc * sup, Co = sup * C;
+    const size_t out_id = (size_t)bh * ((NC + sup - 1) / sup) + sc;
 
     // ---- A: loads and scan.  Tokens past `len` are neutral (alpha = 1, theta = 0, beta = 0, k = 0).
     {
@@ -293,7 +296,10 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
     if (Gamma) {
         for (int j = tid; j < M; j += kFacThreads) {
             const float a = ex2f(sm.lg2C[j]);
-            reinterpret_cast<float2 *>(Gamma)[chunk_id * M + j] = make_float2(a * sm.gcr[j], a * sm.gci[j]);
+            const float2 gam = make_float2(a * sm.gcr[j], a * sm.gci[j]);
+            if (sup == 1) reinterpret_cast<float2 *>(Gamma)[out_id * M + j] = gam;
+            // a tile's Gamma waits in row `part` of the block of M above the diagonal, which ends up zero
+            else reinterpret_cast<float2 *>(Mo)[(out_id * Co + part) * Co + C + j] = gam;
         }
     }
     if (W || Y) {
@@ -301,10 +307,10 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
         constexpr int JS = kFacThreads / C;                 // coordinates per sweep of the CTA
         const int t = tid % C;
         const float bt = sm.beta[t];
-        float2 *Wp = reinterpret_cast<float2 *>(W) + (chunk_id * M + tid / C) * C + t;
-        float2 *Yp = reinterpret_cast<float2 *>(Y) + (chunk_id * M + tid / C) * C + t;
+        float2 *Wp = reinterpret_cast<float2 *>(W) + (out_id * M + tid / C) * Co + part * C + t;
+        float2 *Yp = reinterpret_cast<float2 *>(Y) + (out_id * M + tid / C) * Co + part * C + t;
 #pragma unroll 4
-        for (int j = tid / C; j < M; j += JS, Wp += JS * C, Yp += JS * C) {
+        for (int j = tid / C; j < M; j += JS, Wp += JS * Co, Yp += JS * Co) {
             const float2 kk = sm.kp[t * S::KS + j];
             const float l = sm.lg2[t * S::LS + j];
             if (W) {   // W[:,t] = conj(gamma_t) k_t = a_t k'_t
@@ -502,13 +508,14 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
         merge_level<S, C, 32>(sm, tid);
         for (int idx = tid; idx < C * C; idx += kFacThreads) {
             const int t = idx / C, i = idx % C;
-            reinterpret_cast<float2 *>(Mo)[chunk_id * C * C + idx] = i <= t ? sm.nx[t * S::NS + i] : make_float2(0.f, 0.f);
+            reinterpret_cast<float2 *>(Mo)[(out_id * Co + part * C + t) * Co + part * C + i] =
+                i <= t ? sm.nx[t * S::NS + i] : make_float2(0.f, 0.f);
         }
     }
 }
 
 template <int DK, int C, typename T>
-cudaError_t launch_fac(const FactorArgs &a, cudaStream_t stream)
+cudaError_t launch_fac(const FactorArgs &a, cudaStream_t stream, int sup = 1)
 {
     constexpr size_t smem = FacSmem<DK, C>::bytes;
     auto kern = sfda_chunk_factors_kernel<DK, C, T>;
@@ -517,7 +524,133 @@ cudaError_t launch_fac(const FactorArgs &a, cudaStream_t stream)
     const int NC = (a.T + C - 1) / C;
     const unsigned grid = (unsigned)a.B * a.H * NC;
     kern<<<grid, kFacThreads, smem, stream>>>(static_cast<const T *>(a.k), a.alpha, a.theta, a.beta, a.Gamma, a.Y, a.M,
-                                              a.W, a.phase_turns, a.T, a.H, NC);
+                                              a.W, a.phase_turns, a.T, a.H, NC, sup);
+    return cudaGetLastError();
+}
+
+// Factors of a 128-token chunk out of those of its two 64-token tiles (Section 6, "superchunks"; the block form of
+// Eq. "constructive-M"): with P_1 = Gamma_1 - Y_1 M_1 W_1^*, P_2 likewise,
+//
+//   P_2 P_1 = Gamma - Y M W^*,   Gamma = Gamma_2 Gamma_1,   Y = [Gamma_2 Y_1 | Y_2],   W = [W_1 | Gamma_1^* W_2],
+//   M = [[M_1, 0], [-M_2 (W_2^* Y_1) M_1, M_2]],
+//
+// exact, and every factor is a product of numbers of modulus at most one.  The tile kernel has left Y_1, Y_2, W_1,
+// W_2, M_1, M_2 at their places in the 128-token layout and Gamma_1, Gamma_2 in rows 0 and 1 of M's upper right
+// block; this kernel, one CTA per chunk, forms the lower left block of M in fp32 on the CUDA cores (three 64 x 64
+// complex products through shared memory), scales Y_1 and W_2, zeroes the upper right block, writes Gamma and adds
+// the first tile's closing phase to the integer phases of the second tile's tokens.  A chunk whose second tile has
+// no token (the sequence ends inside the first) gets the neutral tile: zero columns, identity block.
+constexpr int kCmpThreads = 256;
+constexpr int kCmpStride = 68;                              // float2 row stride of the three 64 x 64 regions (4 mod 16)
+template <int DK>
+__global__ void __launch_bounds__(kCmpThreads)
+sfda_compose_factors_kernel(float *__restrict__ Gamma, float *__restrict__ Y, float *__restrict__ Mo,
+                            float *__restrict__ W, uint32_t *__restrict__ turns, int T_, int H, int NCo)
+{
+    constexpr int M = DK / 2, h = 64, Co = 128, RS = kCmpStride;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float2 *ra = reinterpret_cast<float2 *>(smem_raw), *rb = ra + 64 * RS, *rc = rb + 64 * RS, *g1 = rc + 64 * RS, *g2 = g1 + M;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, c = lane & 3;
+    const size_t out_id = blockIdx.x;
+    const int bh = (int)(out_id / NCo), sc = (int)(out_id % NCo), b = bh / H, hh = bh % H;
+    const int t0 = sc * Co;
+    const bool has2 = t0 + h < T_;
+    float2 *Y2 = reinterpret_cast<float2 *>(Y) + out_id * M * Co, *W2 = reinterpret_cast<float2 *>(W) + out_id * M * Co;
+    float2 *M2 = reinterpret_cast<float2 *>(Mo) + out_id * Co * Co, *G2 = reinterpret_cast<float2 *>(Gamma) + out_id * M;
+    auto cmul = [](float2 x, float2 y) { return make_float2(x.x * y.x - x.y * y.y, x.x * y.y + x.y * y.x); };
+    // one 64 x 64 complex product as 32 tiles of 16 x 8 (four per warp), 3 x TF32, k-steps ks0(tile) .. ks1(tile) - 1;
+    // `put` receives every result element
+    auto product = [&](const float2 *A, const float2 *Bm, auto ks0, auto ks1, auto put) {
+        for (int tile = warp; tile < 32; tile += kCmpThreads / 32) {
+            const int mt = tile >> 3, nt = tile & 7;
+            float acc[4][4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x)
+#pragma unroll
+                for (int y = 0; y < 4; ++y) acc[x][y] = 0.f;
+            const int k1 = ks1(mt, nt);
+#pragma unroll 1
+            for (int ks = ks0(mt, nt); ks < k1; ++ks)
+                cmma3_step(acc, A + (16 * mt + g) * RS + 8 * ks + c, RS, Bm + (8 * ks + c) * RS + 8 * nt + g, RS);
+#pragma unroll
+            for (int e = 0; e < 4; ++e)        // c0 (g, 2c), c1 (g, 2c + 1), c2 (g + 8, 2c), c3 (g + 8, 2c + 1)
+                put(16 * mt + g + 8 * (e >> 1), 8 * nt + 2 * c + (e & 1), make_float2(acc[0][e] - acc[1][e], acc[2][e] + acc[3][e]));
+        }
+    };
+
+    for (int j = tid; j < M; j += kCmpThreads) {
+        g1[j] = M2[h + j];
+        g2[j] = has2 ? M2[Co + h + j] : make_float2(1.f, 0.f);
+    }
+    if (has2) {
+        for (int i = tid; i < M * h; i += kCmpThreads) {     // Y_1 -> ra[j][t1], W_2^* -> rb[t2][j]
+            const int j = i / h, t = i % h;
+            ra[j * RS + t] = Y2[j * Co + t];
+            const float2 w = W2[j * Co + h + t];
+            rb[t * RS + j] = make_float2(w.x, -w.y);
+        }
+        __syncthreads();
+        // Z = W_2^* Y_1  (sum over the m coordinates)
+        product(rb, ra, [](int, int) { return 0; }, [](int, int) { return M / 8; },
+                [&](int r, int cc, float2 v) { rc[r * RS + cc] = v; });
+        // Y_1 <- Gamma_2 Y_1,  W_2 <- conj(Gamma_1) W_2  (from the copies in shared memory)
+        for (int i = tid; i < M * h; i += kCmpThreads) {
+            const int j = i / h, t = i % h;
+            Y2[j * Co + t] = cmul(g2[j], ra[j * RS + t]);
+            const float2 w = cmul(g1[j], rb[t * RS + j]);                       // conj(conj(Gamma_1) W_2)
+            W2[j * Co + h + t] = make_float2(w.x, -w.y);
+        }
+        __syncthreads();
+        for (int i = tid; i < h * h; i += kCmpThreads) ra[(i / h) * RS + i % h] = M2[(size_t)(i / h) * Co + i % h];   // M_1
+        __syncthreads();
+        // T = Z M_1  (M_1 is lower triangular: k-blocks from the column's on)
+        product(rc, ra, [](int, int nt) { return nt; }, [](int, int) { return 8; },
+                [&](int r, int cc, float2 v) { rb[r * RS + cc] = v; });
+        __syncthreads();
+        for (int i = tid; i < h * h; i += kCmpThreads)
+            ra[(i / h) * RS + i % h] = M2[(size_t)(h + i / h) * Co + h + i % h];                                    // M_2
+        __syncthreads();
+        // lower left block of M = -M_2 T  (M_2 is lower triangular: k-blocks up to the rows')
+        product(ra, rb, [](int, int) { return 0; }, [](int mt, int) { return 2 * mt + 2; },
+                [&](int r, int cc, float2 v) { M2[(size_t)(h + r) * Co + cc] = make_float2(-v.x, -v.y); });
+    } else {
+        // the neutral second tile
+        for (int i = tid; i < M * h; i += kCmpThreads) {
+            const int j = i / h, t = i % h;
+            Y2[j * Co + h + t] = make_float2(0.f, 0.f);
+            W2[j * Co + h + t] = make_float2(0.f, 0.f);
+        }
+        for (int i = tid; i < h * h; i += kCmpThreads) {
+            const int rr = i / h, cc = i % h;
+            M2[(size_t)(h + rr) * Co + cc] = make_float2(0.f, 0.f);
+            M2[(size_t)(h + rr) * Co + h + cc] = make_float2(rr == cc ? 1.f : 0.f, 0.f);
+        }
+    }
+    __syncthreads();                                     // g1, g2 were read from the block that is zeroed now
+    for (int i = tid; i < h * h; i += kCmpThreads) M2[(size_t)(i / h) * Co + h + i % h] = make_float2(0.f, 0.f);
+    for (int j = tid; j < M; j += kCmpThreads) G2[j] = cmul(g2[j], g1[j]);
+    if (turns && has2) {
+        const int n2 = min(h, T_ - t0 - h);
+        const uint32_t *close1 = turns + (((size_t)b * T_ + t0 + h - 1) * H + hh) * M;
+        for (int i = tid; i < n2 * M; i += kCmpThreads) {
+            const int t = i / M, j = i % M;
+            turns[(((size_t)b * T_ + t0 + h + t) * H + hh) * M + j] += close1[j];
+        }
+    }
+}
+
+template <int DK, typename T>
+cudaError_t launch_fac_128(const FactorArgs &a, cudaStream_t stream, int *launches)
+{
+    cudaError_t e = launch_fac<DK, 64, T>(a, stream, 2);
+    if (e != cudaSuccess) return e;
+    if (launches) ++*launches;
+    constexpr size_t smem = (size_t)3 * 64 * kCmpStride * 8 + (size_t)DK * 8;
+    auto kern = sfda_compose_factors_kernel<DK>;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const int NCo = (a.T + 127) / 128;
+    kern<<<(unsigned)a.B * a.H * NCo, kCmpThreads, smem, stream>>>(a.Gamma, a.Y, a.M, a.W, a.phase_turns, a.T, a.H, NCo);
     return cudaGetLastError();
 }
 
@@ -537,6 +670,14 @@ cudaError_t dispatch_fac(const FactorArgs &a, cudaStream_t s)
 
 cudaError_t launch_chunk_factors(const FactorArgs &a, cudaStream_t stream, int *launches)
 {
+    if (a.chunk == 128) {   // two tiles of 64 and their composition (needs every factor array: the tiles' Gamma wait in M)
+        if (!a.Gamma || !a.Y || !a.M || !a.W) return cudaErrorInvalidValue;
+        cudaError_t e2;
+        if (a.d_k == 64) e2 = a.dtype == 1 ? launch_fac_128<64, __nv_bfloat16>(a, stream, launches) : launch_fac_128<64, float>(a, stream, launches);
+        else e2 = a.dtype == 1 ? launch_fac_128<128, __nv_bfloat16>(a, stream, launches) : launch_fac_128<128, float>(a, stream, launches);
+        if (e2 == cudaSuccess && launches) ++*launches;
+        return e2;
+    }
     const cudaError_t e = a.dtype == 1 ? dispatch_fac<__nv_bfloat16>(a, stream) : dispatch_fac<float>(a, stream);
     if (e == cudaSuccess && launches) ++*launches;
     return e;

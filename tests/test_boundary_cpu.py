@@ -70,6 +70,34 @@ def test_host_arena_gives_every_piece_of_the_batch_an_aligned_beta_region(lib):
         assert (per * T * H * 4) % 16 != 0 or (B, T, H) in ((8, 64, 2),)      # the cases above do leave the grid
 
 
+def test_chunks_of_128_and_256_tokens_are_superchunks_of_64_token_tiles(lib):
+    """Section 6 ("superchunks": chunk transfers compose exactly): a chunk of 128 or 256 tokens runs as two or four
+    64-token tiles, so the plan is the caller's, the workspace and the launcher's partition are those of the tiles, and
+    other sizes stay unsupported; the factor export composes 128-token chunks out of two tiles and needs all four
+    factor arrays for it (host logic only)."""
+    vp, ci = ctypes.c_void_p, ctypes.c_int
+    for chunk in (128, 256):
+        assert sfda.sfda_plan(1000, chunk) == bookkeeping.chunk_plan(1000, chunk)
+        assert sfda.sfda_workspace_bytes(8, 8192, 32, 128, 128, chunk, sfda.SFDA_BF16) == \
+            sfda.sfda_workspace_bytes(8, 8192, 32, 128, 128, 64, sfda.SFDA_BF16) > 0
+        assert sfda.sfda_forward_partition(8, 8192, 32, 128, 128, chunk, sfda.SFDA_BF16, 1 << 30, 148) == \
+            sfda.sfda_forward_partition(8, 8192, 32, 128, 128, 64, sfda.SFDA_BF16, 1 << 30, 148)
+        assert sfda.sfda_forward_two_level_workspace_bytes(1, 131072, 16, 128, 128, chunk, sfda.SFDA_BF16, 0) == \
+            sfda.sfda_forward_two_level_workspace_bytes(1, 131072, 16, 128, 128, 64, sfda.SFDA_BF16, 0) > 0
+    assert sfda.sfda_workspace_bytes(1, 1024, 1, 128, 128, 512, sfda.SFDA_BF16) == 0
+    assert sfda.sfda_workspace_bytes(1, 1024, 1, 128, 128, 96, sfda.SFDA_BF16) == 0
+    ok = vp(0x1000)
+    fac = lambda ptrs, d: lib.sfda_chunk_factors(*ptrs, *[ci(x) for x in d], None)
+    assert fac([ok] * 4 + [ok] * 4 + [None], [1, 256, 1, 128, 256, 0]) == -3          # factors: up to 128 tokens
+    assert fac([ok] * 4 + [ok, ok, None, ok] + [None], [1, 256, 1, 128, 128, 0]) == -1  # M missing
+    assert fac([ok] * 4 + [None, ok, ok, ok] + [None], [1, 256, 1, 128, 128, 0]) == -1  # Gamma missing
+    # the diagnostic phase export is per 64-token tile
+    ph = lambda chunk: lib.sfda_forward_phase(*([ok] * 6 + [None, ok, None, None]), ok,
+                                              *[ci(d) for d in (1, 256, 1, 128, 128, chunk, 1)], vp(0x2000),
+                                              ctypes.c_size_t(256), None)
+    assert ph(128) == -3
+
+
 def test_argument_validation_happens_before_any_launch(lib):
     """Every error below is found on the host; nothing touches a device (there is none here)."""
     vp, ci = ctypes.c_void_p, ctypes.c_int

@@ -559,6 +559,78 @@ def test_chunk_factors_decay_and_write_extremes(case, d_k, chunk):
     assert worst < 1e-4, worst
 
 
+@pytest.mark.parametrize("d_k,T,dtype", [(128, 200, "bf16"), (128, 150, "f32"), (64, 128, "f32"), (128, 64, "bf16"),
+                                         (64, 333, "bf16")])
+def test_chunk_factors_of_128_token_chunks(d_k, T, dtype):
+    """Factors of 128-token chunks (Section 6 "Chunk size": C = 64-256; App. E protocol C in {64, 128}), which the
+    library composes exactly out of two 64-token tiles (block form of Eq. "constructive-M"), against the constructive
+    recursion run over 128 tokens: full chunks, a second tile with a ragged tail, a chunk whose second tile is empty
+    (T = 150: the last chunk holds 22 tokens, T = 64: the only chunk holds 64), and the chunk-local integer phases."""
+    C = 128
+    cfg = workloads.CONFIGS[0].scaled(name="fac128", B=2, T=T, H=2, d_k=d_k, chunk=64, dtype=dtype, seed=900 + T)
+    inp = workloads.forward_inputs(cfg)
+    B, H, m = cfg.B, cfg.H, cfg.m
+    NC, tail = sfda.sfda_plan(T, C)
+    assert (NC, tail) == bookkeeping.chunk_plan(T, C)
+    G = torch.full((B, H, NC, m, 2), float("nan"), device=DEV)
+    Y = torch.full((B, H, NC, m, C, 2), float("nan"), device=DEV)
+    M = torch.full((B, H, NC, C, C, 2), float("nan"), device=DEV)
+    W = torch.full((B, H, NC, m, C, 2), float("nan"), device=DEV)
+    turns = torch.zeros(B, T, H, m, device=DEV, dtype=torch.int32)
+    sfda.sfda_chunk_factors(to_dev(inp["k"], cfg, "k"), to_dev(inp["alpha"], cfg, "alpha"),
+                            to_dev(inp["theta"], cfg, "theta"), to_dev(inp["beta"], cfg, "beta"), G, Y, M, W, turns, C)
+    torch.cuda.synchronize()
+    assert sfda.last_launch_count() == 2
+    cx = lambda t: t.cpu().numpy().astype(np.float64)[..., 0] + 1j * t.cpu().numpy().astype(np.float64)[..., 1]
+    G, Y, M, W = cx(G), cx(Y), cx(M), cx(W)
+    want_turns = np.moveaxis(bookkeeping.cumulative_phase_turns(np.moveaxis(inp["theta"], 1, 2), C), 2, 1)
+    assert np.array_equal(turns.cpu().numpy().view(np.uint32), want_turns)
+    worst = 0.0
+    for b in range(B):
+        for h in range(H):
+            kc = chunk_wy.pair(inp["k"][b, :, h])
+            for c in range(NC):
+                sl = slice(c * C, min((c + 1) * C, T))
+                L = sl.stop - sl.start
+                g, y, w, mm = chunk_wy.chunk_factors(kc[sl], inp["alpha"][b, sl, h].astype(np.float64),
+                                                     inp["theta"][b, sl, h].astype(np.float64),
+                                                     inp["beta"][b, sl, h].astype(np.float64))
+                worst = max(worst, rel_err(G[b, h, c].view(np.float64), g.view(np.float64)),
+                            rel_err(Y[b, h, c][:, :L].copy().view(np.float64), y.copy().view(np.float64)),
+                            rel_err(W[b, h, c][:, :L].copy().view(np.float64), w.copy().view(np.float64)),
+                            rel_err(M[b, h, c][:L, :L].copy().view(np.float64), mm.copy().view(np.float64)))
+                # padded tail tokens are neutral: zero columns, identity rows; nothing above the diagonal
+                assert np.all(Y[b, h, c][:, L:] == 0) and np.all(W[b, h, c][:, L:] == 0)
+                assert np.array_equal(M[b, h, c][L:, :], np.eye(C)[L:, :])
+                assert np.all(np.triu(M[b, h, c], 1) == 0)
+                P_gpu = np.diag(G[b, h, c]) - Y[b, h, c] @ M[b, h, c] @ W[b, h, c].conj().T
+                assert np.abs(P_gpu - (np.diag(g) - y @ mm @ w.conj().T)).max() < 2e-5
+    assert worst < 1e-4, worst
+
+
+@pytest.mark.parametrize("chunk", [128, 256])
+def test_forward_with_chunks_of_128_and_256_tokens(chunk):
+    """A chunk of 128 or 256 tokens runs as an exact superchunk of 64-token tiles (Section 6: chunk transfers compose
+    exactly, and the recurrence's result does not depend on where a sequence is cut): same bits as chunk = 64 on the
+    tensor-core path and on the CUDA-core path, and the oracle's values."""
+    cfg = workloads.CONFIGS[1].scaled(name="sup", B=2, T=4 * 256 + 37, H=3, s0_std=0.02)
+    inp = workloads.forward_inputs(cfg)
+    o64, oi64, S64 = run_forward(cfg, inp)
+    o, oi, S = run_forward(cfg.scaled(chunk=chunk), inp)
+    assert np.array_equal(o, o64) and np.array_equal(oi, oi64) and np.array_equal(S, S64)
+    pairs = [(0, 0), (1, 2)]
+    s = workloads.sequences(inp, pairs)
+    w_re, w_im, w_S = recurrence.sfda_recurrence(s["q"], s["k"], s["v"], s["alpha"], s["theta"], s["beta"], s["S0"])
+    assert rel_err(np.stack([o[b, :, h] for b, h in pairs]), w_re) <= 2e-2
+    assert rel_err(np.stack([S[b, h] for b, h in pairs]), w_S) <= 2e-2
+    # CUDA-core path (fp32, d_k = 64)
+    cfg32 = workloads.CONFIGS[0].scaled(name="sup32", B=1, T=300, H=2, d_k=64, d_v=64, chunk=32, dtype="f32")
+    inp32 = workloads.forward_inputs(cfg32)
+    a = run_forward(cfg32.scaled(chunk=64), inp32)
+    b_ = run_forward(cfg32.scaled(chunk=chunk), inp32)
+    assert all(np.array_equal(x, y) for x, y in zip(a, b_))
+
+
 # ------------------------------------------------------------------------------------------------
 # decode
 # ------------------------------------------------------------------------------------------------
