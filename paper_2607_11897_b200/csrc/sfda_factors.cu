@@ -540,7 +540,7 @@ cudaError_t launch_fac(const FactorArgs &a, cudaStream_t stream, int sup = 1)
 // complex products through shared memory), scales Y_1 and W_2, zeroes the upper right block, writes Gamma and adds
 // the first tile's closing phase to the integer phases of the second tile's tokens.  A chunk whose second tile has
 // no token (the sequence ends inside the first) gets the neutral tile: zero columns, identity block.
-constexpr int kCmpThreads = 256;
+constexpr int kCmpThreads = 512;
 constexpr int kCmpStride = 68;                              // float2 row stride of the three 64 x 64 regions (4 mod 16)
 template <int DK>
 __global__ void __launch_bounds__(kCmpThreads)
