@@ -258,6 +258,43 @@ def test_forward_tensor_core_balanced_partition():
         assert np.array_equal(x, y)
 
 
+def _random_tensor_core_shapes():
+    """Fourteen seeded shapes around the launcher's decisions: fewer and more (batch, head) pairs than SMs, chunk counts
+    that halve and that do not, T below one tile, exact multiples and ragged tails, with and without S0."""
+    rng = np.random.default_rng(20260711)
+    shapes = [(1, 1, 1, 0.0), (1, 63, 149, 0.1), (3, 64 * 9, 50, 0.0), (2, 64 * 16 + 1, 75, 0.05),
+              (4, 64 * 7 + 5, 60, 0.05), (2, 64 * 12, 100, 0.0)]
+    while len(shapes) < 14:
+        B, H = int(rng.integers(1, 6)), int(rng.integers(1, 80))
+        T = int(rng.integers(1, 40)) * 64 + int(rng.integers(0, 64)) * int(rng.integers(0, 2))
+        if B * T * H <= 700_000:
+            shapes.append((B, T, H, float(rng.choice([0.0, 0.05, 0.5]))))
+    return shapes
+
+
+@pytest.mark.parametrize("B,T,H,s0", _random_tensor_core_shapes())
+def test_forward_tensor_core_random_shapes(B, T, H, s0):
+    """The tensor-core forward on seeded random shapes: first, last and three random sequences against the oracle at
+    the bar and the regression guards, and the whole output bit for bit against the same call with only the status
+    block as workspace (the launcher then cuts nothing)."""
+    cfg = workloads.CONFIGS[1].scaled(name="rnd_%d_%d_%d" % (B, T, H), B=B, T=T, H=H, s0_std=s0, seed=7000 + B + T + H)
+    inp = workloads.forward_inputs(cfg)
+    rng = np.random.default_rng(cfg.seed)
+    pairs = sorted({(0, 0), (B - 1, H - 1)} | {(int(rng.integers(B)), int(rng.integers(H))) for _ in range(3)})
+    d = {k: (None if v is None else to_dev(v, cfg, k)) for k, v in inp.items()}
+    outs = []
+    for nbytes in (sfda.sfda_workspace_bytes(B, T, H, 128, 128, 64, 1), 256):
+        o = torch.full((B, T, H, 128), float("nan"), device=DEV, dtype=torch.bfloat16)
+        o_im, S_T = torch.full_like(o, float("nan")), torch.full((B, H, 128, 128), float("nan"), device=DEV)
+        ws = torch.empty(nbytes, device=DEV, dtype=torch.uint8)
+        sfda.sfda_forward(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im, S_T, 64, ws)
+        assert sfda.sfda_workspace_status(ws) == 0 and sfda.last_launch_count() == 1
+        outs.append((o.float().cpu().numpy(), o_im.float().cpu().numpy(), S_T.cpu().numpy()))
+    for x, y in zip(*outs):
+        assert np.isfinite(x).all() and np.array_equal(x, y)
+    check_all_sequences(cfg.name, pairs, lambda sub: oracle_pairs(inp, sub), outs[0], TOL["bf16"], guard=T >= 64)
+
+
 @pytest.mark.parametrize("case", ["product_exactly_e-80", "product_e-77", "product_e-40_uneven"])
 def test_forward_tensor_core_at_the_documented_decay_edge(case):
     """The tensor-core path forms 1 / |gamma_t| inside a chunk and documents prod_chunk alpha >= e^-80 per coordinate
