@@ -498,7 +498,15 @@ def main():
             sg = [torch.empty_like(x) for x in (sq, sk, sv, sal, sth, sbe)] + [torch.empty_like(sS)]
             sbws = torch.empty(sfda.sfda_backward_workspace_bytes(Bs, Ts, Hs, dk, dv, 1), dtype=torch.uint8, device=dev)
             b_ms = timed(lambda: sfda.sfda_backward(sq, sk, sv, sal, sth, sbe, None, so, so_im, sS, *sg, sbws, stream), 1)
+            # the protocol's other chunk size (an exact superchunk of two 64-token tiles: same kernel, same launch)
+            f128_ms = timed(lambda: sfda.sfda_forward(sq, sk, sv, sal, sth, sbe, None, so, so_im, sS, 128, sws, stream), 3)
+            pcfg = cfg.scaled(B=Bs, T=Ts)
+            best = min(f_ms, f2_ms)
             return {"T": Ts, "B": Bs, "H": Hs, "forward_ms": f_ms, "forward_two_level_auto_ms": f2_ms,
+                    "forward_chunk128_ms": f128_ms,
+                    "forward_tflops": algorithmic_flops(pcfg) / (best * 1e-3) / 1e12,
+                    "forward_gbs": algorithmic_bytes(pcfg) / (best * 1e-3) / 1e9,
+                    "forward_workspace_bytes": int(sws.numel()), "backward_workspace_bytes": int(sbws.numel()),
                     "two_level_launches": f2_launches, "backward_ms": b_ms,
                     "forward_tokens_per_s": Bs * Ts / (min(f_ms, f2_ms) * 1e-3),
                     "backward_tokens_per_s": Bs * Ts / (b_ms * 1e-3)}
