@@ -22,10 +22,15 @@ def lib_path() -> str:
 
 
 def load():
-    """Load ``libsfda.so``; raise if it has not been built (no fallback exists)."""
+    """Load ``libsfda.so``; raise if it has not been built (no fallback exists).  A library that was not built from
+    the sources now in the tree is rebuilt first: an out-of-date kernel must never be what a test or a benchmark runs."""
     global _LIB
     if _LIB is None:
-        _LIB = load_library(lib_path())
+        path = lib_path()
+        from . import build as _build
+        if os.path.abspath(path) == os.path.abspath(_build.LIB) and os.path.exists(path) and _build.is_stale():
+            _build.build(force=True)
+        _LIB = load_library(path)
     return _LIB
 
 

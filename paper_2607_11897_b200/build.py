@@ -1,5 +1,9 @@
-"""Build ``libsfda.so`` (the C-ABI CUDA library) in-tree with nvcc for sm_100a."""
+"""Build ``libsfda.so`` (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
+
+A build is current when the hash of its sources, kept in a small file beside the library, equals the hash of the
+sources in the tree: file times say nothing once a source file has been put back to an earlier state."""
 import glob
+import hashlib
 import os
 import subprocess
 
@@ -19,13 +23,36 @@ def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
+def _deps():
+    return sorted(sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(CSRC, "*.h"))
+                  + glob.glob(os.path.join(HERE, "..", "include", "*.h")))
+
+
+def source_hash(extra_flags=()) -> str:
+    """SHA-256 over the compiler flags and the names and contents of every source and header of the library."""
+    h = hashlib.sha256(" ".join(FLAGS + list(extra_flags)).encode())
+    for path in _deps():
+        h.update(os.path.basename(path).encode() + b"\0")
+        with open(path, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def _current(lib: str, extra_flags=()) -> bool:
+    try:
+        with open(lib + ".srchash") as f:
+            return os.path.exists(lib) and f.read().strip() == source_hash(extra_flags)
+    except OSError:
+        return False
+
+
+def is_stale() -> bool:
+    """True when ``libsfda.so`` is missing or was not built from the sources now in the tree."""
+    return not _current(LIB)
+
+
 def _stale() -> bool:
-    if not os.path.exists(LIB):
-        return True
-    t = os.path.getmtime(LIB)
-    deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(CSRC, "*.h")) \
-        + glob.glob(os.path.join(HERE, "..", "include", "*.h"))
-    return any(os.path.getmtime(d) > t for d in deps)
+    return is_stale()
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
@@ -51,6 +78,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     link = [NVCC, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + objs
     subprocess.run(link, check=True)
     os.replace(tmp, LIB)
+    with open(LIB + ".srchash", "w") as f:
+        f.write(source_hash() + "\n")
     return LIB
 
 
@@ -59,9 +88,7 @@ def build_variant(name: str, extra_flags):
     (used by the tests for the development build whose roles pause at random, ``-DSFDA_WS_CHAOS``)."""
     objdir = os.path.join(HERE, "build", name)
     lib = os.path.join(HERE, "build", "libsfda_%s.so" % name)
-    deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(CSRC, "*.h")) \
-        + glob.glob(os.path.join(HERE, "..", "include", "*.h"))
-    if os.path.exists(lib) and all(os.path.getmtime(d) <= os.path.getmtime(lib) for d in deps):
+    if _current(lib, extra_flags):
         return lib
     os.makedirs(objdir, exist_ok=True)
     procs, objs = [], []
@@ -77,6 +104,8 @@ def build_variant(name: str, extra_flags):
     tmp = lib + ".tmp.%d" % os.getpid()
     subprocess.run([NVCC, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + objs, check=True)
     os.replace(tmp, lib)
+    with open(lib + ".srchash", "w") as f:
+        f.write(source_hash(extra_flags) + "\n")
     return lib
 
 

@@ -70,6 +70,21 @@ def test_host_arena_gives_every_piece_of_the_batch_an_aligned_beta_region(lib):
         assert (per * T * H * 4) % 16 != 0 or (B, T, H) in ((8, 64, 2),)      # the cases above do leave the grid
 
 
+def test_a_library_built_from_other_sources_is_recognised(lib, tmp_path, monkeypatch):
+    """The build records a hash of its sources beside the library; a tree whose sources differ from it (a file added,
+    changed, or put back to an earlier state) makes the library stale whatever the file times say, and loading the
+    package then rebuilds it."""
+    assert not cuda_build.is_stale()
+    h = cuda_build.source_hash()
+    assert h == open(cuda_build.LIB + ".srchash").read().strip()
+    assert cuda_build.source_hash(["-DSOMETHING"]) != h
+    extra = tmp_path / "extra.cuh"
+    extra.write_text("// one more header\n")
+    deps = cuda_build._deps()
+    monkeypatch.setattr(cuda_build, "_deps", lambda: sorted(deps + [str(extra)]))
+    assert cuda_build.source_hash() != h and cuda_build.is_stale()
+
+
 def test_chunks_of_128_and_256_tokens_are_superchunks_of_64_token_tiles(lib):
     """Section 6 ("superchunks": chunk transfers compose exactly): a chunk of 128 or 256 tokens runs as two or four
     64-token tiles, so the plan is the caller's, the workspace and the launcher's partition are those of the tiles, and
