@@ -1253,9 +1253,8 @@ __device__ __forceinline__ void run_chain(uint8_t *smem, Misc &mi, uint32_t tmem
                 if (sub_v) {
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
-                        const float v0 = __uint_as_float((uint32_t)lds16(sv + (32 * pc + 2 * i) * 2 * DV) << 16);
-                        const float v1 = __uint_as_float((uint32_t)lds16(sv + (32 * pc + 2 * i + 1) * 2 * DV) << 16);
-                        pk[i] = pack_bf16(__uint_as_float(r[2 * i]) + v0, __uint_as_float(r[2 * i + 1]) + v1);
+                        pk[i] = pack_bf16(add_bf16_f32(lds16(sv + (32 * pc + 2 * i) * 2 * DV), __uint_as_float(r[2 * i])),
+                                          add_bf16_f32(lds16(sv + (32 * pc + 2 * i + 1) * 2 * DV), __uint_as_float(r[2 * i + 1])));
                     }
                 } else {
 #pragma unroll

@@ -192,6 +192,14 @@ __device__ __forceinline__ uint16_t lds16(uint32_t saddr)
     asm volatile("ld.shared.b16 %0, [%1];" : "=h"(v) : "r"(saddr));
     return v;
 }
+// x + y for a bf16 x (its 16 bits as loaded) and an fp32 y, in one instruction (the bf16 is exact in fp32, so the
+// result is the fp32 sum of the two)
+__device__ __forceinline__ float add_bf16_f32(uint16_t x, float y)
+{
+    float r;
+    asm("add.rn.f32.bf16 %0, %1, %2;" : "=f"(r) : "h"(x), "f"(y));
+    return r;
+}
 template <int N>
 __device__ __forceinline__ void tmem_ld(uint32_t addr, uint32_t *r)
 {
