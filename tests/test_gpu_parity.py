@@ -668,6 +668,54 @@ def test_forward_with_chunks_of_128_and_256_tokens(chunk):
     assert all(np.array_equal(x, y) for x, y in zip(a, b_))
 
 
+def test_other_forward_entry_points_with_chunks_of_128_tokens():
+    """The fused forward, the two-level scan, the entry point without allocations and the host-buffer entry point take
+    chunk = 128 as the same exact superchunk: bit for bit what they return with chunk = 64."""
+    cfg = workloads.CONFIGS[1].scaled(name="sup2", B=2, T=2048, H=3, s0_std=0.02, seed=321)
+    inp = workloads.forward_inputs(cfg)
+    raw = workloads.forward_raw_inputs(cfg)
+    d = {k: (None if v is None else to_dev(v, cfg, k)) for k, v in inp.items()}
+    B, T, H = cfg.B, cfg.T, cfg.H
+    new = lambda: (torch.empty(B, T, H, 128, device=DEV, dtype=torch.bfloat16),
+                   torch.empty(B, T, H, 128, device=DEV, dtype=torch.bfloat16), torch.empty(B, H, 128, 128, device=DEV))
+    same = lambda x, y: all(torch.equal(a, b) for a, b in zip(x, y))
+    # fused
+    outs = []
+    for chunk in (64, 128):
+        o, o_im, S, _, _ = run_forward_fused(cfg.scaled(chunk=chunk), raw, PARAM)
+        outs.append((o, o_im, S))
+    assert all(np.array_equal(a, b) for a, b in zip(*outs))
+    # two-level scan (4 slices)
+    outs = []
+    for chunk in (64, 128):
+        o, o_im, S = new()
+        ws = torch.empty(sfda.sfda_forward_two_level_workspace_bytes(B, T, H, 128, 128, chunk, 1, 4), device=DEV, dtype=torch.uint8)
+        sfda.sfda_forward_two_level(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im, S, chunk, 4, ws)
+        assert sfda.sfda_workspace_status(ws) == 0
+        outs.append((o, o_im, S))
+    assert same(*outs)
+    # no allocations
+    outs = []
+    for chunk in (64, 128):
+        o, o_im, S = new()
+        sfda.sfda_forward_noalloc(d["q"], d["k"], d["v"], d["alpha"], d["theta"], d["beta"], d["S0"], o, o_im, S, chunk)
+        assert sfda.sfda_noalloc_status() == 0
+        outs.append((o, o_im, S))
+    assert same(*outs)
+    # host buffers
+    h = {k: (None if v is None else to_dev(v, cfg, k).cpu().pin_memory()) for k, v in inp.items()}
+    outs = []
+    for chunk in (64, 128):
+        oh = torch.empty(B, T, H, 128, dtype=torch.bfloat16).pin_memory()
+        oh_im, Sh = torch.empty_like(oh).pin_memory(), torch.empty(B, H, 128, 128).pin_memory()
+        arena = torch.empty(sfda.sfda_forward_host_arena_bytes(B, T, H, 128, 128, chunk, 1, True, True, True), device=DEV,
+                            dtype=torch.uint8)
+        sfda.sfda_forward_host(h["q"], h["k"], h["v"], h["alpha"], h["theta"], h["beta"], h["S0"], oh, oh_im, Sh, chunk, arena)
+        torch.cuda.synchronize()
+        outs.append((oh.clone(), oh_im.clone(), Sh.clone()))
+    assert same(*outs)
+
+
 # ------------------------------------------------------------------------------------------------
 # decode
 # ------------------------------------------------------------------------------------------------
