@@ -29,7 +29,14 @@ def load():
         path = lib_path()
         from . import build as _build
         if os.path.abspath(path) == os.path.abspath(_build.LIB) and os.path.exists(path) and _build.is_stale():
-            _build.build(force=True)
+            if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+                _build.build(force=True)
+            else:                                   # several ranks on one node: the first one builds, the others wait for it
+                import time
+                for _ in range(1800):
+                    if not _build.is_stale():
+                        break
+                    time.sleep(1.0)
         _LIB = load_library(path)
     return _LIB
 
