@@ -662,6 +662,19 @@ def main():
                                     "note": "forward: exact superchunk of two 64-token tiles, the kernel and launch of "
                                             "chunk = 64; factors: tile kernel plus composition kernel"}
             del G2, Y2, W2, M2
+            if cfg.T % 256 == 0:
+                NC4 = cfg.T // 256
+                G4 = torch.empty(cfg.B, cfg.H, NC4, cfg.m, 2, device=dev)
+                Y4 = torch.empty(cfg.B, cfg.H, NC4, cfg.m, 256, 2, device=dev)
+                W4 = torch.empty_like(Y4)
+                M4 = torch.empty(cfg.B, cfg.H, NC4, 256, 256, 2, device=dev)
+                f256_ms = timed_n(lambda: sfda.sfda_chunk_factors(d["k"], d["alpha"], d["theta"], d["beta"], G4, Y4, M4,
+                                                                  W4, turns, 256, stream), 3)
+                fb4 = rows * (cfg.d_k * 2 + 2 * cfg.m * 4 + 4) + sum(t.numel() * 4 for t in (G4, Y4, W4, M4, turns))
+                factors["chunk_256"] = {"factors_ms_per_call": f256_ms, "factors_launches": 4,
+                                        "factors_algorithmic_bytes": fb4,
+                                        "factors_achieved_gbs": fb4 / (f256_ms * 1e-3) / 1e9}
+                del G4, Y4, W4, M4
         del turns
 
     # one-token decode (sfda_step) on the decode configuration: HBM-bound, reported beside the headline

@@ -290,12 +290,12 @@ SFDA_API int sfda_forward_simt(const void *q, const void *k, const void *v,
  * are those of neutral tokens (zero columns in Y and W, identity rows in M).
  * Any of Gamma, Y, M, W may be NULL to skip that output.  fp32 arithmetic.
  *
- * chunk in {16, 32, 64, 128}.  The factors of a 128-token chunk are composed exactly out
- * of those of its two 64-token tiles (block form of Eq. "constructive-M": Gamma =
- * Gamma_2 Gamma_1, Y = [Gamma_2 Y_1 | Y_2], W = [W_1 | Gamma_1^* W_2], lower left block of
- * M = -M_2 (W_2^* Y_1) M_1) by a second kernel; the tiles' Gamma wait inside M meanwhile,
- * so with chunk = 128 all of Gamma, Y, M, W are required (SFDA_ERR_NULL otherwise).
- * chunk = 256 -> SFDA_ERR_UNSUPPORTED.
+ * chunk in {16, 32, 64, 128, 256}.  The factors of a chunk of 128 or 256 tokens are
+ * composed exactly out of those of its 64-token tiles, one tile appended per launch
+ * (block form of Eq. "constructive-M": appending tile b to a prefix p gives Gamma =
+ * Gamma_b Gamma_p, Y = [Gamma_b Y_p | Y_b], W = [W_p | Gamma_p^* W_b], block row b of
+ * M = -M_b (W_b^* Y_p) M_p); the tiles' Gamma wait inside M meanwhile, so with
+ * chunk > 64 all of Gamma, Y, M, W are required (SFDA_ERR_NULL otherwise).
  */
 SFDA_API int sfda_chunk_factors(const void *k, const float *alpha, const float *theta, const float *beta,
                        float *Gamma, float *Y, float *M, float *W, uint32_t *phase_turns,

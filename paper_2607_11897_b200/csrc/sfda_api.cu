@@ -375,9 +375,8 @@ int sfda_chunk_factors(const void *k, const float *alpha, const float *theta, co
     if (B < 1 || T < 1 || H < 1) return SFDA_ERR_SHAPE;
     const int rc = check_dims(d_k, 64, chunk, dtype);
     if (rc != SFDA_OK) return rc;
-    // 128-token chunks are composed of two 64-token tiles, whose Gamma wait inside M: all four factor arrays are needed
-    if (chunk > 128) return SFDA_ERR_UNSUPPORTED;
-    if (chunk == 128 && (!Gamma || !Y || !M || !W)) return SFDA_ERR_NULL;
+    // chunks of 128 and 256 tokens are composed of 64-token tiles, whose Gamma wait inside M: all four factor arrays are needed
+    if (chunk > 64 && (!Gamma || !Y || !M || !W)) return SFDA_ERR_NULL;
     const void *ptrs[] = {k, alpha, theta, beta, Gamma, Y, M, W, phase_turns};
     for (const void *p : ptrs)
         if (p && !aligned16(p)) return SFDA_ERR_ALIGN;

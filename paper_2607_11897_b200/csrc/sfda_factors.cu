@@ -298,8 +298,9 @@ sfda_chunk_factors_kernel(const T *__restrict__ k, const float *__restrict__ alp
             const float a = ex2f(sm.lg2C[j]);
             const float2 gam = make_float2(a * sm.gcr[j], a * sm.gci[j]);
             if (sup == 1) reinterpret_cast<float2 *>(Gamma)[out_id * M + j] = gam;
-            // a tile's Gamma waits in row `part` of the block of M above the diagonal, which ends up zero
-            else reinterpret_cast<float2 *>(Mo)[(out_id * Co + part) * Co + C + j] = gam;
+            // a tile's Gamma waits in a block of M above the diagonal, which ends up zero: tile 0 in row 1 of block
+            // (0, 1), tile b >= 1 in row 0 of block (0, b)
+            else reinterpret_cast<float2 *>(Mo)[(part == 0 ? out_id * Co + 1 : out_id * Co) * Co + (part == 0 ? C : part * C) + j] = gam;
         }
     }
     if (W || Y) {
@@ -528,37 +529,44 @@ cudaError_t launch_fac(const FactorArgs &a, cudaStream_t stream, int sup = 1)
     return cudaGetLastError();
 }
 
-// Factors of a 128-token chunk out of those of its two 64-token tiles (Section 6, "superchunks"; the block form of
-// Eq. "constructive-M"): with P_1 = Gamma_1 - Y_1 M_1 W_1^*, P_2 likewise,
+// Factors of a chunk of 128 or 256 tokens out of those of its 64-token tiles (Section 6, "superchunks"; the block
+// form of Eq. "constructive-M").  Appending a tile b with P_b = Gamma_b - Y_b M_b W_b^* to a prefix of tiles with
+// P_p = Gamma_p - Y_p M_p W_p^* gives
 //
-//   P_2 P_1 = Gamma - Y M W^*,   Gamma = Gamma_2 Gamma_1,   Y = [Gamma_2 Y_1 | Y_2],   W = [W_1 | Gamma_1^* W_2],
-//   M = [[M_1, 0], [-M_2 (W_2^* Y_1) M_1, M_2]],
+//   P_b P_p = Gamma - Y M W^*,   Gamma = Gamma_b Gamma_p,   Y = [Gamma_b Y_p | Y_b],   W = [W_p | Gamma_p^* W_b],
+//   M = [[M_p, 0], [-M_b (W_b^* Y_p) M_p, M_b]],
 //
-// exact, and every factor is a product of numbers of modulus at most one.  The tile kernel has left Y_1, Y_2, W_1,
-// W_2, M_1, M_2 at their places in the 128-token layout and Gamma_1, Gamma_2 in rows 0 and 1 of M's upper right
-// block; this kernel, one CTA per chunk, forms the lower left block of M in fp32 on the CUDA cores (three 64 x 64
-// complex products through shared memory), scales Y_1 and W_2, zeroes the upper right block, writes Gamma and adds
-// the first tile's closing phase to the integer phases of the second tile's tokens.  A chunk whose second tile has
-// no token (the sequence ends inside the first) gets the neutral tile: zero columns, identity block.
+// exact, and every factor is a product of numbers of modulus at most one.  The tile kernel has left every tile's Y,
+// W and M at their places in the chunk's layout and the tiles' Gamma in the blocks of M above the diagonal (tile 0:
+// row 1 of block (0, 1); tile b >= 1: row 0 of block (0, b)).  This kernel, launched once per appended tile
+// b = 1 .. sup - 1 with one CTA per chunk, forms block row b of M left of the diagonal,
+// X_c = -M_b sum_{k >= c} Z_k M_p[k][c] with Z_k = W_b^* Y_p[:, block k], as 16 x 8 tiles on the tensor cores
+// (3 x TF32) through shared memory, scales the prefix's Y by Gamma_b and W_b by conj(Gamma_p), zeroes the blocks above
+// tile b's diagonal block, keeps the running Gamma in the output array and adds the prefix's closing phase to the
+// integer phases of tile b's tokens.  A tile without tokens (the sequence ends before it) becomes the neutral tile:
+// zero columns, identity block.
 constexpr int kCmpThreads = 512;
-constexpr int kCmpStride = 68;                              // float2 row stride of the three 64 x 64 regions (4 mod 16)
+constexpr int kCmpStride = 68;                              // float2 row stride of the 64 x 64 regions (4 mod 16)
+constexpr size_t compose_smem_bytes(int DK, int b) { return (size_t)(b + 2) * 64 * kCmpStride * 8 + (size_t)DK * 8; }
 template <int DK>
 __global__ void __launch_bounds__(kCmpThreads)
 sfda_compose_factors_kernel(float *__restrict__ Gamma, float *__restrict__ Y, float *__restrict__ Mo,
-                            float *__restrict__ W, uint32_t *__restrict__ turns, int T_, int H, int NCo)
+                            float *__restrict__ W, uint32_t *__restrict__ turns, int T_, int H, int NCo, int sup, int b)
 {
-    constexpr int M = DK / 2, h = 64, Co = 128, RS = kCmpStride;
+    constexpr int M = DK / 2, h = 64, RS = kCmpStride;
+    const int Co = h * sup, P = h * b;                     // chunk length, prefix length
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float2 *ra = reinterpret_cast<float2 *>(smem_raw), *rb = ra + 64 * RS, *rc = rb + 64 * RS, *g1 = rc + 64 * RS, *g2 = g1 + M;
+    float2 *ra = reinterpret_cast<float2 *>(smem_raw), *rb = ra + 64 * RS, *zs = rb + 64 * RS;   // zs: b regions
+    float2 *gb = zs + b * 64 * RS, *gp = gb + M;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, c = lane & 3;
     const size_t out_id = blockIdx.x;
-    const int bh = (int)(out_id / NCo), sc = (int)(out_id % NCo), b = bh / H, hh = bh % H;
+    const int bh = (int)(out_id / NCo), sc = (int)(out_id % NCo), bb = bh / H, hh = bh % H;
     const int t0 = sc * Co;
-    const bool has2 = t0 + h < T_;
+    const bool has = t0 + P < T_;                          // tile b holds at least one token
     float2 *Y2 = reinterpret_cast<float2 *>(Y) + out_id * M * Co, *W2 = reinterpret_cast<float2 *>(W) + out_id * M * Co;
     float2 *M2 = reinterpret_cast<float2 *>(Mo) + out_id * Co * Co, *G2 = reinterpret_cast<float2 *>(Gamma) + out_id * M;
     auto cmul = [](float2 x, float2 y) { return make_float2(x.x * y.x - x.y * y.y, x.x * y.y + x.y * y.x); };
-    // one 64 x 64 complex product as 32 tiles of 16 x 8 (four per warp), 3 x TF32, k-steps ks0(tile) .. ks1(tile) - 1;
+    // one 64 x 64 complex product as 32 tiles of 16 x 8 (two per warp), 3 x TF32, k-steps ks0(tile) .. ks1(tile) - 1;
     // `put` receives every result element
     auto product = [&](const float2 *A, const float2 *Bm, auto ks0, auto ks1, auto put) {
         for (int tile = warp; tile < 32; tile += kCmpThreads / 32) {
@@ -577,81 +585,101 @@ sfda_compose_factors_kernel(float *__restrict__ Gamma, float *__restrict__ Y, fl
                 put(16 * mt + g + 8 * (e >> 1), 8 * nt + 2 * c + (e & 1), make_float2(acc[0][e] - acc[1][e], acc[2][e] + acc[3][e]));
         }
     };
+    auto load_block = [&](float2 *dst, int row0, int col0) {   // a 64 x 64 block of M
+        for (int i = tid; i < h * h; i += kCmpThreads) dst[(i / h) * RS + i % h] = M2[(size_t)(row0 + i / h) * Co + col0 + i % h];
+    };
 
     for (int j = tid; j < M; j += kCmpThreads) {
-        g1[j] = M2[h + j];
-        g2[j] = has2 ? M2[Co + h + j] : make_float2(1.f, 0.f);
+        gb[j] = has ? M2[P + j] : make_float2(1.f, 0.f);                 // tile b: row 0 of block (0, b)
+        gp[j] = b == 1 ? M2[Co + h + j] : G2[j];                         // tile 0: row 1 of block (0, 1); else the running one
     }
-    if (has2) {
-        for (int i = tid; i < M * h; i += kCmpThreads) {     // Y_1 -> ra[j][t1], W_2^* -> rb[t2][j]
+    if (has) {
+        for (int i = tid; i < M * h; i += kCmpThreads) {     // W_b^* -> rb[t][j]
             const int j = i / h, t = i % h;
-            ra[j * RS + t] = Y2[j * Co + t];
-            const float2 w = W2[j * Co + h + t];
+            const float2 w = W2[j * Co + P + t];
             rb[t * RS + j] = make_float2(w.x, -w.y);
         }
-        __syncthreads();
-        // Z = W_2^* Y_1  (sum over the m coordinates)
-        product(rb, ra, [](int, int) { return 0; }, [](int, int) { return M / 8; },
-                [&](int r, int cc, float2 v) { rc[r * RS + cc] = v; });
-        // Y_1 <- Gamma_2 Y_1,  W_2 <- conj(Gamma_1) W_2  (from the copies in shared memory)
-        for (int i = tid; i < M * h; i += kCmpThreads) {
-            const int j = i / h, t = i % h;
-            Y2[j * Co + t] = cmul(g2[j], ra[j * RS + t]);
-            const float2 w = cmul(g1[j], rb[t * RS + j]);                       // conj(conj(Gamma_1) W_2)
-            W2[j * Co + h + t] = make_float2(w.x, -w.y);
+#pragma unroll 1
+        for (int cb = 0; cb < b; ++cb) {                     // Z_cb = W_b^* Y_p[:, block cb]  (sum over the m coordinates)
+            __syncthreads();                                 // (the previous block's products have read ra)
+            for (int i = tid; i < M * h; i += kCmpThreads) ra[(i / h) * RS + i % h] = Y2[(i / h) * Co + h * cb + i % h];
+            __syncthreads();
+            float2 *z = zs + cb * 64 * RS;
+            product(rb, ra, [](int, int) { return 0; }, [](int, int) { return M / 8; },
+                    [&](int r, int cc, float2 v) { z[r * RS + cc] = v; });
+            for (int i = tid; i < M * h; i += kCmpThreads)   // Y_p <- Gamma_b Y_p (from the copy in shared memory)
+                Y2[(i / h) * Co + h * cb + i % h] = cmul(gb[i / h], ra[(i / h) * RS + i % h]);
         }
-        __syncthreads();
-        for (int i = tid; i < h * h; i += kCmpThreads) ra[(i / h) * RS + i % h] = M2[(size_t)(i / h) * Co + i % h];   // M_1
-        __syncthreads();
-        // T = Z M_1  (M_1 is lower triangular: k-blocks from the column's on)
-        product(rc, ra, [](int, int nt) { return nt; }, [](int, int) { return 8; },
-                [&](int r, int cc, float2 v) { rb[r * RS + cc] = v; });
-        __syncthreads();
-        for (int i = tid; i < h * h; i += kCmpThreads)
-            ra[(i / h) * RS + i % h] = M2[(size_t)(h + i / h) * Co + h + i % h];                                    // M_2
-        __syncthreads();
-        // lower left block of M = -M_2 T  (M_2 is lower triangular: k-blocks up to the rows')
-        product(ra, rb, [](int, int) { return 0; }, [](int mt, int) { return 2 * mt + 2; },
-                [&](int r, int cc, float2 v) { M2[(size_t)(h + r) * Co + cc] = make_float2(-v.x, -v.y); });
+        for (int i = tid; i < M * h; i += kCmpThreads) {     // W_b <- conj(Gamma_p) W_b = conj(Gamma_p conj(W_b))
+            const int j = i / h, t = i % h;
+            const float2 w = cmul(gp[j], rb[t * RS + j]);
+            W2[j * Co + P + t] = make_float2(w.x, -w.y);
+        }
+#pragma unroll 1
+        for (int cb = 0; cb < b; ++cb) {
+            // T = sum_{k >= cb} Z_k M_p[k][cb] into rb (the diagonal block of M_p is lower triangular: k-steps from the
+            // column's on), then X_cb = -M_b T (M_b is lower triangular: k-steps up to the rows')
+#pragma unroll 1
+            for (int k = cb; k < b; ++k) {
+                __syncthreads();
+                load_block(ra, h * k, h * cb);
+                __syncthreads();
+                const float2 *z = zs + k * 64 * RS;
+                if (k == cb)
+                    product(z, ra, [](int, int nt) { return nt; }, [](int, int) { return 8; },
+                            [&](int r, int cc, float2 v) { rb[r * RS + cc] = v; });
+                else
+                    product(z, ra, [](int, int) { return 0; }, [](int, int) { return 8; },
+                            [&](int r, int cc, float2 v) { rb[r * RS + cc].x += v.x; rb[r * RS + cc].y += v.y; });
+            }
+            __syncthreads();
+            load_block(ra, P, P);
+            __syncthreads();
+            product(ra, rb, [](int, int) { return 0; }, [](int mt, int) { return 2 * mt + 2; },
+                    [&](int r, int cc, float2 v) { M2[(size_t)(P + r) * Co + h * cb + cc] = make_float2(-v.x, -v.y); });
+        }
     } else {
-        // the neutral second tile
+        // the neutral tile
         for (int i = tid; i < M * h; i += kCmpThreads) {
             const int j = i / h, t = i % h;
-            Y2[j * Co + h + t] = make_float2(0.f, 0.f);
-            W2[j * Co + h + t] = make_float2(0.f, 0.f);
+            Y2[j * Co + P + t] = make_float2(0.f, 0.f);
+            W2[j * Co + P + t] = make_float2(0.f, 0.f);
         }
-        for (int i = tid; i < h * h; i += kCmpThreads) {
-            const int rr = i / h, cc = i % h;
-            M2[(size_t)(h + rr) * Co + cc] = make_float2(0.f, 0.f);
-            M2[(size_t)(h + rr) * Co + h + cc] = make_float2(rr == cc ? 1.f : 0.f, 0.f);
-        }
+        for (int i = tid; i < h * P; i += kCmpThreads) M2[(size_t)(P + i / P) * Co + i % P] = make_float2(0.f, 0.f);
+        for (int i = tid; i < h * h; i += kCmpThreads)
+            M2[(size_t)(P + i / h) * Co + P + i % h] = make_float2(i / h == i % h ? 1.f : 0.f, 0.f);
     }
-    __syncthreads();                                     // g1, g2 were read from the block that is zeroed now
-    for (int i = tid; i < h * h; i += kCmpThreads) M2[(size_t)(i / h) * Co + h + i % h] = make_float2(0.f, 0.f);
-    for (int j = tid; j < M; j += kCmpThreads) G2[j] = cmul(g2[j], g1[j]);
-    if (turns && has2) {
-        const int n2 = min(h, T_ - t0 - h);
-        const uint32_t *close1 = turns + (((size_t)b * T_ + t0 + h - 1) * H + hh) * M;
+    __syncthreads();                                     // gb, gp were read from blocks that are zeroed now
+    for (int i = tid; i < P * h; i += kCmpThreads) M2[(size_t)(i / h) * Co + P + i % h] = make_float2(0.f, 0.f);
+    for (int j = tid; j < M; j += kCmpThreads) G2[j] = cmul(gb[j], gp[j]);
+    if (turns && has) {
+        const int n2 = min(h, T_ - t0 - P);
+        const uint32_t *close1 = turns + (((size_t)bb * T_ + t0 + P - 1) * H + hh) * M;
         for (int i = tid; i < n2 * M; i += kCmpThreads) {
             const int t = i / M, j = i % M;
-            turns[(((size_t)b * T_ + t0 + h + t) * H + hh) * M + j] += close1[j];
+            turns[(((size_t)bb * T_ + t0 + P + t) * H + hh) * M + j] += close1[j];
         }
     }
 }
 
 template <int DK, typename T>
-cudaError_t launch_fac_128(const FactorArgs &a, cudaStream_t stream, int *launches)
+cudaError_t launch_fac_super(const FactorArgs &a, cudaStream_t stream, int *launches)
 {
-    cudaError_t e = launch_fac<DK, 64, T>(a, stream, 2);
+    const int sup = a.chunk / 64;
+    cudaError_t e = launch_fac<DK, 64, T>(a, stream, sup);
     if (e != cudaSuccess) return e;
     if (launches) ++*launches;
-    constexpr size_t smem = (size_t)3 * 64 * kCmpStride * 8 + (size_t)DK * 8;
     auto kern = sfda_compose_factors_kernel<DK>;
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)compose_smem_bytes(DK, sup - 1));
     if (e != cudaSuccess) return e;
-    const int NCo = (a.T + 127) / 128;
-    kern<<<(unsigned)a.B * a.H * NCo, kCmpThreads, smem, stream>>>(a.Gamma, a.Y, a.M, a.W, a.phase_turns, a.T, a.H, NCo);
-    return cudaGetLastError();
+    const int NCo = (a.T + a.chunk - 1) / a.chunk;
+    for (int b = 1; b < sup; ++b) {
+        kern<<<(unsigned)a.B * a.H * NCo, kCmpThreads, compose_smem_bytes(DK, b), stream>>>(a.Gamma, a.Y, a.M, a.W, a.phase_turns,
+                                                                                           a.T, a.H, NCo, sup, b);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        if (launches) ++*launches;
+    }
+    return cudaSuccess;
 }
 
 template <typename T>
@@ -670,13 +698,10 @@ cudaError_t dispatch_fac(const FactorArgs &a, cudaStream_t s)
 
 cudaError_t launch_chunk_factors(const FactorArgs &a, cudaStream_t stream, int *launches)
 {
-    if (a.chunk == 128) {   // two tiles of 64 and their composition (needs every factor array: the tiles' Gamma wait in M)
-        if (!a.Gamma || !a.Y || !a.M || !a.W) return cudaErrorInvalidValue;
-        cudaError_t e2;
-        if (a.d_k == 64) e2 = a.dtype == 1 ? launch_fac_128<64, __nv_bfloat16>(a, stream, launches) : launch_fac_128<64, float>(a, stream, launches);
-        else e2 = a.dtype == 1 ? launch_fac_128<128, __nv_bfloat16>(a, stream, launches) : launch_fac_128<128, float>(a, stream, launches);
-        if (e2 == cudaSuccess && launches) ++*launches;
-        return e2;
+    if (a.chunk > 64) {   // tiles of 64 tokens and their composition (needs every factor array: the tiles' Gamma wait in M)
+        if ((a.chunk != 128 && a.chunk != 256) || !a.Gamma || !a.Y || !a.M || !a.W) return cudaErrorInvalidValue;
+        if (a.d_k == 64) return a.dtype == 1 ? launch_fac_super<64, __nv_bfloat16>(a, stream, launches) : launch_fac_super<64, float>(a, stream, launches);
+        return a.dtype == 1 ? launch_fac_super<128, __nv_bfloat16>(a, stream, launches) : launch_fac_super<128, float>(a, stream, launches);
     }
     const cudaError_t e = a.dtype == 1 ? dispatch_fac<__nv_bfloat16>(a, stream) : dispatch_fac<float>(a, stream);
     if (e == cudaSuccess && launches) ++*launches;

@@ -88,8 +88,8 @@ def test_a_library_built_from_other_sources_is_recognised(lib, tmp_path, monkeyp
 def test_chunks_of_128_and_256_tokens_are_superchunks_of_64_token_tiles(lib):
     """Section 6 ("superchunks": chunk transfers compose exactly): a chunk of 128 or 256 tokens runs as two or four
     64-token tiles, so the plan is the caller's, the workspace and the launcher's partition are those of the tiles, and
-    other sizes stay unsupported; the factor export composes 128-token chunks out of two tiles and needs all four
-    factor arrays for it (host logic only)."""
+    other sizes stay unsupported; the factor export composes chunks of 128 and 256 tokens out of their tiles and needs
+    all four factor arrays for it (host logic only)."""
     vp, ci = ctypes.c_void_p, ctypes.c_int
     for chunk in (128, 256):
         assert sfda.sfda_plan(1000, chunk) == bookkeeping.chunk_plan(1000, chunk)
@@ -103,7 +103,8 @@ def test_chunks_of_128_and_256_tokens_are_superchunks_of_64_token_tiles(lib):
     assert sfda.sfda_workspace_bytes(1, 1024, 1, 128, 128, 96, sfda.SFDA_BF16) == 0
     ok = vp(0x1000)
     fac = lambda ptrs, d: lib.sfda_chunk_factors(*ptrs, *[ci(x) for x in d], None)
-    assert fac([ok] * 4 + [ok] * 4 + [None], [1, 256, 1, 128, 256, 0]) == -3          # factors: up to 128 tokens
+    assert fac([ok] * 4 + [ok] * 4 + [None], [1, 512, 1, 128, 512, 0]) == -3          # factors: up to 256 tokens
+    assert fac([ok] * 4 + [ok, None, ok, ok] + [None], [1, 512, 1, 128, 256, 0]) == -1  # Y missing
     assert fac([ok] * 4 + [ok, ok, None, ok] + [None], [1, 256, 1, 128, 128, 0]) == -1  # M missing
     assert fac([ok] * 4 + [None, ok, ok, ok] + [None], [1, 256, 1, 128, 128, 0]) == -1  # Gamma missing
     # the diagnostic phase export is per 64-token tile

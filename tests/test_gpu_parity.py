@@ -596,14 +596,15 @@ def test_chunk_factors_decay_and_write_extremes(case, d_k, chunk):
     assert worst < 1e-4, worst
 
 
-@pytest.mark.parametrize("d_k,T,dtype", [(128, 200, "bf16"), (128, 150, "f32"), (64, 128, "f32"), (128, 64, "bf16"),
-                                         (64, 333, "bf16")])
-def test_chunk_factors_of_128_token_chunks(d_k, T, dtype):
-    """Factors of 128-token chunks (Section 6 "Chunk size": C = 64-256; App. E protocol C in {64, 128}), which the
-    library composes exactly out of two 64-token tiles (block form of Eq. "constructive-M"), against the constructive
-    recursion run over 128 tokens: full chunks, a second tile with a ragged tail, a chunk whose second tile is empty
-    (T = 150: the last chunk holds 22 tokens, T = 64: the only chunk holds 64), and the chunk-local integer phases."""
-    C = 128
+@pytest.mark.parametrize("C,d_k,T,dtype", [(128, 128, 200, "bf16"), (128, 128, 150, "f32"), (128, 64, 128, "f32"),
+                                           (128, 128, 64, "bf16"), (128, 64, 333, "bf16"), (256, 128, 512, "bf16"),
+                                           (256, 128, 300, "f32"), (256, 64, 700, "bf16"), (256, 128, 130, "f32"),
+                                           (256, 64, 64, "f32")])
+def test_chunk_factors_of_128_and_256_token_chunks(C, d_k, T, dtype):
+    """Factors of chunks of 128 and 256 tokens (Section 6 "Chunk size": C = 64-256; App. E protocol C in {64, 128}),
+    which the library composes exactly out of 64-token tiles (block form of Eq. "constructive-M", one tile appended
+    per launch), against the constructive recursion run over the whole chunk: full chunks, tiles with a ragged tail,
+    chunks whose later tiles are empty, and the chunk-local integer phases."""
     cfg = workloads.CONFIGS[0].scaled(name="fac128", B=2, T=T, H=2, d_k=d_k, chunk=64, dtype=dtype, seed=900 + T)
     inp = workloads.forward_inputs(cfg)
     B, H, m = cfg.B, cfg.H, cfg.m
@@ -617,7 +618,7 @@ def test_chunk_factors_of_128_token_chunks(d_k, T, dtype):
     sfda.sfda_chunk_factors(to_dev(inp["k"], cfg, "k"), to_dev(inp["alpha"], cfg, "alpha"),
                             to_dev(inp["theta"], cfg, "theta"), to_dev(inp["beta"], cfg, "beta"), G, Y, M, W, turns, C)
     torch.cuda.synchronize()
-    assert sfda.last_launch_count() == 2
+    assert sfda.last_launch_count() == C // 64
     cx = lambda t: t.cpu().numpy().astype(np.float64)[..., 0] + 1j * t.cpu().numpy().astype(np.float64)[..., 1]
     G, Y, M, W = cx(G), cx(Y), cx(M), cx(W)
     want_turns = np.moveaxis(bookkeeping.cumulative_phase_turns(np.moveaxis(inp["theta"], 1, 2), C), 2, 1)
